@@ -1,0 +1,174 @@
+"""ctypes front end of the fp64 CPU oracle (``retopk_oracle.c``).
+
+TEST INFRASTRUCTURE ONLY: the tests, the smoke check and the benchmark's CPU-baseline leg
+load this; the CUDA library never does.  ``build()`` compiles the C file with gcc next to
+itself; nothing here does arithmetic, it only marshals numpy arrays.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "retopk_oracle.c")
+_LIB = os.path.join(_HERE, "libretopk_oracle.so")
+
+PATH_REUSE, PATH_FALLBACK, PATH_REFRESH = 0, 1, 2
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle into ``libretopk_oracle.so`` (skipped when up to date)."""
+    if (not force and os.path.exists(_LIB)
+            and os.path.getmtime(_LIB) >= os.path.getmtime(_SRC)):
+        return _LIB
+    cmd = ["gcc", "-O2", "-std=c99", "-fopenmp", "-fPIC", "-shared", "-ffp-contract=off",
+           "-o", _LIB, _SRC, "-lm"]
+    subprocess.run(cmd, check=True)
+    return _LIB
+
+
+_lib = None
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = C.CDLL(build())
+        vp, i32, i64, f64 = C.c_void_p, C.c_int, C.c_int64, C.c_double
+        lib.oracle_create.argtypes = [C.POINTER(vp)] + [i32] * 8 + [f64, i32, i64]
+        lib.oracle_create.restype = i32
+        lib.oracle_destroy.argtypes = [vp]
+        lib.oracle_destroy.restype = None
+        lib.oracle_reset.argtypes = [vp]
+        lib.oracle_reset.restype = None
+        lib.oracle_decode_step.argtypes = [vp, vp, vp, vp, i64, vp]
+        lib.oracle_decode_step.restype = i32
+        lib.oracle_exact_topk.argtypes = [vp, vp, vp, vp, i64, vp, vp]
+        lib.oracle_exact_topk.restype = i32
+        lib.oracle_stats.argtypes = [vp, vp]
+        lib.oracle_stats.restype = None
+        lib.oracle_last_step.argtypes = [vp] * 7
+        lib.oracle_last_step.restype = None
+        lib.oracle_last_candidates.argtypes = [vp, i32, vp]
+        lib.oracle_last_candidates.restype = i32
+        lib.oracle_export_state.argtypes = [vp] * 5
+        lib.oracle_export_state.restype = None
+        lib.oracle_import_state.argtypes = [vp, vp, vp, i64, i64]
+        lib.oracle_import_state.restype = None
+        lib.oracle_num_threads.argtypes = []
+        lib.oracle_num_threads.restype = i32
+        _lib = lib
+    return _lib
+
+
+def num_threads() -> int:
+    return int(_load().oracle_num_threads())
+
+
+def _ptr(a: np.ndarray):
+    return a.ctypes.data_as(C.c_void_p)
+
+
+def _u16(a) -> np.ndarray:
+    a = np.ascontiguousarray(a)
+    if a.dtype != np.uint16:
+        raise TypeError("bf16 inputs are passed as uint16 bit patterns")
+    return a
+
+
+class Oracle:
+    """fp64 ReTopK state machine for ``B`` sequences x ``H_q`` query heads."""
+
+    def __init__(self, B, H_q, H_kv, d, M, r, W, K, tau, R, max_seq_len):
+        self.lib = _load()
+        self.B, self.H_q, self.H_kv, self.d = B, H_q, H_kv, d
+        self.M, self.r, self.W, self.K, self.R = M, r, W, K, R
+        # the C interface of the CUDA library takes tau as a float: compare against the
+        # same value here
+        self.tau = float(np.float32(tau))
+        self.max_seq_len = max_seq_len
+        h = C.c_void_p()
+        rc = self.lib.oracle_create(C.byref(h), B, H_q, H_kv, d, M, r, W, K, self.tau, R,
+                                    max_seq_len)
+        if rc != 0:
+            raise ValueError(f"oracle_create failed with {rc}")
+        self.h = h
+        self.nh = B * H_q
+
+    @classmethod
+    def from_config(cls, cfg, **override):
+        p = dict(B=cfg.B, H_q=cfg.H_q, H_kv=cfg.H_kv, d=cfg.d, M=cfg.M, r=cfg.r, W=cfg.W, K=cfg.K,
+                 tau=cfg.tau, R=cfg.R, max_seq_len=cfg.max_seq_len)
+        p.update(override)
+        return cls(**p)
+
+    def __del__(self):
+        if getattr(self, "h", None):
+            self.lib.oracle_destroy(self.h)
+            self.h = None
+
+    def reset(self):
+        self.lib.oracle_reset(self.h)
+
+    def _check_kv(self, k, v):
+        shape = (self.B, self.H_kv, self.max_seq_len, self.d)
+        if k.shape != shape or v.shape != shape:
+            raise ValueError(f"k/v must have shape {shape}, got {k.shape} / {v.shape}")
+
+    def decode_step(self, q, k, v, seq_len) -> np.ndarray:
+        q, k, v = _u16(q), _u16(k), _u16(v)
+        self._check_kv(k, v)
+        out = np.empty((self.B, self.H_q, self.d), dtype=np.float64)
+        rc = self.lib.oracle_decode_step(self.h, _ptr(q), _ptr(k), _ptr(v), seq_len, _ptr(out))
+        if rc != 0:
+            raise ValueError(f"oracle_decode_step failed with {rc}")
+        return out
+
+    def exact_topk(self, q, k, v, seq_len):
+        q, k, v = _u16(q), _u16(k), _u16(v)
+        self._check_kv(k, v)
+        out = np.empty((self.B, self.H_q, self.d), dtype=np.float64)
+        idx = np.empty((self.B, self.H_q, self.K), dtype=np.int32)
+        rc = self.lib.oracle_exact_topk(self.h, _ptr(q), _ptr(k), _ptr(v), seq_len, _ptr(out),
+                                        _ptr(idx))
+        if rc != 0:
+            raise ValueError(f"oracle_exact_topk failed with {rc}")
+        return out, idx
+
+    def stats(self) -> dict:
+        five = np.zeros(5, dtype=np.int64)
+        self.lib.oracle_stats(self.h, _ptr(five))
+        return dict(zip(("steps", "reuse", "fallback", "refresh", "cand_sum"), map(int, five)))
+
+    def last_step(self) -> dict:
+        sup = np.empty((self.B, self.H_q, self.K), dtype=np.int32)
+        path = np.empty((self.B, self.H_q), dtype=np.uint8)
+        rho = np.empty((self.B, self.H_q), dtype=np.float64)
+        ncand = np.empty((self.B, self.H_q), dtype=np.int32)
+        kth = np.empty((self.B, self.H_q), dtype=np.float64)
+        sel = np.empty((self.B, self.H_q, self.r), dtype=np.int32)
+        self.lib.oracle_last_step(self.h, _ptr(sup), _ptr(path), _ptr(rho), _ptr(ncand), _ptr(kth),
+                                  _ptr(sel))
+        return dict(support=sup, path=path, rho_max=rho, n_cand=ncand, kth_score=kth, sel=sel)
+
+    def last_candidates(self, b, h):
+        cand = np.empty(self.r * self.K + self.W + 1, dtype=np.int32)
+        n = self.lib.oracle_last_candidates(self.h, b * self.H_q + h, _ptr(cand))
+        return None if n < 0 else cand[:n].copy()
+
+    def export_state(self):
+        qbar = np.empty((self.B, self.H_q, self.M, self.d), dtype=np.float64)
+        sup = np.empty((self.B, self.H_q, self.M, self.K), dtype=np.int32)
+        n_ins, t_dec = C.c_int64(), C.c_int64()
+        self.lib.oracle_export_state(self.h, _ptr(qbar), _ptr(sup), C.byref(n_ins), C.byref(t_dec))
+        return qbar, sup, int(n_ins.value), int(t_dec.value)
+
+    def import_state(self, qbar, sup, n_ins, t_dec):
+        qbar = np.ascontiguousarray(qbar, dtype=np.float64)
+        sup = np.ascontiguousarray(sup, dtype=np.int32)
+        assert qbar.shape == (self.B, self.H_q, self.M, self.d)
+        assert sup.shape == (self.B, self.H_q, self.M, self.K)
+        self.lib.oracle_import_state(self.h, _ptr(qbar), _ptr(sup), n_ins, t_dec)
