@@ -1,0 +1,162 @@
+/*
+ * retopk.h - C interface of the ReTopK decode-step library (CUDA, sm_100a).
+ *
+ * One call of retopk_decode_step() is one attention layer's decode step for a batch of
+ * B independent sequences: per query head it recalls the supports of the most similar
+ * cached queries, reranks the compact candidate set with exact current-query scores,
+ * attends over the K winners, falls back to full-history Exact Top-K when similarity is
+ * low or a refresh is due, and inserts the new (query, support) pair into its cache
+ * (Sec. 3.3 "Recall-Before-Rerank Selection", Sec. 3.4 "Reliable Reuse via Fallback and
+ * Refresh").  exact_topk_decode() is the paper's Exact Top-K attention (Sec. 3.2, Eq. 4,
+ * Eq. 1, Eq. 12), the comparator and the fallback path.
+ *
+ * Names: M = cache capacity (the paper's C), r = recalled entries (the paper's R),
+ * W = recent window, K = support size, tau = similarity threshold, R = refresh period in
+ * decode steps (the paper's T_r; 0 disables refresh).
+ *
+ * Conventions shared by every call
+ *   - All tensor pointers are DEVICE pointers on the device that was current at
+ *     retopk_create time, unless the argument name ends in _host.
+ *   - bf16 tensors are raw 16-bit patterns, innermost dimension d contiguous:
+ *       q, out           [B, H_q, d]
+ *       k_cache, v_cache [B, H_kv, max_seq_len, d]
+ *     Query head h reads KV head h / (H_q / H_kv).  Key indices are 0-based int32.
+ *   - seq_len counts the keys available INCLUDING the current token: the caller appends
+ *     k_t, v_t at position seq_len - 1 before the call.  The library never writes the
+ *     KV cache (except retopk_decode_step_host, which performs that append itself).
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls only
+ *     enqueue work; none synchronises except where stated.  A context must be driven from
+ *     one stream at a time.
+ *   - The caller owns q / k_cache / v_cache / out; the context owns its cache state and
+ *     workspaces, allocated once in create and released in destroy.  decode calls allocate
+ *     nothing.
+ *   - Return value: 0 on success, a negative RETOPK_E* code otherwise.  Inputs containing
+ *     NaN or Inf give unspecified (but memory-safe) results.  The kernels never trap.
+ */
+#ifndef RETOPK_H
+#define RETOPK_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct retopk_ctx retopk_ctx;
+
+enum {
+    RETOPK_OK = 0,
+    RETOPK_EINVAL = -1,      /* bad argument (null pointer, size out of range) */
+    RETOPK_EUNSUPPORTED = -2,/* legal but not built (d not 64/128, H_q/H_kv > 16, ...) */
+    RETOPK_ENOMEM = -3,      /* device allocation failed in create */
+    RETOPK_ECUDA = -4        /* a CUDA runtime call or launch failed */
+};
+
+enum { RETOPK_PATH_REUSE = 0, RETOPK_PATH_FALLBACK = 1, RETOPK_PATH_REFRESH = 2 };
+
+/* Bits of retopk_stats_t.status (sticky until retopk_reset). */
+enum {
+    RETOPK_STATUS_BAD_INDEX = 1u  /* a stored support held an index >= seq_len; it was skipped */
+};
+
+/* Counters since create/reset, summed over every (sequence, query head). */
+typedef struct {
+    int64_t steps;       /* head-steps taken = reuse + fallback + refresh */
+    int64_t reuse;       /* Eq. 13 "otherwise" branch */
+    int64_t fallback;    /* rho_max < tau (includes the empty cache) */
+    int64_t refresh;     /* scheduled refresh (counted as refresh even if rho_max < tau) */
+    int64_t cand_sum;    /* sum of candidate-set sizes |A_t| over reuse head-steps (Eq. 9) */
+    int64_t slow_select; /* exact-path selections that needed the multi-pass fallback */
+    uint32_t status;     /* RETOPK_STATUS_* bits */
+    uint32_t reserved;
+} retopk_stats_t;
+
+#define RETOPK_DEFAULT_MAX_SEQ_LEN 139264  /* 128K context + 8K decode steps */
+
+/*
+ * Create a context for one sequence (B = 1) with the default max_seq_len.  The nine
+ * parameters are the method's: head counts and head dim (Sec. 3.2), cache capacity M,
+ * recall count r, window W, support size K (Sec. 3.3), threshold tau and refresh period
+ * R (Sec. 3.4, Eq. 13).  The cache starts empty, so the first step takes the exact path.
+ * Constraints: H_q % H_kv == 0, H_q / H_kv <= 16, d in {64, 128}, 1 <= r <= M <= 1024,
+ * W >= 0, 1 <= K <= 4096, R >= 0; tau may be any float (<= -1 never falls back on
+ * similarity, > 1 always does).
+ */
+int retopk_create(retopk_ctx** ctx, int H_q, int H_kv, int d, int M, int r, int W, int K,
+                  float tau, int R);
+
+/* Same, for B independent sequences sharing seq_len, and an explicit KV-cache row count
+ * (max_seq_len fixes the k_cache / v_cache strides and the workspace sizes;
+ * 1 <= max_seq_len <= 1048576). */
+int retopk_create_batched(retopk_ctx** ctx, int B, int H_q, int H_kv, int d, int M, int r, int W,
+                          int K, float tau, int R, int64_t max_seq_len);
+
+/* Release the context and its device memory (synchronises the device). */
+int retopk_destroy(retopk_ctx* ctx);
+
+/* Empty every cache, set the decode offset t_dec to 0 and clear the counters. */
+int retopk_reset(retopk_ctx* ctx, void* stream);
+
+/*
+ * One ReTopK decode step (Sec. 3.3-3.4: Eq. 6-13 and the cache insert) for all B * H_q
+ * heads.  q, k_cache, v_cache are read, out is written; 1 <= seq_len <= max_seq_len.
+ * The path of each head is decided on the device; no host synchronisation happens.
+ * Advances t_dec and the insert count by one.
+ */
+int retopk_decode_step(retopk_ctx* ctx, const void* q, const void* k_cache, const void* v_cache,
+                       int64_t seq_len, void* out, void* stream);
+
+/*
+ * The same step for a caller whose per-token tensors live in HOST memory: copies q_host
+ * [B,H_q,d] to the device, appends k_new_host / v_new_host [B,H_kv,d] at position
+ * seq_len - 1 of the device-resident k_cache / v_cache, runs the step, copies the result
+ * to out_host [B,H_q,d] and synchronises `stream`.  Pinned host buffers keep the copies
+ * asynchronous; pageable ones work but serialise.
+ */
+int retopk_decode_step_host(retopk_ctx* ctx, const void* q_host, const void* k_new_host,
+                            const void* v_new_host, void* k_cache, void* v_cache,
+                            int64_t seq_len, void* out_host, void* stream);
+
+/*
+ * Exact Top-K attention (Eq. 4: score every key; Eq. 1: global Top-K, ties to the lower
+ * index; Eq. 12: softmax . V over the support) for all B * H_q heads.  Stateless with
+ * respect to the caches (uses the context only for shapes and workspaces).
+ * idx_out: device int32 [B,H_q,K], ascending, -1 padded when seq_len < K; may be NULL.
+ */
+int exact_topk_decode(retopk_ctx* ctx, const void* q, const void* k_cache, const void* v_cache,
+                      int64_t seq_len, void* out, int32_t* idx_out, void* stream);
+
+/* Copy the counters to host memory.  Synchronises the device. */
+int retopk_stats(retopk_ctx* ctx, retopk_stats_t* stats_host);
+
+/*
+ * What the most recent retopk_decode_step did, per head (device pointers, any may be
+ * NULL): support [B,H_q,K] int32 ascending (-1 padded), path [B,H_q] uint8
+ * (RETOPK_PATH_*), rho_max [B,H_q] float (-inf for an empty cache), n_cand [B,H_q] int32
+ * (|A_t| on reuse steps, seq_len otherwise).  Enqueued on `stream`.
+ */
+int retopk_last_step(retopk_ctx* ctx, int32_t* support, uint8_t* path, float* rho_max,
+                     int32_t* n_cand, void* stream);
+
+/*
+ * Cache state out / in (device pointers): qbar [B,H_q,M,d] float32 normalised queries,
+ * supports [B,H_q,M,K] int32 (ascending, -1 padded); the entry inserted n-th sits in slot
+ * n % M.  n_inserted and t_dec are host scalars.  Import replaces the whole state (this
+ * is how a test re-seeds the caches from a reference each step); it does not touch the
+ * counters.  Enqueued on `stream`.
+ */
+int retopk_export_state(retopk_ctx* ctx, float* qbar, int32_t* supports, int64_t* n_inserted,
+                        int64_t* t_dec, void* stream);
+int retopk_import_state(retopk_ctx* ctx, const float* qbar, const int32_t* supports,
+                        int64_t n_inserted, int64_t t_dec, void* stream);
+
+/* Number of kernels the last decode call of this context launched (host-side count). */
+int retopk_last_launch_count(const retopk_ctx* ctx);
+
+/* Static description of an error code. */
+const char* retopk_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RETOPK_H */

@@ -1,0 +1,347 @@
+// Host side of the ReTopK library: context, argument checks, launch sequence, C interface.
+#include "retopk_kernels.cuh"
+
+#include <math.h>
+#include <new>
+#include <stdio.h>
+#include <string.h>
+
+#include "../../include/retopk.h"
+
+using namespace retopk;
+
+struct retopk_ctx {
+    int device;
+    int B, Hq, Hkv, G, d, M, r, W, K, R, cap;
+    float tau;
+    long long max_seq_len, score_stride;
+    long long n_ins, t_dec;
+    int NS;
+    int num_sms;
+    size_t smem_recall, smem_finish;
+    // device state
+    float* qbar_cache;
+    int32_t* sup_cache;
+    uint8_t* ws_path;
+    float* ws_rho;
+    int32_t* ws_ncand;
+    int32_t* ws_cand;
+    float* ws_scores;
+    long long* counters;
+    unsigned int* status;
+    unsigned long long* slow_select;
+    // staging for the host-buffer entry point
+    uint16_t* stage_q;
+    uint16_t* stage_out;
+    uint16_t* stage_kv;   // [2][B*Hkv*d]
+    int last_launches;
+};
+
+namespace {
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+struct DeviceGuard {
+    int prev;
+    bool ok;
+    explicit DeviceGuard(int dev) : prev(-1), ok(false) {
+        if (cudaGetDevice(&prev) != cudaSuccess) return;
+        ok = (prev == dev) || cudaSetDevice(dev) == cudaSuccess;
+    }
+    ~DeviceGuard() { if (ok && prev >= 0) cudaSetDevice(prev); }
+};
+
+template <class T>
+bool dev_alloc(T** p, size_t count) {
+    return cudaMalloc(reinterpret_cast<void**>(p), count * sizeof(T) > 0 ? count * sizeof(T) : 16) == cudaSuccess;
+}
+
+void free_all(retopk_ctx* c) {
+    cudaFree(c->qbar_cache); cudaFree(c->sup_cache); cudaFree(c->ws_path); cudaFree(c->ws_rho);
+    cudaFree(c->ws_ncand); cudaFree(c->ws_cand); cudaFree(c->ws_scores); cudaFree(c->counters);
+    cudaFree(c->status); cudaFree(c->slow_select); cudaFree(c->stage_q); cudaFree(c->stage_out);
+    cudaFree(c->stage_kv);
+}
+
+StepArgs make_args(const retopk_ctx* c, const void* q, const void* k, const void* v, long long L,
+                   void* out, int mode) {
+    StepArgs a;
+    memset(&a, 0, sizeof a);
+    a.B = c->B; a.Hq = c->Hq; a.Hkv = c->Hkv; a.G = c->G; a.d = c->d; a.M = c->M; a.r = c->r;
+    a.W = c->W; a.K = c->K; a.cap = c->cap;
+    a.max_seq_len = c->max_seq_len; a.score_stride = c->score_stride;
+    a.L = (int)L;
+    a.tau = c->tau;
+    a.scale = 1.0f / sqrtf((float)c->d);
+    a.fill = (int)(c->n_ins < c->M ? c->n_ins : c->M);
+    a.slot = (int)(c->n_ins % c->M);
+    a.refresh = (c->R > 0 && c->t_dec > 0 && c->t_dec % c->R == 0) ? 1 : 0;
+    a.mode = mode;
+    a.NS = c->NS;
+    // scan grid: enough CTAs to fill the machine several times over, in whole 128-row blocks
+    long long rows = (L * c->B * c->Hkv + (long long)c->num_sms * 8 - 1) / ((long long)c->num_sms * 8);
+    rows = (rows + 127) / 128 * 128;
+    if (rows < 128) rows = 128;
+    if (rows > 1024) rows = 1024;
+    a.rows_per_cta = (int)rows;
+    a.q = static_cast<const uint16_t*>(q);
+    a.k = static_cast<const uint16_t*>(k);
+    a.v = static_cast<const uint16_t*>(v);
+    a.out = static_cast<uint16_t*>(out);
+    a.qbar_cache = c->qbar_cache; a.sup_cache = c->sup_cache;
+    a.ws_path = c->ws_path; a.ws_rho = c->ws_rho; a.ws_ncand = c->ws_ncand; a.ws_cand = c->ws_cand;
+    a.ws_scores = c->ws_scores; a.counters = c->counters; a.status = c->status;
+    a.slow_select = c->slow_select;
+    a.idx_out = nullptr;
+    return a;
+}
+
+int launch_scan(const retopk_ctx* c, const StepArgs& a, cudaStream_t s) {
+    dim3 grid((unsigned)((a.L + a.rows_per_cta - 1) / a.rows_per_cta), (unsigned)(c->B * c->Hkv));
+    const int ntile = (c->G + 7) / 8;
+    if (c->d == 128 && ntile == 1) scan_kernel<128, 1><<<grid, SCAN_THREADS, 0, s>>>(a);
+    else if (c->d == 128) scan_kernel<128, 2><<<grid, SCAN_THREADS, 0, s>>>(a);
+    else if (ntile == 1) scan_kernel<64, 1><<<grid, SCAN_THREADS, 0, s>>>(a);
+    else scan_kernel<64, 2><<<grid, SCAN_THREADS, 0, s>>>(a);
+    return cudaGetLastError() == cudaSuccess ? RETOPK_OK : RETOPK_ECUDA;
+}
+
+int launch_finish(const retopk_ctx* c, const StepArgs& a, cudaStream_t s) {
+    const unsigned grid = (unsigned)(c->B * c->Hq);
+    if (c->d == 128) finish_kernel<128><<<grid, FINISH_THREADS, c->smem_finish, s>>>(a);
+    else finish_kernel<64><<<grid, FINISH_THREADS, c->smem_finish, s>>>(a);
+    return cudaGetLastError() == cudaSuccess ? RETOPK_OK : RETOPK_ECUDA;
+}
+
+int check_step_args(const retopk_ctx* c, const void* q, const void* k, const void* v, long long L,
+                    const void* out) {
+    if (!c || !q || !k || !v || !out) return RETOPK_EINVAL;
+    if (L < 1 || L > c->max_seq_len) return RETOPK_EINVAL;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v)) return RETOPK_EINVAL;
+    return RETOPK_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int retopk_create_batched(retopk_ctx** out, int B, int H_q, int H_kv, int d, int M, int r, int W,
+                          int K, float tau, int R, int64_t max_seq_len) {
+    if (!out) return RETOPK_EINVAL;
+    *out = nullptr;
+    if (B < 1 || H_q < 1 || H_kv < 1 || H_q % H_kv != 0 || M < 1 || r < 1 || r > M || W < 0 || K < 1 ||
+        R < 0 || max_seq_len < 1 || d < 1)
+        return RETOPK_EINVAL;
+    if ((d != 64 && d != 128) || H_q / H_kv > 16 || M > 1024 || K > 4096 || max_seq_len > 1048576 ||
+        (long long)B * H_kv > 65535)
+        return RETOPK_EUNSUPPORTED;
+    if (tau != tau) return RETOPK_EINVAL;
+    retopk_ctx* c = new (std::nothrow) retopk_ctx;
+    if (!c) return RETOPK_ENOMEM;
+    memset(c, 0, sizeof *c);
+    if (cudaGetDevice(&c->device) != cudaSuccess) { delete c; return RETOPK_ECUDA; }
+    c->B = B; c->Hq = H_q; c->Hkv = H_kv; c->G = H_q / H_kv; c->d = d; c->M = M; c->r = r; c->W = W;
+    c->K = K; c->R = R; c->tau = tau; c->max_seq_len = max_seq_len;
+    c->cap = r * K + W;
+    c->score_stride = (max_seq_len + 3) / 4 * 4;
+    c->NS = c->cap > NS_MIN ? c->cap : NS_MIN;
+    int sms = 0;
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, c->device);
+    c->num_sms = sms > 0 ? sms : 148;
+
+    const size_t head_words = (size_t)d + M + r + 8 + 4;
+    c->smem_recall = (((head_words + 3) & ~(size_t)3) + (size_t)(max_seq_len + 31) / 32) * 4;
+    c->smem_finish = ((size_t)c->NS * 2 + (size_t)K * 3 + SAMPLE_BINS + 32 + 8) * 4;
+    int max_smem = 0;
+    cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, c->device);
+    if ((size_t)max_smem < c->smem_recall || (size_t)max_smem < c->smem_finish) {
+        delete c;
+        return RETOPK_EUNSUPPORTED;
+    }
+    // opt in to the device maximum once; contexts of different sizes then coexist
+    cudaError_t e1 = cudaFuncSetAttribute(recall_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
+    cudaError_t e2 = (d == 128)
+        ? cudaFuncSetAttribute(finish_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem)
+        : cudaFuncSetAttribute(finish_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
+    if (e1 != cudaSuccess || e2 != cudaSuccess) { cudaGetLastError(); delete c; return RETOPK_ECUDA; }
+
+    const size_t nh = (size_t)B * H_q;
+    bool ok = dev_alloc(&c->qbar_cache, nh * M * d) && dev_alloc(&c->sup_cache, nh * M * K) &&
+              dev_alloc(&c->ws_path, nh) && dev_alloc(&c->ws_rho, nh) && dev_alloc(&c->ws_ncand, nh) &&
+              dev_alloc(&c->ws_cand, nh * c->cap) && dev_alloc(&c->ws_scores, nh * (size_t)c->score_stride) &&
+              dev_alloc(&c->counters, nh * 4) && dev_alloc(&c->status, 1) &&
+              dev_alloc(&c->slow_select, 1) && dev_alloc(&c->stage_q, nh * d) &&
+              dev_alloc(&c->stage_out, nh * d) && dev_alloc(&c->stage_kv, (size_t)2 * B * H_kv * d);
+    if (!ok) { cudaGetLastError(); free_all(c); delete c; return RETOPK_ENOMEM; }
+    *out = c;
+    int rc = retopk_reset(c, nullptr);
+    if (rc == RETOPK_OK && cudaStreamSynchronize(nullptr) != cudaSuccess) rc = RETOPK_ECUDA;
+    if (rc != RETOPK_OK) { free_all(c); delete c; *out = nullptr; }
+    return rc;
+}
+
+int retopk_create(retopk_ctx** ctx, int H_q, int H_kv, int d, int M, int r, int W, int K, float tau,
+                  int R) {
+    return retopk_create_batched(ctx, 1, H_q, H_kv, d, M, r, W, K, tau, R, RETOPK_DEFAULT_MAX_SEQ_LEN);
+}
+
+int retopk_destroy(retopk_ctx* c) {
+    if (!c) return RETOPK_EINVAL;
+    DeviceGuard g(c->device);
+    cudaDeviceSynchronize();
+    free_all(c);
+    delete c;
+    return RETOPK_OK;
+}
+
+int retopk_reset(retopk_ctx* c, void* stream) {
+    if (!c) return RETOPK_EINVAL;
+    const size_t nh = (size_t)c->B * c->Hq;
+    reset_kernel<<<c->num_sms * 4, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        c->qbar_cache, nh * c->M * c->d, c->sup_cache, nh * c->M * c->K, c->counters, nh * 4, c->status,
+        c->slow_select);
+    c->n_ins = 0;
+    c->t_dec = 0;
+    return cudaGetLastError() == cudaSuccess ? RETOPK_OK : RETOPK_ECUDA;
+}
+
+int retopk_decode_step(retopk_ctx* c, const void* q, const void* k_cache, const void* v_cache,
+                       int64_t seq_len, void* out, void* stream) {
+    int rc = check_step_args(c, q, k_cache, v_cache, seq_len, out);
+    if (rc != RETOPK_OK) return rc;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    StepArgs a = make_args(c, q, k_cache, v_cache, seq_len, out, MODE_RETOPK);
+    recall_kernel<<<(unsigned)(c->B * c->Hq), RECALL_THREADS, c->smem_recall, s>>>(a);
+    if (cudaGetLastError() != cudaSuccess) return RETOPK_ECUDA;
+    if ((rc = launch_scan(c, a, s)) != RETOPK_OK) return rc;
+    if ((rc = launch_finish(c, a, s)) != RETOPK_OK) return rc;
+    c->last_launches = 3;
+    c->n_ins += 1;
+    c->t_dec += 1;
+    return RETOPK_OK;
+}
+
+int exact_topk_decode(retopk_ctx* c, const void* q, const void* k_cache, const void* v_cache,
+                      int64_t seq_len, void* out, int32_t* idx_out, void* stream) {
+    int rc = check_step_args(c, q, k_cache, v_cache, seq_len, out);
+    if (rc != RETOPK_OK) return rc;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    StepArgs a = make_args(c, q, k_cache, v_cache, seq_len, out, MODE_EXACT);
+    a.idx_out = idx_out;
+    if ((rc = launch_scan(c, a, s)) != RETOPK_OK) return rc;
+    if ((rc = launch_finish(c, a, s)) != RETOPK_OK) return rc;
+    c->last_launches = 2;
+    return RETOPK_OK;
+}
+
+int retopk_decode_step_host(retopk_ctx* c, const void* q_host, const void* k_new_host,
+                            const void* v_new_host, void* k_cache, void* v_cache, int64_t seq_len,
+                            void* out_host, void* stream) {
+    if (!c || !q_host || !k_new_host || !v_new_host || !k_cache || !v_cache || !out_host)
+        return RETOPK_EINVAL;
+    if (seq_len < 1 || seq_len > c->max_seq_len) return RETOPK_EINVAL;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t row = (size_t)c->d * 2;
+    const size_t nq = (size_t)c->B * c->Hq * row, nkv = (size_t)c->B * c->Hkv;
+    if (cudaMemcpyAsync(c->stage_q, q_host, nq, cudaMemcpyHostToDevice, s) != cudaSuccess)
+        return RETOPK_ECUDA;
+    // append the current token's key / value row of every (sequence, KV head)
+    const size_t pitch = (size_t)c->max_seq_len * row;
+    char* kdst = static_cast<char*>(k_cache) + (size_t)(seq_len - 1) * row;
+    char* vdst = static_cast<char*>(v_cache) + (size_t)(seq_len - 1) * row;
+    if (cudaMemcpy2DAsync(kdst, pitch, k_new_host, row, row, nkv, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+        cudaMemcpy2DAsync(vdst, pitch, v_new_host, row, row, nkv, cudaMemcpyHostToDevice, s) != cudaSuccess)
+        return RETOPK_ECUDA;
+    int rc = retopk_decode_step(c, c->stage_q, k_cache, v_cache, seq_len, c->stage_out, stream);
+    if (rc != RETOPK_OK) return rc;
+    if (cudaMemcpyAsync(out_host, c->stage_out, nq, cudaMemcpyDeviceToHost, s) != cudaSuccess)
+        return RETOPK_ECUDA;
+    return cudaStreamSynchronize(s) == cudaSuccess ? RETOPK_OK : RETOPK_ECUDA;
+}
+
+int retopk_stats(retopk_ctx* c, retopk_stats_t* st) {
+    if (!c || !st) return RETOPK_EINVAL;
+    DeviceGuard g(c->device);
+    const size_t nh = (size_t)c->B * c->Hq;
+    long long* host = new (std::nothrow) long long[nh * 4];
+    if (!host) return RETOPK_ENOMEM;
+    unsigned int status = 0;
+    unsigned long long slow = 0;
+    bool ok = cudaDeviceSynchronize() == cudaSuccess &&
+              cudaMemcpy(host, c->counters, nh * 4 * sizeof(long long), cudaMemcpyDeviceToHost) == cudaSuccess &&
+              cudaMemcpy(&status, c->status, sizeof status, cudaMemcpyDeviceToHost) == cudaSuccess &&
+              cudaMemcpy(&slow, c->slow_select, sizeof slow, cudaMemcpyDeviceToHost) == cudaSuccess;
+    if (ok) {
+        memset(st, 0, sizeof *st);
+        for (size_t i = 0; i < nh; ++i) {
+            st->reuse += host[i * 4 + 0];
+            st->fallback += host[i * 4 + 1];
+            st->refresh += host[i * 4 + 2];
+            st->cand_sum += host[i * 4 + 3];
+        }
+        st->steps = st->reuse + st->fallback + st->refresh;
+        st->slow_select = (int64_t)slow;
+        st->status = status;
+    }
+    delete[] host;
+    return ok ? RETOPK_OK : RETOPK_ECUDA;
+}
+
+int retopk_last_step(retopk_ctx* c, int32_t* support, uint8_t* path, float* rho_max, int32_t* n_cand,
+                     void* stream) {
+    if (!c) return RETOPK_EINVAL;
+    if (c->n_ins < 1) return RETOPK_EINVAL;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t nh = (size_t)c->B * c->Hq;
+    bool ok = true;
+    if (support) {
+        const int slot = (int)((c->n_ins - 1) % c->M);
+        const size_t width = (size_t)c->K * 4;
+        ok = ok && cudaMemcpy2DAsync(support, width, c->sup_cache + (size_t)slot * c->K,
+                                     (size_t)c->M * width, width, nh, cudaMemcpyDeviceToDevice, s) == cudaSuccess;
+    }
+    if (path) ok = ok && cudaMemcpyAsync(path, c->ws_path, nh, cudaMemcpyDeviceToDevice, s) == cudaSuccess;
+    if (rho_max) ok = ok && cudaMemcpyAsync(rho_max, c->ws_rho, nh * 4, cudaMemcpyDeviceToDevice, s) == cudaSuccess;
+    if (n_cand) ok = ok && cudaMemcpyAsync(n_cand, c->ws_ncand, nh * 4, cudaMemcpyDeviceToDevice, s) == cudaSuccess;
+    return ok ? RETOPK_OK : RETOPK_ECUDA;
+}
+
+int retopk_export_state(retopk_ctx* c, float* qbar, int32_t* supports, int64_t* n_inserted,
+                        int64_t* t_dec, void* stream) {
+    if (!c) return RETOPK_EINVAL;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t nh = (size_t)c->B * c->Hq;
+    bool ok = true;
+    if (qbar) ok = ok && cudaMemcpyAsync(qbar, c->qbar_cache, nh * c->M * c->d * 4, cudaMemcpyDeviceToDevice, s) == cudaSuccess;
+    if (supports) ok = ok && cudaMemcpyAsync(supports, c->sup_cache, nh * c->M * c->K * 4, cudaMemcpyDeviceToDevice, s) == cudaSuccess;
+    if (n_inserted) *n_inserted = c->n_ins;
+    if (t_dec) *t_dec = c->t_dec;
+    return ok ? RETOPK_OK : RETOPK_ECUDA;
+}
+
+int retopk_import_state(retopk_ctx* c, const float* qbar, const int32_t* supports, int64_t n_inserted,
+                        int64_t t_dec, void* stream) {
+    if (!c || !qbar || !supports || n_inserted < 0 || t_dec < 0) return RETOPK_EINVAL;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t nh = (size_t)c->B * c->Hq;
+    bool ok = cudaMemcpyAsync(c->qbar_cache, qbar, nh * c->M * c->d * 4, cudaMemcpyDeviceToDevice, s) == cudaSuccess &&
+              cudaMemcpyAsync(c->sup_cache, supports, nh * c->M * c->K * 4, cudaMemcpyDeviceToDevice, s) == cudaSuccess;
+    c->n_ins = n_inserted;
+    c->t_dec = t_dec;
+    return ok ? RETOPK_OK : RETOPK_ECUDA;
+}
+
+int retopk_last_launch_count(const retopk_ctx* c) { return c ? c->last_launches : 0; }
+
+const char* retopk_strerror(int code) {
+    switch (code) {
+        case RETOPK_OK: return "ok";
+        case RETOPK_EINVAL: return "invalid argument";
+        case RETOPK_EUNSUPPORTED: return "configuration not supported by this build";
+        case RETOPK_ENOMEM: return "device memory allocation failed";
+        case RETOPK_ECUDA: return "CUDA runtime call or kernel launch failed";
+        default: return "unknown error";
+    }
+}
+
+}  // extern "C"

@@ -1,0 +1,100 @@
+"""Shared comparison code for the GPU parity tests (CUDA library vs the fp64 oracle)."""
+import math
+
+import numpy as np
+import torch
+
+from paper_2607_27692_b200 import retopk as rt
+from paper_2607_27692_b200 import workload as wl
+
+ABS_TOL, REL_TOL = 2e-2, 1e-2        # outputs: bf16 I/O, fp32 accumulate
+SCORE_BAND = 1e-3                    # relative band around the K-th score
+TAU_BAND = 1e-4                      # similarity band around tau
+
+
+def to_dev(bits):
+    return rt.bf16_tensor_from_bits(bits, device="cuda")
+
+
+def assert_outputs_close(out_gpu, out_ref, what=""):
+    g = out_gpu.float().cpu().numpy().astype(np.float64)
+    err = np.abs(g - out_ref)
+    tol = ABS_TOL + REL_TOL * np.abs(out_ref)
+    assert (err <= tol).all(), f"{what}: max err {err.max():.4g} (worst excess {(err - tol).max():.4g})"
+
+
+def assert_support_matches(sup_gpu, sup_ref, q_bits, k_head_bits, kth_score, what=""):
+    """Index sets must agree except for positions scoring within the band of the K-th score."""
+    sg, sr = sup_gpu[sup_gpu >= 0], sup_ref[sup_ref >= 0]
+    assert len(sg) == len(sr), f"{what}: support sizes differ ({len(sg)} vs {len(sr)})"
+    assert (np.diff(sg) > 0).all(), f"{what}: GPU support not strictly ascending"
+    diff = np.setxor1d(sg, sr)
+    if len(diff) == 0:
+        return 0
+    q64 = wl.bf16_bits_to_f64(q_bits)
+    s = wl.bf16_bits_to_f64(k_head_bits[diff]) @ q64 / math.sqrt(len(q64))
+    band = SCORE_BAND * max(abs(kth_score), 1e-30)
+    assert (np.abs(s - kth_score) <= band).all(), (
+        f"{what}: {len(diff)} positions differ, worst gap {np.abs(s - kth_score).max():.3g} "
+        f"vs band {band:.3g}")
+    return len(diff)
+
+
+def teacher_forced_run(cfg, st, steps, oracle, gpu, k_dev, v_dev, b_map=None, check_out=True):
+    """Step both sides with the GPU caches re-seeded from the oracle before every step.
+
+    ``oracle`` may cover a subset of the GPU's sequences: ``b_map[i]`` is the GPU batch row of
+    oracle row ``i`` (the stream ``st`` then holds the oracle's rows).
+    Returns counts of excused events.
+    """
+    G = cfg.H_q // cfg.H_kv
+    b_map = list(range(oracle.B)) if b_map is None else b_map
+    full = len(b_map) == gpu.B
+    excused_flips = excused_pos = 0
+    q_full = None
+    for t in range(steps):
+        L = st.seq_len(t)
+        qbar, sup, n_ins, t_dec = oracle.export_state()
+        if full:
+            gq = torch.from_numpy(qbar.astype(np.float32)).cuda()
+            gs = torch.from_numpy(sup).cuda()
+        else:
+            gq, gs, _, _ = gpu.export_state()
+            idx = torch.tensor(b_map, device="cuda")
+            gq[idx] = torch.from_numpy(qbar.astype(np.float32)).cuda()
+            gs[idx] = torch.from_numpy(sup).cuda()
+        gpu.import_state(gq, gs, n_ins, t_dec)
+        if full:
+            q_dev = to_dev(st.q[t])
+        else:
+            q_full = torch.zeros(gpu.q_shape, dtype=torch.bfloat16, device="cuda") if q_full is None else q_full
+            q_full[torch.tensor(b_map, device="cuda")] = to_dev(st.q[t])
+            q_dev = q_full
+        out_g = gpu.decode_step(q_dev, k_dev, v_dev, L)
+        out_o = oracle.decode_step(st.q[t], st.k, st.v, L)
+        lo, lg = oracle.last_step(), gpu.last_step()
+        g_path = lg["path"].cpu().numpy()
+        g_sup = lg["support"].cpu().numpy()
+        g_rho = lg["rho_max"].cpu().numpy()
+        g_nc = lg["n_cand"].cpu().numpy()
+        for i, b in enumerate(b_map):
+            for h in range(cfg.H_q):
+                what = f"step {t} seq {b} head {h}"
+                rho_o = lo["rho_max"][i, h]
+                if np.isfinite(rho_o):
+                    assert abs(g_rho[b, h] - rho_o) <= 2e-5, f"{what}: rho_max {g_rho[b, h]} vs {rho_o}"
+                else:
+                    assert g_rho[b, h] == rho_o
+                if g_path[b, h] != lo["path"][i, h]:
+                    assert abs(rho_o - oracle.tau) <= TAU_BAND, (
+                        f"{what}: path {g_path[b, h]} vs {lo['path'][i, h]}, rho_max {rho_o}")
+                    excused_flips += 1
+                    continue
+                if lo["path"][i, h] == 0:
+                    assert g_nc[b, h] == lo["n_cand"][i, h], f"{what}: n_cand"
+                excused_pos += assert_support_matches(
+                    g_sup[b, h], lo["support"][i, h], st.q[t, i, h], st.k[i, h // G],
+                    lo["kth_score"][i, h], what)
+                if check_out:
+                    assert_outputs_close(out_g[b, h], out_o[i, h], what)
+    return dict(flips=excused_flips, positions=excused_pos)

@@ -1,0 +1,277 @@
+"""GPU parity: the CUDA library against the fp64 oracle, element by element (run with -m gpu).
+
+Rules: path decisions and index sets are bit-exact except for positions whose fp64 score is
+within 1e-3 relative of the K-th score and steps whose rho_max is within 1e-4 of tau;
+outputs within 2e-2 absolute + 1e-2 relative (bf16 I/O, fp32 accumulation).  In the
+teacher-forced runs the GPU caches are overwritten with the oracle's before every step so
+that an excused difference cannot compound.
+"""
+import json
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2607_27692_b200 import workload as wl
+
+pytestmark = pytest.mark.gpu
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+@pytest.fixture(scope="module")
+def rt():
+    from paper_2607_27692_b200 import build, retopk
+    build.build()
+    retopk.load()
+    return retopk
+
+
+@pytest.fixture(scope="module")
+def P():
+    import parity
+    return parity
+
+
+def bits(x):
+    return wl.f32_to_bf16_bits(np.asarray(x, dtype=np.float32))
+
+
+# ------------------------------------------------------------------ Exact Top-K
+
+@pytest.mark.parametrize("B,H_q,H_kv,d,L,K,Lmax", [
+    (1, 1, 1, 64, 2112, 64, 2112),        # the tiny configuration's shape
+    (2, 8, 2, 128, 5000, 512, 5003),      # several scan tiles and a ragged tail
+    (1, 4, 4, 128, 9000, 100, 9001),      # longer than the threshold sample
+    (1, 16, 1, 64, 777, 33, 800),         # two head tiles per group
+    (1, 2, 1, 128, 300, 512, 300),        # fewer keys than K
+    (1, 32, 8, 128, 20000, 2048, 20480),  # large K
+])
+def test_exact_topk_decode_matches_oracle(rt, P, oracle_mod, B, H_q, H_kv, d, L, K, Lmax):
+    rng = np.random.default_rng(L + K)
+    k = bits(rng.standard_normal((B, H_kv, Lmax, d)))
+    v = bits(rng.standard_normal((B, H_kv, Lmax, d)))
+    q = bits(rng.standard_normal((B, H_q, d)))
+    o = oracle_mod.Oracle(B, H_q, H_kv, d, 4, 2, 8, K, 0.9, 0, Lmax)
+    ref_out, ref_idx = o.exact_topk(q, k, v, L)
+    g = rt.ReTopK(B, H_q, H_kv, d, 4, 2, 8, K, 0.9, 0, Lmax)
+    idx = torch.full((B, H_q, K), -7, dtype=torch.int32, device="cuda")
+    out = g.exact_topk_decode(P.to_dev(q), P.to_dev(k), P.to_dev(v), L, idx_out=idx)
+    idx = idx.cpu().numpy()
+    G = H_q // H_kv
+    for b in range(B):
+        for h in range(H_q):
+            srt = np.sort(ref_idx[b, h][ref_idx[b, h] >= 0])
+            q64 = wl.bf16_bits_to_f64(q[b, h])
+            kth = (wl.bf16_bits_to_f64(k[b, h // G, srt]) @ q64 / np.sqrt(d)).min()
+            P.assert_support_matches(idx[b, h], ref_idx[b, h], q[b, h], k[b, h // G], kth,
+                                     f"seq {b} head {h}")
+    P.assert_outputs_close(out, ref_out, "exact_topk_decode")
+    assert g.stats()["slow_select"] == 0
+    assert g.last_launch_count() == 2
+
+
+def test_exact_ties_are_bit_exact(rt, P, oracle_mod):
+    """Integer inputs: scores tie exactly and are exact in fp32, so indices must be identical."""
+    B, H_q, H_kv, d, L, K = 1, 4, 2, 64, 3000, 128
+    rng = np.random.default_rng(11)
+    kf = rng.integers(-2, 3, size=(B, H_kv, L, d)).astype(np.float32)
+    kf[0, 0, 5] = 0.0
+    kf[0, 0, 6] = -0.0
+    qf = rng.integers(-1, 2, size=(B, H_q, d)).astype(np.float32)
+    k, v, q = bits(kf), bits(rng.standard_normal((B, H_kv, L, d))), bits(qf)
+    o = oracle_mod.Oracle(B, H_q, H_kv, d, 4, 2, 8, K, 0.9, 0, L)
+    ref_out, ref_idx = o.exact_topk(q, k, v, L)
+    g = rt.ReTopK(B, H_q, H_kv, d, 4, 2, 8, K, 0.9, 0, L)
+    idx = torch.empty((B, H_q, K), dtype=torch.int32, device="cuda")
+    out = g.exact_topk_decode(P.to_dev(q), P.to_dev(k), P.to_dev(v), L, idx_out=idx)
+    assert np.array_equal(idx.cpu().numpy(), ref_idx)
+    P.assert_outputs_close(out, ref_out, "ties")
+
+
+def test_degenerate_scores_take_the_multi_pass_path(rt, P, oracle_mod):
+    """All keys identical: every score ties, the support is the first K indices."""
+    B, H_q, H_kv, d, L, K = 1, 2, 1, 128, 20000, 512
+    rng = np.random.default_rng(12)
+    k = np.broadcast_to(bits(rng.standard_normal((1, 1, 1, d))), (B, H_kv, L, d)).copy()
+    v = bits(rng.standard_normal((B, H_kv, L, d)))
+    q = bits(rng.standard_normal((B, H_q, d)))
+    o = oracle_mod.Oracle(B, H_q, H_kv, d, 4, 2, 8, K, 0.9, 0, L)
+    ref_out, ref_idx = o.exact_topk(q, k, v, L)
+    assert np.array_equal(ref_idx[0, 0], np.arange(K))
+    g = rt.ReTopK(B, H_q, H_kv, d, 4, 2, 8, K, 0.9, 0, L)
+    idx = torch.empty((B, H_q, K), dtype=torch.int32, device="cuda")
+    out = g.exact_topk_decode(P.to_dev(q), P.to_dev(k), P.to_dev(v), L, idx_out=idx)
+    assert np.array_equal(idx.cpu().numpy(), ref_idx)
+    P.assert_outputs_close(out, ref_out, "degenerate")
+    assert g.stats()["slow_select"] == B * H_q
+
+
+# ------------------------------------------------------------------ ReTopK steps
+
+def stream_case(rt, P, oracle_mod, cfg, steps, **override):
+    st = wl.make_stream(cfg, steps=steps)
+    o = oracle_mod.Oracle.from_config(cfg, **override)
+    g = rt.ReTopK.from_config(cfg, **override)
+    return st, o, g, P.to_dev(st.k), P.to_dev(st.v)
+
+
+def test_tiny_config_teacher_forced(rt, P, oracle_mod):
+    cfg = wl.CONFIGS["tiny"]
+    st, o, g, k, v = stream_case(rt, P, oracle_mod, cfg, cfg.steps)
+    ex = P.teacher_forced_run(cfg, st, cfg.steps, o, g, k, v)
+    so, sg = o.stats(), g.stats()
+    assert ex["flips"] == 0
+    for key in ("steps", "reuse", "fallback", "refresh", "cand_sum"):
+        assert sg[key] == so[key], key
+    assert so["reuse"] > so["fallback"] > 0 and so["refresh"] == 3
+    assert sg["status"] == 0
+
+
+@pytest.mark.parametrize("override", [{"r": 1}, {"M": 1, "r": 1}, {"W": 0}, {"R": 0}, {"tau": -2.0},
+                                      {"tau": 2.0}, {"K": 300, "W": 5}])
+def test_parameter_corners_teacher_forced(rt, P, oracle_mod, override):
+    cfg = wl.CONFIGS["tiny"].replace(context=700, steps=24, B=2, H_q=4, H_kv=2)
+    st, o, g, k, v = stream_case(rt, P, oracle_mod, cfg, 24, **override)
+    P.teacher_forced_run(cfg, st, 24, o, g, k, v)
+    so, sg = o.stats(), g.stats()
+    for key in ("steps", "reuse", "fallback", "refresh", "cand_sum"):
+        assert sg[key] == so[key], key
+
+
+def test_llama_shape_teacher_forced(rt, P, oracle_mod):
+    """32 query / 8 KV heads, d = 128, 16K context: the second configuration, first 40 steps."""
+    cfg = wl.CONFIGS["llama16k"]
+    steps = 40
+    st, o, g, k, v = stream_case(rt, P, oracle_mod, cfg, steps)
+    ex = P.teacher_forced_run(cfg, st, steps, o, g, k, v)
+    so, sg = o.stats(), g.stats()
+    assert so["reuse"] > 0 and so["fallback"] > 0 and so["refresh"] == 32
+    # counters agree up to the excused decisions
+    assert abs(sg["reuse"] - so["reuse"]) <= ex["flips"]
+    assert sg["slow_select"] == 0 and sg["status"] == 0
+
+
+def test_free_running_stays_close(rt, P, oracle_mod):
+    """No re-seeding: decisions may drift apart at excused ties, outputs must stay aligned."""
+    cfg = wl.CONFIGS["tiny"].replace(B=2, H_q=4, H_kv=2)
+    steps = 48
+    st, o, g, k, v = stream_case(rt, P, oracle_mod, cfg, steps)
+    cos = []
+    for t in range(steps):
+        L = st.seq_len(t)
+        out_g = g.decode_step(P.to_dev(st.q[t]), k, v, L).float().cpu().numpy().astype(np.float64)
+        out_o = o.decode_step(st.q[t], st.k, st.v, L)
+        cos.append((out_g * out_o).sum(-1) / (np.linalg.norm(out_g, axis=-1) * np.linalg.norm(out_o, axis=-1)))
+    cos = np.array(cos)
+    assert np.median(cos) > 0.999 and cos.min() > 0.98
+    so, sg = o.stats(), g.stats()
+    assert sg["steps"] == so["steps"] and sg["refresh"] == so["refresh"]
+    assert abs(sg["reuse"] - so["reuse"]) <= 0.05 * so["steps"]
+
+
+def test_forced_fallback_equals_exact_topk_decode(rt, P, oracle_mod):
+    """tau > 1: every step is the exact path, so decode_step and exact_topk_decode agree bit for bit."""
+    cfg = wl.CONFIGS["tiny"].replace(context=3000, steps=6, B=2, H_q=8, H_kv=2, d=128)
+    st = wl.make_stream(cfg, steps=6)
+    g = rt.ReTopK.from_config(cfg, tau=2.0, R=0)
+    k, v = P.to_dev(st.k), P.to_dev(st.v)
+    for t in range(6):
+        q = P.to_dev(st.q[t])
+        a = g.decode_step(q, k, v, st.seq_len(t))
+        idx = torch.empty((cfg.B, cfg.H_q, cfg.K), dtype=torch.int32, device="cuda")
+        b = g.exact_topk_decode(q, k, v, st.seq_len(t), idx_out=idx)
+        assert torch.equal(a.view(torch.int16), b.view(torch.int16))
+        assert torch.equal(g.last_step()["support"], idx)
+    s = g.stats()
+    assert s["fallback"] == 6 * cfg.B * cfg.H_q and s["reuse"] == 0
+
+
+def test_hand_trace_decisions_on_gpu(rt, P):
+    """The six-step hand trace, zero-padded to d = 64 (decisions and supports only)."""
+    with open(os.path.join(GOLDEN, "hand_trace.json")) as f:
+        gold = json.load(f)
+    p = gold["params"]
+    d = 64
+    keys = np.zeros((1, 1, len(gold["keys"]), d), dtype=np.float32)
+    keys[0, 0, :, :2] = np.array(gold["keys"], dtype=np.float32)
+    vals = np.zeros_like(keys)
+    vals[0, 0, :, :2] = np.array(gold["values"], dtype=np.float32)
+    k, v = P.to_dev(bits(keys)), P.to_dev(bits(vals))
+    g = rt.ReTopK(1, 1, 1, d, p["M"], p["r"], p["W"], p["K"], p["tau"], p["R"], keys.shape[2])
+    names = {"REUSE": 0, "FALLBACK": 1, "REFRESH": 2}
+    for t, step in enumerate(gold["steps"]):
+        q = np.zeros((1, 1, d), dtype=np.float32)
+        q[0, 0, :2] = step["q"]
+        g.decode_step(P.to_dev(bits(q)), k, v, step["L"])
+        last = g.last_step()
+        assert int(last["path"][0, 0]) == names[step["path"]], f"step {t}"
+        assert last["support"][0, 0].tolist() == step["support"], f"step {t}"
+        if step["candidates"] is not None:
+            assert int(last["n_cand"][0, 0]) == len(step["candidates"])
+    s = g.stats()
+    assert {key: s[key] for key in gold["stats"]} == gold["stats"]
+
+
+def test_steps_are_deterministic(rt, P):
+    cfg = wl.CONFIGS["tiny"].replace(context=4000, steps=20, B=2, H_q=8, H_kv=2, d=128)
+    st = wl.make_stream(cfg, steps=20)
+    k, v = P.to_dev(st.k), P.to_dev(st.v)
+    runs = []
+    for _ in range(2):
+        g = rt.ReTopK.from_config(cfg)
+        outs = [g.decode_step(P.to_dev(st.q[t]), k, v, st.seq_len(t)).clone() for t in range(20)]
+        runs.append((torch.stack(outs), g.export_state(), g.stats()))
+    assert torch.equal(runs[0][0].view(torch.int16), runs[1][0].view(torch.int16))
+    assert torch.equal(runs[0][1][0], runs[1][1][0]) and torch.equal(runs[0][1][1], runs[1][1][1])
+    assert runs[0][2] == runs[1][2]
+
+
+def test_host_entry_point_matches_device_entry_point(rt, P):
+    cfg = wl.CONFIGS["tiny"].replace(context=1500, steps=10, B=2, H_q=8, H_kv=2, d=128)
+    st = wl.make_stream(cfg, steps=10)
+    g_dev, g_host = rt.ReTopK.from_config(cfg), rt.ReTopK.from_config(cfg)
+    k, v = P.to_dev(st.k), P.to_dev(st.v)
+    # the host path appends each token's key / value itself: start from the prefill only
+    k2, v2 = k.clone(), v.clone()
+    k2[:, :, cfg.context:] = 0
+    v2[:, :, cfg.context:] = 0
+    out_host = torch.empty(g_host.q_shape, dtype=torch.bfloat16).pin_memory()
+    for t in range(10):
+        L = st.seq_len(t)
+        a = g_dev.decode_step(P.to_dev(st.q[t]), k, v, L)
+        qh = rt.bf16_tensor_from_bits(st.q[t], pin=True)
+        kn = rt.bf16_tensor_from_bits(st.k[:, :, L - 1], pin=True)
+        vn = rt.bf16_tensor_from_bits(st.v[:, :, L - 1], pin=True)
+        g_host.decode_step_host(qh, kn, vn, k2, v2, L, out_host)
+        assert torch.equal(a.cpu().view(torch.int16), out_host.view(torch.int16))
+    assert torch.equal(k, k2) and torch.equal(v, v2)
+
+
+def test_corrupt_imported_support_is_flagged_not_followed(rt, P):
+    cfg = wl.CONFIGS["tiny"].replace(context=500, steps=4)
+    st = wl.make_stream(cfg, steps=4)
+    g = rt.ReTopK.from_config(cfg, tau=-2.0)
+    k, v = P.to_dev(st.k), P.to_dev(st.v)
+    g.decode_step(P.to_dev(st.q[0]), k, v, st.seq_len(0))
+    qbar, sup, n_ins, t_dec = g.export_state()
+    sup[0, 0, 0, :5] = 10 ** 6          # far beyond seq_len
+    g.import_state(qbar, sup, n_ins, t_dec)
+    out = g.decode_step(P.to_dev(st.q[1]), k, v, st.seq_len(1))
+    assert torch.isfinite(out.float()).all()
+    s = g.stats()
+    assert s["status"] & rt.STATUS_BAD_INDEX
+    assert int(g.last_step()["support"].max()) < st.seq_len(1)
+
+
+def test_bad_arguments_return_errors(rt, P):
+    g = rt.ReTopK(1, 2, 1, 64, 4, 2, 8, 16, 0.9, 0, 256)
+    q = torch.zeros(g.q_shape, dtype=torch.bfloat16, device="cuda")
+    kv = torch.zeros(g.kv_shape, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(rt.RetopkError):
+        g.decode_step(q, kv, kv, 0)
+    with pytest.raises(rt.RetopkError):
+        g.decode_step(q, kv, kv, 257)
+    with pytest.raises(rt.RetopkError):
+        rt.ReTopK(1, 2, 1, 64, 4, 5, 8, 16, 0.9, 0, 256)     # r > M
