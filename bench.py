@@ -1,0 +1,435 @@
+#!/usr/bin/env python
+"""Benchmark of the ReTopK decode step: microseconds per decode step per layer.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config NAME] [--impl reference]
+
+One *step* is one ``retopk_decode_step`` call: the whole hot path (recall, candidate
+union, candidate or full-history scoring, Top-K, softmax.V, cache insert) for all
+``B * H_q`` heads of one attention layer.  Calls rotate over ``--layers`` independent
+layers (own KV cache, own query stream, own context) so that consecutive calls do not
+find their key rows in L2.  Inputs are seeded synthetic decode streams.
+
+The printed JSON line holds the stream-average time at the configured tau / R (``value``),
+the same metric through the host-buffer entry point (``e2e``), the library's own Exact
+Top-K on identical inputs, forced pure-reuse and pure-exact passes, the paper-default
+tau = 0.85 mix, the roofline of the dominant kernel and the oracle timed on the host cores.
+
+The path shards over (sequence, head) with no exchange, so ``--gpus N`` runs N independent
+replicas (one process per GPU) and reports the job-wide cost per step.
+"""
+from __future__ import annotations
+
+import argparse
+import ctypes as C
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2607_27692_b200 import workload as wl  # noqa: E402
+
+METRIC = "retopk_us_per_decode_step_per_layer"
+UNIT = "us"
+FALLBACK_HBM_GBS = 6650.0
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return float(p["hbm_gbs"]), "measured"
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+# --------------------------------------------------------------------------- clocks
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while a region runs (read only)."""
+
+    def __init__(self, index: int, period_s: float = 0.01):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        self.period = period_s
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.dev = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.dev, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self.nv = None
+
+    def _run(self):
+        nv = self.nv
+        names = {
+            getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8): "hw_slowdown",
+            getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4): "sw_power_cap",
+        }
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.dev, nv.NVML_CLOCK_SM)))
+                try:
+                    mask = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.dev))
+                except Exception:
+                    mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.dev))
+                for bit, name in names.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            self._stop.wait(self.period)
+
+    def __enter__(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0}
+        return {"sm_mhz": float(np.median(self.samples)), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+# --------------------------------------------------------------------------- GPU arm
+class Layers:
+    """Device-resident inputs and contexts of the rotating layers, plus raw-pointer calls."""
+
+    def __init__(self, cfg, n_layers, t_per_layer, rank, torch, rt):
+        self.cfg, self.n, self.T = cfg, n_layers, t_per_layer
+        self.torch, self.rt, self.lib = torch, rt, rt.load()
+        self.streams = [wl.make_stream(cfg, steps=t_per_layer, layer=l + 10 * rank) for l in range(n_layers)]
+        self.k = [rt.bf16_tensor_from_bits(s.k, device="cuda") for s in self.streams]
+        self.v = [rt.bf16_tensor_from_bits(s.v, device="cuda") for s in self.streams]
+        self.q = [rt.bf16_tensor_from_bits(s.q, device="cuda") for s in self.streams]
+        self.out = torch.empty((cfg.B, cfg.H_q, cfg.d), dtype=torch.bfloat16, device="cuda")
+        # pinned host copies of the per-step tensors for the end-to-end pass
+        self.q_host = [rt.bf16_tensor_from_bits(s.q, pin=True) for s in self.streams]
+        self.knew_host, self.vnew_host = [], []
+        for s in self.streams:
+            rows = slice(cfg.context, cfg.context + t_per_layer)
+            self.knew_host.append(rt.bf16_tensor_from_bits(
+                np.ascontiguousarray(s.k[:, :, rows].transpose(2, 0, 1, 3)), pin=True))
+            self.vnew_host.append(rt.bf16_tensor_from_bits(
+                np.ascontiguousarray(s.v[:, :, rows].transpose(2, 0, 1, 3)), pin=True))
+        self.out_host = torch.empty((cfg.B, cfg.H_q, cfg.d), dtype=torch.bfloat16).pin_memory()
+        self.ctx = []
+
+    def make_contexts(self, **override):
+        for c in self.ctx:
+            c.close()
+        self.ctx = [self.rt.ReTopK.from_config(self.cfg, **override) for _ in range(self.n)]
+
+    def stats(self):
+        tot = {}
+        for c in self.ctx:
+            for key, val in c.stats().items():
+                tot[key] = (tot.get(key, 0) | val) if key == "status" else tot.get(key, 0) + val
+        return tot
+
+    def call(self, i, kind, stream):
+        """Call number i of a pass: layer i % n at decode offset i // n."""
+        l, t = i % self.n, i // self.n
+        L = self.cfg.context + t + 1
+        h = self.ctx[l].h
+        qstep = self.cfg.B * self.cfg.H_q * self.cfg.d * 2
+        if kind == "retopk":
+            rc = self.lib.retopk_decode_step(h, self.q[l].data_ptr() + t * qstep, self.k[l].data_ptr(),
+                                             self.v[l].data_ptr(), L, self.out.data_ptr(), stream)
+        elif kind == "exact":
+            rc = self.lib.exact_topk_decode(h, self.q[l].data_ptr() + t * qstep, self.k[l].data_ptr(),
+                                            self.v[l].data_ptr(), L, self.out.data_ptr(), None, stream)
+        else:  # host buffers: h2d of q, k_t, v_t and d2h of the output inside the call
+            kvstep = self.cfg.B * self.cfg.H_kv * self.cfg.d * 2
+            rc = self.lib.retopk_decode_step_host(
+                h, self.q_host[l].data_ptr() + t * qstep, self.knew_host[l].data_ptr() + t * kvstep,
+                self.vnew_host[l].data_ptr() + t * kvstep, self.k[l].data_ptr(), self.v[l].data_ptr(), L,
+                self.out_host.data_ptr(), stream)
+        if rc != 0:
+            raise RuntimeError(f"{kind} call {i} failed with {rc}")
+
+
+def sync_all(torch, dist):
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+
+
+def timed_pass(layers, kind, warmup, steps, torch, dist, profile=False, sampler=None):
+    """Reset, run `warmup` untimed calls, then time exactly `steps` calls with CUDA events."""
+    stream = torch.cuda.current_stream().cuda_stream
+    for c in layers.ctx:
+        c.reset()
+    for i in range(warmup):
+        layers.call(i, kind, stream)
+    sync_all(torch, dist)
+    before = layers.stats()
+    if profile:
+        for c in layers.ctx:
+            c.profile_begin(steps // layers.n + 2)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    launches = 0
+    if sampler is not None:
+        sampler.__enter__()
+    sync_all(torch, dist)
+    e0.record()
+    for i in range(warmup, warmup + steps):
+        layers.call(i, kind, stream)
+    e1.record()
+    sync_all(torch, dist)
+    if sampler is not None:
+        sampler.__exit__(None, None, None)
+    ms = e0.elapsed_time(e1)
+    if dist is not None:
+        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    prof = None
+    if profile:
+        prof = {}
+        for c in layers.ctx:
+            for name, rec in c.profile_end().items():
+                agg = prof.setdefault(name, dict(ms=0.0, launches=0))
+                agg["ms"] += rec["ms"]
+                agg["launches"] += rec["launches"]
+    after = layers.stats()
+    delta = {key: (after[key] if key == "status" else after[key] - before[key]) for key in after}
+    launches = steps * (2 if kind == "exact" else 3)
+    return dict(ms=ms, us_per_step=1e3 * ms / steps, stats=delta, prof=prof, launches=launches)
+
+
+def algorithmic_bytes(cfg, stats, mean_L, mean_fill):
+    """Bytes the method has to move for the head-steps in `stats` (not score spills)."""
+    d, K = cfg.d, cfg.K
+    heads = stats["steps"]
+    n_sel = min(cfg.r, mean_fill)
+    tail = K * d * 2 + K * 4 + d * 2          # value rows, support insert, output
+    reuse = (heads * (mean_fill * d * 4 + d * 4 + d * 2) + stats["reuse"] * (n_sel * K * 4 + tail)
+             + stats["cand_sum"] * d * 2)
+    scan = stats["scan_groups"] * mean_L * d * 2
+    exact_finish = (heads - stats["reuse"]) * tail
+    return dict(reuse=reuse, scan=scan, exact_finish=exact_finish)
+
+
+def path_mix(stats):
+    n = max(stats["steps"], 1)
+    return {k: round(stats[k] / n, 4) for k in ("reuse", "fallback", "refresh")} | {
+        "mean_candidates": round(stats["cand_sum"] / max(stats["reuse"], 1), 1)}
+
+
+def cpu_baseline(cfg, stream, budget_s=12.0, max_steps=48):
+    """The fp64 oracle, as it stands, on the first decode steps of layer 0."""
+    from oracle import retopk_oracle
+    o = retopk_oracle.Oracle.from_config(cfg)
+    n, t0 = 0, time.perf_counter()
+    while n < min(max_steps, stream.q.shape[0]) and time.perf_counter() - t0 < budget_s:
+        o.decode_step(stream.q[n], stream.k, stream.v, stream.seq_len(n))
+        n += 1
+    el = time.perf_counter() - t0
+    s = o.stats()
+    return {"value": round(1e6 * el / n, 1), "unit": UNIT, "cores": retopk_oracle.num_threads(), "kind": "oracle",
+            "sample": f"first {n} decode steps of layer 0, all {cfg.B}x{cfg.H_q} heads, "
+                      f"{s['reuse']}/{s['fallback']}/{s['refresh']} reuse/fallback/refresh head-steps"}
+
+
+def run_gpu(args):
+    import torch
+    from paper_2607_27692_b200 import build, retopk as rt
+    build.build()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    cfg = wl.CONFIGS[args.config]
+    W, K = args.warmup, args.steps
+    n_layers = args.layers
+    t_per_layer = -(-(W + K) // n_layers)
+    if t_per_layer > cfg.steps:      # a longer run than the configuration's: extend the KV layout
+        cfg = cfg.replace(steps=t_per_layer)
+    layers = Layers(cfg, n_layers, t_per_layer, rank, torch, rt)
+    peak, peak_kind = measured_peaks()
+    mean_t = (W + K / 2) / n_layers
+    mean_L = cfg.context + mean_t + 1
+    mean_fill = min(cfg.M, mean_t)
+
+    # headline: configured tau / R, device-resident inputs
+    layers.make_contexts()
+    sampler = ClockSampler(local)
+    head = timed_pass(layers, "retopk", W, K, torch, dist, sampler=sampler)
+    # the same pass with per-kernel events (not the headline number)
+    prof = timed_pass(layers, "retopk", W, K, torch, dist, profile=True)
+    # end to end: host buffers in, host buffer out, every step
+    e2e = timed_pass(layers, "host", W, K, torch, dist)
+    # the library's own Exact Top-K on identical inputs
+    exact = timed_pass(layers, "exact", W, K, torch, dist)
+    # forced paths and the paper-default threshold
+    layers.make_contexts(tau=-2.0, R=0)
+    reuse = timed_pass(layers, "retopk", W, K, torch, dist)
+    layers.make_contexts(tau=2.0, R=0)
+    fallb = timed_pass(layers, "retopk", W, K, torch, dist)
+    layers.make_contexts(tau=0.85)
+    paper = timed_pass(layers, "retopk", W, K, torch, dist)
+
+    # roofline of the dominant kernel of the headline pass
+    abytes = algorithmic_bytes(cfg, prof["stats"], mean_L, mean_fill)
+    total_ms = sum(r["ms"] for r in prof["prof"].values())
+    kernels = {}
+    for name, rec in prof["prof"].items():
+        gbs = abytes[name] / (rec["ms"] * 1e-3) / 1e9 if rec["ms"] > 0 else 0.0
+        kernels[name] = {"launches": rec["launches"], "avg_us": round(1e3 * rec["ms"] / max(rec["launches"], 1), 2),
+                         "share": round(rec["ms"] / total_ms, 4),
+                         "alg_bytes_per_launch": int(abytes[name] / max(rec["launches"], 1)),
+                         "GBps": round(gbs, 1), "frac": round(gbs / peak, 4)}
+    top = max(kernels, key=lambda n: kernels[n]["share"])
+    roofline = {"bound": "hbm", "kernel": top + "_kernel", "achieved": kernels[top]["GBps"], "peak": peak,
+                "peak_kind": peak_kind, "unit": "GB/s", "frac": kernels[top]["frac"],
+                "frac_of_8TBps": round(kernels[top]["GBps"] / 8000.0, 4),
+                "traffic": NCU_TRAFFIC.get((args.config, top)), "kernels": kernels}
+
+    def path_report(res, exact_like):
+        st = res["stats"]
+        b = algorithmic_bytes(cfg, st, mean_L, mean_fill)
+        tot = sum(b.values())
+        gbs = tot / (res["ms"] * 1e-3) / 1e9
+        return {"us_per_step": round(res["us_per_step"], 2), "alg_bytes_per_step": int(tot / K),
+                "GBps": round(gbs, 1), "frac_of_measured": round(gbs / peak, 4),
+                "frac_of_8TBps": round(gbs / 8000.0, 4), "mix": path_mix(st)}
+
+    exact_bytes = (cfg.B * cfg.H_kv * mean_L * cfg.d * 2 + cfg.B * cfg.H_q * cfg.K * cfg.d * 2) * K
+    exact_gbs = exact_bytes / (exact["ms"] * 1e-3) / 1e9
+    qbytes = cfg.B * cfg.H_q * cfg.d * 2
+    kvbytes = 2 * cfg.B * cfg.H_kv * cfg.d * 2
+    line = {
+        "metric": METRIC, "value": round(head["us_per_step"] / world, 3), "unit": UNIT, "n_gpus": world,
+        "steps": K, "warmup": W, "ms_per_step": round(head["ms"] / K, 6), "higher_is_better": False,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": cfg.name, "B": cfg.B, "H_q": cfg.H_q, "H_kv": cfg.H_kv, "d": cfg.d,
+                   "context": cfg.context, "K": cfg.K, "M": cfg.M, "r": cfg.r, "W": cfg.W, "tau": cfg.tau,
+                   "R": cfg.R, "layers_rotated": n_layers, "decode_steps_per_layer": t_per_layer,
+                   "l2": "inputs larger than L2: calls rotate over independent layers",
+                   "parallelism": "replicas only" if world > 1 else "single GPU"},
+        "clocks": sampler.summary(),
+        "e2e": {"value": round(e2e["us_per_step"] / world, 3), "unit": UNIT,
+                "h2d_bytes_per_step": qbytes + kvbytes, "d2h_bytes_per_step": qbytes},
+        "gpu_launches": head["launches"],
+        "path_mix": path_mix(head["stats"]),
+        "exact_topk": {"us_per_step": round(exact["us_per_step"], 2), "GBps": round(exact_gbs, 1),
+                       "frac_of_measured": round(exact_gbs / peak, 4),
+                       "frac_of_8TBps": round(exact_gbs / 8000.0, 4)},
+        "speedup_vs_exact_topk": {"configured_tau": round(exact["us_per_step"] / head["us_per_step"], 3),
+                                  "tau_0.85": round(exact["us_per_step"] / paper["us_per_step"], 3),
+                                  "pure_reuse": round(exact["us_per_step"] / reuse["us_per_step"], 3)},
+        "paths": {"pure_reuse": path_report(reuse, False), "pure_exact": path_report(fallb, True),
+                  "tau_0.85": path_report(paper, False)},
+        "slow_select": head["stats"]["slow_select"],
+        "roofline": roofline,
+        "paper_context": "paper: 3.07x attention speedup over Exact Top-K at 128K, K=512 on one NVIDIA L20 "
+                         "(Qwen2.5-7B, PG19, tau=0.85); about 115 us per layer at 128K (Table 4 / 28 layers)",
+    }
+    if rank == 0:
+        if world == 1 and not args.no_cpu_baseline:
+            line["cpu_baseline"] = cpu_baseline(cfg, layers.streams[0])
+        print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+# Per-launch DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu
+# captures summarised under profiles/; filled in when a capture of that workload exists.
+NCU_TRAFFIC = {}
+
+
+# --------------------------------------------------------------------------- reference arm
+def run_reference(args):
+    """Time the fp64 oracle on the host cores: same metric, unit and configuration."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import retopk_oracle
+    cfg = wl.CONFIGS[args.config]
+    W, K = args.warmup, args.steps
+    if W + K > cfg.steps:
+        cfg = cfg.replace(steps=W + K)
+    # a bounded sample: one sequence of the batch (sequences are independent), scaled by B
+    sub = wl.make_stream(cfg, steps=W + K, sequences=range(0, 1))
+    o = retopk_oracle.Oracle.from_config(sub.cfg)
+    heads, scale = cfg.H_q, cfg.B
+    t_probe = time.perf_counter()
+    o.exact_topk(sub.q[0], sub.k, sub.v, sub.seq_len(0))
+    probe = time.perf_counter() - t_probe
+    note = f"one of {cfg.B} sequences per step ({heads} heads), time scaled by {scale}"
+    if probe * (W + K) > 240.0:
+        # one KV group of that sequence
+        G = cfg.G
+        sub = wl.Stream(sub.cfg.replace(H_q=G, H_kv=1), np.ascontiguousarray(sub.k[:, :1]),
+                        np.ascontiguousarray(sub.v[:, :1]), np.ascontiguousarray(sub.q[:, :, :G]))
+        o = retopk_oracle.Oracle.from_config(sub.cfg)
+        heads, scale = G, cfg.B * cfg.H_kv
+        note = f"one KV group ({G} heads) of one sequence per step, time scaled by {scale}"
+    for t in range(W):
+        o.decode_step(sub.q[t], sub.k, sub.v, sub.seq_len(t))
+    t0 = time.perf_counter()
+    for t in range(W, W + K):
+        o.decode_step(sub.q[t], sub.k, sub.v, sub.seq_len(t))
+    el = time.perf_counter() - t0
+    us = 1e6 * el / K * scale
+    cores = retopk_oracle.num_threads()
+    line = {
+        "impl": "reference", "metric": METRIC, "value": round(us, 1), "unit": UNIT,
+        "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": K, "warmup": W,
+        "ms_per_step": round(us / 1e3, 4), "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic",
+        "config": {"workload": cfg.name, "B": cfg.B, "H_q": cfg.H_q, "H_kv": cfg.H_kv, "d": cfg.d,
+                   "context": cfg.context, "K": cfg.K, "M": cfg.M, "r": cfg.r, "W": cfg.W, "tau": cfg.tau,
+                   "R": cfg.R},
+        "cpu_baseline": {"value": round(us, 1), "unit": UNIT, "cores": cores, "kind": "oracle", "sample": note},
+        "e2e": {"value": round(us, 1), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--config", default="headline128k", choices=sorted(wl.CONFIGS))
+    ap.add_argument("--layers", type=int, default=4, help="independent layers rotated over (L2 hygiene)")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        args.steps = 32 if args.steps is None else args.steps
+        args.warmup = 3 if args.warmup is None else args.warmup
+        run_reference(args)
+    else:
+        args.steps = 1024 if args.steps is None else args.steps
+        args.warmup = 64 if args.warmup is None else args.warmup
+        run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()

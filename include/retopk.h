@@ -67,6 +67,7 @@ typedef struct {
     int64_t refresh;     /* scheduled refresh (counted as refresh even if rho_max < tau) */
     int64_t cand_sum;    /* sum of candidate-set sizes |A_t| over reuse head-steps (Eq. 9) */
     int64_t slow_select; /* exact-path selections that needed the multi-pass fallback */
+    int64_t scan_groups; /* (sequence, KV head) groups whose keys were scanned in full, summed over steps */
     uint32_t status;     /* RETOPK_STATUS_* bits */
     uint32_t reserved;
 } retopk_stats_t;
@@ -149,6 +150,17 @@ int retopk_export_state(retopk_ctx* ctx, float* qbar, int32_t* supports, int64_t
                         int64_t* t_dec, void* stream);
 int retopk_import_state(retopk_ctx* ctx, const float* qbar, const int32_t* supports,
                         int64_t n_inserted, int64_t t_dec, void* stream);
+
+/*
+ * Measurement hooks (no counterpart in the paper).  Between begin and end, every decode
+ * call of this context brackets each of its kernels with CUDA events on the call's stream
+ * (up to max_calls calls; later calls run unrecorded).  retopk_profile_end synchronises
+ * the device and returns, per kernel slot {0: reuse, 1: scan, 2: exact finish}, the summed
+ * device time in milliseconds and the number of launches.  Not for use inside a timed
+ * region: the events themselves cost a little.
+ */
+int retopk_profile_begin(retopk_ctx* ctx, int max_calls);
+int retopk_profile_end(retopk_ctx* ctx, double ms_host[3], int64_t launches_host[3]);
 
 /* Number of kernels the last decode call of this context launched (host-side count). */
 int retopk_last_launch_count(const retopk_ctx* ctx);

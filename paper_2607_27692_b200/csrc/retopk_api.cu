@@ -17,19 +17,25 @@ struct retopk_ctx {
     long long max_seq_len, score_stride;
     long long n_ins, t_dec;
     int NS;
-    int num_sms;
-    size_t smem_recall, smem_finish;
+    int num_sms, scan_grid;
+    int call_serial;
+    size_t smem_reuse, smem_exact;
     // device state
     float* qbar_cache;
     int32_t* sup_cache;
     uint8_t* ws_path;
     float* ws_rho;
     int32_t* ws_ncand;
-    int32_t* ws_cand;
+    int32_t* ws_gflag;
     float* ws_scores;
     long long* counters;
     unsigned int* status;
     unsigned long long* slow_select;
+    unsigned long long* scan_groups;
+    // per-kernel event timing (measurement hook)
+    cudaEvent_t* prof_events;
+    int prof_max, prof_calls;
+    unsigned char* prof_kind;   // per call: 0 = retopk step, 1 = exact_topk_decode
     // staging for the host-buffer entry point
     uint16_t* stage_q;
     uint16_t* stage_out;
@@ -58,8 +64,8 @@ bool dev_alloc(T** p, size_t count) {
 
 void free_all(retopk_ctx* c) {
     cudaFree(c->qbar_cache); cudaFree(c->sup_cache); cudaFree(c->ws_path); cudaFree(c->ws_rho);
-    cudaFree(c->ws_ncand); cudaFree(c->ws_cand); cudaFree(c->ws_scores); cudaFree(c->counters);
-    cudaFree(c->status); cudaFree(c->slow_select); cudaFree(c->stage_q); cudaFree(c->stage_out);
+    cudaFree(c->ws_ncand); cudaFree(c->ws_gflag); cudaFree(c->ws_scores); cudaFree(c->counters);
+    cudaFree(c->status); cudaFree(c->slow_select); cudaFree(c->scan_groups); cudaFree(c->stage_q); cudaFree(c->stage_out);
     cudaFree(c->stage_kv);
 }
 
@@ -78,26 +84,31 @@ StepArgs make_args(const retopk_ctx* c, const void* q, const void* k, const void
     a.refresh = (c->R > 0 && c->t_dec > 0 && c->t_dec % c->R == 0) ? 1 : 0;
     a.mode = mode;
     a.NS = c->NS;
-    // scan grid: enough CTAs to fill the machine several times over, in whole 128-row blocks
-    long long rows = (L * c->B * c->Hkv + (long long)c->num_sms * 8 - 1) / ((long long)c->num_sms * 8);
-    rows = (rows + 127) / 128 * 128;
-    if (rows < 128) rows = 128;
-    if (rows > 1024) rows = 1024;
-    a.rows_per_cta = (int)rows;
+    a.step_id = c->call_serial;
     a.q = static_cast<const uint16_t*>(q);
     a.k = static_cast<const uint16_t*>(k);
     a.v = static_cast<const uint16_t*>(v);
     a.out = static_cast<uint16_t*>(out);
     a.qbar_cache = c->qbar_cache; a.sup_cache = c->sup_cache;
-    a.ws_path = c->ws_path; a.ws_rho = c->ws_rho; a.ws_ncand = c->ws_ncand; a.ws_cand = c->ws_cand;
+    a.ws_path = c->ws_path; a.ws_rho = c->ws_rho; a.ws_ncand = c->ws_ncand; a.ws_gflag = c->ws_gflag;
     a.ws_scores = c->ws_scores; a.counters = c->counters; a.status = c->status;
     a.slow_select = c->slow_select;
+    a.scan_groups = c->scan_groups;
     a.idx_out = nullptr;
     return a;
 }
 
+int launch_reuse(const retopk_ctx* c, const StepArgs& a, cudaStream_t s) {
+    const unsigned grid = (unsigned)(c->B * c->Hq);
+    if (c->d == 128) reuse_kernel<128><<<grid, REUSE_THREADS, c->smem_reuse, s>>>(a);
+    else reuse_kernel<64><<<grid, REUSE_THREADS, c->smem_reuse, s>>>(a);
+    return cudaGetLastError() == cudaSuccess ? RETOPK_OK : RETOPK_ECUDA;
+}
+
 int launch_scan(const retopk_ctx* c, const StepArgs& a, cudaStream_t s) {
-    dim3 grid((unsigned)((a.L + a.rows_per_cta - 1) / a.rows_per_cta), (unsigned)(c->B * c->Hkv));
+    // persistent CTAs; no more of them than there are 256-row work items
+    const long long items = (long long)c->B * c->Hkv * ((a.L + SCAN_TILE_ROWS - 1) / SCAN_TILE_ROWS);
+    const unsigned grid = (unsigned)(items < c->scan_grid ? items : c->scan_grid);
     const int ntile = (c->G + 7) / 8;
     if (c->d == 128 && ntile == 1) scan_kernel<128, 1><<<grid, SCAN_THREADS, 0, s>>>(a);
     else if (c->d == 128) scan_kernel<128, 2><<<grid, SCAN_THREADS, 0, s>>>(a);
@@ -106,11 +117,20 @@ int launch_scan(const retopk_ctx* c, const StepArgs& a, cudaStream_t s) {
     return cudaGetLastError() == cudaSuccess ? RETOPK_OK : RETOPK_ECUDA;
 }
 
-int launch_finish(const retopk_ctx* c, const StepArgs& a, cudaStream_t s) {
+int launch_exact_finish(const retopk_ctx* c, const StepArgs& a, cudaStream_t s) {
     const unsigned grid = (unsigned)(c->B * c->Hq);
-    if (c->d == 128) finish_kernel<128><<<grid, FINISH_THREADS, c->smem_finish, s>>>(a);
-    else finish_kernel<64><<<grid, FINISH_THREADS, c->smem_finish, s>>>(a);
+    if (c->d == 128) exact_finish_kernel<128><<<grid, EXACT_THREADS, c->smem_exact, s>>>(a);
+    else exact_finish_kernel<64><<<grid, EXACT_THREADS, c->smem_exact, s>>>(a);
     return cudaGetLastError() == cudaSuccess ? RETOPK_OK : RETOPK_ECUDA;
+}
+
+// Measurement hook: event number `which` (0..3) of the current call, if recording.
+void prof_mark(retopk_ctx* c, int which, cudaStream_t s) {
+    if (c->prof_events && c->prof_calls < c->prof_max)
+        cudaEventRecord(c->prof_events[(size_t)c->prof_calls * 4 + which], s);
+}
+void prof_done(retopk_ctx* c, int kind) {
+    if (c->prof_events && c->prof_calls < c->prof_max) c->prof_kind[c->prof_calls++] = (unsigned char)kind;
 }
 
 int check_step_args(const retopk_ctx* c, const void* q, const void* k, const void* v, long long L,
@@ -133,7 +153,7 @@ int retopk_create_batched(retopk_ctx** out, int B, int H_q, int H_kv, int d, int
         R < 0 || max_seq_len < 1 || d < 1)
         return RETOPK_EINVAL;
     if ((d != 64 && d != 128) || H_q / H_kv > 16 || M > 1024 || K > 4096 || max_seq_len > 1048576 ||
-        (long long)B * H_kv > 65535)
+        (long long)B * H_kv > MAX_GROUPS)
         return RETOPK_EUNSUPPORTED;
     if (tau != tau) return RETOPK_EINVAL;
     retopk_ctx* c = new (std::nothrow) retopk_ctx;
@@ -144,33 +164,48 @@ int retopk_create_batched(retopk_ctx** out, int B, int H_q, int H_kv, int d, int
     c->K = K; c->R = R; c->tau = tau; c->max_seq_len = max_seq_len;
     c->cap = r * K + W;
     c->score_stride = (max_seq_len + 3) / 4 * 4;
-    c->NS = c->cap > NS_MIN ? c->cap : NS_MIN;
+    c->NS = K <= 1024 ? 8192 : 16384;
     int sms = 0;
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, c->device);
     c->num_sms = sms > 0 ? sms : 148;
 
-    const size_t head_words = (size_t)d + M + r + 8 + 4;
-    c->smem_recall = (((head_words + 3) & ~(size_t)3) + (size_t)(max_seq_len + 31) / 32) * 4;
-    c->smem_finish = ((size_t)c->NS * 2 + (size_t)K * 3 + SAMPLE_BINS + 32 + 8) * 4;
+    // shared-memory footprints (must mirror the carve-up at the top of each kernel)
+    const size_t red_words = (size_t)(REUSE_THREADS / 32) * d + REUSE_THREADS;
+    const size_t head_words = ((size_t)d + M + r + 32 + 8 + 256 + 3 * (size_t)K + 3) & ~(size_t)3;
+    const size_t big_words = (((size_t)2 * c->cap > red_words ? (size_t)2 * c->cap : red_words) + 3) & ~(size_t)3;
+    const size_t bm_words = (((size_t)max_seq_len + 31) / 32 + 3) & ~(size_t)3;
+    c->smem_reuse = (head_words + big_words + bm_words) * 4;
+    c->smem_exact = ((size_t)c->NS * 2 + (size_t)K * 3 + SAMPLE_BINS + 32 + 8 + 2 * (EXACT_THREADS / 32)) * 4;
     int max_smem = 0;
     cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, c->device);
-    if ((size_t)max_smem < c->smem_recall || (size_t)max_smem < c->smem_finish) {
+    if ((size_t)max_smem < c->smem_reuse || (size_t)max_smem < c->smem_exact) {
         delete c;
         return RETOPK_EUNSUPPORTED;
     }
     // opt in to the device maximum once; contexts of different sizes then coexist
-    cudaError_t e1 = cudaFuncSetAttribute(recall_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
-    cudaError_t e2 = (d == 128)
-        ? cudaFuncSetAttribute(finish_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem)
-        : cudaFuncSetAttribute(finish_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
+    cudaError_t e1, e2;
+    int occ = 0;
+    const int ntile = (c->G + 7) / 8;
+    if (d == 128) {
+        e1 = cudaFuncSetAttribute(reuse_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
+        e2 = cudaFuncSetAttribute(exact_finish_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
+        if (ntile == 1) cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, scan_kernel<128, 1>, SCAN_THREADS, 0);
+        else cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, scan_kernel<128, 2>, SCAN_THREADS, 0);
+    } else {
+        e1 = cudaFuncSetAttribute(reuse_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
+        e2 = cudaFuncSetAttribute(exact_finish_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
+        if (ntile == 1) cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, scan_kernel<64, 1>, SCAN_THREADS, 0);
+        else cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, scan_kernel<64, 2>, SCAN_THREADS, 0);
+    }
     if (e1 != cudaSuccess || e2 != cudaSuccess) { cudaGetLastError(); delete c; return RETOPK_ECUDA; }
+    c->scan_grid = c->num_sms * (occ > 0 ? occ : 2);
 
     const size_t nh = (size_t)B * H_q;
     bool ok = dev_alloc(&c->qbar_cache, nh * M * d) && dev_alloc(&c->sup_cache, nh * M * K) &&
               dev_alloc(&c->ws_path, nh) && dev_alloc(&c->ws_rho, nh) && dev_alloc(&c->ws_ncand, nh) &&
-              dev_alloc(&c->ws_cand, nh * c->cap) && dev_alloc(&c->ws_scores, nh * (size_t)c->score_stride) &&
+              dev_alloc(&c->ws_gflag, (size_t)B * H_kv) && dev_alloc(&c->ws_scores, nh * (size_t)c->score_stride) &&
               dev_alloc(&c->counters, nh * 4) && dev_alloc(&c->status, 1) &&
-              dev_alloc(&c->slow_select, 1) && dev_alloc(&c->stage_q, nh * d) &&
+              dev_alloc(&c->slow_select, 1) && dev_alloc(&c->scan_groups, 1) && dev_alloc(&c->stage_q, nh * d) &&
               dev_alloc(&c->stage_out, nh * d) && dev_alloc(&c->stage_kv, (size_t)2 * B * H_kv * d);
     if (!ok) { cudaGetLastError(); free_all(c); delete c; return RETOPK_ENOMEM; }
     *out = c;
@@ -198,8 +233,8 @@ int retopk_reset(retopk_ctx* c, void* stream) {
     if (!c) return RETOPK_EINVAL;
     const size_t nh = (size_t)c->B * c->Hq;
     reset_kernel<<<c->num_sms * 4, 256, 0, static_cast<cudaStream_t>(stream)>>>(
-        c->qbar_cache, nh * c->M * c->d, c->sup_cache, nh * c->M * c->K, c->counters, nh * 4, c->status,
-        c->slow_select);
+        c->qbar_cache, nh * c->M * c->d, c->sup_cache, nh * c->M * c->K, c->counters, nh * 4, c->ws_gflag,
+        (size_t)c->B * c->Hkv, c->status, c->slow_select, c->scan_groups);
     c->n_ins = 0;
     c->t_dec = 0;
     return cudaGetLastError() == cudaSuccess ? RETOPK_OK : RETOPK_ECUDA;
@@ -211,10 +246,16 @@ int retopk_decode_step(retopk_ctx* c, const void* q, const void* k_cache, const 
     if (rc != RETOPK_OK) return rc;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     StepArgs a = make_args(c, q, k_cache, v_cache, seq_len, out, MODE_RETOPK);
-    recall_kernel<<<(unsigned)(c->B * c->Hq), RECALL_THREADS, c->smem_recall, s>>>(a);
-    if (cudaGetLastError() != cudaSuccess) return RETOPK_ECUDA;
+    c->call_serial = (c->call_serial + 1) & 0x3fffffff;
+    a.step_id = c->call_serial;
+    prof_mark(c, 0, s);
+    if ((rc = launch_reuse(c, a, s)) != RETOPK_OK) return rc;
+    prof_mark(c, 1, s);
     if ((rc = launch_scan(c, a, s)) != RETOPK_OK) return rc;
-    if ((rc = launch_finish(c, a, s)) != RETOPK_OK) return rc;
+    prof_mark(c, 2, s);
+    if ((rc = launch_exact_finish(c, a, s)) != RETOPK_OK) return rc;
+    prof_mark(c, 3, s);
+    prof_done(c, 0);
     c->last_launches = 3;
     c->n_ins += 1;
     c->t_dec += 1;
@@ -228,8 +269,13 @@ int exact_topk_decode(retopk_ctx* c, const void* q, const void* k_cache, const v
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     StepArgs a = make_args(c, q, k_cache, v_cache, seq_len, out, MODE_EXACT);
     a.idx_out = idx_out;
+    prof_mark(c, 0, s);
+    prof_mark(c, 1, s);
     if ((rc = launch_scan(c, a, s)) != RETOPK_OK) return rc;
-    if ((rc = launch_finish(c, a, s)) != RETOPK_OK) return rc;
+    prof_mark(c, 2, s);
+    if ((rc = launch_exact_finish(c, a, s)) != RETOPK_OK) return rc;
+    prof_mark(c, 3, s);
+    prof_done(c, 1);
     c->last_launches = 2;
     return RETOPK_OK;
 }
@@ -266,8 +312,9 @@ int retopk_stats(retopk_ctx* c, retopk_stats_t* st) {
     long long* host = new (std::nothrow) long long[nh * 4];
     if (!host) return RETOPK_ENOMEM;
     unsigned int status = 0;
-    unsigned long long slow = 0;
+    unsigned long long slow = 0, groups = 0;
     bool ok = cudaDeviceSynchronize() == cudaSuccess &&
+              cudaMemcpy(&groups, c->scan_groups, sizeof groups, cudaMemcpyDeviceToHost) == cudaSuccess &&
               cudaMemcpy(host, c->counters, nh * 4 * sizeof(long long), cudaMemcpyDeviceToHost) == cudaSuccess &&
               cudaMemcpy(&status, c->status, sizeof status, cudaMemcpyDeviceToHost) == cudaSuccess &&
               cudaMemcpy(&slow, c->slow_select, sizeof slow, cudaMemcpyDeviceToHost) == cudaSuccess;
@@ -281,6 +328,7 @@ int retopk_stats(retopk_ctx* c, retopk_stats_t* st) {
         }
         st->steps = st->reuse + st->fallback + st->refresh;
         st->slow_select = (int64_t)slow;
+        st->scan_groups = (int64_t)groups;
         st->status = status;
     }
     delete[] host;
@@ -328,6 +376,42 @@ int retopk_import_state(retopk_ctx* c, const float* qbar, const int32_t* support
               cudaMemcpyAsync(c->sup_cache, supports, nh * c->M * c->K * 4, cudaMemcpyDeviceToDevice, s) == cudaSuccess;
     c->n_ins = n_inserted;
     c->t_dec = t_dec;
+    return ok ? RETOPK_OK : RETOPK_ECUDA;
+}
+
+int retopk_profile_begin(retopk_ctx* c, int max_calls) {
+    if (!c || max_calls < 1 || c->prof_events) return RETOPK_EINVAL;
+    DeviceGuard g(c->device);
+    c->prof_events = new (std::nothrow) cudaEvent_t[(size_t)max_calls * 4];
+    c->prof_kind = new (std::nothrow) unsigned char[max_calls];
+    if (!c->prof_events || !c->prof_kind) return RETOPK_ENOMEM;
+    for (int i = 0; i < max_calls * 4; ++i)
+        if (cudaEventCreate(&c->prof_events[i]) != cudaSuccess) return RETOPK_ECUDA;
+    c->prof_max = max_calls;
+    c->prof_calls = 0;
+    return RETOPK_OK;
+}
+
+int retopk_profile_end(retopk_ctx* c, double ms_host[3], int64_t launches_host[3]) {
+    if (!c || !c->prof_events || !ms_host || !launches_host) return RETOPK_EINVAL;
+    DeviceGuard g(c->device);
+    bool ok = cudaDeviceSynchronize() == cudaSuccess;
+    for (int j = 0; j < 3; ++j) { ms_host[j] = 0.0; launches_host[j] = 0; }
+    for (int i = 0; ok && i < c->prof_calls; ++i) {
+        cudaEvent_t* e = c->prof_events + (size_t)i * 4;
+        for (int j = (c->prof_kind[i] == 1 ? 1 : 0); j < 3; ++j) {
+            float ms = 0.f;
+            ok = ok && cudaEventElapsedTime(&ms, e[j], e[j + 1]) == cudaSuccess;
+            ms_host[j] += ms;
+            launches_host[j] += 1;
+        }
+    }
+    for (int i = 0; i < c->prof_max * 4; ++i) cudaEventDestroy(c->prof_events[i]);
+    delete[] c->prof_events;
+    delete[] c->prof_kind;
+    c->prof_events = nullptr;
+    c->prof_kind = nullptr;
+    c->prof_max = c->prof_calls = 0;
     return ok ? RETOPK_OK : RETOPK_ECUDA;
 }
 

@@ -25,7 +25,7 @@ class RetopkError(RuntimeError):
 
 class _Stats(C.Structure):
     _fields_ = [("steps", C.c_int64), ("reuse", C.c_int64), ("fallback", C.c_int64),
-                ("refresh", C.c_int64), ("cand_sum", C.c_int64), ("slow_select", C.c_int64),
+                ("refresh", C.c_int64), ("cand_sum", C.c_int64), ("slow_select", C.c_int64), ("scan_groups", C.c_int64),
                 ("status", C.c_uint32), ("reserved", C.c_uint32)]
 
 
@@ -45,6 +45,8 @@ SIGNATURES = {
     "retopk_last_step": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp]),
     "retopk_export_state": (_i32, [_vp, _vp, _vp, C.POINTER(_i64), C.POINTER(_i64), _vp]),
     "retopk_import_state": (_i32, [_vp, _vp, _vp, _i64, _i64, _vp]),
+    "retopk_profile_begin": (_i32, [_vp, _i32]),
+    "retopk_profile_end": (_i32, [_vp, C.POINTER(C.c_double), C.POINTER(_i64)]),
     "retopk_last_launch_count": (_i32, [_vp]),
     "retopk_strerror": (C.c_char_p, [_i32]),
 }
@@ -202,6 +204,15 @@ class ReTopK:
             self.h, _dev(qbar, torch.float32, (self.B, self.H_q, self.M, self.d)),
             _dev(supports, torch.int32, (self.B, self.H_q, self.M, self.K)), n_inserted, t_dec, _stream())
         _check(rc, "retopk_import_state")
+
+    def profile_begin(self, max_calls: int):
+        _check(self.lib.retopk_profile_begin(self.h, max_calls), "retopk_profile_begin")
+
+    def profile_end(self) -> dict:
+        ms, n = (C.c_double * 3)(), (_i64 * 3)()
+        _check(self.lib.retopk_profile_end(self.h, ms, n), "retopk_profile_end")
+        return {name: dict(ms=float(ms[i]), launches=int(n[i]))
+                for i, name in enumerate(("reuse", "scan", "exact_finish"))}
 
     def last_launch_count(self) -> int:
         return int(self.lib.retopk_last_launch_count(self.h))
