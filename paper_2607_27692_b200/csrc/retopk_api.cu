@@ -14,9 +14,9 @@ struct retopk_ctx {
     int device;
     int B, Hq, Hkv, G, d, M, r, W, K, R, cap;
     float tau;
-    long long max_seq_len, score_stride;
+    long long max_seq_len, score_stride, tmax_stride;
     long long n_ins, t_dec;
-    int NS;
+    int NS, stage_depth, exact_stage_depth;
     int num_sms, scan_grid;
     int call_serial;
     size_t smem_reuse, smem_exact;
@@ -28,6 +28,7 @@ struct retopk_ctx {
     int32_t* ws_ncand;
     int32_t* ws_gflag;
     float* ws_scores;
+    float* ws_tmax;
     long long* counters;
     unsigned int* status;
     unsigned long long* slow_select;
@@ -64,7 +65,7 @@ bool dev_alloc(T** p, size_t count) {
 
 void free_all(retopk_ctx* c) {
     cudaFree(c->qbar_cache); cudaFree(c->sup_cache); cudaFree(c->ws_path); cudaFree(c->ws_rho);
-    cudaFree(c->ws_ncand); cudaFree(c->ws_gflag); cudaFree(c->ws_scores); cudaFree(c->counters);
+    cudaFree(c->ws_ncand); cudaFree(c->ws_gflag); cudaFree(c->ws_scores); cudaFree(c->ws_tmax); cudaFree(c->counters);
     cudaFree(c->status); cudaFree(c->slow_select); cudaFree(c->scan_groups); cudaFree(c->stage_q); cudaFree(c->stage_out);
     cudaFree(c->stage_kv);
 }
@@ -85,13 +86,15 @@ StepArgs make_args(const retopk_ctx* c, const void* q, const void* k, const void
     a.mode = mode;
     a.NS = c->NS;
     a.step_id = c->call_serial;
+    a.stage_depth = c->stage_depth;
+    a.exact_stage_depth = c->exact_stage_depth;
     a.q = static_cast<const uint16_t*>(q);
     a.k = static_cast<const uint16_t*>(k);
     a.v = static_cast<const uint16_t*>(v);
     a.out = static_cast<uint16_t*>(out);
     a.qbar_cache = c->qbar_cache; a.sup_cache = c->sup_cache;
     a.ws_path = c->ws_path; a.ws_rho = c->ws_rho; a.ws_ncand = c->ws_ncand; a.ws_gflag = c->ws_gflag;
-    a.ws_scores = c->ws_scores; a.counters = c->counters; a.status = c->status;
+    a.ws_scores = c->ws_scores; a.ws_tmax = c->ws_tmax; a.tmax_stride = c->tmax_stride; a.counters = c->counters; a.status = c->status;
     a.slow_select = c->slow_select;
     a.scan_groups = c->scan_groups;
     a.idx_out = nullptr;
@@ -163,8 +166,9 @@ int retopk_create_batched(retopk_ctx** out, int B, int H_q, int H_kv, int d, int
     c->B = B; c->Hq = H_q; c->Hkv = H_kv; c->G = H_q / H_kv; c->d = d; c->M = M; c->r = r; c->W = W;
     c->K = K; c->R = R; c->tau = tau; c->max_seq_len = max_seq_len;
     c->cap = r * K + W;
-    c->score_stride = (max_seq_len + 3) / 4 * 4;
-    c->NS = K <= 1024 ? 8192 : 16384;
+    c->score_stride = (max_seq_len + TILE_ROWS - 1) / TILE_ROWS * TILE_ROWS;   // whole 16-row tiles
+    c->tmax_stride = ((max_seq_len + TILE_ROWS - 1) / TILE_ROWS + 3) / 4 * 4;
+    c->NS = 16 * K <= 8192 ? 8192 : 16384;
     int sms = 0;
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, c->device);
     c->num_sms = sms > 0 ? sms : 148;
@@ -175,13 +179,31 @@ int retopk_create_batched(retopk_ctx** out, int B, int H_q, int H_kv, int d, int
     const size_t big_words = (((size_t)2 * c->cap > red_words ? (size_t)2 * c->cap : red_words) + 3) & ~(size_t)3;
     const size_t bm_words = (((size_t)max_seq_len + 31) / 32 + 3) & ~(size_t)3;
     c->smem_reuse = (head_words + big_words + bm_words) * 4;
-    c->smem_exact = ((size_t)c->NS * 2 + (size_t)K * 3 + SAMPLE_BINS + 32 + 8 + 2 * (EXACT_THREADS / 32)) * 4;
+    c->smem_exact = (((size_t)c->NS * 2 + (size_t)c->NS / 2 + (size_t)K * 3 + 256 + 32 + 8 + 3) & ~(size_t)3) * 4;
     int max_smem = 0;
     cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, c->device);
-    if ((size_t)max_smem < c->smem_reuse || (size_t)max_smem < c->smem_exact) {
+    // the rest of shared memory is the landing zone of the asynchronous row copies:
+    // 16 KB (one 16-byte piece per thread) per row kept in flight per row slot
+    const size_t wave = (size_t)REUSE_THREADS * 16;
+    if ((size_t)max_smem < c->smem_reuse + wave || (size_t)max_smem < c->smem_exact + wave) {
         delete c;
         return RETOPK_EUNSUPPORTED;
     }
+    const int slots = REUSE_THREADS / (d / 8);
+    auto depth_for = [&](size_t fixed, int rows) {
+        long long fit = (long long)(((size_t)max_smem - fixed) / wave);
+        long long want = (rows + slots - 1) / slots;          // one wave covers `rows` rows
+        long long dep = fit < want ? fit : want;
+        return (int)(dep < 1 ? 1 : (dep > 16 ? 16 : dep));
+    };
+    c->stage_depth = depth_for(c->smem_reuse, K + K / 4 > c->cap ? c->cap : K + K / 4);
+    c->exact_stage_depth = depth_for(c->smem_exact, K);
+    if (c->stage_depth * slots < K) {            // the value rows use the same zone
+        int dv = depth_for(c->smem_reuse, K);
+        if (dv > c->stage_depth) c->stage_depth = dv;
+    }
+    c->smem_reuse += (size_t)c->stage_depth * wave;
+    c->smem_exact += (size_t)c->exact_stage_depth * wave;
     // opt in to the device maximum once; contexts of different sizes then coexist
     cudaError_t e1, e2;
     int occ = 0;
@@ -204,6 +226,7 @@ int retopk_create_batched(retopk_ctx** out, int B, int H_q, int H_kv, int d, int
     bool ok = dev_alloc(&c->qbar_cache, nh * M * d) && dev_alloc(&c->sup_cache, nh * M * K) &&
               dev_alloc(&c->ws_path, nh) && dev_alloc(&c->ws_rho, nh) && dev_alloc(&c->ws_ncand, nh) &&
               dev_alloc(&c->ws_gflag, (size_t)B * H_kv) && dev_alloc(&c->ws_scores, nh * (size_t)c->score_stride) &&
+              dev_alloc(&c->ws_tmax, nh * (size_t)c->tmax_stride) &&
               dev_alloc(&c->counters, nh * 4) && dev_alloc(&c->status, 1) &&
               dev_alloc(&c->slow_select, 1) && dev_alloc(&c->scan_groups, 1) && dev_alloc(&c->stage_q, nh * d) &&
               dev_alloc(&c->stage_out, nh * d) && dev_alloc(&c->stage_kv, (size_t)2 * B * H_kv * d);
@@ -416,6 +439,14 @@ int retopk_profile_end(retopk_ctx* c, double ms_host[3], int64_t launches_host[3
 }
 
 int retopk_last_launch_count(const retopk_ctx* c) { return c ? c->last_launches : 0; }
+
+#ifdef RETOPK_PHASE_CLOCKS
+// Development aid (not part of the public interface): copy the phase clock table to the host.
+int retopk_debug_read_phases(long long* host) {
+    cudaDeviceSynchronize();
+    return cudaMemcpyFromSymbol(host, g_phase_clk, sizeof(long long) * 3 * 1024 * 16) == cudaSuccess ? 0 : -4;
+}
+#endif
 
 const char* retopk_strerror(int code) {
     switch (code) {

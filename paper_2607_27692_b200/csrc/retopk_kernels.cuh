@@ -12,13 +12,26 @@
 //                  e_i = q.k_i/sqrt(d) (Eq. 4); every key row streams once through the
 //                  tensor cores for all G query heads of its group.
 //   exact_finish_kernel  one CTA per exact-path head: global Top-K (Eq. 1) of the scanned
-//                  scores by threshold collection + radix select, softmax.V (Eq. 12),
-//                  support insert.  Exact Top-K attention is scan + this kernel.
+//                  scores (tile maxima give a lower bound for the K-th score, only the
+//                  tiles that reach it are read back), softmax.V (Eq. 12), support insert.
+//                  Exact Top-K attention is scan + this kernel.
 #pragma once
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <math_constants.h>
 #include <stdint.h>
+
+// Development aid: with -DRETOPK_PHASE_CLOCKS thread 0 of every CTA stamps the SM clock at
+// phase boundaries into a global table (read back through retopk_debug_read_phases).
+#ifdef RETOPK_PHASE_CLOCKS
+__device__ long long g_phase_clk[3][1024][16];
+#define RETOPK_PHASE(kernel, n)                                                            \
+    do {                                                                                   \
+        if (threadIdx.x == 0 && blockIdx.x < 1024) g_phase_clk[kernel][blockIdx.x][n] = clock64(); \
+    } while (0)
+#else
+#define RETOPK_PHASE(kernel, n) do { } while (0)
+#endif
 
 namespace retopk {
 
@@ -30,8 +43,7 @@ constexpr int EXACT_THREADS = 1024;
 constexpr int SCAN_THREADS = 256;
 constexpr int SCAN_TILE_ROWS = 256;  // key rows per scan work item
 constexpr int MAX_GROUPS = 4096;     // B * H_kv limit (shared list in scan_kernel)
-constexpr int SAMPLE_MAX = 8192;     // scores sampled to place the collection threshold
-constexpr int SAMPLE_BINS = 2048;    // histogram over the top 11 bits of the score key
+constexpr int TILE_ROWS = 16;        // rows per score tile whose maximum the scan records
 
 struct StepArgs {
     int B, Hq, Hkv, G, d, M, r, W, K, cap;
@@ -45,6 +57,8 @@ struct StepArgs {
     int mode;                // MODE_RETOPK or MODE_EXACT
     int NS;                  // entries in exact_finish_kernel's shared collection lists
     int step_id;             // call serial number; a KV group is flagged by storing it
+    int stage_depth;         // rows in flight per row slot in reuse_kernel's landing zone
+    int exact_stage_depth;   // same for exact_finish_kernel
     const uint16_t* q;
     const uint16_t* k;
     const uint16_t* v;
@@ -56,6 +70,8 @@ struct StepArgs {
     int32_t* ws_ncand;       // [B*Hq]
     int32_t* ws_gflag;       // [B*Hkv] == step_id when the group needs a full scan
     float* ws_scores;        // [B*Hq][score_stride]
+    float* ws_tmax;          // [B*Hq][tmax_stride] largest score of every 16-row key tile
+    long long tmax_stride;   // multiple of 4
     long long* counters;     // [B*Hq][4] reuse, fallback, refresh, cand_sum
     unsigned int* status;
     unsigned long long* slow_select;
@@ -85,6 +101,14 @@ __device__ __forceinline__ uint4 ldg_stream(const void* p) {
                  : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p));
     return r;
 }
+
+// 16-byte asynchronous global -> shared copy (L2 only), and its completion wait.
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
+    const unsigned dst = (unsigned)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" :: "r"(dst), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
 
 __device__ __forceinline__ float dot8(const uint4& x, const float* qf) {
     float a = bf16_lo(x.x) * qf[0];
@@ -156,9 +180,13 @@ __device__ void radix_select(const Src& src, int n, int K, uint32_t* s_hist, int
     for (int shift = 24; shift >= 0; shift -= 8) {
         for (int i = tid; i < 256; i += NT) s_hist[i] = 0;
         __syncthreads();
-        for (int i = tid; i < n; i += NT) {
-            const uint32_t key = src.k(i);
-            if ((key & mask) == prefix) atomicAdd(&s_hist[(key >> shift) & 255u], 1u);
+        for (int base = 0; base < n; base += NT) {
+            const int i = base + tid;
+            const uint32_t key = i < n ? src.k(i) : 0u;
+            const bool in = i < n && (key & mask) == prefix;
+            const unsigned dgt = in ? (key >> shift) & 255u : 256u;     // 256 = not counted
+            const unsigned peers = __match_any_sync(0xffffffffu, dgt);  // one add per distinct digit
+            if (in && lane == __ffs(peers) - 1) atomicAdd(&s_hist[dgt], (uint32_t)__popc(peers));
         }
         __syncthreads();
         if (tid < 32) {
@@ -193,6 +221,113 @@ __device__ void radix_select(const Src& src, int n, int K, uint32_t* s_hist, int
     need_eq = kk;
 }
 
+// Threshold by counting.  Finds v, a multiple of 2^low_bit, with at least K of key[0..n)
+// >= v (n >= K >= 1, n < 65536), bisecting the key bits from the first bit in which the
+// keys differ at all.  If some candidate is reached by exactly K keys the search stops
+// there (`count` == K: the keys >= v ARE the top K); otherwise it runs to low_bit and v is
+// the largest such multiple (for low_bit 0: the K-th largest key) with `count` >= K.
+// No shared-memory atomics, so heavily clustered keys cost the same as spread ones.
+//
+// Short lists take five bits per round: warp w counts the keys >= prefix | w << shift over
+// the whole list and the highest w whose count reaches K extends the prefix.  Long lists
+// take two bits per round, every thread counting its share against three candidates.
+// s_cnt: 192 ints.  Every thread returns the same result; kmax = largest key.
+struct Threshold {
+    uint32_t v;
+    int count;
+    uint32_t kmax;
+};
+
+template <int NT>
+__device__ Threshold count_threshold(const uint32_t* key, int n, int K, int low_bit, int* s_cnt) {
+    static_assert(NT == 1024, "one warp per 5-bit candidate");
+    constexpr int NW = NT / 32;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    // common leading bits of all keys
+    uint32_t kmin = 0xffffffffu, kmax = 0u;
+    for (int i = tid; i < n; i += NT) { const uint32_t k = key[i]; kmin = min(kmin, k); kmax = max(kmax, k); }
+    kmin = __reduce_min_sync(0xffffffffu, kmin);
+    kmax = __reduce_max_sync(0xffffffffu, kmax);
+    if (lane == 0) { s_cnt[128 + warp] = (int)kmin; s_cnt[160 + warp] = (int)kmax; }
+    __syncthreads();
+    kmin = __reduce_min_sync(0xffffffffu, (uint32_t)s_cnt[128 + lane]);
+    kmax = __reduce_max_sync(0xffffffffu, (uint32_t)s_cnt[160 + lane]);
+    Threshold res;
+    res.kmax = kmax;
+    res.count = n;
+    int hi = 32 - __clz(kmin ^ kmax);                 // bits [hi-1:0] may differ
+    uint32_t prefix = hi >= 32 ? 0u : (kmax >> hi) << hi;
+    int buf = 0;
+    if (n <= 1024) {
+        while (hi > low_bit && res.count != K) {
+            const int width = hi - low_bit < 5 ? hi - low_bit : 5;
+            const int shift = hi - width;
+            int cnt = 0;
+            if (warp > 0 && warp < (1 << width)) {
+                const uint32_t T = prefix | ((uint32_t)warp << shift);
+#pragma unroll 4
+                for (int i = lane; i < n; i += 32) cnt += key[i] >= T;
+                cnt = __reduce_add_sync(0xffffffffu, cnt);
+            }
+            if (lane == 0) s_cnt[buf * 32 + warp] = cnt;
+            __syncthreads();
+            const int c = s_cnt[buf * 32 + lane];
+            const bool ok = lane == 0 || (lane < (1 << width) && c >= K);
+            const unsigned bal = __ballot_sync(0xffffffffu, ok);   // counts fall with w: a lane prefix
+            const int best = 31 - __clz(bal);
+            const int cbest = __shfl_sync(0xffffffffu, c, best);
+            if (best > 0) res.count = cbest;
+            prefix |= (uint32_t)best << shift;
+            hi = shift;
+            buf ^= 1;
+        }
+    } else {
+        if (((hi - low_bit) & 1) && hi < 32) ++hi;     // whole 2-bit fields; a common bit re-enters
+        if (hi > 32) hi = 32;
+        prefix = hi >= 32 ? 0u : (kmax >> hi) << hi;
+        for (int bit = hi - 2; bit >= low_bit && res.count != K; bit -= 2) {
+            const uint32_t c1 = prefix | (1u << bit), c2 = prefix | (2u << bit), c3 = prefix | (3u << bit);
+            int n12 = 0, n3 = 0;
+            for (int i = tid; i < n; i += NT) {
+                const uint32_t k = key[i];
+                n12 += (k >= c1) + ((k >= c2) << 16);
+                n3 += k >= c3;
+            }
+            n12 = __reduce_add_sync(0xffffffffu, n12);
+            n3 = __reduce_add_sync(0xffffffffu, n3);
+            int* slot = s_cnt + buf * 2 * NW;
+            if (lane == 0) { slot[2 * warp] = n12; slot[2 * warp + 1] = n3; }
+            __syncthreads();
+            int t12 = lane < NW ? slot[2 * lane] : 0, t3 = lane < NW ? slot[2 * lane + 1] : 0;
+            t12 = __reduce_add_sync(0xffffffffu, t12);
+            t3 = __reduce_add_sync(0xffffffffu, t3);
+            if (t3 >= K) { prefix = c3; res.count = t3; }
+            else if ((t12 >> 16) >= K) { prefix = c2; res.count = t12 >> 16; }
+            else if ((t12 & 0xffff) >= K) { prefix = c1; res.count = t12 & 0xffff; }
+            buf ^= 1;
+        }
+    }
+    __syncthreads();
+    res.v = prefix;
+    return res;
+}
+
+// Number of key[0..n) strictly greater than v (block-wide, every thread gets it).
+template <int NT>
+__device__ int count_greater(const uint32_t* key, int n, uint32_t v, int* s_cnt) {
+    constexpr int NW = NT / 32;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    int c = 0;
+    for (int i = tid; i < n; i += NT) c += key[i] > v;
+    c = __reduce_add_sync(0xffffffffu, c);
+    if (lane == 0) s_cnt[warp] = c;
+    __syncthreads();
+    int t = lane < NW ? s_cnt[lane] : 0;
+    t = __reduce_add_sync(0xffffffffu, t);
+    __syncthreads();
+    return t;
+}
+
 // Write, in source order, every element with key > v and the first need_eq elements with
 // key == v into s_sup_idx / s_sup_key.  Source order is ascending index, so the output is
 // the support in ascending index order with ties resolved to the lower index.
@@ -220,52 +355,105 @@ __device__ void ordered_emit(const Src& src, int n, uint32_t vstar, int need_eq,
 }
 
 // Top-K of the n listed entries (ascending index order in, ascending index order out).
+// kmax_out: largest listed key when known (n > K), else 0 with *kmax_known = false.
 template <int NT>
 __device__ int select_listed(const uint32_t* s_key, const int32_t* s_idx, int n, int K,
-                             int32_t* s_sup_idx, uint32_t* s_sup_key, uint32_t* s_hist, int* s_misc,
-                             int* s_ws) {
+                             int32_t* s_sup_idx, uint32_t* s_sup_key, uint32_t* s_hist, int* s_ws,
+                             uint32_t& kmax, bool& kmax_known) {
     int ns;
     if (n <= K) {
         for (int i = threadIdx.x; i < n; i += NT) { s_sup_idx[i] = s_idx[i]; s_sup_key[i] = s_key[i]; }
         ns = n;
+        kmax = 0;
+        kmax_known = false;
     } else {
         SmemSrc src{s_key, s_idx};
+        int* s_cnt = reinterpret_cast<int*>(s_hist);
+        const Threshold t = count_threshold<NT>(s_key, n, K, 0, s_cnt);
         uint32_t vstar;
         int need_eq;
-        radix_select<NT>(src, n, K, s_hist, s_misc, vstar, need_eq);
+        if (t.count == K) { vstar = t.v - 1u; need_eq = 0; }            // exactly K keys are >= v
+        else { vstar = t.v; need_eq = K - count_greater<NT>(s_key, n, vstar, s_cnt); }   // v = K-th largest
         ordered_emit<NT>(src, n, vstar, need_eq, s_sup_idx, s_sup_key, s_ws);
         ns = K;
+        kmax = t.kmax;
+        kmax_known = true;
     }
     __syncthreads();
     return ns;
 }
 
+// Sum each of eight per-lane partials a[0..7] over the LPR lanes of a row group, trading
+// values between lanes as the tree narrows (7-8 shuffles instead of 8 * log2(LPR)).
+// Returns the total of row `row`; for LPR = 16 both lanes of a pair hold the same row.
+template <int LPR>
+__device__ __forceinline__ float reduce8_across(const float* a, int sub, int& row) {
+    float b[4], c[2], d;
+    if (LPR == 16) {
+        const bool h8 = sub & 8, h4 = sub & 4, h2 = sub & 2;
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            b[j] = (h8 ? a[j + 4] : a[j]) + __shfl_xor_sync(0xffffffffu, h8 ? a[j] : a[j + 4], 8);
+#pragma unroll
+        for (int j = 0; j < 2; ++j)
+            c[j] = (h4 ? b[j + 2] : b[j]) + __shfl_xor_sync(0xffffffffu, h4 ? b[j] : b[j + 2], 4);
+        d = (h2 ? c[1] : c[0]) + __shfl_xor_sync(0xffffffffu, h2 ? c[0] : c[1], 2);
+        d += __shfl_xor_sync(0xffffffffu, d, 1);
+        row = sub >> 1;
+    } else {
+        const bool h4 = sub & 4, h2 = sub & 2, h1 = sub & 1;
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            b[j] = (h4 ? a[j + 4] : a[j]) + __shfl_xor_sync(0xffffffffu, h4 ? a[j] : a[j + 4], 4);
+#pragma unroll
+        for (int j = 0; j < 2; ++j)
+            c[j] = (h2 ? b[j + 2] : b[j]) + __shfl_xor_sync(0xffffffffu, h2 ? b[j] : b[j + 2], 2);
+        d = (h1 ? c[1] : c[0]) + __shfl_xor_sync(0xffffffffu, h1 ? c[0] : c[1], 1);
+        row = sub;
+    }
+    return d;
+}
+
 // ------------------------------------------------------------------------------------
 // Eq. 12: out = sum_i softmax(e)_i v_i over the ns selected rows.
-// s_w: ns floats; s_red: (NT/32) * D + NT floats; s_ws: 32 words.
+// The value rows are fetched with 16-byte asynchronous copies into a per-thread landing
+// zone (depth rows per row slot in flight at once); the softmax weights are computed while
+// the first wave is in the air.  s_w: ns floats; s_red: (NT/32) * D + NT floats; s_ws: 32
+// words; s_stage: depth * NT uint4.
 // ------------------------------------------------------------------------------------
 template <int D, int NT>
 __device__ void attend(const uint16_t* vbase, int ns, const int32_t* s_sup_idx, const uint32_t* s_sup_key,
-                       float* s_w, float* s_red, int* s_ws, uint16_t* out_row) {
+                       float* s_w, float* s_red, int* s_ws, uint4* s_stage, int depth, uint32_t kmax,
+                       bool kmax_known, uint16_t* out_row) {
     constexpr int LPR = D / 8;                  // lanes per bf16 row (16 bytes each)
     constexpr int RPW = 32 / LPR;               // rows per warp load
-    constexpr int SLOTS = (NT / 32) * RPW;      // rows per block load
-    constexpr int U = 8;                        // rows in flight per slot
+    constexpr int SLOTS = (NT / 32) * RPW;      // row slots per block
     constexpr int NW = NT / 32;
     constexpr int PARTS = NT / D;               // second-stage partial sums
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int sub = lane % LPR, myslot = warp * RPW + lane / LPR;
+    const char* vsrc = reinterpret_cast<const char*>(vbase) + sub * 16;
+    uint4* my_stage = s_stage + tid;
 
-    uint32_t kmax = 0;
-    for (int i = tid; i < ns; i += NT) kmax = max(kmax, s_sup_key[i]);
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) kmax = max(kmax, __shfl_xor_sync(0xffffffffu, kmax, o));
-    if (lane == 0) s_ws[warp] = (int)kmax;
-    __syncthreads();
-    kmax = 0;
-    for (int w = 0; w < NW; ++w) kmax = max(kmax, (uint32_t)s_ws[w]);
+    auto issue = [&](int base) {
+        for (int u = 0; u < depth; ++u) {
+            const int i = base + u * SLOTS + myslot;
+            if (i < ns) cp_async16(my_stage + u * NT, vsrc + (size_t)s_sup_idx[i] * (D * 2));
+        }
+        cp_async_commit();
+    };
+    issue(0);
+
+    if (!kmax_known) {
+        kmax = 0;
+        for (int i = tid; i < ns; i += NT) kmax = max(kmax, s_sup_key[i]);
+        kmax = __reduce_max_sync(0xffffffffu, kmax);
+        if (lane == 0) s_ws[warp] = (int)kmax;
+        __syncthreads();
+        kmax = __reduce_max_sync(0xffffffffu, (uint32_t)s_ws[lane]);
+        __syncthreads();
+    }
     const float smax = key_score(kmax);
-    __syncthreads();
     float wsum = 0.f;
     for (int i = tid; i < ns; i += NT) {
         const float w = expf(key_score(s_sup_key[i]) - smax);
@@ -278,28 +466,26 @@ __device__ void attend(const uint16_t* vbase, int ns, const int32_t* s_sup_idx, 
     if (lane == 0) s_wsf[warp] = wsum;
     __syncthreads();
     float denom = 0.f;
-    for (int w = 0; w < NW; ++w) denom += s_wsf[w];
+    for (int w = 0; w < NW; ++w) denom += s_wsf[w];      // fixed order
 
     float acc[8];
 #pragma unroll
     for (int e = 0; e < 8; ++e) acc[e] = 0.f;
-    for (int base = 0; base < ns; base += SLOTS * U) {
-        uint4 x[U];
-        float w[U];
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
+    for (int base = 0;;) {
+        cp_async_wait_all();
+        for (int u = 0; u < depth; ++u) {
             const int i = base + u * SLOTS + myslot;
-            const bool ok = i < ns;
-            w[u] = ok ? s_w[i] : 0.f;
-            x[u] = ok ? ldg_stream(vbase + (size_t)s_sup_idx[i] * D + sub * 8) : make_uint4(0, 0, 0, 0);
-        }
+            if (i < ns) {
+                const float w = s_w[i];
+                float f[8];
+                unpack8(my_stage[u * NT], f);
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
-            float f[8];
-            unpack8(x[u], f);
-#pragma unroll
-            for (int e = 0; e < 8; ++e) acc[e] = fmaf(w[u], f[e], acc[e]);
+                for (int e = 0; e < 8; ++e) acc[e] = fmaf(w, f[e], acc[e]);
+            }
         }
+        base += SLOTS * depth;
+        if (base >= ns) break;
+        issue(base);
     }
     // fixed-order reduction: row slots of a warp, then warps in groups, then groups
 #pragma unroll
@@ -314,17 +500,17 @@ __device__ void attend(const uint16_t* vbase, int ns, const int32_t* s_sup_idx, 
     {
         const int j = tid % D, part = tid / D;
         constexpr int WPP = NW / PARTS;          // warps per part
-        float s = 0.f;
+        float sum = 0.f;
 #pragma unroll
-        for (int w = 0; w < WPP; ++w) s += s_red[(part * WPP + w) * D + j];
-        s_red[NW * D + part * D + j] = s;
+        for (int w = 0; w < WPP; ++w) sum += s_red[(part * WPP + w) * D + j];
+        s_red[NW * D + part * D + j] = sum;
     }
     __syncthreads();
     if (tid < D) {
-        float s = 0.f;
+        float sum = 0.f;
 #pragma unroll
-        for (int p = 0; p < PARTS; ++p) s += s_red[NW * D + p * D + tid];
-        const float o = ns > 0 ? s / denom : 0.f;
+        for (int p = 0; p < PARTS; ++p) sum += s_red[NW * D + p * D + tid];
+        const float o = ns > 0 ? sum / denom : 0.f;
         out_row[tid] = __bfloat16_as_ushort(__float2bfloat16_rn(o));
     }
 }
@@ -339,7 +525,7 @@ __global__ void __launch_bounds__(REUSE_THREADS, 1) reuse_kernel(const StepArgs 
     constexpr int LPR = D / 8, RPW = 32 / LPR, SLOTS = NW * RPW;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     // layout (words): q[D] rho[M] sel[r] ws[32] misc[8] hist[256] sup_idx[K] sup_key[K] w[K]
-    //                 | big: idx[cap] key[cap], aliased later by red[NW*D+NT] | bitmap
+    //                 | big: idx[cap] key[cap], aliased later by red[NW*D+NT] | bitmap | stage[depth*NT*4]
     float* s_q = reinterpret_cast<float*>(smem_raw);
     float* s_rho = s_q + D;
     int* s_sel = reinterpret_cast<int*>(s_rho + a.M);
@@ -355,6 +541,7 @@ __global__ void __launch_bounds__(REUSE_THREADS, 1) reuse_kernel(const StepArgs 
     float* s_red = reinterpret_cast<float*>(s_idx);
     const int big_words = (max(2 * a.cap, NW * D + NT) + 3) & ~3;
     uint32_t* s_bm = reinterpret_cast<uint32_t*>(s_idx) + big_words;
+    uint4* s_stage = reinterpret_cast<uint4*>(s_bm + ((((int)a.max_seq_len + 31) / 32 + 3) & ~3));
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int bh = blockIdx.x;
@@ -363,28 +550,18 @@ __global__ void __launch_bounds__(REUSE_THREADS, 1) reuse_kernel(const StepArgs 
     const int M = a.M, fill = a.fill, L = a.L, K = a.K;
     const int nwords = (L + 31) >> 5;
 
-    // normalised query (text above Eq. 6) on warp 0 while the others clear the bitmap
-    if (warp == 0) {
-        const uint16_t* qrow = a.q + (size_t)bh * D;
-        float x[D / 32], acc = 0.f;
-#pragma unroll
-        for (int u = 0; u < D / 32; ++u) {
-            x[u] = __uint_as_float((uint32_t)qrow[lane + 32 * u] << 16);
-            acc = fmaf(x[u], x[u], acc);
-        }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-        const float nrm = sqrtf(acc);
-#pragma unroll
-        for (int u = 0; u < D / 32; ++u) s_q[lane + 32 * u] = nrm > 0.f ? x[u] / nrm : 0.f;
-    } else if (!a.refresh) {
-        uint4* bm4 = reinterpret_cast<uint4*>(s_bm);
-        for (int w = tid - 32; w < (nwords + 3) >> 2; w += NT - 32) bm4[w] = make_uint4(0, 0, 0, 0);
+    RETOPK_PHASE(0, 0);
+    // Every warp reads the query itself (four elements per lane) next to its cache rows, so
+    // one memory latency covers both:  rho_c = (qbar_c . q) / |q|   (Eq. 6)
+    float q4[4] = {0.f, 0.f, 0.f, 0.f};
+    if (lane < D / 4) {
+        const uint2 raw = *reinterpret_cast<const uint2*>(a.q + (size_t)bh * D + 4 * lane);
+        q4[0] = bf16_lo(raw.x); q4[1] = bf16_hi(raw.x); q4[2] = bf16_lo(raw.y); q4[3] = bf16_hi(raw.y);
     }
-    __syncthreads();
-
-    // Eq. 6: rho_c for every cached entry, four entries in flight per warp
-    for (int c0 = warp; c0 < fill; c0 += NW * 4) {
+    if (tid < a.r) s_sel[tid] = -1;
+    if (tid == 0) reinterpret_cast<float*>(s_misc)[0] = -CUDART_INF_F;
+    float inv_nrm = 0.f;
+    for (int c0 = warp; c0 < fill || c0 == warp; c0 += NW * 4) {
         float4 x[4];
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
@@ -393,51 +570,57 @@ __global__ void __launch_bounds__(REUSE_THREADS, 1) reuse_kernel(const StepArgs 
                 ? reinterpret_cast<const float4*>(a.qbar_cache + ((size_t)bh * M + c) * D)[lane]
                 : make_float4(0.f, 0.f, 0.f, 0.f);
         }
+        if (c0 == warp) {
+            // first trip: clear the bitmap while the loads fly, then the query norm
+            if (!a.refresh) {
+                uint4* bm4 = reinterpret_cast<uint4*>(s_bm);
+                for (int w = tid; w < (nwords + 3) >> 2; w += NT) bm4[w] = make_uint4(0, 0, 0, 0);
+            }
+            float n2 = q4[0] * q4[0];
+            n2 = fmaf(q4[1], q4[1], n2); n2 = fmaf(q4[2], q4[2], n2); n2 = fmaf(q4[3], q4[3], n2);
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) n2 += __shfl_xor_sync(0xffffffffu, n2, o);
+            const float nrm = sqrtf(n2);
+            inv_nrm = nrm > 0.f ? 1.f / nrm : 0.f;
+            if (warp == 0 && lane < D / 4) {
+#pragma unroll
+                for (int e = 0; e < 4; ++e) s_q[4 * lane + e] = nrm > 0.f ? q4[e] / nrm : 0.f;
+            }
+        }
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
             const int c = c0 + NW * u;
-            float acc = 0.f;
-            if (lane < D / 4) {
-                acc = x[u].x * s_q[4 * lane];
-                acc = fmaf(x[u].y, s_q[4 * lane + 1], acc);
-                acc = fmaf(x[u].z, s_q[4 * lane + 2], acc);
-                acc = fmaf(x[u].w, s_q[4 * lane + 3], acc);
-            }
+            float acc = x[u].x * q4[0];
+            acc = fmaf(x[u].y, q4[1], acc);
+            acc = fmaf(x[u].z, q4[2], acc);
+            acc = fmaf(x[u].w, q4[3], acc);
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-            if (lane == 0 && c < fill) s_rho[c] = acc;
+            if (lane == 0 && c < fill) s_rho[c] = acc * inv_nrm;
         }
     }
     __syncthreads();
+    RETOPK_PHASE(0, 2);
 
-    // Eq. 7: rho_max and the min(r, fill) most similar slots (ties -> lower slot)
+    // Eq. 7: rho_max and the min(r, fill) most similar slots.  Every cached entry ranks
+    // itself against the others (larger rho first, ties -> lower slot).
     const int n_sel = a.r < fill ? a.r : fill;
-    if (warp == 0) {
-        float rho_max = -CUDART_INF_F;
-        for (int s = 0; s < n_sel; ++s) {
-            float bv = -CUDART_INF_F;
-            int bc = 0x7fffffff;
-            for (int c = lane; c < fill; c += 32) {
-                float v = s_rho[c];
-                if (v != -CUDART_INF_F && (v > bv || (v == bv && c < bc))) { bv = v; bc = c; }
-            }
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) {
-                float ov = __shfl_xor_sync(0xffffffffu, bv, o);
-                int oc = __shfl_xor_sync(0xffffffffu, bc, o);
-                if (ov > bv || (ov == bv && oc < bc)) { bv = ov; bc = oc; }
-            }
-            if (s == 0) rho_max = bv;
-            if (lane == 0) {
-                s_sel[s] = (bc == 0x7fffffff) ? -1 : bc;
-                if (bc != 0x7fffffff) s_rho[bc] = -CUDART_INF_F;   // taken
-            }
-            __syncwarp();
+    if (tid < fill) {
+        const float mine = s_rho[tid];
+        int rank = 0;
+        for (int c = 0; c < fill; c += 4) {
+            const float4 o = *reinterpret_cast<const float4*>(s_rho + c);
+            rank += (c < fill) && (o.x > mine || (o.x == mine && c < tid));
+            rank += (c + 1 < fill) && (o.y > mine || (o.y == mine && c + 1 < tid));
+            rank += (c + 2 < fill) && (o.z > mine || (o.z == mine && c + 2 < tid));
+            rank += (c + 3 < fill) && (o.w > mine || (o.w == mine && c + 3 < tid));
         }
-        if (lane == 0) reinterpret_cast<float*>(s_misc)[0] = rho_max;
+        if (rank < n_sel) s_sel[rank] = tid;
+        if (rank == 0) reinterpret_cast<float*>(s_misc)[0] = mine;
     }
     __syncthreads();
     const float rho_max = reinterpret_cast<float*>(s_misc)[0];
+    RETOPK_PHASE(0, 3);
 
     // Eq. 13
     int path;
@@ -486,6 +669,7 @@ __global__ void __launch_bounds__(REUSE_THREADS, 1) reuse_kernel(const StepArgs 
         if (bad) atomicOr(a.status, 1u);
     }
     __syncthreads();
+    RETOPK_PHASE(0, 4);
     int n;
     {
         const int wpt = (nwords + NT - 1) / NT;
@@ -511,41 +695,54 @@ __global__ void __launch_bounds__(REUSE_THREADS, 1) reuse_kernel(const StepArgs 
         a.counters[(size_t)bh * 4 + 3] += n;
     }
     __syncthreads();
+    RETOPK_PHASE(0, 5);
 
-    // Eq. 10: exact current-query scores on the candidate rows only
+    // Eq. 10: exact current-query scores on the candidate rows only.  Every lane copies its
+    // 16 bytes of each row asynchronously into its own landing zone and reads them back
+    // itself, so a whole wave of rows is in flight with no registers held and no barrier.
     {
         const int sub = lane % LPR, myslot = warp * RPW + lane / LPR;
-        const uint16_t* kbase = a.k + (size_t)bkv * a.max_seq_len * D;
+        const char* ksrc = reinterpret_cast<const char*>(a.k + (size_t)bkv * a.max_seq_len * D) + sub * 16;
         float qf[8];
         unpack8(*reinterpret_cast<const uint4*>(a.q + (size_t)bh * D + sub * 8), qf);
-        constexpr int U = 8;
-        for (int base = 0; base < n; base += SLOTS * U) {
-            uint4 x[U];
-#pragma unroll
-            for (int u = 0; u < U; ++u) {
+        const int depth = a.stage_depth;
+        uint4* my_stage = s_stage + tid;
+        for (int base = 0; base < n; base += SLOTS * depth) {
+            for (int u = 0; u < depth; ++u) {
                 const int i = base + u * SLOTS + myslot;
-                x[u] = i < n ? ldg_stream(kbase + (size_t)s_idx[i] * D + sub * 8) : make_uint4(0, 0, 0, 0);
+                if (i < n) cp_async16(my_stage + u * NT, ksrc + (size_t)s_idx[i] * (D * 2));
             }
+            cp_async_commit();
+            cp_async_wait_all();
+            for (int u0 = 0; u0 < depth; u0 += 8) {
+                float part[8];
 #pragma unroll
-            for (int u = 0; u < U; ++u) {
-                const int i = base + u * SLOTS + myslot;
-                float acc = dot8(x[u], qf);
-#pragma unroll
-                for (int o = LPR / 2; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-                if (sub == 0 && i < n) s_key[i] = score_key(acc * a.scale);
+                for (int uu = 0; uu < 8; ++uu) {
+                    const int i = base + (u0 + uu) * SLOTS + myslot;
+                    part[uu] = (u0 + uu < depth && i < n) ? dot8(my_stage[(u0 + uu) * NT], qf) : 0.f;
+                }
+                int row;
+                const float tot = reduce8_across<LPR>(part, sub, row);
+                const int i = base + (u0 + row) * SLOTS + myslot;
+                if ((LPR == 8 || (sub & 1) == 0) && u0 + row < depth && i < n) s_key[i] = score_key(tot * a.scale);
             }
         }
     }
     __syncthreads();
+    RETOPK_PHASE(0, 6);
 
     // Eq. 11: Top-K of the candidates; insert the support
-    const int ns = select_listed<NT>(s_key, s_idx, n, K, s_sup_idx, s_sup_key, s_hist, s_misc, s_ws);
+    uint32_t kmax;
+    bool kmax_known;
+    const int ns = select_listed<NT>(s_key, s_idx, n, K, s_sup_idx, s_sup_key, s_hist, s_ws, kmax, kmax_known);
+    RETOPK_PHASE(0, 7);
     int32_t* sup_out = a.sup_cache + ((size_t)bh * M + a.slot) * K;
     for (int i = tid; i < K; i += NT) sup_out[i] = i < ns ? s_sup_idx[i] : -1;
 
     // Eq. 12 (s_red aliases the candidate lists, which are dead now)
-    attend<D, NT>(a.v + (size_t)bkv * a.max_seq_len * D, ns, s_sup_idx, s_sup_key, s_w, s_red, s_ws,
-                  a.out + (size_t)bh * D);
+    attend<D, NT>(a.v + (size_t)bkv * a.max_seq_len * D, ns, s_sup_idx, s_sup_key, s_w, s_red, s_ws, s_stage,
+                  a.stage_depth, kmax, kmax_known, a.out + (size_t)bh * D);
+    RETOPK_PHASE(0, 8);
 }
 
 // ------------------------------------------------------------------------------------
@@ -660,13 +857,21 @@ __global__ void __launch_bounds__(SCAN_THREADS) scan_kernel(const StepArgs a) {
                     mma_bf16_16816(c, x[s][j].z, y[s][j].z, x[s][j].w, y[s][j].w, bq[nt][j][1][0], bq[nt][j][1][1]);
                 }
                 // c0,c1: row r0, heads 2t, 2t+1 of this tile; c2,c3: row r1
+                const int tile_row = rbase + s * 128;
 #pragma unroll
                 for (int e = 0; e < 2; ++e) {
                     const int head = nt * 8 + 2 * t + e;
+                    // tile maximum over the 16 rows (rows past L repeat row L-1: harmless)
+                    float m = fmaxf(c[e], c[2 + e]);
+                    m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 4));
+                    m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 8));
+                    m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 16));
                     if (head < G && ((need >> head) & 1u)) {
                         float* srow = a.ws_scores + (size_t)(head0 + head) * a.score_stride;
                         if (r0 < L) srow[r0] = c[e] * scale;
                         if (r1 < L) srow[r1] = c[2 + e] * scale;
+                        if (g == 0 && tile_row < L)
+                            a.ws_tmax[(size_t)(head0 + head) * a.tmax_stride + (tile_row >> 4)] = m * scale;
                     }
                 }
             }
@@ -676,173 +881,139 @@ __global__ void __launch_bounds__(SCAN_THREADS) scan_kernel(const StepArgs a) {
 
 // ------------------------------------------------------------------------------------
 // exact_finish_kernel
+//
+// Global Top-K without reading all L scores again.  The scan left the maximum of every
+// 16-row tile.  If v is the K-th largest of (groups of) tile maxima, at least K different
+// tiles hold a score >= v, so the K-th largest score is >= v: every member of the exact
+// support lies in a tile whose maximum reaches v.  Only those tiles (about K of them) are
+// read back, their scores >= v are listed in index order, and the exact Top-K with the
+// lower-index tie rule is taken from that list.
 // ------------------------------------------------------------------------------------
 template <int D>
 __global__ void __launch_bounds__(EXACT_THREADS, 1) exact_finish_kernel(const StepArgs a) {
     constexpr int NT = EXACT_THREADS;
-    constexpr int NW = NT / 32;
     const int bh = blockIdx.x;
     if (a.mode == MODE_RETOPK && a.ws_path[bh] == PATH_REUSE) return;
 
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    // layout (words): key[NS] idx[NS] (aliased later by red[NW*D+NT]) sup_idx[K] sup_key[K] w[K]
-    //                 hist[SAMPLE_BINS] ws[32] misc[8] wcnt[NW] woff[NW]
+    // layout (words): key[NS] idx[NS] (aliased later by red[NW*D+NT]) tile[NS/2]
+    //                 sup_idx[K] sup_key[K] w[K] cnt[256] ws[32] misc[8] stage[depth*NT*4]
     uint32_t* s_key = reinterpret_cast<uint32_t*>(smem_raw);
     int32_t* s_idx = reinterpret_cast<int32_t*>(s_key + a.NS);
     float* s_red = reinterpret_cast<float*>(smem_raw);
-    int32_t* s_sup_idx = s_idx + a.NS;
+    int32_t* s_tile = s_idx + a.NS;
+    int32_t* s_sup_idx = s_tile + a.NS / 2;
     uint32_t* s_sup_key = reinterpret_cast<uint32_t*>(s_sup_idx + a.K);
     float* s_w = reinterpret_cast<float*>(s_sup_key + a.K);
     uint32_t* s_hist = reinterpret_cast<uint32_t*>(s_w + a.K);
-    int* s_ws = reinterpret_cast<int*>(s_hist + SAMPLE_BINS);
+    int* s_ws = reinterpret_cast<int*>(s_hist + 256);
     int* s_misc = s_ws + 32;
-    int* s_wcnt = s_misc + 8;
-    int* s_woff = s_wcnt + NW;
+    // landing zone of the value-row copies, on a 16-byte boundary
+    uint4* s_stage = reinterpret_cast<uint4*>(
+        reinterpret_cast<uint32_t*>(smem_raw) + ((2 * a.NS + a.NS / 2 + 3 * a.K + 256 + 32 + 8 + 3) & ~3));
 
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int tid = threadIdx.x;
     const int b = bh / a.Hq, h = bh % a.Hq;
     const int bkv = b * a.Hkv + h / a.G;
     const int K = a.K, L = a.L, NS = a.NS;
     const float* sc = a.ws_scores + (size_t)bh * a.score_stride;
+    const float* tm = a.ws_tmax + (size_t)bh * a.tmax_stride;
 
     int ns = -1;      // selected entries in s_sup_*; -1 = not selected yet
-    int n = 0;        // collected entries in s_key / s_idx
+    int n = 0;        // listed entries in s_key / s_idx
     bool slow = false;
+    RETOPK_PHASE(2, 0);
 
     if (L <= K) {
         for (int i = tid; i < L; i += NT) { s_sup_idx[i] = i; s_sup_key[i] = score_key(sc[i]); }
         ns = L;
         __syncthreads();
     } else {
-        // 1. threshold from a block-strided sample, so that about 2K scores pass it
-        const bool all = L <= SAMPLE_MAX;
-        const int n_s = all ? L : SAMPLE_MAX;
-        for (int i = tid; i < SAMPLE_BINS; i += NT) s_hist[i] = 0;
-        {
-            const int blk = L >> 3;
-            float sv[SAMPLE_MAX / NT];
-#pragma unroll
-            for (int u = 0; u < SAMPLE_MAX / NT; ++u) {
-                const int i = tid + u * NT;
-                const int pos = all ? i : (i >> 10) * blk + (i & 1023);
-                sv[u] = i < n_s ? sc[pos] : 0.f;
-            }
-            __syncthreads();
-#pragma unroll
-            for (int u = 0; u < SAMPLE_MAX / NT; ++u)
-                if (tid + u * NT < n_s) atomicAdd(&s_hist[score_key(sv[u]) >> 21], 1u);
-        }
-        __syncthreads();
-        int j;
-        if (all) j = K;
-        else {
-            const float kf = (float)K * (float)n_s / (float)L;
-            j = (int)ceilf(kf + 4.f * sqrtf(kf) + 8.f);
-        }
+        const int ntile = (L + TILE_ROWS - 1) / TILE_ROWS;
+        const int tcap = NS / 2;
+        // 1. lower bound v for the K-th score from the tile maxima (grouped so the list is short)
         uint32_t thr_key = 0;
-        if (j < n_s) {
-            // lowest bin edge with at least j sampled scores at or above it
-            constexpr int BPT = SAMPLE_BINS / NT;
-            int c = 0;
-#pragma unroll
-            for (int u = 0; u < BPT; ++u) c += (int)s_hist[SAMPLE_BINS - 1 - BPT * tid - u];
-            int total;
-            const int above = block_excl_scan<NT>(c, s_ws, total);
-            if (above < j && j <= above + c) {
-                int acc = above;
-                for (int u = 0; u < BPT; ++u) {
-                    const int bin = SAMPLE_BINS - 1 - BPT * tid - u;
-                    acc += (int)s_hist[bin];
-                    if (acc >= j) { s_misc[2] = bin; break; }
-                }
+        int g2 = 1;
+        while ((ntile + g2 - 1) / g2 > 2048 && ntile / (2 * g2) >= 2 * K) g2 *= 2;
+        while ((ntile + g2 - 1) / g2 > NS) g2 *= 2;
+        const int n2 = (ntile + g2 - 1) / g2;
+        if (n2 >= K) {
+            for (int i2 = tid; i2 < n2; i2 += NT) {
+                const int t0 = i2 * g2;
+                float m = tm[t0];
+                for (int j = 1; j < g2 && t0 + j < ntile; ++j) m = fmaxf(m, tm[t0 + j]);
+                s_key[i2] = score_key(m);
             }
             __syncthreads();
-            thr_key = (uint32_t)s_misc[2] << 21;
+            thr_key = count_threshold<NT>(s_key, n2, K, 7, reinterpret_cast<int*>(s_hist)).v;
         }
-
-        // 2. every warp collects, in index order, the scores of its own contiguous segment
-        //    that reach the threshold, into its own slice of the shared lists
-        const int cap_w = NS / NW;
-        const int wseg = ((L + NW * 128 - 1) / (NW * 128)) * 128;
-        const int begin = warp * wseg;
-        const int end = begin + wseg < L ? begin + wseg : L;
-        uint32_t* wkey = s_key + warp * cap_w;
-        int32_t* widx = s_idx + warp * cap_w;
-        const unsigned lt = (1u << lane) - 1u;
-        int cnt_w = 0;
-        for (int base = begin; base < end; base += 128 * 4) {
-            float4 x[4];
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const int i0 = base + u * 128 + lane * 4;
-                x[u] = i0 < end ? *reinterpret_cast<const float4*>(sc + i0) : make_float4(0.f, 0.f, 0.f, 0.f);
+        RETOPK_PHASE(2, 1);
+        // 2. the tiles whose maximum reaches v, in ascending order
+        int nhit = 0;
+        for (int base = 0; base < ntile; base += NT * 4) {
+            const int t0 = base + tid * 4;
+            int f[4] = {0, 0, 0, 0}, cnt = 0;
+            if (t0 < ntile) {
+                const float4 m4 = *reinterpret_cast<const float4*>(tm + t0);
+                f[0] = score_key(m4.x) >= thr_key;
+                f[1] = (t0 + 1 < ntile) && score_key(m4.y) >= thr_key;
+                f[2] = (t0 + 2 < ntile) && score_key(m4.z) >= thr_key;
+                f[3] = (t0 + 3 < ntile) && score_key(m4.w) >= thr_key;
+                cnt = f[0] + f[1] + f[2] + f[3];
             }
+            int total;
+            int pos = nhit + block_excl_scan<NT>(cnt, s_ws, total);
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const int i0 = base + u * 128 + lane * 4;
-                uint32_t key[4] = {score_key(x[u].x), score_key(x[u].y), score_key(x[u].z), score_key(x[u].w)};
-                int f[4];
-                unsigned bal[4];
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    f[e] = (i0 + e < end) && key[e] >= thr_key;
-                    bal[e] = __ballot_sync(0xffffffffu, f[e]);
+            for (int e = 0; e < 4; ++e)
+                if (f[e]) {
+                    if (pos < tcap) s_tile[pos] = t0 + e;
+                    ++pos;
                 }
-                if (bal[0] | bal[1] | bal[2] | bal[3]) {
-                    int pos = cnt_w + __popc(bal[0] & lt) + __popc(bal[1] & lt) + __popc(bal[2] & lt) +
-                              __popc(bal[3] & lt);
-#pragma unroll
-                    for (int e = 0; e < 4; ++e)
-                        if (f[e]) {
-                            if (pos < cap_w) { wkey[pos] = key[e]; widx[pos] = i0 + e; }
-                            ++pos;
-                        }
-                    cnt_w += __popc(bal[0]) + __popc(bal[1]) + __popc(bal[2]) + __popc(bal[3]);
-                }
-            }
-        }
-        if (lane == 0) s_wcnt[warp] = cnt_w;
-        __syncthreads();
-        if (warp == 0) {
-            const int c = s_wcnt[lane];
-            int inc = c;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                int tt = __shfl_up_sync(0xffffffffu, inc, o);
-                if (lane >= o) inc += tt;
-            }
-            s_woff[lane] = inc - c;
-            const unsigned over = __ballot_sync(0xffffffffu, c > cap_w);
-            if (lane == 31) { s_misc[3] = inc; s_misc[4] = over != 0; }
+            nhit += total;
         }
         __syncthreads();
-        n = s_misc[3];
-        if (s_misc[4] || n < K) slow = true;
+        RETOPK_PHASE(2, 2);
+        if (nhit > tcap) slow = true;
         else {
-            // 3. close the gaps between the warp slices (through registers: slices overlap targets)
-            uint32_t mk[8];
-            int32_t mi[8];
-            const int per_thread = (NS + NT - 1) / NT;     // <= 8 for NS <= 8192; more handled below
-            for (int chunk = 0; chunk < per_thread; chunk += 8) {
+            // 3. one thread per hit tile: its 16 scores, those >= v listed in index order
+            for (int base = 0; base < nhit; base += NT) {
+                const int it = base + tid;
+                float4 x[4];
+                int row0 = 0;
+                unsigned fl = 0;
+                if (it < nhit) {
+                    row0 = s_tile[it] * TILE_ROWS;
 #pragma unroll
-                for (int u = 0; u < 8; ++u) {
-                    const int e = (chunk + u) * NT + tid;
-                    const int w = e / cap_w, jj = e - w * cap_w;
-                    const bool ok = e < NS && jj < s_wcnt[w];
-                    mk[u] = ok ? s_key[e] : 0u;
-                    mi[u] = ok ? s_idx[e] : -1;
-                }
-                __syncthreads();
+                    for (int u = 0; u < 4; ++u) x[u] = *reinterpret_cast<const float4*>(sc + row0 + 4 * u);
 #pragma unroll
-                for (int u = 0; u < 8; ++u) {
-                    const int e = (chunk + u) * NT + tid;
-                    const int w = e / cap_w, jj = e - w * cap_w;
-                    if (mi[u] >= 0) { s_key[s_woff[w] + jj] = mk[u]; s_idx[s_woff[w] + jj] = mi[u]; }
+                    for (int u = 0; u < 4; ++u) {
+                        const float v4[4] = {x[u].x, x[u].y, x[u].z, x[u].w};
+#pragma unroll
+                        for (int e = 0; e < 4; ++e)
+                            if (row0 + 4 * u + e < L && score_key(v4[e]) >= thr_key) fl |= 1u << (4 * u + e);
+                    }
                 }
-                __syncthreads();
+                int total;
+                int pos = n + block_excl_scan<NT>(__popc(fl), s_ws, total);
+                if (fl) {
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const float v4[4] = {x[u].x, x[u].y, x[u].z, x[u].w};
+#pragma unroll
+                        for (int e = 0; e < 4; ++e)
+                            if ((fl >> (4 * u + e)) & 1u) {
+                                if (pos < NS) { s_key[pos] = score_key(v4[e]); s_idx[pos] = row0 + 4 * u + e; }
+                                ++pos;
+                            }
+                    }
+                }
+                n += total;
             }
+            __syncthreads();
+            if (n > NS) slow = true;
         }
     }
+    RETOPK_PHASE(2, 3);
     if (slow) {
         // multi-pass select straight from the score array (heavy ties, odd distributions)
         ScoreSrc src{sc};
@@ -854,7 +1025,10 @@ __global__ void __launch_bounds__(EXACT_THREADS, 1) exact_finish_kernel(const St
         if (tid == 0) atomicAdd(a.slow_select, 1ull);
         __syncthreads();
     }
-    if (ns < 0) ns = select_listed<NT>(s_key, s_idx, n, K, s_sup_idx, s_sup_key, s_hist, s_misc, s_ws);
+    uint32_t kmax = 0;
+    bool kmax_known = false;
+    if (ns < 0) ns = select_listed<NT>(s_key, s_idx, n, K, s_sup_idx, s_sup_key, s_hist, s_ws, kmax, kmax_known);
+    RETOPK_PHASE(2, 4);
 
     // record the support (cache insert / caller's index output)
     int32_t* sup_out = nullptr;
@@ -863,8 +1037,9 @@ __global__ void __launch_bounds__(EXACT_THREADS, 1) exact_finish_kernel(const St
     if (sup_out)
         for (int i = tid; i < K; i += NT) sup_out[i] = i < ns ? s_sup_idx[i] : -1;
 
-    attend<D, NT>(a.v + (size_t)bkv * a.max_seq_len * D, ns, s_sup_idx, s_sup_key, s_w, s_red, s_ws,
-                  a.out + (size_t)bh * D);
+    attend<D, NT>(a.v + (size_t)bkv * a.max_seq_len * D, ns, s_sup_idx, s_sup_key, s_w, s_red, s_ws, s_stage,
+                  a.exact_stage_depth, kmax, kmax_known, a.out + (size_t)bh * D);
+    RETOPK_PHASE(2, 5);
 }
 
 // Clear the caches (supports to -1, queries and counters to 0).

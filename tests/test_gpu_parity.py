@@ -46,7 +46,8 @@ def bits(x):
     (1, 4, 4, 128, 9000, 100, 9001),      # longer than the threshold sample
     (1, 16, 1, 64, 777, 33, 800),         # two head tiles per group
     (1, 2, 1, 128, 300, 512, 300),        # fewer keys than K
-    (1, 32, 8, 128, 20000, 2048, 20480),  # large K
+    (1, 32, 8, 128, 20000, 2048, 20480),  # large K, fewer 16-row tiles than K: multi-pass select
+    (1, 8, 2, 128, 40000, 2048, 40000),   # large K with enough tiles for the tile-maximum bound
 ])
 def test_exact_topk_decode_matches_oracle(rt, P, oracle_mod, B, H_q, H_kv, d, L, K, Lmax):
     rng = np.random.default_rng(L + K)
@@ -68,7 +69,10 @@ def test_exact_topk_decode_matches_oracle(rt, P, oracle_mod, B, H_q, H_kv, d, L,
             P.assert_support_matches(idx[b, h], ref_idx[b, h], q[b, h], k[b, h // G], kth,
                                      f"seq {b} head {h}")
     P.assert_outputs_close(out, ref_out, "exact_topk_decode")
-    assert g.stats()["slow_select"] == 0
+    # the tile-maximum bound needs at least K 16-row tiles, or all of L must fit the shared list
+    list_capacity = 8192 if 16 * K <= 8192 else 16384
+    fast = L <= K or -(-L // 16) >= K or L <= list_capacity
+    assert g.stats()["slow_select"] == (0 if fast else B * H_q)
     assert g.last_launch_count() == 2
 
 
