@@ -43,6 +43,7 @@ constexpr int EXACT_THREADS = 1024;
 constexpr int SCAN_THREADS = 256;
 constexpr int SCAN_TILE_ROWS = 256;  // key rows per scan work item
 constexpr int MAX_GROUPS = 4096;     // B * H_kv limit (shared list in scan_kernel)
+constexpr int SCRATCH_WORDS = 1056;  // histogram scratch of the threshold search (32 x 32 + 32)
 constexpr int TILE_ROWS = 16;        // rows per score tile whose maximum the scan records
 
 struct StepArgs {
@@ -72,7 +73,7 @@ struct StepArgs {
     float* ws_scores;        // [B*Hq][score_stride]
     float* ws_tmax;          // [B*Hq][tmax_stride] largest score of every 16-row key tile
     long long tmax_stride;   // multiple of 4
-    long long* counters;     // [B*Hq][4] reuse, fallback, refresh, cand_sum
+    unsigned long long* counters;   // [B*Hq][4] reuse, fallback, refresh, cand_sum
     unsigned int* status;
     unsigned long long* slow_select;
     unsigned long long* scan_groups;
@@ -101,6 +102,11 @@ __device__ __forceinline__ uint4 ldg_stream(const void* p) {
                  : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p));
     return r;
 }
+
+// Programmatic dependent launch: a kernel launched with the stream-serialisation attribute
+// may start while its predecessor still runs; it must call pdl_wait() before touching
+// anything the predecessor writes.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
 // 16-byte asynchronous global -> shared copy (L2 only), and its completion wait.
 __device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
@@ -221,111 +227,79 @@ __device__ void radix_select(const Src& src, int n, int K, uint32_t* s_hist, int
     need_eq = kk;
 }
 
-// Threshold by counting.  Finds v, a multiple of 2^low_bit, with at least K of key[0..n)
-// >= v (n >= K >= 1, n < 65536), bisecting the key bits from the first bit in which the
-// keys differ at all.  If some candidate is reached by exactly K keys the search stops
-// there (`count` == K: the keys >= v ARE the top K); otherwise it runs to low_bit and v is
-// the largest such multiple (for low_bit 0: the K-th largest key) with `count` >= K.
-// No shared-memory atomics, so heavily clustered keys cost the same as spread ones.
-//
-// Short lists take five bits per round: warp w counts the keys >= prefix | w << shift over
-// the whole list and the highest w whose count reaches K extends the prefix.  Long lists
-// take two bits per round, every thread counting its share against three candidates.
-// s_cnt: 192 ints.  Every thread returns the same result; kmax = largest key.
+// Threshold by radix bisection.  Finds v, a multiple of 2^low_bit, with at least K of
+// key[0..n) >= v (n >= K >= 1), five key bits per round, starting at the first bit in
+// which the keys differ at all.  Each round histograms the next digit of the keys that
+// still match the prefix into 32 bins x 32 lane columns (a lane only ever adds to its own
+// column, so clustered keys do not serialise), sums the columns, and descends into the
+// digit that holds the K-th largest key.
+//   count == K : exactly K keys are >= v (the search stopped as soon as that held);
+//   count  > K : v is the largest multiple with >= K keys at or above it; for low_bit 0 it
+//                is the K-th largest key itself and `need` of the keys equal to it belong
+//                to the top K.
+// s_h: 1024 + 32 ints.  Every thread returns the same result; kmax = largest key.
 struct Threshold {
     uint32_t v;
     int count;
+    int need;
     uint32_t kmax;
 };
 
 template <int NT>
-__device__ Threshold count_threshold(const uint32_t* key, int n, int K, int low_bit, int* s_cnt) {
-    static_assert(NT == 1024, "one warp per 5-bit candidate");
-    constexpr int NW = NT / 32;
+__device__ Threshold count_threshold(const uint32_t* key, int n, int K, int low_bit, int* s_h) {
+    static_assert(NT == 1024, "one histogram word per thread, one digit per warp");
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    int* s_tot = s_h + 1024;
     // common leading bits of all keys
     uint32_t kmin = 0xffffffffu, kmax = 0u;
     for (int i = tid; i < n; i += NT) { const uint32_t k = key[i]; kmin = min(kmin, k); kmax = max(kmax, k); }
     kmin = __reduce_min_sync(0xffffffffu, kmin);
     kmax = __reduce_max_sync(0xffffffffu, kmax);
-    if (lane == 0) { s_cnt[128 + warp] = (int)kmin; s_cnt[160 + warp] = (int)kmax; }
+    if (lane == 0) { s_h[warp] = (int)kmin; s_h[32 + warp] = (int)kmax; }
     __syncthreads();
-    kmin = __reduce_min_sync(0xffffffffu, (uint32_t)s_cnt[128 + lane]);
-    kmax = __reduce_max_sync(0xffffffffu, (uint32_t)s_cnt[160 + lane]);
+    kmin = __reduce_min_sync(0xffffffffu, (uint32_t)s_h[lane]);
+    kmax = __reduce_max_sync(0xffffffffu, (uint32_t)s_h[32 + lane]);
+    __syncthreads();
     Threshold res;
     res.kmax = kmax;
     res.count = n;
     int hi = 32 - __clz(kmin ^ kmax);                 // bits [hi-1:0] may differ
     uint32_t prefix = hi >= 32 ? 0u : (kmax >> hi) << hi;
-    int buf = 0;
-    if (n <= 1024) {
-        while (hi > low_bit && res.count != K) {
-            const int width = hi - low_bit < 5 ? hi - low_bit : 5;
-            const int shift = hi - width;
-            int cnt = 0;
-            if (warp > 0 && warp < (1 << width)) {
-                const uint32_t T = prefix | ((uint32_t)warp << shift);
-#pragma unroll 4
-                for (int i = lane; i < n; i += 32) cnt += key[i] >= T;
-                cnt = __reduce_add_sync(0xffffffffu, cnt);
-            }
-            if (lane == 0) s_cnt[buf * 32 + warp] = cnt;
-            __syncthreads();
-            const int c = s_cnt[buf * 32 + lane];
-            const bool ok = lane == 0 || (lane < (1 << width) && c >= K);
-            const unsigned bal = __ballot_sync(0xffffffffu, ok);   // counts fall with w: a lane prefix
-            const int best = 31 - __clz(bal);
-            const int cbest = __shfl_sync(0xffffffffu, c, best);
-            if (best > 0) res.count = cbest;
-            prefix |= (uint32_t)best << shift;
-            hi = shift;
-            buf ^= 1;
+    int kk = K;                                       // rank wanted among the keys matching prefix
+    while (hi > low_bit && res.count != K) {
+        const int width = hi - low_bit < 5 ? hi - low_bit : 5;
+        const int shift = hi - width;
+        const uint32_t himask = hi >= 32 ? 0u : 0xffffffffu << hi;
+        s_h[tid] = 0;
+        __syncthreads();
+        for (int i = tid; i < n; i += NT) {
+            const uint32_t k = key[i];
+            if ((k & himask) == prefix) atomicAdd(&s_h[(((k >> shift) & ((1u << width) - 1u)) << 5) + lane], 1);
         }
-    } else {
-        if (((hi - low_bit) & 1) && hi < 32) ++hi;     // whole 2-bit fields; a common bit re-enters
-        if (hi > 32) hi = 32;
-        prefix = hi >= 32 ? 0u : (kmax >> hi) << hi;
-        for (int bit = hi - 2; bit >= low_bit && res.count != K; bit -= 2) {
-            const uint32_t c1 = prefix | (1u << bit), c2 = prefix | (2u << bit), c3 = prefix | (3u << bit);
-            int n12 = 0, n3 = 0;
-            for (int i = tid; i < n; i += NT) {
-                const uint32_t k = key[i];
-                n12 += (k >= c1) + ((k >= c2) << 16);
-                n3 += k >= c3;
-            }
-            n12 = __reduce_add_sync(0xffffffffu, n12);
-            n3 = __reduce_add_sync(0xffffffffu, n3);
-            int* slot = s_cnt + buf * 2 * NW;
-            if (lane == 0) { slot[2 * warp] = n12; slot[2 * warp + 1] = n3; }
-            __syncthreads();
-            int t12 = lane < NW ? slot[2 * lane] : 0, t3 = lane < NW ? slot[2 * lane + 1] : 0;
-            t12 = __reduce_add_sync(0xffffffffu, t12);
-            t3 = __reduce_add_sync(0xffffffffu, t3);
-            if (t3 >= K) { prefix = c3; res.count = t3; }
-            else if ((t12 >> 16) >= K) { prefix = c2; res.count = t12 >> 16; }
-            else if ((t12 & 0xffff) >= K) { prefix = c1; res.count = t12 & 0xffff; }
-            buf ^= 1;
+        __syncthreads();
+        const int tot = __reduce_add_sync(0xffffffffu, s_h[(warp << 5) + lane]);   // digit `warp`
+        if (lane == 0) s_tot[warp] = tot;
+        __syncthreads();
+        const int c = s_tot[31 - lane];               // lane l looks at digit 31 - l: descending
+        int inc = c;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int t = __shfl_up_sync(0xffffffffu, inc, o);
+            if (lane >= o) inc += t;
         }
+        const int above = inc - c;
+        const unsigned bal = __ballot_sync(0xffffffffu, above < kk && kk <= above + c);
+        const int sel = __ffs(bal) - 1;
+        const int above_sel = __shfl_sync(0xffffffffu, above, sel);
+        const int c_sel = __shfl_sync(0xffffffffu, c, sel);
+        prefix |= (uint32_t)(31 - sel) << shift;
+        kk -= above_sel;
+        res.count = (K - kk) + c_sel;                 // keys >= the new prefix
+        hi = shift;
     }
-    __syncthreads();
     res.v = prefix;
+    res.need = kk;
     return res;
-}
-
-// Number of key[0..n) strictly greater than v (block-wide, every thread gets it).
-template <int NT>
-__device__ int count_greater(const uint32_t* key, int n, uint32_t v, int* s_cnt) {
-    constexpr int NW = NT / 32;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    int c = 0;
-    for (int i = tid; i < n; i += NT) c += key[i] > v;
-    c = __reduce_add_sync(0xffffffffu, c);
-    if (lane == 0) s_cnt[warp] = c;
-    __syncthreads();
-    int t = lane < NW ? s_cnt[lane] : 0;
-    t = __reduce_add_sync(0xffffffffu, t);
-    __syncthreads();
-    return t;
 }
 
 // Write, in source order, every element with key > v and the first need_eq elements with
@@ -373,7 +347,7 @@ __device__ int select_listed(const uint32_t* s_key, const int32_t* s_idx, int n,
         uint32_t vstar;
         int need_eq;
         if (t.count == K) { vstar = t.v - 1u; need_eq = 0; }            // exactly K keys are >= v
-        else { vstar = t.v; need_eq = K - count_greater<NT>(s_key, n, vstar, s_cnt); }   // v = K-th largest
+        else { vstar = t.v; need_eq = t.need; }                          // v = K-th largest key
         ordered_emit<NT>(src, n, vstar, need_eq, s_sup_idx, s_sup_key, s_ws);
         ns = K;
         kmax = t.kmax;
@@ -524,18 +498,19 @@ __global__ void __launch_bounds__(REUSE_THREADS, 1) reuse_kernel(const StepArgs 
     constexpr int NW = NT / 32;
     constexpr int LPR = D / 8, RPW = 32 / LPR, SLOTS = NW * RPW;
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    // layout (words): q[D] rho[M] sel[r] ws[32] misc[8] hist[256] sup_idx[K] sup_key[K] w[K]
+    // layout (words): q[D] qraw[D] rho[M] sel[r] ws[32] misc[8] hist[SCRATCH_WORDS] sup_idx[K] sup_key[K] w[K]
     //                 | big: idx[cap] key[cap], aliased later by red[NW*D+NT] | bitmap | stage[depth*NT*4]
     float* s_q = reinterpret_cast<float*>(smem_raw);
-    float* s_rho = s_q + D;
+    float* s_qraw = s_q + D;
+    float* s_rho = s_qraw + D;
     int* s_sel = reinterpret_cast<int*>(s_rho + a.M);
     int* s_ws = s_sel + a.r;
     int* s_misc = s_ws + 32;
     uint32_t* s_hist = reinterpret_cast<uint32_t*>(s_misc + 8);
-    int32_t* s_sup_idx = reinterpret_cast<int32_t*>(s_hist + 256);
+    int32_t* s_sup_idx = reinterpret_cast<int32_t*>(s_hist + SCRATCH_WORDS);
     uint32_t* s_sup_key = reinterpret_cast<uint32_t*>(s_sup_idx + a.K);
     float* s_w = reinterpret_cast<float*>(s_sup_key + a.K);
-    const int head_words = (D + a.M + a.r + 32 + 8 + 256 + 3 * a.K + 3) & ~3;
+    const int head_words = (2 * D + a.M + a.r + 32 + 8 + SCRATCH_WORDS + 3 * a.K + 3) & ~3;
     int32_t* s_idx = reinterpret_cast<int32_t*>(smem_raw) + head_words;
     uint32_t* s_key = reinterpret_cast<uint32_t*>(s_idx + a.cap);
     float* s_red = reinterpret_cast<float*>(s_idx);
@@ -584,7 +559,10 @@ __global__ void __launch_bounds__(REUSE_THREADS, 1) reuse_kernel(const StepArgs 
             inv_nrm = nrm > 0.f ? 1.f / nrm : 0.f;
             if (warp == 0 && lane < D / 4) {
 #pragma unroll
-                for (int e = 0; e < 4; ++e) s_q[4 * lane + e] = nrm > 0.f ? q4[e] / nrm : 0.f;
+                for (int e = 0; e < 4; ++e) {
+                    s_q[4 * lane + e] = nrm > 0.f ? q4[e] / nrm : 0.f;
+                    s_qraw[4 * lane + e] = q4[e];
+                }
             }
         }
 #pragma unroll
@@ -637,7 +615,7 @@ __global__ void __launch_bounds__(REUSE_THREADS, 1) reuse_kernel(const StepArgs 
             a.ws_path[bh] = (uint8_t)path;
             a.ws_rho[bh] = rho_max;
             a.ws_ncand[bh] = L;
-            a.counters[(size_t)bh * 4 + path] += 1;
+            atomicAdd(a.counters + (size_t)bh * 4 + path, 1ull);     // no return value: not waited for
         }
         return;
     }
@@ -691,8 +669,8 @@ __global__ void __launch_bounds__(REUSE_THREADS, 1) reuse_kernel(const StepArgs 
         a.ws_path[bh] = (uint8_t)path;
         a.ws_rho[bh] = rho_max;
         a.ws_ncand[bh] = n;
-        a.counters[(size_t)bh * 4 + PATH_REUSE] += 1;
-        a.counters[(size_t)bh * 4 + 3] += n;
+        atomicAdd(a.counters + (size_t)bh * 4 + PATH_REUSE, 1ull);
+        atomicAdd(a.counters + (size_t)bh * 4 + 3, (unsigned long long)n);
     }
     __syncthreads();
     RETOPK_PHASE(0, 5);
@@ -704,16 +682,20 @@ __global__ void __launch_bounds__(REUSE_THREADS, 1) reuse_kernel(const StepArgs 
         const int sub = lane % LPR, myslot = warp * RPW + lane / LPR;
         const char* ksrc = reinterpret_cast<const char*>(a.k + (size_t)bkv * a.max_seq_len * D) + sub * 16;
         float qf[8];
-        unpack8(*reinterpret_cast<const uint4*>(a.q + (size_t)bh * D + sub * 8), qf);
+        *reinterpret_cast<float4*>(qf) = *reinterpret_cast<const float4*>(s_qraw + sub * 8);
+        *reinterpret_cast<float4*>(qf + 4) = *reinterpret_cast<const float4*>(s_qraw + sub * 8 + 4);
         const int depth = a.stage_depth;
         uint4* my_stage = s_stage + tid;
+        RETOPK_PHASE(0, 9);
         for (int base = 0; base < n; base += SLOTS * depth) {
             for (int u = 0; u < depth; ++u) {
                 const int i = base + u * SLOTS + myslot;
                 if (i < n) cp_async16(my_stage + u * NT, ksrc + (size_t)s_idx[i] * (D * 2));
             }
             cp_async_commit();
+            RETOPK_PHASE(0, 10);
             cp_async_wait_all();
+            RETOPK_PHASE(0, 11);
             for (int u0 = 0; u0 < depth; u0 += 8) {
                 float part[8];
 #pragma unroll
@@ -727,6 +709,7 @@ __global__ void __launch_bounds__(REUSE_THREADS, 1) reuse_kernel(const StepArgs 
                 if ((LPR == 8 || (sub & 1) == 0) && u0 + row < depth && i < n) s_key[i] = score_key(tot * a.scale);
             }
         }
+        RETOPK_PHASE(0, 12);
     }
     __syncthreads();
     RETOPK_PHASE(0, 6);
@@ -773,6 +756,8 @@ __global__ void __launch_bounds__(SCAN_THREADS) scan_kernel(const StepArgs a) {
     const int g = lane >> 2, t = lane & 3;
     const int G = a.G, L = a.L;
     const int n_groups = a.B * a.Hkv;
+    // No trigger for the dependent launch behind this kernel: its CTAs take a whole SM each
+    // and start as this kernel's CTAs exit; that already hides its launch latency.
 
     // the groups to scan, in ascending order (all of them for Exact Top-K attention)
     int n_act = 0;
@@ -893,11 +878,12 @@ template <int D>
 __global__ void __launch_bounds__(EXACT_THREADS, 1) exact_finish_kernel(const StepArgs a) {
     constexpr int NT = EXACT_THREADS;
     const int bh = blockIdx.x;
+    pdl_wait();        // scores and tile maxima come from the scan, path flags from the step's first kernel
     if (a.mode == MODE_RETOPK && a.ws_path[bh] == PATH_REUSE) return;
 
     extern __shared__ __align__(16) unsigned char smem_raw[];
     // layout (words): key[NS] idx[NS] (aliased later by red[NW*D+NT]) tile[NS/2]
-    //                 sup_idx[K] sup_key[K] w[K] cnt[256] ws[32] misc[8] stage[depth*NT*4]
+    //                 sup_idx[K] sup_key[K] w[K] cnt[SCRATCH_WORDS] ws[32] misc[8] stage[depth*NT*4]
     uint32_t* s_key = reinterpret_cast<uint32_t*>(smem_raw);
     int32_t* s_idx = reinterpret_cast<int32_t*>(s_key + a.NS);
     float* s_red = reinterpret_cast<float*>(smem_raw);
@@ -906,11 +892,11 @@ __global__ void __launch_bounds__(EXACT_THREADS, 1) exact_finish_kernel(const St
     uint32_t* s_sup_key = reinterpret_cast<uint32_t*>(s_sup_idx + a.K);
     float* s_w = reinterpret_cast<float*>(s_sup_key + a.K);
     uint32_t* s_hist = reinterpret_cast<uint32_t*>(s_w + a.K);
-    int* s_ws = reinterpret_cast<int*>(s_hist + 256);
+    int* s_ws = reinterpret_cast<int*>(s_hist + SCRATCH_WORDS);
     int* s_misc = s_ws + 32;
     // landing zone of the value-row copies, on a 16-byte boundary
     uint4* s_stage = reinterpret_cast<uint4*>(
-        reinterpret_cast<uint32_t*>(smem_raw) + ((2 * a.NS + a.NS / 2 + 3 * a.K + 256 + 32 + 8 + 3) & ~3));
+        reinterpret_cast<uint32_t*>(smem_raw) + ((2 * a.NS + a.NS / 2 + 3 * a.K + SCRATCH_WORDS + 32 + 8 + 3) & ~3));
 
     const int tid = threadIdx.x;
     const int b = bh / a.Hq, h = bh % a.Hq;
@@ -1043,7 +1029,7 @@ __global__ void __launch_bounds__(EXACT_THREADS, 1) exact_finish_kernel(const St
 }
 
 // Clear the caches (supports to -1, queries and counters to 0).
-__global__ void reset_kernel(float* qbar, size_t n_q, int32_t* sup, size_t n_sup, long long* counters,
+__global__ void reset_kernel(float* qbar, size_t n_q, int32_t* sup, size_t n_sup, unsigned long long* counters,
                              size_t n_cnt, int32_t* gflag, size_t n_flag, unsigned int* status,
                              unsigned long long* slow, unsigned long long* groups) {
     const size_t stride = (size_t)gridDim.x * blockDim.x;
