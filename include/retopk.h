@@ -49,7 +49,8 @@ enum {
     RETOPK_EINVAL = -1,      /* bad argument (null pointer, size out of range) */
     RETOPK_EUNSUPPORTED = -2,/* legal but not built (d not 64/128, H_q/H_kv > 16, ...) */
     RETOPK_ENOMEM = -3,      /* device allocation failed in create */
-    RETOPK_ECUDA = -4        /* a CUDA runtime call or launch failed */
+    RETOPK_ECUDA = -4,       /* a CUDA runtime call or launch failed */
+    RETOPK_ETOOLARGE = -5    /* the shape does not fit the fixed scratch of exact_topk_decode_static */
 };
 
 enum { RETOPK_PATH_REUSE = 0, RETOPK_PATH_FALLBACK = 1, RETOPK_PATH_REFRESH = 2 };
@@ -150,6 +151,37 @@ int retopk_export_state(retopk_ctx* ctx, float* qbar, int32_t* supports, int64_t
                         int64_t* t_dec, void* stream);
 int retopk_import_state(retopk_ctx* ctx, const float* qbar, const int32_t* supports,
                         int64_t n_inserted, int64_t t_dec, void* stream);
+
+/*
+ * Exact Top-K attention without a context and without any allocation (the paper has no
+ * counterpart: this entry point exists for callers that must not allocate device memory).
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits - inside a region whose memory
+ * is fully owned by another allocator (an inference server's arena, a framework's caching
+ * allocator that forbids raw allocations), while a stream capture is being recorded, or
+ * in a plug-in that is only handed input and output buffers.  retopk_create allocates the
+ * score workspace with cudaMalloc; this call instead keeps its workspace in a fixed array
+ * that is part of the library image (RETOPK_STATIC_SCRATCH_BYTES of device memory on every
+ * GPU that loads the library, held until the process exits).
+ *
+ * Same computation and same results as exact_topk_decode (Eq. 4, Eq. 1, Eq. 12) for
+ * q [B,H_q,d], k_cache / v_cache [B,H_kv,max_seq_len,d] -> out [B,H_q,d], idx_out [B,H_q,K]
+ * or NULL; all device pointers, caller-owned.  Constraints as for retopk_create_batched.
+ * The workspace holds B * H_q rows of max_seq_len scores plus their tile maxima, so
+ *     B * H_q * (ceil16(max_seq_len) + ceil4(ceil(max_seq_len / 16))) * 4 + 256
+ * must not exceed RETOPK_STATIC_SCRATCH_BYTES; larger shapes return RETOPK_ETOOLARGE and
+ * nothing is launched.
+ *
+ * The first call on a device looks up the array's device address and opts the kernels in to
+ * large shared memory; make that first call outside any stream capture.  No call allocates,
+ * frees or synchronises.  All calls on a device share the one array: its contents are
+ * rewritten by every call before they are read (nothing needs to start at zero), and two
+ * calls that overlap on the GPU (different streams, no dependency) race on it.
+ */
+#define RETOPK_STATIC_SCRATCH_BYTES (32u << 20)
+int exact_topk_decode_static(int B, int H_q, int H_kv, int d, int K, int64_t max_seq_len, const void* q,
+                             const void* k_cache, const void* v_cache, int64_t seq_len, void* out,
+                             int32_t* idx_out, void* stream);
 
 /*
  * Measurement hooks (no counterpart in the paper).  Between begin and end, every decode

@@ -460,6 +460,125 @@ int retopk_profile_end(retopk_ctx* c, double ms_host[3], int64_t launches_host[3
 
 int retopk_last_launch_count(const retopk_ctx* c) { return c ? c->last_launches : 0; }
 
+// ---------------------------------------------------------------------------------------
+// Exact Top-K attention for callers that may not allocate.
+//
+// The score workspace lives in this fixed array instead of cudaMalloc'ed memory.  In host
+// code the name `g_static_scratch` is only a handle for the runtime, not a device address:
+// the address every kernel gets is looked up once per device with cudaGetSymbolAddress
+// while that device is current.
+// ---------------------------------------------------------------------------------------
+static __device__ __align__(256) unsigned char g_static_scratch[RETOPK_STATIC_SCRATCH_BYTES];
+
+namespace {
+constexpr int STATIC_MAX_DEVICES = 64;
+struct StaticSetup {
+    bool ready;
+    unsigned char* scratch;      // device address of g_static_scratch on this device
+    int num_sms, max_smem;
+    int occ[2][2];               // scan CTAs per SM for d in {64,128} x head tiles in {1,2}
+};
+StaticSetup g_static_setup[STATIC_MAX_DEVICES];
+
+// First use on the current device: resolve the array's address, opt in to large shared memory.
+int static_setup(int dev, StaticSetup** out) {
+    if (dev < 0 || dev >= STATIC_MAX_DEVICES) return RETOPK_EUNSUPPORTED;
+    StaticSetup* st = &g_static_setup[dev];
+    if (!st->ready) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) { cudaGetLastError(); return RETOPK_ECUDA; }
+        st->scratch = static_cast<unsigned char*>(p);
+        if (cudaDeviceGetAttribute(&st->num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&st->max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess)
+            return RETOPK_ECUDA;
+        if (cudaFuncSetAttribute(exact_finish_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, st->max_smem) != cudaSuccess ||
+            cudaFuncSetAttribute(exact_finish_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, st->max_smem) != cudaSuccess)
+            return RETOPK_ECUDA;
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&st->occ[0][0], scan_kernel<64, 1>, SCAN_THREADS, 0);
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&st->occ[0][1], scan_kernel<64, 2>, SCAN_THREADS, 0);
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&st->occ[1][0], scan_kernel<128, 1>, SCAN_THREADS, 0);
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&st->occ[1][1], scan_kernel<128, 2>, SCAN_THREADS, 0);
+        st->ready = true;
+    }
+    *out = st;
+    return RETOPK_OK;
+}
+}  // namespace
+
+int exact_topk_decode_static(int B, int H_q, int H_kv, int d, int K, int64_t max_seq_len, const void* q,
+                             const void* k_cache, const void* v_cache, int64_t seq_len, void* out,
+                             int32_t* idx_out, void* stream) {
+    if (!q || !k_cache || !v_cache || !out) return RETOPK_EINVAL;
+    if (B < 1 || H_q < 1 || H_kv < 1 || H_q % H_kv != 0 || K < 1 || max_seq_len < 1 || seq_len < 1 ||
+        seq_len > max_seq_len)
+        return RETOPK_EINVAL;
+    if ((d != 64 && d != 128) || H_q / H_kv > 16 || K > 4096 || max_seq_len > 1048576 ||
+        (long long)B * H_kv > MAX_GROUPS)
+        return RETOPK_EUNSUPPORTED;
+    if (!aligned16(q) || !aligned16(k_cache) || !aligned16(v_cache)) return RETOPK_EINVAL;
+
+    // does the shape fit the fixed array?  (256 bytes of counters, then scores, then tile maxima)
+    const long long nh = (long long)B * H_q;
+    const long long score_stride = (max_seq_len + TILE_ROWS - 1) / TILE_ROWS * TILE_ROWS;
+    const long long tmax_stride = ((max_seq_len + TILE_ROWS - 1) / TILE_ROWS + 3) / 4 * 4;
+    const long long need = 256 + nh * (score_stride + tmax_stride) * 4;
+    if (need > (long long)RETOPK_STATIC_SCRATCH_BYTES) return RETOPK_ETOOLARGE;
+
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return RETOPK_ECUDA;
+    StaticSetup* st = nullptr;
+    int rc = static_setup(dev, &st);
+    if (rc != RETOPK_OK) return rc;
+
+    const int NS = 16 * K <= 8192 ? 8192 : 16384;
+    size_t smem = (((size_t)NS * 2 + (size_t)NS / 2 + (size_t)K * 3 + SCRATCH_WORDS + 32 + 8 + 3) & ~(size_t)3) * 4;
+    const size_t wave = (size_t)EXACT_THREADS * 16;
+    if ((size_t)st->max_smem < smem + wave) return RETOPK_EUNSUPPORTED;
+    const int slots = EXACT_THREADS / (d / 8);
+    long long depth = (long long)(((size_t)st->max_smem - smem) / wave);
+    const long long want = (K + slots - 1) / slots;
+    if (depth > want) depth = want;
+    if (depth > 16) depth = 16;
+    smem += (size_t)depth * wave;
+
+    StepArgs a;
+    memset(&a, 0, sizeof a);
+    a.B = B; a.Hq = H_q; a.Hkv = H_kv; a.G = H_q / H_kv; a.d = d; a.M = 1; a.r = 1; a.W = 0; a.K = K; a.cap = K;
+    a.max_seq_len = max_seq_len;
+    a.score_stride = score_stride;
+    a.tmax_stride = tmax_stride;
+    a.L = (int)seq_len;
+    a.scale = 1.0f / sqrtf((float)d);
+    a.mode = MODE_EXACT;
+    a.NS = NS;
+    a.exact_stage_depth = (int)depth;
+    a.q = static_cast<const uint16_t*>(q);
+    a.k = static_cast<const uint16_t*>(k_cache);
+    a.v = static_cast<const uint16_t*>(v_cache);
+    a.out = static_cast<uint16_t*>(out);
+    a.idx_out = idx_out;
+    // the two diagnostic counters the kernels add to are sinks here; they need no clearing
+    a.slow_select = reinterpret_cast<unsigned long long*>(st->scratch);
+    a.scan_groups = reinterpret_cast<unsigned long long*>(st->scratch + 8);
+    a.ws_scores = reinterpret_cast<float*>(st->scratch + 256);
+    a.ws_tmax = a.ws_scores + nh * score_stride;
+
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int ntile = (a.G + 7) / 8;
+    const int occ = st->occ[d == 128][ntile - 1];
+    const long long items = (long long)B * H_kv * ((a.L + SCAN_TILE_ROWS - 1) / SCAN_TILE_ROWS);
+    const long long cap_grid = (long long)st->num_sms * (occ > 0 ? occ : 2);
+    const unsigned grid = (unsigned)(items < cap_grid ? items : cap_grid);
+    if (d == 128 && ntile == 1) scan_kernel<128, 1><<<grid, SCAN_THREADS, 0, s>>>(a);
+    else if (d == 128) scan_kernel<128, 2><<<grid, SCAN_THREADS, 0, s>>>(a);
+    else if (ntile == 1) scan_kernel<64, 1><<<grid, SCAN_THREADS, 0, s>>>(a);
+    else scan_kernel<64, 2><<<grid, SCAN_THREADS, 0, s>>>(a);
+    if (cudaGetLastError() != cudaSuccess) return RETOPK_ECUDA;
+    if (d == 128) exact_finish_kernel<128><<<(unsigned)nh, EXACT_THREADS, smem, s>>>(a);
+    else exact_finish_kernel<64><<<(unsigned)nh, EXACT_THREADS, smem, s>>>(a);
+    return cudaGetLastError() == cudaSuccess ? RETOPK_OK : RETOPK_ECUDA;
+}
+
 #ifdef RETOPK_PHASE_CLOCKS
 // Development aid (not part of the public interface): copy the phase clock table to the host.
 int retopk_debug_read_phases(long long* host) {
@@ -475,6 +594,7 @@ const char* retopk_strerror(int code) {
         case RETOPK_EUNSUPPORTED: return "configuration not supported by this build";
         case RETOPK_ENOMEM: return "device memory allocation failed";
         case RETOPK_ECUDA: return "CUDA runtime call or kernel launch failed";
+        case RETOPK_ETOOLARGE: return "shape exceeds the fixed scratch array of exact_topk_decode_static";
         default: return "unknown error";
     }
 }

@@ -41,6 +41,7 @@ SIGNATURES = {
     "retopk_decode_step": (_i32, [_vp, _vp, _vp, _vp, _i64, _vp, _vp]),
     "retopk_decode_step_host": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _i64, _vp, _vp]),
     "exact_topk_decode": (_i32, [_vp, _vp, _vp, _vp, _i64, _vp, _vp, _vp]),
+    "exact_topk_decode_static": (_i32, [_i32] * 5 + [_i64, _vp, _vp, _vp, _i64, _vp, _vp, _vp]),
     "retopk_stats": (_i32, [_vp, C.POINTER(_Stats)]),
     "retopk_last_step": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp]),
     "retopk_export_state": (_i32, [_vp, _vp, _vp, C.POINTER(_i64), C.POINTER(_i64), _vp]),
@@ -216,6 +217,33 @@ class ReTopK:
 
     def last_launch_count(self) -> int:
         return int(self.lib.retopk_last_launch_count(self.h))
+
+
+STATIC_SCRATCH_BYTES = 32 << 20
+
+
+def exact_topk_decode_static(q, k_cache, v_cache, seq_len, K, out=None, idx_out=None):
+    """Exact Top-K attention through the entry point that allocates nothing.
+
+    For callers that cannot call cudaMalloc (memory owned by another allocator, plug-ins that
+    only get buffers): the library's score workspace is a fixed array inside the library
+    instead of context memory, so the shape must fit ``STATIC_SCRATCH_BYTES``.  ``out`` and
+    ``idx_out`` should be passed in by such callers; they are only created here for
+    convenience when omitted.
+    """
+    bf = torch.bfloat16
+    B, H_q, d = q.shape
+    _, H_kv, max_seq_len, _ = k_cache.shape
+    if out is None:
+        out = torch.empty((B, H_q, d), dtype=bf, device=q.device)
+    idx_ptr = None if idx_out is None else _dev(idx_out, torch.int32, (B, H_q, K))
+    with torch.cuda.device(q.device):
+        rc = load().exact_topk_decode_static(
+            B, H_q, H_kv, d, K, max_seq_len, _dev(q, bf), _dev(k_cache, bf, (B, H_kv, max_seq_len, d)),
+            _dev(v_cache, bf, (B, H_kv, max_seq_len, d)), seq_len, _dev(out, bf, (B, H_q, d)), idx_ptr,
+            _stream())
+    _check(rc, "exact_topk_decode_static")
+    return out
 
 
 def bf16_tensor_from_bits(bits, device=None, pin=False) -> torch.Tensor:
