@@ -196,11 +196,8 @@ def timed_pass(layers, kind, warmup, steps, torch, dist, profile=False, sampler=
     sync_all(torch, dist)
     if sampler is not None:
         sampler.__exit__(None, None, None)
-    ms = e0.elapsed_time(e1)
-    if dist is not None:
-        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    from paper_2607_27692_b200 import replicas
+    ms = replicas.max_over_ranks(e0.elapsed_time(e1), dist, "cuda")
     prof = None
     if profile:
         prof = {}
@@ -253,14 +250,10 @@ def run_gpu(args):
     import torch
     from paper_2607_27692_b200 import build, retopk as rt
     build.build()
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    from paper_2607_27692_b200 import replicas
+    rank, world, local = replicas.rank_info()
     torch.cuda.set_device(local)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    dist = replicas.init("nccl", torch.device("cuda", local))
     cfg = wl.CONFIGS[args.config]
     W, K = args.warmup, args.steps
     n_layers = args.layers
@@ -321,7 +314,7 @@ def run_gpu(args):
     qbytes = cfg.B * cfg.H_q * cfg.d * 2
     kvbytes = 2 * cfg.B * cfg.H_kv * cfg.d * 2
     line = {
-        "metric": METRIC, "value": round(head["us_per_step"] / world, 3), "unit": UNIT, "n_gpus": world,
+        "metric": METRIC, "value": round(replicas.job_cost_per_step(head["us_per_step"], world), 3), "unit": UNIT, "n_gpus": world,
         "steps": K, "warmup": W, "ms_per_step": round(head["ms"] / K, 6), "higher_is_better": False,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": cfg.name, "B": cfg.B, "H_q": cfg.H_q, "H_kv": cfg.H_kv, "d": cfg.d,
@@ -330,7 +323,7 @@ def run_gpu(args):
                    "l2": "inputs larger than L2: calls rotate over independent layers",
                    "parallelism": "replicas only" if world > 1 else "single GPU"},
         "clocks": sampler.summary(),
-        "e2e": {"value": round(e2e["us_per_step"] / world, 3), "unit": UNIT,
+        "e2e": {"value": round(replicas.job_cost_per_step(e2e["us_per_step"], world), 3), "unit": UNIT,
                 "h2d_bytes_per_step": qbytes + kvbytes, "d2h_bytes_per_step": qbytes},
         "gpu_launches": head["launches"],
         "path_mix": path_mix(head["stats"]),

@@ -41,6 +41,10 @@
  * left-to-right fp64 loop; selection is a full sort.  OpenMP only spreads independent
  * (sequence, head) pairs over threads.
  *
+ * Parity unpinned by the paper (fixed only by this file's readings, which the hand trace and
+ * the integer-tie tests pin): the tie-breaks of Top-r and Top-K, and whether the first decode
+ * step has offset 0 or 1 for the refresh schedule.
+ *
  * Pins (tests/test_oracle_pins.py): brute-force selection on small inputs, dense softmax
  * attention when K >= L, closed forms for K = 1 and K = 2, exact-path equality when
  * tau > 1 or W >= L, the hand-enumerated six-step trace in tests/golden, counter

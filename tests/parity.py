@@ -40,12 +40,13 @@ def assert_support_matches(sup_gpu, sup_ref, q_bits, k_head_bits, kth_score, wha
     return len(diff)
 
 
-def teacher_forced_run(cfg, st, steps, oracle, gpu, k_dev, v_dev, b_map=None, check_out=True):
+def teacher_forced_run(cfg, st, steps, oracle, gpu, k_dev, v_dev, b_map=None, check_out=True,
+                       full_stream=None):
     """Step both sides with the GPU caches re-seeded from the oracle before every step.
 
     ``oracle`` may cover a subset of the GPU's sequences: ``b_map[i]`` is the GPU batch row of
-    oracle row ``i`` (the stream ``st`` then holds the oracle's rows).
-    Returns counts of excused events.
+    oracle row ``i`` (the stream ``st`` then holds the oracle's rows, ``full_stream`` the
+    queries of every GPU sequence).  Returns counts of excused events.
     """
     G = cfg.H_q // cfg.H_kv
     b_map = list(range(oracle.B)) if b_map is None else b_map
@@ -66,6 +67,8 @@ def teacher_forced_run(cfg, st, steps, oracle, gpu, k_dev, v_dev, b_map=None, ch
         gpu.import_state(gq, gs, n_ins, t_dec)
         if full:
             q_dev = to_dev(st.q[t])
+        elif full_stream is not None:
+            q_dev = to_dev(full_stream.q[t])
         else:
             q_full = torch.zeros(gpu.q_shape, dtype=torch.bfloat16, device="cuda") if q_full is None else q_full
             q_full[torch.tensor(b_map, device="cuda")] = to_dev(st.q[t])
