@@ -298,7 +298,10 @@ def run_gpu(args):
     roofline = {"bound": "hbm", "kernel": top + "_kernel", "achieved": kernels[top]["GBps"], "peak": peak,
                 "peak_kind": peak_kind, "unit": "GB/s", "frac": kernels[top]["frac"],
                 "frac_of_8TBps": round(kernels[top]["GBps"] / 8000.0, 4),
-                "traffic": NCU_TRAFFIC.get((args.config, top)), "kernels": kernels}
+                "traffic": (int(NCU_TRAFFIC_PER_GROUP[args.config] * prof["stats"]["scan_groups"] / prof["prof"]["scan"]["launches"])
+                            if top == "scan" and args.config in NCU_TRAFFIC_PER_GROUP else None),
+                "traffic_source": "profiles/scan_kernel_headline128k_single_layer.md, scaled by scanned groups per launch",
+                "kernels": kernels}
 
     def path_report(res, exact_like):
         st = res["stats"]
@@ -349,9 +352,11 @@ def run_gpu(args):
         dist.destroy_process_group()
 
 
-# Per-launch DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu
-# captures summarised under profiles/; filled in when a capture of that workload exists.
-NCU_TRAFFIC = {}
+# DRAM traffic of scan_kernel per scanned KV group (dram__bytes_read.sum + dram__bytes_write.sum
+# of one launch over its 32 groups) from the ncu capture summarised in
+# profiles/scan_kernel_headline128k_single_layer.md; a launch's traffic is this times the
+# groups it scanned (traffic grows in proportion to the rows streamed).
+NCU_TRAFFIC_PER_GROUP = {"headline128k": 34.29e6}
 
 
 # --------------------------------------------------------------------------- reference arm
