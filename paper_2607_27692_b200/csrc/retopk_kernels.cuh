@@ -43,7 +43,7 @@ constexpr int EXACT_THREADS = 1024;
 constexpr int SCAN_THREADS = 256;
 constexpr int SCAN_TILE_ROWS = 256;  // key rows per scan work item
 constexpr int MAX_GROUPS = 4096;     // B * H_kv limit (shared list in scan_kernel)
-constexpr int SCRATCH_WORDS = 1056;  // histogram scratch of the threshold search (32 x 32 + 32)
+constexpr int SCRATCH_WORDS = 2144;  // scratch of the threshold search (2 x 32 x 32 + 96)
 constexpr int TILE_ROWS = 16;        // rows per score tile whose maximum the scan records
 
 struct StepArgs {
@@ -237,7 +237,7 @@ __device__ void radix_select(const Src& src, int n, int K, uint32_t* s_hist, int
 //   count  > K : v is the largest multiple with >= K keys at or above it; for low_bit 0 it
 //                is the K-th largest key itself and `need` of the keys equal to it belong
 //                to the top K.
-// s_h: 1024 + 32 ints.  Every thread returns the same result; kmax = largest key.
+// s_h: SCRATCH_WORDS ints.  Every thread returns the same result; kmax = largest key.
 struct Threshold {
     uint32_t v;
     int count;
@@ -249,38 +249,40 @@ template <int NT>
 __device__ Threshold count_threshold(const uint32_t* key, int n, int K, int low_bit, int* s_h) {
     static_assert(NT == 1024, "one histogram word per thread, one digit per warp");
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    int* s_tot = s_h + 1024;
+    // scratch: two histograms of 32 x 32 words used alternately, then 96 words of totals
+    int* s_tot = s_h + 2048;
     // common leading bits of all keys
     uint32_t kmin = 0xffffffffu, kmax = 0u;
     for (int i = tid; i < n; i += NT) { const uint32_t k = key[i]; kmin = min(kmin, k); kmax = max(kmax, k); }
     kmin = __reduce_min_sync(0xffffffffu, kmin);
     kmax = __reduce_max_sync(0xffffffffu, kmax);
-    if (lane == 0) { s_h[warp] = (int)kmin; s_h[32 + warp] = (int)kmax; }
+    if (lane == 0) { s_tot[warp] = (int)kmin; s_tot[32 + warp] = (int)kmax; }
+    s_h[tid] = 0;
+    s_h[1024 + tid] = 0;
     __syncthreads();
-    kmin = __reduce_min_sync(0xffffffffu, (uint32_t)s_h[lane]);
-    kmax = __reduce_max_sync(0xffffffffu, (uint32_t)s_h[32 + lane]);
-    __syncthreads();
+    kmin = __reduce_min_sync(0xffffffffu, (uint32_t)s_tot[lane]);
+    kmax = __reduce_max_sync(0xffffffffu, (uint32_t)s_tot[32 + lane]);
     Threshold res;
     res.kmax = kmax;
     res.count = n;
     int hi = 32 - __clz(kmin ^ kmax);                 // bits [hi-1:0] may differ
     uint32_t prefix = hi >= 32 ? 0u : (kmax >> hi) << hi;
     int kk = K;                                       // rank wanted among the keys matching prefix
+    int* hist = s_h;
     while (hi > low_bit && res.count != K) {
         const int width = hi - low_bit < 5 ? hi - low_bit : 5;
         const int shift = hi - width;
         const uint32_t himask = hi >= 32 ? 0u : 0xffffffffu << hi;
-        s_h[tid] = 0;
-        __syncthreads();
         for (int i = tid; i < n; i += NT) {
             const uint32_t k = key[i];
-            if ((k & himask) == prefix) atomicAdd(&s_h[(((k >> shift) & ((1u << width) - 1u)) << 5) + lane], 1);
+            if ((k & himask) == prefix) atomicAdd(&hist[(((k >> shift) & ((1u << width) - 1u)) << 5) + lane], 1);
         }
         __syncthreads();
-        const int tot = __reduce_add_sync(0xffffffffu, s_h[(warp << 5) + lane]);   // digit `warp`
-        if (lane == 0) s_tot[warp] = tot;
+        const int tot = __reduce_add_sync(0xffffffffu, hist[(warp << 5) + lane]);   // digit `warp`
+        hist[tid] = 0;                                // ready for the round after next
+        if (lane == 0) s_tot[64 + warp] = tot;
         __syncthreads();
-        const int c = s_tot[31 - lane];               // lane l looks at digit 31 - l: descending
+        const int c = s_tot[64 + 31 - lane];          // lane l looks at digit 31 - l: descending
         int inc = c;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
@@ -296,7 +298,9 @@ __device__ Threshold count_threshold(const uint32_t* key, int n, int K, int low_
         kk -= above_sel;
         res.count = (K - kk) + c_sel;                 // keys >= the new prefix
         hi = shift;
+        hist = (hist == s_h) ? s_h + 1024 : s_h;
     }
+    __syncthreads();
     res.v = prefix;
     res.need = kk;
     return res;
@@ -344,11 +348,13 @@ __device__ int select_listed(const uint32_t* s_key, const int32_t* s_idx, int n,
         SmemSrc src{s_key, s_idx};
         int* s_cnt = reinterpret_cast<int*>(s_hist);
         const Threshold t = count_threshold<NT>(s_key, n, K, 0, s_cnt);
+        RETOPK_PHASE(2, 6);
         uint32_t vstar;
         int need_eq;
         if (t.count == K) { vstar = t.v - 1u; need_eq = 0; }            // exactly K keys are >= v
         else { vstar = t.v; need_eq = t.need; }                          // v = K-th largest key
         ordered_emit<NT>(src, n, vstar, need_eq, s_sup_idx, s_sup_key, s_ws);
+        RETOPK_PHASE(2, 7);
         ns = K;
         kmax = t.kmax;
         kmax_known = true;
@@ -620,7 +626,10 @@ __global__ void __launch_bounds__(REUSE_THREADS, 1) reuse_kernel(const StepArgs 
         return;
     }
 
-    // Eq. 8-9: bitmap over key positions, then ordered extraction = sorted unique list
+    // Eq. 8-9: sorted unique candidate list.  Recalled indices below the window go through a
+    // bitmap over key positions (ordered extraction = sorted and deduplicated for free); the
+    // window itself is a contiguous run appended behind them, whatever the supports held there.
+    const int w_lo = L - a.W > 0 ? L - a.W : 0;
     {
         bool bad = false;
         const int E = n_sel * K;
@@ -638,24 +647,24 @@ __global__ void __launch_bounds__(REUSE_THREADS, 1) reuse_kernel(const StepArgs 
 #pragma unroll
             for (int u = 0; u < 4; ++u)
                 if (idx[u] >= 0) {
-                    if (idx[u] < L) atomicOr(&s_bm[idx[u] >> 5], 1u << (idx[u] & 31));
-                    else bad = true;
+                    if (idx[u] < w_lo) atomicOr(&s_bm[idx[u] >> 5], 1u << (idx[u] & 31));
+                    else if (idx[u] >= L) bad = true;
                 }
         }
-        const int w_lo = L - a.W > 0 ? L - a.W : 0;
-        for (int i = w_lo + tid; i < L; i += NT) atomicOr(&s_bm[i >> 5], 1u << (i & 31));
         if (bad) atomicOr(a.status, 1u);
     }
     __syncthreads();
     RETOPK_PHASE(0, 4);
     int n;
     {
-        const int wpt = (nwords + NT - 1) / NT;
+        const int nw_lo = (w_lo + 31) >> 5;               // words that can hold bits below the window
+        const int wpt = (nw_lo + NT - 1) / NT;
         const int w0 = tid * wpt;
-        const int w1 = (w0 + wpt < nwords) ? w0 + wpt : nwords;
+        const int w1 = (w0 + wpt < nw_lo) ? w0 + wpt : nw_lo;
         int cnt = 0;
         for (int w = w0; w < w1; ++w) cnt += __popc(s_bm[w]);
-        int pos = block_excl_scan<NT>(cnt, s_ws, n);
+        int n_low;
+        int pos = block_excl_scan<NT>(cnt, s_ws, n_low);
         for (int w = w0; w < w1; ++w) {
             uint32_t bits = s_bm[w];
             while (bits) {
@@ -664,13 +673,8 @@ __global__ void __launch_bounds__(REUSE_THREADS, 1) reuse_kernel(const StepArgs 
                 bits &= bits - 1;
             }
         }
-    }
-    if (tid == 0) {
-        a.ws_path[bh] = (uint8_t)path;
-        a.ws_rho[bh] = rho_max;
-        a.ws_ncand[bh] = n;
-        atomicAdd(a.counters + (size_t)bh * 4 + PATH_REUSE, 1ull);
-        atomicAdd(a.counters + (size_t)bh * 4 + 3, (unsigned long long)n);
+        for (int i = w_lo + tid; i < L; i += NT) s_idx[n_low + (i - w_lo)] = i;
+        n = n_low + (L - w_lo);
     }
     __syncthreads();
     RETOPK_PHASE(0, 5);
@@ -725,6 +729,13 @@ __global__ void __launch_bounds__(REUSE_THREADS, 1) reuse_kernel(const StepArgs 
     // Eq. 12 (s_red aliases the candidate lists, which are dead now)
     attend<D, NT>(a.v + (size_t)bkv * a.max_seq_len * D, ns, s_sup_idx, s_sup_key, s_w, s_red, s_ws, s_stage,
                   a.stage_depth, kmax, kmax_known, a.out + (size_t)bh * D);
+    if (tid == 0) {      // the step record is written last: nothing in this kernel waits for it
+        a.ws_path[bh] = (uint8_t)path;
+        a.ws_rho[bh] = rho_max;
+        a.ws_ncand[bh] = n;
+        atomicAdd(a.counters + (size_t)bh * 4 + PATH_REUSE, 1ull);
+        atomicAdd(a.counters + (size_t)bh * 4 + 3, (unsigned long long)n);
+    }
     RETOPK_PHASE(0, 8);
 }
 
@@ -920,42 +931,74 @@ __global__ void __launch_bounds__(EXACT_THREADS, 1) exact_finish_kernel(const St
         // 1. lower bound v for the K-th score from the tile maxima (grouped so the list is short)
         uint32_t thr_key = 0;
         int g2 = 1;
-        while ((ntile + g2 - 1) / g2 > 2048 && ntile / (2 * g2) >= 2 * K) g2 *= 2;
+        while ((ntile + g2 - 1) / g2 > 1024 && ntile / (2 * g2) >= 2 * K) g2 *= 2;
         while ((ntile + g2 - 1) / g2 > NS) g2 *= 2;
         const int n2 = (ntile + g2 - 1) / g2;
         if (n2 >= K) {
             for (int i2 = tid; i2 < n2; i2 += NT) {
                 const int t0 = i2 * g2;
-                float m = tm[t0];
-                for (int j = 1; j < g2 && t0 + j < ntile; ++j) m = fmaxf(m, tm[t0 + j]);
+                float m;
+                if (g2 >= 4) {
+                    // g2 is a power of two: whole float4 chunks, all requested before any is used
+                    m = -CUDART_INF_F;
+                    for (int c0 = 0; c0 < g2; c0 += 16) {
+                        float4 x[4];
+#pragma unroll
+                        for (int u = 0; u < 4; ++u)
+                            x[u] = (c0 + 4 * u < g2 && t0 + c0 + 4 * u < ntile)
+                                ? *reinterpret_cast<const float4*>(tm + t0 + c0 + 4 * u)
+                                : make_float4(-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F);
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            const int tt = t0 + c0 + 4 * u;
+                            m = fmaxf(m, x[u].x);
+                            if (tt + 1 < ntile) m = fmaxf(m, x[u].y);
+                            if (tt + 2 < ntile) m = fmaxf(m, x[u].z);
+                            if (tt + 3 < ntile) m = fmaxf(m, x[u].w);
+                        }
+                    }
+                } else {
+                    m = tm[t0];
+                    if (g2 == 2 && t0 + 1 < ntile) m = fmaxf(m, tm[t0 + 1]);
+                }
                 s_key[i2] = score_key(m);
             }
             __syncthreads();
-            thr_key = count_threshold<NT>(s_key, n2, K, 7, reinterpret_cast<int*>(s_hist)).v;
+            RETOPK_PHASE(2, 8);
+            thr_key = count_threshold<NT>(s_key, n2, K, 12, reinterpret_cast<int*>(s_hist)).v;
         }
         RETOPK_PHASE(2, 1);
-        // 2. the tiles whose maximum reaches v, in ascending order
+        // 2. the tiles whose maximum reaches v, in ascending order (two chunks of four tile
+        //    maxima per thread are requested before the first prefix sum)
         int nhit = 0;
-        for (int base = 0; base < ntile; base += NT * 4) {
-            const int t0 = base + tid * 4;
-            int f[4] = {0, 0, 0, 0}, cnt = 0;
-            if (t0 < ntile) {
-                const float4 m4 = *reinterpret_cast<const float4*>(tm + t0);
-                f[0] = score_key(m4.x) >= thr_key;
-                f[1] = (t0 + 1 < ntile) && score_key(m4.y) >= thr_key;
-                f[2] = (t0 + 2 < ntile) && score_key(m4.z) >= thr_key;
-                f[3] = (t0 + 3 < ntile) && score_key(m4.w) >= thr_key;
-                cnt = f[0] + f[1] + f[2] + f[3];
-            }
-            int total;
-            int pos = nhit + block_excl_scan<NT>(cnt, s_ws, total);
+        for (int base = 0; base < ntile; base += NT * 8) {
+            float4 m4[2];
 #pragma unroll
-            for (int e = 0; e < 4; ++e)
-                if (f[e]) {
-                    if (pos < tcap) s_tile[pos] = t0 + e;
-                    ++pos;
+            for (int u = 0; u < 2; ++u) {
+                const int t0 = base + u * NT * 4 + tid * 4;
+                m4[u] = t0 < ntile ? *reinterpret_cast<const float4*>(tm + t0) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+                const int t0 = base + u * NT * 4 + tid * 4;
+                int f[4] = {0, 0, 0, 0}, cnt = 0;
+                if (t0 < ntile) {
+                    f[0] = score_key(m4[u].x) >= thr_key;
+                    f[1] = (t0 + 1 < ntile) && score_key(m4[u].y) >= thr_key;
+                    f[2] = (t0 + 2 < ntile) && score_key(m4[u].z) >= thr_key;
+                    f[3] = (t0 + 3 < ntile) && score_key(m4[u].w) >= thr_key;
+                    cnt = f[0] + f[1] + f[2] + f[3];
                 }
-            nhit += total;
+                int total;
+                int pos = nhit + block_excl_scan<NT>(cnt, s_ws, total);
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                    if (f[e]) {
+                        if (pos < tcap) s_tile[pos] = t0 + e;
+                        ++pos;
+                    }
+                nhit += total;
+            }
         }
         __syncthreads();
         RETOPK_PHASE(2, 2);
