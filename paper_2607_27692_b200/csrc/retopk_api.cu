@@ -195,8 +195,8 @@ int retopk_create_batched(retopk_ctx** out, int B, int H_q, int H_kv, int d, int
 
     // shared-memory footprints (must mirror the carve-up at the top of each kernel)
     const size_t red_words = (size_t)(REUSE_THREADS / 32) * d + REUSE_THREADS;
-    const size_t head_words = ((size_t)2 * d + M + r + 32 + 8 + SCRATCH_WORDS + 4 * (size_t)K + 3) & ~(size_t)3;
-    const size_t big_words = ((size_t)c->cap + ((size_t)2 * c->cap > red_words ? (size_t)2 * c->cap : red_words) + 3) & ~(size_t)3;
+    const size_t head_words = ((size_t)2 * d + M + r + 32 + 8 + SCRATCH_WORDS + 3 * (size_t)K + 3) & ~(size_t)3;
+    const size_t big_words = (((size_t)2 * c->cap > red_words ? (size_t)2 * c->cap : red_words) + 3) & ~(size_t)3;
     const size_t bm_words = (((size_t)max_seq_len + 31) / 32 + 3) & ~(size_t)3;
     c->smem_reuse = (head_words + big_words + bm_words) * 4;
     c->smem_exact = (((size_t)c->NS * 2 + (size_t)c->NS / 2 + (size_t)K * 3 + SCRATCH_WORDS + 32 + 8 + 3) & ~(size_t)3) * 4;

@@ -115,6 +115,7 @@ __device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src)
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_but_one() { asm volatile("cp.async.wait_group 1;" ::: "memory"); }
 
 __device__ __forceinline__ float dot8(const uint4& x, const float* qf) {
     float a = bf16_lo(x.x) * qf[0];
@@ -311,7 +312,7 @@ __device__ Threshold count_threshold(const uint32_t* key, int n, int K, int low_
 // the support in ascending index order with ties resolved to the lower index.
 template <int NT, class Src>
 __device__ void ordered_emit(const Src& src, int n, uint32_t vstar, int need_eq, int32_t* s_sup_idx,
-                             uint32_t* s_sup_key, int* s_ws, int32_t* s_sup_src = nullptr) {
+                             uint32_t* s_sup_key, int* s_ws) {
     const int tid = threadIdx.x;
     int gt_run = 0, eq_run = 0;
     for (int base = 0; base < n; base += NT) {
@@ -326,7 +327,6 @@ __device__ void ordered_emit(const Src& src, int n, uint32_t vstar, int need_eq,
             const int pos = g_before + (e_before < need_eq ? e_before : need_eq);
             s_sup_idx[pos] = src.x(i);
             s_sup_key[pos] = key;
-            if (s_sup_src) s_sup_src[pos] = i;       // where in the list the winner sat
         }
         gt_run += total & 0xffff;
         eq_run += total >> 16;
@@ -338,14 +338,10 @@ __device__ void ordered_emit(const Src& src, int n, uint32_t vstar, int need_eq,
 template <int NT>
 __device__ int select_listed(const uint32_t* s_key, const int32_t* s_idx, int n, int K,
                              int32_t* s_sup_idx, uint32_t* s_sup_key, uint32_t* s_hist, int* s_ws,
-                             uint32_t& kmax, bool& kmax_known, int32_t* s_sup_src = nullptr) {
+                             uint32_t& kmax, bool& kmax_known) {
     int ns;
     if (n <= K) {
-        for (int i = threadIdx.x; i < n; i += NT) {
-            s_sup_idx[i] = s_idx[i];
-            s_sup_key[i] = s_key[i];
-            if (s_sup_src) s_sup_src[i] = i;
-        }
+        for (int i = threadIdx.x; i < n; i += NT) { s_sup_idx[i] = s_idx[i]; s_sup_key[i] = s_key[i]; }
         ns = n;
         kmax = 0;
         kmax_known = false;
@@ -358,7 +354,7 @@ __device__ int select_listed(const uint32_t* s_key, const int32_t* s_idx, int n,
         int need_eq;
         if (t.count == K) { vstar = t.v - 1u; need_eq = 0; }            // exactly K keys are >= v
         else { vstar = t.v; need_eq = t.need; }                          // v = K-th largest key
-        ordered_emit<NT>(src, n, vstar, need_eq, s_sup_idx, s_sup_key, s_ws, s_sup_src);
+        ordered_emit<NT>(src, n, vstar, need_eq, s_sup_idx, s_sup_key, s_ws);
         RETOPK_PHASE(2, 7);
         ns = K;
         kmax = t.kmax;
@@ -409,8 +405,7 @@ __device__ __forceinline__ float reduce8_across(const float* a, int sub, int& ro
 template <int D, int NT>
 __device__ void attend(const uint16_t* vbase, int ns, const int32_t* s_sup_idx, const uint32_t* s_sup_key,
                        float* s_w, float* s_red, int* s_ws, uint4* s_stage, int depth, uint32_t kmax,
-                       bool kmax_known, uint16_t* out_row, const int32_t* s_sup_src = nullptr,
-                       float* s_wc = nullptr, int n_listed = 0) {
+                       bool kmax_known, uint16_t* out_row) {
     constexpr int LPR = D / 8;                  // lanes per bf16 row (16 bytes each)
     constexpr int RPW = 32 / LPR;               // rows per warp load
     constexpr int SLOTS = (NT / 32) * RPW;      // row slots per block
@@ -428,11 +423,7 @@ __device__ void attend(const uint16_t* vbase, int ns, const int32_t* s_sup_idx, 
         }
         cp_async_commit();
     };
-    // n_listed > 0: the caller already requested the value rows of ALL n_listed candidates
-    // (row i into wave slot i / SLOTS of row slot i % SLOTS) while the selection ran; the
-    // weights are then scattered to candidate order (zero = not selected) in s_wc.
-    const bool ahead = n_listed > 0;
-    if (!ahead) issue(0);
+    issue(0);
 
     if (!kmax_known) {
         kmax = 0;
@@ -447,8 +438,7 @@ __device__ void attend(const uint16_t* vbase, int ns, const int32_t* s_sup_idx, 
     float wsum = 0.f;
     for (int i = tid; i < ns; i += NT) {
         const float w = expf(key_score(s_sup_key[i]) - smax);
-        if (ahead) s_wc[s_sup_src[i]] = w;
-        else s_w[i] = w;
+        s_w[i] = w;
         wsum += w;
     }
 #pragma unroll
@@ -462,19 +452,6 @@ __device__ void attend(const uint16_t* vbase, int ns, const int32_t* s_sup_idx, 
     float acc[8];
 #pragma unroll
     for (int e = 0; e < 8; ++e) acc[e] = 0.f;
-    if (ahead) {
-        cp_async_wait_all();
-        for (int u = 0; u < depth; ++u) {
-            const int i = u * SLOTS + myslot;
-            const float w = i < n_listed ? s_wc[i] : 0.f;
-            if (w != 0.f) {
-                float f[8];
-                unpack8(my_stage[u * NT], f);
-#pragma unroll
-                for (int e = 0; e < 8; ++e) acc[e] = fmaf(w, f[e], acc[e]);
-            }
-        }
-    } else
     for (int base = 0;;) {
         cp_async_wait_all();
         for (int u = 0; u < depth; ++u) {
@@ -529,8 +506,7 @@ __global__ void __launch_bounds__(REUSE_THREADS, 1) reuse_kernel(const StepArgs 
     constexpr int LPR = D / 8, RPW = 32 / LPR, SLOTS = NW * RPW;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     // layout (words): q[D] qraw[D] rho[M] sel[r] ws[32] misc[8] hist[SCRATCH_WORDS] sup_idx[K] sup_key[K] w[K]
-    //                 sup_src[K] | big: wc[cap] idx[cap] key[cap] (idx/key aliased later by red[NW*D+NT])
-    //                 | bitmap | stage[depth*NT*4]
+    //                 | big: idx[cap] key[cap], aliased later by red[NW*D+NT] | bitmap | stage[depth*NT*4]
     float* s_q = reinterpret_cast<float*>(smem_raw);
     float* s_qraw = s_q + D;
     float* s_rho = s_qraw + D;
@@ -541,14 +517,12 @@ __global__ void __launch_bounds__(REUSE_THREADS, 1) reuse_kernel(const StepArgs 
     int32_t* s_sup_idx = reinterpret_cast<int32_t*>(s_hist + SCRATCH_WORDS);
     uint32_t* s_sup_key = reinterpret_cast<uint32_t*>(s_sup_idx + a.K);
     float* s_w = reinterpret_cast<float*>(s_sup_key + a.K);
-    int32_t* s_sup_src = reinterpret_cast<int32_t*>(s_w + a.K);
-    const int head_words = (2 * D + a.M + a.r + 32 + 8 + SCRATCH_WORDS + 4 * a.K + 3) & ~3;
-    float* s_wc = reinterpret_cast<float*>(smem_raw) + head_words;          // [cap] weights in candidate order
-    int32_t* s_idx = reinterpret_cast<int32_t*>(s_wc + a.cap);
+    const int head_words = (2 * D + a.M + a.r + 32 + 8 + SCRATCH_WORDS + 3 * a.K + 3) & ~3;
+    int32_t* s_idx = reinterpret_cast<int32_t*>(smem_raw) + head_words;
     uint32_t* s_key = reinterpret_cast<uint32_t*>(s_idx + a.cap);
     float* s_red = reinterpret_cast<float*>(s_idx);
-    const int big_words = (a.cap + max(2 * a.cap, NW * D + NT) + 3) & ~3;
-    uint32_t* s_bm = reinterpret_cast<uint32_t*>(s_wc) + big_words;
+    const int big_words = (max(2 * a.cap, NW * D + NT) + 3) & ~3;
+    uint32_t* s_bm = reinterpret_cast<uint32_t*>(s_idx) + big_words;
     uint4* s_stage = reinterpret_cast<uint4*>(s_bm + ((((int)a.max_seq_len + 31) / 32 + 3) & ~3));
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -718,26 +692,34 @@ __global__ void __launch_bounds__(REUSE_THREADS, 1) reuse_kernel(const StepArgs 
         const int depth = a.stage_depth;
         uint4* my_stage = s_stage + tid;
         RETOPK_PHASE(0, 9);
+        // each wave goes out as two groups of copies, so that the dot products of the first
+        // half run while the second half is still arriving
+        const int half = (depth + 1) / 2;
         for (int base = 0; base < n; base += SLOTS * depth) {
             for (int u = 0; u < depth; ++u) {
                 const int i = base + u * SLOTS + myslot;
                 if (i < n) cp_async16(my_stage + u * NT, ksrc + (size_t)s_idx[i] * (D * 2));
+                if (u == half - 1) cp_async_commit();
             }
             cp_async_commit();
             RETOPK_PHASE(0, 10);
-            cp_async_wait_all();
-            RETOPK_PHASE(0, 11);
-            for (int u0 = 0; u0 < depth; u0 += 8) {
-                float part[8];
+            for (int g2 = 0; g2 < 2; ++g2) {
+                if (g2 == 0) cp_async_wait_but_one();
+                else cp_async_wait_all();
+                if (g2 == 0) RETOPK_PHASE(0, 11);
+                const int u_begin = g2 == 0 ? 0 : half, u_end = g2 == 0 ? half : depth;
+                for (int u0 = u_begin; u0 < u_end; u0 += 8) {
+                    float part[8];
 #pragma unroll
-                for (int uu = 0; uu < 8; ++uu) {
-                    const int i = base + (u0 + uu) * SLOTS + myslot;
-                    part[uu] = (u0 + uu < depth && i < n) ? dot8(my_stage[(u0 + uu) * NT], qf) : 0.f;
+                    for (int uu = 0; uu < 8; ++uu) {
+                        const int i = base + (u0 + uu) * SLOTS + myslot;
+                        part[uu] = (u0 + uu < u_end && i < n) ? dot8(my_stage[(u0 + uu) * NT], qf) : 0.f;
+                    }
+                    int row;
+                    const float tot = reduce8_across<LPR>(part, sub, row);
+                    const int i = base + (u0 + row) * SLOTS + myslot;
+                    if ((LPR == 8 || (sub & 1) == 0) && u0 + row < u_end && i < n) s_key[i] = score_key(tot * a.scale);
                 }
-                int row;
-                const float tot = reduce8_across<LPR>(part, sub, row);
-                const int i = base + (u0 + row) * SLOTS + myslot;
-                if ((LPR == 8 || (sub & 1) == 0) && u0 + row < depth && i < n) s_key[i] = score_key(tot * a.scale);
             }
         }
         RETOPK_PHASE(0, 12);
@@ -745,34 +727,17 @@ __global__ void __launch_bounds__(REUSE_THREADS, 1) reuse_kernel(const StepArgs 
     __syncthreads();
     RETOPK_PHASE(0, 6);
 
-    // Nearly every candidate ends up selected when the recalled supports overlap (n close to K):
-    // then request the value rows of ALL candidates now, so that they arrive while the
-    // selection runs, and let the softmax weights (zero for the losers) pick among them.
-    const bool ahead = n > 0 && n <= a.stage_depth * SLOTS && 2 * n <= 3 * K;
-    if (ahead) {
-        const int sub = lane % LPR, myslot = warp * RPW + lane / LPR;
-        const char* vsrc = reinterpret_cast<const char*>(a.v + (size_t)bkv * a.max_seq_len * D) + sub * 16;
-        uint4* my_stage = s_stage + tid;     // this thread has read back its own key pieces already
-        for (int u = 0; u < a.stage_depth; ++u) {
-            const int i = u * SLOTS + myslot;
-            if (i < n) cp_async16(my_stage + u * NT, vsrc + (size_t)s_idx[i] * (D * 2));
-        }
-        cp_async_commit();
-        for (int i = tid; i < n; i += NT) s_wc[i] = 0.f;
-    }
-
     // Eq. 11: Top-K of the candidates; insert the support
     uint32_t kmax;
     bool kmax_known;
-    const int ns = select_listed<NT>(s_key, s_idx, n, K, s_sup_idx, s_sup_key, s_hist, s_ws, kmax, kmax_known,
-                                     s_sup_src);
+    const int ns = select_listed<NT>(s_key, s_idx, n, K, s_sup_idx, s_sup_key, s_hist, s_ws, kmax, kmax_known);
     RETOPK_PHASE(0, 7);
     int32_t* sup_out = a.sup_cache + ((size_t)bh * M + a.slot) * K;
     for (int i = tid; i < K; i += NT) sup_out[i] = i < ns ? s_sup_idx[i] : -1;
 
     // Eq. 12 (s_red aliases the candidate lists, which are dead now)
     attend<D, NT>(a.v + (size_t)bkv * a.max_seq_len * D, ns, s_sup_idx, s_sup_key, s_w, s_red, s_ws, s_stage,
-                  a.stage_depth, kmax, kmax_known, a.out + (size_t)bh * D, s_sup_src, s_wc, ahead ? n : 0);
+                  a.stage_depth, kmax, kmax_known, a.out + (size_t)bh * D);
     if (tid == 0) {      // the step record is written last: nothing in this kernel waits for it
         a.ws_path[bh] = (uint8_t)path;
         a.ws_rho[bh] = rho_max;
