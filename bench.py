@@ -218,11 +218,10 @@ def algorithmic_bytes(cfg, stats, mean_L, mean_fill):
     heads = stats["steps"]
     n_sel = min(cfg.r, mean_fill)
     tail = K * d * 2 + K * 4 + d * 2          # value rows, support insert, output
-    reuse = (heads * (mean_fill * d * 4 + d * 4 + d * 2) + stats["reuse"] * (n_sel * K * 4 + tail)
-             + stats["cand_sum"] * d * 2)
+    recall = heads * (mean_fill * d * 4 + d * 4 + d * 2)
     scan = stats["scan_groups"] * mean_L * d * 2
-    exact_finish = (heads - stats["reuse"]) * tail
-    return dict(reuse=reuse, scan=scan, exact_finish=exact_finish)
+    finish = heads * tail + stats["reuse"] * (n_sel * K * 4 + d * 2) + stats["cand_sum"] * d * 2
+    return dict(recall=recall, scan=scan, finish=finish)
 
 
 def path_mix(stats):

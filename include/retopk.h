@@ -187,7 +187,7 @@ int exact_topk_decode_static(int B, int H_q, int H_kv, int d, int K, int64_t max
  * Measurement hooks (no counterpart in the paper).  Between begin and end, every decode
  * call of this context brackets each of its kernels with CUDA events on the call's stream
  * (up to max_calls calls; later calls run unrecorded).  retopk_profile_end synchronises
- * the device and returns, per kernel slot {0: reuse, 1: scan, 2: exact finish}, the summed
+ * the device and returns, per kernel slot {0: recall, 1: scan, 2: finish}, the summed
  * device time in milliseconds and the number of launches.  Not for use inside a timed
  * region: the events themselves cost a little.
  */

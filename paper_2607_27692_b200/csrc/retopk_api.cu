@@ -19,13 +19,14 @@ struct retopk_ctx {
     int NS, stage_depth, exact_stage_depth;
     int num_sms, scan_grid;
     int call_serial;
-    size_t smem_reuse, smem_exact;
+    size_t smem_recall, smem_reuse, smem_exact, smem_finish;
     // device state
     float* qbar_cache;
     int32_t* sup_cache;
     uint8_t* ws_path;
     float* ws_rho;
     int32_t* ws_ncand;
+    int32_t* ws_sel;
     int32_t* ws_gflag;
     float* ws_scores;
     float* ws_tmax;
@@ -65,7 +66,7 @@ bool dev_alloc(T** p, size_t count) {
 
 void free_all(retopk_ctx* c) {
     cudaFree(c->qbar_cache); cudaFree(c->sup_cache); cudaFree(c->ws_path); cudaFree(c->ws_rho);
-    cudaFree(c->ws_ncand); cudaFree(c->ws_gflag); cudaFree(c->ws_scores); cudaFree(c->ws_tmax); cudaFree(c->counters);
+    cudaFree(c->ws_ncand); cudaFree(c->ws_sel); cudaFree(c->ws_gflag); cudaFree(c->ws_scores); cudaFree(c->ws_tmax); cudaFree(c->counters);
     cudaFree(c->status); cudaFree(c->slow_select); cudaFree(c->scan_groups); cudaFree(c->stage_q); cudaFree(c->stage_out);
     cudaFree(c->stage_kv);
 }
@@ -93,19 +94,12 @@ StepArgs make_args(const retopk_ctx* c, const void* q, const void* k, const void
     a.v = static_cast<const uint16_t*>(v);
     a.out = static_cast<uint16_t*>(out);
     a.qbar_cache = c->qbar_cache; a.sup_cache = c->sup_cache;
-    a.ws_path = c->ws_path; a.ws_rho = c->ws_rho; a.ws_ncand = c->ws_ncand; a.ws_gflag = c->ws_gflag;
+    a.ws_path = c->ws_path; a.ws_rho = c->ws_rho; a.ws_ncand = c->ws_ncand; a.ws_sel = c->ws_sel; a.ws_gflag = c->ws_gflag;
     a.ws_scores = c->ws_scores; a.ws_tmax = c->ws_tmax; a.tmax_stride = c->tmax_stride; a.counters = c->counters; a.status = c->status;
     a.slow_select = c->slow_select;
     a.scan_groups = c->scan_groups;
     a.idx_out = nullptr;
     return a;
-}
-
-int launch_reuse(const retopk_ctx* c, const StepArgs& a, cudaStream_t s) {
-    const unsigned grid = (unsigned)(c->B * c->Hq);
-    if (c->d == 128) reuse_kernel<128><<<grid, REUSE_THREADS, c->smem_reuse, s>>>(a);
-    else reuse_kernel<64><<<grid, REUSE_THREADS, c->smem_reuse, s>>>(a);
-    return cudaGetLastError() == cudaSuccess ? RETOPK_OK : RETOPK_ECUDA;
 }
 
 // Launch with programmatic stream serialisation: the kernel may be set up while its
@@ -127,13 +121,20 @@ int launch_dependent(Kernel kernel, unsigned grid, unsigned block, size_t smem, 
     return cudaLaunchKernelEx(&cfg, kernel, a) == cudaSuccess ? RETOPK_OK : RETOPK_ECUDA;
 }
 
+int launch_recall(const retopk_ctx* c, const StepArgs& a, cudaStream_t s) {
+    const unsigned grid = (unsigned)(c->B * c->Hq);
+    if (c->d == 128) return launch_dependent(recall_kernel<128>, grid, RECALL_THREADS, c->smem_recall, s, a);
+    return launch_dependent(recall_kernel<64>, grid, RECALL_THREADS, c->smem_recall, s, a);
+}
+
 int launch_scan(const retopk_ctx* c, const StepArgs& a, cudaStream_t s) {
     // persistent CTAs; no more of them than there are 256-row work items
     const long long items = (long long)c->B * c->Hkv * ((a.L + SCAN_TILE_ROWS - 1) / SCAN_TILE_ROWS);
     const unsigned grid = (unsigned)(items < c->scan_grid ? items : c->scan_grid);
     const int ntile = (c->G + 7) / 8;
-    // An ordinary launch: started as a dependent launch behind the 1024-thread kernel, the scan
-    // measured 1.6x slower (its CTAs land on SMs still carved up for the other kernel).
+    // An ordinary launch: started as a dependent launch behind a kernel that takes all of an
+    // SM's shared memory, the scan measured 1.6x slower (its CTAs land on SMs still carved up
+    // for that kernel, and it needs about 100 KB of L1 to keep its loads in flight).
     if (c->d == 128 && ntile == 1) scan_kernel<128, 1><<<grid, SCAN_THREADS, 0, s>>>(a);
     else if (c->d == 128) scan_kernel<128, 2><<<grid, SCAN_THREADS, 0, s>>>(a);
     else if (ntile == 1) scan_kernel<64, 1><<<grid, SCAN_THREADS, 0, s>>>(a);
@@ -141,10 +142,11 @@ int launch_scan(const retopk_ctx* c, const StepArgs& a, cudaStream_t s) {
     return cudaGetLastError() == cudaSuccess ? RETOPK_OK : RETOPK_ECUDA;
 }
 
-int launch_exact_finish(const retopk_ctx* c, const StepArgs& a, cudaStream_t s) {
+int launch_finish(const retopk_ctx* c, const StepArgs& a, cudaStream_t s) {
     const unsigned grid = (unsigned)(c->B * c->Hq);
-    if (c->d == 128) return launch_dependent(exact_finish_kernel<128>, grid, EXACT_THREADS, c->smem_exact, s, a);
-    return launch_dependent(exact_finish_kernel<64>, grid, EXACT_THREADS, c->smem_exact, s, a);
+    const size_t smem = a.mode == MODE_EXACT ? c->smem_exact : c->smem_finish;
+    if (c->d == 128) return launch_dependent(finish_kernel<128>, grid, FINISH_THREADS, smem, s, a);
+    return launch_dependent(finish_kernel<64>, grid, FINISH_THREADS, smem, s, a);
 }
 
 // Measurement hook: event number `which` (0..3) of the current call, if recording.
@@ -194,22 +196,23 @@ int retopk_create_batched(retopk_ctx** out, int B, int H_q, int H_kv, int d, int
     c->num_sms = sms > 0 ? sms : 148;
 
     // shared-memory footprints (must mirror the carve-up at the top of each kernel)
-    const size_t red_words = (size_t)(REUSE_THREADS / 32) * d + REUSE_THREADS;
-    const size_t head_words = ((size_t)2 * d + M + r + 32 + 8 + SCRATCH_WORDS + 3 * (size_t)K + 3) & ~(size_t)3;
+    const size_t red_words = (size_t)(FINISH_THREADS / 32) * d + FINISH_THREADS;
+    const size_t head_words = ((size_t)d + r + 32 + SCRATCH_WORDS + 3 * (size_t)K + 3) & ~(size_t)3;
     const size_t big_words = (((size_t)2 * c->cap > red_words ? (size_t)2 * c->cap : red_words) + 3) & ~(size_t)3;
     const size_t bm_words = (((size_t)max_seq_len + 31) / 32 + 3) & ~(size_t)3;
+    c->smem_recall = ((size_t)d + ((M + 3) & ~3) + r + 4) * 4;
     c->smem_reuse = (head_words + big_words + bm_words) * 4;
     c->smem_exact = (((size_t)c->NS * 2 + (size_t)c->NS / 2 + (size_t)K * 3 + SCRATCH_WORDS + 32 + 8 + 3) & ~(size_t)3) * 4;
     int max_smem = 0;
     cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, c->device);
     // the rest of shared memory is the landing zone of the asynchronous row copies:
     // 16 KB (one 16-byte piece per thread) per row kept in flight per row slot
-    const size_t wave = (size_t)REUSE_THREADS * 16;
+    const size_t wave = (size_t)FINISH_THREADS * 16;
     if ((size_t)max_smem < c->smem_reuse + wave || (size_t)max_smem < c->smem_exact + wave) {
         delete c;
         return RETOPK_EUNSUPPORTED;
     }
-    const int slots = REUSE_THREADS / (d / 8);
+    const int slots = FINISH_THREADS / (d / 8);
     auto depth_for = [&](size_t fixed, int rows) {
         long long fit = (long long)(((size_t)max_smem - fixed) / wave);
         long long want = (rows + slots - 1) / slots;          // one wave covers `rows` rows
@@ -224,28 +227,28 @@ int retopk_create_batched(retopk_ctx** out, int B, int H_q, int H_kv, int d, int
     }
     c->smem_reuse += (size_t)c->stage_depth * wave;
     c->smem_exact += (size_t)c->exact_stage_depth * wave;
+    c->smem_finish = c->smem_reuse > c->smem_exact ? c->smem_reuse : c->smem_exact;
     // opt in to the device maximum once; contexts of different sizes then coexist
-    cudaError_t e1, e2;
+    cudaError_t e1, e2 = cudaSuccess;
     int occ = 0;
     const int ntile = (c->G + 7) / 8;
     if (d == 128) {
-        e1 = cudaFuncSetAttribute(reuse_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
-        e2 = cudaFuncSetAttribute(exact_finish_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
+        e1 = cudaFuncSetAttribute(finish_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
         if (ntile == 1) cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, scan_kernel<128, 1>, SCAN_THREADS, 0);
         else cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, scan_kernel<128, 2>, SCAN_THREADS, 0);
     } else {
-        e1 = cudaFuncSetAttribute(reuse_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
-        e2 = cudaFuncSetAttribute(exact_finish_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
+        e1 = cudaFuncSetAttribute(finish_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
         if (ntile == 1) cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, scan_kernel<64, 1>, SCAN_THREADS, 0);
         else cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, scan_kernel<64, 2>, SCAN_THREADS, 0);
     }
     if (e1 != cudaSuccess || e2 != cudaSuccess) { cudaGetLastError(); delete c; return RETOPK_ECUDA; }
     c->scan_grid = c->num_sms * (occ > 0 ? occ : 2);
 
+
     const size_t nh = (size_t)B * H_q;
     bool ok = dev_alloc(&c->qbar_cache, nh * M * d) && dev_alloc(&c->sup_cache, nh * M * K) &&
               dev_alloc(&c->ws_path, nh) && dev_alloc(&c->ws_rho, nh) && dev_alloc(&c->ws_ncand, nh) &&
-              dev_alloc(&c->ws_gflag, (size_t)B * H_kv) && dev_alloc(&c->ws_scores, nh * (size_t)c->score_stride) &&
+              dev_alloc(&c->ws_sel, nh * r) && dev_alloc(&c->ws_gflag, (size_t)B * H_kv) && dev_alloc(&c->ws_scores, nh * (size_t)c->score_stride) &&
               dev_alloc(&c->ws_tmax, nh * (size_t)c->tmax_stride) &&
               dev_alloc(&c->counters, nh * 4) && dev_alloc(&c->status, 1) &&
               dev_alloc(&c->slow_select, 1) && dev_alloc(&c->scan_groups, 1) && dev_alloc(&c->stage_q, nh * d) &&
@@ -292,11 +295,11 @@ int retopk_decode_step(retopk_ctx* c, const void* q, const void* k_cache, const 
     c->call_serial = (c->call_serial + 1) & 0x3fffffff;
     a.step_id = c->call_serial;
     prof_mark(c, 0, s);
-    if ((rc = launch_reuse(c, a, s)) != RETOPK_OK) return rc;
+    if ((rc = launch_recall(c, a, s)) != RETOPK_OK) return rc;
     prof_mark(c, 1, s);
     if ((rc = launch_scan(c, a, s)) != RETOPK_OK) return rc;
     prof_mark(c, 2, s);
-    if ((rc = launch_exact_finish(c, a, s)) != RETOPK_OK) return rc;
+    if ((rc = launch_finish(c, a, s)) != RETOPK_OK) return rc;
     prof_mark(c, 3, s);
     prof_done(c, 0);
     c->last_launches = 3;
@@ -316,7 +319,7 @@ int exact_topk_decode(retopk_ctx* c, const void* q, const void* k_cache, const v
     prof_mark(c, 1, s);
     if ((rc = launch_scan(c, a, s)) != RETOPK_OK) return rc;
     prof_mark(c, 2, s);
-    if ((rc = launch_exact_finish(c, a, s)) != RETOPK_OK) return rc;
+    if ((rc = launch_finish(c, a, s)) != RETOPK_OK) return rc;
     prof_mark(c, 3, s);
     prof_done(c, 1);
     c->last_launches = 2;
@@ -491,8 +494,8 @@ int static_setup(int dev, StaticSetup** out) {
         if (cudaDeviceGetAttribute(&st->num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
             cudaDeviceGetAttribute(&st->max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess)
             return RETOPK_ECUDA;
-        if (cudaFuncSetAttribute(exact_finish_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, st->max_smem) != cudaSuccess ||
-            cudaFuncSetAttribute(exact_finish_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, st->max_smem) != cudaSuccess)
+        if (cudaFuncSetAttribute(finish_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, st->max_smem) != cudaSuccess ||
+            cudaFuncSetAttribute(finish_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, st->max_smem) != cudaSuccess)
             return RETOPK_ECUDA;
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&st->occ[0][0], scan_kernel<64, 1>, SCAN_THREADS, 0);
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&st->occ[0][1], scan_kernel<64, 2>, SCAN_THREADS, 0);
@@ -532,9 +535,9 @@ int exact_topk_decode_static(int B, int H_q, int H_kv, int d, int K, int64_t max
 
     const int NS = 16 * K <= 8192 ? 8192 : 16384;
     size_t smem = (((size_t)NS * 2 + (size_t)NS / 2 + (size_t)K * 3 + SCRATCH_WORDS + 32 + 8 + 3) & ~(size_t)3) * 4;
-    const size_t wave = (size_t)EXACT_THREADS * 16;
+    const size_t wave = (size_t)FINISH_THREADS * 16;
     if ((size_t)st->max_smem < smem + wave) return RETOPK_EUNSUPPORTED;
-    const int slots = EXACT_THREADS / (d / 8);
+    const int slots = FINISH_THREADS / (d / 8);
     long long depth = (long long)(((size_t)st->max_smem - smem) / wave);
     const long long want = (K + slots - 1) / slots;
     if (depth > want) depth = want;
@@ -574,8 +577,8 @@ int exact_topk_decode_static(int B, int H_q, int H_kv, int d, int K, int64_t max
     else if (ntile == 1) scan_kernel<64, 1><<<grid, SCAN_THREADS, 0, s>>>(a);
     else scan_kernel<64, 2><<<grid, SCAN_THREADS, 0, s>>>(a);
     if (cudaGetLastError() != cudaSuccess) return RETOPK_ECUDA;
-    if (d == 128) exact_finish_kernel<128><<<(unsigned)nh, EXACT_THREADS, smem, s>>>(a);
-    else exact_finish_kernel<64><<<(unsigned)nh, EXACT_THREADS, smem, s>>>(a);
+    if (d == 128) finish_kernel<128><<<(unsigned)nh, FINISH_THREADS, smem, s>>>(a);
+    else finish_kernel<64><<<(unsigned)nh, FINISH_THREADS, smem, s>>>(a);
     return cudaGetLastError() == cudaSuccess ? RETOPK_OK : RETOPK_ECUDA;
 }
 

@@ -1,20 +1,21 @@
 // Device code of the ReTopK decode step (sm_100a).
 //
 // Three kernels per step, all reading caller-owned bf16 q / K / V:
-//   reuse_kernel   one CTA per (sequence, query head): normalise the query, cosine
+//   recall_kernel  one CTA per (sequence, query head): normalise the query, cosine
 //                  similarity to the cached queries (Eq. 6), Top-r recall and rho_max
-//                  (Eq. 7), path decision (Eq. 13), insert of the normalised query.  A
-//                  head on the reuse path then stays in this CTA to the end: candidate
-//                  union (Eq. 8-9) in a shared-memory bitmap, exact scores of the gathered
-//                  key rows (Eq. 10), Top-K (Eq. 11), softmax.V (Eq. 12), support insert.
-//                  A head on the exact path only flags its KV group and leaves.
+//                  (Eq. 7), path decision (Eq. 13), insert of the normalised query.  A head
+//                  on the exact path flags its KV group.
 //   scan_kernel    persistent CTAs over the flagged KV groups: full-history scores
 //                  e_i = q.k_i/sqrt(d) (Eq. 4); every key row streams once through the
-//                  tensor cores for all G query heads of its group.
-//   exact_finish_kernel  one CTA per exact-path head: global Top-K (Eq. 1) of the scanned
-//                  scores (tile maxima give a lower bound for the K-th score, only the
-//                  tiles that reach it are read back), softmax.V (Eq. 12), support insert.
-//                  Exact Top-K attention is scan + this kernel.
+//                  tensor cores for all G query heads of its group; also the maximum of
+//                  every 16-row tile.
+//   finish_kernel  one CTA per (sequence, query head), heads of both paths side by side.
+//                  Reuse path: candidate union (Eq. 8-9) in a shared-memory bitmap, exact
+//                  scores of the gathered key rows (Eq. 10), Top-K (Eq. 11).  Exact path:
+//                  global Top-K (Eq. 1) of the scanned scores (tile maxima give a lower
+//                  bound for the K-th score, only the tiles that reach it are read back).
+//                  Both: softmax.V (Eq. 12) and the support insert.
+//                  Exact Top-K attention is scan + finish with every head on the exact path.
 #pragma once
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -38,8 +39,8 @@ namespace retopk {
 constexpr int PATH_REUSE = 0, PATH_FALLBACK = 1, PATH_REFRESH = 2;
 constexpr int MODE_RETOPK = 0, MODE_EXACT = 1;
 
-constexpr int REUSE_THREADS = 1024;
-constexpr int EXACT_THREADS = 1024;
+constexpr int RECALL_THREADS = 1024;
+constexpr int FINISH_THREADS = 1024;
 constexpr int SCAN_THREADS = 256;
 constexpr int SCAN_TILE_ROWS = 256;  // key rows per scan work item
 constexpr int MAX_GROUPS = 4096;     // B * H_kv limit (shared list in scan_kernel)
@@ -69,6 +70,7 @@ struct StepArgs {
     uint8_t* ws_path;        // [B*Hq]
     float* ws_rho;           // [B*Hq]
     int32_t* ws_ncand;       // [B*Hq]
+    int32_t* ws_sel;         // [B*Hq][r] recalled cache slots, -1 padded
     int32_t* ws_gflag;       // [B*Hkv] == step_id when the group needs a full scan
     float* ws_scores;        // [B*Hq][score_stride]
     float* ws_tmax;          // [B*Hq][tmax_stride] largest score of every 16-row key tile
@@ -497,42 +499,29 @@ __device__ void attend(const uint16_t* vbase, int ns, const int32_t* s_sup_idx, 
 }
 
 // ------------------------------------------------------------------------------------
-// reuse_kernel
+// recall_kernel: Eq. 6, Eq. 7, Eq. 13 and the insert of the normalised query, per head.
+// Leaves the recalled slots, rho_max and the path in global memory and flags the KV group
+// of every head that takes the exact path.
 // ------------------------------------------------------------------------------------
 template <int D>
-__global__ void __launch_bounds__(REUSE_THREADS, 1) reuse_kernel(const StepArgs a) {
-    constexpr int NT = REUSE_THREADS;
+__global__ void __launch_bounds__(RECALL_THREADS, 1) recall_kernel(const StepArgs a) {
+    constexpr int NT = RECALL_THREADS;
     constexpr int NW = NT / 32;
-    constexpr int LPR = D / 8, RPW = 32 / LPR, SLOTS = NW * RPW;
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    // layout (words): q[D] qraw[D] rho[M] sel[r] ws[32] misc[8] hist[SCRATCH_WORDS] sup_idx[K] sup_key[K] w[K]
-    //                 | big: idx[cap] key[cap], aliased later by red[NW*D+NT] | bitmap | stage[depth*NT*4]
+    // layout (words): q[D] rho[M + 3] sel[r] misc[4]
     float* s_q = reinterpret_cast<float*>(smem_raw);
-    float* s_qraw = s_q + D;
-    float* s_rho = s_qraw + D;
-    int* s_sel = reinterpret_cast<int*>(s_rho + a.M);
-    int* s_ws = s_sel + a.r;
-    int* s_misc = s_ws + 32;
-    uint32_t* s_hist = reinterpret_cast<uint32_t*>(s_misc + 8);
-    int32_t* s_sup_idx = reinterpret_cast<int32_t*>(s_hist + SCRATCH_WORDS);
-    uint32_t* s_sup_key = reinterpret_cast<uint32_t*>(s_sup_idx + a.K);
-    float* s_w = reinterpret_cast<float*>(s_sup_key + a.K);
-    const int head_words = (2 * D + a.M + a.r + 32 + 8 + SCRATCH_WORDS + 3 * a.K + 3) & ~3;
-    int32_t* s_idx = reinterpret_cast<int32_t*>(smem_raw) + head_words;
-    uint32_t* s_key = reinterpret_cast<uint32_t*>(s_idx + a.cap);
-    float* s_red = reinterpret_cast<float*>(s_idx);
-    const int big_words = (max(2 * a.cap, NW * D + NT) + 3) & ~3;
-    uint32_t* s_bm = reinterpret_cast<uint32_t*>(s_idx) + big_words;
-    uint4* s_stage = reinterpret_cast<uint4*>(s_bm + ((((int)a.max_seq_len + 31) / 32 + 3) & ~3));
+    float* s_rho = s_q + D;
+    int* s_sel = reinterpret_cast<int*>(s_rho + ((a.M + 3) & ~3));
+    float* s_misc = reinterpret_cast<float*>(s_sel + a.r);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int bh = blockIdx.x;
     const int b = bh / a.Hq, h = bh % a.Hq;
     const int bkv = b * a.Hkv + h / a.G;
-    const int M = a.M, fill = a.fill, L = a.L, K = a.K;
-    const int nwords = (L + 31) >> 5;
+    const int M = a.M, fill = a.fill;
 
-    RETOPK_PHASE(0, 0);
+    pdl_wait();        // the caches were written by the step before; q by whatever ran before this call
+    RETOPK_PHASE(1, 0);
     // Every warp reads the query itself (four elements per lane) next to its cache rows, so
     // one memory latency covers both:  rho_c = (qbar_c . q) / |q|   (Eq. 6)
     float q4[4] = {0.f, 0.f, 0.f, 0.f};
@@ -541,7 +530,7 @@ __global__ void __launch_bounds__(REUSE_THREADS, 1) reuse_kernel(const StepArgs 
         q4[0] = bf16_lo(raw.x); q4[1] = bf16_hi(raw.x); q4[2] = bf16_lo(raw.y); q4[3] = bf16_hi(raw.y);
     }
     if (tid < a.r) s_sel[tid] = -1;
-    if (tid == 0) reinterpret_cast<float*>(s_misc)[0] = -CUDART_INF_F;
+    if (tid == 0) s_misc[0] = -CUDART_INF_F;
     float inv_nrm = 0.f;
     for (int c0 = warp; c0 < fill || c0 == warp; c0 += NW * 4) {
         float4 x[4];
@@ -553,11 +542,7 @@ __global__ void __launch_bounds__(REUSE_THREADS, 1) reuse_kernel(const StepArgs 
                 : make_float4(0.f, 0.f, 0.f, 0.f);
         }
         if (c0 == warp) {
-            // first trip: clear the bitmap while the loads fly, then the query norm
-            if (!a.refresh) {
-                uint4* bm4 = reinterpret_cast<uint4*>(s_bm);
-                for (int w = tid; w < (nwords + 3) >> 2; w += NT) bm4[w] = make_uint4(0, 0, 0, 0);
-            }
+            // first trip: the query norm while the loads fly
             float n2 = q4[0] * q4[0];
             n2 = fmaf(q4[1], q4[1], n2); n2 = fmaf(q4[2], q4[2], n2); n2 = fmaf(q4[3], q4[3], n2);
 #pragma unroll
@@ -566,10 +551,7 @@ __global__ void __launch_bounds__(REUSE_THREADS, 1) reuse_kernel(const StepArgs 
             inv_nrm = nrm > 0.f ? 1.f / nrm : 0.f;
             if (warp == 0 && lane < D / 4) {
 #pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    s_q[4 * lane + e] = nrm > 0.f ? q4[e] / nrm : 0.f;
-                    s_qraw[4 * lane + e] = q4[e];
-                }
+                for (int e = 0; e < 4; ++e) s_q[4 * lane + e] = nrm > 0.f ? q4[e] / nrm : 0.f;
             }
         }
 #pragma unroll
@@ -585,7 +567,7 @@ __global__ void __launch_bounds__(REUSE_THREADS, 1) reuse_kernel(const StepArgs 
         }
     }
     __syncthreads();
-    RETOPK_PHASE(0, 2);
+    RETOPK_PHASE(1, 1);
 
     // Eq. 7: rho_max and the min(r, fill) most similar slots.  Every cached entry ranks
     // itself against the others (larger rho first, ties -> lower slot).
@@ -601,11 +583,10 @@ __global__ void __launch_bounds__(REUSE_THREADS, 1) reuse_kernel(const StepArgs 
             rank += (c + 3 < fill) && (o.w > mine || (o.w == mine && c + 3 < tid));
         }
         if (rank < n_sel) s_sel[rank] = tid;
-        if (rank == 0) reinterpret_cast<float*>(s_misc)[0] = mine;
+        if (rank == 0) s_misc[0] = mine;
     }
     __syncthreads();
-    const float rho_max = reinterpret_cast<float*>(s_misc)[0];
-    RETOPK_PHASE(0, 3);
+    const float rho_max = s_misc[0];
 
     // Eq. 13
     int path;
@@ -615,17 +596,66 @@ __global__ void __launch_bounds__(REUSE_THREADS, 1) reuse_kernel(const StepArgs 
 
     // insert the normalised query now: every similarity of this step has been taken
     if (tid < D) a.qbar_cache[((size_t)bh * M + a.slot) * D + tid] = s_q[tid];
-
-    if (path != PATH_REUSE) {
-        if (tid == 0) {
+    if (tid < a.r) a.ws_sel[(size_t)bh * a.r + tid] = s_sel[tid];
+    if (tid == 0) {
+        a.ws_path[bh] = (uint8_t)path;
+        a.ws_rho[bh] = rho_max;
+        if (path != PATH_REUSE) {
             a.ws_gflag[bkv] = a.step_id;       // same value from every head of the group
-            a.ws_path[bh] = (uint8_t)path;
-            a.ws_rho[bh] = rho_max;
-            a.ws_ncand[bh] = L;
+            a.ws_ncand[bh] = a.L;
             atomicAdd(a.counters + (size_t)bh * 4 + path, 1ull);     // no return value: not waited for
         }
-        return;
     }
+    RETOPK_PHASE(1, 2);
+}
+
+// ------------------------------------------------------------------------------------
+// reuse path of finish_kernel: candidate union (Eq. 8-9), candidate scores (Eq. 10), Top-K
+// (Eq. 11), softmax.V (Eq. 12) and the support insert for one head, all in shared memory.
+// ------------------------------------------------------------------------------------
+template <int D, int NT>
+__device__ void reuse_path(const StepArgs& a, unsigned char* smem_raw) {
+    constexpr int NW = NT / 32;
+    constexpr int LPR = D / 8, RPW = 32 / LPR, SLOTS = NW * RPW;
+    // layout (words): qraw[D] sel[r] ws[32] hist[SCRATCH_WORDS] sup_idx[K] sup_key[K] w[K]
+    //                 | big: idx[cap] key[cap], aliased later by red[NW*D+NT] | bitmap | stage[depth*NT*4]
+    float* s_qraw = reinterpret_cast<float*>(smem_raw);
+    int* s_sel = reinterpret_cast<int*>(s_qraw + D);
+    int* s_ws = s_sel + a.r;
+    uint32_t* s_hist = reinterpret_cast<uint32_t*>(s_ws + 32);
+    int32_t* s_sup_idx = reinterpret_cast<int32_t*>(s_hist + SCRATCH_WORDS);
+    uint32_t* s_sup_key = reinterpret_cast<uint32_t*>(s_sup_idx + a.K);
+    float* s_w = reinterpret_cast<float*>(s_sup_key + a.K);
+    const int head_words = (D + a.r + 32 + SCRATCH_WORDS + 3 * a.K + 3) & ~3;
+    int32_t* s_idx = reinterpret_cast<int32_t*>(smem_raw) + head_words;
+    uint32_t* s_key = reinterpret_cast<uint32_t*>(s_idx + a.cap);
+    float* s_red = reinterpret_cast<float*>(s_idx);
+    const int big_words = (max(2 * a.cap, NW * D + NT) + 3) & ~3;
+    uint32_t* s_bm = reinterpret_cast<uint32_t*>(s_idx) + big_words;
+    uint4* s_stage = reinterpret_cast<uint4*>(s_bm + ((((int)a.max_seq_len + 31) / 32 + 3) & ~3));
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int bh = blockIdx.x;
+    const int b = bh / a.Hq, h = bh % a.Hq;
+    const int bkv = b * a.Hkv + h / a.G;
+    const int M = a.M, fill = a.fill, L = a.L, K = a.K;
+    const int n_sel = a.r < fill ? a.r : fill;
+    RETOPK_PHASE(0, 0);
+
+    // recalled slots and the raw query from global memory; clear the bitmap meanwhile
+    if (tid < a.r) s_sel[tid] = a.ws_sel[(size_t)bh * a.r + tid];
+    if (tid >= 32 && tid < 32 + D / 2) {
+        const uint32_t raw = reinterpret_cast<const uint32_t*>(a.q + (size_t)bh * D)[tid - 32];
+        s_qraw[2 * (tid - 32)] = bf16_lo(raw);
+        s_qraw[2 * (tid - 32) + 1] = bf16_hi(raw);
+    }
+    {
+        const int nwords = (L + 31) >> 5;
+        uint4* bm4 = reinterpret_cast<uint4*>(s_bm);
+        for (int w = tid; w < (nwords + 3) >> 2; w += NT) bm4[w] = make_uint4(0, 0, 0, 0);
+    }
+    __syncthreads();
+    RETOPK_PHASE(0, 3);
 
     // Eq. 8-9: sorted unique candidate list.  Recalled indices below the window go through a
     // bitmap over key positions (ordered extraction = sorted and deduplicated for free); the
@@ -633,25 +663,21 @@ __global__ void __launch_bounds__(REUSE_THREADS, 1) reuse_kernel(const StepArgs 
     const int w_lo = L - a.W > 0 ? L - a.W : 0;
     {
         bool bad = false;
-        const int E = n_sel * K;
-        for (int e0 = tid; e0 < E; e0 += NT * 4) {
-            int idx[4];
+        for (int s0 = 0; s0 < n_sel; s0 += 4)
+            for (int i = tid; i < K; i += NT) {
+                int idx[4];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const int e = e0 + u * NT;
-                idx[u] = -1;
-                if (e < E) {
-                    const int s = e / K, c = s_sel[s];
-                    if (c >= 0) idx[u] = a.sup_cache[((size_t)bh * M + c) * K + (e - s * K)];
+                for (int u = 0; u < 4; ++u) {
+                    const int c = s0 + u < n_sel ? s_sel[s0 + u] : -1;
+                    idx[u] = c >= 0 ? a.sup_cache[((size_t)bh * M + c) * K + i] : -1;
                 }
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+                    if (idx[u] >= 0) {
+                        if (idx[u] < w_lo) atomicOr(&s_bm[idx[u] >> 5], 1u << (idx[u] & 31));
+                        else if (idx[u] >= L) bad = true;
+                    }
             }
-#pragma unroll
-            for (int u = 0; u < 4; ++u)
-                if (idx[u] >= 0) {
-                    if (idx[u] < w_lo) atomicOr(&s_bm[idx[u] >> 5], 1u << (idx[u] & 31));
-                    else if (idx[u] >= L) bad = true;
-                }
-        }
         if (bad) atomicOr(a.status, 1u);
     }
     __syncthreads();
@@ -739,8 +765,6 @@ __global__ void __launch_bounds__(REUSE_THREADS, 1) reuse_kernel(const StepArgs 
     attend<D, NT>(a.v + (size_t)bkv * a.max_seq_len * D, ns, s_sup_idx, s_sup_key, s_w, s_red, s_ws, s_stage,
                   a.stage_depth, kmax, kmax_known, a.out + (size_t)bh * D);
     if (tid == 0) {      // the step record is written last: nothing in this kernel waits for it
-        a.ws_path[bh] = (uint8_t)path;
-        a.ws_rho[bh] = rho_max;
         a.ws_ncand[bh] = n;
         atomicAdd(a.counters + (size_t)bh * 4 + PATH_REUSE, 1ull);
         atomicAdd(a.counters + (size_t)bh * 4 + 3, (unsigned long long)n);
@@ -885,7 +909,7 @@ __global__ void __launch_bounds__(SCAN_THREADS) scan_kernel(const StepArgs a) {
 }
 
 // ------------------------------------------------------------------------------------
-// exact_finish_kernel
+// exact path of finish_kernel
 //
 // Global Top-K without reading all L scores again.  The scan left the maximum of every
 // 16-row tile.  If v is the K-th largest of (groups of) tile maxima, at least K different
@@ -894,14 +918,9 @@ __global__ void __launch_bounds__(SCAN_THREADS) scan_kernel(const StepArgs a) {
 // read back, their scores >= v are listed in index order, and the exact Top-K with the
 // lower-index tie rule is taken from that list.
 // ------------------------------------------------------------------------------------
-template <int D>
-__global__ void __launch_bounds__(EXACT_THREADS, 1) exact_finish_kernel(const StepArgs a) {
-    constexpr int NT = EXACT_THREADS;
+template <int D, int NT>
+__device__ void exact_path(const StepArgs& a, unsigned char* smem_raw) {
     const int bh = blockIdx.x;
-    pdl_wait();        // scores and tile maxima come from the scan, path flags from the step's first kernel
-    if (a.mode == MODE_RETOPK && a.ws_path[bh] == PATH_REUSE) return;
-
-    extern __shared__ __align__(16) unsigned char smem_raw[];
     // layout (words): key[NS] idx[NS] (aliased later by red[NW*D+NT]) tile[NS/2]
     //                 sup_idx[K] sup_key[K] w[K] cnt[SCRATCH_WORDS] ws[32] misc[8] stage[depth*NT*4]
     uint32_t* s_key = reinterpret_cast<uint32_t*>(smem_raw);
@@ -1079,6 +1098,19 @@ __global__ void __launch_bounds__(EXACT_THREADS, 1) exact_finish_kernel(const St
     attend<D, NT>(a.v + (size_t)bkv * a.max_seq_len * D, ns, s_sup_idx, s_sup_key, s_w, s_red, s_ws, s_stage,
                   a.exact_stage_depth, kmax, kmax_known, a.out + (size_t)bh * D);
     RETOPK_PHASE(2, 5);
+}
+
+// ------------------------------------------------------------------------------------
+// finish_kernel: one CTA per (sequence, query head), launched behind the scan.  A head on
+// the reuse path never waited for the scan's results, a head on the exact path selects from
+// them; both end with softmax.V and the support insert.  Heads of one step run side by side.
+// ------------------------------------------------------------------------------------
+template <int D>
+__global__ void __launch_bounds__(FINISH_THREADS, 1) finish_kernel(const StepArgs a) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    pdl_wait();        // scores and tile maxima come from the scan, recalled slots and paths from recall_kernel
+    if (a.mode == MODE_RETOPK && a.ws_path[blockIdx.x] == PATH_REUSE) reuse_path<D, FINISH_THREADS>(a, smem_raw);
+    else exact_path<D, FINISH_THREADS>(a, smem_raw);
 }
 
 // Clear the caches (supports to -1, queries and counters to 0).

@@ -213,7 +213,7 @@ class ReTopK:
         ms, n = (C.c_double * 3)(), (_i64 * 3)()
         _check(self.lib.retopk_profile_end(self.h, ms, n), "retopk_profile_end")
         return {name: dict(ms=float(ms[i]), launches=int(n[i]))
-                for i, name in enumerate(("reuse", "scan", "exact_finish"))}
+                for i, name in enumerate(("recall", "scan", "finish"))}
 
     def last_launch_count(self) -> int:
         return int(self.lib.retopk_last_launch_count(self.h))
