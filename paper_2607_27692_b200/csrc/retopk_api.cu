@@ -87,6 +87,7 @@ StepArgs make_args(const retopk_ctx* c, const void* q, const void* k, const void
     a.mode = mode;
     a.NS = c->NS;
     a.step_id = c->call_serial;
+    a.g_shift = (c->G & (c->G - 1)) == 0 ? __builtin_ctz((unsigned)c->G) : -1;
     a.stage_depth = c->stage_depth;
     a.exact_stage_depth = c->exact_stage_depth;
     a.q = static_cast<const uint16_t*>(q);
@@ -248,7 +249,7 @@ int retopk_create_batched(retopk_ctx** out, int B, int H_q, int H_kv, int d, int
     const size_t nh = (size_t)B * H_q;
     bool ok = dev_alloc(&c->qbar_cache, nh * M * d) && dev_alloc(&c->sup_cache, nh * M * K) &&
               dev_alloc(&c->ws_path, nh) && dev_alloc(&c->ws_rho, nh) && dev_alloc(&c->ws_ncand, nh) &&
-              dev_alloc(&c->ws_sel, nh * r) && dev_alloc(&c->ws_gflag, (size_t)B * H_kv) && dev_alloc(&c->ws_scores, nh * (size_t)c->score_stride) &&
+              dev_alloc(&c->ws_sel, nh * r) && dev_alloc(&c->ws_gflag, (size_t)B * H_kv + 1) && dev_alloc(&c->ws_scores, nh * (size_t)c->score_stride) &&
               dev_alloc(&c->ws_tmax, nh * (size_t)c->tmax_stride) &&
               dev_alloc(&c->counters, nh * 4) && dev_alloc(&c->status, 1) &&
               dev_alloc(&c->slow_select, 1) && dev_alloc(&c->scan_groups, 1) && dev_alloc(&c->stage_q, nh * d) &&
@@ -280,7 +281,7 @@ int retopk_reset(retopk_ctx* c, void* stream) {
     const size_t nh = (size_t)c->B * c->Hq;
     reset_kernel<<<c->num_sms * 4, 256, 0, static_cast<cudaStream_t>(stream)>>>(
         c->qbar_cache, nh * c->M * c->d, c->sup_cache, nh * c->M * c->K, c->counters, nh * 4, c->ws_gflag,
-        (size_t)c->B * c->Hkv, c->status, c->slow_select, c->scan_groups);
+        (size_t)c->B * c->Hkv + 1, c->status, c->slow_select, c->scan_groups);
     c->n_ins = 0;
     c->t_dec = 0;
     return cudaGetLastError() == cudaSuccess ? RETOPK_OK : RETOPK_ECUDA;
@@ -554,6 +555,7 @@ int exact_topk_decode_static(int B, int H_q, int H_kv, int d, int K, int64_t max
     a.scale = 1.0f / sqrtf((float)d);
     a.mode = MODE_EXACT;
     a.NS = NS;
+    a.g_shift = (a.G & (a.G - 1)) == 0 ? __builtin_ctz((unsigned)a.G) : -1;
     a.exact_stage_depth = (int)depth;
     a.q = static_cast<const uint16_t*>(q);
     a.k = static_cast<const uint16_t*>(k_cache);

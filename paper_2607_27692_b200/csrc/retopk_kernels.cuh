@@ -58,6 +58,7 @@ struct StepArgs {
     int refresh;             // 1 when Eq. 13's first case holds (known on the host)
     int mode;                // MODE_RETOPK or MODE_EXACT
     int NS;                  // entries in exact_finish_kernel's shared collection lists
+    int g_shift;             // log2(G) when G is a power of two, else -1
     int step_id;             // call serial number; a KV group is flagged by storing it
     int stage_depth;         // rows in flight per row slot in reuse_kernel's landing zone
     int exact_stage_depth;   // same for exact_finish_kernel
@@ -71,7 +72,7 @@ struct StepArgs {
     float* ws_rho;           // [B*Hq]
     int32_t* ws_ncand;       // [B*Hq]
     int32_t* ws_sel;         // [B*Hq][r] recalled cache slots, -1 padded
-    int32_t* ws_gflag;       // [B*Hkv] == step_id when the group needs a full scan
+    int32_t* ws_gflag;       // [B*Hkv + 1] == step_id when the group needs a full scan; last word: any group
     float* ws_scores;        // [B*Hq][score_stride]
     float* ws_tmax;          // [B*Hq][tmax_stride] largest score of every 16-row key tile
     long long tmax_stride;   // multiple of 4
@@ -134,6 +135,11 @@ __device__ __forceinline__ float dot8(const uint4& x, const float* qf) {
 __device__ __forceinline__ void unpack8(const uint4& x, float* f) {
     f[0] = bf16_lo(x.x); f[1] = bf16_hi(x.x); f[2] = bf16_lo(x.y); f[3] = bf16_hi(x.y);
     f[4] = bf16_lo(x.z); f[5] = bf16_hi(x.z); f[6] = bf16_lo(x.w); f[7] = bf16_hi(x.w);
+}
+
+// (sequence, KV head) index of query head bh: bh / G without a division when G is 2^k.
+__device__ __forceinline__ int kv_group_of(int bh, const StepArgs& a) {
+    return a.g_shift >= 0 ? bh >> a.g_shift : bh / a.G;
 }
 
 // Exclusive prefix sum of v over the block in thread order; `total` gets the block sum.
@@ -516,8 +522,7 @@ __global__ void __launch_bounds__(RECALL_THREADS, 1) recall_kernel(const StepArg
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int bh = blockIdx.x;
-    const int b = bh / a.Hq, h = bh % a.Hq;
-    const int bkv = b * a.Hkv + h / a.G;
+    const int bkv = kv_group_of(bh, a);
     const int M = a.M, fill = a.fill;
 
     pdl_wait();        // the caches were written by the step before; q by whatever ran before this call
@@ -571,19 +576,25 @@ __global__ void __launch_bounds__(RECALL_THREADS, 1) recall_kernel(const StepArg
 
     // Eq. 7: rho_max and the min(r, fill) most similar slots.  Every cached entry ranks
     // itself against the others (larger rho first, ties -> lower slot).
+    // P threads share an entry (P a power of two <= 32): each counts the better entries in
+    // its slice of the cache, a shuffle tree adds the slices.
     const int n_sel = a.r < fill ? a.r : fill;
-    if (tid < fill) {
-        const float mine = s_rho[tid];
+    {
+        int lp = 5;
+        while (lp > 0 && (fill << lp) > NT) --lp;
+        const int P = 1 << lp, me = tid >> lp, part = tid & (P - 1);
+        const bool live = me < fill;
+        const float mine = live ? s_rho[me] : 0.f;
         int rank = 0;
-        for (int c = 0; c < fill; c += 4) {
-            const float4 o = *reinterpret_cast<const float4*>(s_rho + c);
-            rank += (c < fill) && (o.x > mine || (o.x == mine && c < tid));
-            rank += (c + 1 < fill) && (o.y > mine || (o.y == mine && c + 1 < tid));
-            rank += (c + 2 < fill) && (o.z > mine || (o.z == mine && c + 2 < tid));
-            rank += (c + 3 < fill) && (o.w > mine || (o.w == mine && c + 3 < tid));
+        for (int c = part; c < fill; c += P) {
+            const float o = s_rho[c];
+            rank += (int)(o > mine) | ((int)(o == mine) & (int)(c < me));
         }
-        if (rank < n_sel) s_sel[rank] = tid;
-        if (rank == 0) s_misc[0] = mine;
+        for (int o = P >> 1; o > 0; o >>= 1) rank += __shfl_xor_sync(0xffffffffu, rank, o);
+        if (live && part == 0) {
+            if (rank < n_sel) s_sel[rank] = me;
+            if (rank == 0) s_misc[0] = mine;
+        }
     }
     __syncthreads();
     const float rho_max = s_misc[0];
@@ -602,6 +613,7 @@ __global__ void __launch_bounds__(RECALL_THREADS, 1) recall_kernel(const StepArg
         a.ws_rho[bh] = rho_max;
         if (path != PATH_REUSE) {
             a.ws_gflag[bkv] = a.step_id;       // same value from every head of the group
+            a.ws_gflag[a.B * a.Hkv] = a.step_id;   // "some group needs a scan in this step"
             a.ws_ncand[bh] = a.L;
             atomicAdd(a.counters + (size_t)bh * 4 + path, 1ull);     // no return value: not waited for
         }
@@ -636,8 +648,7 @@ __device__ void reuse_path(const StepArgs& a, unsigned char* smem_raw) {
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int bh = blockIdx.x;
-    const int b = bh / a.Hq, h = bh % a.Hq;
-    const int bkv = b * a.Hkv + h / a.G;
+    const int bkv = kv_group_of(bh, a);
     const int M = a.M, fill = a.fill, L = a.L, K = a.K;
     const int n_sel = a.r < fill ? a.r : fill;
     RETOPK_PHASE(0, 0);
@@ -803,6 +814,9 @@ __global__ void __launch_bounds__(SCAN_THREADS) scan_kernel(const StepArgs a) {
     // No trigger for the dependent launch behind this kernel: its CTAs take a whole SM each
     // and start as this kernel's CTAs exit; that already hides its launch latency.
 
+    // nothing flagged in this step: leave at once (the common case on the reuse path)
+    if (a.mode != MODE_EXACT && a.ws_gflag[n_groups] != a.step_id) return;
+
     // the groups to scan, in ascending order (all of them for Exact Top-K attention)
     int n_act = 0;
     if (a.mode == MODE_EXACT) n_act = n_groups;
@@ -820,10 +834,12 @@ __global__ void __launch_bounds__(SCAN_THREADS) scan_kernel(const StepArgs a) {
     if (blockIdx.x == 0 && tid == 0) atomicAdd(a.scan_groups, (unsigned long long)n_act);
 
     const int tpg = (L + SCAN_TILE_ROWS - 1) / SCAN_TILE_ROWS;     // work items per group
-    const long long total_items = (long long)n_act * tpg;
-    const long long per = (total_items + gridDim.x - 1) / gridDim.x;
-    const long long it0 = (long long)blockIdx.x * per;
-    const long long it1 = it0 + per < total_items ? it0 + per : total_items;
+    const int total_items = n_act * tpg;                            // < 2^31: checked on the host
+    const int per = (total_items + (int)gridDim.x - 1) / (int)gridDim.x;
+    const int it0 = (int)blockIdx.x * per;
+    const int it1 = it0 + per < total_items ? it0 + per : total_items;
+    if (it0 >= it1) return;
+    int gi = it0 / tpg, rb = it0 - gi * tpg;
 
     uint32_t bq[NTILE][NJ][2][2];
     unsigned need = 0;
@@ -831,13 +847,12 @@ __global__ void __launch_bounds__(SCAN_THREADS) scan_kernel(const StepArgs a) {
     const uint16_t* kbase = nullptr;
     const float scale = a.scale;
 
-    for (long long item = it0; item < it1; ++item) {
-        const int gi = (int)(item / tpg), rb = (int)(item - (long long)gi * tpg);
+    for (int item = it0; item < it1; ++item, ++rb) {
+        if (rb == tpg) { rb = 0; ++gi; }
         const int bkv = (a.mode == MODE_EXACT) ? gi : s_list[gi];
         if (bkv != cur) {
             cur = bkv;
-            const int b = bkv / a.Hkv, kvh = bkv % a.Hkv;
-            head0 = b * a.Hq + kvh * G;
+            head0 = bkv * G;                 // first query head of the group
             kbase = a.k + (size_t)bkv * a.max_seq_len * D;
             need = 0;
             if (a.mode == MODE_EXACT) need = (1u << G) - 1u;
@@ -938,8 +953,7 @@ __device__ void exact_path(const StepArgs& a, unsigned char* smem_raw) {
         reinterpret_cast<uint32_t*>(smem_raw) + ((2 * a.NS + a.NS / 2 + 3 * a.K + SCRATCH_WORDS + 32 + 8 + 3) & ~3));
 
     const int tid = threadIdx.x;
-    const int b = bh / a.Hq, h = bh % a.Hq;
-    const int bkv = b * a.Hkv + h / a.G;
+    const int bkv = kv_group_of(bh, a);
     const int K = a.K, L = a.L, NS = a.NS;
     const float* sc = a.ws_scores + (size_t)bh * a.score_stride;
     const float* tm = a.ws_tmax + (size_t)bh * a.tmax_stride;
