@@ -35,7 +35,11 @@
  *     current token;
  *   - grouped-query attention: cache, decision and support per query head h, keys and
  *     values of KV head h / (H_q / H_kv);
- *   - a zero query normalises to zero.
+ *   - a zero query normalises to zero;
+ *   - prefill seeding (Sec. 3.3: the cache "is initialized from the final C prompt tokens"):
+ *     the paper does not say which support a prompt token gets; here each of the last
+ *     n_tail <= M prompt positions p contributes its normalised query and its CAUSAL Exact
+ *     Top-K support over keys 0..p, oldest first; the decode offset stays 0.
  *
  * Inputs are bf16 bit patterns, widened exactly to double; every sum is a plain
  * left-to-right fp64 loop; selection is a full sort.  OpenMP only spreads independent
@@ -339,6 +343,43 @@ int oracle_decode_step(oracle_t *o, const uint16_t *q, const uint16_t *k, const 
     }
     o->n_ins += 1;
     o->t_dec += 1;
+    return 0;
+}
+
+/*
+ * Seed the caches from the last n_tail prompt positions (Sec. 3.3, first paragraph).
+ * q_tail [n_tail,B,Hq,d]: query of prompt position prompt_len - n_tail + j in slab j.
+ * Entry j gets the causal Exact Top-K support over keys 0 .. prompt_len - n_tail + j (Eq. 1).
+ */
+int oracle_prefill(oracle_t *o, const uint16_t *q_tail, const uint16_t *k, const uint16_t *v,
+                   int64_t prompt_len, int n_tail) {
+    if (n_tail < 1 || n_tail > o->M || n_tail > prompt_len || prompt_len > o->max_seq_len) return -1;
+    const int d = o->d, G = o->Hq / o->Hkv, K = o->K, M = o->M;
+    const size_t nh = (size_t)o->B * o->Hq;
+    for (int j = 0; j < n_tail; ++j) {
+        const int64_t L = prompt_len - n_tail + j + 1;
+        const int slot = (int)(o->n_ins % M);
+#pragma omp parallel for schedule(dynamic, 1)
+        for (long bh = 0; bh < (long)nh; ++bh) {
+            const int b = (int)(bh / o->Hq), h = (int)(bh % o->Hq);
+            const size_t kv = ((size_t)b * o->Hkv + h / G) * (size_t)o->max_seq_len * d;
+            double *qd = (double *)malloc((size_t)d * sizeof(double));
+            double *out = (double *)malloc((size_t)d * sizeof(double));
+            int32_t *sup = (int32_t *)malloc((size_t)K * sizeof(int32_t));
+            double kth, nrm2 = 0.0;
+            for (int t = 0; t < d; ++t) {
+                qd[t] = bf16_to_double(q_tail[((size_t)j * nh + bh) * d + t]);
+                nrm2 += qd[t] * qd[t];
+            }
+            exact_head(qd, k + kv, v + kv, L, d, K, sup, out, &kth);
+            const double nrm = sqrt(nrm2);
+            double *cq = o->qbar + ((size_t)bh * M + slot) * d;
+            for (int t = 0; t < d; ++t) cq[t] = nrm > 0.0 ? qd[t] / nrm : 0.0;
+            memcpy(o->sup + ((size_t)bh * M + slot) * K, sup, (size_t)K * sizeof(int32_t));
+            free(qd); free(out); free(sup);
+        }
+        o->n_ins += 1;
+    }
     return 0;
 }
 

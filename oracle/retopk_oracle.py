@@ -48,6 +48,8 @@ def _load():
         lib.oracle_decode_step.restype = i32
         lib.oracle_exact_topk.argtypes = [vp, vp, vp, vp, i64, vp, vp]
         lib.oracle_exact_topk.restype = i32
+        lib.oracle_prefill.argtypes = [vp, vp, vp, vp, i64, i32]
+        lib.oracle_prefill.restype = i32
         lib.oracle_stats.argtypes = [vp, vp]
         lib.oracle_stats.restype = None
         lib.oracle_last_step.argtypes = [vp] * 7
@@ -137,6 +139,17 @@ class Oracle:
         if rc != 0:
             raise ValueError(f"oracle_exact_topk failed with {rc}")
         return out, idx
+
+    def prefill(self, q_tail, k, v, prompt_len):
+        """Seed the caches from the last ``len(q_tail)`` prompt positions (causal Exact Top-K supports)."""
+        q_tail, k, v = _u16(q_tail), _u16(k), _u16(v)
+        self._check_kv(k, v)
+        n_tail = q_tail.shape[0]
+        if q_tail.shape != (n_tail, self.B, self.H_q, self.d):
+            raise ValueError("q_tail must be [n_tail, B, H_q, d]")
+        rc = self.lib.oracle_prefill(self.h, _ptr(q_tail), _ptr(k), _ptr(v), prompt_len, n_tail)
+        if rc != 0:
+            raise ValueError(f"oracle_prefill failed with {rc}")
 
     def stats(self) -> dict:
         five = np.zeros(5, dtype=np.int64)

@@ -349,3 +349,60 @@ def test_similarity_equal_to_tau_reuses(oracle_mod):
         o.decode_step(q, k, v, 10 + t)
         assert o.last_step()["path"][0, 0] == want[t]
     assert o.last_step()["rho_max"][0, 0] == 0.0
+
+
+# ------------------------------------------------------------------ prefill seeding (Sec. 3.3)
+
+def test_prefill_seeds_causal_exact_supports(oracle_mod):
+    """Each of the last n_tail prompt positions p enters with q/|q| and Top-K over keys 0..p."""
+    B, H_q, H_kv, d, M, K, P, n_tail = 1, 4, 2, 16, 6, 5, 40, 4
+    rng = np.random.default_rng(21)
+    k = bits(rng.standard_normal((B, H_kv, 64, d)))
+    v = bits(rng.standard_normal((B, H_kv, 64, d)))
+    q_tail = bits(rng.standard_normal((n_tail, B, H_q, d)))
+    o = oracle_mod.Oracle(B, H_q, H_kv, d, M, 2, 3, K, 0.5, 0, 64)
+    o.prefill(q_tail, k, v, P)
+    qbar, sup, n_ins, t_dec = o.export_state()
+    assert n_ins == n_tail and t_dec == 0
+    for j in range(n_tail):
+        L = P - n_tail + j + 1
+        for h in range(H_q):
+            q64 = wl.bf16_bits_to_f64(q_tail[j, 0, h])
+            want, _ = brute_topk(q64, wl.bf16_bits_to_f64(k[0, h // 2, :L]), K)
+            assert np.array_equal(sup[0, h, j], want)
+            assert sup[0, h, j].max() < L                       # causal: nothing beyond its own position
+            np.testing.assert_allclose(qbar[0, h, j], q64 / np.linalg.norm(q64), rtol=1e-15)
+    assert (sup[0, :, n_tail:] == -1).all()
+    assert sum(o.stats().values()) == 0                         # seeding is not a decode step
+
+
+def test_prefilled_cache_lets_the_first_step_reuse(oracle_mod):
+    """With a seeded cache the first decode step is no longer a forced fallback."""
+    cfg = wl.CONFIGS["tiny"].replace(context=300, steps=8, H_q=2, H_kv=1)
+    st = wl.make_stream(cfg, steps=8)
+    n_tail = cfg.M
+    # the prompt's last queries: the stream's first query repeated keeps every similarity at 1
+    q_tail = np.broadcast_to(st.q[0], (n_tail,) + st.q[0].shape).copy()
+    o = oracle_mod.Oracle.from_config(cfg, R=0)
+    o.prefill(q_tail, st.k, st.v, cfg.context)
+    for t in range(8):
+        o.decode_step(st.q[t], st.k, st.v, st.seq_len(t))
+        if t == 0:
+            last = o.last_step()
+            assert (last["path"] == oracle_mod.PATH_REUSE).all()
+            assert np.allclose(last["rho_max"], 1.0, atol=1e-12)
+    s = o.stats()
+    assert s["reuse"] >= 2 and s["refresh"] == 0
+    # without seeding the first step of every head falls back
+    o2 = oracle_mod.Oracle.from_config(cfg, R=0)
+    o2.decode_step(st.q[0], st.k, st.v, st.seq_len(0))
+    assert (o2.last_step()["path"] == oracle_mod.PATH_FALLBACK).all()
+
+
+def test_prefill_argument_checks(oracle_mod):
+    o = oracle_mod.Oracle(1, 1, 1, 8, 2, 1, 1, 2, 0.5, 0, 16)
+    k = bits(np.zeros((1, 1, 16, 8)))
+    with pytest.raises(ValueError):
+        o.prefill(bits(np.zeros((3, 1, 1, 8))), k, k, 10)      # more tail positions than cache slots
+    with pytest.raises(ValueError):
+        o.prefill(bits(np.zeros((2, 1, 1, 8))), k, k, 1)       # more tail positions than prompt tokens
