@@ -109,6 +109,19 @@ int retopk_decode_step(retopk_ctx* ctx, const void* q, const void* k_cache, cons
                        int64_t seq_len, void* out, void* stream);
 
 /*
+ * Seed the caches from the end of the prompt (Sec. 3.3: the cache "is initialized from the
+ * final C prompt tokens during prefill").  q_tail [n_tail,B,H_q,d] (device) holds the queries
+ * of prompt positions prompt_len - n_tail .. prompt_len - 1, oldest first; k_cache / v_cache
+ * hold the prompt's keys and values.  Entry j gets the normalised query of its position p and
+ * the CAUSAL Exact Top-K support over keys 0..p (Eq. 1 with L = p + 1; the paper leaves the
+ * supports of prompt tokens undefined).  1 <= n_tail <= min(M, prompt_len).  The insert count
+ * advances by n_tail, the decode offset t_dec and the counters do not change.  Costs n_tail
+ * full-history scans: a one-off at the end of prefill.
+ */
+int retopk_prefill(retopk_ctx* ctx, const void* q_tail, const void* k_cache, const void* v_cache,
+                   int64_t prompt_len, int n_tail, void* stream);
+
+/*
  * The same step for a caller whose per-token tensors live in HOST memory: copies q_host
  * [B,H_q,d] to the device, appends k_new_host / v_new_host [B,H_kv,d] at position
  * seq_len - 1 of the device-resident k_cache / v_cache, runs the step, copies the result

@@ -309,6 +309,31 @@ int retopk_decode_step(retopk_ctx* c, const void* q, const void* k_cache, const 
     return RETOPK_OK;
 }
 
+int retopk_prefill(retopk_ctx* c, const void* q_tail, const void* k_cache, const void* v_cache,
+                   int64_t prompt_len, int n_tail, void* stream) {
+    if (!c || !q_tail || !k_cache || !v_cache) return RETOPK_EINVAL;
+    if (n_tail < 1 || n_tail > c->M || n_tail > prompt_len || prompt_len > c->max_seq_len) return RETOPK_EINVAL;
+    if (!aligned16(q_tail) || !aligned16(k_cache) || !aligned16(v_cache)) return RETOPK_EINVAL;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t slab = (size_t)c->B * c->Hq * c->d;          // elements per prompt position
+    for (int j = 0; j < n_tail; ++j) {
+        // position p = prompt_len - n_tail + j sees keys 0..p: the exact path with L = p + 1
+        StepArgs a = make_args(c, static_cast<const uint16_t*>(q_tail) + (size_t)j * slab, k_cache, v_cache,
+                               prompt_len - n_tail + j + 1, c->stage_out, MODE_RETOPK);
+        a.refresh = 1;                 // every head takes the exact path
+        a.prefill = 1;                 // and nothing is counted
+        c->call_serial = (c->call_serial + 1) & 0x3fffffff;
+        a.step_id = c->call_serial;
+        int rc;
+        if ((rc = launch_recall(c, a, s)) != RETOPK_OK) return rc;
+        if ((rc = launch_scan(c, a, s)) != RETOPK_OK) return rc;
+        if ((rc = launch_finish(c, a, s)) != RETOPK_OK) return rc;
+        c->n_ins += 1;
+    }
+    c->last_launches = 3 * n_tail;
+    return RETOPK_OK;
+}
+
 int exact_topk_decode(retopk_ctx* c, const void* q, const void* k_cache, const void* v_cache,
                       int64_t seq_len, void* out, int32_t* idx_out, void* stream) {
     int rc = check_step_args(c, q, k_cache, v_cache, seq_len, out);

@@ -57,6 +57,7 @@ struct StepArgs {
     int slot;                // ring slot written by this step = n_inserted % M
     int refresh;             // 1 when Eq. 13's first case holds (known on the host)
     int mode;                // MODE_RETOPK or MODE_EXACT
+    int prefill;             // 1: cache seeding (every head exact, nothing counted)
     int NS;                  // entries in exact_finish_kernel's shared collection lists
     int g_shift;             // log2(G) when G is a power of two, else -1
     int step_id;             // call serial number; a KV group is flagged by storing it
@@ -615,7 +616,7 @@ __global__ void __launch_bounds__(RECALL_THREADS, 1) recall_kernel(const StepArg
             a.ws_gflag[bkv] = a.step_id;       // same value from every head of the group
             a.ws_gflag[a.B * a.Hkv] = a.step_id;   // "some group needs a scan in this step"
             a.ws_ncand[bh] = a.L;
-            atomicAdd(a.counters + (size_t)bh * 4 + path, 1ull);     // no return value: not waited for
+            if (!a.prefill) atomicAdd(a.counters + (size_t)bh * 4 + path, 1ull);   // no return value: not waited for
         }
     }
     RETOPK_PHASE(1, 2);
@@ -831,7 +832,7 @@ __global__ void __launch_bounds__(SCAN_THREADS) scan_kernel(const StepArgs a) {
         }
     if (n_act == 0) return;
     __syncthreads();
-    if (blockIdx.x == 0 && tid == 0) atomicAdd(a.scan_groups, (unsigned long long)n_act);
+    if (blockIdx.x == 0 && tid == 0 && !a.prefill) atomicAdd(a.scan_groups, (unsigned long long)n_act);
 
     const int tpg = (L + SCAN_TILE_ROWS - 1) / SCAN_TILE_ROWS;     // work items per group
     const int total_items = n_act * tpg;                            // < 2^31: checked on the host

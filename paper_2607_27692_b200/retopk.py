@@ -39,6 +39,7 @@ SIGNATURES = {
     "retopk_destroy": (_i32, [_vp]),
     "retopk_reset": (_i32, [_vp, _vp]),
     "retopk_decode_step": (_i32, [_vp, _vp, _vp, _vp, _i64, _vp, _vp]),
+    "retopk_prefill": (_i32, [_vp, _vp, _vp, _vp, _i64, _i32, _vp]),
     "retopk_decode_step_host": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _i64, _vp, _vp]),
     "exact_topk_decode": (_i32, [_vp, _vp, _vp, _vp, _i64, _vp, _vp, _vp]),
     "exact_topk_decode_static": (_i32, [_i32] * 5 + [_i64, _vp, _vp, _vp, _i64, _vp, _vp, _vp]),
@@ -152,6 +153,15 @@ class ReTopK:
                                          _dev(out, bf, self.q_shape), _stream())
         _check(rc, "retopk_decode_step")
         return out
+
+    def prefill(self, q_tail, k_cache, v_cache, prompt_len):
+        """Seed the caches from the last ``len(q_tail)`` prompt positions (q_tail [n_tail,B,H_q,d])."""
+        bf = torch.bfloat16
+        n_tail = int(q_tail.shape[0])
+        rc = self.lib.retopk_prefill(self.h, _dev(q_tail, bf, (n_tail,) + self.q_shape),
+                                     _dev(k_cache, bf, self.kv_shape), _dev(v_cache, bf, self.kv_shape),
+                                     prompt_len, n_tail, _stream())
+        _check(rc, "retopk_prefill")
 
     def decode_step_host(self, q_host, k_new_host, v_new_host, k_cache, v_cache, seq_len, out_host):
         bf = torch.bfloat16

@@ -279,3 +279,52 @@ def test_bad_arguments_return_errors(rt, P):
         g.decode_step(q, kv, kv, 257)
     with pytest.raises(rt.RetopkError):
         rt.ReTopK(1, 2, 1, 64, 4, 5, 8, 16, 0.9, 0, 256)     # r > M
+
+
+# ------------------------------------------------------------------ prefill seeding
+
+def test_prefill_seeding_matches_oracle(rt, P, oracle_mod):
+    """Caches seeded from the last M prompt positions, then free-running decode steps."""
+    cfg = wl.CONFIGS["tiny"].replace(context=3000, steps=12, B=2, H_q=8, H_kv=2, d=128, M=8, K=128)
+    st = wl.make_stream(cfg, steps=12)
+    rng = np.random.default_rng(5)
+    n_tail = cfg.M
+    q_tail = bits(rng.standard_normal((n_tail, cfg.B, cfg.H_q, cfg.d)))
+    # make the prompt's last query equal the first decode query: the first step can then reuse
+    q_tail[-1] = st.q[0]
+    o = oracle_mod.Oracle.from_config(cfg)
+    g = rt.ReTopK.from_config(cfg)
+    k, v = P.to_dev(st.k), P.to_dev(st.v)
+    o.prefill(q_tail, st.k, st.v, cfg.context)
+    g.prefill(P.to_dev(q_tail), k, v, cfg.context)
+    assert g.last_launch_count() == 3 * n_tail
+    qo, so, n_o, t_o = o.export_state()
+    qg, sg, n_g, t_g = g.export_state()
+    assert (n_g, t_g) == (n_o, t_o) == (n_tail, 0)
+    np.testing.assert_allclose(qg.cpu().numpy(), qo, atol=2e-6)
+    sg = sg.cpu().numpy()
+    G = cfg.H_q // cfg.H_kv
+    for j in range(n_tail):
+        L = cfg.context - n_tail + j + 1
+        for b in range(cfg.B):
+            for h in range(cfg.H_q):
+                q64 = wl.bf16_bits_to_f64(q_tail[j, b, h])
+                kth = (wl.bf16_bits_to_f64(st.k[b, h // G, so[b, h, j]]) @ q64 / np.sqrt(cfg.d)).min()
+                P.assert_support_matches(sg[b, h, j], so[b, h, j], q_tail[j, b, h], st.k[b, h // G], kth,
+                                         f"entry {j} seq {b} head {h}")
+                assert sg[b, h, j].max() < L
+    assert sum(v for key, v in g.stats().items() if key != "status") == 0     # seeding counts nothing
+    ex = P.teacher_forced_run(cfg, st, 12, o, g, k, v)
+    first_paths = None
+    assert o.stats()["reuse"] > 0
+    for key in ("steps", "refresh"):
+        assert g.stats()[key] == o.stats()[key]
+
+
+def test_prefill_argument_checks(rt, P):
+    g = rt.ReTopK(1, 2, 1, 64, 4, 2, 8, 16, 0.9, 0, 256)
+    kv = torch.zeros(g.kv_shape, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(rt.RetopkError):
+        g.prefill(torch.zeros((5, 1, 2, 64), dtype=torch.bfloat16, device="cuda"), kv, kv, 100)   # n_tail > M
+    with pytest.raises(rt.RetopkError):
+        g.prefill(torch.zeros((3, 1, 2, 64), dtype=torch.bfloat16, device="cuda"), kv, kv, 2)     # n_tail > prompt
