@@ -16,7 +16,7 @@ struct retopk_ctx {
     float tau;
     long long max_seq_len, score_stride, tmax_stride;
     long long n_ins, t_dec;
-    int NS, stage_depth, exact_stage_depth;
+    int NS, tile_cap, stage_depth, exact_stage_depth;
     int num_sms, scan_grid;
     int call_serial;
     size_t smem_recall, smem_reuse, smem_exact, smem_finish;
@@ -86,6 +86,7 @@ StepArgs make_args(const retopk_ctx* c, const void* q, const void* k, const void
     a.refresh = (c->R > 0 && c->t_dec > 0 && c->t_dec % c->R == 0) ? 1 : 0;
     a.mode = mode;
     a.NS = c->NS;
+    a.tile_cap = c->tile_cap;
     a.step_id = c->call_serial;
     a.g_shift = (c->G & (c->G - 1)) == 0 ? __builtin_ctz((unsigned)c->G) : -1;
     a.stage_depth = c->stage_depth;
@@ -159,6 +160,15 @@ void prof_done(retopk_ctx* c, int kind) {
     if (c->prof_events && c->prof_calls < c->prof_max) c->prof_kind[c->prof_calls++] = (unsigned char)kind;
 }
 
+// Sizes of the exact path's shared lists for a support size K (a trade between the range of
+// short histories handled without the tile bound and the room left for value-row copies).
+void exact_list_sizes(int K, int* NS, int* tile_cap) {
+    if (K <= 512) { *NS = 8192; *tile_cap = 4096; }
+    else if (K <= 1024) { *NS = 16384; *tile_cap = 8192; }
+    else if (K <= 2048) { *NS = 8192; *tile_cap = 4096; }
+    else { *NS = 8192; *tile_cap = 8192; }
+}
+
 int check_step_args(const retopk_ctx* c, const void* q, const void* k, const void* v, long long L,
                     const void* out) {
     if (!c || !q || !k || !v || !out) return RETOPK_EINVAL;
@@ -191,7 +201,9 @@ int retopk_create_batched(retopk_ctx** out, int B, int H_q, int H_kv, int d, int
     c->cap = r * K + W;
     c->score_stride = (max_seq_len + TILE_ROWS - 1) / TILE_ROWS * TILE_ROWS;   // whole 16-row tiles
     c->tmax_stride = ((max_seq_len + TILE_ROWS - 1) / TILE_ROWS + 3) / 4 * 4;
-    c->NS = 16 * K <= 8192 ? 8192 : 16384;
+    // exact path: shared lists for the scores that reach the tile bound (about 1.1-1.4 K of them,
+    // or all of L when L is short) and for the tiles that hold them
+    exact_list_sizes(K, &c->NS, &c->tile_cap);
     int sms = 0;
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, c->device);
     c->num_sms = sms > 0 ? sms : 148;
@@ -203,7 +215,7 @@ int retopk_create_batched(retopk_ctx** out, int B, int H_q, int H_kv, int d, int
     const size_t bm_words = (((size_t)max_seq_len + 31) / 32 + 3) & ~(size_t)3;
     c->smem_recall = ((size_t)d + ((M + 3) & ~3) + r + 4) * 4;
     c->smem_reuse = (head_words + big_words + bm_words) * 4;
-    c->smem_exact = (((size_t)c->NS * 2 + (size_t)c->NS / 2 + (size_t)K * 3 + SCRATCH_WORDS + 32 + 8 + 3) & ~(size_t)3) * 4;
+    c->smem_exact = (((size_t)c->NS * 2 + (size_t)c->tile_cap + (size_t)K * 3 + SCRATCH_WORDS + 32 + 8 + 3) & ~(size_t)3) * 4;
     int max_smem = 0;
     cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, c->device);
     // the rest of shared memory is the landing zone of the asynchronous row copies:
@@ -559,8 +571,9 @@ int exact_topk_decode_static(int B, int H_q, int H_kv, int d, int K, int64_t max
     int rc = static_setup(dev, &st);
     if (rc != RETOPK_OK) return rc;
 
-    const int NS = 16 * K <= 8192 ? 8192 : 16384;
-    size_t smem = (((size_t)NS * 2 + (size_t)NS / 2 + (size_t)K * 3 + SCRATCH_WORDS + 32 + 8 + 3) & ~(size_t)3) * 4;
+    int NS = 0, tile_cap = 0;
+    exact_list_sizes(K, &NS, &tile_cap);
+    size_t smem = (((size_t)NS * 2 + (size_t)tile_cap + (size_t)K * 3 + SCRATCH_WORDS + 32 + 8 + 3) & ~(size_t)3) * 4;
     const size_t wave = (size_t)FINISH_THREADS * 16;
     if ((size_t)st->max_smem < smem + wave) return RETOPK_EUNSUPPORTED;
     const int slots = FINISH_THREADS / (d / 8);
@@ -580,6 +593,7 @@ int exact_topk_decode_static(int B, int H_q, int H_kv, int d, int K, int64_t max
     a.scale = 1.0f / sqrtf((float)d);
     a.mode = MODE_EXACT;
     a.NS = NS;
+    a.tile_cap = tile_cap;
     a.g_shift = (a.G & (a.G - 1)) == 0 ? __builtin_ctz((unsigned)a.G) : -1;
     a.exact_stage_depth = (int)depth;
     a.q = static_cast<const uint16_t*>(q);

@@ -58,7 +58,8 @@ struct StepArgs {
     int refresh;             // 1 when Eq. 13's first case holds (known on the host)
     int mode;                // MODE_RETOPK or MODE_EXACT
     int prefill;             // 1: cache seeding (every head exact, nothing counted)
-    int NS;                  // entries in exact_finish_kernel's shared collection lists
+    int NS;                  // entries in the exact path's shared collection lists
+    int tile_cap;            // entries in the exact path's list of hit tiles
     int g_shift;             // log2(G) when G is a power of two, else -1
     int step_id;             // call serial number; a KV group is flagged by storing it
     int stage_depth;         // rows in flight per row slot in reuse_kernel's landing zone
@@ -937,13 +938,13 @@ __global__ void __launch_bounds__(SCAN_THREADS) scan_kernel(const StepArgs a) {
 template <int D, int NT>
 __device__ void exact_path(const StepArgs& a, unsigned char* smem_raw) {
     const int bh = blockIdx.x;
-    // layout (words): key[NS] idx[NS] (aliased later by red[NW*D+NT]) tile[NS/2]
+    // layout (words): key[NS] idx[NS] (aliased later by red[NW*D+NT]) tile[tile_cap]
     //                 sup_idx[K] sup_key[K] w[K] cnt[SCRATCH_WORDS] ws[32] misc[8] stage[depth*NT*4]
     uint32_t* s_key = reinterpret_cast<uint32_t*>(smem_raw);
     int32_t* s_idx = reinterpret_cast<int32_t*>(s_key + a.NS);
     float* s_red = reinterpret_cast<float*>(smem_raw);
     int32_t* s_tile = s_idx + a.NS;
-    int32_t* s_sup_idx = s_tile + a.NS / 2;
+    int32_t* s_sup_idx = s_tile + a.tile_cap;
     uint32_t* s_sup_key = reinterpret_cast<uint32_t*>(s_sup_idx + a.K);
     float* s_w = reinterpret_cast<float*>(s_sup_key + a.K);
     uint32_t* s_hist = reinterpret_cast<uint32_t*>(s_w + a.K);
@@ -951,7 +952,7 @@ __device__ void exact_path(const StepArgs& a, unsigned char* smem_raw) {
     int* s_misc = s_ws + 32;
     // landing zone of the value-row copies, on a 16-byte boundary
     uint4* s_stage = reinterpret_cast<uint4*>(
-        reinterpret_cast<uint32_t*>(smem_raw) + ((2 * a.NS + a.NS / 2 + 3 * a.K + SCRATCH_WORDS + 32 + 8 + 3) & ~3));
+        reinterpret_cast<uint32_t*>(smem_raw) + ((2 * a.NS + a.tile_cap + 3 * a.K + SCRATCH_WORDS + 32 + 8 + 3) & ~3));
 
     const int tid = threadIdx.x;
     const int bkv = kv_group_of(bh, a);
@@ -970,7 +971,7 @@ __device__ void exact_path(const StepArgs& a, unsigned char* smem_raw) {
         __syncthreads();
     } else {
         const int ntile = (L + TILE_ROWS - 1) / TILE_ROWS;
-        const int tcap = NS / 2;
+        const int tcap = a.tile_cap;
         // 1. lower bound v for the K-th score from the tile maxima (grouped so the list is short)
         uint32_t thr_key = 0;
         int sh = 0;                                  // groups of g2 = 2^sh tiles
