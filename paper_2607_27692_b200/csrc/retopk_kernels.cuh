@@ -1010,7 +1010,7 @@ __device__ void exact_path(const StepArgs& a, unsigned char* smem_raw) {
             }
             __syncthreads();
             RETOPK_PHASE(2, 8);
-            thr_key = count_threshold<NT>(s_key, n2, K, 12, reinterpret_cast<int*>(s_hist)).v;
+            thr_key = count_threshold<NT>(s_key, n2, K, 16, reinterpret_cast<int*>(s_hist)).v;
         }
         RETOPK_PHASE(2, 1);
         // 2. the tiles whose maximum reaches v, in ascending order (two chunks of four tile
