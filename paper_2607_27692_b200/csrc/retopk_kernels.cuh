@@ -1013,37 +1013,31 @@ __device__ void exact_path(const StepArgs& a, unsigned char* smem_raw) {
             thr_key = count_threshold<NT>(s_key, n2, K, 16, reinterpret_cast<int*>(s_hist)).v;
         }
         RETOPK_PHASE(2, 1);
-        // 2. the tiles whose maximum reaches v, in ascending order (two chunks of four tile
-        //    maxima per thread are requested before the first prefix sum)
+        // 2. the tiles whose maximum reaches v, in ascending order: eight consecutive tile
+        //    maxima per thread and one prefix sum per 8 * NT tiles
         int nhit = 0;
         for (int base = 0; base < ntile; base += NT * 8) {
+            const int t0 = base + tid * 8;
             float4 m4[2];
 #pragma unroll
-            for (int u = 0; u < 2; ++u) {
-                const int t0 = base + u * NT * 4 + tid * 4;
-                m4[u] = t0 < ntile ? *reinterpret_cast<const float4*>(tm + t0) : make_float4(0.f, 0.f, 0.f, 0.f);
-            }
+            for (int u = 0; u < 2; ++u)
+                m4[u] = t0 + 4 * u < ntile ? *reinterpret_cast<const float4*>(tm + t0 + 4 * u)
+                                           : make_float4(0.f, 0.f, 0.f, 0.f);
+            if (base == 0) RETOPK_PHASE(2, 11);
+            const float mv[8] = {m4[0].x, m4[0].y, m4[0].z, m4[0].w, m4[1].x, m4[1].y, m4[1].z, m4[1].w};
+            unsigned hits = 0;
 #pragma unroll
-            for (int u = 0; u < 2; ++u) {
-                const int t0 = base + u * NT * 4 + tid * 4;
-                int f[4] = {0, 0, 0, 0}, cnt = 0;
-                if (t0 < ntile) {
-                    f[0] = score_key(m4[u].x) >= thr_key;
-                    f[1] = (t0 + 1 < ntile) && score_key(m4[u].y) >= thr_key;
-                    f[2] = (t0 + 2 < ntile) && score_key(m4[u].z) >= thr_key;
-                    f[3] = (t0 + 3 < ntile) && score_key(m4[u].w) >= thr_key;
-                    cnt = f[0] + f[1] + f[2] + f[3];
-                }
-                int total;
-                int pos = nhit + block_excl_scan<NT>(cnt, s_ws, total);
-#pragma unroll
-                for (int e = 0; e < 4; ++e)
-                    if (f[e]) {
-                        if (pos < tcap) s_tile[pos] = t0 + e;
-                        ++pos;
-                    }
-                nhit += total;
+            for (int e = 0; e < 8; ++e)
+                if (t0 + e < ntile && score_key(mv[e]) >= thr_key) hits |= 1u << e;
+            int total;
+            int pos = nhit + block_excl_scan<NT>(__popc(hits), s_ws, total);
+            while (hits) {
+                const int e = __ffs(hits) - 1;
+                if (pos < tcap) s_tile[pos] = t0 + e;
+                ++pos;
+                hits &= hits - 1;
             }
+            nhit += total;
         }
         __syncthreads();
         RETOPK_PHASE(2, 2);
@@ -1067,19 +1061,15 @@ __device__ void exact_path(const StepArgs& a, unsigned char* smem_raw) {
                             if (row0 + 4 * u + e < L && score_key(v4[e]) >= thr_key) fl |= 1u << (4 * u + e);
                     }
                 }
+                RETOPK_PHASE(2, 9);
                 int total;
                 int pos = n + block_excl_scan<NT>(__popc(fl), s_ws, total);
-                if (fl) {
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        const float v4[4] = {x[u].x, x[u].y, x[u].z, x[u].w};
-#pragma unroll
-                        for (int e = 0; e < 4; ++e)
-                            if ((fl >> (4 * u + e)) & 1u) {
-                                if (pos < NS) { s_key[pos] = score_key(v4[e]); s_idx[pos] = row0 + 4 * u + e; }
-                                ++pos;
-                            }
-                    }
+                RETOPK_PHASE(2, 10);
+                while (fl) {
+                    const int e = __ffs(fl) - 1;
+                    if (pos < NS) { s_key[pos] = score_key(sc[row0 + e]); s_idx[pos] = row0 + e; }
+                    ++pos;
+                    fl &= fl - 1;
                 }
                 n += total;
             }
