@@ -122,6 +122,28 @@ __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commi
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void cp_async_wait_but_one() { asm volatile("cp.async.wait_group 1;" ::: "memory"); }
 
+// L2 residency hints for the scan: key rows are read once (first to go), scores and tile
+// maxima are read again by the finish kernel (last to go).
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_last() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ uint4 ldg_stream_hint(const void* p, uint64_t policy) {
+    uint4 r;
+    asm volatile("ld.global.nc.L1::no_allocate.L2::cache_hint.v4.u32 {%0,%1,%2,%3}, [%4], %5;"
+                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p), "l"(policy));
+    return r;
+}
+__device__ __forceinline__ void stg_hint(float* p, float v, uint64_t policy) {
+    asm volatile("st.global.L2::cache_hint.f32 [%0], %1, %2;" :: "l"(p), "f"(v), "l"(policy) : "memory");
+}
+
 __device__ __forceinline__ float dot8(const uint4& x, const float* qf) {
     float a = bf16_lo(x.x) * qf[0];
     a = fmaf(bf16_hi(x.x), qf[1], a);
@@ -843,6 +865,7 @@ __global__ void __launch_bounds__(SCAN_THREADS) scan_kernel(const StepArgs a) {
     if (it0 >= it1) return;
     int gi = it0 / tpg, rb = it0 - gi * tpg;
 
+    const uint64_t pol_first = l2_policy_evict_first(), pol_last = l2_policy_evict_last();
     uint32_t bq[NTILE][NJ][2][2];
     unsigned need = 0;
     int cur = -1, head0 = 0;
@@ -887,8 +910,8 @@ __global__ void __launch_bounds__(SCAN_THREADS) scan_kernel(const StepArgs a) {
             const uint16_t* p1 = kbase + (size_t)c1 * D + t * 8;
 #pragma unroll
             for (int j = 0; j < NJ; ++j) {
-                x[s][j] = ldg_stream(p0 + j * 32);
-                y[s][j] = ldg_stream(p1 + j * 32);
+                x[s][j] = ldg_stream_hint(p0 + j * 32, pol_first);
+                y[s][j] = ldg_stream_hint(p1 + j * 32, pol_first);
             }
         }
 #pragma unroll
@@ -914,10 +937,10 @@ __global__ void __launch_bounds__(SCAN_THREADS) scan_kernel(const StepArgs a) {
                     m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 16));
                     if (head < G && ((need >> head) & 1u)) {
                         float* srow = a.ws_scores + (size_t)(head0 + head) * a.score_stride;
-                        if (r0 < L) srow[r0] = c[e] * scale;
-                        if (r1 < L) srow[r1] = c[2 + e] * scale;
+                        if (r0 < L) stg_hint(srow + r0, c[e] * scale, pol_last);
+                        if (r1 < L) stg_hint(srow + r1, c[2 + e] * scale, pol_last);
                         if (g == 0 && tile_row < L)
-                            a.ws_tmax[(size_t)(head0 + head) * a.tmax_stride + (tile_row >> 4)] = m * scale;
+                            stg_hint(a.ws_tmax + (size_t)(head0 + head) * a.tmax_stride + (tile_row >> 4), m * scale, pol_last);
                     }
                 }
             }
