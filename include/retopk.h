@@ -187,9 +187,11 @@ int retopk_import_state(retopk_ctx* ctx, const float* qbar, const int32_t* suppo
  *
  * The first call on a device looks up the array's device address and opts the kernels in to
  * large shared memory; make that first call outside any stream capture.  No call allocates,
- * frees or synchronises.  All calls on a device share the one array: its contents are
- * rewritten by every call before they are read (nothing needs to start at zero), and two
- * calls that overlap on the GPU (different streams, no dependency) race on it.
+ * frees or synchronises.  All calls on a device share the one array: scores and tile maxima
+ * are rewritten by every call before they are read; the one word that must start at zero
+ * (the scan's work counter) is zero in the library image and is put back to zero by the
+ * last kernel of every call.  Two calls that overlap on the GPU (different streams, no
+ * dependency) race on the array.
  */
 #define RETOPK_STATIC_SCRATCH_BYTES (32u << 20)
 int exact_topk_decode_static(int B, int H_q, int H_kv, int d, int K, int64_t max_seq_len, const void* q,

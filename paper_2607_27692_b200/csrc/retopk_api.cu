@@ -34,6 +34,7 @@ struct retopk_ctx {
     unsigned int* status;
     unsigned long long* slow_select;
     unsigned long long* scan_groups;
+    unsigned int* scan_counter;
     // per-kernel event timing (measurement hook)
     cudaEvent_t* prof_events;
     int prof_max, prof_calls;
@@ -67,7 +68,7 @@ bool dev_alloc(T** p, size_t count) {
 void free_all(retopk_ctx* c) {
     cudaFree(c->qbar_cache); cudaFree(c->sup_cache); cudaFree(c->ws_path); cudaFree(c->ws_rho);
     cudaFree(c->ws_ncand); cudaFree(c->ws_sel); cudaFree(c->ws_gflag); cudaFree(c->ws_scores); cudaFree(c->ws_tmax); cudaFree(c->counters);
-    cudaFree(c->status); cudaFree(c->slow_select); cudaFree(c->scan_groups); cudaFree(c->stage_q); cudaFree(c->stage_out);
+    cudaFree(c->status); cudaFree(c->slow_select); cudaFree(c->scan_groups); cudaFree(c->scan_counter); cudaFree(c->stage_q); cudaFree(c->stage_out);
     cudaFree(c->stage_kv);
 }
 
@@ -100,6 +101,7 @@ StepArgs make_args(const retopk_ctx* c, const void* q, const void* k, const void
     a.ws_scores = c->ws_scores; a.ws_tmax = c->ws_tmax; a.tmax_stride = c->tmax_stride; a.counters = c->counters; a.status = c->status;
     a.slow_select = c->slow_select;
     a.scan_groups = c->scan_groups;
+    a.scan_counter = c->scan_counter;
     a.idx_out = nullptr;
     return a;
 }
@@ -264,7 +266,7 @@ int retopk_create_batched(retopk_ctx** out, int B, int H_q, int H_kv, int d, int
               dev_alloc(&c->ws_sel, nh * r) && dev_alloc(&c->ws_gflag, (size_t)B * H_kv + 1) && dev_alloc(&c->ws_scores, nh * (size_t)c->score_stride) &&
               dev_alloc(&c->ws_tmax, nh * (size_t)c->tmax_stride) &&
               dev_alloc(&c->counters, nh * 4) && dev_alloc(&c->status, 1) &&
-              dev_alloc(&c->slow_select, 1) && dev_alloc(&c->scan_groups, 1) && dev_alloc(&c->stage_q, nh * d) &&
+              dev_alloc(&c->slow_select, 1) && dev_alloc(&c->scan_groups, 1) && dev_alloc(&c->scan_counter, 1) && dev_alloc(&c->stage_q, nh * d) &&
               dev_alloc(&c->stage_out, nh * d) && dev_alloc(&c->stage_kv, (size_t)2 * B * H_kv * d);
     if (!ok) { cudaGetLastError(); free_all(c); delete c; return RETOPK_ENOMEM; }
     *out = c;
@@ -293,7 +295,7 @@ int retopk_reset(retopk_ctx* c, void* stream) {
     const size_t nh = (size_t)c->B * c->Hq;
     reset_kernel<<<c->num_sms * 4, 256, 0, static_cast<cudaStream_t>(stream)>>>(
         c->qbar_cache, nh * c->M * c->d, c->sup_cache, nh * c->M * c->K, c->counters, nh * 4, c->ws_gflag,
-        (size_t)c->B * c->Hkv + 1, c->status, c->slow_select, c->scan_groups);
+        (size_t)c->B * c->Hkv + 1, c->status, c->slow_select, c->scan_groups, c->scan_counter);
     c->n_ins = 0;
     c->t_dec = 0;
     return cudaGetLastError() == cudaSuccess ? RETOPK_OK : RETOPK_ECUDA;
@@ -604,6 +606,7 @@ int exact_topk_decode_static(int B, int H_q, int H_kv, int d, int K, int64_t max
     // the two diagnostic counters the kernels add to are sinks here; they need no clearing
     a.slow_select = reinterpret_cast<unsigned long long*>(st->scratch);
     a.scan_groups = reinterpret_cast<unsigned long long*>(st->scratch + 8);
+    a.scan_counter = reinterpret_cast<unsigned int*>(st->scratch + 16);   // zero in the image, reset by every finish
     a.ws_scores = reinterpret_cast<float*>(st->scratch + 256);
     a.ws_tmax = a.ws_scores + nh * score_stride;
 

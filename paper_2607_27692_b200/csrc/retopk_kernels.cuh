@@ -30,8 +30,17 @@ __device__ long long g_phase_clk[3][1024][16];
     do {                                                                                   \
         if (threadIdx.x == 0 && blockIdx.x < 1024) g_phase_clk[kernel][blockIdx.x][n] = clock64(); \
     } while (0)
+#define RETOPK_WALL(kernel, n)                                                              \
+    do {                                                                                   \
+        if (threadIdx.x == 0 && blockIdx.x < 1024) {                                       \
+            unsigned long long t_;                                                         \
+            asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_));                          \
+            g_phase_clk[kernel][blockIdx.x][n] = (long long)t_;                            \
+        }                                                                                  \
+    } while (0)
 #else
 #define RETOPK_PHASE(kernel, n) do { } while (0)
+#define RETOPK_WALL(kernel, n) do { } while (0)
 #endif
 
 namespace retopk {
@@ -82,6 +91,7 @@ struct StepArgs {
     unsigned int* status;
     unsigned long long* slow_select;
     unsigned long long* scan_groups;
+    unsigned int* scan_counter;  // pool cursor of scan_kernel; finish_kernel resets it
     int32_t* idx_out;        // MODE_EXACT only, may be null
 };
 
@@ -549,7 +559,9 @@ __global__ void __launch_bounds__(RECALL_THREADS, 1) recall_kernel(const StepArg
     const int bkv = kv_group_of(bh, a);
     const int M = a.M, fill = a.fill;
 
+    RETOPK_WALL(1, 13);
     pdl_wait();        // the caches were written by the step before; q by whatever ran before this call
+    RETOPK_WALL(1, 14);
     RETOPK_PHASE(1, 0);
     // Every warp reads the query itself (four elements per lane) next to its cache rows, so
     // one memory latency covers both:  rho_c = (qbar_c . q) / |q|   (Eq. 6)
@@ -643,6 +655,7 @@ __global__ void __launch_bounds__(RECALL_THREADS, 1) recall_kernel(const StepArg
         }
     }
     RETOPK_PHASE(1, 2);
+    RETOPK_WALL(1, 15);
 }
 
 // ------------------------------------------------------------------------------------
@@ -835,6 +848,7 @@ __global__ void __launch_bounds__(SCAN_THREADS) scan_kernel(const StepArgs a) {
     const int g = lane >> 2, t = lane & 3;
     const int G = a.G, L = a.L;
     const int n_groups = a.B * a.Hkv;
+    RETOPK_WALL(0, 13);
     // No trigger for the dependent launch behind this kernel: its CTAs take a whole SM each
     // and start as this kernel's CTAs exit; that already hides its launch latency.
 
@@ -857,13 +871,15 @@ __global__ void __launch_bounds__(SCAN_THREADS) scan_kernel(const StepArgs a) {
     __syncthreads();
     if (blockIdx.x == 0 && tid == 0 && !a.prefill) atomicAdd(a.scan_groups, (unsigned long long)n_act);
 
+    // Work items of 256 rows.  Seven eighths of them are handed out as one contiguous share
+    // per CTA (locality, no traffic on the counter); the rest sit in a pool that the CTAs
+    // drain one item at a time as they finish, so that the kernel ends on all SMs together
+    // (with fixed shares alone the last CTA finished 13 us after the first).
     const int tpg = (L + SCAN_TILE_ROWS - 1) / SCAN_TILE_ROWS;     // work items per group
     const int total_items = n_act * tpg;                            // < 2^31: checked on the host
-    const int per = (total_items + (int)gridDim.x - 1) / (int)gridDim.x;
-    const int it0 = (int)blockIdx.x * per;
-    const int it1 = it0 + per < total_items ? it0 + per : total_items;
-    if (it0 >= it1) return;
-    int gi = it0 / tpg, rb = it0 - gi * tpg;
+    const int per = (int)(((long long)total_items * 7 / 8) / (int)gridDim.x);
+    const int pool0 = per * (int)gridDim.x;                         // first item of the pool
+    __shared__ int s_next;
 
     const uint64_t pol_first = l2_policy_evict_first(), pol_last = l2_policy_evict_last();
     uint32_t bq[NTILE][NJ][2][2];
@@ -872,8 +888,21 @@ __global__ void __launch_bounds__(SCAN_THREADS) scan_kernel(const StepArgs a) {
     const uint16_t* kbase = nullptr;
     const float scale = a.scale;
 
-    for (int item = it0; item < it1; ++item, ++rb) {
-        if (rb == tpg) { rb = 0; ++gi; }
+    int item = (int)blockIdx.x * per;
+    int left = per;                      // items left in the fixed share
+    int grabbed = 0;                     // thread 0: pool item requested ahead of time
+    if (left == 0) {
+        if (tid == 0) s_next = pool0 + (int)atomicAdd(a.scan_counter, 1u);
+        __syncthreads();
+        item = s_next;
+        __syncthreads();
+    }
+    while (item < total_items) {
+        // ask for the next pool item now; the answer is only needed after this item
+        const bool last_fixed = left == 1, in_pool = left == 0;
+        if ((last_fixed || in_pool) && tid == 0) grabbed = pool0 + (int)atomicAdd(a.scan_counter, 1u);
+        const int gi = item / tpg, rb = item - gi * tpg;
+
         const int bkv = (a.mode == MODE_EXACT) ? gi : s_list[gi];
         if (bkv != cur) {
             cur = bkv;
@@ -945,7 +974,16 @@ __global__ void __launch_bounds__(SCAN_THREADS) scan_kernel(const StepArgs a) {
                 }
             }
         }
+        if (left > 1) { ++item; --left; }
+        else {
+            if (left == 1) left = 0;
+            if (tid == 0) s_next = grabbed;
+            __syncthreads();
+            item = s_next;
+            __syncthreads();
+        }
     }
+    RETOPK_WALL(0, 15);
 }
 
 // ------------------------------------------------------------------------------------
@@ -1137,22 +1175,26 @@ __device__ void exact_path(const StepArgs& a, unsigned char* smem_raw) {
 template <int D>
 __global__ void __launch_bounds__(FINISH_THREADS, 1) finish_kernel(const StepArgs a) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
+    RETOPK_WALL(2, 13);
     pdl_wait();        // scores and tile maxima come from the scan, recalled slots and paths from recall_kernel
+    RETOPK_WALL(2, 14);
+    if (blockIdx.x == 0 && threadIdx.x == 0) *a.scan_counter = 0u;      // the scan before this kernel is complete
     if (a.mode == MODE_RETOPK && a.ws_path[blockIdx.x] == PATH_REUSE) reuse_path<D, FINISH_THREADS>(a, smem_raw);
     else exact_path<D, FINISH_THREADS>(a, smem_raw);
+    RETOPK_WALL(2, 15);
 }
 
 // Clear the caches (supports to -1, queries and counters to 0).
 __global__ void reset_kernel(float* qbar, size_t n_q, int32_t* sup, size_t n_sup, unsigned long long* counters,
                              size_t n_cnt, int32_t* gflag, size_t n_flag, unsigned int* status,
-                             unsigned long long* slow, unsigned long long* groups) {
+                             unsigned long long* slow, unsigned long long* groups, unsigned int* scan_counter) {
     const size_t stride = (size_t)gridDim.x * blockDim.x;
     const size_t t0 = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     for (size_t i = t0; i < n_q; i += stride) qbar[i] = 0.f;
     for (size_t i = t0; i < n_sup; i += stride) sup[i] = -1;
     for (size_t i = t0; i < n_cnt; i += stride) counters[i] = 0;
     for (size_t i = t0; i < n_flag; i += stride) gflag[i] = -1;
-    if (t0 == 0) { *status = 0u; *slow = 0ull; *groups = 0ull; }
+    if (t0 == 0) { *status = 0u; *slow = 0ull; *groups = 0ull; *scan_counter = 0u; }
 }
 
 }  // namespace retopk
