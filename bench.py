@@ -230,6 +230,43 @@ def path_mix(stats):
         "mean_candidates": round(stats["cand_sum"] / max(stats["reuse"], 1), 1)}
 
 
+def fidelity_pass(layers, torch, calls=96):
+    """Support recall and output cosine of ReTopK against Exact Top-K on the same inputs.
+
+    A diagnostic outside every timed region (torch only compares index sets and outputs):
+    after each ReTopK call the library's Exact Top-K runs on the identical inputs.
+    """
+    cfg = layers.cfg
+    stream = torch.cuda.current_stream().cuda_stream
+    for c in layers.ctx:
+        c.reset()
+    idx = torch.empty((cfg.B, cfg.H_q, cfg.K), dtype=torch.int32, device="cuda")
+    out_exact = torch.empty_like(layers.out)
+    qstep = cfg.B * cfg.H_q * cfg.d * 2
+    recalls, cosines = [], []
+    for i in range(calls):
+        l, t = i % layers.n, i // layers.n
+        L = cfg.context + t + 1
+        layers.call(i, "retopk", stream)
+        last = layers.ctx[l].last_step()
+        rc = layers.lib.exact_topk_decode(layers.ctx[l].h, layers.q[l].data_ptr() + t * qstep, layers.k[l].data_ptr(),
+                                          layers.v[l].data_ptr(), L, out_exact.data_ptr(), idx.data_ptr(), stream)
+        if rc != 0:
+            raise RuntimeError(f"exact_topk_decode failed with {rc}")
+        hit = (last["support"].unsqueeze(-1) == idx.unsqueeze(-2)).any(-1).sum(-1).float() / cfg.K
+        reuse = last["path"] == 0
+        if reuse.any():
+            recalls.append(hit[reuse])
+        a, b = layers.out.float(), out_exact.float()
+        cosines.append((a * b).sum(-1) / (a.norm(dim=-1) * b.norm(dim=-1)).clamp_min(1e-20))
+    rec = torch.cat(recalls) if recalls else torch.zeros(1, device="cuda")
+    cos = torch.cat([c.flatten() for c in cosines])
+    return {"calls": calls, "support_recall_on_reuse_heads": round(float(rec.mean()), 4),
+            "output_cosine_mean": round(float(cos.mean()), 5), "output_cosine_min": round(float(cos.min()), 4),
+            "note": "vs this library's Exact Top-K on identical inputs; the paper reports 56.9% recall and "
+                    "97.4% output cosine on reuse steps for Qwen2.5-7B on PG19 (other data: context only)"}
+
+
 def cpu_baseline(cfg, stream, budget_s=12.0, max_steps=48):
     """The fp64 oracle, as it stands, on the first decode steps of layer 0."""
     from oracle import retopk_oracle
@@ -282,6 +319,7 @@ def run_gpu(args):
     fallb = timed_pass(layers, "retopk", W, K, torch, dist)
     layers.make_contexts(tau=0.85)
     paper = timed_pass(layers, "retopk", W, K, torch, dist)
+    fidelity = fidelity_pass(layers, torch, calls=min(96, W + K)) if rank == 0 else None
 
     # roofline of the dominant kernel of the headline pass
     abytes = algorithmic_bytes(cfg, prof["stats"], mean_L, mean_fill)
@@ -338,6 +376,7 @@ def run_gpu(args):
         "paths": {"pure_reuse": path_report(reuse, False), "pure_exact": path_report(fallb, True),
                   "tau_0.85": path_report(paper, False)},
         "slow_select": head["stats"]["slow_select"],
+        "fidelity_tau_0.85": fidelity,
         "roofline": roofline,
         "paper_context": "paper: 3.07x attention speedup over Exact Top-K at 128K, K=512 on one NVIDIA L20 "
                          "(Qwen2.5-7B, PG19, tau=0.85); about 115 us per layer at 128K (Table 4 / 28 layers)",
