@@ -36,6 +36,10 @@
  *   - grouped-query attention: cache, decision and support per query head h, keys and
  *     values of KV head h / (H_q / H_kv);
  *   - a zero query normalises to zero;
+ *   - "recent" recall (the component study's Recent-R row, Table 3): the min(r, fill) most
+ *     recently inserted entries are recalled instead of the most similar ones, and rho_max is
+ *     the largest similarity among THOSE entries (the paper gives no formula; the row's
+ *     higher exact-path share fits a maximum taken over fewer entries);
  *   - prefill seeding (Sec. 3.3: the cache "is initialized from the final C prompt tokens"):
  *     the paper does not say which support a prompt token gets; here each of the last
  *     n_tail <= M prompt positions p contributes its normalised query and its CAUSAL Exact
@@ -67,6 +71,7 @@ enum { PATH_REUSE = 0, PATH_FALLBACK = 1, PATH_REFRESH = 2 };
 
 typedef struct {
     int B, Hq, Hkv, d, M, r, W, K, R;
+    int recall_mode; /* 0: the r most similar cached queries (Eq. 7); 1: the r most recent ones */
     double tau;
     int64_t max_seq_len;
     int64_t n_ins;   /* entries inserted so far (same for every head) */
@@ -138,6 +143,13 @@ int oracle_create(oracle_t **out, int B, int Hq, int Hkv, int d, int M, int r, i
     memset(o->last_sup, 0xFF, nh * K * sizeof(int32_t));
     memset(o->last_sel, 0xFF, nh * r * sizeof(int32_t));
     *out = o;
+    return 0;
+}
+
+/* 0: similarity recall (the method); 1: recency recall (the Recent-R ablation row); r <= 64 then. */
+int oracle_set_recall_mode(oracle_t *o, int mode) {
+    if ((mode != 0 && mode != 1) || (mode == 1 && o->r > 64)) return -1;
+    o->recall_mode = mode;
     return 0;
 }
 
@@ -258,6 +270,17 @@ static void retopk_head(oracle_t *o, size_t bh, const double *q, const uint16_t 
         if (acc > rho_max) rho_max = acc;
     }
 
+    /* recall set: all entries ranked by similarity, or just the newest min(r, fill) */
+    const int n_recall = r < fill ? r : fill;
+    int recent[64];
+    if (o->recall_mode == 1) {
+        rho_max = -INFINITY;
+        for (int j = 0; j < n_recall; ++j) {
+            recent[j] = (int)(((o->n_ins - 1 - j) % M + M) % M);      /* j = 0 is the newest */
+            if (rho[recent[j]].val > rho_max) rho_max = rho[recent[j]].val;
+        }
+    }
+
     /* Eq. 13 */
     int path;
     if (o->R > 0 && o->t_dec > 0 && o->t_dec % o->R == 0) path = PATH_REFRESH;
@@ -271,8 +294,14 @@ static void retopk_head(oracle_t *o, size_t bh, const double *q, const uint16_t 
     int n_scored;
 
     if (path == PATH_REUSE) {
-        int n_sel = r < fill ? r : fill;
-        qsort(rho, (size_t)fill, sizeof *rho, cmp_scored);
+        int n_sel = n_recall;
+        if (o->recall_mode == 1) {
+            scored_t tmp[64];
+            for (int j = 0; j < n_sel; ++j) tmp[j] = rho[recent[j]];
+            for (int j = 0; j < n_sel; ++j) rho[j] = tmp[j];          /* newest first */
+        } else {
+            qsort(rho, (size_t)fill, sizeof *rho, cmp_scored);
+        }
         /* Eq. 8-9: union of recalled supports and the recent window, sorted, unique */
         int32_t *raw = (int32_t *)malloc((size_t)(cap + 1) * sizeof(int32_t));
         int n_raw = 0;

@@ -50,6 +50,8 @@ def _load():
         lib.oracle_exact_topk.restype = i32
         lib.oracle_prefill.argtypes = [vp, vp, vp, vp, i64, i32]
         lib.oracle_prefill.restype = i32
+        lib.oracle_set_recall_mode.argtypes = [vp, i32]
+        lib.oracle_set_recall_mode.restype = i32
         lib.oracle_stats.argtypes = [vp, vp]
         lib.oracle_stats.restype = None
         lib.oracle_last_step.argtypes = [vp] * 7
@@ -150,6 +152,11 @@ class Oracle:
         rc = self.lib.oracle_prefill(self.h, _ptr(q_tail), _ptr(k), _ptr(v), prompt_len, n_tail)
         if rc != 0:
             raise ValueError(f"oracle_prefill failed with {rc}")
+
+    def set_recall_mode(self, mode: int):
+        """0: recall the most similar entries (the method); 1: the most recent ones (Recent-R ablation)."""
+        if self.lib.oracle_set_recall_mode(self.h, mode) != 0:
+            raise ValueError("bad recall mode")
 
     def stats(self) -> dict:
         five = np.zeros(5, dtype=np.int64)

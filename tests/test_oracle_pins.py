@@ -406,3 +406,52 @@ def test_prefill_argument_checks(oracle_mod):
         o.prefill(bits(np.zeros((3, 1, 1, 8))), k, k, 10)      # more tail positions than cache slots
     with pytest.raises(ValueError):
         o.prefill(bits(np.zeros((2, 1, 1, 8))), k, k, 1)       # more tail positions than prompt tokens
+
+
+# ------------------------------------------------------------------ Recent-R recall (Table 3 ablation row)
+
+def test_recent_recall_takes_the_newest_entries(oracle_mod):
+    B, H, d, M, r, K, L = 1, 2, 16, 6, 3, 4, 64
+    rng = np.random.default_rng(31)
+    qc = rng.standard_normal((B, H, M, d))
+    qc /= np.linalg.norm(qc, axis=-1, keepdims=True)
+    sup = np.sort(rng.permuted(np.tile(np.arange(L - 4), (B, H, M, 1)), axis=-1)[..., :K], axis=-1).astype(np.int32)
+    n_ins = 10                                   # ring of 6: newest entries sit in slots 3, 2, 1
+    q, k, v = random_case(9, B, H, H, d, L, L)
+    o = oracle_mod.Oracle(B, H, H, d, M, r, 2, K, -2.0, 0, L)
+    o.set_recall_mode(1)
+    o.import_state(qc, sup, n_ins, 4)
+    o.decode_step(q, k, v, L)
+    last = o.last_step()
+    q64 = wl.bf16_bits_to_f64(q)
+    for h in range(H):
+        assert list(last["sel"][0, h]) == [3, 2, 1]
+        qb = q64[0, h] / np.linalg.norm(q64[0, h])
+        assert last["rho_max"][0, h] == pytest.approx((qc[0, h, [3, 2, 1]] @ qb).max(), abs=1e-14)
+        union = np.union1d(np.unique(sup[0, h, [3, 2, 1]]), np.arange(L - 2, L))
+        assert np.array_equal(o.last_candidates(0, h), union)
+    # similarity mode on the same state picks by rho instead
+    o2 = oracle_mod.Oracle(B, H, H, d, M, r, 2, K, -2.0, 0, L)
+    o2.import_state(qc, sup, n_ins, 4)
+    o2.decode_step(q, k, v, L)
+    rho = qc[0, 0] @ (q64[0, 0] / np.linalg.norm(q64[0, 0]))
+    assert list(o2.last_step()["sel"][0, 0]) == sorted(range(M), key=lambda c: (-rho[c], c))[:r]
+
+
+def test_recent_recall_falls_back_on_its_own_maximum(oracle_mod):
+    """rho_max is taken over the recalled (recent) entries only."""
+    d, M, L = 8, 4, 32
+    qc = np.zeros((1, 1, M, d))
+    qc[0, 0, 0, 0] = 1.0            # old entry identical to the query
+    qc[0, 0, 1, 1] = 1.0
+    qc[0, 0, 2, 2] = 1.0            # newest two entries are orthogonal to it
+    qc[0, 0, 3, 3] = 1.0
+    sup = np.tile(np.arange(4, dtype=np.int32), (1, 1, M, 1))
+    k = bits(np.random.default_rng(1).standard_normal((1, 1, L, d)))
+    q = bits(np.array([[[1.0] + [0.0] * (d - 1)]]))
+    for mode, want in ((0, oracle_mod.PATH_REUSE), (1, oracle_mod.PATH_FALLBACK)):
+        o = oracle_mod.Oracle(1, 1, 1, d, M, 2, 2, 4, 0.5, 0, L)
+        o.set_recall_mode(mode)
+        o.import_state(qc, sup, 4, 1)       # ring full: newest are slots 3 and 2
+        o.decode_step(q, k, k, 20)
+        assert o.last_step()["path"][0, 0] == want
