@@ -93,6 +93,15 @@ int retopk_create(retopk_ctx** ctx, int H_q, int H_kv, int d, int M, int r, int 
 int retopk_create_batched(retopk_ctx** ctx, int B, int H_q, int H_kv, int d, int M, int r, int W,
                           int K, float tau, int R, int64_t max_seq_len);
 
+/*
+ * Recall rule.  RETOPK_RECALL_SIMILAR (default) is the method's Eq. 7: the r most similar
+ * cached queries.  RETOPK_RECALL_RECENT is the component study's "Recent-R" row (Table 3):
+ * the min(r, filled) most recently inserted entries are recalled instead and rho_max is the
+ * largest similarity among those (the paper prints no formula for this row).
+ */
+enum { RETOPK_RECALL_SIMILAR = 0, RETOPK_RECALL_RECENT = 1 };
+int retopk_set_recall_mode(retopk_ctx* ctx, int mode);
+
 /* Release the context and its device memory (synchronises the device). */
 int retopk_destroy(retopk_ctx* ctx);
 

@@ -19,6 +19,7 @@ struct retopk_ctx {
     int NS, tile_cap, stage_depth, exact_stage_depth;
     int num_sms, scan_grid;
     int call_serial;
+    int recall_recent;
     size_t smem_recall, smem_reuse, smem_exact, smem_finish;
     // device state
     float* qbar_cache;
@@ -86,6 +87,7 @@ StepArgs make_args(const retopk_ctx* c, const void* q, const void* k, const void
     a.slot = (int)(c->n_ins % c->M);
     a.refresh = (c->R > 0 && c->t_dec > 0 && c->t_dec % c->R == 0) ? 1 : 0;
     a.mode = mode;
+    a.recall_recent = c->recall_recent;
     a.NS = c->NS;
     a.tile_cap = c->tile_cap;
     a.step_id = c->call_serial;
@@ -279,6 +281,12 @@ int retopk_create_batched(retopk_ctx** out, int B, int H_q, int H_kv, int d, int
 int retopk_create(retopk_ctx** ctx, int H_q, int H_kv, int d, int M, int r, int W, int K, float tau,
                   int R) {
     return retopk_create_batched(ctx, 1, H_q, H_kv, d, M, r, W, K, tau, R, RETOPK_DEFAULT_MAX_SEQ_LEN);
+}
+
+int retopk_set_recall_mode(retopk_ctx* c, int mode) {
+    if (!c || (mode != RETOPK_RECALL_SIMILAR && mode != RETOPK_RECALL_RECENT)) return RETOPK_EINVAL;
+    c->recall_recent = mode == RETOPK_RECALL_RECENT;
+    return RETOPK_OK;
 }
 
 int retopk_destroy(retopk_ctx* c) {

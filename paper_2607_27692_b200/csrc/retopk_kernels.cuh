@@ -67,6 +67,7 @@ struct StepArgs {
     int refresh;             // 1 when Eq. 13's first case holds (known on the host)
     int mode;                // MODE_RETOPK or MODE_EXACT
     int prefill;             // 1: cache seeding (every head exact, nothing counted)
+    int recall_recent;       // 1: recall the newest entries instead of the most similar (Recent-R ablation)
     int NS;                  // entries in the exact path's shared collection lists
     int tile_cap;            // entries in the exact path's list of hit tiles
     int g_shift;             // log2(G) when G is a power of two, else -1
@@ -615,7 +616,20 @@ __global__ void __launch_bounds__(RECALL_THREADS, 1) recall_kernel(const StepArg
     // P threads share an entry (P a power of two <= 32): each counts the better entries in
     // its slice of the cache, a shuffle tree adds the slices.
     const int n_sel = a.r < fill ? a.r : fill;
-    {
+    if (a.recall_recent) {
+        // Recent-R ablation: the newest n_sel entries (newest first), rho_max over those only
+        if (tid < 32) {
+            float best = -CUDART_INF_F;
+            for (int j = lane; j < n_sel; j += 32) {
+                const int c = ((a.slot - 1 - j) % M + M) % M;
+                s_sel[j] = c;
+                best = fmaxf(best, s_rho[c]);
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) best = fmaxf(best, __shfl_xor_sync(0xffffffffu, best, o));
+            if (lane == 0) s_misc[0] = best;
+        }
+    } else {
         int lp = 5;
         while (lp > 0 && (fill << lp) > NT) --lp;
         const int P = 1 << lp, me = tid >> lp, part = tid & (P - 1);

@@ -36,6 +36,7 @@ _vp, _i32, _i64, _f32 = C.c_void_p, C.c_int, C.c_int64, C.c_float
 SIGNATURES = {
     "retopk_create": (_i32, [C.POINTER(_vp)] + [_i32] * 7 + [_f32, _i32]),
     "retopk_create_batched": (_i32, [C.POINTER(_vp)] + [_i32] * 8 + [_f32, _i32, _i64]),
+    "retopk_set_recall_mode": (_i32, [_vp, _i32]),
     "retopk_destroy": (_i32, [_vp]),
     "retopk_reset": (_i32, [_vp, _vp]),
     "retopk_decode_step": (_i32, [_vp, _vp, _vp, _vp, _i64, _vp, _vp]),
@@ -141,6 +142,10 @@ class ReTopK:
         return (self.B, self.H_kv, self.max_seq_len, self.d)
 
     # -- calls ----------------------------------------------------------------------
+    def set_recall_mode(self, mode: int):
+        """0: recall the most similar entries (Eq. 7); 1: the most recent ones (Recent-R ablation row)."""
+        _check(self.lib.retopk_set_recall_mode(self.h, mode), "retopk_set_recall_mode")
+
     def reset(self):
         _check(self.lib.retopk_reset(self.h, _stream()), "retopk_reset")
 

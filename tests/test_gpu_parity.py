@@ -328,3 +328,20 @@ def test_prefill_argument_checks(rt, P):
         g.prefill(torch.zeros((5, 1, 2, 64), dtype=torch.bfloat16, device="cuda"), kv, kv, 100)   # n_tail > M
     with pytest.raises(rt.RetopkError):
         g.prefill(torch.zeros((3, 1, 2, 64), dtype=torch.bfloat16, device="cuda"), kv, kv, 2)     # n_tail > prompt
+
+
+def test_recent_recall_variant_teacher_forced(rt, P, oracle_mod):
+    """The Recent-R ablation row: newest entries recalled, rho_max over them only."""
+    cfg = wl.CONFIGS["tiny"].replace(context=900, steps=30, B=2, H_q=4, H_kv=2, M=6, r=3)
+    st, o, g, k, v = stream_case(rt, P, oracle_mod, cfg, 30)
+    o.set_recall_mode(1)
+    g.set_recall_mode(1)
+    P.teacher_forced_run(cfg, st, 30, o, g, k, v)
+    so, sg = o.stats(), g.stats()
+    for key in ("steps", "reuse", "fallback", "refresh", "cand_sum"):
+        assert sg[key] == so[key], key
+    # and it really differs from similarity recall on this stream
+    st2, o2, g2, _, _ = stream_case(rt, P, oracle_mod, cfg, 30)
+    for t in range(30):
+        o2.decode_step(st2.q[t], st2.k, st2.v, st2.seq_len(t))
+    assert o2.stats()["fallback"] != so["fallback"] or o2.stats()["cand_sum"] != so["cand_sum"]
