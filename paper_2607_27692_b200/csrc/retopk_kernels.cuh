@@ -30,17 +30,8 @@ __device__ long long g_phase_clk[3][1024][16];
     do {                                                                                   \
         if (threadIdx.x == 0 && blockIdx.x < 1024) g_phase_clk[kernel][blockIdx.x][n] = clock64(); \
     } while (0)
-#define RETOPK_WALL(kernel, n)                                                              \
-    do {                                                                                   \
-        if (threadIdx.x == 0 && blockIdx.x < 1024) {                                       \
-            unsigned long long t_;                                                         \
-            asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_));                          \
-            g_phase_clk[kernel][blockIdx.x][n] = (long long)t_;                            \
-        }                                                                                  \
-    } while (0)
 #else
 #define RETOPK_PHASE(kernel, n) do { } while (0)
-#define RETOPK_WALL(kernel, n) do { } while (0)
 #endif
 
 namespace retopk {
@@ -111,13 +102,6 @@ __device__ __forceinline__ float key_score(uint32_t k) {
 }
 __device__ __forceinline__ float bf16_lo(uint32_t u) { return __uint_as_float(u << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t u) { return __uint_as_float(u & 0xffff0000u); }
-
-__device__ __forceinline__ uint4 ldg_stream(const void* p) {
-    uint4 r;
-    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p));
-    return r;
-}
 
 // Programmatic dependent launch: a kernel launched with the stream-serialisation attribute
 // may start while its predecessor still runs; it must call pdl_wait() before touching
@@ -392,13 +376,11 @@ __device__ int select_listed(const uint32_t* s_key, const int32_t* s_idx, int n,
         SmemSrc src{s_key, s_idx};
         int* s_cnt = reinterpret_cast<int*>(s_hist);
         const Threshold t = count_threshold<NT>(s_key, n, K, 0, s_cnt);
-        RETOPK_PHASE(2, 6);
         uint32_t vstar;
         int need_eq;
         if (t.count == K) { vstar = t.v - 1u; need_eq = 0; }            // exactly K keys are >= v
         else { vstar = t.v; need_eq = t.need; }                          // v = K-th largest key
         ordered_emit<NT>(src, n, vstar, need_eq, s_sup_idx, s_sup_key, s_ws);
-        RETOPK_PHASE(2, 7);
         ns = K;
         kmax = t.kmax;
         kmax_known = true;
@@ -560,9 +542,7 @@ __global__ void __launch_bounds__(RECALL_THREADS, 1) recall_kernel(const StepArg
     const int bkv = kv_group_of(bh, a);
     const int M = a.M, fill = a.fill;
 
-    RETOPK_WALL(1, 13);
     pdl_wait();        // the caches were written by the step before; q by whatever ran before this call
-    RETOPK_WALL(1, 14);
     RETOPK_PHASE(1, 0);
     // Every warp reads the query itself (four elements per lane) next to its cache rows, so
     // one memory latency covers both:  rho_c = (qbar_c . q) / |q|   (Eq. 6)
@@ -669,7 +649,6 @@ __global__ void __launch_bounds__(RECALL_THREADS, 1) recall_kernel(const StepArg
         }
     }
     RETOPK_PHASE(1, 2);
-    RETOPK_WALL(1, 15);
 }
 
 // ------------------------------------------------------------------------------------
@@ -779,7 +758,6 @@ __device__ void reuse_path(const StepArgs& a, unsigned char* smem_raw) {
         *reinterpret_cast<float4*>(qf + 4) = *reinterpret_cast<const float4*>(s_qraw + sub * 8 + 4);
         const int depth = a.stage_depth;
         uint4* my_stage = s_stage + tid;
-        RETOPK_PHASE(0, 9);
         // each wave goes out as two groups of copies, so that the dot products of the first
         // half run while the second half is still arriving
         const int half = (depth + 1) / 2;
@@ -790,11 +768,9 @@ __device__ void reuse_path(const StepArgs& a, unsigned char* smem_raw) {
                 if (u == half - 1) cp_async_commit();
             }
             cp_async_commit();
-            RETOPK_PHASE(0, 10);
             for (int g2 = 0; g2 < 2; ++g2) {
                 if (g2 == 0) cp_async_wait_but_one();
                 else cp_async_wait_all();
-                if (g2 == 0) RETOPK_PHASE(0, 11);
                 const int u_begin = g2 == 0 ? 0 : half, u_end = g2 == 0 ? half : depth;
                 for (int u0 = u_begin; u0 < u_end; u0 += 8) {
                     float part[8];
@@ -810,7 +786,6 @@ __device__ void reuse_path(const StepArgs& a, unsigned char* smem_raw) {
                 }
             }
         }
-        RETOPK_PHASE(0, 12);
     }
     __syncthreads();
     RETOPK_PHASE(0, 6);
@@ -862,7 +837,6 @@ __global__ void __launch_bounds__(SCAN_THREADS) scan_kernel(const StepArgs a) {
     const int g = lane >> 2, t = lane & 3;
     const int G = a.G, L = a.L;
     const int n_groups = a.B * a.Hkv;
-    RETOPK_WALL(0, 13);
     // No trigger for the dependent launch behind this kernel: its CTAs take a whole SM each
     // and start as this kernel's CTAs exit; that already hides its launch latency.
 
@@ -997,7 +971,6 @@ __global__ void __launch_bounds__(SCAN_THREADS) scan_kernel(const StepArgs a) {
             __syncthreads();
         }
     }
-    RETOPK_WALL(0, 15);
 }
 
 // ------------------------------------------------------------------------------------
@@ -1084,7 +1057,6 @@ __device__ void exact_path(const StepArgs& a, unsigned char* smem_raw) {
                 s_key[i2] = score_key(m);
             }
             __syncthreads();
-            RETOPK_PHASE(2, 8);
             thr_key = count_threshold<NT>(s_key, n2, K, 16, reinterpret_cast<int*>(s_hist)).v;
         }
         RETOPK_PHASE(2, 1);
@@ -1098,7 +1070,6 @@ __device__ void exact_path(const StepArgs& a, unsigned char* smem_raw) {
             for (int u = 0; u < 2; ++u)
                 m4[u] = t0 + 4 * u < ntile ? *reinterpret_cast<const float4*>(tm + t0 + 4 * u)
                                            : make_float4(0.f, 0.f, 0.f, 0.f);
-            if (base == 0) RETOPK_PHASE(2, 11);
             const float mv[8] = {m4[0].x, m4[0].y, m4[0].z, m4[0].w, m4[1].x, m4[1].y, m4[1].z, m4[1].w};
             unsigned hits = 0;
 #pragma unroll
@@ -1136,10 +1107,8 @@ __device__ void exact_path(const StepArgs& a, unsigned char* smem_raw) {
                             if (row0 + 4 * u + e < L && score_key(v4[e]) >= thr_key) fl |= 1u << (4 * u + e);
                     }
                 }
-                RETOPK_PHASE(2, 9);
                 int total;
                 int pos = n + block_excl_scan<NT>(__popc(fl), s_ws, total);
-                RETOPK_PHASE(2, 10);
                 while (fl) {
                     const int e = __ffs(fl) - 1;
                     if (pos < NS) { s_key[pos] = score_key(sc[row0 + e]); s_idx[pos] = row0 + e; }
@@ -1189,13 +1158,10 @@ __device__ void exact_path(const StepArgs& a, unsigned char* smem_raw) {
 template <int D>
 __global__ void __launch_bounds__(FINISH_THREADS, 1) finish_kernel(const StepArgs a) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    RETOPK_WALL(2, 13);
     pdl_wait();        // scores and tile maxima come from the scan, recalled slots and paths from recall_kernel
-    RETOPK_WALL(2, 14);
     if (blockIdx.x == 0 && threadIdx.x == 0) *a.scan_counter = 0u;      // the scan before this kernel is complete
     if (a.mode == MODE_RETOPK && a.ws_path[blockIdx.x] == PATH_REUSE) reuse_path<D, FINISH_THREADS>(a, smem_raw);
     else exact_path<D, FINISH_THREADS>(a, smem_raw);
-    RETOPK_WALL(2, 15);
 }
 
 // Clear the caches (supports to -1, queries and counters to 0).
