@@ -138,14 +138,15 @@ int launch_scan(const retopk_ctx* c, const StepArgs& a, cudaStream_t s) {
     const long long items = (long long)c->B * c->Hkv * ((a.L + SCAN_TILE_ROWS - 1) / SCAN_TILE_ROWS);
     const unsigned grid = (unsigned)(items < c->scan_grid ? items : c->scan_grid);
     const int ntile = (c->G + 7) / 8;
-    // An ordinary launch: started as a dependent launch behind a kernel that takes all of an
-    // SM's shared memory, the scan measured 1.6x slower (its CTAs land on SMs still carved up
-    // for that kernel, and it needs about 100 KB of L1 to keep its loads in flight).
-    if (c->d == 128 && ntile == 1) scan_kernel<128, 1><<<grid, SCAN_THREADS, 0, s>>>(a);
-    else if (c->d == 128) scan_kernel<128, 2><<<grid, SCAN_THREADS, 0, s>>>(a);
-    else if (ntile == 1) scan_kernel<64, 1><<<grid, SCAN_THREADS, 0, s>>>(a);
-    else scan_kernel<64, 2><<<grid, SCAN_THREADS, 0, s>>>(a);
-    return cudaGetLastError() == cudaSuccess ? RETOPK_OK : RETOPK_ECUDA;
+    // A dependent launch behind recall_kernel (or behind the previous call's last kernel for
+    // Exact Top-K).  Behind a kernel that takes ALL of an SM's shared memory the scan ran 1.6x
+    // slower: its CTAs then land on SMs still carved up for that kernel, and it needs about
+    // 100 KB of L1 per SM to keep its loads in flight.  recall_kernel uses a few KB, so the SMs
+    // are back in the default split by the time the scan's CTAs start.
+    if (c->d == 128 && ntile == 1) return launch_dependent(scan_kernel<128, 1>, grid, SCAN_THREADS, 0, s, a);
+    if (c->d == 128) return launch_dependent(scan_kernel<128, 2>, grid, SCAN_THREADS, 0, s, a);
+    if (ntile == 1) return launch_dependent(scan_kernel<64, 1>, grid, SCAN_THREADS, 0, s, a);
+    return launch_dependent(scan_kernel<64, 2>, grid, SCAN_THREADS, 0, s, a);
 }
 
 int launch_finish(const retopk_ctx* c, const StepArgs& a, cudaStream_t s) {

@@ -839,6 +839,7 @@ __global__ void __launch_bounds__(SCAN_THREADS) scan_kernel(const StepArgs a) {
     const int n_groups = a.B * a.Hkv;
     // No trigger for the dependent launch behind this kernel: its CTAs take a whole SM each
     // and start as this kernel's CTAs exit; that already hides its launch latency.
+    pdl_wait();        // group flags and paths come from recall_kernel
 
     // nothing flagged in this step: leave at once (the common case on the reuse path)
     if (a.mode != MODE_EXACT && a.ws_gflag[n_groups] != a.step_id) return;
