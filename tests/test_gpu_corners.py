@@ -32,6 +32,8 @@ CASES = [
     (1, 3, 3, 64, 1234, 512, 5, 5, 3000, 0.7, 2, 7),      # window longer than the history
     (3, 2, 1, 128, 40000, 1000, 9, 3, 17, 0.8, 5, 6),     # several sequences, K not a power of two
     (1, 8, 8, 128, 70000, 2048, 3, 3, 1, 0.3, 0, 5),      # K = 2048 with enough tiles for the bound
+    (1, 2, 1, 128, 1048570, 512, 4, 2, 64, 0.4, 0, 4),    # the longest supported history (1 Mi keys)
+    (1, 4, 2, 64, 300000, 64, 4, 2, 8, 0.4, 3, 4),        # beyond 256 Ki keys, d = 64
 ]
 
 
