@@ -337,7 +337,7 @@ def run_gpu(args):
                 "frac_of_8TBps": round(kernels[top]["GBps"] / 8000.0, 4),
                 "traffic": (int(NCU_TRAFFIC_PER_GROUP[args.config] * prof["stats"]["scan_groups"] / prof["prof"]["scan"]["launches"])
                             if top == "scan" and args.config in NCU_TRAFFIC_PER_GROUP else None),
-                "traffic_source": "profiles/scan_kernel_headline128k_single_layer.md, scaled by scanned groups per launch",
+                "traffic_source": "ncu capture of a one-layer run of this workload (summary under profiles/), scaled by scanned groups per launch",
                 "kernels": kernels}
 
     def path_report(res, exact_like):
@@ -391,10 +391,10 @@ def run_gpu(args):
 
 
 # DRAM traffic of scan_kernel per scanned KV group (dram__bytes_read.sum + dram__bytes_write.sum
-# of one launch over its 32 groups) from the ncu capture summarised in
-# profiles/scan_kernel_headline128k_single_layer.md; a launch's traffic is this times the
-# groups it scanned (traffic grows in proportion to the rows streamed).
-NCU_TRAFFIC_PER_GROUP = {"headline128k": 34.29e6}
+# of one launch over its 32 groups) from the ncu capture of a one-layer run whose summary is kept
+# under profiles/; a launch's traffic is this times the groups it scanned (traffic grows in
+# proportion to the rows streamed).  The K = 1024 variant streams the same rows per group.
+NCU_TRAFFIC_PER_GROUP = {"headline128k": 34.29e6, "headline128k_k1024": 34.29e6}
 
 
 # --------------------------------------------------------------------------- reference arm

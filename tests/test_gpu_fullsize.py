@@ -54,6 +54,13 @@ def test_headline_config(rt, P, oracle_mod):
     assert sg["steps"] == 34 * 4 * 32 and sg["slow_select"] == 0 and sg["status"] == 0
 
 
+def test_headline_shapes_with_k1024(rt, P, oracle_mod):
+    """The cross-model 128K setting (Table 2) keeps K = 1024 keys per head."""
+    so, sg, ex = run_sampled(rt, P, oracle_mod, "headline128k_k1024", 10, [2], tau=0.85)
+    assert so["reuse"] > 0 and so["fallback"] > 0
+    assert sg["steps"] == 10 * 4 * 32 and sg["slow_select"] == 0 and sg["status"] == 0
+
+
 def test_stress_config(rt, P, oracle_mod):
     """128K, batch 16, K = 2048, r = 8, W = 512, refresh every 8 steps: mostly exact steps."""
     so, sg, ex = run_sampled(rt, P, oracle_mod, "stress128k", 10, [9])
