@@ -522,37 +522,22 @@ __device__ void attend(const uint16_t* vbase, int ns, const int32_t* s_sup_idx, 
 }
 
 // ------------------------------------------------------------------------------------
-// recall_kernel: Eq. 6, Eq. 7, Eq. 13 and the insert of the normalised query, per head.
-// Leaves the recalled slots, rho_max and the path in global memory and flags the KV group
-// of every head that takes the exact path.
+// Pieces of the recall stage (one block per head).
 // ------------------------------------------------------------------------------------
-template <int D>
-__global__ void __launch_bounds__(RECALL_THREADS, 1) recall_kernel(const StepArgs a) {
-    constexpr int NT = RECALL_THREADS;
+
+// Eq. 6: rho_c = (qbar_c . q) / |q| for every cached entry c < fill into s_rho[c], and the
+// normalised query into s_q[0..D).  Every warp reads the query itself (four elements per
+// lane) next to its cache rows, so one memory latency covers both.  No barrier at the end.
+template <int D, int NT>
+__device__ __forceinline__ void cache_similarities(const StepArgs& a, int bh, float* s_q, float* s_rho) {
     constexpr int NW = NT / 32;
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    // layout (words): q[D] rho[M + 3] sel[r] misc[4]
-    float* s_q = reinterpret_cast<float*>(smem_raw);
-    float* s_rho = s_q + D;
-    int* s_sel = reinterpret_cast<int*>(s_rho + ((a.M + 3) & ~3));
-    float* s_misc = reinterpret_cast<float*>(s_sel + a.r);
-
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int bh = blockIdx.x;
-    const int bkv = kv_group_of(bh, a);
     const int M = a.M, fill = a.fill;
-
-    pdl_wait();        // the caches were written by the step before; q by whatever ran before this call
-    RETOPK_PHASE(1, 0);
-    // Every warp reads the query itself (four elements per lane) next to its cache rows, so
-    // one memory latency covers both:  rho_c = (qbar_c . q) / |q|   (Eq. 6)
     float q4[4] = {0.f, 0.f, 0.f, 0.f};
     if (lane < D / 4) {
         const uint2 raw = *reinterpret_cast<const uint2*>(a.q + (size_t)bh * D + 4 * lane);
         q4[0] = bf16_lo(raw.x); q4[1] = bf16_hi(raw.x); q4[2] = bf16_lo(raw.y); q4[3] = bf16_hi(raw.y);
     }
-    if (tid < a.r) s_sel[tid] = -1;
-    if (tid == 0) s_misc[0] = -CUDART_INF_F;
     float inv_nrm = 0.f;
     for (int c0 = warp; c0 < fill || c0 == warp; c0 += NW * 4) {
         float4 x[4];
@@ -588,13 +573,17 @@ __global__ void __launch_bounds__(RECALL_THREADS, 1) recall_kernel(const StepArg
             if (lane == 0 && c < fill) s_rho[c] = acc * inv_nrm;
         }
     }
-    __syncthreads();
-    RETOPK_PHASE(1, 1);
+}
 
-    // Eq. 7: rho_max and the min(r, fill) most similar slots.  Every cached entry ranks
-    // itself against the others (larger rho first, ties -> lower slot).
-    // P threads share an entry (P a power of two <= 32): each counts the better entries in
-    // its slice of the cache, a shuffle tree adds the slices.
+// Eq. 7: rho_max and the min(r, fill) most similar slots into s_sel (places beyond that keep
+// the -1 the caller put there; s_misc[0] must hold -inf).  Every cached entry ranks itself
+// against the others (larger rho first, ties -> lower slot).  P threads share an entry (P a
+// power of two <= 32): each counts the better entries in its slice of the cache, a shuffle
+// tree adds the slices.  s_rho must be complete (barrier before the call).
+template <int NT>
+__device__ __forceinline__ float recall_slots(const StepArgs& a, const float* s_rho, int* s_sel, float* s_misc) {
+    const int tid = threadIdx.x, lane = tid & 31;
+    const int M = a.M, fill = a.fill;
     const int n_sel = a.r < fill ? a.r : fill;
     if (a.recall_recent) {
         // Recent-R ablation: the newest n_sel entries (newest first), rho_max over those only
@@ -627,16 +616,20 @@ __global__ void __launch_bounds__(RECALL_THREADS, 1) recall_kernel(const StepArg
         }
     }
     __syncthreads();
-    const float rho_max = s_misc[0];
+    return s_misc[0];
+}
 
-    // Eq. 13
-    int path;
-    if (a.refresh) path = PATH_REFRESH;
-    else if (rho_max < a.tau) path = PATH_FALLBACK;
-    else path = PATH_REUSE;
+// Eq. 13
+__device__ __forceinline__ int decide_path(const StepArgs& a, float rho_max) {
+    if (a.refresh) return PATH_REFRESH;
+    return rho_max < a.tau ? PATH_FALLBACK : PATH_REUSE;
+}
 
-    // insert the normalised query now: every similarity of this step has been taken
-    if (tid < D) a.qbar_cache[((size_t)bh * M + a.slot) * D + tid] = s_q[tid];
+// Leave the decision of one head where the later kernels (and the caller) find it; a head
+// on the exact path flags its KV group for the scan.
+__device__ __forceinline__ void record_decision(const StepArgs& a, int bh, int bkv, const int* s_sel, int path,
+                                                float rho_max) {
+    const int tid = threadIdx.x;
     if (tid < a.r) a.ws_sel[(size_t)bh * a.r + tid] = s_sel[tid];
     if (tid == 0) {
         a.ws_path[bh] = (uint8_t)path;
@@ -648,59 +641,57 @@ __global__ void __launch_bounds__(RECALL_THREADS, 1) recall_kernel(const StepArg
             if (!a.prefill) atomicAdd(a.counters + (size_t)bh * 4 + path, 1ull);   // no return value: not waited for
         }
     }
+}
+
+// ------------------------------------------------------------------------------------
+// recall_kernel: Eq. 6, Eq. 7, Eq. 13 and the insert of the normalised query, per head.
+// Leaves the recalled slots, rho_max and the path in global memory and flags the KV group
+// of every head that takes the exact path.
+// ------------------------------------------------------------------------------------
+template <int D>
+__global__ void __launch_bounds__(RECALL_THREADS, 1) recall_kernel(const StepArgs a) {
+    constexpr int NT = RECALL_THREADS;
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    // layout (words): q[D] rho[M + 3] sel[r] misc[4]
+    float* s_q = reinterpret_cast<float*>(smem_raw);
+    float* s_rho = s_q + D;
+    int* s_sel = reinterpret_cast<int*>(s_rho + ((a.M + 3) & ~3));
+    float* s_misc = reinterpret_cast<float*>(s_sel + a.r);
+
+    const int tid = threadIdx.x;
+    const int bh = blockIdx.x;
+    const int bkv = kv_group_of(bh, a);
+
+    pdl_wait();        // the caches were written by the step before; q by whatever ran before this call
+    RETOPK_PHASE(1, 0);
+    if (tid < a.r) s_sel[tid] = -1;
+    if (tid == 0) s_misc[0] = -CUDART_INF_F;
+    cache_similarities<D, NT>(a, bh, s_q, s_rho);
+    __syncthreads();
+    RETOPK_PHASE(1, 1);
+    const float rho_max = recall_slots<NT>(a, s_rho, s_sel, s_misc);
+    const int path = decide_path(a, rho_max);
+
+    // insert the normalised query now: every similarity of this step has been taken
+    if (tid < D) a.qbar_cache[((size_t)bh * a.M + a.slot) * D + tid] = s_q[tid];
+    record_decision(a, bh, bkv, s_sel, path, rho_max);
     RETOPK_PHASE(1, 2);
 }
 
 // ------------------------------------------------------------------------------------
-// reuse path of finish_kernel: candidate union (Eq. 8-9), candidate scores (Eq. 10), Top-K
-// (Eq. 11), softmax.V (Eq. 12) and the support insert for one head, all in shared memory.
+// Pieces of the reuse path (one block per head).
 // ------------------------------------------------------------------------------------
-template <int D, int NT>
-__device__ void reuse_path(const StepArgs& a, unsigned char* smem_raw) {
-    constexpr int NW = NT / 32;
-    constexpr int LPR = D / 8, RPW = 32 / LPR, SLOTS = NW * RPW;
-    // layout (words): qraw[D] sel[r] ws[32] hist[SCRATCH_WORDS] sup_idx[K] sup_key[K] w[K]
-    //                 | big: idx[cap] key[cap], aliased later by red[NW*D+NT] | bitmap | stage[depth*NT*4]
-    float* s_qraw = reinterpret_cast<float*>(smem_raw);
-    int* s_sel = reinterpret_cast<int*>(s_qraw + D);
-    int* s_ws = s_sel + a.r;
-    uint32_t* s_hist = reinterpret_cast<uint32_t*>(s_ws + 32);
-    int32_t* s_sup_idx = reinterpret_cast<int32_t*>(s_hist + SCRATCH_WORDS);
-    uint32_t* s_sup_key = reinterpret_cast<uint32_t*>(s_sup_idx + a.K);
-    float* s_w = reinterpret_cast<float*>(s_sup_key + a.K);
-    const int head_words = (D + a.r + 32 + SCRATCH_WORDS + 3 * a.K + 3) & ~3;
-    int32_t* s_idx = reinterpret_cast<int32_t*>(smem_raw) + head_words;
-    uint32_t* s_key = reinterpret_cast<uint32_t*>(s_idx + a.cap);
-    float* s_red = reinterpret_cast<float*>(s_idx);
-    const int big_words = (max(2 * a.cap, NW * D + NT) + 3) & ~3;
-    uint32_t* s_bm = reinterpret_cast<uint32_t*>(s_idx) + big_words;
-    uint4* s_stage = reinterpret_cast<uint4*>(s_bm + ((((int)a.max_seq_len + 31) / 32 + 3) & ~3));
 
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int bh = blockIdx.x;
-    const int bkv = kv_group_of(bh, a);
-    const int M = a.M, fill = a.fill, L = a.L, K = a.K;
-    const int n_sel = a.r < fill ? a.r : fill;
-    RETOPK_PHASE(0, 0);
-
-    // recalled slots and the raw query from global memory; clear the bitmap meanwhile
-    if (tid < a.r) s_sel[tid] = a.ws_sel[(size_t)bh * a.r + tid];
-    if (tid >= 32 && tid < 32 + D / 2) {
-        const uint32_t raw = reinterpret_cast<const uint32_t*>(a.q + (size_t)bh * D)[tid - 32];
-        s_qraw[2 * (tid - 32)] = bf16_lo(raw);
-        s_qraw[2 * (tid - 32) + 1] = bf16_hi(raw);
-    }
-    {
-        const int nwords = (L + 31) >> 5;
-        uint4* bm4 = reinterpret_cast<uint4*>(s_bm);
-        for (int w = tid; w < (nwords + 3) >> 2; w += NT) bm4[w] = make_uint4(0, 0, 0, 0);
-    }
-    __syncthreads();
-    RETOPK_PHASE(0, 3);
-
-    // Eq. 8-9: sorted unique candidate list.  Recalled indices below the window go through a
-    // bitmap over key positions (ordered extraction = sorted and deduplicated for free); the
-    // window itself is a contiguous run appended behind them, whatever the supports held there.
+// Eq. 8-9: the sorted unique candidate list of head bh into s_idx; returns its length.
+// Recalled indices below the window go through a bitmap over key positions (ordered
+// extraction = sorted and deduplicated for free); the window itself is a contiguous run
+// appended behind them, whatever the supports held there.  The bitmap must be clear and
+// s_sel loaded (barrier before the call); no barrier at the end.
+template <int NT>
+__device__ __forceinline__ int candidate_union(const StepArgs& a, int bh, const int* s_sel, int n_sel,
+                                               uint32_t* s_bm, int32_t* s_idx, int* s_ws) {
+    const int tid = threadIdx.x;
+    const int M = a.M, L = a.L, K = a.K;
     const int w_lo = L - a.W > 0 ? L - a.W : 0;
     {
         bool bad = false;
@@ -723,70 +714,127 @@ __device__ void reuse_path(const StepArgs& a, unsigned char* smem_raw) {
     }
     __syncthreads();
     RETOPK_PHASE(0, 4);
-    int n;
-    {
-        const int nw_lo = (w_lo + 31) >> 5;               // words that can hold bits below the window
-        const int wpt = (nw_lo + NT - 1) / NT;
-        const int w0 = tid * wpt;
-        const int w1 = (w0 + wpt < nw_lo) ? w0 + wpt : nw_lo;
-        int cnt = 0;
-        for (int w = w0; w < w1; ++w) cnt += __popc(s_bm[w]);
-        int n_low;
-        int pos = block_excl_scan<NT>(cnt, s_ws, n_low);
-        for (int w = w0; w < w1; ++w) {
-            uint32_t bits = s_bm[w];
-            while (bits) {
-                const int bit = __ffs(bits) - 1;
-                s_idx[pos++] = w * 32 + bit;
-                bits &= bits - 1;
+    const int nw_lo = (w_lo + 31) >> 5;               // words that can hold bits below the window
+    const int wpt = (nw_lo + NT - 1) / NT;
+    const int w0 = tid * wpt;
+    const int w1 = (w0 + wpt < nw_lo) ? w0 + wpt : nw_lo;
+    int cnt = 0;
+    for (int w = w0; w < w1; ++w) cnt += __popc(s_bm[w]);
+    int n_low;
+    int pos = block_excl_scan<NT>(cnt, s_ws, n_low);
+    for (int w = w0; w < w1; ++w) {
+        uint32_t bits = s_bm[w];
+        while (bits) {
+            const int bit = __ffs(bits) - 1;
+            s_idx[pos++] = w * 32 + bit;
+            bits &= bits - 1;
+        }
+    }
+    for (int i = w_lo + tid; i < L; i += NT) s_idx[n_low + (i - w_lo)] = i;
+    return n_low + (L - w_lo);
+}
+
+// Eq. 10: exact current-query scores of n key rows as order-preserving keys into key_out.
+// Row i is kbase[row_of[i]] (INDEXED) or kbase[i] (rows already packed).  Every lane copies
+// its 16 bytes of each row asynchronously into its own landing zone and reads them back
+// itself, so a whole wave of rows is in flight with no registers held and no barrier.
+// s_qraw: the raw query as D floats; s_stage: depth * NT uint4.  No barrier at the end.
+template <int D, int NT, bool INDEXED>
+__device__ __forceinline__ void score_candidates(const uint16_t* kbase, const int32_t* row_of, int n,
+                                                 const float* s_qraw, uint4* s_stage, int depth, float scale,
+                                                 uint32_t* key_out) {
+    constexpr int LPR = D / 8, RPW = 32 / LPR, SLOTS = (NT / 32) * RPW;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int sub = lane % LPR, myslot = warp * RPW + lane / LPR;
+    const char* ksrc = reinterpret_cast<const char*>(kbase) + sub * 16;
+    float qf[8];
+    *reinterpret_cast<float4*>(qf) = *reinterpret_cast<const float4*>(s_qraw + sub * 8);
+    *reinterpret_cast<float4*>(qf + 4) = *reinterpret_cast<const float4*>(s_qraw + sub * 8 + 4);
+    uint4* my_stage = s_stage + tid;
+    // each wave goes out as two groups of copies, so that the dot products of the first
+    // half run while the second half is still arriving
+    const int half = (depth + 1) / 2;
+    for (int base = 0; base < n; base += SLOTS * depth) {
+        for (int u = 0; u < depth; ++u) {
+            const int i = base + u * SLOTS + myslot;
+            if (i < n) cp_async16(my_stage + u * NT, ksrc + (size_t)(INDEXED ? row_of[i] : i) * (D * 2));
+            if (u == half - 1) cp_async_commit();
+        }
+        cp_async_commit();
+        for (int g2 = 0; g2 < 2; ++g2) {
+            if (g2 == 0) cp_async_wait_but_one();
+            else cp_async_wait_all();
+            const int u_begin = g2 == 0 ? 0 : half, u_end = g2 == 0 ? half : depth;
+            for (int u0 = u_begin; u0 < u_end; u0 += 8) {
+                float part[8];
+#pragma unroll
+                for (int uu = 0; uu < 8; ++uu) {
+                    const int i = base + (u0 + uu) * SLOTS + myslot;
+                    part[uu] = (u0 + uu < u_end && i < n) ? dot8(my_stage[(u0 + uu) * NT], qf) : 0.f;
+                }
+                int row;
+                const float tot = reduce8_across<LPR>(part, sub, row);
+                const int i = base + (u0 + row) * SLOTS + myslot;
+                if ((LPR == 8 || (sub & 1) == 0) && u0 + row < u_end && i < n) key_out[i] = score_key(tot * scale);
             }
         }
-        for (int i = w_lo + tid; i < L; i += NT) s_idx[n_low + (i - w_lo)] = i;
-        n = n_low + (L - w_lo);
     }
+}
+
+// ------------------------------------------------------------------------------------
+// reuse path of finish_kernel: candidate union (Eq. 8-9), candidate scores (Eq. 10), Top-K
+// (Eq. 11), softmax.V (Eq. 12) and the support insert for one head, all in shared memory.
+// ------------------------------------------------------------------------------------
+template <int D, int NT>
+__device__ void reuse_path(const StepArgs& a, unsigned char* smem_raw) {
+    constexpr int NW = NT / 32;
+    // layout (words): qraw[D] sel[r] ws[32] hist[SCRATCH_WORDS] sup_idx[K] sup_key[K] w[K]
+    //                 | big: idx[cap] key[cap], aliased later by red[NW*D+NT] | bitmap | stage[depth*NT*4]
+    float* s_qraw = reinterpret_cast<float*>(smem_raw);
+    int* s_sel = reinterpret_cast<int*>(s_qraw + D);
+    int* s_ws = s_sel + a.r;
+    uint32_t* s_hist = reinterpret_cast<uint32_t*>(s_ws + 32);
+    int32_t* s_sup_idx = reinterpret_cast<int32_t*>(s_hist + SCRATCH_WORDS);
+    uint32_t* s_sup_key = reinterpret_cast<uint32_t*>(s_sup_idx + a.K);
+    float* s_w = reinterpret_cast<float*>(s_sup_key + a.K);
+    const int head_words = (D + a.r + 32 + SCRATCH_WORDS + 3 * a.K + 3) & ~3;
+    int32_t* s_idx = reinterpret_cast<int32_t*>(smem_raw) + head_words;
+    uint32_t* s_key = reinterpret_cast<uint32_t*>(s_idx + a.cap);
+    float* s_red = reinterpret_cast<float*>(s_idx);
+    const int big_words = (max(2 * a.cap, NW * D + NT) + 3) & ~3;
+    uint32_t* s_bm = reinterpret_cast<uint32_t*>(s_idx) + big_words;
+    uint4* s_stage = reinterpret_cast<uint4*>(s_bm + ((((int)a.max_seq_len + 31) / 32 + 3) & ~3));
+
+    const int tid = threadIdx.x;
+    const int bh = blockIdx.x;
+    const int bkv = kv_group_of(bh, a);
+    const int M = a.M, fill = a.fill, L = a.L, K = a.K;
+    const int n_sel = a.r < fill ? a.r : fill;
+    RETOPK_PHASE(0, 0);
+
+    // recalled slots and the raw query from global memory; clear the bitmap meanwhile
+    if (tid < a.r) s_sel[tid] = a.ws_sel[(size_t)bh * a.r + tid];
+    if (tid >= 32 && tid < 32 + D / 2) {
+        const uint32_t raw = reinterpret_cast<const uint32_t*>(a.q + (size_t)bh * D)[tid - 32];
+        s_qraw[2 * (tid - 32)] = bf16_lo(raw);
+        s_qraw[2 * (tid - 32) + 1] = bf16_hi(raw);
+    }
+    {
+        const int nwords = (L + 31) >> 5;
+        uint4* bm4 = reinterpret_cast<uint4*>(s_bm);
+        for (int w = tid; w < (nwords + 3) >> 2; w += NT) bm4[w] = make_uint4(0, 0, 0, 0);
+    }
+    __syncthreads();
+    RETOPK_PHASE(0, 3);
+
+    // Eq. 8-9
+    const int n = candidate_union<NT>(a, bh, s_sel, n_sel, s_bm, s_idx, s_ws);
     __syncthreads();
     RETOPK_PHASE(0, 5);
 
-    // Eq. 10: exact current-query scores on the candidate rows only.  Every lane copies its
-    // 16 bytes of each row asynchronously into its own landing zone and reads them back
-    // itself, so a whole wave of rows is in flight with no registers held and no barrier.
-    {
-        const int sub = lane % LPR, myslot = warp * RPW + lane / LPR;
-        const char* ksrc = reinterpret_cast<const char*>(a.k + (size_t)bkv * a.max_seq_len * D) + sub * 16;
-        float qf[8];
-        *reinterpret_cast<float4*>(qf) = *reinterpret_cast<const float4*>(s_qraw + sub * 8);
-        *reinterpret_cast<float4*>(qf + 4) = *reinterpret_cast<const float4*>(s_qraw + sub * 8 + 4);
-        const int depth = a.stage_depth;
-        uint4* my_stage = s_stage + tid;
-        // each wave goes out as two groups of copies, so that the dot products of the first
-        // half run while the second half is still arriving
-        const int half = (depth + 1) / 2;
-        for (int base = 0; base < n; base += SLOTS * depth) {
-            for (int u = 0; u < depth; ++u) {
-                const int i = base + u * SLOTS + myslot;
-                if (i < n) cp_async16(my_stage + u * NT, ksrc + (size_t)s_idx[i] * (D * 2));
-                if (u == half - 1) cp_async_commit();
-            }
-            cp_async_commit();
-            for (int g2 = 0; g2 < 2; ++g2) {
-                if (g2 == 0) cp_async_wait_but_one();
-                else cp_async_wait_all();
-                const int u_begin = g2 == 0 ? 0 : half, u_end = g2 == 0 ? half : depth;
-                for (int u0 = u_begin; u0 < u_end; u0 += 8) {
-                    float part[8];
-#pragma unroll
-                    for (int uu = 0; uu < 8; ++uu) {
-                        const int i = base + (u0 + uu) * SLOTS + myslot;
-                        part[uu] = (u0 + uu < u_end && i < n) ? dot8(my_stage[(u0 + uu) * NT], qf) : 0.f;
-                    }
-                    int row;
-                    const float tot = reduce8_across<LPR>(part, sub, row);
-                    const int i = base + (u0 + row) * SLOTS + myslot;
-                    if ((LPR == 8 || (sub & 1) == 0) && u0 + row < u_end && i < n) s_key[i] = score_key(tot * a.scale);
-                }
-            }
-        }
-    }
+    // Eq. 10
+    score_candidates<D, NT, true>(a.k + (size_t)bkv * a.max_seq_len * D, s_idx, n, s_qraw, s_stage, a.stage_depth,
+                                  a.scale, s_key);
     __syncthreads();
     RETOPK_PHASE(0, 6);
 
