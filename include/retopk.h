@@ -102,6 +102,29 @@ int retopk_create_batched(retopk_ctx** ctx, int B, int H_q, int H_kv, int d, int
 enum { RETOPK_RECALL_SIMILAR = 0, RETOPK_RECALL_RECENT = 1 };
 int retopk_set_recall_mode(retopk_ctx* ctx, int mode);
 
+/*
+ * Fusion level of the reuse path, for measuring what kernel fusion buys (the paper's kernel
+ * efficiency analysis, Table 4, reports five cumulative stages for its own kernels; the cut
+ * points here follow its description of them and are this library's own).  Results do not
+ * depend on the level: supports and outputs are bit-identical.
+ *   1  separate kernels: similarity | top-r and path | candidate union | pack candidate key
+ *      rows | score packed rows | top-K | softmax.V | cache insert
+ *   2  one kernel for cache search + support union; candidate rows scored through their indices
+ *   3  top-K, softmax.V and the support insert in one kernel
+ *   4  as 3, the intermediate buffers owned by the context; levels 1-3 take them from a
+ *      stream-ordered memory pool (created on first use, blocks kept between steps) and give
+ *      them back in every step
+ *   5  candidate union through output in one kernel (the default)
+ * dependent_launches = 1 (default, only valid with level 5) launches the step's kernels with
+ * programmatic stream serialisation, 0 as plain stream-ordered launches.  Heads on the exact
+ * path run scan + finish at every level.  Levels below 5 allocate device memory: level 4 in
+ * this call (about B*H_q*(2*(r*K+W)) words), levels 1-3 from the pool inside
+ * retopk_decode_step, which then must not run under stream capture.  This call
+ * synchronises the device.  Errors: EINVAL (bad level / flag), EUNSUPPORTED (a kernel of the
+ * level does not fit shared memory), ENOMEM, ECUDA.
+ */
+int retopk_set_fusion_level(retopk_ctx* ctx, int level, int dependent_launches);
+
 /* Release the context and its device memory (synchronises the device). */
 int retopk_destroy(retopk_ctx* ctx);
 

@@ -1,5 +1,6 @@
 // Host side of the ReTopK library: context, argument checks, launch sequence, C interface.
 #include "retopk_kernels.cuh"
+#include "retopk_ladder.cuh"
 
 #include <math.h>
 #include <new>
@@ -45,6 +46,13 @@ struct retopk_ctx {
     uint16_t* stage_out;
     uint16_t* stage_kv;   // [2][B*Hkv*d]
     int last_launches;
+    // fusion ladder (measurement): level 1..5, dependent launches on or off, and the buffers
+    // the unfused levels hand their intermediates through
+    int fusion_level, dependent_launches;
+    cudaMemPool_t pool;          // levels 1-3 draw the buffers from here in every step
+    void* lw_persist[8];         // level 4 keeps them
+    size_t lw_bytes[8];
+    size_t sm_sim, sm_topr, sm_union, sm_discover, sm_score, sm_select, sm_attend, sm_fused;
 };
 
 namespace {
@@ -71,6 +79,8 @@ void free_all(retopk_ctx* c) {
     cudaFree(c->ws_ncand); cudaFree(c->ws_sel); cudaFree(c->ws_gflag); cudaFree(c->ws_scores); cudaFree(c->ws_tmax); cudaFree(c->counters);
     cudaFree(c->status); cudaFree(c->slow_select); cudaFree(c->scan_groups); cudaFree(c->scan_counter); cudaFree(c->stage_q); cudaFree(c->stage_out);
     cudaFree(c->stage_kv);
+    for (int i = 0; i < 8; ++i) cudaFree(c->lw_persist[i]);
+    if (c->pool) cudaMemPoolDestroy(c->pool);
 }
 
 StepArgs make_args(const retopk_ctx* c, const void* q, const void* k, const void* v, long long L,
@@ -112,7 +122,7 @@ StepArgs make_args(const retopk_ctx* c, const void* q, const void* k, const void
 // predecessor in the stream still runs; it waits (pdl_wait) before reading its inputs.
 template <class Kernel>
 int launch_dependent(Kernel kernel, unsigned grid, unsigned block, size_t smem, cudaStream_t s,
-                     const StepArgs& a) {
+                     const StepArgs& a, int allowed = 1) {
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof cfg);
     cfg.gridDim = dim3(grid);
@@ -121,7 +131,7 @@ int launch_dependent(Kernel kernel, unsigned grid, unsigned block, size_t smem, 
     cfg.stream = s;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[0].val.programmaticStreamSerializationAllowed = allowed;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, kernel, a) == cudaSuccess ? RETOPK_OK : RETOPK_ECUDA;
@@ -129,8 +139,8 @@ int launch_dependent(Kernel kernel, unsigned grid, unsigned block, size_t smem, 
 
 int launch_recall(const retopk_ctx* c, const StepArgs& a, cudaStream_t s) {
     const unsigned grid = (unsigned)(c->B * c->Hq);
-    if (c->d == 128) return launch_dependent(recall_kernel<128>, grid, RECALL_THREADS, c->smem_recall, s, a);
-    return launch_dependent(recall_kernel<64>, grid, RECALL_THREADS, c->smem_recall, s, a);
+    if (c->d == 128) return launch_dependent(recall_kernel<128>, grid, RECALL_THREADS, c->smem_recall, s, a, c->dependent_launches);
+    return launch_dependent(recall_kernel<64>, grid, RECALL_THREADS, c->smem_recall, s, a, c->dependent_launches);
 }
 
 int launch_scan(const retopk_ctx* c, const StepArgs& a, cudaStream_t s) {
@@ -143,17 +153,17 @@ int launch_scan(const retopk_ctx* c, const StepArgs& a, cudaStream_t s) {
     // slower: its CTAs then land on SMs still carved up for that kernel, and it needs about
     // 100 KB of L1 per SM to keep its loads in flight.  recall_kernel uses a few KB, so the SMs
     // are back in the default split by the time the scan's CTAs start.
-    if (c->d == 128 && ntile == 1) return launch_dependent(scan_kernel<128, 1>, grid, SCAN_THREADS, 0, s, a);
-    if (c->d == 128) return launch_dependent(scan_kernel<128, 2>, grid, SCAN_THREADS, 0, s, a);
-    if (ntile == 1) return launch_dependent(scan_kernel<64, 1>, grid, SCAN_THREADS, 0, s, a);
-    return launch_dependent(scan_kernel<64, 2>, grid, SCAN_THREADS, 0, s, a);
+    if (c->d == 128 && ntile == 1) return launch_dependent(scan_kernel<128, 1>, grid, SCAN_THREADS, 0, s, a, c->dependent_launches);
+    if (c->d == 128) return launch_dependent(scan_kernel<128, 2>, grid, SCAN_THREADS, 0, s, a, c->dependent_launches);
+    if (ntile == 1) return launch_dependent(scan_kernel<64, 1>, grid, SCAN_THREADS, 0, s, a, c->dependent_launches);
+    return launch_dependent(scan_kernel<64, 2>, grid, SCAN_THREADS, 0, s, a, c->dependent_launches);
 }
 
 int launch_finish(const retopk_ctx* c, const StepArgs& a, cudaStream_t s) {
     const unsigned grid = (unsigned)(c->B * c->Hq);
     const size_t smem = a.mode == MODE_EXACT ? c->smem_exact : c->smem_finish;
-    if (c->d == 128) return launch_dependent(finish_kernel<128>, grid, FINISH_THREADS, smem, s, a);
-    return launch_dependent(finish_kernel<64>, grid, FINISH_THREADS, smem, s, a);
+    if (c->d == 128) return launch_dependent(finish_kernel<128>, grid, FINISH_THREADS, smem, s, a, c->dependent_launches);
+    return launch_dependent(finish_kernel<64>, grid, FINISH_THREADS, smem, s, a, c->dependent_launches);
 }
 
 // Measurement hook: event number `which` (0..3) of the current call, if recording.
@@ -182,6 +192,162 @@ int check_step_args(const retopk_ctx* c, const void* q, const void* k, const voi
     return RETOPK_OK;
 }
 
+// ---------------------------------------------------------------------------------------
+// Fusion ladder (levels 1-4): the reuse path as separate kernels.
+// ---------------------------------------------------------------------------------------
+enum { LW_RHO, LW_QBAR, LW_CAND, LW_KEY, LW_ROWS, LW_SUP_IDX, LW_SUP_KEY, LW_META };
+
+// Which buffers a level needs.
+bool ladder_needs(int level, int which) {
+    switch (which) {
+        case LW_RHO: case LW_QBAR: case LW_ROWS: return level == 1;
+        case LW_SUP_IDX: case LW_SUP_KEY: case LW_META: return level <= 2;
+        default: return true;     // candidates and their keys: every unfused level
+    }
+}
+
+template <class Kernel>
+bool opt_in(Kernel kernel, size_t smem) {
+    return smem <= 48 * 1024 ||
+           cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) == cudaSuccess;
+}
+
+// Shared-memory footprints of the ladder kernels (mirror the carve-ups at their tops).
+int ladder_prepare(retopk_ctx* c) {
+    const size_t d = c->d, K = c->K, cap = c->cap, r = c->r;
+    const size_t Mp = (c->M + 3) & ~3, capp = (cap + 3) & ~(size_t)3;
+    const size_t bm_words = (((size_t)c->max_seq_len + 31) / 32 + 3) & ~(size_t)3;
+    const size_t red_words = (size_t)(LADDER_THREADS / 32) * d + LADDER_THREADS;
+    const size_t wave = (size_t)LADDER_THREADS * 16 * c->stage_depth;
+    const size_t union_words = ((r + 3) & ~(size_t)3) + 32 + capp + bm_words;
+    c->sm_sim = (d + Mp) * 4;
+    c->sm_topr = (Mp + r + 4) * 4;
+    c->sm_union = union_words * 4;
+    c->sm_discover = (d + Mp + 4 + union_words) * 4;
+    c->sm_score = (d + capp) * 4 + wave;
+    c->sm_select = (32 + SCRATCH_WORDS + 2 * K + 2 * cap) * 4;
+    c->sm_attend = (32 + ((3 * K + 3) & ~(size_t)3) + red_words) * 4 + wave;
+    const size_t head_words = (32 + SCRATCH_WORDS + 3 * K + 3) & ~(size_t)3;
+    const size_t big_words = ((2 * cap > red_words ? 2 * cap : red_words) + 3) & ~(size_t)3;
+    c->sm_fused = (head_words + big_words) * 4 + wave;
+    int max_smem = 0;
+    cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, c->device);
+    const size_t all[] = {c->sm_sim, c->sm_topr, c->sm_union, c->sm_discover, c->sm_score, c->sm_select,
+                          c->sm_attend, c->sm_fused};
+    for (size_t v : all)
+        if (v > (size_t)max_smem) return RETOPK_EUNSUPPORTED;
+    bool ok = opt_in(ladder_topr_kernel, c->sm_topr) && opt_in(ladder_union_kernel, c->sm_union) &&
+              opt_in(ladder_select_kernel, c->sm_select);
+    if (c->d == 128)
+        ok = ok && opt_in(ladder_similarity_kernel<128>, c->sm_sim) && opt_in(ladder_discover_kernel<128>, c->sm_discover) &&
+             opt_in(ladder_score_kernel<128, true>, c->sm_score) && opt_in(ladder_score_kernel<128, false>, c->sm_score) &&
+             opt_in(ladder_attend_kernel<128>, c->sm_attend) &&
+             opt_in(ladder_select_attend_insert_kernel<128>, c->sm_fused);
+    else
+        ok = ok && opt_in(ladder_similarity_kernel<64>, c->sm_sim) && opt_in(ladder_discover_kernel<64>, c->sm_discover) &&
+             opt_in(ladder_score_kernel<64, true>, c->sm_score) && opt_in(ladder_score_kernel<64, false>, c->sm_score) &&
+             opt_in(ladder_attend_kernel<64>, c->sm_attend) &&
+             opt_in(ladder_select_attend_insert_kernel<64>, c->sm_fused);
+    if (!ok) { cudaGetLastError(); return RETOPK_ECUDA; }
+    const size_t nh = (size_t)c->B * c->Hq;
+    c->lw_bytes[LW_RHO] = nh * c->M * 4;
+    c->lw_bytes[LW_QBAR] = nh * d * 4;
+    c->lw_bytes[LW_CAND] = nh * cap * 4;
+    c->lw_bytes[LW_KEY] = nh * cap * 4;
+    c->lw_bytes[LW_ROWS] = nh * cap * d * 2;
+    c->lw_bytes[LW_SUP_IDX] = nh * K * 4;
+    c->lw_bytes[LW_SUP_KEY] = nh * K * 4;
+    c->lw_bytes[LW_META] = nh * 4 * 4;
+    return RETOPK_OK;
+}
+
+void ladder_bind(StepArgs& a, void* const* buf) {
+    a.lw_rho = static_cast<float*>(buf[LW_RHO]);
+    a.lw_qbar = static_cast<float*>(buf[LW_QBAR]);
+    a.lw_cand = static_cast<int32_t*>(buf[LW_CAND]);
+    a.lw_key = static_cast<uint32_t*>(buf[LW_KEY]);
+    a.lw_rows = static_cast<uint16_t*>(buf[LW_ROWS]);
+    a.lw_sup_idx = static_cast<int32_t*>(buf[LW_SUP_IDX]);
+    a.lw_sup_key = static_cast<uint32_t*>(buf[LW_SUP_KEY]);
+    a.lw_meta = static_cast<int32_t*>(buf[LW_META]);
+}
+
+#define LADDER_LAUNCH(kernel, smem, ...)                                    \
+    do {                                                                    \
+        kernel<<<grid, LADDER_THREADS, smem, s>>>(__VA_ARGS__);             \
+        if (cudaGetLastError() != cudaSuccess) return RETOPK_ECUDA;         \
+        ++launches;                                                         \
+    } while (0)
+
+// One decode step at fusion level 1..4.  Order: decision kernels, scan (exact heads), the
+// reuse path's kernels, finish_kernel (exact heads only).
+int ladder_step(retopk_ctx* c, StepArgs a, cudaStream_t s) {
+    const int level = c->fusion_level;
+    const unsigned grid = (unsigned)(c->B * c->Hq);
+    int launches = 0, rc;
+    void* buf[8] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
+    if (level == 4) {
+        for (int i = 0; i < 8; ++i) buf[i] = c->lw_persist[i];
+    } else {
+        for (int i = 0; i < 8; ++i)
+            if (ladder_needs(level, i) &&
+                cudaMallocFromPoolAsync(&buf[i], c->lw_bytes[i] ? c->lw_bytes[i] : 16, c->pool, s) != cudaSuccess) {
+                for (int j = 0; j < i; ++j) if (buf[j]) cudaFreeAsync(buf[j], s);
+                cudaGetLastError();
+                return RETOPK_ENOMEM;
+            }
+    }
+    ladder_bind(a, buf);
+    a.skip_reuse = 1;
+    const bool d128 = c->d == 128;
+
+    prof_mark(c, 0, s);
+    if (level == 1) {
+        if (d128) LADDER_LAUNCH(ladder_similarity_kernel<128>, c->sm_sim, a);
+        else LADDER_LAUNCH(ladder_similarity_kernel<64>, c->sm_sim, a);
+        LADDER_LAUNCH(ladder_topr_kernel, c->sm_topr, a);
+    } else {
+        if (d128) LADDER_LAUNCH(ladder_discover_kernel<128>, c->sm_discover, a);
+        else LADDER_LAUNCH(ladder_discover_kernel<64>, c->sm_discover, a);
+    }
+    prof_mark(c, 1, s);
+    if ((rc = launch_scan(c, a, s)) != RETOPK_OK) return rc;
+    ++launches;
+    prof_mark(c, 2, s);
+    if (level == 1) {
+        LADDER_LAUNCH(ladder_union_kernel, c->sm_union, a);
+        if (d128) {
+            LADDER_LAUNCH(ladder_pack_rows_kernel<128>, 0, a);
+            LADDER_LAUNCH((ladder_score_kernel<128, false>), c->sm_score, a);
+        } else {
+            LADDER_LAUNCH(ladder_pack_rows_kernel<64>, 0, a);
+            LADDER_LAUNCH((ladder_score_kernel<64, false>), c->sm_score, a);
+        }
+    } else {
+        if (d128) LADDER_LAUNCH((ladder_score_kernel<128, true>), c->sm_score, a);
+        else LADDER_LAUNCH((ladder_score_kernel<64, true>), c->sm_score, a);
+    }
+    if (level <= 2) {
+        LADDER_LAUNCH(ladder_select_kernel, c->sm_select, a);
+        if (d128) LADDER_LAUNCH(ladder_attend_kernel<128>, c->sm_attend, a);
+        else LADDER_LAUNCH(ladder_attend_kernel<64>, c->sm_attend, a);
+        LADDER_LAUNCH(ladder_insert_kernel, 0, a, level == 1 ? 1 : 0);
+    } else {
+        if (d128) LADDER_LAUNCH(ladder_select_attend_insert_kernel<128>, c->sm_fused, a);
+        else LADDER_LAUNCH(ladder_select_attend_insert_kernel<64>, c->sm_fused, a);
+    }
+    if ((rc = launch_finish(c, a, s)) != RETOPK_OK) return rc;
+    ++launches;
+    prof_mark(c, 3, s);
+    prof_done(c, 0);
+    if (level != 4)
+        for (int i = 0; i < 8; ++i)
+            if (buf[i] && cudaFreeAsync(buf[i], s) != cudaSuccess) return RETOPK_ECUDA;
+    c->last_launches = launches;
+    return RETOPK_OK;
+}
+#undef LADDER_LAUNCH
+
 }  // namespace
 
 extern "C" {
@@ -204,6 +370,8 @@ int retopk_create_batched(retopk_ctx** out, int B, int H_q, int H_kv, int d, int
     c->B = B; c->Hq = H_q; c->Hkv = H_kv; c->G = H_q / H_kv; c->d = d; c->M = M; c->r = r; c->W = W;
     c->K = K; c->R = R; c->tau = tau; c->max_seq_len = max_seq_len;
     c->cap = r * K + W;
+    c->fusion_level = 5;
+    c->dependent_launches = 1;
     c->score_stride = (max_seq_len + TILE_ROWS - 1) / TILE_ROWS * TILE_ROWS;   // whole 16-row tiles
     c->tmax_stride = ((max_seq_len + TILE_ROWS - 1) / TILE_ROWS + 3) / 4 * 4;
     // exact path: shared lists for the scores that reach the tile bound (about 1.1-1.4 K of them,
@@ -290,6 +458,37 @@ int retopk_set_recall_mode(retopk_ctx* c, int mode) {
     return RETOPK_OK;
 }
 
+int retopk_set_fusion_level(retopk_ctx* c, int level, int dependent_launches) {
+    if (!c || level < 1 || level > 5 || (dependent_launches != 0 && dependent_launches != 1)) return RETOPK_EINVAL;
+    if (dependent_launches && level != 5) return RETOPK_EINVAL;   // the unfused kernels are plain launches
+    DeviceGuard g(c->device);
+    if (level < 5) {
+        int rc = ladder_prepare(c);
+        if (rc != RETOPK_OK) return rc;
+        if (cudaDeviceSynchronize() != cudaSuccess) return RETOPK_ECUDA;
+        if (level == 4) {
+            for (int i = 0; i < 8; ++i)
+                if (ladder_needs(4, i) && !c->lw_persist[i] &&
+                    cudaMalloc(&c->lw_persist[i], c->lw_bytes[i] ? c->lw_bytes[i] : 16) != cudaSuccess) {
+                    cudaGetLastError();
+                    return RETOPK_ENOMEM;
+                }
+        } else if (!c->pool) {
+            cudaMemPoolProps props;
+            memset(&props, 0, sizeof props);
+            props.allocType = cudaMemAllocationTypePinned;
+            props.location.type = cudaMemLocationTypeDevice;
+            props.location.id = c->device;
+            if (cudaMemPoolCreate(&c->pool, &props) != cudaSuccess) { cudaGetLastError(); c->pool = nullptr; return RETOPK_ECUDA; }
+            unsigned long long keep = ~0ull;     // freed blocks stay with the pool for the next step
+            cudaMemPoolSetAttribute(c->pool, cudaMemPoolAttrReleaseThreshold, &keep);
+        }
+    }
+    c->fusion_level = level;
+    c->dependent_launches = dependent_launches;
+    return RETOPK_OK;
+}
+
 int retopk_destroy(retopk_ctx* c) {
     if (!c) return RETOPK_EINVAL;
     DeviceGuard g(c->device);
@@ -318,6 +517,12 @@ int retopk_decode_step(retopk_ctx* c, const void* q, const void* k_cache, const 
     StepArgs a = make_args(c, q, k_cache, v_cache, seq_len, out, MODE_RETOPK);
     c->call_serial = (c->call_serial + 1) & 0x3fffffff;
     a.step_id = c->call_serial;
+    if (c->fusion_level < 5) {
+        if ((rc = ladder_step(c, a, s)) != RETOPK_OK) return rc;
+        c->n_ins += 1;
+        c->t_dec += 1;
+        return RETOPK_OK;
+    }
     prof_mark(c, 0, s);
     if ((rc = launch_recall(c, a, s)) != RETOPK_OK) return rc;
     prof_mark(c, 1, s);

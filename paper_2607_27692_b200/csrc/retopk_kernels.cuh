@@ -85,6 +85,18 @@ struct StepArgs {
     unsigned long long* scan_groups;
     unsigned int* scan_counter;  // pool cursor of scan_kernel; finish_kernel resets it
     int32_t* idx_out;        // MODE_EXACT only, may be null
+    // Fusion-ladder levels below the production one (see retopk_ladder.cuh): the reuse path runs
+    // as separate kernels that hand their intermediates on through these global buffers, and
+    // finish_kernel then leaves heads on the reuse path alone.
+    int skip_reuse;
+    float* lw_rho;           // [B*Hq][M] similarities
+    float* lw_qbar;          // [B*Hq][d] normalised query
+    int32_t* lw_cand;        // [B*Hq][cap] candidate indices
+    uint32_t* lw_key;        // [B*Hq][cap] candidate score keys
+    uint16_t* lw_rows;       // [B*Hq][cap][d] packed candidate key rows (level 1 only)
+    int32_t* lw_sup_idx;     // [B*Hq][K] selected indices
+    uint32_t* lw_sup_key;    // [B*Hq][K] their score keys
+    int32_t* lw_meta;        // [B*Hq][4] ns, kmax, kmax_known, -
 };
 
 // ------------------------------------------------------------------------------------
@@ -1209,8 +1221,11 @@ __global__ void __launch_bounds__(FINISH_THREADS, 1) finish_kernel(const StepArg
     extern __shared__ __align__(16) unsigned char smem_raw[];
     pdl_wait();        // scores and tile maxima come from the scan, recalled slots and paths from recall_kernel
     if (blockIdx.x == 0 && threadIdx.x == 0) *a.scan_counter = 0u;      // the scan before this kernel is complete
-    if (a.mode == MODE_RETOPK && a.ws_path[blockIdx.x] == PATH_REUSE) reuse_path<D, FINISH_THREADS>(a, smem_raw);
-    else exact_path<D, FINISH_THREADS>(a, smem_raw);
+    if (a.mode == MODE_RETOPK && a.ws_path[blockIdx.x] == PATH_REUSE) {
+        if (!a.skip_reuse) reuse_path<D, FINISH_THREADS>(a, smem_raw);
+    } else {
+        exact_path<D, FINISH_THREADS>(a, smem_raw);
+    }
 }
 
 // Clear the caches (supports to -1, queries and counters to 0).

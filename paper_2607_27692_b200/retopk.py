@@ -37,6 +37,7 @@ SIGNATURES = {
     "retopk_create": (_i32, [C.POINTER(_vp)] + [_i32] * 7 + [_f32, _i32]),
     "retopk_create_batched": (_i32, [C.POINTER(_vp)] + [_i32] * 8 + [_f32, _i32, _i64]),
     "retopk_set_recall_mode": (_i32, [_vp, _i32]),
+    "retopk_set_fusion_level": (_i32, [_vp, _i32, _i32]),
     "retopk_destroy": (_i32, [_vp]),
     "retopk_reset": (_i32, [_vp, _vp]),
     "retopk_decode_step": (_i32, [_vp, _vp, _vp, _vp, _i64, _vp, _vp]),
@@ -145,6 +146,10 @@ class ReTopK:
     def set_recall_mode(self, mode: int):
         """0: recall the most similar entries (Eq. 7); 1: the most recent ones (Recent-R ablation row)."""
         _check(self.lib.retopk_set_recall_mode(self.h, mode), "retopk_set_recall_mode")
+
+    def set_fusion_level(self, level: int, dependent_launches: bool = False):
+        """Fusion level 1..5 of the reuse path (Table 4's ladder); results do not depend on it."""
+        _check(self.lib.retopk_set_fusion_level(self.h, level, int(dependent_launches)), "retopk_set_fusion_level")
 
     def reset(self):
         _check(self.lib.retopk_reset(self.h, _stream()), "retopk_reset")
