@@ -267,6 +267,30 @@ def fidelity_pass(layers, torch, calls=96):
                     "97.4% output cosine on reuse steps for Qwen2.5-7B on PG19 (other data: context only)"}
 
 
+def fusion_ladder(layers, W, K, torch, dist):
+    """The reuse path at every fusion level (Table 4's experiment), same inputs and path mixture.
+
+    Levels 1-5 are plain stream-ordered launches; "5+dependent" is the default configuration.
+    """
+    out = {}
+    for mix, override in (("tau_0.85", dict(tau=0.85)), ("pure_reuse", dict(tau=-2.0, R=0))):
+        rows = {}
+        for name, level, dependent in (("L1", 1, False), ("L2", 2, False), ("L3", 3, False), ("L4", 4, False),
+                                       ("L5", 5, False), ("L5+dependent", 5, True)):
+            layers.make_contexts(**override)
+            for c in layers.ctx:
+                c.set_fusion_level(level, dependent)
+            res = timed_pass(layers, "retopk", W, K, torch, dist)
+            rows[name] = {"us_per_step": round(res["us_per_step"], 2),
+                          "launches_per_step": layers.ctx[0].last_launch_count(),
+                          "mix": path_mix(res["stats"])}
+        base = rows["L1"]["us_per_step"]
+        for r in rows.values():
+            r["vs_L1"] = round(base / r["us_per_step"], 3)
+        out[mix] = rows
+    return out
+
+
 def cpu_baseline(cfg, stream, budget_s=12.0, max_steps=48):
     """The fp64 oracle, as it stands, on the first decode steps of layer 0."""
     from oracle import retopk_oracle
@@ -320,6 +344,7 @@ def run_gpu(args):
     layers.make_contexts(tau=0.85)
     paper = timed_pass(layers, "retopk", W, K, torch, dist)
     fidelity = fidelity_pass(layers, torch, calls=min(96, W + K)) if rank == 0 else None
+    ladder = fusion_ladder(layers, W, K, torch, dist) if args.ladder else None
 
     # roofline of the dominant kernel of the headline pass
     abytes = algorithmic_bytes(cfg, prof["stats"], mean_L, mean_fill)
@@ -378,6 +403,7 @@ def run_gpu(args):
         "slow_select": head["stats"]["slow_select"],
         "fidelity_tau_0.85": fidelity,
         "roofline": roofline,
+        "fusion_ladder": ladder,
         "paper_context": "paper: 3.07x attention speedup over Exact Top-K at 128K, K=512 on one NVIDIA L20 "
                          "(Qwen2.5-7B, PG19, tau=0.85); about 115 us per layer at 128K (Table 4 / 28 layers)",
     }
@@ -452,6 +478,8 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--ladder", action="store_true",
+                    help="also time the reuse path at every fusion level (adds \"fusion_ladder\" to the line)")
     ap.add_argument("--config", default="headline128k", choices=sorted(wl.CONFIGS))
     ap.add_argument("--layers", type=int, default=4, help="independent layers rotated over (L2 hygiene)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
