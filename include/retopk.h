@@ -186,6 +186,13 @@ int retopk_last_step(retopk_ctx* ctx, int32_t* support, uint8_t* path, float* rh
                      int32_t* n_cand, void* stream);
 
 /*
+ * The cache slots recalled by the most recent retopk_decode_step (Eq. 7), most similar
+ * first: sel [B,H_q,r] int32 (device pointer), -1 where fewer than r entries were cached.
+ * Written for every head, whatever path it then took.  Enqueued on `stream`.
+ */
+int retopk_last_recall(retopk_ctx* ctx, int32_t* sel, void* stream);
+
+/*
  * Cache state out / in (device pointers): qbar [B,H_q,M,d] float32 normalised queries,
  * supports [B,H_q,M,K] int32 (ascending, -1 padded); the entry inserted n-th sits in slot
  * n % M.  n_inserted and t_dec are host scalars.  Import replaces the whole state (this

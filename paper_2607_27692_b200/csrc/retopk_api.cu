@@ -654,6 +654,13 @@ int retopk_last_step(retopk_ctx* c, int32_t* support, uint8_t* path, float* rho_
     return ok ? RETOPK_OK : RETOPK_ECUDA;
 }
 
+int retopk_last_recall(retopk_ctx* c, int32_t* sel, void* stream) {
+    if (!c || !sel || c->n_ins < 1) return RETOPK_EINVAL;
+    const size_t bytes = (size_t)c->B * c->Hq * c->r * 4;
+    return cudaMemcpyAsync(sel, c->ws_sel, bytes, cudaMemcpyDeviceToDevice, static_cast<cudaStream_t>(stream)) == cudaSuccess
+               ? RETOPK_OK : RETOPK_ECUDA;
+}
+
 int retopk_export_state(retopk_ctx* c, float* qbar, int32_t* supports, int64_t* n_inserted,
                         int64_t* t_dec, void* stream) {
     if (!c) return RETOPK_EINVAL;

@@ -47,6 +47,7 @@ SIGNATURES = {
     "exact_topk_decode_static": (_i32, [_i32] * 5 + [_i64, _vp, _vp, _vp, _i64, _vp, _vp, _vp]),
     "retopk_stats": (_i32, [_vp, C.POINTER(_Stats)]),
     "retopk_last_step": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp]),
+    "retopk_last_recall": (_i32, [_vp, _vp, _vp]),
     "retopk_export_state": (_i32, [_vp, _vp, _vp, C.POINTER(_i64), C.POINTER(_i64), _vp]),
     "retopk_import_state": (_i32, [_vp, _vp, _vp, _i64, _i64, _vp]),
     "retopk_profile_begin": (_i32, [_vp, _i32]),
@@ -209,6 +210,12 @@ class ReTopK:
                                        ncand.data_ptr(), _stream())
         _check(rc, "retopk_last_step")
         return dict(support=sup, path=path, rho_max=rho, n_cand=ncand)
+
+    def last_recall(self):
+        """Cache slots recalled by the last step (Eq. 7), most similar first, -1 padded: [B, H_q, r] int32."""
+        sel = torch.empty((self.B, self.H_q, self.r), dtype=torch.int32, device=self.device)
+        _check(self.lib.retopk_last_recall(self.h, sel.data_ptr(), _stream()), "retopk_last_recall")
+        return sel
 
     def export_state(self):
         dev = self.device

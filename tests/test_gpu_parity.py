@@ -345,3 +345,38 @@ def test_recent_recall_variant_teacher_forced(rt, P, oracle_mod):
     for t in range(30):
         o2.decode_step(st2.q[t], st2.k, st2.v, st2.seq_len(t))
     assert o2.stats()["fallback"] != so["fallback"] or o2.stats()["cand_sum"] != so["cand_sum"]
+
+
+def test_last_recall_reports_the_most_similar_slots(rt, P, oracle_mod):
+    """retopk_last_recall against similarities recomputed in fp64 from the oracle's cache (Eq. 6-7)."""
+    cfg = wl.CONFIGS["tiny"].replace(context=600, steps=28, B=2, H_q=4, H_kv=2, M=8, r=3)
+    st, o, g, k, v = stream_case(rt, P, oracle_mod, cfg, cfg.steps)
+    same_as_oracle = 0
+    for t in range(cfg.steps):
+        qbar, sup, n_ins, t_dec = o.export_state()
+        g.import_state(torch.from_numpy(qbar.astype(np.float32)).cuda(), torch.from_numpy(sup).cuda(), n_ins, t_dec)
+        g.decode_step(P.to_dev(st.q[t]), k, v, st.seq_len(t))
+        o.decode_step(st.q[t], st.k, st.v, st.seq_len(t))
+        sel = g.last_recall().cpu().numpy()
+        fill = min(n_ins, cfg.M)
+        q = wl.bf16_bits_to_f64(st.q[t])
+        rho = np.einsum("bhmd,bhd->bhm", qbar, q) / np.linalg.norm(q, axis=-1)[..., None]
+        for b in range(cfg.B):
+            for h in range(cfg.H_q):
+                got = sel[b, h]
+                n_sel = min(cfg.r, fill)
+                assert (got[n_sel:] == -1).all() and (got[:n_sel] >= 0).all() and (got[:n_sel] < fill).all()
+                assert len(set(got[:n_sel])) == n_sel
+                if n_sel == 0:
+                    continue
+                r_sorted = np.sort(rho[b, h, :fill])[::-1]
+                mine = rho[b, h, got[:n_sel]]
+                assert (np.diff(mine) <= 1e-5).all()                 # most similar first
+                assert (mine >= r_sorted[n_sel - 1] - 1e-5).all()     # and none better left out
+                last = o.last_step()
+                if last["path"][b, h] == 0:        # the oracle records its recall on reuse steps
+                    gaps = -np.diff(r_sorted[:n_sel + 1])
+                    if gaps.size == 0 or gaps.min() > 1e-5:
+                        assert list(got) == list(last["sel"][b, h])
+                        same_as_oracle += 1
+    assert same_as_oracle > 0.3 * cfg.steps * cfg.B * cfg.H_q
