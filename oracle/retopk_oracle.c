@@ -43,7 +43,11 @@
  *   - prefill seeding (Sec. 3.3: the cache "is initialized from the final C prompt tokens"):
  *     the paper does not say which support a prompt token gets; here each of the last
  *     n_tail <= M prompt positions p contributes its normalised query and its CAUSAL Exact
- *     Top-K support over keys 0..p, oldest first; the decode offset stays 0.
+ *     Top-K support over keys 0..p, oldest first; the decode offset stays 0;
+ *   - bf16 query cache (a storage variant; the paper runs everything in BF16 and does not say
+ *     how the cached queries are kept): each element of the normalised query is rounded once,
+ *     to nearest even, to bf16 when it is stored; the similarity of a later step is the dot
+ *     product of that step's unrounded normalised query with the stored rounded one.
  *
  * Inputs are bf16 bit patterns, widened exactly to double; every sum is a plain
  * left-to-right fp64 loop; selection is a full sort.  OpenMP only spreads independent
@@ -72,6 +76,7 @@ enum { PATH_REUSE = 0, PATH_FALLBACK = 1, PATH_REFRESH = 2 };
 typedef struct {
     int B, Hq, Hkv, d, M, r, W, K, R;
     int recall_mode; /* 0: the r most similar cached queries (Eq. 7); 1: the r most recent ones */
+    int qbar_bf16;   /* 1: cached normalised queries are rounded to bf16 when stored */
     double tau;
     int64_t max_seq_len;
     int64_t n_ins;   /* entries inserted so far (same for every head) */
@@ -150,6 +155,23 @@ int oracle_create(oracle_t **out, int B, int Hq, int Hkv, int d, int M, int r, i
 int oracle_set_recall_mode(oracle_t *o, int mode) {
     if ((mode != 0 && mode != 1) || (mode == 1 && o->r > 64)) return -1;
     o->recall_mode = mode;
+    return 0;
+}
+
+/* Nearest bf16 value (8 significand bits, ties to even) of a double, as a double. */
+static double round_to_bf16(double x) {
+    if (x == 0.0 || !isfinite(x)) return x;
+    int e;
+    frexp(x, &e);                 /* |x| = f * 2^e with f in [0.5, 1) */
+    if (e < -125) e = -125;       /* below the normal range the spacing stays 2^-133 */
+    return ldexp(nearbyint(ldexp(x, 8 - e)), e - 8);   /* nearbyint: round half to even */
+}
+
+/* 0: cached queries kept as computed (default); 1: rounded to bf16 when stored.  Only while
+ * the cache is empty. */
+int oracle_set_qbar_format(oracle_t *o, int fmt) {
+    if ((fmt != 0 && fmt != 1) || o->n_ins != 0) return -1;
+    o->qbar_bf16 = fmt;
     return 0;
 }
 
@@ -335,7 +357,8 @@ static void retopk_head(oracle_t *o, size_t bh, const double *q, const uint16_t 
 
     /* insert (qbar_t, S_t) at the ring position; happens after recall on either path */
     int slot = (int)(o->n_ins % M);
-    memcpy(cache_q + (size_t)slot * d, qbar, (size_t)d * sizeof(double));
+    for (int j = 0; j < d; ++j)
+        cache_q[(size_t)slot * d + j] = o->qbar_bf16 ? round_to_bf16(qbar[j]) : qbar[j];
     memcpy(cache_s + (size_t)slot * K, sup, (size_t)K * sizeof(int32_t));
 
     o->last_path[bh] = (uint8_t)path;
@@ -403,7 +426,10 @@ int oracle_prefill(oracle_t *o, const uint16_t *q_tail, const uint16_t *k, const
             exact_head(qd, k + kv, v + kv, L, d, K, sup, out, &kth);
             const double nrm = sqrt(nrm2);
             double *cq = o->qbar + ((size_t)bh * M + slot) * d;
-            for (int t = 0; t < d; ++t) cq[t] = nrm > 0.0 ? qd[t] / nrm : 0.0;
+            for (int t = 0; t < d; ++t) {
+                cq[t] = nrm > 0.0 ? qd[t] / nrm : 0.0;
+                if (o->qbar_bf16) cq[t] = round_to_bf16(cq[t]);
+            }
             memcpy(o->sup + ((size_t)bh * M + slot) * K, sup, (size_t)K * sizeof(int32_t));
             free(qd); free(out); free(sup);
         }

@@ -52,6 +52,8 @@ def _load():
         lib.oracle_prefill.restype = i32
         lib.oracle_set_recall_mode.argtypes = [vp, i32]
         lib.oracle_set_recall_mode.restype = i32
+        lib.oracle_set_qbar_format.argtypes = [vp, i32]
+        lib.oracle_set_qbar_format.restype = i32
         lib.oracle_stats.argtypes = [vp, vp]
         lib.oracle_stats.restype = None
         lib.oracle_last_step.argtypes = [vp] * 7
@@ -157,6 +159,11 @@ class Oracle:
         """0: recall the most similar entries (the method); 1: the most recent ones (Recent-R ablation)."""
         if self.lib.oracle_set_recall_mode(self.h, mode) != 0:
             raise ValueError("bad recall mode")
+
+    def set_qbar_format(self, fmt: int):
+        """0: cached queries kept in full precision; 1: rounded to bf16 when stored (empty cache only)."""
+        if self.lib.oracle_set_qbar_format(self.h, fmt) != 0:
+            raise ValueError("bad format, or the cache is not empty")
 
     def stats(self) -> dict:
         five = np.zeros(5, dtype=np.int64)

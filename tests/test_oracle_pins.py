@@ -455,3 +455,46 @@ def test_recent_recall_falls_back_on_its_own_maximum(oracle_mod):
         o.import_state(qc, sup, 4, 1)       # ring full: newest are slots 3 and 2
         o.decode_step(q, k, k, 20)
         assert o.last_step()["path"][0, 0] == want
+
+
+def test_bf16_query_cache_rounds_once_to_nearest(oracle_mod):
+    """bf16 storage of the cached queries: every stored element is a bf16 value, the nearest one
+    to the fp64 normalised query, and later similarities use the stored values as they are."""
+    cfg = wl.CONFIGS["tiny"].replace(context=200, steps=10, H_q=2, H_kv=1, B=2, M=4)
+    st = wl.make_stream(cfg, steps=cfg.steps)
+    o = oracle_mod.Oracle.from_config(cfg)
+    o.set_qbar_format(1)
+    off_grid = 0
+    for t in range(cfg.steps):
+        qbar_before, _, n_ins, _ = o.export_state()
+        o.decode_step(st.q[t], st.k, st.v, st.seq_len(t))
+        q = wl.bf16_bits_to_f64(st.q[t])
+        exact = q / np.linalg.norm(q, axis=-1, keepdims=True)
+        # similarities of this step: unrounded current query against the stored entries
+        fill = min(n_ins, cfg.M)
+        if fill:
+            rho = np.einsum("bhmd,bhd->bhm", qbar_before[:, :, :fill], exact)
+            assert np.allclose(o.last_step()["rho_max"], rho.max(-1), rtol=0, atol=1e-13)
+        stored = o.export_state()[0][:, :, n_ins % cfg.M]
+        # representable: a round trip through the 16-bit pattern changes nothing
+        assert np.array_equal(wl.bf16_bits_to_f64(wl.f32_to_bf16_bits(stored.astype(np.float32))), stored)
+        # nearest: within half a unit in the last of bf16's 8 significand bits
+        ulp = 2.0 ** (np.floor(np.log2(np.abs(exact))) - 7)
+        assert (np.abs(stored - exact) <= 0.5 * ulp * (1 + 1e-12)).all()
+        off_grid += int((stored != exact).sum())
+    assert off_grid > 0.9 * cfg.steps * cfg.B * cfg.H_q * cfg.d      # the rounding really happened
+
+
+def test_bf16_query_cache_is_off_by_default_and_only_set_on_an_empty_cache(oracle_mod):
+    cfg = wl.CONFIGS["tiny"].replace(context=100, steps=3, H_q=1, H_kv=1)
+    st = wl.make_stream(cfg, steps=3)
+    o = oracle_mod.Oracle.from_config(cfg)
+    o.decode_step(st.q[0], st.k, st.v, st.seq_len(0))
+    q = wl.bf16_bits_to_f64(st.q[0])
+    assert np.allclose(o.export_state()[0][:, :, 0], q / np.linalg.norm(q, axis=-1, keepdims=True), rtol=0, atol=1e-15)
+    with pytest.raises(ValueError):
+        o.set_qbar_format(1)
+    o.reset()
+    o.set_qbar_format(1)
+    with pytest.raises(ValueError):
+        o.set_qbar_format(2)
