@@ -130,11 +130,15 @@ class Layers:
                 np.ascontiguousarray(s.v[:, :, rows].transpose(2, 0, 1, 3)), pin=True))
         self.out_host = torch.empty((cfg.B, cfg.H_q, cfg.d), dtype=torch.bfloat16).pin_memory()
         self.ctx = []
+        self.qbar_bf16 = False
 
     def make_contexts(self, **override):
         for c in self.ctx:
             c.close()
         self.ctx = [self.rt.ReTopK.from_config(self.cfg, **override) for _ in range(self.n)]
+        if self.qbar_bf16:
+            for c in self.ctx:
+                c.set_qbar_format(1)
 
     def stats(self):
         tot = {}
@@ -212,13 +216,16 @@ def timed_pass(layers, kind, warmup, steps, torch, dist, profile=False, sampler=
     return dict(ms=ms, us_per_step=1e3 * ms / steps, stats=delta, prof=prof, launches=launches)
 
 
+QBAR_BYTES = 4      # bytes per cached query element; 2 with --qbar-bf16
+
+
 def algorithmic_bytes(cfg, stats, mean_L, mean_fill):
     """Bytes the method has to move for the head-steps in `stats` (not score spills)."""
     d, K = cfg.d, cfg.K
     heads = stats["steps"]
     n_sel = min(cfg.r, mean_fill)
     tail = K * d * 2 + K * 4 + d * 2          # value rows, support insert, output
-    recall = heads * (mean_fill * d * 4 + d * 4 + d * 2)
+    recall = heads * (mean_fill * d * QBAR_BYTES + d * QBAR_BYTES + d * 2)
     scan = stats["scan_groups"] * mean_L * d * 2
     finish = heads * tail + stats["reuse"] * (n_sel * K * 4 + d * 2) + stats["cand_sum"] * d * 2
     return dict(recall=recall, scan=scan, finish=finish)
@@ -355,6 +362,9 @@ def run_gpu(args):
     if t_per_layer > cfg.steps:      # a longer run than the configuration's: extend the KV layout
         cfg = cfg.replace(steps=t_per_layer)
     layers = Layers(cfg, n_layers, t_per_layer, rank, torch, rt)
+    layers.qbar_bf16 = args.qbar_bf16
+    global QBAR_BYTES
+    QBAR_BYTES = 2 if args.qbar_bf16 else 4
     peak, peak_kind = measured_peaks()
     mean_t = (W + K / 2) / n_layers
     mean_L = cfg.context + mean_t + 1
@@ -418,7 +428,7 @@ def run_gpu(args):
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": cfg.name, "B": cfg.B, "H_q": cfg.H_q, "H_kv": cfg.H_kv, "d": cfg.d,
                    "context": cfg.context, "K": cfg.K, "M": cfg.M, "r": cfg.r, "W": cfg.W, "tau": cfg.tau,
-                   "R": cfg.R, "layers_rotated": n_layers, "decode_steps_per_layer": t_per_layer,
+                   "R": cfg.R, "qbar_cache": "bf16" if args.qbar_bf16 else "fp32", "layers_rotated": n_layers, "decode_steps_per_layer": t_per_layer,
                    "l2": "inputs larger than L2: calls rotate over independent layers",
                    "parallelism": "replicas only" if world > 1 else "single GPU"},
         "clocks": sampler.summary(),
@@ -512,6 +522,8 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--qbar-bf16", action="store_true",
+                    help="keep the cached normalised queries in bf16 (storage variant) in every pass")
     ap.add_argument("--ladder", action="store_true",
                     help="also time the reuse path at every fusion level (adds \"fusion_ladder\" to the line)")
     ap.add_argument("--config", default="headline128k", choices=sorted(wl.CONFIGS))

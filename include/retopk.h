@@ -103,6 +103,19 @@ enum { RETOPK_RECALL_SIMILAR = 0, RETOPK_RECALL_RECENT = 1 };
 int retopk_set_recall_mode(retopk_ctx* ctx, int mode);
 
 /*
+ * Storage format of the cached normalised queries.  RETOPK_QBAR_FP32 (default) keeps them as
+ * computed; RETOPK_QBAR_BF16 rounds every element once, to nearest even, to bf16 when it is
+ * stored and halves the bytes the similarity search (Eq. 6) reads.  The paper runs in BF16
+ * and does not say how its cached queries are kept; the similarity of a later step is the
+ * dot product of that step's unrounded normalised query with the stored rounded entry.
+ * Only while the cache is empty (after create or reset), else EINVAL; allocates the bf16
+ * cache on first use (ENOMEM).  retopk_export_state / retopk_import_state keep their fp32
+ * layout in both formats (values are widened / rounded on the way).
+ */
+enum { RETOPK_QBAR_FP32 = 0, RETOPK_QBAR_BF16 = 1 };
+int retopk_set_qbar_format(retopk_ctx* ctx, int format);
+
+/*
  * Fusion level of the reuse path, for measuring what kernel fusion buys (the paper's kernel
  * efficiency analysis, Table 4, reports five cumulative stages for its own kernels; the cut
  * points here follow its description of them and are this library's own).  Results do not

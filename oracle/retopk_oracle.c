@@ -54,8 +54,9 @@
  * (sequence, head) pairs over threads.
  *
  * Parity unpinned by the paper (fixed only by this file's readings, which the hand trace and
- * the integer-tie tests pin): the tie-breaks of Top-r and Top-K, and whether the first decode
- * step has offset 0 or 1 for the refresh schedule.
+ * the integer-tie tests pin): the tie-breaks of Top-r and Top-K, whether the first decode
+ * step has offset 0 or 1 for the refresh schedule, the recent-recall rule, the supports of
+ * prompt tokens in prefill seeding, and the bf16 storage rule of cached queries.
  *
  * Pins (tests/test_oracle_pins.py): brute-force selection on small inputs, dense softmax
  * attention when K >= L, closed forms for K = 1 and K = 2, exact-path equality when

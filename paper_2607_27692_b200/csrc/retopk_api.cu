@@ -24,6 +24,8 @@ struct retopk_ctx {
     size_t smem_recall, smem_reuse, smem_exact, smem_finish;
     // device state
     float* qbar_cache;
+    uint16_t* qbar16;            // bf16 copy of the layout, allocated when that format is chosen
+    int qbar_bf16;
     int32_t* sup_cache;
     uint8_t* ws_path;
     float* ws_rho;
@@ -79,6 +81,7 @@ void free_all(retopk_ctx* c) {
     cudaFree(c->ws_ncand); cudaFree(c->ws_sel); cudaFree(c->ws_gflag); cudaFree(c->ws_scores); cudaFree(c->ws_tmax); cudaFree(c->counters);
     cudaFree(c->status); cudaFree(c->slow_select); cudaFree(c->scan_groups); cudaFree(c->scan_counter); cudaFree(c->stage_q); cudaFree(c->stage_out);
     cudaFree(c->stage_kv);
+    cudaFree(c->qbar16);
     for (int i = 0; i < 8; ++i) cudaFree(c->lw_persist[i]);
     if (c->pool) cudaMemPoolDestroy(c->pool);
 }
@@ -109,6 +112,7 @@ StepArgs make_args(const retopk_ctx* c, const void* q, const void* k, const void
     a.v = static_cast<const uint16_t*>(v);
     a.out = static_cast<uint16_t*>(out);
     a.qbar_cache = c->qbar_cache; a.sup_cache = c->sup_cache;
+    a.qbar16 = c->qbar_bf16 ? c->qbar16 : nullptr;
     a.ws_path = c->ws_path; a.ws_rho = c->ws_rho; a.ws_ncand = c->ws_ncand; a.ws_sel = c->ws_sel; a.ws_gflag = c->ws_gflag;
     a.ws_scores = c->ws_scores; a.ws_tmax = c->ws_tmax; a.tmax_stride = c->tmax_stride; a.counters = c->counters; a.status = c->status;
     a.slow_select = c->slow_select;
@@ -458,6 +462,18 @@ int retopk_set_recall_mode(retopk_ctx* c, int mode) {
     return RETOPK_OK;
 }
 
+int retopk_set_qbar_format(retopk_ctx* c, int format) {
+    if (!c || (format != RETOPK_QBAR_FP32 && format != RETOPK_QBAR_BF16) || c->n_ins != 0) return RETOPK_EINVAL;
+    DeviceGuard g(c->device);
+    if (format == RETOPK_QBAR_BF16 && !c->qbar16) {
+        const size_t n = (size_t)c->B * c->Hq * c->M * c->d;
+        if (cudaMalloc(reinterpret_cast<void**>(&c->qbar16), n * 2) != cudaSuccess) { cudaGetLastError(); c->qbar16 = nullptr; return RETOPK_ENOMEM; }
+        if (cudaMemset(c->qbar16, 0, n * 2) != cudaSuccess) return RETOPK_ECUDA;
+    }
+    c->qbar_bf16 = format == RETOPK_QBAR_BF16;
+    return RETOPK_OK;
+}
+
 int retopk_set_fusion_level(retopk_ctx* c, int level, int dependent_launches) {
     if (!c || level < 1 || level > 5 || (dependent_launches != 0 && dependent_launches != 1)) return RETOPK_EINVAL;
     if (dependent_launches && level != 5) return RETOPK_EINVAL;   // the unfused kernels are plain launches
@@ -506,7 +522,10 @@ int retopk_reset(retopk_ctx* c, void* stream) {
         (size_t)c->B * c->Hkv + 1, c->status, c->slow_select, c->scan_groups, c->scan_counter);
     c->n_ins = 0;
     c->t_dec = 0;
-    return cudaGetLastError() == cudaSuccess ? RETOPK_OK : RETOPK_ECUDA;
+    if (cudaGetLastError() != cudaSuccess) return RETOPK_ECUDA;
+    if (c->qbar16 && cudaMemsetAsync(c->qbar16, 0, nh * c->M * c->d * 2, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+        return RETOPK_ECUDA;
+    return RETOPK_OK;
 }
 
 int retopk_decode_step(retopk_ctx* c, const void* q, const void* k_cache, const void* v_cache,
@@ -667,7 +686,12 @@ int retopk_export_state(retopk_ctx* c, float* qbar, int32_t* supports, int64_t* 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const size_t nh = (size_t)c->B * c->Hq;
     bool ok = true;
-    if (qbar) ok = ok && cudaMemcpyAsync(qbar, c->qbar_cache, nh * c->M * c->d * 4, cudaMemcpyDeviceToDevice, s) == cudaSuccess;
+    if (qbar && c->qbar_bf16) {
+        widen_kernel<<<c->num_sms * 4, 256, 0, s>>>(c->qbar16, qbar, nh * c->M * c->d);
+        ok = ok && cudaGetLastError() == cudaSuccess;
+    } else if (qbar) {
+        ok = ok && cudaMemcpyAsync(qbar, c->qbar_cache, nh * c->M * c->d * 4, cudaMemcpyDeviceToDevice, s) == cudaSuccess;
+    }
     if (supports) ok = ok && cudaMemcpyAsync(supports, c->sup_cache, nh * c->M * c->K * 4, cudaMemcpyDeviceToDevice, s) == cudaSuccess;
     if (n_inserted) *n_inserted = c->n_ins;
     if (t_dec) *t_dec = c->t_dec;
@@ -679,7 +703,14 @@ int retopk_import_state(retopk_ctx* c, const float* qbar, const int32_t* support
     if (!c || !qbar || !supports || n_inserted < 0 || t_dec < 0) return RETOPK_EINVAL;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const size_t nh = (size_t)c->B * c->Hq;
-    bool ok = cudaMemcpyAsync(c->qbar_cache, qbar, nh * c->M * c->d * 4, cudaMemcpyDeviceToDevice, s) == cudaSuccess &&
+    bool ok;
+    if (c->qbar_bf16) {
+        narrow_kernel<<<c->num_sms * 4, 256, 0, s>>>(qbar, c->qbar16, nh * c->M * c->d);
+        ok = cudaGetLastError() == cudaSuccess;
+    } else {
+        ok = cudaMemcpyAsync(c->qbar_cache, qbar, nh * c->M * c->d * 4, cudaMemcpyDeviceToDevice, s) == cudaSuccess;
+    }
+    ok = ok &&
               cudaMemcpyAsync(c->sup_cache, supports, nh * c->M * c->K * 4, cudaMemcpyDeviceToDevice, s) == cudaSuccess;
     c->n_ins = n_inserted;
     c->t_dec = t_dec;

@@ -70,6 +70,7 @@ struct StepArgs {
     const uint16_t* v;
     uint16_t* out;
     float* qbar_cache;       // [B*Hq][M][d]
+    uint16_t* qbar16;        // same, kept as bf16 (storage variant); null: qbar_cache is in use
     int32_t* sup_cache;      // [B*Hq][M][K]
     uint8_t* ws_path;        // [B*Hq]
     float* ws_rho;           // [B*Hq]
@@ -166,6 +167,20 @@ __device__ __forceinline__ float dot8(const uint4& x, const float* qf) {
 __device__ __forceinline__ void unpack8(const uint4& x, float* f) {
     f[0] = bf16_lo(x.x); f[1] = bf16_hi(x.x); f[2] = bf16_lo(x.y); f[3] = bf16_hi(x.y);
     f[4] = bf16_lo(x.z); f[5] = bf16_hi(x.z); f[6] = bf16_lo(x.w); f[7] = bf16_hi(x.w);
+}
+
+// The cached normalised queries live in fp32 or, as a storage variant, in bf16 (rounded once,
+// to nearest even, when stored).  Four consecutive elements of a cache row / one element.
+__device__ __forceinline__ float4 load_qbar4(const StepArgs& a, size_t row_off, int lane) {
+    if (a.qbar16) {
+        const uint2 raw = reinterpret_cast<const uint2*>(a.qbar16 + row_off)[lane];
+        return make_float4(bf16_lo(raw.x), bf16_hi(raw.x), bf16_lo(raw.y), bf16_hi(raw.y));
+    }
+    return reinterpret_cast<const float4*>(a.qbar_cache + row_off)[lane];
+}
+__device__ __forceinline__ void store_qbar(const StepArgs& a, size_t off, float v) {
+    if (a.qbar16) a.qbar16[off] = __bfloat16_as_ushort(__float2bfloat16_rn(v));
+    else a.qbar_cache[off] = v;
 }
 
 // (sequence, KV head) index of query head bh: bh / G without a division when G is 2^k.
@@ -556,9 +571,8 @@ __device__ __forceinline__ void cache_similarities(const StepArgs& a, int bh, fl
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
             const int c = c0 + NW * u;
-            x[u] = (c < fill && lane < D / 4)
-                ? reinterpret_cast<const float4*>(a.qbar_cache + ((size_t)bh * M + c) * D)[lane]
-                : make_float4(0.f, 0.f, 0.f, 0.f);
+            x[u] = (c < fill && lane < D / 4) ? load_qbar4(a, ((size_t)bh * M + c) * D, lane)
+                                              : make_float4(0.f, 0.f, 0.f, 0.f);
         }
         if (c0 == warp) {
             // first trip: the query norm while the loads fly
@@ -685,7 +699,7 @@ __global__ void __launch_bounds__(RECALL_THREADS, 1) recall_kernel(const StepArg
     const int path = decide_path(a, rho_max);
 
     // insert the normalised query now: every similarity of this step has been taken
-    if (tid < D) a.qbar_cache[((size_t)bh * a.M + a.slot) * D + tid] = s_q[tid];
+    if (tid < D) store_qbar(a, ((size_t)bh * a.M + a.slot) * D + tid, s_q[tid]);
     record_decision(a, bh, bkv, s_sel, path, rho_max);
     RETOPK_PHASE(1, 2);
 }
@@ -1226,6 +1240,16 @@ __global__ void __launch_bounds__(FINISH_THREADS, 1) finish_kernel(const StepArg
     } else {
         exact_path<D, FINISH_THREADS>(a, smem_raw);
     }
+}
+
+// Conversions between the bf16 cache and the fp32 layout of export / import.
+__global__ void widen_kernel(const uint16_t* src, float* dst, size_t n) {
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
+        dst[i] = __uint_as_float((uint32_t)src[i] << 16);
+}
+__global__ void narrow_kernel(const float* src, uint16_t* dst, size_t n) {
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
+        dst[i] = __bfloat16_as_ushort(__float2bfloat16_rn(src[i]));
 }
 
 // Clear the caches (supports to -1, queries and counters to 0).

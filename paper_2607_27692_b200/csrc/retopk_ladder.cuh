@@ -209,7 +209,7 @@ __global__ void __launch_bounds__(LADDER_THREADS, 1) ladder_attend_kernel(const 
 __global__ void __launch_bounds__(LADDER_THREADS, 1) ladder_insert_kernel(const StepArgs a, int insert_q) {
     const int tid = threadIdx.x, bh = blockIdx.x;
     if (insert_q && tid < a.d)
-        a.qbar_cache[((size_t)bh * a.M + a.slot) * a.d + tid] = a.lw_qbar[(size_t)bh * a.d + tid];
+        store_qbar(a, ((size_t)bh * a.M + a.slot) * a.d + tid, a.lw_qbar[(size_t)bh * a.d + tid]);
     if (a.ws_path[bh] != PATH_REUSE) return;
     const int ns = a.lw_meta[bh * 4 + 0];
     int32_t* sup_out = a.sup_cache + ((size_t)bh * a.M + a.slot) * a.K;
@@ -236,7 +236,7 @@ __global__ void __launch_bounds__(LADDER_THREADS, 1) ladder_discover_kernel(cons
     __syncthreads();
     const float rho_max = recall_slots<NT>(a, s_rho, u.sel, s_misc);
     const int path = decide_path(a, rho_max);
-    if (tid < D) a.qbar_cache[((size_t)bh * a.M + a.slot) * D + tid] = s_q[tid];
+    if (tid < D) store_qbar(a, ((size_t)bh * a.M + a.slot) * D + tid, s_q[tid]);
     record_decision(a, bh, kv_group_of(bh, a), u.sel, path, rho_max);
     if (path == PATH_REUSE) union_to_global<NT>(a, bh, u);
 }

@@ -37,6 +37,7 @@ SIGNATURES = {
     "retopk_create": (_i32, [C.POINTER(_vp)] + [_i32] * 7 + [_f32, _i32]),
     "retopk_create_batched": (_i32, [C.POINTER(_vp)] + [_i32] * 8 + [_f32, _i32, _i64]),
     "retopk_set_recall_mode": (_i32, [_vp, _i32]),
+    "retopk_set_qbar_format": (_i32, [_vp, _i32]),
     "retopk_set_fusion_level": (_i32, [_vp, _i32, _i32]),
     "retopk_destroy": (_i32, [_vp]),
     "retopk_reset": (_i32, [_vp, _vp]),
@@ -147,6 +148,10 @@ class ReTopK:
     def set_recall_mode(self, mode: int):
         """0: recall the most similar entries (Eq. 7); 1: the most recent ones (Recent-R ablation row)."""
         _check(self.lib.retopk_set_recall_mode(self.h, mode), "retopk_set_recall_mode")
+
+    def set_qbar_format(self, fmt: int):
+        """0: cached queries in fp32 (default); 1: rounded to bf16 when stored (empty cache only)."""
+        _check(self.lib.retopk_set_qbar_format(self.h, fmt), "retopk_set_qbar_format")
 
     def set_fusion_level(self, level: int, dependent_launches: bool = False):
         """Fusion level 1..5 of the reuse path (Table 4's ladder); results do not depend on it."""

@@ -380,3 +380,49 @@ def test_last_recall_reports_the_most_similar_slots(rt, P, oracle_mod):
                         assert list(got) == list(last["sel"][b, h])
                         same_as_oracle += 1
     assert same_as_oracle > 0.3 * cfg.steps * cfg.B * cfg.H_q
+
+
+@pytest.mark.parametrize("d", [64, 128])
+def test_bf16_query_cache_teacher_forced(rt, P, oracle_mod, d):
+    """The bf16 storage variant of the cached queries on both sides."""
+    cfg = wl.CONFIGS["tiny"].replace(context=1200, steps=36, B=2, H_q=4, H_kv=2, d=d, M=8, r=3)
+    st, o, g, k, v = stream_case(rt, P, oracle_mod, cfg, cfg.steps)
+    o.set_qbar_format(1)
+    g.set_qbar_format(1)
+    P.teacher_forced_run(cfg, st, cfg.steps, o, g, k, v)
+    so, sg = o.stats(), g.stats()
+    assert so["reuse"] > 0 and so["fallback"] > 0
+    for key in ("steps", "reuse", "fallback", "refresh", "cand_sum"):
+        assert sg[key] == so[key], key
+    # the entry the last step stored: the same bf16 value on both sides, but for elements whose
+    # fp32 quotient lands on the other side of a rounding boundary (one bf16 step at most)
+    slot = (cfg.steps - 1) % cfg.M
+    mine = g.export_state()[0][:, :, slot].cpu().numpy().astype(np.float64)
+    ref = o.export_state()[0][:, :, slot]
+    assert np.array_equal(wl.bf16_bits_to_f64(wl.f32_to_bf16_bits(mine.astype(np.float32))), mine)
+    step = 2.0 ** (np.floor(np.log2(np.maximum(np.abs(ref), 1e-30))) - 7)
+    assert (np.abs(mine - ref) <= step * 1.0001).all()
+    assert (mine == ref).mean() > 0.99
+
+
+def test_bf16_query_cache_free_running_and_argument_checks(rt, P, oracle_mod):
+    cfg = wl.CONFIGS["tiny"].replace(context=800, steps=40, B=2, H_q=4, H_kv=2)
+    st, o, g, k, v = stream_case(rt, P, oracle_mod, cfg, cfg.steps)
+    o.set_qbar_format(1)
+    g.set_qbar_format(1)
+    g.set_qbar_format(0)
+    g.set_qbar_format(1)
+    cos = []
+    for t in range(cfg.steps):
+        out_g = g.decode_step(P.to_dev(st.q[t]), k, v, st.seq_len(t)).float().cpu().numpy().astype(np.float64)
+        out_o = o.decode_step(st.q[t], st.k, st.v, st.seq_len(t))
+        cos.append((out_g * out_o).sum(-1) / (np.linalg.norm(out_g, axis=-1) * np.linalg.norm(out_o, axis=-1)))
+    assert np.median(np.array(cos)) > 0.999
+    so, sg = o.stats(), g.stats()
+    assert sg["steps"] == so["steps"] and abs(sg["reuse"] - so["reuse"]) <= 0.05 * so["steps"]
+    lib = rt.load()
+    assert lib.retopk_set_qbar_format(g.h, 0) == -1          # the cache is not empty any more
+    assert lib.retopk_set_qbar_format(None, 1) == -1
+    g.reset()
+    assert lib.retopk_set_qbar_format(g.h, 2) == -1
+    assert lib.retopk_set_qbar_format(g.h, 0) == 0
