@@ -116,6 +116,18 @@ enum { RETOPK_QBAR_FP32 = 0, RETOPK_QBAR_BF16 = 1 };
 int retopk_set_qbar_format(retopk_ctx* ctx, int format);
 
 /*
+ * CTAs per (sequence, query head) in the finish kernel: 1, 2, 4 or 8.  With more than one, the
+ * CTAs of a head form a thread-block cluster on as many SMs: each scores a share of the
+ * candidate rows (Eq. 10) and fetches a share of the selected value rows (Eq. 12); keys and
+ * partial sums cross through distributed shared memory.  The paper has no counterpart; it is
+ * how a small batch uses the SMs that one CTA per head would leave idle.  retopk_create*
+ * picks the largest size with B*H_q*size <= the SM count (1 from B*H_q = 75 up on B200).
+ * Supports and decisions do not depend on the size; outputs differ in the last bits of the
+ * fp32 sum order.  EINVAL for any other size.
+ */
+int retopk_set_cluster_size(retopk_ctx* ctx, int ctas_per_head);
+
+/*
  * Fusion level of the reuse path, for measuring what kernel fusion buys (the paper's kernel
  * efficiency analysis, Table 4, reports five cumulative stages for its own kernels; the cut
  * points here follow its description of them and are this library's own).  Results do not

@@ -50,6 +50,7 @@ struct retopk_ctx {
     int last_launches;
     // fusion ladder (measurement): level 1..5, dependent launches on or off, and the buffers
     // the unfused levels hand their intermediates through
+    int cluster;                 // CTAs per head in finish_kernel (1, 2, 4 or 8)
     int fusion_level, dependent_launches;
     cudaMemPool_t pool;          // levels 1-3 draw the buffers from here in every step
     void* lw_persist[8];         // level 4 keeps them
@@ -119,25 +120,41 @@ StepArgs make_args(const retopk_ctx* c, const void* q, const void* k, const void
     a.scan_groups = c->scan_groups;
     a.scan_counter = c->scan_counter;
     a.idx_out = nullptr;
+    a.cl_shift = __builtin_ctz((unsigned)(c->cluster > 0 ? c->cluster : 1));
     return a;
+}
+
+// CTAs per head in finish_kernel: with few heads, as many (a power of two up to 8, one SM each)
+// as still fit one wave.
+int auto_cluster(long long heads, int num_sms) {
+    int cl = 1;
+    while (cl < 8 && heads * cl * 2 <= num_sms) cl *= 2;
+    return cl;
 }
 
 // Launch with programmatic stream serialisation: the kernel may be set up while its
 // predecessor in the stream still runs; it waits (pdl_wait) before reading its inputs.
 template <class Kernel>
 int launch_dependent(Kernel kernel, unsigned grid, unsigned block, size_t smem, cudaStream_t s,
-                     const StepArgs& a, int allowed = 1) {
+                     const StepArgs& a, int allowed = 1, int cluster = 1) {
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof cfg);
     cfg.gridDim = dim3(grid);
     cfg.blockDim = dim3(block);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = s;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = allowed;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
+    if (cluster > 1) {
+        attr[1].id = cudaLaunchAttributeClusterDimension;
+        attr[1].val.clusterDim.x = (unsigned)cluster;
+        attr[1].val.clusterDim.y = 1;
+        attr[1].val.clusterDim.z = 1;
+        cfg.numAttrs = 2;
+    }
     return cudaLaunchKernelEx(&cfg, kernel, a) == cudaSuccess ? RETOPK_OK : RETOPK_ECUDA;
 }
 
@@ -164,10 +181,10 @@ int launch_scan(const retopk_ctx* c, const StepArgs& a, cudaStream_t s) {
 }
 
 int launch_finish(const retopk_ctx* c, const StepArgs& a, cudaStream_t s) {
-    const unsigned grid = (unsigned)(c->B * c->Hq);
+    const unsigned grid = (unsigned)(c->B * c->Hq * c->cluster);      // one cluster of CTAs per head
     const size_t smem = a.mode == MODE_EXACT ? c->smem_exact : c->smem_finish;
-    if (c->d == 128) return launch_dependent(finish_kernel<128>, grid, FINISH_THREADS, smem, s, a, c->dependent_launches);
-    return launch_dependent(finish_kernel<64>, grid, FINISH_THREADS, smem, s, a, c->dependent_launches);
+    if (c->d == 128) return launch_dependent(finish_kernel<128>, grid, FINISH_THREADS, smem, s, a, c->dependent_launches, c->cluster);
+    return launch_dependent(finish_kernel<64>, grid, FINISH_THREADS, smem, s, a, c->dependent_launches, c->cluster);
 }
 
 // Measurement hook: event number `which` (0..3) of the current call, if recording.
@@ -433,6 +450,8 @@ int retopk_create_batched(retopk_ctx** out, int B, int H_q, int H_kv, int d, int
     }
     if (e1 != cudaSuccess || e2 != cudaSuccess) { cudaGetLastError(); delete c; return RETOPK_ECUDA; }
     c->scan_grid = c->num_sms * (occ > 0 ? occ : 2);
+    // finish_kernel: with few heads, a cluster of CTAs (one SM each) per head, as many as fit one wave
+    c->cluster = auto_cluster((long long)B * H_q, c->num_sms);
 
 
     const size_t nh = (size_t)B * H_q;
@@ -471,6 +490,12 @@ int retopk_set_qbar_format(retopk_ctx* c, int format) {
         if (cudaMemset(c->qbar16, 0, n * 2) != cudaSuccess) return RETOPK_ECUDA;
     }
     c->qbar_bf16 = format == RETOPK_QBAR_BF16;
+    return RETOPK_OK;
+}
+
+int retopk_set_cluster_size(retopk_ctx* c, int ctas_per_head) {
+    if (!c || (ctas_per_head != 1 && ctas_per_head != 2 && ctas_per_head != 4 && ctas_per_head != 8)) return RETOPK_EINVAL;
+    c->cluster = ctas_per_head;
     return RETOPK_OK;
 }
 
@@ -873,9 +898,10 @@ int exact_topk_decode_static(int B, int H_q, int H_kv, int d, int K, int64_t max
     else if (ntile == 1) scan_kernel<64, 1><<<grid, SCAN_THREADS, 0, s>>>(a);
     else scan_kernel<64, 2><<<grid, SCAN_THREADS, 0, s>>>(a);
     if (cudaGetLastError() != cudaSuccess) return RETOPK_ECUDA;
-    if (d == 128) finish_kernel<128><<<(unsigned)nh, FINISH_THREADS, smem, s>>>(a);
-    else finish_kernel<64><<<(unsigned)nh, FINISH_THREADS, smem, s>>>(a);
-    return cudaGetLastError() == cudaSuccess ? RETOPK_OK : RETOPK_ECUDA;
+    const int cluster = auto_cluster(nh, st->num_sms);
+    a.cl_shift = __builtin_ctz((unsigned)cluster);
+    if (d == 128) return launch_dependent(finish_kernel<128>, (unsigned)(nh * cluster), FINISH_THREADS, smem, s, a, 0, cluster);
+    return launch_dependent(finish_kernel<64>, (unsigned)(nh * cluster), FINISH_THREADS, smem, s, a, 0, cluster);
 }
 
 #ifdef RETOPK_PHASE_CLOCKS

@@ -17,6 +17,7 @@
 //                  Both: softmax.V (Eq. 12) and the support insert.
 //                  Exact Top-K attention is scan + finish with every head on the exact path.
 #pragma once
+#include <cooperative_groups.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <math_constants.h>
@@ -86,6 +87,7 @@ struct StepArgs {
     unsigned long long* scan_groups;
     unsigned int* scan_counter;  // pool cursor of scan_kernel; finish_kernel resets it
     int32_t* idx_out;        // MODE_EXACT only, may be null
+    int cl_shift;            // finish_kernel runs 2^cl_shift CTAs (one thread-block cluster) per head
     // Fusion-ladder levels below the production one (see retopk_ladder.cuh): the reuse path runs
     // as separate kernels that hand their intermediates on through these global buffers, and
     // finish_kernel then leaves heads on the reuse path alone.
@@ -182,6 +184,10 @@ __device__ __forceinline__ void store_qbar(const StepArgs& a, size_t off, float 
     if (a.qbar16) a.qbar16[off] = __bfloat16_as_ushort(__float2bfloat16_rn(v));
     else a.qbar_cache[off] = v;
 }
+
+// finish_kernel may give a head a whole thread-block cluster: head and rank of this CTA.
+__device__ __forceinline__ int finish_head(const StepArgs& a) { return (int)(blockIdx.x >> a.cl_shift); }
+__device__ __forceinline__ int finish_rank(const StepArgs& a) { return (int)(blockIdx.x & ((1u << a.cl_shift) - 1u)); }
 
 // (sequence, KV head) index of query head bh: bh / G without a division when G is 2^k.
 __device__ __forceinline__ int kv_group_of(int bh, const StepArgs& a) {
@@ -453,11 +459,14 @@ __device__ __forceinline__ float reduce8_across(const float* a, int sub, int& ro
 // zone (depth rows per row slot in flight at once); the softmax weights are computed while
 // the first wave is in the air.  s_w: ns floats; s_red: (NT/32) * D + NT floats; s_ws: 32
 // words; s_stage: depth * NT uint4.
+// With a cluster of cl_size CTAs per head (every CTA holding the same support), CTA cl_rank
+// fetches and weighs its contiguous share of the rows; the partial sums meet in rank 0
+// through distributed shared memory and are added there in rank order.
 // ------------------------------------------------------------------------------------
 template <int D, int NT>
 __device__ void attend(const uint16_t* vbase, int ns, const int32_t* s_sup_idx, const uint32_t* s_sup_key,
                        float* s_w, float* s_red, int* s_ws, uint4* s_stage, int depth, uint32_t kmax,
-                       bool kmax_known, uint16_t* out_row) {
+                       bool kmax_known, uint16_t* out_row, int cl_rank = 0, int cl_size = 1) {
     constexpr int LPR = D / 8;                  // lanes per bf16 row (16 bytes each)
     constexpr int RPW = 32 / LPR;               // rows per warp load
     constexpr int SLOTS = (NT / 32) * RPW;      // row slots per block
@@ -467,15 +476,18 @@ __device__ void attend(const uint16_t* vbase, int ns, const int32_t* s_sup_idx, 
     const int sub = lane % LPR, myslot = warp * RPW + lane / LPR;
     const char* vsrc = reinterpret_cast<const char*>(vbase) + sub * 16;
     uint4* my_stage = s_stage + tid;
+    // this CTA's share of the support: [i_lo, i_hi)
+    const int share = (ns + cl_size - 1) / cl_size;
+    const int i_lo = min(ns, cl_rank * share), i_hi = min(ns, i_lo + share);
 
     auto issue = [&](int base) {
         for (int u = 0; u < depth; ++u) {
             const int i = base + u * SLOTS + myslot;
-            if (i < ns) cp_async16(my_stage + u * NT, vsrc + (size_t)s_sup_idx[i] * (D * 2));
+            if (i < i_hi) cp_async16(my_stage + u * NT, vsrc + (size_t)s_sup_idx[i] * (D * 2));
         }
         cp_async_commit();
     };
-    issue(0);
+    issue(i_lo);
 
     if (!kmax_known) {
         kmax = 0;
@@ -504,11 +516,11 @@ __device__ void attend(const uint16_t* vbase, int ns, const int32_t* s_sup_idx, 
     float acc[8];
 #pragma unroll
     for (int e = 0; e < 8; ++e) acc[e] = 0.f;
-    for (int base = 0;;) {
+    for (int base = i_lo;;) {
         cp_async_wait_all();
         for (int u = 0; u < depth; ++u) {
             const int i = base + u * SLOTS + myslot;
-            if (i < ns) {
+            if (i < i_hi) {
                 const float w = s_w[i];
                 float f[8];
                 unpack8(my_stage[u * NT], f);
@@ -517,7 +529,7 @@ __device__ void attend(const uint16_t* vbase, int ns, const int32_t* s_sup_idx, 
             }
         }
         base += SLOTS * depth;
-        if (base >= ns) break;
+        if (base >= i_hi) break;
         issue(base);
     }
     // fixed-order reduction: row slots of a warp, then warps in groups, then groups
@@ -539,10 +551,25 @@ __device__ void attend(const uint16_t* vbase, int ns, const int32_t* s_sup_idx, 
         s_red[NW * D + part * D + j] = sum;
     }
     __syncthreads();
+    float sum = 0.f;
     if (tid < D) {
-        float sum = 0.f;
 #pragma unroll
         for (int p = 0; p < PARTS; ++p) sum += s_red[NW * D + p * D + tid];
+    }
+    if (cl_size > 1) {
+        // s_red[0..D) is free again (its readers passed the barrier above)
+        namespace cg = cooperative_groups;
+        cg::cluster_group cluster = cg::this_cluster();
+        if (tid < D) s_red[tid] = sum;
+        cluster.sync();
+        if (cl_rank == 0 && tid < D) {
+            sum = 0.f;
+            for (int r = 0; r < cl_size; ++r) sum += *cluster.map_shared_rank(s_red + tid, r);
+        }
+        cluster.sync();           // nobody leaves while its shared memory may still be read
+        if (cl_rank != 0) return;
+    }
+    if (tid < D) {
         const float o = ns > 0 ? sum / denom : 0.f;
         out_row[tid] = __bfloat16_as_ushort(__float2bfloat16_rn(o));
     }
@@ -832,11 +859,14 @@ __device__ void reuse_path(const StepArgs& a, unsigned char* smem_raw) {
     uint4* s_stage = reinterpret_cast<uint4*>(s_bm + ((((int)a.max_seq_len + 31) / 32 + 3) & ~3));
 
     const int tid = threadIdx.x;
-    const int bh = blockIdx.x;
+    const int bh = finish_head(a);
+    const int cl_rank = finish_rank(a), cl_size = 1 << a.cl_shift;
     const int bkv = kv_group_of(bh, a);
     const int M = a.M, fill = a.fill, L = a.L, K = a.K;
     const int n_sel = a.r < fill ? a.r : fill;
     RETOPK_PHASE(0, 0);
+    // peers write into this CTA's shared memory later on: all of them must be running by then
+    if (cl_size > 1) cooperative_groups::this_cluster().sync();
 
     // recalled slots and the raw query from global memory; clear the bitmap meanwhile
     if (tid < a.r) s_sel[tid] = a.ws_sel[(size_t)bh * a.r + tid];
@@ -858,10 +888,26 @@ __device__ void reuse_path(const StepArgs& a, unsigned char* smem_raw) {
     __syncthreads();
     RETOPK_PHASE(0, 5);
 
-    // Eq. 10
-    score_candidates<D, NT, true>(a.k + (size_t)bkv * a.max_seq_len * D, s_idx, n, s_qraw, s_stage, a.stage_depth,
-                                  a.scale, s_key);
-    __syncthreads();
+    // Eq. 10.  In a cluster every CTA built the same list; each scores a contiguous share of
+    // it and hands the keys to the others through distributed shared memory.
+    if (cl_size == 1) {
+        score_candidates<D, NT, true>(a.k + (size_t)bkv * a.max_seq_len * D, s_idx, n, s_qraw, s_stage,
+                                      a.stage_depth, a.scale, s_key);
+        __syncthreads();
+    } else {
+        namespace cg = cooperative_groups;
+        cg::cluster_group cluster = cg::this_cluster();
+        const int share = (n + cl_size - 1) / cl_size;
+        const int lo = min(n, cl_rank * share), hi = min(n, lo + share);
+        score_candidates<D, NT, true>(a.k + (size_t)bkv * a.max_seq_len * D, s_idx + lo, hi - lo, s_qraw, s_stage,
+                                      a.stage_depth, a.scale, s_key + lo);
+        __syncthreads();
+        for (int r = 1; r < cl_size; ++r) {
+            uint32_t* peer = cluster.map_shared_rank(s_key, (cl_rank + r) & (cl_size - 1));
+            for (int i = lo + tid; i < hi; i += NT) peer[i] = s_key[i];
+        }
+        cluster.sync();
+    }
     RETOPK_PHASE(0, 6);
 
     // Eq. 11: Top-K of the candidates; insert the support
@@ -869,13 +915,15 @@ __device__ void reuse_path(const StepArgs& a, unsigned char* smem_raw) {
     bool kmax_known;
     const int ns = select_listed<NT>(s_key, s_idx, n, K, s_sup_idx, s_sup_key, s_hist, s_ws, kmax, kmax_known);
     RETOPK_PHASE(0, 7);
-    int32_t* sup_out = a.sup_cache + ((size_t)bh * M + a.slot) * K;
-    for (int i = tid; i < K; i += NT) sup_out[i] = i < ns ? s_sup_idx[i] : -1;
+    if (cl_rank == 0) {
+        int32_t* sup_out = a.sup_cache + ((size_t)bh * M + a.slot) * K;
+        for (int i = tid; i < K; i += NT) sup_out[i] = i < ns ? s_sup_idx[i] : -1;
+    }
 
     // Eq. 12 (s_red aliases the candidate lists, which are dead now)
     attend<D, NT>(a.v + (size_t)bkv * a.max_seq_len * D, ns, s_sup_idx, s_sup_key, s_w, s_red, s_ws, s_stage,
-                  a.stage_depth, kmax, kmax_known, a.out + (size_t)bh * D);
-    if (tid == 0) {      // the step record is written last: nothing in this kernel waits for it
+                  a.stage_depth, kmax, kmax_known, a.out + (size_t)bh * D, cl_rank, cl_size);
+    if (tid == 0 && cl_rank == 0) {      // the step record is written last: nothing in this kernel waits for it
         a.ws_ncand[bh] = n;
         atomicAdd(a.counters + (size_t)bh * 4 + PATH_REUSE, 1ull);
         atomicAdd(a.counters + (size_t)bh * 4 + 3, (unsigned long long)n);
@@ -1060,7 +1108,10 @@ __global__ void __launch_bounds__(SCAN_THREADS) scan_kernel(const StepArgs a) {
 // ------------------------------------------------------------------------------------
 template <int D, int NT>
 __device__ void exact_path(const StepArgs& a, unsigned char* smem_raw) {
-    const int bh = blockIdx.x;
+    // In a cluster every CTA of a head selects the same support on its own (the lists are short
+    // and come from L2); only the value rows are shared out, and rank 0 writes the results.
+    const int bh = finish_head(a);
+    const int cl_rank = finish_rank(a), cl_size = 1 << a.cl_shift;
     // layout (words): key[NS] idx[NS] (aliased later by red[NW*D+NT]) tile[tile_cap]
     //                 sup_idx[K] sup_key[K] w[K] cnt[SCRATCH_WORDS] ws[32] misc[8] stage[depth*NT*4]
     uint32_t* s_key = reinterpret_cast<uint32_t*>(smem_raw);
@@ -1205,7 +1256,7 @@ __device__ void exact_path(const StepArgs& a, unsigned char* smem_raw) {
         radix_select<NT>(src, L, K, s_hist, s_misc, vstar, need_eq);
         ordered_emit<NT>(src, L, vstar, need_eq, s_sup_idx, s_sup_key, s_ws);
         ns = K;
-        if (tid == 0) atomicAdd(a.slow_select, 1ull);
+        if (tid == 0 && cl_rank == 0) atomicAdd(a.slow_select, 1ull);
         __syncthreads();
     }
     uint32_t kmax = 0;
@@ -1217,11 +1268,11 @@ __device__ void exact_path(const StepArgs& a, unsigned char* smem_raw) {
     int32_t* sup_out = nullptr;
     if (a.mode == MODE_RETOPK) sup_out = a.sup_cache + ((size_t)bh * a.M + a.slot) * K;
     else if (a.idx_out) sup_out = a.idx_out + (size_t)bh * K;
-    if (sup_out)
+    if (sup_out && cl_rank == 0)
         for (int i = tid; i < K; i += NT) sup_out[i] = i < ns ? s_sup_idx[i] : -1;
 
     attend<D, NT>(a.v + (size_t)bkv * a.max_seq_len * D, ns, s_sup_idx, s_sup_key, s_w, s_red, s_ws, s_stage,
-                  a.exact_stage_depth, kmax, kmax_known, a.out + (size_t)bh * D);
+                  a.exact_stage_depth, kmax, kmax_known, a.out + (size_t)bh * D, cl_rank, cl_size);
     RETOPK_PHASE(2, 5);
 }
 
@@ -1235,7 +1286,7 @@ __global__ void __launch_bounds__(FINISH_THREADS, 1) finish_kernel(const StepArg
     extern __shared__ __align__(16) unsigned char smem_raw[];
     pdl_wait();        // scores and tile maxima come from the scan, recalled slots and paths from recall_kernel
     if (blockIdx.x == 0 && threadIdx.x == 0) *a.scan_counter = 0u;      // the scan before this kernel is complete
-    if (a.mode == MODE_RETOPK && a.ws_path[blockIdx.x] == PATH_REUSE) {
+    if (a.mode == MODE_RETOPK && a.ws_path[finish_head(a)] == PATH_REUSE) {
         if (!a.skip_reuse) reuse_path<D, FINISH_THREADS>(a, smem_raw);
     } else {
         exact_path<D, FINISH_THREADS>(a, smem_raw);

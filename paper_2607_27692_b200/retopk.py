@@ -38,6 +38,7 @@ SIGNATURES = {
     "retopk_create_batched": (_i32, [C.POINTER(_vp)] + [_i32] * 8 + [_f32, _i32, _i64]),
     "retopk_set_recall_mode": (_i32, [_vp, _i32]),
     "retopk_set_qbar_format": (_i32, [_vp, _i32]),
+    "retopk_set_cluster_size": (_i32, [_vp, _i32]),
     "retopk_set_fusion_level": (_i32, [_vp, _i32, _i32]),
     "retopk_destroy": (_i32, [_vp]),
     "retopk_reset": (_i32, [_vp, _vp]),
@@ -152,6 +153,10 @@ class ReTopK:
     def set_qbar_format(self, fmt: int):
         """0: cached queries in fp32 (default); 1: rounded to bf16 when stored (empty cache only)."""
         _check(self.lib.retopk_set_qbar_format(self.h, fmt), "retopk_set_qbar_format")
+
+    def set_cluster_size(self, ctas_per_head: int):
+        """CTAs (one SM each) per head in the finish kernel: 1, 2, 4 or 8."""
+        _check(self.lib.retopk_set_cluster_size(self.h, ctas_per_head), "retopk_set_cluster_size")
 
     def set_fusion_level(self, level: int, dependent_launches: bool = False):
         """Fusion level 1..5 of the reuse path (Table 4's ladder); results do not depend on it."""
