@@ -481,6 +481,7 @@ __device__ void attend(const uint16_t* vbase, int ns, const int32_t* s_sup_idx, 
     const int i_lo = min(ns, cl_rank * share), i_hi = min(ns, i_lo + share);
 
     auto issue = [&](int base) {
+#pragma unroll 4
         for (int u = 0; u < depth; ++u) {
             const int i = base + u * SLOTS + myslot;
             if (i < i_hi) cp_async16(my_stage + u * NT, vsrc + (size_t)s_sup_idx[i] * (D * 2));
@@ -510,8 +511,9 @@ __device__ void attend(const uint16_t* vbase, int ns, const int32_t* s_sup_idx, 
     float* s_wsf = reinterpret_cast<float*>(s_ws);
     if (lane == 0) s_wsf[warp] = wsum;
     __syncthreads();
-    float denom = 0.f;
-    for (int w = 0; w < NW; ++w) denom += s_wsf[w];      // fixed order
+    float denom = lane < NW ? s_wsf[lane] : 0.f;         // fixed tree: the same sum on every lane and run
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) denom += __shfl_xor_sync(0xffffffffu, denom, o);
 
     float acc[8];
 #pragma unroll
@@ -808,6 +810,7 @@ __device__ __forceinline__ void score_candidates(const uint16_t* kbase, const in
     // half run while the second half is still arriving
     const int half = (depth + 1) / 2;
     for (int base = 0; base < n; base += SLOTS * depth) {
+#pragma unroll 4
         for (int u = 0; u < depth; ++u) {
             const int i = base + u * SLOTS + myslot;
             if (i < n) cp_async16(my_stage + u * NT, ksrc + (size_t)(INDEXED ? row_of[i] : i) * (D * 2));
