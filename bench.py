@@ -439,7 +439,9 @@ def run_gpu(args):
                    "parallelism": "replicas only" if world > 1 else "single GPU"},
         "clocks": sampler.summary(),
         "e2e": {"value": round(replicas.job_cost_per_step(e2e["us_per_step"], world), 3), "unit": UNIT,
-                "h2d_bytes_per_step": qbytes + kvbytes, "d2h_bytes_per_step": qbytes},
+                "h2d_bytes_per_step": qbytes + kvbytes, "d2h_bytes_per_step": qbytes,
+                "transport": "pinned host buffers read and written by the step's kernels over the host link; "
+                             "stream synchronised every step"},
         "gpu_launches": head["launches"],
         "path_mix": path_mix(head["stats"]),
         "exact_topk": {"us_per_step": round(exact["us_per_step"], 2), "GBps": round(exact_gbs, 1),

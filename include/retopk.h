@@ -182,8 +182,11 @@ int retopk_prefill(retopk_ctx* ctx, const void* q_tail, const void* k_cache, con
  * The same step for a caller whose per-token tensors live in HOST memory: copies q_host
  * [B,H_q,d] to the device, appends k_new_host / v_new_host [B,H_kv,d] at position
  * seq_len - 1 of the device-resident k_cache / v_cache, runs the step, copies the result
- * to out_host [B,H_q,d] and synchronises `stream`.  Pinned host buffers keep the copies
- * asynchronous; pageable ones work but serialise.
+ * to out_host [B,H_q,d] and synchronises `stream`.  When all four host buffers are pinned
+ * and mapped (cudaHostAlloc / cudaHostRegister memory, 16-byte aligned) no copy is enqueued:
+ * one small kernel reads q and the new rows straight from host memory and the last kernel
+ * stores the output rows to out_host.  Otherwise the tensors go through staged copies
+ * (pageable buffers work but serialise).
  */
 int retopk_decode_step_host(retopk_ctx* ctx, const void* q_host, const void* k_new_host,
                             const void* v_new_host, void* k_cache, void* v_cache,

@@ -624,6 +624,14 @@ int exact_topk_decode(retopk_ctx* c, const void* q, const void* k_cache, const v
     return RETOPK_OK;
 }
 
+// Device-side alias of a host pointer the GPU can address directly (pinned and mapped), or null.
+static void* device_alias(const void* host) {
+    cudaPointerAttributes at;
+    if (cudaPointerGetAttributes(&at, host) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+    if (at.type != cudaMemoryTypeHost) return nullptr;
+    return at.devicePointer;
+}
+
 int retopk_decode_step_host(retopk_ctx* c, const void* q_host, const void* k_new_host,
                             const void* v_new_host, void* k_cache, void* v_cache, int64_t seq_len,
                             void* out_host, void* stream) {
@@ -633,6 +641,28 @@ int retopk_decode_step_host(retopk_ctx* c, const void* q_host, const void* k_new
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const size_t row = (size_t)c->d * 2;
     const size_t nq = (size_t)c->B * c->Hq * row, nkv = (size_t)c->B * c->Hkv;
+    // Pinned, mapped host buffers are read and written by the kernels themselves: one small
+    // launch brings q and the new rows across, finish_kernel stores the output rows to the
+    // host.  Anything else goes through staged copies.
+    void* q_dev = device_alias(q_host);
+    void* k_dev = device_alias(k_new_host);
+    void* v_dev = device_alias(v_new_host);
+    void* out_dev = device_alias(out_host);
+    const bool direct = q_dev && k_dev && v_dev && out_dev && aligned16(q_dev) && aligned16(k_dev) &&
+                        aligned16(v_dev) && aligned16(k_cache) && aligned16(v_cache);
+    if (direct) {
+        const int q_vecs = (int)(nq / 16), row_vecs = (int)(nkv * row / 16);
+        const int total = q_vecs + 2 * row_vecs;
+        ingest_kernel<<<(total + 255) / 256, 256, 0, s>>>(
+            static_cast<const uint4*>(q_dev), reinterpret_cast<uint4*>(c->stage_q), q_vecs,
+            static_cast<const uint4*>(k_dev), static_cast<const uint4*>(v_dev), static_cast<uint16_t*>(k_cache),
+            static_cast<uint16_t*>(v_cache), (int)nkv, c->d, c->max_seq_len, seq_len - 1);
+        if (cudaGetLastError() != cudaSuccess) return RETOPK_ECUDA;
+        int rc = retopk_decode_step(c, c->stage_q, k_cache, v_cache, seq_len, out_dev, stream);
+        if (rc != RETOPK_OK) return rc;
+        c->last_launches += 1;
+        return cudaStreamSynchronize(s) == cudaSuccess ? RETOPK_OK : RETOPK_ECUDA;
+    }
     if (cudaMemcpyAsync(c->stage_q, q_host, nq, cudaMemcpyHostToDevice, s) != cudaSuccess)
         return RETOPK_ECUDA;
     // append the current token's key / value row of every (sequence, KV head)

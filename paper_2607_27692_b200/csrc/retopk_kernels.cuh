@@ -1296,6 +1296,29 @@ __global__ void __launch_bounds__(FINISH_THREADS, 1) finish_kernel(const StepArg
     }
 }
 
+// Host-buffer entry point, when the caller's buffers are pinned and mapped: one launch reads
+// the step's query block and the new key / value row of every (sequence, KV head) straight
+// from host memory, 16 bytes per thread, into the staging copy of q and into row `pos` of the
+// caches.  q_vecs = B*H_q*d/8; rows: [B*H_kv][d] each.
+__global__ void ingest_kernel(const uint4* q_src, uint4* q_dst, int q_vecs, const uint4* k_src, const uint4* v_src,
+                              uint16_t* k_cache, uint16_t* v_cache, int groups, int d, long long max_seq_len,
+                              long long pos) {
+    const int lpr = d / 8;                              // 16-byte pieces per row
+    const int row_vecs = groups * lpr;
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < q_vecs) {
+        q_dst[i] = q_src[i];
+    } else if (i < q_vecs + 2 * row_vecs) {
+        const int j = i - q_vecs;
+        const bool is_v = j >= row_vecs;
+        const int jj = is_v ? j - row_vecs : j;
+        const int g = jj / lpr, sub = jj - g * lpr;
+        uint16_t* cache = is_v ? v_cache : k_cache;
+        uint4* dst = reinterpret_cast<uint4*>(cache + ((size_t)g * max_seq_len + pos) * d) + sub;
+        *dst = (is_v ? v_src : k_src)[jj];
+    }
+}
+
 // Conversions between the bf16 cache and the fp32 layout of export / import.
 __global__ void widen_kernel(const uint16_t* src, float* dst, size_t n) {
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)

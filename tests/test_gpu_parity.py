@@ -232,7 +232,9 @@ def test_steps_are_deterministic(rt, P):
     assert runs[0][2] == runs[1][2]
 
 
-def test_host_entry_point_matches_device_entry_point(rt, P):
+@pytest.mark.parametrize("pinned", [True, False])
+def test_host_entry_point_matches_device_entry_point(rt, P, pinned):
+    """Pinned buffers are read and written by the kernels directly, pageable ones are staged."""
     cfg = wl.CONFIGS["tiny"].replace(context=1500, steps=10, B=2, H_q=8, H_kv=2, d=128)
     st = wl.make_stream(cfg, steps=10)
     g_dev, g_host = rt.ReTopK.from_config(cfg), rt.ReTopK.from_config(cfg)
@@ -241,15 +243,18 @@ def test_host_entry_point_matches_device_entry_point(rt, P):
     k2, v2 = k.clone(), v.clone()
     k2[:, :, cfg.context:] = 0
     v2[:, :, cfg.context:] = 0
-    out_host = torch.empty(g_host.q_shape, dtype=torch.bfloat16).pin_memory()
+    out_host = torch.empty(g_host.q_shape, dtype=torch.bfloat16)
+    if pinned:
+        out_host = out_host.pin_memory()
     for t in range(10):
         L = st.seq_len(t)
         a = g_dev.decode_step(P.to_dev(st.q[t]), k, v, L)
-        qh = rt.bf16_tensor_from_bits(st.q[t], pin=True)
-        kn = rt.bf16_tensor_from_bits(st.k[:, :, L - 1], pin=True)
-        vn = rt.bf16_tensor_from_bits(st.v[:, :, L - 1], pin=True)
+        qh = rt.bf16_tensor_from_bits(st.q[t], pin=pinned)
+        kn = rt.bf16_tensor_from_bits(st.k[:, :, L - 1], pin=pinned)
+        vn = rt.bf16_tensor_from_bits(st.v[:, :, L - 1], pin=pinned)
         g_host.decode_step_host(qh, kn, vn, k2, v2, L, out_host)
         assert torch.equal(a.cpu().view(torch.int16), out_host.view(torch.int16))
+        assert g_host.last_launch_count() == (4 if pinned else 3)
     assert torch.equal(k, k2) and torch.equal(v, v2)
 
 
