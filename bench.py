@@ -132,6 +132,7 @@ class Layers:
         self.ctx = []
         self.qbar_bf16 = False
         self.cluster = 0
+        self.finish_threads = 0
 
     def make_contexts(self, **override):
         for c in self.ctx:
@@ -143,6 +144,9 @@ class Layers:
         if self.cluster:
             for c in self.ctx:
                 c.set_cluster_size(self.cluster)
+        if self.finish_threads:
+            for c in self.ctx:
+                c.set_finish_threads(self.finish_threads)
 
     def stats(self):
         tot = {}
@@ -368,6 +372,7 @@ def run_gpu(args):
     layers = Layers(cfg, n_layers, t_per_layer, rank, torch, rt)
     layers.qbar_bf16 = args.qbar_bf16
     layers.cluster = args.cluster
+    layers.finish_threads = args.finish_threads
     global QBAR_BYTES
     QBAR_BYTES = 2 if args.qbar_bf16 else 4
     peak, peak_kind = measured_peaks()
@@ -434,7 +439,7 @@ def run_gpu(args):
         "config": {"workload": cfg.name, "B": cfg.B, "H_q": cfg.H_q, "H_kv": cfg.H_kv, "d": cfg.d,
                    "context": cfg.context, "K": cfg.K, "M": cfg.M, "r": cfg.r, "W": cfg.W, "tau": cfg.tau,
                    "R": cfg.R, "qbar_cache": "bf16" if args.qbar_bf16 else "fp32",
-                   "finish_ctas_per_head": args.cluster or "auto", "layers_rotated": n_layers, "decode_steps_per_layer": t_per_layer,
+                   "finish_ctas_per_head": args.cluster or "auto", "finish_threads": args.finish_threads or "auto", "layers_rotated": n_layers, "decode_steps_per_layer": t_per_layer,
                    "l2": "inputs larger than L2: calls rotate over independent layers",
                    "parallelism": "replicas only" if world > 1 else "single GPU"},
         "clocks": sampler.summary(),
@@ -532,6 +537,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--cluster", type=int, default=0, choices=[0, 1, 2, 4, 8],
                     help="CTAs per head in the finish kernel (0: the library's own choice)")
+    ap.add_argument("--finish-threads", type=int, default=0, choices=[0, 512, 1024],
+                    help="block shape of the finish kernel (0: the library's own choice)")
     ap.add_argument("--qbar-bf16", action="store_true",
                     help="keep the cached normalised queries in bf16 (storage variant) in every pass")
     ap.add_argument("--ladder", action="store_true",

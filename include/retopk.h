@@ -128,6 +128,16 @@ int retopk_set_qbar_format(retopk_ctx* ctx, int format);
 int retopk_set_cluster_size(retopk_ctx* ctx, int ctas_per_head);
 
 /*
+ * Block shape of the finish kernel: 1024 threads (one CTA per SM) or 512 (two CTAs per SM,
+ * each with half of the SM's shared memory, so that the selection of one head overlaps the
+ * row copies of another).  retopk_create* picks 512 when there are more heads than SMs and
+ * the shape fits.  Results do not depend on the number of CTAs per SM; outputs differ between
+ * the two shapes in the fp32 sum order only.  EUNSUPPORTED when the narrow shape does not fit
+ * (large K or r*K+W, or a long max_seq_len), EINVAL for other values or below fusion level 5.
+ */
+int retopk_set_finish_threads(retopk_ctx* ctx, int threads);
+
+/*
  * Fusion level of the reuse path, for measuring what kernel fusion buys (the paper's kernel
  * efficiency analysis, Table 4, reports five cumulative stages for its own kernels; the cut
  * points here follow its description of them and are this library's own).  Results do not

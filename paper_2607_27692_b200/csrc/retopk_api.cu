@@ -17,7 +17,9 @@ struct retopk_ctx {
     float tau;
     long long max_seq_len, score_stride, tmax_stride;
     long long n_ins, t_dec;
-    int NS, tile_cap, stage_depth, exact_stage_depth;
+    int NS, tile_cap, stage_depth, exact_stage_depth;      // of the finish shape in use
+    int finish_threads;          // 1024, or 512 with two CTAs per SM when there are more heads than SMs
+    struct FinishShape { int ok, stage_depth, exact_stage_depth; size_t smem_reuse, smem_exact, smem_finish; } shape[2];   // [0]: 1024, [1]: 512
     int num_sms, scan_grid;
     int call_serial;
     int recall_recent;
@@ -132,6 +134,22 @@ int auto_cluster(long long heads, int num_sms) {
     return cl;
 }
 
+// More heads than SMs: two narrower CTAs per SM, so that one head's selection overlaps
+// another's row copies.
+int auto_finish_threads(const retopk_ctx* c) {
+    return (long long)c->B * c->Hq > c->num_sms && c->shape[1].ok ? 512 : 1024;
+}
+
+void use_finish_shape(retopk_ctx* c, int threads) {
+    const retopk_ctx::FinishShape& sh = c->shape[threads == 512 ? 1 : 0];
+    c->finish_threads = threads;
+    c->stage_depth = sh.stage_depth;
+    c->exact_stage_depth = sh.exact_stage_depth;
+    c->smem_reuse = sh.smem_reuse;
+    c->smem_exact = sh.smem_exact;
+    c->smem_finish = sh.smem_finish;
+}
+
 // Launch with programmatic stream serialisation: the kernel may be set up while its
 // predecessor in the stream still runs; it waits (pdl_wait) before reading its inputs.
 template <class Kernel>
@@ -183,8 +201,12 @@ int launch_scan(const retopk_ctx* c, const StepArgs& a, cudaStream_t s) {
 int launch_finish(const retopk_ctx* c, const StepArgs& a, cudaStream_t s) {
     const unsigned grid = (unsigned)(c->B * c->Hq * c->cluster);      // one cluster of CTAs per head
     const size_t smem = a.mode == MODE_EXACT ? c->smem_exact : c->smem_finish;
-    if (c->d == 128) return launch_dependent(finish_kernel<128>, grid, FINISH_THREADS, smem, s, a, c->dependent_launches, c->cluster);
-    return launch_dependent(finish_kernel<64>, grid, FINISH_THREADS, smem, s, a, c->dependent_launches, c->cluster);
+    if (c->finish_threads == 512) {
+        if (c->d == 128) return launch_dependent(finish_kernel<128, 512>, grid, 512, smem, s, a, c->dependent_launches, c->cluster);
+        return launch_dependent(finish_kernel<64, 512>, grid, 512, smem, s, a, c->dependent_launches, c->cluster);
+    }
+    if (c->d == 128) return launch_dependent(finish_kernel<128, 1024>, grid, FINISH_THREADS, smem, s, a, c->dependent_launches, c->cluster);
+    return launch_dependent(finish_kernel<64, 1024>, grid, FINISH_THREADS, smem, s, a, c->dependent_launches, c->cluster);
 }
 
 // Measurement hook: event number `which` (0..3) of the current call, if recording.
@@ -203,6 +225,25 @@ void exact_list_sizes(int K, int* NS, int* tile_cap) {
     else if (K <= 1024) { *NS = 16384; *tile_cap = 8192; }
     else if (K <= 2048) { *NS = 8192; *tile_cap = 4096; }
     else { *NS = 8192; *tile_cap = 8192; }
+}
+
+// Shared memory of the exact path for a block of nt threads within `budget` bytes (mirrors the
+// carve-up at the top of exact_path): the live arrays, then the lists, whose space the
+// reduction scratch and the value-row landing zone take over once the support is emitted.
+// Returns 0 if not even `min_waves` rows per row slot fit; else the bytes, and the depth.
+size_t exact_smem(int K, int NS, int tile_cap, int d, int nt, size_t budget, int min_waves, int* depth) {
+    const size_t live = ((size_t)3 * K + SCRATCH_WORDS + 32 + 8 + 3) & ~(size_t)3;
+    const size_t lists = (size_t)2 * NS + tile_cap;
+    const size_t red = ((size_t)(nt / 32) * d + nt + 3) & ~(size_t)3;
+    const size_t wave = (size_t)nt * 16;
+    if (budget < (live + lists) * 4 || budget < (live + red) * 4 + (size_t)min_waves * wave) return 0;
+    const int slots = nt / (d / 8);
+    long long fit = (long long)((budget - (live + red) * 4) / wave);
+    long long want = (K + slots - 1) / slots;
+    long long dep = fit < want ? fit : want;
+    *depth = (int)(dep < 1 ? 1 : (dep > 16 ? 16 : dep));
+    const size_t tail = red + (size_t)*depth * wave / 4;
+    return (live + (lists > tail ? lists : tail)) * 4;
 }
 
 int check_step_args(const retopk_ctx* c, const void* q, const void* k, const void* v, long long L,
@@ -403,48 +444,57 @@ int retopk_create_batched(retopk_ctx** out, int B, int H_q, int H_kv, int d, int
     c->num_sms = sms > 0 ? sms : 148;
 
     // shared-memory footprints (must mirror the carve-up at the top of each kernel)
-    const size_t red_words = (size_t)(FINISH_THREADS / 32) * d + FINISH_THREADS;
-    const size_t head_words = ((size_t)d + r + 32 + SCRATCH_WORDS + 3 * (size_t)K + 3) & ~(size_t)3;
-    const size_t big_words = (((size_t)2 * c->cap > red_words ? (size_t)2 * c->cap : red_words) + 3) & ~(size_t)3;
-    const size_t bm_words = (((size_t)max_seq_len + 31) / 32 + 3) & ~(size_t)3;
     c->smem_recall = ((size_t)d + ((M + 3) & ~3) + r + 4) * 4;
-    c->smem_reuse = (head_words + big_words + bm_words) * 4;
-    c->smem_exact = (((size_t)c->NS * 2 + (size_t)c->tile_cap + (size_t)K * 3 + SCRATCH_WORDS + 32 + 8 + 3) & ~(size_t)3) * 4;
-    int max_smem = 0;
+    int max_smem = 0, sm_smem = 0;
     cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, c->device);
-    // the rest of shared memory is the landing zone of the asynchronous row copies:
-    // 16 KB (one 16-byte piece per thread) per row kept in flight per row slot
-    const size_t wave = (size_t)FINISH_THREADS * 16;
-    if ((size_t)max_smem < c->smem_reuse + wave || (size_t)max_smem < c->smem_exact + wave) {
-        delete c;
-        return RETOPK_EUNSUPPORTED;
+    cudaDeviceGetAttribute(&sm_smem, cudaDevAttrMaxSharedMemoryPerMultiprocessor, c->device);
+    for (int v = 0; v < 2; ++v) {
+        // v = 0: one CTA of 1024 threads per SM; v = 1: two of 512, each with half of the SM's
+        // shared memory (1 KB per CTA is the system's)
+        const int nt = v == 0 ? 1024 : 512;
+        const size_t budget = v == 0 ? (size_t)max_smem : (size_t)(sm_smem / 2 - 1024);
+        retopk_ctx::FinishShape& sh = c->shape[v];
+        const size_t red_words = (size_t)(nt / 32) * d + nt;
+        const size_t head_words = ((size_t)d + r + 32 + SCRATCH_WORDS + 3 * (size_t)K + 3) & ~(size_t)3;
+        const size_t big_words = (((size_t)2 * c->cap > red_words ? (size_t)2 * c->cap : red_words) + 3) & ~(size_t)3;
+        const size_t bm_words = (((size_t)max_seq_len + 31) / 32 + 3) & ~(size_t)3;
+        sh.smem_reuse = (head_words + big_words + bm_words) * 4;
+        sh.smem_exact = exact_smem(K, c->NS, c->tile_cap, d, nt, budget, v == 0 ? 1 : 3, &sh.exact_stage_depth);
+        // the rest of shared memory is the landing zone of the asynchronous row copies: one
+        // 16-byte piece per thread per row kept in flight per row slot
+        const size_t wave = (size_t)nt * 16;
+        // the narrow shape only pays with a few waves of rows in flight on either path
+        const size_t min_waves = v == 0 ? 1 : 3;
+        sh.ok = budget >= sh.smem_reuse + min_waves * wave && sh.smem_exact > 0;
+        if (!sh.ok) continue;
+        const int slots = nt / (d / 8);
+        auto depth_for = [&](size_t fixed, int rows) {
+            long long fit = (long long)((budget - fixed) / wave);
+            long long want = (rows + slots - 1) / slots;          // one wave covers `rows` rows
+            long long dep = fit < want ? fit : want;
+            return (int)(dep < 1 ? 1 : (dep > 16 ? 16 : dep));
+        };
+        sh.stage_depth = depth_for(sh.smem_reuse, K + K / 4 > c->cap ? c->cap : K + K / 4);
+        if (sh.stage_depth * slots < K) {            // the value rows use the same zone
+            int dv = depth_for(sh.smem_reuse, K);
+            if (dv > sh.stage_depth) sh.stage_depth = dv;
+        }
+        sh.smem_reuse += (size_t)sh.stage_depth * wave;
+        sh.smem_finish = sh.smem_reuse > sh.smem_exact ? sh.smem_reuse : sh.smem_exact;
     }
-    const int slots = FINISH_THREADS / (d / 8);
-    auto depth_for = [&](size_t fixed, int rows) {
-        long long fit = (long long)(((size_t)max_smem - fixed) / wave);
-        long long want = (rows + slots - 1) / slots;          // one wave covers `rows` rows
-        long long dep = fit < want ? fit : want;
-        return (int)(dep < 1 ? 1 : (dep > 16 ? 16 : dep));
-    };
-    c->stage_depth = depth_for(c->smem_reuse, K + K / 4 > c->cap ? c->cap : K + K / 4);
-    c->exact_stage_depth = depth_for(c->smem_exact, K);
-    if (c->stage_depth * slots < K) {            // the value rows use the same zone
-        int dv = depth_for(c->smem_reuse, K);
-        if (dv > c->stage_depth) c->stage_depth = dv;
-    }
-    c->smem_reuse += (size_t)c->stage_depth * wave;
-    c->smem_exact += (size_t)c->exact_stage_depth * wave;
-    c->smem_finish = c->smem_reuse > c->smem_exact ? c->smem_reuse : c->smem_exact;
+    if (!c->shape[0].ok) { delete c; return RETOPK_EUNSUPPORTED; }
     // opt in to the device maximum once; contexts of different sizes then coexist
     cudaError_t e1, e2 = cudaSuccess;
     int occ = 0;
     const int ntile = (c->G + 7) / 8;
     if (d == 128) {
-        e1 = cudaFuncSetAttribute(finish_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
+        e1 = cudaFuncSetAttribute(finish_kernel<128, 1024>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
+        e2 = cudaFuncSetAttribute(finish_kernel<128, 512>, cudaFuncAttributeMaxDynamicSharedMemorySize, sm_smem / 2 - 1024);
         if (ntile == 1) cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, scan_kernel<128, 1>, SCAN_THREADS, 0);
         else cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, scan_kernel<128, 2>, SCAN_THREADS, 0);
     } else {
-        e1 = cudaFuncSetAttribute(finish_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
+        e1 = cudaFuncSetAttribute(finish_kernel<64, 1024>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
+        e2 = cudaFuncSetAttribute(finish_kernel<64, 512>, cudaFuncAttributeMaxDynamicSharedMemorySize, sm_smem / 2 - 1024);
         if (ntile == 1) cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, scan_kernel<64, 1>, SCAN_THREADS, 0);
         else cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, scan_kernel<64, 2>, SCAN_THREADS, 0);
     }
@@ -452,6 +502,7 @@ int retopk_create_batched(retopk_ctx** out, int B, int H_q, int H_kv, int d, int
     c->scan_grid = c->num_sms * (occ > 0 ? occ : 2);
     // finish_kernel: with few heads, a cluster of CTAs (one SM each) per head, as many as fit one wave
     c->cluster = auto_cluster((long long)B * H_q, c->num_sms);
+    use_finish_shape(c, auto_finish_threads(c));
 
 
     const size_t nh = (size_t)B * H_q;
@@ -499,10 +550,20 @@ int retopk_set_cluster_size(retopk_ctx* c, int ctas_per_head) {
     return RETOPK_OK;
 }
 
+int retopk_set_finish_threads(retopk_ctx* c, int threads) {
+    if (!c || (threads != 1024 && threads != 512)) return RETOPK_EINVAL;
+    if (threads == 512 && !c->shape[1].ok) return RETOPK_EUNSUPPORTED;
+    if (threads == 512 && c->fusion_level < 5) return RETOPK_EINVAL;
+    use_finish_shape(c, threads);
+    return RETOPK_OK;
+}
+
 int retopk_set_fusion_level(retopk_ctx* c, int level, int dependent_launches) {
     if (!c || level < 1 || level > 5 || (dependent_launches != 0 && dependent_launches != 1)) return RETOPK_EINVAL;
     if (dependent_launches && level != 5) return RETOPK_EINVAL;   // the unfused kernels are plain launches
     DeviceGuard g(c->device);
+    // the unfused kernels are sized for the wide finish shape; level 5 goes back to the default
+    use_finish_shape(c, level < 5 ? 1024 : auto_finish_threads(c));
     if (level < 5) {
         int rc = ladder_prepare(c);
         if (rc != RETOPK_OK) return rc;
@@ -841,8 +902,8 @@ int static_setup(int dev, StaticSetup** out) {
         if (cudaDeviceGetAttribute(&st->num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
             cudaDeviceGetAttribute(&st->max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess)
             return RETOPK_ECUDA;
-        if (cudaFuncSetAttribute(finish_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, st->max_smem) != cudaSuccess ||
-            cudaFuncSetAttribute(finish_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, st->max_smem) != cudaSuccess)
+        if (cudaFuncSetAttribute(finish_kernel<128, 1024>, cudaFuncAttributeMaxDynamicSharedMemorySize, st->max_smem) != cudaSuccess ||
+            cudaFuncSetAttribute(finish_kernel<64, 1024>, cudaFuncAttributeMaxDynamicSharedMemorySize, st->max_smem) != cudaSuccess)
             return RETOPK_ECUDA;
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&st->occ[0][0], scan_kernel<64, 1>, SCAN_THREADS, 0);
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&st->occ[0][1], scan_kernel<64, 2>, SCAN_THREADS, 0);
@@ -882,15 +943,9 @@ int exact_topk_decode_static(int B, int H_q, int H_kv, int d, int K, int64_t max
 
     int NS = 0, tile_cap = 0;
     exact_list_sizes(K, &NS, &tile_cap);
-    size_t smem = (((size_t)NS * 2 + (size_t)tile_cap + (size_t)K * 3 + SCRATCH_WORDS + 32 + 8 + 3) & ~(size_t)3) * 4;
-    const size_t wave = (size_t)FINISH_THREADS * 16;
-    if ((size_t)st->max_smem < smem + wave) return RETOPK_EUNSUPPORTED;
-    const int slots = FINISH_THREADS / (d / 8);
-    long long depth = (long long)(((size_t)st->max_smem - smem) / wave);
-    const long long want = (K + slots - 1) / slots;
-    if (depth > want) depth = want;
-    if (depth > 16) depth = 16;
-    smem += (size_t)depth * wave;
+    int depth = 1;
+    const size_t smem = exact_smem(K, NS, tile_cap, d, FINISH_THREADS, (size_t)st->max_smem, 1, &depth);
+    if (smem == 0) return RETOPK_EUNSUPPORTED;
 
     StepArgs a;
     memset(&a, 0, sizeof a);
@@ -930,8 +985,8 @@ int exact_topk_decode_static(int B, int H_q, int H_kv, int d, int K, int64_t max
     if (cudaGetLastError() != cudaSuccess) return RETOPK_ECUDA;
     const int cluster = auto_cluster(nh, st->num_sms);
     a.cl_shift = __builtin_ctz((unsigned)cluster);
-    if (d == 128) return launch_dependent(finish_kernel<128>, (unsigned)(nh * cluster), FINISH_THREADS, smem, s, a, 0, cluster);
-    return launch_dependent(finish_kernel<64>, (unsigned)(nh * cluster), FINISH_THREADS, smem, s, a, 0, cluster);
+    if (d == 128) return launch_dependent(finish_kernel<128, 1024>, (unsigned)(nh * cluster), FINISH_THREADS, smem, s, a, 0, cluster);
+    return launch_dependent(finish_kernel<64, 1024>, (unsigned)(nh * cluster), FINISH_THREADS, smem, s, a, 0, cluster);
 }
 
 #ifdef RETOPK_PHASE_CLOCKS

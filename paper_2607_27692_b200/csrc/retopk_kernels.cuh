@@ -308,7 +308,8 @@ struct Threshold {
 
 template <int NT>
 __device__ Threshold count_threshold(const uint32_t* key, int n, int K, int low_bit, int* s_h) {
-    static_assert(NT == 1024, "one histogram word per thread, one digit per warp");
+    static_assert(NT == 1024 || NT == 512, "32 digits are shared out over NT / 32 warps");
+    constexpr int NW = NT / 32;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     // scratch: two histograms of 32 x 32 words used alternately, then 96 words of totals
     int* s_tot = s_h + 2048;
@@ -318,11 +319,11 @@ __device__ Threshold count_threshold(const uint32_t* key, int n, int K, int low_
     kmin = __reduce_min_sync(0xffffffffu, kmin);
     kmax = __reduce_max_sync(0xffffffffu, kmax);
     if (lane == 0) { s_tot[warp] = (int)kmin; s_tot[32 + warp] = (int)kmax; }
-    s_h[tid] = 0;
-    s_h[1024 + tid] = 0;
+#pragma unroll
+    for (int i = tid; i < 2048; i += NT) s_h[i] = 0;
     __syncthreads();
-    kmin = __reduce_min_sync(0xffffffffu, (uint32_t)s_tot[lane]);
-    kmax = __reduce_max_sync(0xffffffffu, (uint32_t)s_tot[32 + lane]);
+    kmin = __reduce_min_sync(0xffffffffu, lane < NW ? (uint32_t)s_tot[lane] : 0xffffffffu);
+    kmax = __reduce_max_sync(0xffffffffu, lane < NW ? (uint32_t)s_tot[32 + lane] : 0u);
     Threshold res;
     res.kmax = kmax;
     res.count = n;
@@ -339,9 +340,12 @@ __device__ Threshold count_threshold(const uint32_t* key, int n, int K, int low_
             if ((k & himask) == prefix) atomicAdd(&hist[(((k >> shift) & ((1u << width) - 1u)) << 5) + lane], 1);
         }
         __syncthreads();
-        const int tot = __reduce_add_sync(0xffffffffu, hist[(warp << 5) + lane]);   // digit `warp`
-        hist[tid] = 0;                                // ready for the round after next
-        if (lane == 0) s_tot[64 + warp] = tot;
+#pragma unroll
+        for (int dgt = warp; dgt < 32; dgt += NW) {   // a warp sums the lane columns of its digit(s)
+            const int tot = __reduce_add_sync(0xffffffffu, hist[(dgt << 5) + lane]);
+            hist[(dgt << 5) + lane] = 0;              // ready for the round after next
+            if (lane == 0) s_tot[64 + dgt] = tot;
+        }
         __syncthreads();
         const int c = s_tot[64 + 31 - lane];          // lane l looks at digit 31 - l: descending
         int inc = c;
@@ -496,7 +500,7 @@ __device__ void attend(const uint16_t* vbase, int ns, const int32_t* s_sup_idx, 
         kmax = __reduce_max_sync(0xffffffffu, kmax);
         if (lane == 0) s_ws[warp] = (int)kmax;
         __syncthreads();
-        kmax = __reduce_max_sync(0xffffffffu, (uint32_t)s_ws[lane]);
+        kmax = __reduce_max_sync(0xffffffffu, lane < NW ? (uint32_t)s_ws[lane] : 0u);
         __syncthreads();
     }
     const float smax = key_score(kmax);
@@ -1115,21 +1119,21 @@ __device__ void exact_path(const StepArgs& a, unsigned char* smem_raw) {
     // and come from L2); only the value rows are shared out, and rank 0 writes the results.
     const int bh = finish_head(a);
     const int cl_rank = finish_rank(a), cl_size = 1 << a.cl_shift;
-    // layout (words): key[NS] idx[NS] (aliased later by red[NW*D+NT]) tile[tile_cap]
-    //                 sup_idx[K] sup_key[K] w[K] cnt[SCRATCH_WORDS] ws[32] misc[8] stage[depth*NT*4]
-    uint32_t* s_key = reinterpret_cast<uint32_t*>(smem_raw);
-    int32_t* s_idx = reinterpret_cast<int32_t*>(s_key + a.NS);
-    float* s_red = reinterpret_cast<float*>(smem_raw);
-    int32_t* s_tile = s_idx + a.NS;
-    int32_t* s_sup_idx = s_tile + a.tile_cap;
+    // layout (words): sup_idx[K] sup_key[K] w[K] cnt[SCRATCH_WORDS] ws[32] misc[8]
+    //                 | lists: key[NS] idx[NS] tile[tile_cap]; dead once the support is emitted and
+    //                   then reused by attend: red[NW*D+NT], stage[depth*NT*4] (may run past the lists)
+    constexpr int NW = NT / 32;
+    int32_t* s_sup_idx = reinterpret_cast<int32_t*>(smem_raw);
     uint32_t* s_sup_key = reinterpret_cast<uint32_t*>(s_sup_idx + a.K);
     float* s_w = reinterpret_cast<float*>(s_sup_key + a.K);
     uint32_t* s_hist = reinterpret_cast<uint32_t*>(s_w + a.K);
     int* s_ws = reinterpret_cast<int*>(s_hist + SCRATCH_WORDS);
     int* s_misc = s_ws + 32;
-    // landing zone of the value-row copies, on a 16-byte boundary
-    uint4* s_stage = reinterpret_cast<uint4*>(
-        reinterpret_cast<uint32_t*>(smem_raw) + ((2 * a.NS + a.tile_cap + 3 * a.K + SCRATCH_WORDS + 32 + 8 + 3) & ~3));
+    uint32_t* s_key = reinterpret_cast<uint32_t*>(smem_raw) + ((3 * a.K + SCRATCH_WORDS + 32 + 8 + 3) & ~3);
+    int32_t* s_idx = reinterpret_cast<int32_t*>(s_key + a.NS);
+    int32_t* s_tile = s_idx + a.NS;
+    float* s_red = reinterpret_cast<float*>(s_key);
+    uint4* s_stage = reinterpret_cast<uint4*>(s_key + ((NW * D + NT + 3) & ~3));
 
     const int tid = threadIdx.x;
     const int bkv = kv_group_of(bh, a);
@@ -1284,15 +1288,15 @@ __device__ void exact_path(const StepArgs& a, unsigned char* smem_raw) {
 // the reuse path never waited for the scan's results, a head on the exact path selects from
 // them; both end with softmax.V and the support insert.  Heads of one step run side by side.
 // ------------------------------------------------------------------------------------
-template <int D>
-__global__ void __launch_bounds__(FINISH_THREADS, 1) finish_kernel(const StepArgs a) {
+template <int D, int NT>
+__global__ void __launch_bounds__(NT, 1024 / NT) finish_kernel(const StepArgs a) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     pdl_wait();        // scores and tile maxima come from the scan, recalled slots and paths from recall_kernel
     if (blockIdx.x == 0 && threadIdx.x == 0) *a.scan_counter = 0u;      // the scan before this kernel is complete
     if (a.mode == MODE_RETOPK && a.ws_path[finish_head(a)] == PATH_REUSE) {
-        if (!a.skip_reuse) reuse_path<D, FINISH_THREADS>(a, smem_raw);
+        if (!a.skip_reuse) reuse_path<D, NT>(a, smem_raw);
     } else {
-        exact_path<D, FINISH_THREADS>(a, smem_raw);
+        exact_path<D, NT>(a, smem_raw);
     }
 }
 

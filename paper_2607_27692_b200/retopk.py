@@ -39,6 +39,7 @@ SIGNATURES = {
     "retopk_set_recall_mode": (_i32, [_vp, _i32]),
     "retopk_set_qbar_format": (_i32, [_vp, _i32]),
     "retopk_set_cluster_size": (_i32, [_vp, _i32]),
+    "retopk_set_finish_threads": (_i32, [_vp, _i32]),
     "retopk_set_fusion_level": (_i32, [_vp, _i32, _i32]),
     "retopk_destroy": (_i32, [_vp]),
     "retopk_reset": (_i32, [_vp, _vp]),
@@ -157,6 +158,10 @@ class ReTopK:
     def set_cluster_size(self, ctas_per_head: int):
         """CTAs (one SM each) per head in the finish kernel: 1, 2, 4 or 8."""
         _check(self.lib.retopk_set_cluster_size(self.h, ctas_per_head), "retopk_set_cluster_size")
+
+    def set_finish_threads(self, threads: int):
+        """Block shape of the finish kernel: 1024 (one CTA per SM) or 512 (two per SM)."""
+        _check(self.lib.retopk_set_finish_threads(self.h, threads), "retopk_set_finish_threads")
 
     def set_fusion_level(self, level: int, dependent_launches: bool = False):
         """Fusion level 1..5 of the reuse path (Table 4's ladder); results do not depend on it."""

@@ -1,8 +1,9 @@
-"""Thread-block cluster per head in the finish kernel (run with -m gpu).
+"""Launch shapes of the finish kernel (run with -m gpu).
 
-With 2, 4 or 8 CTAs per head the candidate scores and the value rows are shared out over the
-CTAs.  Decisions, supports and candidate counts must not depend on the cluster size; outputs
-may differ in the order of the fp32 partial sums only.
+Thread-block cluster per head: with 2, 4 or 8 CTAs per head the candidate scores and the value
+rows are shared out over the CTAs.  Narrow blocks: 512 threads, two CTAs per SM.  Decisions,
+supports and candidate counts must not depend on either; outputs may differ in the order of the
+fp32 partial sums only.
 """
 import pytest
 import torch
@@ -42,9 +43,10 @@ def test_cluster_sizes_agree(rt, P, case):
     st = wl.make_stream(cfg, steps=cfg.steps)
     k, v = P.to_dev(st.k), P.to_dev(st.v)
 
-    def run(size):
+    def run(size, threads=1024):
         g = rt.ReTopK.from_config(cfg)
         g.set_cluster_size(size)
+        g.set_finish_threads(threads)
         rec = []
         for t in range(cfg.steps):
             out = g.decode_step(P.to_dev(st.q[t]), k, v, st.seq_len(t))
@@ -57,8 +59,8 @@ def test_cluster_sizes_agree(rt, P, case):
 
     ref, ref_stats = run(1)
     assert ref_stats["reuse"] > 0 and ref_stats["fallback"] + ref_stats["refresh"] > 0
-    for size in (2, 4, 8):
-        rec, stats = run(size)
+    for size, threads in ((2, 1024), (4, 1024), (8, 1024), (1, 512), (2, 512)):
+        rec, stats = run(size, threads)
         assert stats == ref_stats, (size, stats, ref_stats)
         for t, (a, b) in enumerate(zip(ref, rec)):
             for name, x, y in zip(("out", "support", "path", "rho_max", "n_cand", "exact_out", "exact_idx"), a, b):
@@ -69,13 +71,14 @@ def test_cluster_sizes_agree(rt, P, case):
                     assert torch.equal(x, y), (size, t, name)
 
 
-def test_cluster_against_the_oracle(rt, P, oracle_mod):
+def test_shapes_against_the_oracle(rt, P, oracle_mod):
     cfg = wl.CONFIGS["tiny"].replace(context=2500, steps=24, B=1, H_q=8, H_kv=2, d=128, K=96, M=8, r=3, W=40)
     st = wl.make_stream(cfg, steps=cfg.steps)
-    for size in (4, 8):
+    for size, threads in ((4, 1024), (8, 1024), (1, 512)):
         o = oracle_mod.Oracle.from_config(cfg)
         g = rt.ReTopK.from_config(cfg)
         g.set_cluster_size(size)
+        g.set_finish_threads(threads)
         P.teacher_forced_run(cfg, st, cfg.steps, o, g, P.to_dev(st.k), P.to_dev(st.v))
         so, sg = o.stats(), g.stats()
         assert so["reuse"] > 0
@@ -91,3 +94,9 @@ def test_cluster_argument_checks(rt):
     assert lib.retopk_set_cluster_size(None, 2) == -1
     for ok in (1, 2, 4, 8):
         assert lib.retopk_set_cluster_size(g.h, ok) == 0
+    for bad in (0, 256, 768, 2048):
+        assert lib.retopk_set_finish_threads(g.h, bad) == -1
+    assert lib.retopk_set_finish_threads(g.h, 512) == 0 and lib.retopk_set_finish_threads(g.h, 1024) == 0
+    # a support size whose lists do not fit half an SM's shared memory
+    big = rt.ReTopK.from_config(wl.CONFIGS["tiny"].replace(K=2048, r=8, W=512, context=20000, steps=4))
+    assert lib.retopk_set_finish_threads(big.h, 512) == -2
