@@ -218,13 +218,12 @@ void prof_done(retopk_ctx* c, int kind) {
     if (c->prof_events && c->prof_calls < c->prof_max) c->prof_kind[c->prof_calls++] = (unsigned char)kind;
 }
 
-// Sizes of the exact path's shared lists for a support size K (a trade between the range of
-// short histories handled without the tile bound and the room left for value-row copies).
+// Sizes of the exact path's shared lists for a support size K.  The landing zone of the value
+// rows reuses their space, so they cost nothing up to the size of that zone; 8192 entries for
+// K <= 512 keep the narrow (two CTAs per SM) shape within half an SM's shared memory.
 void exact_list_sizes(int K, int* NS, int* tile_cap) {
     if (K <= 512) { *NS = 8192; *tile_cap = 4096; }
-    else if (K <= 1024) { *NS = 16384; *tile_cap = 8192; }
-    else if (K <= 2048) { *NS = 8192; *tile_cap = 4096; }
-    else { *NS = 8192; *tile_cap = 8192; }
+    else { *NS = 16384; *tile_cap = 8192; }
 }
 
 // Shared memory of the exact path for a block of nt threads within `budget` bytes (mirrors the

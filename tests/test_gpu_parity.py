@@ -70,7 +70,7 @@ def test_exact_topk_decode_matches_oracle(rt, P, oracle_mod, B, H_q, H_kv, d, L,
                                      f"seq {b} head {h}")
     P.assert_outputs_close(out, ref_out, "exact_topk_decode")
     # the tile-maximum bound needs at least K 16-row tiles, or all of L must fit the shared list
-    list_capacity = 16384 if 512 < K <= 1024 else 8192
+    list_capacity = 16384 if K > 512 else 8192
     fast = L <= K or -(-L // 16) >= K or L <= list_capacity
     assert g.stats()["slow_select"] == (0 if fast else B * H_q)
     assert g.last_launch_count() == 2
