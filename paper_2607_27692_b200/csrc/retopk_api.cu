@@ -340,26 +340,12 @@ void ladder_bind(StepArgs& a, void* const* buf) {
         ++launches;                                                         \
     } while (0)
 
-// One decode step at fusion level 1..4.  Order: decision kernels, scan (exact heads), the
-// reuse path's kernels, finish_kernel (exact heads only).
-int ladder_step(retopk_ctx* c, StepArgs a, cudaStream_t s) {
+// The launches of one decode step at fusion level 1..4.  Order: decision kernels, scan (exact
+// heads), the reuse path's kernels, finish_kernel (exact heads only).
+int ladder_launches(retopk_ctx* c, const StepArgs& a, cudaStream_t s, int* n_launches) {
     const int level = c->fusion_level;
     const unsigned grid = (unsigned)(c->B * c->Hq);
     int launches = 0, rc;
-    void* buf[8] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
-    if (level == 4) {
-        for (int i = 0; i < 8; ++i) buf[i] = c->lw_persist[i];
-    } else {
-        for (int i = 0; i < 8; ++i)
-            if (ladder_needs(level, i) &&
-                cudaMallocFromPoolAsync(&buf[i], c->lw_bytes[i] ? c->lw_bytes[i] : 16, c->pool, s) != cudaSuccess) {
-                for (int j = 0; j < i; ++j) if (buf[j]) cudaFreeAsync(buf[j], s);
-                cudaGetLastError();
-                return RETOPK_ENOMEM;
-            }
-    }
-    ladder_bind(a, buf);
-    a.skip_reuse = 1;
     const bool d128 = c->d == 128;
 
     prof_mark(c, 0, s);
@@ -401,11 +387,38 @@ int ladder_step(retopk_ctx* c, StepArgs a, cudaStream_t s) {
     ++launches;
     prof_mark(c, 3, s);
     prof_done(c, 0);
+    *n_launches = launches;
+    return RETOPK_OK;
+}
+
+// One decode step at fusion level 1..4: the buffers (kept by the context at level 4, from the
+// pool otherwise) around the launches.
+int ladder_step(retopk_ctx* c, StepArgs a, cudaStream_t s) {
+    const int level = c->fusion_level;
+    void* buf[8] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
+    int rc = RETOPK_OK;
+    if (level == 4) {
+        for (int i = 0; i < 8; ++i) buf[i] = c->lw_persist[i];
+    } else {
+        for (int i = 0; i < 8 && rc == RETOPK_OK; ++i)
+            if (ladder_needs(level, i) &&
+                cudaMallocFromPoolAsync(&buf[i], c->lw_bytes[i] ? c->lw_bytes[i] : 16, c->pool, s) != cudaSuccess) {
+                cudaGetLastError();
+                buf[i] = nullptr;
+                rc = RETOPK_ENOMEM;
+            }
+    }
+    int launches = 0;
+    if (rc == RETOPK_OK) {
+        ladder_bind(a, buf);
+        a.skip_reuse = 1;
+        rc = ladder_launches(c, a, s, &launches);
+    }
     if (level != 4)
         for (int i = 0; i < 8; ++i)
-            if (buf[i] && cudaFreeAsync(buf[i], s) != cudaSuccess) return RETOPK_ECUDA;
-    c->last_launches = launches;
-    return RETOPK_OK;
+            if (buf[i] && cudaFreeAsync(buf[i], s) != cudaSuccess && rc == RETOPK_OK) rc = RETOPK_ECUDA;
+    if (rc == RETOPK_OK) c->last_launches = launches;
+    return rc;
 }
 #undef LADDER_LAUNCH
 
