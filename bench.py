@@ -155,9 +155,9 @@ class Layers:
                 tot[key] = (tot.get(key, 0) | val) if key == "status" else tot.get(key, 0) + val
         return tot
 
-    def call(self, i, kind, stream):
-        """Call number i of a pass: layer i % n at decode offset i // n."""
-        l, t = i % self.n, i // self.n
+    def call(self, i, kind, stream, single=False):
+        """Call number i of a pass: layer i % n at decode offset i // n (single: layer 0 at offset i)."""
+        l, t = (0, i) if single else (i % self.n, i // self.n)
         L = self.cfg.context + t + 1
         h = self.ctx[l].h
         qstep = self.cfg.B * self.cfg.H_q * self.cfg.d * 2
@@ -184,13 +184,18 @@ def sync_all(torch, dist):
     torch.cuda.synchronize()
 
 
-def timed_pass(layers, kind, warmup, steps, torch, dist, profile=False, sampler=None):
-    """Reset, run `warmup` untimed calls, then time exactly `steps` calls with CUDA events."""
+def timed_pass(layers, kind, warmup, steps, torch, dist, profile=False, sampler=None, per_step=False, single=False):
+    """Reset, run `warmup` untimed calls, then time exactly `steps` calls with CUDA events.
+
+    per_step: also record an event after every call and return the distribution of the intervals
+    (the extra stream entries keep consecutive calls from overlapping their launches, so these are
+    a little longer than the pass average).  single: every call goes to layer 0 (hot L2).
+    """
     stream = torch.cuda.current_stream().cuda_stream
     for c in layers.ctx:
         c.reset()
     for i in range(warmup):
-        layers.call(i, kind, stream)
+        layers.call(i, kind, stream, single)
     sync_all(torch, dist)
     before = layers.stats()
     if profile:
@@ -201,9 +206,12 @@ def timed_pass(layers, kind, warmup, steps, torch, dist, profile=False, sampler=
     if sampler is not None:
         sampler.__enter__()
     sync_all(torch, dist)
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(steps)] if per_step else None
     e0.record()
     for i in range(warmup, warmup + steps):
-        layers.call(i, kind, stream)
+        layers.call(i, kind, stream, single)
+        if per_step:
+            marks[i - warmup].record()
     e1.record()
     sync_all(torch, dist)
     if sampler is not None:
@@ -221,7 +229,12 @@ def timed_pass(layers, kind, warmup, steps, torch, dist, profile=False, sampler=
     after = layers.stats()
     delta = {key: (after[key] if key == "status" else after[key] - before[key]) for key in after}
     launches = steps * (2 if kind == "exact" else 3)
-    return dict(ms=ms, us_per_step=1e3 * ms / steps, stats=delta, prof=prof, launches=launches)
+    dist_us = None
+    if per_step:
+        ts = np.array([1e3 * a.elapsed_time(b) for a, b in zip([e0] + marks[:-1], marks)])
+        dist_us = {"median": round(float(np.median(ts)), 2), "p10": round(float(np.percentile(ts, 10)), 2),
+                   "p90": round(float(np.percentile(ts, 90)), 2)}
+    return dict(ms=ms, us_per_step=1e3 * ms / steps, stats=delta, prof=prof, launches=launches, dist_us=dist_us)
 
 
 QBAR_BYTES = 4      # bytes per cached query element; 2 with --qbar-bf16
@@ -350,9 +363,19 @@ def cpu_baseline(cfg, stream, budget_s=12.0, max_steps=48):
         n += 1
     el = time.perf_counter() - t0
     s = o.stats()
+    per_path = {}
+    for label, override, budget in (("pure_reuse", dict(tau=-2.0, R=0), 3.0), ("pure_exact", dict(tau=2.0, R=0), 6.0)):
+        op = retopk_oracle.Oracle.from_config(cfg, **override)
+        op.decode_step(stream.q[0], stream.k, stream.v, stream.seq_len(0))       # fills the cache; not timed
+        m, t1 = 0, time.perf_counter()
+        while m < min(24, stream.q.shape[0] - 1) and time.perf_counter() - t1 < budget:
+            op.decode_step(stream.q[m + 1], stream.k, stream.v, stream.seq_len(m + 1))
+            m += 1
+        per_path[label] = {"us_per_step": round(1e6 * (time.perf_counter() - t1) / max(m, 1), 1), "steps": m}
     return {"value": round(1e6 * el / n, 1), "unit": UNIT, "cores": retopk_oracle.num_threads(), "kind": "oracle",
             "sample": f"first {n} decode steps of layer 0, all {cfg.B}x{cfg.H_q} heads, "
-                      f"{s['reuse']}/{s['fallback']}/{s['refresh']} reuse/fallback/refresh head-steps"}
+                      f"{s['reuse']}/{s['fallback']}/{s['refresh']} reuse/fallback/refresh head-steps",
+            "per_path": per_path}
 
 
 def run_gpu(args):
@@ -393,10 +416,18 @@ def run_gpu(args):
     # forced paths and the paper-default threshold
     layers.make_contexts(tau=-2.0, R=0)
     reuse = timed_pass(layers, "retopk", W, K, torch, dist)
+    reuse_d = timed_pass(layers, "retopk", W, K, torch, dist, per_step=True)
+    # one layer only: candidate rows and caches of the step before are still in L2
+    n_hot = min(t_per_layer, W + K)
+    w_hot = min(W, n_hot // 4)
+    reuse_hot = timed_pass(layers, "retopk", w_hot, n_hot - w_hot, torch, dist, single=True)
     layers.make_contexts(tau=2.0, R=0)
     fallb = timed_pass(layers, "retopk", W, K, torch, dist)
+    fallb_d = timed_pass(layers, "retopk", W, K, torch, dist, per_step=True)
     layers.make_contexts(tau=0.85)
     paper = timed_pass(layers, "retopk", W, K, torch, dist)
+    paper_d = timed_pass(layers, "retopk", W, K, torch, dist, per_step=True)
+    paper_hot = timed_pass(layers, "retopk", w_hot, n_hot - w_hot, torch, dist, single=True)
     fidelity = fidelity_pass(layers, torch, calls=min(96, W + K)) if rank == 0 else None
     ladder = fusion_ladder(layers, W, K, torch, dist) if args.ladder else None
 
@@ -457,6 +488,11 @@ def run_gpu(args):
                                   "pure_reuse": round(exact["us_per_step"] / reuse["us_per_step"], 3)},
         "paths": {"pure_reuse": path_report(reuse, False), "pure_exact": path_report(fallb, True),
                   "tau_0.85": path_report(paper, False)},
+        "per_step_us": {"note": "an event after every call (calls then do not overlap their launches)",
+                        "pure_reuse": reuse_d["dist_us"], "pure_exact": fallb_d["dist_us"], "tau_0.85": paper_d["dist_us"]},
+        "single_layer_hot_l2_us": {"note": "every call on layer 0: the step before left its rows in L2; not the headline",
+                                   "pure_reuse": round(reuse_hot["us_per_step"], 2),
+                                   "tau_0.85": round(paper_hot["us_per_step"], 2)},
         "slow_select": head["stats"]["slow_select"],
         "fidelity_tau_0.85": fidelity,
         "roofline": roofline,
