@@ -104,3 +104,28 @@ def test_random_small_configurations_teacher_forced(rt, P, oracle_mod, seed):
     for key in ("steps", "reuse", "fallback", "refresh"):
         assert abs(sg[key] - so[key]) <= 2, (cfg, key, sg, so)       # an excused flip at the tau band at most
     assert sg["status"] == 0
+
+
+def test_non_finite_inputs_stay_in_bounds(rt, P):
+    """NaN and infinities in q / K / V: results are unspecified, but every index the library
+    reports lies inside the history, the status word stays clear and the calls return."""
+    cfg = wl.CONFIGS["tiny"].replace(context=3000, steps=12, B=2, H_q=4, H_kv=2, d=128, K=100, M=6, r=3, W=20, R=5)
+    st = wl.make_stream(cfg, steps=cfg.steps)
+    rng = np.random.default_rng(5)
+    k, v, q = st.k.copy(), st.v.copy(), st.q.copy()
+    specials = np.array([0x7FC0, 0xFFC0, 0x7F80, 0xFF80], dtype=np.uint16)      # +-NaN, +-inf as bf16 bits
+    for arr, count in ((k, 4000), (v, 4000), (q, 300)):
+        flat = arr.reshape(-1)
+        flat[rng.integers(0, flat.size, count)] = specials[rng.integers(0, 4, count)]
+    q[3] = 0x7FC0                                                            # one step with an all-NaN query
+    g = rt.ReTopK.from_config(cfg)
+    kd, vd = P.to_dev(k), P.to_dev(v)
+    for t in range(cfg.steps):
+        L = st.seq_len(t)
+        g.decode_step(P.to_dev(q[t]), kd, vd, L)
+        sup = g.last_step()["support"].cpu().numpy()
+        assert ((sup >= -1) & (sup < L)).all()
+        for row in sup.reshape(-1, cfg.K):
+            live = row[row >= 0]
+            assert (np.diff(live) > 0).all()                                 # ascending, no duplicates
+    assert g.stats()["status"] == 0 and g.stats()["steps"] == cfg.steps * cfg.B * cfg.H_q
