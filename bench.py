@@ -427,6 +427,7 @@ def run_gpu(args):
     layers.make_contexts(tau=0.85)
     paper = timed_pass(layers, "retopk", W, K, torch, dist)
     paper_d = timed_pass(layers, "retopk", W, K, torch, dist, per_step=True)
+    paper_p = timed_pass(layers, "retopk", W, K, torch, dist, profile=True)
     paper_hot = timed_pass(layers, "retopk", w_hot, n_hot - w_hot, torch, dist, single=True)
     fidelity = fidelity_pass(layers, torch, calls=min(96, W + K)) if rank == 0 else None
     ladder = fusion_ladder(layers, W, K, torch, dist) if args.ladder else None
@@ -487,7 +488,8 @@ def run_gpu(args):
                                   "tau_0.85": round(exact["us_per_step"] / paper["us_per_step"], 3),
                                   "pure_reuse": round(exact["us_per_step"] / reuse["us_per_step"], 3)},
         "paths": {"pure_reuse": path_report(reuse, False), "pure_exact": path_report(fallb, True),
-                  "tau_0.85": path_report(paper, False)},
+                  "tau_0.85": path_report(paper, False) | {"kernel_avg_us": {
+                      name: round(1e3 * rec["ms"] / max(rec["launches"], 1), 2) for name, rec in paper_p["prof"].items()}}},
         "per_step_us": {"note": "an event after every call (calls then do not overlap their launches)",
                         "pure_reuse": reuse_d["dist_us"], "pure_exact": fallb_d["dist_us"], "tau_0.85": paper_d["dist_us"]},
         "single_layer_hot_l2_us": {"note": "every call on layer 0: the step before left its rows in L2; not the headline",
