@@ -7,6 +7,7 @@ itself; nothing here does arithmetic, it only marshals numpy arrays.
 from __future__ import annotations
 
 import ctypes as C
+import fcntl
 import os
 import subprocess
 
@@ -19,14 +20,26 @@ _LIB = os.path.join(_HERE, "libretopk_oracle.so")
 PATH_REUSE, PATH_FALLBACK, PATH_REFRESH = 0, 1, 2
 
 
+def _stale() -> bool:
+    return not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC)
+
+
 def build(force: bool = False) -> str:
-    """Compile the oracle into ``libretopk_oracle.so`` (skipped when up to date)."""
-    if (not force and os.path.exists(_LIB)
-            and os.path.getmtime(_LIB) >= os.path.getmtime(_SRC)):
+    """Compile the oracle into ``libretopk_oracle.so`` (skipped when up to date; safe to call
+    from several processes at once)."""
+    if not force and not _stale():
         return _LIB
-    cmd = ["gcc", "-O2", "-std=c99", "-fopenmp", "-fPIC", "-shared", "-ffp-contract=off",
-           "-o", _LIB, _SRC, "-lm"]
-    subprocess.run(cmd, check=True)
+    with open(_LIB + ".lock", "w") as lock:
+        fcntl.flock(lock, fcntl.LOCK_EX)
+        try:
+            if force or _stale():
+                tmp = f"{_LIB}.{os.getpid()}.tmp"
+                cmd = ["gcc", "-O2", "-std=c99", "-fopenmp", "-fPIC", "-shared", "-ffp-contract=off",
+                       "-o", tmp, _SRC, "-lm"]
+                subprocess.run(cmd, check=True)
+                os.replace(tmp, _LIB)
+        finally:
+            fcntl.flock(lock, fcntl.LOCK_UN)
     return _LIB
 
 

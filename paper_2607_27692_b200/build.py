@@ -1,6 +1,7 @@
 """Compile the CUDA library in-tree: ``csrc/retopk_api.cu`` -> ``libretopk.so`` (sm_100a)."""
 from __future__ import annotations
 
+import fcntl
 import os
 import shutil
 import subprocess
@@ -25,15 +26,27 @@ def is_stale() -> bool:
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
-    """Run nvcc if the library is missing or older than its sources; return its path."""
+    """Run nvcc if the library is missing or older than its sources; return its path.
+
+    Several processes may call this at once (one rank per GPU): the check and the build run
+    under a file lock, and the library appears under its final name in one rename.
+    """
     if not force and not is_stale():
         return LIB_PATH
     nvcc = shutil.which("nvcc") or "/usr/local/cuda/bin/nvcc"
     if not os.path.exists(nvcc):
         raise RuntimeError("nvcc not found: cannot build libretopk.so")
-    units = [s for s in _sources() if s.endswith(".cu")]
-    cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-o", LIB_PATH] + units
-    subprocess.run(cmd, check=True)
+    with open(LIB_PATH + ".lock", "w") as lock:
+        fcntl.flock(lock, fcntl.LOCK_EX)
+        try:
+            if force or is_stale():          # another process may have built it meanwhile
+                units = [s for s in _sources() if s.endswith(".cu")]
+                tmp = f"{LIB_PATH}.{os.getpid()}.tmp"
+                cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-o", tmp] + units
+                subprocess.run(cmd, check=True)
+                os.replace(tmp, LIB_PATH)
+        finally:
+            fcntl.flock(lock, fcntl.LOCK_UN)
     return LIB_PATH
 
 
