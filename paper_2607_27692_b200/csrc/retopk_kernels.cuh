@@ -9,13 +9,16 @@
 //                  e_i = q.k_i/sqrt(d) (Eq. 4); every key row streams once through the
 //                  tensor cores for all G query heads of its group; also the maximum of
 //                  every 16-row tile.
-//   finish_kernel  one CTA per (sequence, query head), heads of both paths side by side.
+//   finish_kernel  one CTA per (sequence, query head) - or a thread-block cluster of 2-8 CTAs
+//                  when there are few heads, or 512-thread CTAs two to an SM when there are
+//                  more heads than SMs - with heads of both paths side by side.
 //                  Reuse path: candidate union (Eq. 8-9) in a shared-memory bitmap, exact
 //                  scores of the gathered key rows (Eq. 10), Top-K (Eq. 11).  Exact path:
 //                  global Top-K (Eq. 1) of the scanned scores (tile maxima give a lower
 //                  bound for the K-th score, only the tiles that reach it are read back).
 //                  Both: softmax.V (Eq. 12) and the support insert.
 //                  Exact Top-K attention is scan + finish with every head on the exact path.
+// All three are programmatic dependent launches; ingest_kernel serves the host-buffer entry point.
 #pragma once
 #include <cooperative_groups.h>
 #include <cuda_bf16.h>
