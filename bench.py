@@ -515,7 +515,7 @@ def run_gpu(args):
 # of one launch over its 32 groups) from the ncu capture of a one-layer run whose summary is kept
 # under profiles/; a launch's traffic is this times the groups it scanned (traffic grows in
 # proportion to the rows streamed).  The K = 1024 variant streams the same rows per group.
-NCU_TRAFFIC_PER_GROUP = {"headline128k": 34.29e6, "headline128k_k1024": 34.29e6}
+NCU_TRAFFIC_PER_GROUP = {"headline128k": 33.88e6, "headline128k_k1024": 33.88e6}
 
 
 # --------------------------------------------------------------------------- reference arm
