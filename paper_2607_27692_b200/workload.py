@@ -85,6 +85,8 @@ CONFIGS = {
     # the paper's cross-model setting at 128K uses K = 1024 (Table 2); same streams as the headline
     "headline128k_k1024": Config("headline128k_k1024", 4, 4, 32, 8, 128, 131072, 512, 1024, 128, 4, 256, 0.9, 32,
                                  256, 0.02),
+    # one sequence at 128K: the batch size of the paper's own latency measurements
+    "single128k": Config("single128k", 6, 1, 32, 8, 128, 131072, 512, 512, 128, 4, 256, 0.9, 32, 256, 0.02),
     "stress128k": Config("stress128k", 5, 16, 32, 8, 128, 131072, 256, 2048, 128, 8, 512, 0.95, 8,
                          256, 0.02, regime_switch=16),
 }

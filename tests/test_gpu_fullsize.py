@@ -61,6 +61,13 @@ def test_headline_shapes_with_k1024(rt, P, oracle_mod):
     assert sg["steps"] == 10 * 4 * 32 and sg["slow_select"] == 0 and sg["status"] == 0
 
 
+def test_single_sequence_at_128k(rt, P, oracle_mod):
+    """Batch 1 at 128K (the paper's latency setting): four CTAs per head in the finish kernel."""
+    so, sg, ex = run_sampled(rt, P, oracle_mod, "single128k", 8, [0], tau=0.85)
+    assert so["reuse"] > 0 and so["fallback"] > 0
+    assert sg["steps"] == 8 * 32 and sg["slow_select"] == 0 and sg["status"] == 0
+
+
 def test_stress_config(rt, P, oracle_mod):
     """128K, batch 16, K = 2048, r = 8, W = 512, refresh every 8 steps: mostly exact steps."""
     so, sg, ex = run_sampled(rt, P, oracle_mod, "stress128k", 10, [9])
