@@ -29,7 +29,7 @@
  *     one stream at a time.
  *   - The caller owns q / k_cache / v_cache / out; the context owns its cache state and
  *     workspaces, allocated once in create and released in destroy.  decode calls allocate
- *     nothing.
+ *     nothing (the measurement-only fusion levels 1-3 of retopk_set_fusion_level excepted).
  *   - Return value: 0 on success, a negative RETOPK_E* code otherwise.  Inputs containing
  *     NaN or Inf give unspecified (but memory-safe) results.  The kernels never trap.
  */
