@@ -40,8 +40,8 @@
  *     recently inserted entries are recalled instead of the most similar ones, and rho_max is
  *     the largest similarity among THOSE entries (the paper gives no formula; the row's
  *     higher exact-path share fits a maximum taken over fewer entries);
- *   - prefill seeding (Sec. 3.3: the cache "is initialized from the final C prompt tokens"):
- *     the paper does not say which support a prompt token gets; here each of the last
+ *   - prefill seeding (Sec. 3.3, cache paragraph: the cache starts from the last C prompt
+ *     tokens): the paper does not say which support a prompt token gets; here each of the last
  *     n_tail <= M prompt positions p contributes its normalised query and its CAUSAL Exact
  *     Top-K support over keys 0..p, oldest first; the decode offset stays 0;
  *   - bf16 query cache (a storage variant; the paper runs everything in BF16 and does not say
@@ -61,7 +61,8 @@
  * Pins (tests/test_oracle_pins.py): brute-force selection on small inputs, dense softmax
  * attention when K >= L, closed forms for K = 1 and K = 2, exact-path equality when
  * tau > 1 or W >= L, the hand-enumerated six-step trace in tests/golden, counter
- * identities, the candidate bound of Eq. 14, and tie cases with integer inputs.
+ * identities, the candidate bound of Eq. 14, and tie cases with integer inputs; the fidelity
+ * quantities (oracle_fidelity) by the hand trace, the W >= L case and a numpy restatement.
  */
 #include <math.h>
 #include <stdint.h>
@@ -94,6 +95,9 @@ typedef struct {
     double *last_kth;    /* [B*Hq] smallest selected score */
     int32_t *last_cand;  /* [B*Hq][r*K+W] candidate list of reuse steps */
     int32_t *last_sel;   /* [B*Hq][r] recalled slots, -1 padded */
+    double *last_out;    /* [B*Hq][d] attention output of the step */
+    int32_t *last_uni;   /* [B*Hq][r*K] union of the recalled supports U_t (Eq. 3), ascending */
+    int32_t *last_nuni;  /* [B*Hq] its size (reuse steps only) */
 } oracle_t;
 
 static double bf16_to_double(uint16_t bits) {
@@ -142,6 +146,10 @@ int oracle_create(oracle_t **out, int B, int Hq, int Hkv, int d, int M, int r, i
     o->last_kth = (double *)calloc(nh, sizeof(double));
     o->last_cand = (int32_t *)malloc(nh * ((size_t)r * K + W + 1) * sizeof(int32_t));
     o->last_sel = (int32_t *)malloc(nh * r * sizeof(int32_t));
+    o->last_out = (double *)calloc(nh * d, sizeof(double));
+    o->last_uni = (int32_t *)malloc(nh * ((size_t)r * K + 1) * sizeof(int32_t));
+    o->last_nuni = (int32_t *)calloc(nh, sizeof(int32_t));
+    if (!o->last_out || !o->last_uni || !o->last_nuni) return -2;
     if (!o->qbar || !o->sup || !o->last_sup || !o->last_path || !o->last_rho || !o->last_ncand ||
         !o->last_kth || !o->last_cand || !o->last_sel)
         return -2;
@@ -180,6 +188,7 @@ void oracle_destroy(oracle_t *o) {
     if (!o) return;
     free(o->qbar); free(o->sup); free(o->last_sup); free(o->last_path); free(o->last_rho);
     free(o->last_ncand); free(o->last_kth); free(o->last_cand); free(o->last_sel);
+    free(o->last_out); free(o->last_uni); free(o->last_nuni);
     free(o);
 }
 
@@ -334,6 +343,15 @@ static void retopk_head(oracle_t *o, size_t bh, const double *q, const uint16_t 
             for (int i = 0; i < K; ++i)
                 if (stored[i] >= 0) raw[n_raw++] = stored[i];
         }
+        /* U_t of Eq. 3: the recalled supports alone, before the window joins them */
+        {
+            int32_t *uni = o->last_uni + bh * ((size_t)r * K + 1);
+            int n_uni = 0;
+            qsort(raw, (size_t)n_raw, sizeof(int32_t), cmp_int32);
+            for (int i = 0; i < n_raw; ++i)
+                if (i == 0 || raw[i] != raw[i - 1]) uni[n_uni++] = raw[i];
+            o->last_nuni[bh] = n_uni;
+        }
         int64_t w_lo = L - W > 0 ? L - W : 0;
         for (int64_t i = w_lo; i < L; ++i) raw[n_raw++] = (int32_t)i;
         qsort(raw, (size_t)n_raw, sizeof(int32_t), cmp_int32);
@@ -366,6 +384,7 @@ static void retopk_head(oracle_t *o, size_t bh, const double *q, const uint16_t 
     o->last_rho[bh] = rho_max;
     o->last_ncand[bh] = n_scored;
     o->last_kth[bh] = kth;
+    for (int j = 0; j < d; ++j) o->last_out[bh * d + j] = out[j];
     free(rho); free(qbar);
 }
 
@@ -436,6 +455,67 @@ int oracle_prefill(oracle_t *o, const uint16_t *q_tail, const uint16_t *k, const
         }
         o->n_ins += 1;
     }
+    return 0;
+}
+
+/*
+ * Fidelity of the most recent decode step against Exact Top-K attention on the same inputs
+ * (the quantities of Eq. 2-3 and of the fidelity paragraph of Sec. 4).  Call right after
+ * oracle_decode_step with that step's q, k, v and L.  Per (sequence, head), four doubles:
+ *   [0] support recall   |S^_t & S_t| / |S_t|   (S_t exact support of Eq. 1, S^_t the step's support)
+ *   [1] retained mass    sum over i in S_t & S^_t of softmax(e restricted to S_t)_i
+ *   [2] output cosine    <o^_t, o_t> / (|o^_t| |o_t|), o_t the Exact Top-K output (Eq. 12 over S_t)
+ *   [3] coverage         |S_t & U_t| / |S_t| with U_t the union of the recalled supports (Eq. 3);
+ *                        -1 on steps that did not take the reuse path
+ * Plain definitions: one membership scan per index, left-to-right sums.
+ */
+int oracle_fidelity(const oracle_t *o, const uint16_t *q, const uint16_t *k, const uint16_t *v,
+                    int64_t L, double *four) {
+    if (L < 1 || L > o->max_seq_len) return -1;
+    const int d = o->d, G = o->Hq / o->Hkv, K = o->K;
+#pragma omp parallel for collapse(2) schedule(dynamic, 1)
+    for (int b = 0; b < o->B; ++b)
+        for (int h = 0; h < o->Hq; ++h) {
+            size_t bh = (size_t)b * o->Hq + h;
+            size_t kv = ((size_t)b * o->Hkv + h / G) * (size_t)o->max_seq_len * d;
+            double *qd = (double *)malloc((size_t)d * sizeof(double));
+            double *oe = (double *)malloc((size_t)d * sizeof(double));
+            int32_t *se = (int32_t *)malloc((size_t)K * sizeof(int32_t));
+            double kth;
+            for (int j = 0; j < d; ++j) qd[j] = bf16_to_double(q[bh * d + j]);
+            exact_head(qd, k + kv, v + kv, L, d, K, se, oe, &kth);
+            const int32_t *sr = o->last_sup + bh * K;
+            const int32_t *uni = o->last_uni + bh * ((size_t)o->r * K + 1);
+            const int n_uni = o->last_nuni[bh];
+            int ne = 0, both = 0, covered = 0;
+            double m = -INFINITY;
+            for (int i = 0; i < K && se[i] >= 0; ++i) {
+                double e = score_key(qd, k + kv + (size_t)se[i] * d, d);
+                if (e > m) m = e;
+                ++ne;
+            }
+            double denom = 0.0, kept = 0.0;
+            for (int i = 0; i < ne; ++i) {
+                double w = exp(score_key(qd, k + kv + (size_t)se[i] * d, d) - m);
+                int in_r = 0, in_u = 0;
+                for (int j = 0; j < K; ++j) if (sr[j] == se[i]) in_r = 1;
+                for (int j = 0; j < n_uni; ++j) if (uni[j] == se[i]) in_u = 1;
+                denom += w;
+                if (in_r) { kept += w; ++both; }
+                covered += in_u;
+            }
+            double dot = 0.0, na = 0.0, nb = 0.0;
+            for (int j = 0; j < d; ++j) {
+                double a = o->last_out[bh * d + j];
+                dot += a * oe[j]; na += a * a; nb += oe[j] * oe[j];
+            }
+            double *f = four + bh * 4;
+            f[0] = ne > 0 ? (double)both / ne : 0.0;
+            f[1] = denom > 0.0 ? kept / denom : 0.0;
+            f[2] = (na > 0.0 && nb > 0.0) ? dot / (sqrt(na) * sqrt(nb)) : 0.0;
+            f[3] = o->last_path[bh] == PATH_REUSE && ne > 0 ? (double)covered / ne : -1.0;
+            free(qd); free(oe); free(se);
+        }
     return 0;
 }
 

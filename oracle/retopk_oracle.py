@@ -71,6 +71,8 @@ def _load():
         lib.oracle_stats.restype = None
         lib.oracle_last_step.argtypes = [vp] * 7
         lib.oracle_last_step.restype = None
+        lib.oracle_fidelity.argtypes = [vp, vp, vp, vp, i64, vp]
+        lib.oracle_fidelity.restype = i32
         lib.oracle_last_candidates.argtypes = [vp, i32, vp]
         lib.oracle_last_candidates.restype = i32
         lib.oracle_export_state.argtypes = [vp] * 5
@@ -193,6 +195,21 @@ class Oracle:
         self.lib.oracle_last_step(self.h, _ptr(sup), _ptr(path), _ptr(rho), _ptr(ncand), _ptr(kth),
                                   _ptr(sel))
         return dict(support=sup, path=path, rho_max=rho, n_cand=ncand, kth_score=kth, sel=sel)
+
+    def fidelity(self, q, k, v, seq_len) -> dict:
+        """Fidelity of the step just taken against Exact Top-K on the same inputs (Eq. 2-3, Sec. 4).
+
+        Call right after ``decode_step`` with that step's arguments.  Per (sequence, head):
+        ``support_recall``, ``retained_mass``, ``output_cosine`` and ``coverage`` (of the exact
+        support by the recalled supports, -1 where the step did not reuse).
+        """
+        q, k, v = _u16(q), _u16(k), _u16(v)
+        self._check_kv(k, v)
+        four = np.empty((self.B, self.H_q, 4), dtype=np.float64)
+        if self.lib.oracle_fidelity(self.h, _ptr(q), _ptr(k), _ptr(v), seq_len, _ptr(four)) != 0:
+            raise ValueError("oracle_fidelity failed")
+        return dict(support_recall=four[..., 0], retained_mass=four[..., 1], output_cosine=four[..., 2],
+                    coverage=four[..., 3])
 
     def last_candidates(self, b, h):
         cand = np.empty(self.r * self.K + self.W + 1, dtype=np.int32)

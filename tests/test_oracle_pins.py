@@ -498,3 +498,98 @@ def test_bf16_query_cache_is_off_by_default_and_only_set_on_an_empty_cache(oracl
     o.set_qbar_format(1)
     with pytest.raises(ValueError):
         o.set_qbar_format(2)
+
+
+# ------------------------------------------------------------------ fidelity diagnostics (Eq. 2-3, Sec. 4)
+def test_fidelity_on_the_hand_trace(oracle_mod):
+    """Step 3 of the hand trace keeps {0,2} where the exact support is {1,2}: recall 1/2,
+    coverage 1/2 (the recalled support is {0,2}), retained mass = the logistic weight of key 2
+    against key 1 (q.k = 21 vs 16, d = 2).  Steps 1 and 5 rerank to the exact support."""
+    with open(os.path.join(GOLDEN, "hand_trace.json")) as f:
+        g = json.load(f)
+    p = g["params"]
+    keys = np.array(g["keys"], dtype=np.float32)
+    vals = np.array(g["values"], dtype=np.float32)
+    Lmax = len(keys)
+    k = bits(keys.reshape(1, 1, Lmax, 2))
+    v = bits(vals.reshape(1, 1, Lmax, 2))
+    o = oracle_mod.Oracle(p["B"], p["H_q"], p["H_kv"], p["d"], p["M"], p["r"], p["W"], p["K"],
+                          p["tau"], p["R"], Lmax)
+    seen = {}
+    for t, step in enumerate(g["steps"]):
+        q = bits(np.array(step["q"], dtype=np.float32).reshape(1, 1, 2))
+        o.decode_step(q, k, v, step["L"])
+        seen[t] = {name: float(val[0, 0]) for name, val in o.fidelity(q, k, v, step["L"]).items()}
+    # exact-path steps reproduce Exact Top-K by construction; coverage is only defined on reuse steps
+    for t in (0, 2, 4):
+        assert seen[t]["support_recall"] == 1.0 and seen[t]["retained_mass"] == pytest.approx(1.0, abs=1e-15)
+        assert seen[t]["output_cosine"] == pytest.approx(1.0, abs=1e-15) and seen[t]["coverage"] == -1.0
+    assert seen[1]["support_recall"] == 1.0 and seen[1]["coverage"] == 1.0     # recalled {0,2} = exact {0,2}
+    assert seen[3]["support_recall"] == 0.5 and seen[3]["coverage"] == 0.5
+    assert seen[3]["retained_mass"] == pytest.approx(1.0 / (1.0 + math.exp((16.0 - 21.0) / math.sqrt(2.0))), rel=1e-13)
+    # step 3's output mixes v0, v2 instead of v1, v2: cosine of the two logistic mixes
+    v64 = vals.astype(np.float64)
+    pa = lambda ea, eb: 1.0 / (1.0 + math.exp((eb - ea) / math.sqrt(2.0)))
+    mix = lambda a, b, ea, eb: pa(ea, eb) * v64[a] + (1.0 - pa(ea, eb)) * v64[b]
+    got, exact = mix(0, 2, 12.0, 21.0), mix(1, 2, 16.0, 21.0)
+    assert seen[3]["output_cosine"] == pytest.approx(
+        float(got @ exact / (np.linalg.norm(got) * np.linalg.norm(exact))), rel=1e-12)
+    assert seen[5]["support_recall"] == 1.0 and seen[5]["coverage"] == 1.0     # recalled {1,2} = exact {1,2}
+
+
+def test_fidelity_is_perfect_when_the_window_covers_the_history(oracle_mod):
+    """W >= L: the candidates are every key, rerank recovers the exact support, so recall, mass
+    and cosine are exactly 1; coverage by the recalled supports alone stays a fraction."""
+    cfg = wl.CONFIGS["tiny"].replace(context=300, steps=12, W=400, tau=-2.0, R=0, K=32)
+    st = wl.make_stream(cfg)
+    o = oracle_mod.Oracle.from_config(cfg)
+    for t in range(cfg.steps):
+        o.decode_step(st.q[t], st.k, st.v, st.seq_len(t))
+        f = o.fidelity(st.q[t], st.k, st.v, st.seq_len(t))
+        assert (f["support_recall"] == 1.0).all()
+        np.testing.assert_allclose(f["retained_mass"], 1.0, rtol=0, atol=1e-14)
+        np.testing.assert_allclose(f["output_cosine"], 1.0, rtol=0, atol=1e-14)
+        if t > 0:
+            assert ((f["coverage"] >= 0.0) & (f["coverage"] <= 1.0)).all()
+
+
+def test_fidelity_matches_a_numpy_restatement(oracle_mod):
+    """The four quantities recomputed with numpy set operations from the oracle's own step
+    record (support, recalled slots, cache state before the step) and a brute-force exact support."""
+    cfg = wl.CONFIGS["tiny"].replace(B=2, H_q=4, H_kv=2, context=400, steps=24, K=16, W=8, M=8, r=3, tau=0.5, R=0)
+    st = wl.make_stream(cfg)
+    o = oracle_mod.Oracle.from_config(cfg)
+    G = cfg.H_q // cfg.H_kv
+    saw_reuse = False
+    for t in range(cfg.steps):
+        L = st.seq_len(t)
+        _, sup_before, _, _ = o.export_state()
+        out = o.decode_step(st.q[t], st.k, st.v, L)
+        last = o.last_step()
+        f = o.fidelity(st.q[t], st.k, st.v, L)
+        for b in range(cfg.B):
+            for h in range(cfg.H_q):
+                q64 = wl.bf16_bits_to_f64(st.q[t, b, h])
+                k64 = wl.bf16_bits_to_f64(st.k[b, h // G, :L])
+                v64 = wl.bf16_bits_to_f64(st.v[b, h // G, :L])
+                s_exact, scores = brute_topk(q64, k64, cfg.K)
+                s_got = set(int(x) for x in last["support"][b, h] if x >= 0)
+                w = np.exp(scores[s_exact] - scores[s_exact].max())
+                w /= w.sum()
+                kept = np.array([i in s_got for i in s_exact])
+                assert f["support_recall"][b, h] == pytest.approx(kept.mean(), abs=1e-15)
+                assert f["retained_mass"][b, h] == pytest.approx(float(w[kept].sum()), rel=1e-12, abs=1e-15)
+                o_exact = w @ v64[s_exact]
+                cos = float(out[b, h] @ o_exact / (np.linalg.norm(out[b, h]) * np.linalg.norm(o_exact)))
+                assert f["output_cosine"][b, h] == pytest.approx(cos, rel=1e-12)
+                if last["path"][b, h] == oracle_mod.PATH_REUSE:
+                    saw_reuse = True
+                    union = set()
+                    for c in last["sel"][b, h]:
+                        if c >= 0:
+                            union |= set(int(x) for x in sup_before[b, h, c] if x >= 0)
+                    cov = np.mean([i in union for i in s_exact])
+                    assert f["coverage"][b, h] == pytest.approx(cov, abs=1e-15)
+                else:
+                    assert f["coverage"][b, h] == -1.0
+    assert saw_reuse
