@@ -2,6 +2,8 @@
 """Benchmark of the ReTopK decode step: microseconds per decode step per layer.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--config NAME] [--impl reference]
+    python bench.py --one-layer {reuse,exact,mix} --steps K      (a small case for profiler captures)
+    python bench.py --phases                                     (per-phase SM clocks of the kernels)
 
 One *step* is one ``retopk_decode_step`` call: the whole hot path (recall, candidate
 union, candidate or full-history scoring, Top-K, softmax.V, cache insert) for all
@@ -14,8 +16,13 @@ the same metric through the host-buffer entry point (``e2e``), the library's own
 Top-K on identical inputs, forced pure-reuse and pure-exact passes, the paper-default
 tau = 0.85 mix, the roofline of the dominant kernel and the oracle timed on the host cores.
 
-The path shards over (sequence, head) with no exchange, so ``--gpus N`` runs N independent
-replicas (one process per GPU) and reports the job-wide cost per step.
+Every pass first fills the caches with ``M`` untimed decode calls per layer (the pre-roll), so
+that a short run measures the same steady state as a long one: full caches, the stream's own
+path mix.
+
+The path shards over (sequence, head) with no exchange, so ``--gpus N`` starts N independent
+replicas (one process per GPU, spawned from here unless a launcher already did) and reports
+the job-wide cost per step.
 """
 from __future__ import annotations
 
@@ -111,8 +118,9 @@ class ClockSampler:
 class Layers:
     """Device-resident inputs and contexts of the rotating layers, plus raw-pointer calls."""
 
-    def __init__(self, cfg, n_layers, t_per_layer, rank, torch, rt):
+    def __init__(self, cfg, n_layers, t_per_layer, rank, torch, rt, preroll=0):
         self.cfg, self.n, self.T = cfg, n_layers, t_per_layer
+        self.preroll = preroll               # decode steps per layer that only fill the caches
         self.torch, self.rt, self.lib = torch, rt, rt.load()
         self.streams = [wl.make_stream(cfg, steps=t_per_layer, layer=l + 10 * rank) for l in range(n_layers)]
         self.k = [rt.bf16_tensor_from_bits(s.k, device="cuda") for s in self.streams]
@@ -155,9 +163,18 @@ class Layers:
                 tot[key] = (tot.get(key, 0) | val) if key == "status" else tot.get(key, 0) + val
         return tot
 
+    def fill_caches(self, stream):
+        """The pre-roll: ``preroll`` ReTopK decode calls per layer from an empty cache (untimed)."""
+        for c in self.ctx:
+            c.reset()
+        for i in range(self.preroll * self.n):
+            self.call(i - self.preroll * self.n, "retopk", stream)
+
     def call(self, i, kind, stream, single=False):
-        """Call number i of a pass: layer i % n at decode offset i // n (single: layer 0 at offset i)."""
-        l, t = (0, i) if single else (i % self.n, i // self.n)
+        """Call number i of a pass: layer i % n at decode offset preroll + i // n (single: layer 0
+        at offset preroll + i); negative i are the pre-roll calls."""
+        i += self.preroll * self.n
+        l, t = (0, i - self.preroll * (self.n - 1)) if single and i >= self.preroll * self.n else (i % self.n, i // self.n)
         L = self.cfg.context + t + 1
         h = self.ctx[l].h
         qstep = self.cfg.B * self.cfg.H_q * self.cfg.d * 2
@@ -185,15 +202,15 @@ def sync_all(torch, dist):
 
 
 def timed_pass(layers, kind, warmup, steps, torch, dist, profile=False, sampler=None, per_step=False, single=False):
-    """Reset, run `warmup` untimed calls, then time exactly `steps` calls with CUDA events.
+    """Fill the caches (pre-roll), run `warmup` untimed calls, then time exactly `steps` calls
+    with CUDA events.
 
     per_step: also record an event after every call and return the distribution of the intervals
     (the extra stream entries keep consecutive calls from overlapping their launches, so these are
     a little longer than the pass average).  single: every call goes to layer 0 (hot L2).
     """
     stream = torch.cuda.current_stream().cuda_stream
-    for c in layers.ctx:
-        c.reset()
+    layers.fill_caches(stream)
     for i in range(warmup):
         layers.call(i, kind, stream, single)
     sync_all(torch, dist)
@@ -246,10 +263,13 @@ def algorithmic_bytes(cfg, stats, mean_L, mean_fill):
     heads = stats["steps"]
     n_sel = min(cfg.r, mean_fill)
     tail = K * d * 2 + K * 4 + d * 2          # value rows, support insert, output
+    exact_heads = heads - stats["reuse"]
     recall = heads * (mean_fill * d * QBAR_BYTES + d * QBAR_BYTES + d * 2)
     scan = stats["scan_groups"] * mean_L * d * 2
-    finish = heads * tail + stats["reuse"] * (n_sel * K * 4 + d * 2) + stats["cand_sum"] * d * 2
-    return dict(recall=recall, scan=scan, finish=finish)
+    # step kernel: the recall stage of every head plus the whole reuse path of the heads that reuse
+    step = recall + stats["reuse"] * (tail + n_sel * K * 4) + stats["cand_sum"] * d * 2
+    finish = exact_heads * (tail + d * 2)
+    return dict(step=step, scan=scan, finish=finish)
 
 
 def path_mix(stats):
@@ -258,65 +278,80 @@ def path_mix(stats):
         "mean_candidates": round(stats["cand_sum"] / max(stats["reuse"], 1), 1)}
 
 
-def fidelity_pass(layers, torch, calls=96):
-    """ReTopK against Exact Top-K on the same inputs: the paper's fidelity quantities.
+def fidelity_of_step(torch, q, k_cache, idx_exact, out_exact, out_retopk, support, path, cached_supports=None, sel=None):
+    """The paper's fidelity quantities for one step, per (sequence, head), from what the library
+    returned for ReTopK and for its own Exact Top-K on identical inputs (a diagnostic: torch only
+    compares index sets and outputs and re-weighs the exact support).
 
-    A diagnostic outside every timed region (torch only compares index sets, outputs and
-    re-weighs the exact support): after each ReTopK call the library's Exact Top-K runs on the
-    identical inputs.  Per head-step: support recall |S_retopk & S_exact| / K, retained mass (share
-    of the softmax weight over the exact support that lies on keys ReTopK kept), output cosine,
-    and Eq. 3's coverage |S_exact & U| / K of the exact support by the union U of the recalled
-    cached supports (without the recent window).
+    q [B,H_q,d], k_cache [B,H_kv,L_max,d] bf16; idx_exact / support [B,H_q,K] int32 (-1 padded);
+    out_* [B,H_q,d]; path [B,H_q]; cached_supports [B,H_q,M,K] as they were BEFORE the step and
+    sel [B,H_q,r] the recalled slots, for Eq. 3's coverage (omitted: coverage is not computed).
+    Returns support_recall |S^ & S| / |S|, retained_mass (share of the softmax weight over the
+    exact support that lies on keys ReTopK kept), output_cosine, and coverage |S & U| / |S| by
+    the union U of the recalled supports (-1 where the head did not reuse).
     """
-    cfg = layers.cfg
-    stream = torch.cuda.current_stream().cuda_stream
-    for c in layers.ctx:
-        c.reset()
-    idx = torch.empty((cfg.B, cfg.H_q, cfg.K), dtype=torch.int32, device="cuda")
-    out_exact = torch.empty_like(layers.out)
-    qstep = cfg.B * cfg.H_q * cfg.d * 2
-    G = cfg.H_q // cfg.H_kv
-    recalls, cosines, cos_reuse, masses, mass_reuse, coverages = [], [], [], [], [], []
+    B, H_q, K = idx_exact.shape
+    H_kv, d = k_cache.shape[1], k_cache.shape[3]
+    G = H_q // H_kv
 
     def member(a, b):          # per head: which entries of a [.., n] occur in b [.., m]
         return (a.unsqueeze(-1) == b.unsqueeze(-2)).any(-1)
 
+    valid = idx_exact >= 0
+    n_exact = valid.sum(-1).clamp_min(1).float()
+    in_both = member(idx_exact, support) & valid
+    recall = in_both.sum(-1).float() / n_exact
+    # softmax over the exact support, recomputed here from the key rows
+    kv_head = torch.arange(H_q, device=q.device) // G
+    group = torch.arange(B, device=q.device).view(-1, 1, 1) * H_kv + kv_head.view(1, -1, 1)
+    row_id = group * k_cache.shape[2] + idx_exact.long().clamp_min(0)
+    keys = k_cache.reshape(-1, d)[row_id.flatten()].view(B, H_q, K, d).float()
+    e = (keys * q.float().unsqueeze(-2)).sum(-1) / d ** 0.5
+    w = torch.softmax(e.masked_fill(~valid, float("-inf")), dim=-1)
+    mass = (w * in_both).sum(-1)
+    a, b = out_retopk.float(), out_exact.float()
+    cos = (a * b).sum(-1) / (a.norm(dim=-1) * b.norm(dim=-1)).clamp_min(1e-20)
+    res = {"support_recall": recall, "retained_mass": mass, "output_cosine": cos}
+    if cached_supports is not None and sel is not None:
+        sel = sel.long()                                       # [B, H_q, r], -1 padded
+        picked = torch.gather(cached_supports, 2, sel.clamp_min(0).unsqueeze(-1).expand(-1, -1, -1, K))
+        picked = picked.masked_fill((sel < 0).unsqueeze(-1), -2).flatten(2)     # [B, H_q, r*K]
+        cov = torch.stack([(member(idx_exact[bb], picked[bb]) & valid[bb]).sum(-1).float() / n_exact[bb] for bb in range(B)])
+        res["coverage"] = torch.where(path == 0, cov, torch.full_like(cov, -1.0))
+    return res
+
+
+def fidelity_pass(layers, torch, calls=96):
+    """ReTopK against Exact Top-K on the same inputs over the first decode calls of a run (caches
+    filled by the pre-roll): means of fidelity_of_step's quantities, outside every timed region."""
+    cfg = layers.cfg
+    stream = torch.cuda.current_stream().cuda_stream
+    layers.fill_caches(stream)
+    idx = torch.empty((cfg.B, cfg.H_q, cfg.K), dtype=torch.int32, device="cuda")
+    out_exact = torch.empty_like(layers.out)
+    qstep = cfg.B * cfg.H_q * cfg.d * 2
+    recalls, cosines, cos_reuse, masses, mass_reuse, coverages = [], [], [], [], [], []
     for i in range(calls):
-        l, t = i % layers.n, i // layers.n
+        l, t = i % layers.n, layers.preroll + i // layers.n
         L = cfg.context + t + 1
         ctx = layers.ctx[l]
-        cached = ctx.export_state()[1] if t > 0 else None          # supports before this step's insert
+        cached = ctx.export_state()[1]                             # supports before this step's insert
         layers.call(i, "retopk", stream)
         last = ctx.last_step()
         rc = layers.lib.exact_topk_decode(ctx.h, layers.q[l].data_ptr() + t * qstep, layers.k[l].data_ptr(),
                                           layers.v[l].data_ptr(), L, out_exact.data_ptr(), idx.data_ptr(), stream)
         if rc != 0:
             raise RuntimeError(f"exact_topk_decode failed with {rc}")
+        f = fidelity_of_step(torch, layers.q[l][t], layers.k[l], idx, out_exact, layers.out, last["support"], last["path"],
+                             cached, ctx.last_recall())
         reuse = last["path"] == 0
-        in_both = member(idx, last["support"])                     # [B, H_q, K] over the exact support
-        hit = in_both.sum(-1).float() / cfg.K
-        # softmax over the exact support, recomputed here from the key rows
-        kv_head = torch.arange(cfg.H_q, device="cuda") // G
-        group = torch.arange(cfg.B, device="cuda").view(-1, 1, 1) * cfg.H_kv + kv_head.view(1, -1, 1)
-        row_id = group * layers.k[l].shape[2] + idx.long().clamp_min(0)
-        keys = layers.k[l].view(-1, cfg.d)[row_id.flatten()].view(cfg.B, cfg.H_q, cfg.K, cfg.d).float()
-        e = (keys * layers.q[l][t].float().unsqueeze(-2)).sum(-1) / cfg.d ** 0.5
-        w = torch.softmax(e.masked_fill(idx < 0, float("-inf")), dim=-1)
-        mass = (w * in_both).sum(-1)
-        a, b = layers.out.float(), out_exact.float()
-        cos = (a * b).sum(-1) / (a.norm(dim=-1) * b.norm(dim=-1)).clamp_min(1e-20)
-        cosines.append(cos.flatten())
-        masses.append(mass.flatten())
+        cosines.append(f["output_cosine"].flatten())
+        masses.append(f["retained_mass"].flatten())
         if reuse.any():
-            recalls.append(hit[reuse])
-            cos_reuse.append(cos[reuse])
-            mass_reuse.append(mass[reuse])
-            if cached is not None:
-                sel = ctx.last_recall().long()                     # [B, H_q, r], -1 padded
-                picked = torch.gather(cached, 2, sel.clamp_min(0).unsqueeze(-1).expand(-1, -1, -1, cfg.K))
-                picked = picked.masked_fill((sel < 0).unsqueeze(-1), -1).flatten(2)     # [B, H_q, r*K]
-                cov = torch.stack([member(idx[bb], picked[bb]).sum(-1).float() / cfg.K for bb in range(cfg.B)])
-                coverages.append(cov[reuse])
+            recalls.append(f["support_recall"][reuse])
+            cos_reuse.append(f["output_cosine"][reuse])
+            mass_reuse.append(f["retained_mass"][reuse])
+            coverages.append(f["coverage"][reuse])
     cat = lambda xs: torch.cat(xs) if xs else torch.zeros(1, device="cuda")
     rnd = lambda x, n=4: round(float(x), n)
     return {"calls": calls, "support_recall_on_reuse_heads": rnd(cat(recalls).mean()),
@@ -389,19 +424,23 @@ def run_gpu(args):
     cfg = wl.CONFIGS[args.config]
     W, K = args.warmup, args.steps
     n_layers = args.layers
-    t_per_layer = -(-(W + K) // n_layers)
+    preroll = cfg.M if args.preroll is None else args.preroll       # untimed calls per layer that fill the caches
+    t_timed = -(-(W + K) // n_layers)
+    t_per_layer = preroll + t_timed
     if t_per_layer > cfg.steps:      # a longer run than the configuration's: extend the KV layout
         cfg = cfg.replace(steps=t_per_layer)
-    layers = Layers(cfg, n_layers, t_per_layer, rank, torch, rt)
+    layers = Layers(cfg, n_layers, t_per_layer, rank, torch, rt, preroll=preroll)
     layers.qbar_bf16 = args.qbar_bf16
     layers.cluster = args.cluster
     layers.finish_threads = args.finish_threads
     global QBAR_BYTES
     QBAR_BYTES = 2 if args.qbar_bf16 else 4
     peak, peak_kind = measured_peaks()
-    mean_t = (W + K / 2) / n_layers
+    mean_t = preroll + (W + K / 2) / n_layers
     mean_L = cfg.context + mean_t + 1
     mean_fill = min(cfg.M, mean_t)
+    fill_first = min(cfg.M, preroll + W // n_layers)
+    fill_last = min(cfg.M, preroll + (W + K - 1) // n_layers)
 
     # headline: configured tau / R, device-resident inputs
     layers.make_contexts()
@@ -413,12 +452,13 @@ def run_gpu(args):
     e2e = timed_pass(layers, "host", W, K, torch, dist)
     # the library's own Exact Top-K on identical inputs
     exact = timed_pass(layers, "exact", W, K, torch, dist)
+    exact_p = timed_pass(layers, "exact", W, K, torch, dist, profile=True)
     # forced paths and the paper-default threshold
     layers.make_contexts(tau=-2.0, R=0)
     reuse = timed_pass(layers, "retopk", W, K, torch, dist)
     reuse_d = timed_pass(layers, "retopk", W, K, torch, dist, per_step=True)
     # one layer only: candidate rows and caches of the step before are still in L2
-    n_hot = min(t_per_layer, W + K)
+    n_hot = min(t_timed, W + K)
     w_hot = min(W, n_hot // 4)
     reuse_hot = timed_pass(layers, "retopk", w_hot, n_hot - w_hot, torch, dist, single=True)
     layers.make_contexts(tau=2.0, R=0)
@@ -432,26 +472,21 @@ def run_gpu(args):
     fidelity = fidelity_pass(layers, torch, calls=min(96, W + K)) if rank == 0 else None
     ladder = fusion_ladder(layers, W, K, torch, dist) if args.ladder else None
 
-    # roofline of the dominant kernel of the headline pass
-    abytes = algorithmic_bytes(cfg, prof["stats"], mean_L, mean_fill)
-    total_ms = sum(r["ms"] for r in prof["prof"].values())
-    kernels = {}
-    for name, rec in prof["prof"].items():
-        gbs = abytes[name] / (rec["ms"] * 1e-3) / 1e9 if rec["ms"] > 0 else 0.0
-        kernels[name] = {"launches": rec["launches"], "avg_us": round(1e3 * rec["ms"] / max(rec["launches"], 1), 2),
-                         "share": round(rec["ms"] / total_ms, 4),
-                         "alg_bytes_per_launch": int(abytes[name] / max(rec["launches"], 1)),
-                         "GBps": round(gbs, 1), "frac": round(gbs / peak, 4)}
-    top = max(kernels, key=lambda n: kernels[n]["share"])
-    roofline = {"bound": "hbm", "kernel": top + "_kernel", "achieved": kernels[top]["GBps"], "peak": peak,
-                "peak_kind": peak_kind, "unit": "GB/s", "frac": kernels[top]["frac"],
-                "frac_of_8TBps": round(kernels[top]["GBps"] / 8000.0, 4),
-                "traffic": (int(NCU_TRAFFIC_PER_GROUP[args.config] * prof["stats"]["scan_groups"] / prof["prof"]["scan"]["launches"])
-                            if top == "scan" and args.config in NCU_TRAFFIC_PER_GROUP else None),
-                "traffic_source": "ncu capture of a one-layer run of this workload (summary under profiles/), scaled by scanned groups per launch",
-                "kernels": kernels}
+    def kernel_table(res):
+        """Per kernel of a profiled pass: launches, average time, share, algorithmic GB/s."""
+        b = algorithmic_bytes(cfg, res["stats"], mean_L, mean_fill)
+        total_ms = sum(r["ms"] for r in res["prof"].values())
+        table = {}
+        for name, rec in res["prof"].items():
+            gbs = b[name] / (rec["ms"] * 1e-3) / 1e9 if rec["ms"] > 0 else 0.0
+            table[name] = {"launches": rec["launches"], "avg_us": round(1e3 * rec["ms"] / max(rec["launches"], 1), 2),
+                           "share": round(rec["ms"] / total_ms, 4) if total_ms > 0 else 0.0,
+                           "alg_bytes_per_launch": int(b[name] / max(rec["launches"], 1)),
+                           "GBps": round(gbs, 1), "frac": round(gbs / peak, 4)}
+        return table
 
-    def path_report(res, exact_like):
+    def path_report(res):
+        """A whole pass: time per step and the HBM fraction on the algorithmic bytes of ALL its kernels."""
         st = res["stats"]
         b = algorithmic_bytes(cfg, st, mean_L, mean_fill)
         tot = sum(b.values())
@@ -459,6 +494,28 @@ def run_gpu(args):
         return {"us_per_step": round(res["us_per_step"], 2), "alg_bytes_per_step": int(tot / K),
                 "GBps": round(gbs, 1), "frac_of_measured": round(gbs / peak, 4),
                 "frac_of_8TBps": round(gbs / 8000.0, 4), "mix": path_mix(st)}
+
+    # roofline: the dominant kernel of the headline pass by CUDA-event time, and beside it the
+    # step as a whole (every kernel's algorithmic bytes over the pass time) for every pass
+    kernels = kernel_table(prof)
+    top = max(kernels, key=lambda n: kernels[n]["share"])
+    step_head = path_report(head)
+    paths = {"configured_tau": step_head, "pure_reuse": path_report(reuse), "pure_exact": path_report(fallb),
+             "tau_0.85": path_report(paper) | {"kernel_avg_us": {
+                 name: round(1e3 * rec["ms"] / max(rec["launches"], 1), 2) for name, rec in paper_p["prof"].items()}}}
+    roofline = {"bound": "hbm", "kernel": top + "_kernel", "achieved": kernels[top]["GBps"], "peak": peak,
+                "peak_kind": peak_kind, "unit": "GB/s", "frac": kernels[top]["frac"],
+                "frac_of_8TBps": round(kernels[top]["GBps"] / 8000.0, 4),
+                "traffic": (int(NCU_TRAFFIC_PER_GROUP[args.config] * prof["stats"]["scan_groups"] / prof["prof"]["scan"]["launches"])
+                            if top == "scan" and args.config in NCU_TRAFFIC_PER_GROUP else None),
+                "traffic_source": "ncu capture of a one-layer run of this workload (summary under profiles/), scaled by scanned groups per launch",
+                "kernels": kernels,
+                "step": {"note": "whole decode step: algorithmic bytes of all three kernels over the pass time",
+                         "achieved": step_head["GBps"], "frac": step_head["frac_of_measured"],
+                         "frac_of_8TBps": step_head["frac_of_8TBps"]},
+                "paths": {name: {"achieved": rep["GBps"], "frac": rep["frac_of_measured"], "frac_of_8TBps": rep["frac_of_8TBps"],
+                                 "us_per_step": rep["us_per_step"]} for name, rep in paths.items()},
+                "exact_topk_kernels": {name: rec for name, rec in kernel_table(exact_p).items() if name != "step"}}
 
     exact_bytes = (cfg.B * cfg.H_kv * mean_L * cfg.d * 2 + cfg.B * cfg.H_q * cfg.K * cfg.d * 2) * K
     exact_gbs = exact_bytes / (exact["ms"] * 1e-3) / 1e9
@@ -471,7 +528,10 @@ def run_gpu(args):
         "config": {"workload": cfg.name, "B": cfg.B, "H_q": cfg.H_q, "H_kv": cfg.H_kv, "d": cfg.d,
                    "context": cfg.context, "K": cfg.K, "M": cfg.M, "r": cfg.r, "W": cfg.W, "tau": cfg.tau,
                    "R": cfg.R, "qbar_cache": "bf16" if args.qbar_bf16 else "fp32",
-                   "finish_ctas_per_head": args.cluster or "auto", "finish_threads": args.finish_threads or "auto", "layers_rotated": n_layers, "decode_steps_per_layer": t_per_layer,
+                   "ctas_per_head": args.cluster or "auto", "threads_per_cta": args.finish_threads or "auto",
+                   "layers_rotated": n_layers, "decode_steps_per_layer": t_per_layer,
+                   "preroll_steps_per_layer": preroll, "cache_fill_at_first_timed_call": fill_first,
+                   "cache_fill_at_last_timed_call": fill_last,
                    "l2": "inputs larger than L2: calls rotate over independent layers",
                    "parallelism": "replicas only" if world > 1 else "single GPU"},
         "clocks": sampler.summary(),
@@ -487,9 +547,12 @@ def run_gpu(args):
         "speedup_vs_exact_topk": {"configured_tau": round(exact["us_per_step"] / head["us_per_step"], 3),
                                   "tau_0.85": round(exact["us_per_step"] / paper["us_per_step"], 3),
                                   "pure_reuse": round(exact["us_per_step"] / reuse["us_per_step"], 3)},
-        "paths": {"pure_reuse": path_report(reuse, False), "pure_exact": path_report(fallb, True),
-                  "tau_0.85": path_report(paper, False) | {"kernel_avg_us": {
-                      name: round(1e3 * rec["ms"] / max(rec["launches"], 1), 2) for name, rec in paper_p["prof"].items()}}},
+        "targets": {"note": "north-star targets: >= 0.60 of the 8 TB/s HBM roofline on the bytes the step touches and "
+                            ">= 3x over this library's Exact Top-K",
+                    "frac_of_8TBps_configured_tau": step_head["frac_of_8TBps"],
+                    "speedup_configured_tau": round(exact["us_per_step"] / head["us_per_step"], 3),
+                    "met_at_configured_tau": bool(step_head["frac_of_8TBps"] >= 0.6 and exact["us_per_step"] / head["us_per_step"] >= 3.0)},
+        "paths": paths,
         "per_step_us": {"note": "an event after every call (calls then do not overlap their launches)",
                         "pure_reuse": reuse_d["dist_us"], "pure_exact": fallb_d["dist_us"], "tau_0.85": paper_d["dist_us"]},
         "single_layer_hot_l2_us": {"note": "every call on layer 0: the step before left its rows in L2; not the headline",
@@ -509,6 +572,114 @@ def run_gpu(args):
     if dist is not None:
         dist.barrier()
         dist.destroy_process_group()
+
+
+# --------------------------------------------------------------------------- small cases for profilers
+def run_one_layer(args):
+    """A few decode steps of ONE layer (KV of a few GB at most) for profiler captures of single kernels.
+
+    ``--one-layer reuse``: tau = -2, every head reuses after the first step; ``exact``: tau = 2,
+    every head takes the full-history path; ``mix``: the configuration's own tau and refresh
+    period.  A buffer larger than L2 is rewritten between steps so the key rows come from HBM
+    as they do in the benchmark's layer rotation.  ``--preroll`` steps come first (default 16).
+    """
+    import torch
+    from paper_2607_27692_b200 import build, retopk as rt
+    build.build()
+    cfg = wl.CONFIGS[args.config]
+    pre = 16 if args.preroll is None else args.preroll
+    steps = pre + (args.steps or 6)
+    if steps > cfg.steps:
+        cfg = cfg.replace(steps=steps)
+    st = wl.make_stream(cfg, steps=steps)
+    k = rt.bf16_tensor_from_bits(st.k, device="cuda")
+    v = rt.bf16_tensor_from_bits(st.v, device="cuda")
+    q = rt.bf16_tensor_from_bits(st.q, device="cuda")
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    override = {"reuse": dict(tau=-2.0, R=0), "exact": dict(tau=2.0, R=0), "mix": {}}[args.one_layer]
+    ctx = rt.ReTopK.from_config(cfg, **override)
+    if args.qbar_bf16:
+        ctx.set_qbar_format(1)
+    if args.cluster:
+        ctx.set_cluster_size(args.cluster)
+    if args.finish_threads:
+        ctx.set_finish_threads(args.finish_threads)
+    for t in range(steps):
+        flush.zero_()
+        ctx.decode_step(q[t], k, v, st.seq_len(t))
+    torch.cuda.synchronize()
+    print(json.dumps({"one_layer": args.one_layer, "workload": cfg.name, "steps": steps, "stats": ctx.stats()}), flush=True)
+
+
+PHASES = {
+    "recall stage (every head)": (1, [(0, 1, "similarities (Eq. 6) + window rows requested"), (1, 2, "Top-r, decision, records (Eq. 7, Eq. 13)")]),
+    "reuse path": (0, [(0, 1, "first lists requested + window rows scored"), (1, 2, "bitmap marked (Eq. 8-9)"),
+                       (2, 3, "ordered extraction"), (3, 4, "candidate rows gathered and scored (Eq. 10)"),
+                       (4, 5, "Top-K (Eq. 11)"), (5, 6, "softmax.V, inserts (Eq. 12)")]),
+    "exact finish": (2, [(0, 1, "bound from the tile maxima"), (1, 2, "hit-tile list"), (2, 3, "read-back of hit tiles"),
+                         (3, 4, "Top-K (Eq. 1)"), (4, 5, "softmax.V, insert (Eq. 12)")]),
+}
+
+
+def run_phases(args):
+    """Per-phase SM clock cycles of the kernels (thread 0 of every CTA stamps clock64 at phase
+    boundaries).  Builds a variant of the library with -DRETOPK_PHASE_CLOCKS into a temporary
+    directory, runs one layer of the workload in forced pure-reuse and pure-exact mode with L2
+    flushed between steps, and prints the mean over heads and steps.  A measurement aid: the
+    stamps cost a little, so these are not benchmark numbers."""
+    import subprocess
+    import tempfile
+    import torch
+    from paper_2607_27692_b200 import build, retopk as rt
+    tmp = tempfile.mkdtemp(prefix="retopk_phases_")
+    lib = os.path.join(tmp, "libretopk_phases.so")
+    units = [os.path.join(build.SRC_DIR, f) for f in sorted(os.listdir(build.SRC_DIR)) if f.endswith(".cu")]
+    subprocess.run([build.find_nvcc()] + build.NVCC_FLAGS + ["-DRETOPK_PHASE_CLOCKS", "-o", lib] + units, check=True)
+    rt.library_path = lambda: lib
+    L = rt.load()
+    L.retopk_debug_read_phases.argtypes = [C.c_void_p]
+    L.retopk_debug_read_phases.restype = C.c_int
+    cfg = wl.CONFIGS[args.config]
+    pre = min(cfg.M, 48) if args.preroll is None else args.preroll
+    n_meas = args.steps or 24
+    steps = pre + n_meas
+    if steps > cfg.steps:
+        cfg = cfg.replace(steps=steps)
+    st = wl.make_stream(cfg, steps=steps)
+    k = rt.bf16_tensor_from_bits(st.k, device="cuda")
+    v = rt.bf16_tensor_from_bits(st.v, device="cuda")
+    q = rt.bf16_tensor_from_bits(st.q, device="cuda")
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    nh = min(cfg.B * cfg.H_q, 1024)
+    SLOTS = 24
+    out = {"workload": cfg.name, "steps_measured": n_meas, "cache_fill": min(cfg.M, pre), "unit": "SM clock cycles, mean over heads and steps"}
+    for label, override, tables in (("pure_reuse", dict(tau=-2.0, R=0), ("recall stage (every head)", "reuse path")),
+                                    ("pure_exact", dict(tau=2.0, R=0), ("recall stage (every head)", "exact finish"))):
+        ctx = rt.ReTopK.from_config(cfg, **override)
+        if args.cluster:
+            ctx.set_cluster_size(args.cluster)
+        if args.finish_threads:
+            ctx.set_finish_threads(args.finish_threads)
+        acc = {name: [] for name in tables}
+        for t in range(steps):
+            flush.zero_()
+            ctx.decode_step(q[t], k, v, st.seq_len(t))
+            if t >= pre:
+                buf = np.zeros((3, 1024, SLOTS), dtype=np.int64)
+                if L.retopk_debug_read_phases(buf.ctypes.data) != 0:
+                    raise RuntimeError("retopk_debug_read_phases failed")
+                for name in tables:
+                    acc[name].append(buf[PHASES[name][0], :nh].copy())
+        rep = {}
+        for name in tables:
+            x = np.array(acc[name]).astype(np.float64)
+            rows = {what: round(float((x[..., b] - x[..., a]).mean())) for a, b, what in PHASES[name][1]}
+            first, last = PHASES[name][1][0][0], PHASES[name][1][-1][1]
+            rows["total"] = round(float((x[..., last] - x[..., first]).mean()))
+            rep[name] = rows
+        out[label] = rep
+        ctx.close()
+    print(json.dumps(out, indent=1), flush=True)
 
 
 # DRAM traffic of scan_kernel per scanned KV group (dram__bytes_read.sum + dram__bytes_write.sum
@@ -570,13 +741,15 @@ def run_reference(args):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--gpus", type=int, default=1, help="replicas, one process per GPU (spawned here unless a launcher set RANK/WORLD_SIZE)")
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--preroll", type=int, default=None,
+                    help="untimed decode calls per layer that fill the caches before every pass (default: M)")
     ap.add_argument("--cluster", type=int, default=0, choices=[0, 1, 2, 4, 8],
-                    help="CTAs per head in the finish kernel (0: the library's own choice)")
+                    help="CTAs per head in the per-head kernels (0: the library's own choice)")
     ap.add_argument("--finish-threads", type=int, default=0, choices=[0, 512, 1024],
-                    help="block shape of the finish kernel (0: the library's own choice)")
+                    help="block shape of the per-head kernels (0: the library's own choice)")
     ap.add_argument("--qbar-bf16", action="store_true",
                     help="keep the cached normalised queries in bf16 (storage variant) in every pass")
     ap.add_argument("--ladder", action="store_true",
@@ -585,15 +758,29 @@ def main():
     ap.add_argument("--layers", type=int, default=4, help="independent layers rotated over (L2 hygiene)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--one-layer", default=None, choices=["reuse", "exact", "mix"],
+                    help="run --steps decode steps of one layer in the given mode and exit (for profiler captures)")
+    ap.add_argument("--phases", action="store_true",
+                    help="build a phase-clock variant of the library and print per-phase cycles of the kernels")
     args = ap.parse_args()
     if args.impl == "reference":
         args.steps = 32 if args.steps is None else args.steps
         args.warmup = 3 if args.warmup is None else args.warmup
         run_reference(args)
-    else:
-        args.steps = 1024 if args.steps is None else args.steps
-        args.warmup = 64 if args.warmup is None else args.warmup
-        run_gpu(args)
+        return
+    if args.one_layer:
+        run_one_layer(args)
+        return
+    if args.phases:
+        run_phases(args)
+        return
+    args.steps = 1024 if args.steps is None else args.steps
+    args.warmup = 64 if args.warmup is None else args.warmup
+    from paper_2607_27692_b200 import replicas
+    if args.gpus > 1 and not replicas.under_launcher():
+        # no launcher around: start the replicas from here, one process per GPU
+        sys.exit(replicas.spawn([sys.executable, os.path.abspath(__file__)] + sys.argv[1:], args.gpus))
+    run_gpu(args)
 
 
 if __name__ == "__main__":

@@ -16,7 +16,8 @@
  *
  * Conventions shared by every call
  *   - All tensor pointers are DEVICE pointers on the device that was current at
- *     retopk_create time, unless the argument name ends in _host.
+ *     retopk_create time, unless the argument name ends in _host.  Calls that enqueue work
+ *     return RETOPK_EINVAL when another device is current.
  *   - bf16 tensors are raw 16-bit patterns, innermost dimension d contiguous:
  *       q, out           [B, H_q, d]
  *       k_cache, v_cache [B, H_kv, max_seq_len, d]
@@ -116,19 +117,20 @@ enum { RETOPK_QBAR_FP32 = 0, RETOPK_QBAR_BF16 = 1 };
 int retopk_set_qbar_format(retopk_ctx* ctx, int format);
 
 /*
- * CTAs per (sequence, query head) in the finish kernel: 1, 2, 4 or 8.  With more than one, the
+ * CTAs per (sequence, query head) in the per-head kernels: 1, 2, 4 or 8.  With more than one, the
  * CTAs of a head form a thread-block cluster on as many SMs: each scores a share of the
  * candidate rows (Eq. 10) and fetches a share of the selected value rows (Eq. 12); keys and
  * partial sums cross through distributed shared memory.  The paper has no counterpart; it is
  * how a small batch uses the SMs that one CTA per head would leave idle.  retopk_create*
  * picks the largest size with B*H_q*size <= the SM count (1 from B*H_q = 75 up on B200).
  * Supports and decisions do not depend on the size; outputs differ in the last bits of the
- * fp32 sum order.  EINVAL for any other size.
+ * fp32 sum order.  EINVAL for any other size; EUNSUPPORTED when the device cannot schedule a
+ * cluster of that size for this context's kernels (checked here, not in the middle of a step).
  */
 int retopk_set_cluster_size(retopk_ctx* ctx, int ctas_per_head);
 
 /*
- * Block shape of the finish kernel: 1024 threads (one CTA per SM) or 512 (two CTAs per SM,
+ * Block shape of the per-head kernels: 1024 threads (one CTA per SM) or 512 (two CTAs per SM,
  * each with half of the SM's shared memory, so that the selection of one head overlaps the
  * row copies of another).  retopk_create* picks 512 when there are more heads than SMs and
  * the shape fits.  Results do not depend on the number of CTAs per SM; outputs differ between
@@ -170,14 +172,19 @@ int retopk_reset(retopk_ctx* ctx, void* stream);
  * One ReTopK decode step (Sec. 3.3-3.4: Eq. 6-13 and the cache insert) for all B * H_q
  * heads.  q, k_cache, v_cache are read, out is written; 1 <= seq_len <= max_seq_len.
  * The path of each head is decided on the device; no host synchronisation happens.
- * Advances t_dec and the insert count by one.
+ * Advances t_dec and the insert count by one.  Three launches: the per-head step kernel
+ * (recall, decision, and the whole reuse path of the heads that reuse), the full-history
+ * scan of the flagged KV groups, and the finish of the heads on the exact path; the last two
+ * leave at once when no head fell back.  If a launch fails after the first kernel of the step
+ * was enqueued, the caches are half advanced: the call returns RETOPK_ECUDA and so does every
+ * later step of this context until retopk_reset.
  */
 int retopk_decode_step(retopk_ctx* ctx, const void* q, const void* k_cache, const void* v_cache,
                        int64_t seq_len, void* out, void* stream);
 
 /*
- * Seed the caches from the end of the prompt (Sec. 3.3: the cache "is initialized from the
- * final C prompt tokens during prefill").  q_tail [n_tail,B,H_q,d] (device) holds the queries
+ * Seed the caches from the end of the prompt (Sec. 3.3, cache paragraph: the cache starts
+ * from the last C prompt tokens).  q_tail [n_tail,B,H_q,d] (device) holds the queries
  * of prompt positions prompt_len - n_tail .. prompt_len - 1, oldest first; k_cache / v_cache
  * hold the prompt's keys and values.  Entry j gets the normalised query of its position p and
  * the CAUSAL Exact Top-K support over keys 0..p (Eq. 1 with L = p + 1; the paper leaves the
@@ -231,6 +238,25 @@ int retopk_last_step(retopk_ctx* ctx, int32_t* support, uint8_t* path, float* rh
 int retopk_last_recall(retopk_ctx* ctx, int32_t* sel, void* stream);
 
 /*
+ * Test hook (no counterpart in the paper): keep the candidate list A_t (Eq. 9) of every head
+ * that reuses, so that a test can compare it element by element.  enable = 1 allocates a
+ * buffer of B*H_q*(r*K+W) int32 (ENOMEM), enable = 0 frees it; both synchronise the device.
+ * While it is off (the default) the step kernel writes nothing extra.
+ * retopk_last_candidates copies the buffer to cand [B,H_q,r*K+W] (device pointer): for a head
+ * on the reuse path in the most recent step, its first n_cand entries (retopk_last_step) are
+ * the list in ascending order; other rows are stale.  EINVAL while the hook is off.
+ */
+int retopk_debug_candidates(retopk_ctx* ctx, int enable);
+int retopk_last_candidates(retopk_ctx* ctx, int32_t* cand, void* stream);
+
+/*
+ * Test hook (host side only; nothing on the device fails): the next launch of kernel `which`
+ * (1: step, 2: scan, 3: exact finish; 0 clears the request) is skipped and reported as a failed
+ * launch, so that the error handling of retopk_decode_step can be exercised.
+ */
+int retopk_debug_fail_next_launch(retopk_ctx* ctx, int which);
+
+/*
  * Cache state out / in (device pointers): qbar [B,H_q,M,d] float32 normalised queries,
  * supports [B,H_q,M,K] int32 (ascending, -1 padded); the entry inserted n-th sits in slot
  * n % M.  n_inserted and t_dec are host scalars.  Import replaces the whole state (this
@@ -248,8 +274,8 @@ int retopk_import_state(retopk_ctx* ctx, const float* qbar, const int32_t* suppo
  *
  * Who needs it: code that runs where cudaMalloc is off limits - inside a region whose memory
  * is fully owned by another allocator (an inference server's arena, a framework's caching
- * allocator that forbids raw allocations), while a stream capture is being recorded, or
- * in a plug-in that is only handed input and output buffers.  retopk_create allocates the
+ * allocator that forbids raw allocations), or in a plug-in that is only handed input and
+ * output buffers.  retopk_create allocates the
  * score workspace with cudaMalloc; this call instead keeps its workspace in a fixed array
  * that is part of the library image (RETOPK_STATIC_SCRATCH_BYTES of device memory on every
  * GPU that loads the library, held until the process exits).
@@ -263,12 +289,13 @@ int retopk_import_state(retopk_ctx* ctx, const float* qbar, const int32_t* suppo
  * nothing is launched.
  *
  * The first call on a device looks up the array's device address and opts the kernels in to
- * large shared memory; make that first call outside any stream capture.  No call allocates,
- * frees or synchronises.  All calls on a device share the one array: scores and tile maxima
- * are rewritten by every call before they are read; the one word that must start at zero
- * (the scan's work counter) is zero in the library image and is put back to zero by the
- * last kernel of every call.  Two calls that overlap on the GPU (different streams, no
- * dependency) race on the array.
+ * large shared memory; make that first call before any stream capture begins.  That set-up is
+ * guarded by a lock, so host threads may race for it.  No call allocates, frees or
+ * synchronises.  All calls on a device share the one array, which keeps the last call's
+ * contents: scores and tile maxima are rewritten by every call before they are read, and the
+ * one word that must start at zero (the scan's work counter) is cleared on the stream at the
+ * start of every call, so a call does not depend on how an earlier one ended.  Two calls that
+ * overlap on the GPU (different streams, no dependency) race on the array.
  */
 #define RETOPK_STATIC_SCRATCH_BYTES (32u << 20)
 int exact_topk_decode_static(int B, int H_q, int H_kv, int d, int K, int64_t max_seq_len, const void* q,
@@ -279,9 +306,10 @@ int exact_topk_decode_static(int B, int H_q, int H_kv, int d, int K, int64_t max
  * Measurement hooks (no counterpart in the paper).  Between begin and end, every decode
  * call of this context brackets each of its kernels with CUDA events on the call's stream
  * (up to max_calls calls; later calls run unrecorded).  retopk_profile_end synchronises
- * the device and returns, per kernel slot {0: recall, 1: scan, 2: finish}, the summed
- * device time in milliseconds and the number of launches.  Not for use inside a timed
- * region: the events themselves cost a little.
+ * the device and returns, per kernel slot {0: step (recall + reuse path), 1: scan, 2: exact
+ * finish}, the summed device time in milliseconds and the number of launches.  Not for use
+ * inside a timed region: the events themselves cost a little, and an event between two
+ * kernels keeps the second from starting early.  A failed begin keeps nothing allocated.
  */
 int retopk_profile_begin(retopk_ctx* ctx, int max_calls);
 int retopk_profile_end(retopk_ctx* ctx, double ms_host[3], int64_t launches_host[3]);

@@ -25,6 +25,13 @@ def is_stale() -> bool:
     return any(os.path.getmtime(s) > built for s in _sources())
 
 
+def find_nvcc() -> str:
+    nvcc = shutil.which("nvcc") or "/usr/local/cuda/bin/nvcc"
+    if not os.path.exists(nvcc):
+        raise RuntimeError("nvcc not found: cannot build libretopk.so")
+    return nvcc
+
+
 def build(force: bool = False, verbose: bool = False) -> str:
     """Run nvcc if the library is missing or older than its sources; return its path.
 
@@ -33,9 +40,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     """
     if not force and not is_stale():
         return LIB_PATH
-    nvcc = shutil.which("nvcc") or "/usr/local/cuda/bin/nvcc"
-    if not os.path.exists(nvcc):
-        raise RuntimeError("nvcc not found: cannot build libretopk.so")
+    nvcc = find_nvcc()
     with open(LIB_PATH + ".lock", "w") as lock:
         fcntl.flock(lock, fcntl.LOCK_EX)
         try:

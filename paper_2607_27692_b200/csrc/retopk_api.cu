@@ -3,6 +3,7 @@
 #include "retopk_ladder.cuh"
 
 #include <math.h>
+#include <mutex>
 #include <new>
 #include <stdio.h>
 #include <string.h>
@@ -17,13 +18,15 @@ struct retopk_ctx {
     float tau;
     long long max_seq_len, score_stride, tmax_stride;
     long long n_ins, t_dec;
-    int NS, tile_cap, stage_depth, exact_stage_depth;      // of the finish shape in use
+    int NS, tile_cap, stage_depth, exact_stage_depth, win_prefetch;      // of the block shape in use
     int finish_threads;          // 1024, or 512 with two CTAs per SM when there are more heads than SMs
-    struct FinishShape { int ok, stage_depth, exact_stage_depth; size_t smem_reuse, smem_exact, smem_finish; } shape[2];   // [0]: 1024, [1]: 512
+    struct FinishShape { int ok, stage_depth, exact_stage_depth, win_prefetch; size_t smem_step, smem_exact; } shape[2];   // [0]: 1024, [1]: 512
     int num_sms, scan_grid;
     int call_serial;
     int recall_recent;
-    size_t smem_recall, smem_reuse, smem_exact, smem_finish;
+    int broken;                  // a launch failed in the middle of a step: the caches are inconsistent until reset
+    mutable int fail_launch;     // test hook: the next launch of kernel 1 (step), 2 (scan) or 3 (finish) reports a failure
+    size_t smem_step, smem_exact;
     // device state
     float* qbar_cache;
     uint16_t* qbar16;            // bf16 copy of the layout, allocated when that format is chosen
@@ -34,6 +37,9 @@ struct retopk_ctx {
     int32_t* ws_ncand;
     int32_t* ws_sel;
     int32_t* ws_gflag;
+    int32_t* ws_xlist;
+    unsigned int* ws_xcount;
+    int32_t* dbg_cand;           // candidate lists of the last reuse step (test hook), or null
     float* ws_scores;
     float* ws_tmax;
     unsigned long long* counters;
@@ -85,6 +91,7 @@ void free_all(retopk_ctx* c) {
     cudaFree(c->status); cudaFree(c->slow_select); cudaFree(c->scan_groups); cudaFree(c->scan_counter); cudaFree(c->stage_q); cudaFree(c->stage_out);
     cudaFree(c->stage_kv);
     cudaFree(c->qbar16);
+    cudaFree(c->ws_xlist); cudaFree(c->ws_xcount); cudaFree(c->dbg_cand);
     for (int i = 0; i < 8; ++i) cudaFree(c->lw_persist[i]);
     if (c->pool) cudaMemPoolDestroy(c->pool);
 }
@@ -110,6 +117,8 @@ StepArgs make_args(const retopk_ctx* c, const void* q, const void* k, const void
     a.g_shift = (c->G & (c->G - 1)) == 0 ? __builtin_ctz((unsigned)c->G) : -1;
     a.stage_depth = c->stage_depth;
     a.exact_stage_depth = c->exact_stage_depth;
+    a.win_prefetch = c->win_prefetch;
+    a.ws_xlist = c->ws_xlist; a.ws_xcount = c->ws_xcount; a.dbg_cand = c->dbg_cand;
     a.q = static_cast<const uint16_t*>(q);
     a.k = static_cast<const uint16_t*>(k);
     a.v = static_cast<const uint16_t*>(v);
@@ -126,8 +135,8 @@ StepArgs make_args(const retopk_ctx* c, const void* q, const void* k, const void
     return a;
 }
 
-// CTAs per head in finish_kernel: with few heads, as many (a power of two up to 8, one SM each)
-// as still fit one wave.
+// CTAs per head in step_kernel / exact_finish_kernel: with few heads, as many (a power of two
+// up to 8, one SM each) as still fit one wave.
 int auto_cluster(long long heads, int num_sms) {
     int cl = 1;
     while (cl < 8 && heads * cl * 2 <= num_sms) cl *= 2;
@@ -145,9 +154,9 @@ void use_finish_shape(retopk_ctx* c, int threads) {
     c->finish_threads = threads;
     c->stage_depth = sh.stage_depth;
     c->exact_stage_depth = sh.exact_stage_depth;
-    c->smem_reuse = sh.smem_reuse;
+    c->win_prefetch = sh.win_prefetch;
+    c->smem_step = sh.smem_step;
     c->smem_exact = sh.smem_exact;
-    c->smem_finish = sh.smem_finish;
 }
 
 // Launch with programmatic stream serialisation: the kernel may be set up while its
@@ -176,22 +185,32 @@ int launch_dependent(Kernel kernel, unsigned grid, unsigned block, size_t smem, 
     return cudaLaunchKernelEx(&cfg, kernel, a) == cudaSuccess ? RETOPK_OK : RETOPK_ECUDA;
 }
 
-int launch_recall(const retopk_ctx* c, const StepArgs& a, cudaStream_t s) {
-    const unsigned grid = (unsigned)(c->B * c->Hq);
-    if (c->d == 128) return launch_dependent(recall_kernel<128>, grid, RECALL_THREADS, c->smem_recall, s, a, c->dependent_launches);
-    return launch_dependent(recall_kernel<64>, grid, RECALL_THREADS, c->smem_recall, s, a, c->dependent_launches);
+// Test hook (host side only): pretend that the launch of kernel `which` failed.
+bool injected_failure(const retopk_ctx* c, int which) {
+    if (c->fail_launch != which) return false;
+    c->fail_launch = 0;
+    return true;
+}
+
+int launch_step(const retopk_ctx* c, const StepArgs& a, cudaStream_t s) {
+    if (injected_failure(c, 1)) return RETOPK_ECUDA;
+    const unsigned grid = (unsigned)(c->B * c->Hq * c->cluster);      // one cluster of CTAs per head
+    if (c->finish_threads == 512) {
+        if (c->d == 128) return launch_dependent(step_kernel<128, 512>, grid, 512, c->smem_step, s, a, c->dependent_launches, c->cluster);
+        return launch_dependent(step_kernel<64, 512>, grid, 512, c->smem_step, s, a, c->dependent_launches, c->cluster);
+    }
+    if (c->d == 128) return launch_dependent(step_kernel<128, 1024>, grid, FINISH_THREADS, c->smem_step, s, a, c->dependent_launches, c->cluster);
+    return launch_dependent(step_kernel<64, 1024>, grid, FINISH_THREADS, c->smem_step, s, a, c->dependent_launches, c->cluster);
 }
 
 int launch_scan(const retopk_ctx* c, const StepArgs& a, cudaStream_t s) {
+    if (injected_failure(c, 2)) return RETOPK_ECUDA;
     // persistent CTAs; no more of them than there are 256-row work items
     const long long items = (long long)c->B * c->Hkv * ((a.L + SCAN_TILE_ROWS - 1) / SCAN_TILE_ROWS);
     const unsigned grid = (unsigned)(items < c->scan_grid ? items : c->scan_grid);
     const int ntile = (c->G + 7) / 8;
-    // A dependent launch behind recall_kernel (or behind the previous call's last kernel for
-    // Exact Top-K).  Behind a kernel that takes ALL of an SM's shared memory the scan ran 1.6x
-    // slower: its CTAs then land on SMs still carved up for that kernel, and it needs about
-    // 100 KB of L1 per SM to keep its loads in flight.  recall_kernel uses a few KB, so the SMs
-    // are back in the default split by the time the scan's CTAs start.
+    // A dependent launch behind step_kernel (or behind the previous call's last kernel for
+    // Exact Top-K).
     if (c->d == 128 && ntile == 1) return launch_dependent(scan_kernel<128, 1>, grid, SCAN_THREADS, 0, s, a, c->dependent_launches);
     if (c->d == 128) return launch_dependent(scan_kernel<128, 2>, grid, SCAN_THREADS, 0, s, a, c->dependent_launches);
     if (ntile == 1) return launch_dependent(scan_kernel<64, 1>, grid, SCAN_THREADS, 0, s, a, c->dependent_launches);
@@ -199,14 +218,15 @@ int launch_scan(const retopk_ctx* c, const StepArgs& a, cudaStream_t s) {
 }
 
 int launch_finish(const retopk_ctx* c, const StepArgs& a, cudaStream_t s) {
+    if (injected_failure(c, 3)) return RETOPK_ECUDA;
     const unsigned grid = (unsigned)(c->B * c->Hq * c->cluster);      // one cluster of CTAs per head
-    const size_t smem = a.mode == MODE_EXACT ? c->smem_exact : c->smem_finish;
+    const size_t smem = c->smem_exact;
     if (c->finish_threads == 512) {
-        if (c->d == 128) return launch_dependent(finish_kernel<128, 512>, grid, 512, smem, s, a, c->dependent_launches, c->cluster);
-        return launch_dependent(finish_kernel<64, 512>, grid, 512, smem, s, a, c->dependent_launches, c->cluster);
+        if (c->d == 128) return launch_dependent(exact_finish_kernel<128, 512>, grid, 512, smem, s, a, c->dependent_launches, c->cluster);
+        return launch_dependent(exact_finish_kernel<64, 512>, grid, 512, smem, s, a, c->dependent_launches, c->cluster);
     }
-    if (c->d == 128) return launch_dependent(finish_kernel<128, 1024>, grid, FINISH_THREADS, smem, s, a, c->dependent_launches, c->cluster);
-    return launch_dependent(finish_kernel<64, 1024>, grid, FINISH_THREADS, smem, s, a, c->dependent_launches, c->cluster);
+    if (c->d == 128) return launch_dependent(exact_finish_kernel<128, 1024>, grid, FINISH_THREADS, smem, s, a, c->dependent_launches, c->cluster);
+    return launch_dependent(exact_finish_kernel<64, 1024>, grid, FINISH_THREADS, smem, s, a, c->dependent_launches, c->cluster);
 }
 
 // Measurement hook: event number `which` (0..3) of the current call, if recording.
@@ -231,7 +251,7 @@ void exact_list_sizes(int K, int* NS, int* tile_cap) {
 // reduction scratch and the value-row landing zone take over once the support is emitted.
 // Returns 0 if not even `min_waves` rows per row slot fit; else the bytes, and the depth.
 size_t exact_smem(int K, int NS, int tile_cap, int d, int nt, size_t budget, int min_waves, int* depth) {
-    const size_t live = ((size_t)3 * K + SCRATCH_WORDS + 32 + 8 + 3) & ~(size_t)3;
+    const size_t live = ((size_t)3 * K + SCRATCH_WORDS + WS_WORDS + 8 + 3) & ~(size_t)3;
     const size_t lists = (size_t)2 * NS + tile_cap;
     const size_t red = ((size_t)(nt / 32) * d + nt + 3) & ~(size_t)3;
     const size_t wave = (size_t)nt * 16;
@@ -245,11 +265,19 @@ size_t exact_smem(int K, int NS, int tile_cap, int d, int nt, size_t budget, int
     return (live + (lists > tail ? lists : tail)) * 4;
 }
 
+// The context's buffers live on the device that was current at create: work enqueued with
+// another device current would run there with these pointers.
+bool on_ctx_device(const retopk_ctx* c) {
+    int dev = -1;
+    return cudaGetDevice(&dev) == cudaSuccess && dev == c->device;
+}
+
 int check_step_args(const retopk_ctx* c, const void* q, const void* k, const void* v, long long L,
                     const void* out) {
     if (!c || !q || !k || !v || !out) return RETOPK_EINVAL;
     if (L < 1 || L > c->max_seq_len) return RETOPK_EINVAL;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v)) return RETOPK_EINVAL;
+    if (!on_ctx_device(c)) return RETOPK_EINVAL;
     return RETOPK_OK;
 }
 
@@ -280,15 +308,15 @@ int ladder_prepare(retopk_ctx* c) {
     const size_t bm_words = (((size_t)c->max_seq_len + 31) / 32 + 3) & ~(size_t)3;
     const size_t red_words = (size_t)(LADDER_THREADS / 32) * d + LADDER_THREADS;
     const size_t wave = (size_t)LADDER_THREADS * 16 * c->stage_depth;
-    const size_t union_words = ((r + 3) & ~(size_t)3) + 32 + capp + bm_words;
+    const size_t union_words = ((r + 3) & ~(size_t)3) + WS_WORDS + capp + bm_words;
     c->sm_sim = (d + Mp) * 4;
     c->sm_topr = (Mp + r + 4) * 4;
     c->sm_union = union_words * 4;
     c->sm_discover = (d + Mp + 4 + union_words) * 4;
     c->sm_score = (d + capp) * 4 + wave;
-    c->sm_select = (32 + SCRATCH_WORDS + 2 * K + 2 * cap) * 4;
-    c->sm_attend = (32 + ((3 * K + 3) & ~(size_t)3) + red_words) * 4 + wave;
-    const size_t head_words = (32 + SCRATCH_WORDS + 3 * K + 3) & ~(size_t)3;
+    c->sm_select = (WS_WORDS + SCRATCH_WORDS + 2 * K + 2 * cap) * 4;
+    c->sm_attend = (WS_WORDS + ((3 * K + 3) & ~(size_t)3) + red_words) * 4 + wave;
+    const size_t head_words = (WS_WORDS + SCRATCH_WORDS + 3 * K + 3) & ~(size_t)3;
     const size_t big_words = ((2 * cap > red_words ? 2 * cap : red_words) + 3) & ~(size_t)3;
     c->sm_fused = (head_words + big_words) * 4 + wave;
     int max_smem = 0;
@@ -411,7 +439,6 @@ int ladder_step(retopk_ctx* c, StepArgs a, cudaStream_t s) {
     int launches = 0;
     if (rc == RETOPK_OK) {
         ladder_bind(a, buf);
-        a.skip_reuse = 1;
         rc = ladder_launches(c, a, s, &launches);
     }
     if (level != 4)
@@ -421,6 +448,26 @@ int ladder_step(retopk_ctx* c, StepArgs a, cudaStream_t s) {
     return rc;
 }
 #undef LADDER_LAUNCH
+
+// Can a cluster of `cl` CTAs of `kernel` with this much shared memory be scheduled at all?
+template <class Kernel>
+bool cluster_fits(Kernel kernel, int threads, size_t smem, int cl) {
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof cfg);
+    cfg.gridDim = dim3((unsigned)cl);
+    cfg.blockDim = dim3((unsigned)threads);
+    cfg.dynamicSmemBytes = smem;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)cl;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) != cudaSuccess) { cudaGetLastError(); return false; }
+    return n > 0;
+}
 
 }  // namespace
 
@@ -456,7 +503,6 @@ int retopk_create_batched(retopk_ctx** out, int B, int H_q, int H_kv, int d, int
     c->num_sms = sms > 0 ? sms : 148;
 
     // shared-memory footprints (must mirror the carve-up at the top of each kernel)
-    c->smem_recall = ((size_t)d + ((M + 3) & ~3) + r + 4) * 4;
     int max_smem = 0, sm_smem = 0;
     cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, c->device);
     cudaDeviceGetAttribute(&sm_smem, cudaDevAttrMaxSharedMemoryPerMultiprocessor, c->device);
@@ -467,52 +513,55 @@ int retopk_create_batched(retopk_ctx** out, int B, int H_q, int H_kv, int d, int
         const size_t budget = v == 0 ? (size_t)max_smem : (size_t)(sm_smem / 2 - 1024);
         retopk_ctx::FinishShape& sh = c->shape[v];
         const size_t red_words = (size_t)(nt / 32) * d + nt;
-        const size_t head_words = ((size_t)d + r + 32 + SCRATCH_WORDS + 3 * (size_t)K + 3) & ~(size_t)3;
+        const size_t head_words = (size_t)step_head_words(d, M, r, K, W);
         const size_t big_words = (((size_t)2 * c->cap > red_words ? (size_t)2 * c->cap : red_words) + 3) & ~(size_t)3;
         const size_t bm_words = (((size_t)max_seq_len + 31) / 32 + 3) & ~(size_t)3;
-        sh.smem_reuse = (head_words + big_words + bm_words) * 4;
+        const size_t fixed = (head_words + big_words + bm_words) * 4;
         sh.smem_exact = exact_smem(K, c->NS, c->tile_cap, d, nt, budget, v == 0 ? 1 : 3, &sh.exact_stage_depth);
         // the rest of shared memory is the landing zone of the asynchronous row copies: one
         // 16-byte piece per thread per row kept in flight per row slot
         const size_t wave = (size_t)nt * 16;
         // the narrow shape only pays with a few waves of rows in flight on either path
         const size_t min_waves = v == 0 ? 1 : 3;
-        sh.ok = budget >= sh.smem_reuse + min_waves * wave && sh.smem_exact > 0;
+        sh.ok = budget >= fixed + min_waves * wave && sh.smem_exact > 0;
         if (!sh.ok) continue;
         const int slots = nt / (d / 8);
-        auto depth_for = [&](size_t fixed, int rows) {
-            long long fit = (long long)((budget - fixed) / wave);
-            long long want = (rows + slots - 1) / slots;          // one wave covers `rows` rows
-            long long dep = fit < want ? fit : want;
-            return (int)(dep < 1 ? 1 : (dep > 16 ? 16 : dep));
-        };
-        sh.stage_depth = depth_for(sh.smem_reuse, K + K / 4 > c->cap ? c->cap : K + K / 4);
-        if (sh.stage_depth * slots < K) {            // the value rows use the same zone
-            int dv = depth_for(sh.smem_reuse, K);
-            if (dv > sh.stage_depth) sh.stage_depth = dv;
-        }
-        sh.smem_reuse += (size_t)sh.stage_depth * wave;
-        sh.smem_finish = sh.smem_reuse > sh.smem_exact ? sh.smem_reuse : sh.smem_exact;
+        const long long fit = (long long)((budget - fixed) / wave);
+        auto waves_for = [&](int rows) { return (long long)((rows + slots - 1) / slots); };
+        // enough for the candidates below the window (typically K and a bit), the K value rows
+        // and the window's rows, whichever is most; 16 waves at the very most
+        long long want = waves_for(K + K / 4 > c->cap ? c->cap : K + K / 4);
+        if (waves_for(K) > want) want = waves_for(K);
+        if (waves_for(W) > want) want = waves_for(W);
+        long long dep = fit < want ? fit : want;
+        sh.stage_depth = (int)(dep < 1 ? 1 : (dep > 16 ? 16 : dep));
+        // the window's rows are requested at kernel entry when they fit the landing zone
+        sh.win_prefetch = W > 0 && waves_for(W) <= sh.stage_depth;
+        sh.smem_step = fixed + (size_t)sh.stage_depth * wave;
     }
     if (!c->shape[0].ok) { delete c; return RETOPK_EUNSUPPORTED; }
     // opt in to the device maximum once; contexts of different sizes then coexist
-    cudaError_t e1, e2 = cudaSuccess;
+    cudaError_t e1, e2 = cudaSuccess, e3, e4 = cudaSuccess;
     int occ = 0;
     const int ntile = (c->G + 7) / 8;
     if (d == 128) {
-        e1 = cudaFuncSetAttribute(finish_kernel<128, 1024>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
-        e2 = cudaFuncSetAttribute(finish_kernel<128, 512>, cudaFuncAttributeMaxDynamicSharedMemorySize, sm_smem / 2 - 1024);
+        e1 = cudaFuncSetAttribute(step_kernel<128, 1024>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
+        e2 = cudaFuncSetAttribute(step_kernel<128, 512>, cudaFuncAttributeMaxDynamicSharedMemorySize, sm_smem / 2 - 1024);
+        e3 = cudaFuncSetAttribute(exact_finish_kernel<128, 1024>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
+        e4 = cudaFuncSetAttribute(exact_finish_kernel<128, 512>, cudaFuncAttributeMaxDynamicSharedMemorySize, sm_smem / 2 - 1024);
         if (ntile == 1) cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, scan_kernel<128, 1>, SCAN_THREADS, 0);
         else cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, scan_kernel<128, 2>, SCAN_THREADS, 0);
     } else {
-        e1 = cudaFuncSetAttribute(finish_kernel<64, 1024>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
-        e2 = cudaFuncSetAttribute(finish_kernel<64, 512>, cudaFuncAttributeMaxDynamicSharedMemorySize, sm_smem / 2 - 1024);
+        e1 = cudaFuncSetAttribute(step_kernel<64, 1024>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
+        e2 = cudaFuncSetAttribute(step_kernel<64, 512>, cudaFuncAttributeMaxDynamicSharedMemorySize, sm_smem / 2 - 1024);
+        e3 = cudaFuncSetAttribute(exact_finish_kernel<64, 1024>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
+        e4 = cudaFuncSetAttribute(exact_finish_kernel<64, 512>, cudaFuncAttributeMaxDynamicSharedMemorySize, sm_smem / 2 - 1024);
         if (ntile == 1) cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, scan_kernel<64, 1>, SCAN_THREADS, 0);
         else cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, scan_kernel<64, 2>, SCAN_THREADS, 0);
     }
-    if (e1 != cudaSuccess || e2 != cudaSuccess) { cudaGetLastError(); delete c; return RETOPK_ECUDA; }
+    if (e1 != cudaSuccess || e2 != cudaSuccess || e3 != cudaSuccess || e4 != cudaSuccess) { cudaGetLastError(); delete c; return RETOPK_ECUDA; }
     c->scan_grid = c->num_sms * (occ > 0 ? occ : 2);
-    // finish_kernel: with few heads, a cluster of CTAs (one SM each) per head, as many as fit one wave
+    // with few heads, a cluster of CTAs (one SM each) per head, as many as fit one wave
     c->cluster = auto_cluster((long long)B * H_q, c->num_sms);
     use_finish_shape(c, auto_finish_threads(c));
 
@@ -520,7 +569,8 @@ int retopk_create_batched(retopk_ctx** out, int B, int H_q, int H_kv, int d, int
     const size_t nh = (size_t)B * H_q;
     bool ok = dev_alloc(&c->qbar_cache, nh * M * d) && dev_alloc(&c->sup_cache, nh * M * K) &&
               dev_alloc(&c->ws_path, nh) && dev_alloc(&c->ws_rho, nh) && dev_alloc(&c->ws_ncand, nh) &&
-              dev_alloc(&c->ws_sel, nh * r) && dev_alloc(&c->ws_gflag, (size_t)B * H_kv + 1) && dev_alloc(&c->ws_scores, nh * (size_t)c->score_stride) &&
+              dev_alloc(&c->ws_sel, nh * r) && dev_alloc(&c->ws_gflag, (size_t)B * H_kv + 1) &&
+              dev_alloc(&c->ws_xlist, nh) && dev_alloc(&c->ws_xcount, 2) && dev_alloc(&c->ws_scores, nh * (size_t)c->score_stride) &&
               dev_alloc(&c->ws_tmax, nh * (size_t)c->tmax_stride) &&
               dev_alloc(&c->counters, nh * 4) && dev_alloc(&c->status, 1) &&
               dev_alloc(&c->slow_select, 1) && dev_alloc(&c->scan_groups, 1) && dev_alloc(&c->scan_counter, 1) && dev_alloc(&c->stage_q, nh * d) &&
@@ -558,7 +608,25 @@ int retopk_set_qbar_format(retopk_ctx* c, int format) {
 
 int retopk_set_cluster_size(retopk_ctx* c, int ctas_per_head) {
     if (!c || (ctas_per_head != 1 && ctas_per_head != 2 && ctas_per_head != 4 && ctas_per_head != 8)) return RETOPK_EINVAL;
+    if (ctas_per_head > 1) {
+        // checked here, so that a size the device cannot schedule fails now and not in the middle of a step
+        DeviceGuard g(c->device);
+        bool ok;
+        if (c->finish_threads == 512)
+            ok = c->d == 128 ? cluster_fits(step_kernel<128, 512>, 512, c->smem_step, ctas_per_head) && cluster_fits(exact_finish_kernel<128, 512>, 512, c->smem_exact, ctas_per_head)
+                             : cluster_fits(step_kernel<64, 512>, 512, c->smem_step, ctas_per_head) && cluster_fits(exact_finish_kernel<64, 512>, 512, c->smem_exact, ctas_per_head);
+        else
+            ok = c->d == 128 ? cluster_fits(step_kernel<128, 1024>, 1024, c->smem_step, ctas_per_head) && cluster_fits(exact_finish_kernel<128, 1024>, 1024, c->smem_exact, ctas_per_head)
+                             : cluster_fits(step_kernel<64, 1024>, 1024, c->smem_step, ctas_per_head) && cluster_fits(exact_finish_kernel<64, 1024>, 1024, c->smem_exact, ctas_per_head);
+        if (!ok) return RETOPK_EUNSUPPORTED;
+    }
     c->cluster = ctas_per_head;
+    return RETOPK_OK;
+}
+
+int retopk_debug_fail_next_launch(retopk_ctx* c, int which) {
+    if (!c || which < 0 || which > 3) return RETOPK_EINVAL;
+    c->fail_launch = which;
     return RETOPK_OK;
 }
 
@@ -613,13 +681,14 @@ int retopk_destroy(retopk_ctx* c) {
 }
 
 int retopk_reset(retopk_ctx* c, void* stream) {
-    if (!c) return RETOPK_EINVAL;
+    if (!c || !on_ctx_device(c)) return RETOPK_EINVAL;
     const size_t nh = (size_t)c->B * c->Hq;
     reset_kernel<<<c->num_sms * 4, 256, 0, static_cast<cudaStream_t>(stream)>>>(
         c->qbar_cache, nh * c->M * c->d, c->sup_cache, nh * c->M * c->K, c->counters, nh * 4, c->ws_gflag,
-        (size_t)c->B * c->Hkv + 1, c->status, c->slow_select, c->scan_groups, c->scan_counter);
+        (size_t)c->B * c->Hkv + 1, c->status, c->slow_select, c->scan_groups, c->scan_counter, c->ws_xcount);
     c->n_ins = 0;
     c->t_dec = 0;
+    c->broken = 0;
     if (cudaGetLastError() != cudaSuccess) return RETOPK_ECUDA;
     if (c->qbar16 && cudaMemsetAsync(c->qbar16, 0, nh * c->M * c->d * 2, static_cast<cudaStream_t>(stream)) != cudaSuccess)
         return RETOPK_ECUDA;
@@ -630,22 +699,27 @@ int retopk_decode_step(retopk_ctx* c, const void* q, const void* k_cache, const 
                        int64_t seq_len, void* out, void* stream) {
     int rc = check_step_args(c, q, k_cache, v_cache, seq_len, out);
     if (rc != RETOPK_OK) return rc;
+    if (c->broken) return RETOPK_ECUDA;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     StepArgs a = make_args(c, q, k_cache, v_cache, seq_len, out, MODE_RETOPK);
     c->call_serial = (c->call_serial + 1) & 0x3fffffff;
     a.step_id = c->call_serial;
     if (c->fusion_level < 5) {
-        if ((rc = ladder_step(c, a, s)) != RETOPK_OK) return rc;
+        // a failure inside may have left some of the step's kernels enqueued
+        if ((rc = ladder_step(c, a, s)) != RETOPK_OK) { c->broken = 1; return rc; }
         c->n_ins += 1;
         c->t_dec += 1;
         return RETOPK_OK;
     }
     prof_mark(c, 0, s);
-    if ((rc = launch_recall(c, a, s)) != RETOPK_OK) return rc;
+    if ((rc = launch_step(c, a, s)) != RETOPK_OK) return rc;      // nothing of this step is enqueued yet
     prof_mark(c, 1, s);
-    if ((rc = launch_scan(c, a, s)) != RETOPK_OK) return rc;
+    // From here on the step's first kernel is in the stream (normalised queries inserted, exact
+    // heads listed): a failed launch leaves the caches half advanced, so the context refuses
+    // further steps until retopk_reset.
+    if ((rc = launch_scan(c, a, s)) != RETOPK_OK) { c->broken = 1; return rc; }
     prof_mark(c, 2, s);
-    if ((rc = launch_finish(c, a, s)) != RETOPK_OK) return rc;
+    if ((rc = launch_finish(c, a, s)) != RETOPK_OK) { c->broken = 1; return rc; }
     prof_mark(c, 3, s);
     prof_done(c, 0);
     c->last_launches = 3;
@@ -659,6 +733,8 @@ int retopk_prefill(retopk_ctx* c, const void* q_tail, const void* k_cache, const
     if (!c || !q_tail || !k_cache || !v_cache) return RETOPK_EINVAL;
     if (n_tail < 1 || n_tail > c->M || n_tail > prompt_len || prompt_len > c->max_seq_len) return RETOPK_EINVAL;
     if (!aligned16(q_tail) || !aligned16(k_cache) || !aligned16(v_cache)) return RETOPK_EINVAL;
+    if (!on_ctx_device(c)) return RETOPK_EINVAL;
+    if (c->broken) return RETOPK_ECUDA;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const size_t slab = (size_t)c->B * c->Hq * c->d;          // elements per prompt position
     for (int j = 0; j < n_tail; ++j) {
@@ -670,9 +746,9 @@ int retopk_prefill(retopk_ctx* c, const void* q_tail, const void* k_cache, const
         c->call_serial = (c->call_serial + 1) & 0x3fffffff;
         a.step_id = c->call_serial;
         int rc;
-        if ((rc = launch_recall(c, a, s)) != RETOPK_OK) return rc;
-        if ((rc = launch_scan(c, a, s)) != RETOPK_OK) return rc;
-        if ((rc = launch_finish(c, a, s)) != RETOPK_OK) return rc;
+        if ((rc = launch_step(c, a, s)) != RETOPK_OK) return rc;
+        if ((rc = launch_scan(c, a, s)) != RETOPK_OK) { c->broken = 1; return rc; }
+        if ((rc = launch_finish(c, a, s)) != RETOPK_OK) { c->broken = 1; return rc; }
         c->n_ins += 1;
     }
     c->last_launches = 3 * n_tail;
@@ -690,7 +766,11 @@ int exact_topk_decode(retopk_ctx* c, const void* q, const void* k_cache, const v
     prof_mark(c, 1, s);
     if ((rc = launch_scan(c, a, s)) != RETOPK_OK) return rc;
     prof_mark(c, 2, s);
-    if ((rc = launch_finish(c, a, s)) != RETOPK_OK) return rc;
+    if ((rc = launch_finish(c, a, s)) != RETOPK_OK) {
+        // the scan is enqueued and nothing will put its work counter back: do it here
+        cudaMemsetAsync(c->scan_counter, 0, sizeof(unsigned int), s);
+        return rc;
+    }
     prof_mark(c, 3, s);
     prof_done(c, 1);
     c->last_launches = 2;
@@ -784,7 +864,7 @@ int retopk_stats(retopk_ctx* c, retopk_stats_t* st) {
 
 int retopk_last_step(retopk_ctx* c, int32_t* support, uint8_t* path, float* rho_max, int32_t* n_cand,
                      void* stream) {
-    if (!c) return RETOPK_EINVAL;
+    if (!c || !on_ctx_device(c)) return RETOPK_EINVAL;
     if (c->n_ins < 1) return RETOPK_EINVAL;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const size_t nh = (size_t)c->B * c->Hq;
@@ -802,15 +882,40 @@ int retopk_last_step(retopk_ctx* c, int32_t* support, uint8_t* path, float* rho_
 }
 
 int retopk_last_recall(retopk_ctx* c, int32_t* sel, void* stream) {
-    if (!c || !sel || c->n_ins < 1) return RETOPK_EINVAL;
+    if (!c || !sel || c->n_ins < 1 || !on_ctx_device(c)) return RETOPK_EINVAL;
     const size_t bytes = (size_t)c->B * c->Hq * c->r * 4;
     return cudaMemcpyAsync(sel, c->ws_sel, bytes, cudaMemcpyDeviceToDevice, static_cast<cudaStream_t>(stream)) == cudaSuccess
                ? RETOPK_OK : RETOPK_ECUDA;
 }
 
+int retopk_debug_candidates(retopk_ctx* c, int enable) {
+    if (!c || (enable != 0 && enable != 1)) return RETOPK_EINVAL;
+    DeviceGuard g(c->device);
+    if (cudaDeviceSynchronize() != cudaSuccess) return RETOPK_ECUDA;
+    if (enable && !c->dbg_cand) {
+        const size_t n = (size_t)c->B * c->Hq * c->cap;
+        if (cudaMalloc(reinterpret_cast<void**>(&c->dbg_cand), n * 4 > 0 ? n * 4 : 16) != cudaSuccess) {
+            cudaGetLastError();
+            c->dbg_cand = nullptr;
+            return RETOPK_ENOMEM;
+        }
+    } else if (!enable && c->dbg_cand) {
+        cudaFree(c->dbg_cand);
+        c->dbg_cand = nullptr;
+    }
+    return RETOPK_OK;
+}
+
+int retopk_last_candidates(retopk_ctx* c, int32_t* cand, void* stream) {
+    if (!c || !cand || !c->dbg_cand || c->n_ins < 1 || !on_ctx_device(c)) return RETOPK_EINVAL;
+    const size_t bytes = (size_t)c->B * c->Hq * c->cap * 4;
+    return cudaMemcpyAsync(cand, c->dbg_cand, bytes, cudaMemcpyDeviceToDevice, static_cast<cudaStream_t>(stream)) == cudaSuccess
+               ? RETOPK_OK : RETOPK_ECUDA;
+}
+
 int retopk_export_state(retopk_ctx* c, float* qbar, int32_t* supports, int64_t* n_inserted,
                         int64_t* t_dec, void* stream) {
-    if (!c) return RETOPK_EINVAL;
+    if (!c || !on_ctx_device(c)) return RETOPK_EINVAL;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const size_t nh = (size_t)c->B * c->Hq;
     bool ok = true;
@@ -828,7 +933,7 @@ int retopk_export_state(retopk_ctx* c, float* qbar, int32_t* supports, int64_t* 
 
 int retopk_import_state(retopk_ctx* c, const float* qbar, const int32_t* supports, int64_t n_inserted,
                         int64_t t_dec, void* stream) {
-    if (!c || !qbar || !supports || n_inserted < 0 || t_dec < 0) return RETOPK_EINVAL;
+    if (!c || !qbar || !supports || n_inserted < 0 || t_dec < 0 || !on_ctx_device(c)) return RETOPK_EINVAL;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const size_t nh = (size_t)c->B * c->Hq;
     bool ok;
@@ -848,11 +953,19 @@ int retopk_import_state(retopk_ctx* c, const float* qbar, const int32_t* support
 int retopk_profile_begin(retopk_ctx* c, int max_calls) {
     if (!c || max_calls < 1 || c->prof_events) return RETOPK_EINVAL;
     DeviceGuard g(c->device);
-    c->prof_events = new (std::nothrow) cudaEvent_t[(size_t)max_calls * 4];
-    c->prof_kind = new (std::nothrow) unsigned char[max_calls];
-    if (!c->prof_events || !c->prof_kind) return RETOPK_ENOMEM;
-    for (int i = 0; i < max_calls * 4; ++i)
-        if (cudaEventCreate(&c->prof_events[i]) != cudaSuccess) return RETOPK_ECUDA;
+    cudaEvent_t* ev = new (std::nothrow) cudaEvent_t[(size_t)max_calls * 4];
+    unsigned char* kind = new (std::nothrow) unsigned char[max_calls];
+    int made = 0, rc = (ev && kind) ? RETOPK_OK : RETOPK_ENOMEM;
+    for (; rc == RETOPK_OK && made < max_calls * 4; ++made)
+        if (cudaEventCreate(&ev[made]) != cudaSuccess) { cudaGetLastError(); rc = RETOPK_ECUDA; break; }
+    if (rc != RETOPK_OK) {         // nothing is kept of a half-made set
+        for (int i = 0; i < made; ++i) cudaEventDestroy(ev[i]);
+        delete[] ev;
+        delete[] kind;
+        return rc;
+    }
+    c->prof_events = ev;
+    c->prof_kind = kind;
     c->prof_max = max_calls;
     c->prof_calls = 0;
     return RETOPK_OK;
@@ -902,10 +1015,12 @@ struct StaticSetup {
     int occ[2][2];               // scan CTAs per SM for d in {64,128} x head tiles in {1,2}
 };
 StaticSetup g_static_setup[STATIC_MAX_DEVICES];
+std::mutex g_static_mutex;       // host threads may race for the first call on a device
 
 // First use on the current device: resolve the array's address, opt in to large shared memory.
 int static_setup(int dev, StaticSetup** out) {
     if (dev < 0 || dev >= STATIC_MAX_DEVICES) return RETOPK_EUNSUPPORTED;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
     StaticSetup* st = &g_static_setup[dev];
     if (!st->ready) {
         void* p = nullptr;
@@ -914,8 +1029,8 @@ int static_setup(int dev, StaticSetup** out) {
         if (cudaDeviceGetAttribute(&st->num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
             cudaDeviceGetAttribute(&st->max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess)
             return RETOPK_ECUDA;
-        if (cudaFuncSetAttribute(finish_kernel<128, 1024>, cudaFuncAttributeMaxDynamicSharedMemorySize, st->max_smem) != cudaSuccess ||
-            cudaFuncSetAttribute(finish_kernel<64, 1024>, cudaFuncAttributeMaxDynamicSharedMemorySize, st->max_smem) != cudaSuccess)
+        if (cudaFuncSetAttribute(exact_finish_kernel<128, 1024>, cudaFuncAttributeMaxDynamicSharedMemorySize, st->max_smem) != cudaSuccess ||
+            cudaFuncSetAttribute(exact_finish_kernel<64, 1024>, cudaFuncAttributeMaxDynamicSharedMemorySize, st->max_smem) != cudaSuccess)
             return RETOPK_ECUDA;
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&st->occ[0][0], scan_kernel<64, 1>, SCAN_THREADS, 0);
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&st->occ[0][1], scan_kernel<64, 2>, SCAN_THREADS, 0);
@@ -980,11 +1095,15 @@ int exact_topk_decode_static(int B, int H_q, int H_kv, int d, int K, int64_t max
     // the two diagnostic counters the kernels add to are sinks here; they need no clearing
     a.slow_select = reinterpret_cast<unsigned long long*>(st->scratch);
     a.scan_groups = reinterpret_cast<unsigned long long*>(st->scratch + 8);
-    a.scan_counter = reinterpret_cast<unsigned int*>(st->scratch + 16);   // zero in the image, reset by every finish
+    a.scan_counter = reinterpret_cast<unsigned int*>(st->scratch + 16);
     a.ws_scores = reinterpret_cast<float*>(st->scratch + 256);
     a.ws_tmax = a.ws_scores + nh * score_stride;
 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    // The scan's work counter is the one word of the array that must start at zero.  It is
+    // cleared here in every call (a stream-ordered fill of four bytes: no allocation, no
+    // synchronisation), so a call never depends on how an earlier one ended.
+    if (cudaMemsetAsync(a.scan_counter, 0, sizeof(unsigned int), s) != cudaSuccess) return RETOPK_ECUDA;
     const int ntile = (a.G + 7) / 8;
     const int occ = st->occ[d == 128][ntile - 1];
     const long long items = (long long)B * H_kv * ((a.L + SCAN_TILE_ROWS - 1) / SCAN_TILE_ROWS);
@@ -997,15 +1116,16 @@ int exact_topk_decode_static(int B, int H_q, int H_kv, int d, int K, int64_t max
     if (cudaGetLastError() != cudaSuccess) return RETOPK_ECUDA;
     const int cluster = auto_cluster(nh, st->num_sms);
     a.cl_shift = __builtin_ctz((unsigned)cluster);
-    if (d == 128) return launch_dependent(finish_kernel<128, 1024>, (unsigned)(nh * cluster), FINISH_THREADS, smem, s, a, 0, cluster);
-    return launch_dependent(finish_kernel<64, 1024>, (unsigned)(nh * cluster), FINISH_THREADS, smem, s, a, 0, cluster);
+    if (d == 128) return launch_dependent(exact_finish_kernel<128, 1024>, (unsigned)(nh * cluster), FINISH_THREADS, smem, s, a, 0, cluster);
+    return launch_dependent(exact_finish_kernel<64, 1024>, (unsigned)(nh * cluster), FINISH_THREADS, smem, s, a, 0, cluster);
 }
 
 #ifdef RETOPK_PHASE_CLOCKS
-// Development aid (not part of the public interface): copy the phase clock table to the host.
+// Measurement aid, only in a library built with -DRETOPK_PHASE_CLOCKS (the benchmark's --phases
+// flag builds one): copy the phase clock table [3][1024][RETOPK_PHASE_SLOTS] to the host.
 int retopk_debug_read_phases(long long* host) {
     cudaDeviceSynchronize();
-    return cudaMemcpyFromSymbol(host, g_phase_clk, sizeof(long long) * 3 * 1024 * 16) == cudaSuccess ? 0 : -4;
+    return cudaMemcpyFromSymbol(host, g_phase_clk, sizeof(long long) * 3 * 1024 * RETOPK_PHASE_SLOTS) == cudaSuccess ? 0 : -4;
 }
 #endif
 

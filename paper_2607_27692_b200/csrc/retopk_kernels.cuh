@@ -1,23 +1,24 @@
 // Device code of the ReTopK decode step (sm_100a).
 //
-// Three kernels per step, all reading caller-owned bf16 q / K / V:
-//   recall_kernel  one CTA per (sequence, query head): normalise the query, cosine
-//                  similarity to the cached queries (Eq. 6), Top-r recall and rho_max
-//                  (Eq. 7), path decision (Eq. 13), insert of the normalised query.  A head
-//                  on the exact path flags its KV group.
+// Three launches per step, all reading caller-owned bf16 q / K / V:
+//   step_kernel    one CTA per (sequence, query head) - or a thread-block cluster of 2-8 CTAs
+//                  when there are few heads, or 512-thread CTAs two to an SM when there are
+//                  more heads than SMs.  Normalise the query, cosine similarity to the cached
+//                  queries (Eq. 6), Top-r recall and rho_max (Eq. 7), path decision (Eq. 13),
+//                  insert of the normalised query.  A head that reuses stays in its CTA to the
+//                  end: candidate union (Eq. 8-9) in a shared-memory bitmap, exact scores of
+//                  the gathered key rows (Eq. 10; the recent window's rows are requested at
+//                  kernel entry and arrive while the cache is searched), Top-K (Eq. 11),
+//                  softmax.V (Eq. 12), support insert.  A head on the exact path flags its KV
+//                  group, takes a ticket in the step's list of exact heads and leaves.
 //   scan_kernel    persistent CTAs over the flagged KV groups: full-history scores
 //                  e_i = q.k_i/sqrt(d) (Eq. 4); every key row streams once through the
 //                  tensor cores for all G query heads of its group; also the maximum of
-//                  every 16-row tile.
-//   finish_kernel  one CTA per (sequence, query head) - or a thread-block cluster of 2-8 CTAs
-//                  when there are few heads, or 512-thread CTAs two to an SM when there are
-//                  more heads than SMs - with heads of both paths side by side.
-//                  Reuse path: candidate union (Eq. 8-9) in a shared-memory bitmap, exact
-//                  scores of the gathered key rows (Eq. 10), Top-K (Eq. 11).  Exact path:
-//                  global Top-K (Eq. 1) of the scanned scores (tile maxima give a lower
-//                  bound for the K-th score, only the tiles that reach it are read back).
-//                  Both: softmax.V (Eq. 12) and the support insert.
-//                  Exact Top-K attention is scan + finish with every head on the exact path.
+//                  every 16-row tile.  Leaves at once when no group is flagged.
+//   exact_finish_kernel  one CTA (or cluster) per LISTED head: global Top-K (Eq. 1) of the
+//                  scanned scores (tile maxima give a lower bound for the K-th score, only the
+//                  tiles that reach it are read back), softmax.V (Eq. 12), support insert.
+//                  Exact Top-K attention is scan + exact finish with every head listed.
 // All three are programmatic dependent launches; ingest_kernel serves the host-buffer entry point.
 #pragma once
 #include <cooperative_groups.h>
@@ -26,10 +27,12 @@
 #include <math_constants.h>
 #include <stdint.h>
 
-// Development aid: with -DRETOPK_PHASE_CLOCKS thread 0 of every CTA stamps the SM clock at
-// phase boundaries into a global table (read back through retopk_debug_read_phases).
+// Measurement aid: with -DRETOPK_PHASE_CLOCKS thread 0 of every CTA stamps the SM clock at
+// phase boundaries into a global table (read back through retopk_debug_read_phases; the
+// benchmark's --phases flag builds such a variant of the library and prints the table).
 #ifdef RETOPK_PHASE_CLOCKS
-__device__ long long g_phase_clk[3][1024][16];
+#define RETOPK_PHASE_SLOTS 24
+__device__ long long g_phase_clk[3][1024][RETOPK_PHASE_SLOTS];
 #define RETOPK_PHASE(kernel, n)                                                            \
     do {                                                                                   \
         if (threadIdx.x == 0 && blockIdx.x < 1024) g_phase_clk[kernel][blockIdx.x][n] = clock64(); \
@@ -43,12 +46,14 @@ namespace retopk {
 constexpr int PATH_REUSE = 0, PATH_FALLBACK = 1, PATH_REFRESH = 2;
 constexpr int MODE_RETOPK = 0, MODE_EXACT = 1;
 
-constexpr int RECALL_THREADS = 1024;
 constexpr int FINISH_THREADS = 1024;
 constexpr int SCAN_THREADS = 256;
 constexpr int SCAN_TILE_ROWS = 256;  // key rows per scan work item
 constexpr int MAX_GROUPS = 4096;     // B * H_kv limit (shared list in scan_kernel)
-constexpr int SCRATCH_WORDS = 2144;  // scratch of the threshold search (2 x 32 x 32 + 96)
+constexpr int SEL_BINS = 2048;       // histogram bins of the threshold search
+constexpr int SEL_LIST = 256;        // members of the boundary bin ranked exhaustively
+constexpr int SCRATCH_WORDS = SEL_BINS + 2 * SEL_LIST + 128;  // bins | boundary list (key, position) | totals
+constexpr int WS_WORDS = 64;         // scratch of the block-wide prefix sums
 constexpr int TILE_ROWS = 16;        // rows per score tile whose maximum the scan records
 
 struct StepArgs {
@@ -67,8 +72,9 @@ struct StepArgs {
     int tile_cap;            // entries in the exact path's list of hit tiles
     int g_shift;             // log2(G) when G is a power of two, else -1
     int step_id;             // call serial number; a KV group is flagged by storing it
-    int stage_depth;         // rows in flight per row slot in reuse_kernel's landing zone
+    int stage_depth;         // rows in flight per row slot in step_kernel's landing zone
     int exact_stage_depth;   // same for exact_finish_kernel
+    int win_prefetch;        // 1: the window's key rows are requested at kernel entry (they fit the landing zone)
     const uint16_t* q;
     const uint16_t* k;
     const uint16_t* v;
@@ -81,6 +87,9 @@ struct StepArgs {
     int32_t* ws_ncand;       // [B*Hq]
     int32_t* ws_sel;         // [B*Hq][r] recalled cache slots, -1 padded
     int32_t* ws_gflag;       // [B*Hkv + 1] == step_id when the group needs a full scan; last word: any group
+    int32_t* ws_xlist;       // [B*Hq] heads on the exact path in this step, in ticket order
+    unsigned int* ws_xcount; // [2] length of that list, by parity of step_id (the other word is cleared for the next step)
+    int32_t* dbg_cand;       // [B*Hq][cap] test hook: candidate list of the last reuse step, or null
     float* ws_scores;        // [B*Hq][score_stride]
     float* ws_tmax;          // [B*Hq][tmax_stride] largest score of every 16-row key tile
     long long tmax_stride;   // multiple of 4
@@ -88,13 +97,11 @@ struct StepArgs {
     unsigned int* status;
     unsigned long long* slow_select;
     unsigned long long* scan_groups;
-    unsigned int* scan_counter;  // pool cursor of scan_kernel; finish_kernel resets it
+    unsigned int* scan_counter;  // pool cursor of scan_kernel; exact_finish_kernel resets it
     int32_t* idx_out;        // MODE_EXACT only, may be null
-    int cl_shift;            // finish_kernel runs 2^cl_shift CTAs (one thread-block cluster) per head
+    int cl_shift;            // step_kernel / exact_finish_kernel run 2^cl_shift CTAs (one thread-block cluster) per head
     // Fusion-ladder levels below the production one (see retopk_ladder.cuh): the reuse path runs
-    // as separate kernels that hand their intermediates on through these global buffers, and
-    // finish_kernel then leaves heads on the reuse path alone.
-    int skip_reuse;
+    // as separate kernels that hand their intermediates on through these global buffers.
     float* lw_rho;           // [B*Hq][M] similarities
     float* lw_qbar;          // [B*Hq][d] normalised query
     int32_t* lw_cand;        // [B*Hq][cap] candidate indices
@@ -188,9 +195,9 @@ __device__ __forceinline__ void store_qbar(const StepArgs& a, size_t off, float 
     else a.qbar_cache[off] = v;
 }
 
-// finish_kernel may give a head a whole thread-block cluster: head and rank of this CTA.
-__device__ __forceinline__ int finish_head(const StepArgs& a) { return (int)(blockIdx.x >> a.cl_shift); }
-__device__ __forceinline__ int finish_rank(const StepArgs& a) { return (int)(blockIdx.x & ((1u << a.cl_shift) - 1u)); }
+// A head may get a whole thread-block cluster: cluster number and rank of this CTA.
+__device__ __forceinline__ int cluster_slot(const StepArgs& a) { return (int)(blockIdx.x >> a.cl_shift); }
+__device__ __forceinline__ int cluster_rank(const StepArgs& a) { return (int)(blockIdx.x & ((1u << a.cl_shift) - 1u)); }
 
 // (sequence, KV head) index of query head bh: bh / G without a division when G is 2^k.
 __device__ __forceinline__ int kv_group_of(int bh, const StepArgs& a) {
@@ -221,6 +228,33 @@ __device__ __forceinline__ int block_excl_scan(int v, int* s_ws, int& total) {
     total = __shfl_sync(0xffffffffu, winc, NT / 32 - 1);
     __syncthreads();
     return wexcl + inc - v;
+}
+
+// Same for two counters at once: .x and .y are scanned side by side (totals may pass 2^16).
+// s_ws: 2 * NT/32 ints.
+template <int NT>
+__device__ __forceinline__ int2 block_excl_scan2(int2 v, int* s_ws, int2& total) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int2 inc = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int tx = __shfl_up_sync(0xffffffffu, inc.x, o), ty = __shfl_up_sync(0xffffffffu, inc.y, o);
+        if (lane >= o) { inc.x += tx; inc.y += ty; }
+    }
+    if (lane == 31) { s_ws[warp] = inc.x; s_ws[NT / 32 + warp] = inc.y; }
+    __syncthreads();
+    const int wx = (lane < NT / 32) ? s_ws[lane] : 0, wy = (lane < NT / 32) ? s_ws[NT / 32 + lane] : 0;
+    int ix = wx, iy = wy;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int tx = __shfl_up_sync(0xffffffffu, ix, o), ty = __shfl_up_sync(0xffffffffu, iy, o);
+        if (lane >= o) { ix += tx; iy += ty; }
+    }
+    const int ex = __shfl_sync(0xffffffffu, ix - wx, warp), ey = __shfl_sync(0xffffffffu, iy - wy, warp);
+    total.x = __shfl_sync(0xffffffffu, ix, NT / 32 - 1);
+    total.y = __shfl_sync(0xffffffffu, iy, NT / 32 - 1);
+    __syncthreads();
+    return make_int2(ex + inc.x - v.x, ey + inc.y - v.y);
 }
 
 // ------------------------------------------------------------------------------------
@@ -374,34 +408,156 @@ __device__ Threshold count_threshold(const uint32_t* key, int n, int K, int low_
     return res;
 }
 
+// Threshold by ONE histogram over the span of the scores.  Key i falls into bin
+// floor((score_i - min) / (max - min) * (SEL_BINS - 1)): a monotone map, so every key in a bin
+// above the bin b* that holds the K-th largest key belongs to the top K, and only b*'s members
+// (a handful when the scores are spread) need ranking.  n > K >= 1.
+//   exact = false: v = the smallest key of the bins b* and above, so at least K keys are >= v
+//                  (a lower bound for the K-th largest key); count = keys >= v.
+//   exact = true : b*'s members are ranked exhaustively by (key desc, position asc): v is the
+//                  K-th largest key and `need` of the keys equal to it belong to the top K;
+//                  count = K + 1 marks that form.  More than SEL_LIST members (heavy ties, an
+//                  outlier that flattens the bins): the radix bisection decides instead.
+// s_h: SCRATCH_WORDS ints.  Every thread returns the same result; kmax = largest key.
+template <int NT>
+__device__ Threshold bin_threshold(const uint32_t* key, int n, int K, bool exact, int* s_h) {
+    constexpr int NW = NT / 32, BPT = SEL_BINS / NT;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    int* s_bl = s_h + SEL_BINS;                      // boundary list: key[SEL_LIST] position[SEL_LIST]
+    int* s_tot = s_h + SEL_BINS + 2 * SEL_LIST;      // [0,32) minima [32,64) maxima [64,96) scan scratch [96,104) results
+    int* s_res = s_tot + 96;
+    uint32_t kmin = 0xffffffffu, kmax = 0u;
+    for (int i = tid; i < n; i += NT) { const uint32_t k = key[i]; kmin = min(kmin, k); kmax = max(kmax, k); }
+    kmin = __reduce_min_sync(0xffffffffu, kmin);
+    kmax = __reduce_max_sync(0xffffffffu, kmax);
+    if (lane == 0) { s_tot[warp] = (int)kmin; s_tot[32 + warp] = (int)kmax; }
+#pragma unroll
+    for (int i = tid; i < SEL_BINS; i += NT) s_h[i] = 0;
+    if (tid == 0) { s_res[3] = 0; s_res[4] = (int)0xffffffffu; }
+    __syncthreads();
+    kmin = __reduce_min_sync(0xffffffffu, lane < NW ? (uint32_t)s_tot[lane] : 0xffffffffu);
+    kmax = __reduce_max_sync(0xffffffffu, lane < NW ? (uint32_t)s_tot[32 + lane] : 0u);
+    Threshold res;
+    res.kmax = kmax;
+    res.v = kmax;
+    res.count = n;
+    res.need = K;
+    if (kmin == kmax) {          // every key equal: v is the K-th largest, the first K in order are taken
+        __syncthreads();
+        return res;
+    }
+    const float smin = key_score(kmin);
+    const float scale = (float)(SEL_BINS - 1) / (key_score(kmax) - smin);
+    auto bin_of = [&](uint32_t k) {
+        const int b = __float2int_rd((key_score(k) - smin) * scale);
+        return min(max(b, 0), SEL_BINS - 1);          // also tames non-finite scores
+    };
+    for (int i = tid; i < n; i += NT) atomicAdd(&s_h[bin_of(key[i])], 1);
+    __syncthreads();
+    // bins from the top: thread t owns bins SEL_BINS-1 - (t*BPT + j)
+    int c[BPT], local = 0;
+#pragma unroll
+    for (int j = 0; j < BPT; ++j) { c[j] = s_h[SEL_BINS - 1 - (tid * BPT + j)]; local += c[j]; }
+    int total;
+    int above = block_excl_scan<NT>(local, s_tot + 64, total);
+    if (above < K && K <= above + local) {            // exactly one thread holds b*
+#pragma unroll
+        for (int j = 0; j < BPT; ++j) {
+            if (K <= above + c[j]) { s_res[0] = SEL_BINS - 1 - (tid * BPT + j); s_res[1] = above; s_res[2] = c[j]; break; }
+            above += c[j];
+        }
+    }
+    __syncthreads();
+    const int bstar = s_res[0], m = s_res[2];
+    above = s_res[1];
+    if (!exact) {
+        uint32_t lo = 0xffffffffu;
+        for (int i = tid; i < n; i += NT) { const uint32_t k = key[i]; if (bin_of(k) == bstar) lo = min(lo, k); }
+        lo = __reduce_min_sync(0xffffffffu, lo);
+        if (lane == 0 && lo != 0xffffffffu) atomicMin(reinterpret_cast<unsigned int*>(&s_res[4]), lo);
+        __syncthreads();
+        res.v = (uint32_t)s_res[4];
+        res.count = above + m;
+        res.need = K - above;
+        __syncthreads();
+        return res;
+    }
+    if (m > SEL_LIST) {
+        __syncthreads();
+        return count_threshold<NT>(key, n, K, 0, s_h);
+    }
+    const int need = K - above;                       // 1..m of b*'s members belong to the top K
+    for (int i = tid; i < n; i += NT) {
+        const uint32_t k = key[i];
+        if (bin_of(k) == bstar) {
+            const int p = atomicAdd(&s_res[3], 1);
+            s_bl[p] = (int)k;
+            s_bl[SEL_LIST + p] = i;
+        }
+    }
+    __syncthreads();
+    if (tid < m) {
+        const uint32_t mine = (uint32_t)s_bl[tid];
+        const int pos = s_bl[SEL_LIST + tid];
+        int gt = 0, eq_before = 0;
+        for (int j = 0; j < m; ++j) {
+            const uint32_t o = (uint32_t)s_bl[j];
+            gt += (int)(o > mine);
+            eq_before += (int)(o == mine) & (int)(s_bl[SEL_LIST + j] < pos);
+        }
+        if (gt + eq_before == need - 1) { s_res[5] = (int)mine; s_res[6] = need - gt; }
+    }
+    __syncthreads();
+    res.v = (uint32_t)s_res[5];
+    res.need = s_res[6];
+    res.count = K + 1;
+    __syncthreads();
+    return res;
+}
+
 // Write, in source order, every element with key > v and the first need_eq elements with
 // key == v into s_sup_idx / s_sup_key.  Source order is ascending index, so the output is
-// the support in ascending index order with ties resolved to the lower index.
+// the support in ascending index order with ties resolved to the lower index.  Every thread
+// takes one contiguous run of the source, so a single prefix sum places them all.
+// s_ws: 64 ints.
 template <int NT, class Src>
 __device__ void ordered_emit(const Src& src, int n, uint32_t vstar, int need_eq, int32_t* s_sup_idx,
                              uint32_t* s_sup_key, int* s_ws) {
     const int tid = threadIdx.x;
-    int gt_run = 0, eq_run = 0;
-    for (int base = 0; base < n; base += NT) {
-        const int i = base + tid;
-        const bool valid = i < n;
-        const uint32_t key = valid ? src.k(i) : 0u;
-        const int fg = valid && key > vstar, fe = valid && key == vstar;
-        int total;
-        const int excl = block_excl_scan<NT>(fg | (fe << 16), s_ws, total);
-        const int g_before = gt_run + (excl & 0xffff), e_before = eq_run + (excl >> 16);
-        if (fg || (fe && e_before < need_eq)) {
-            const int pos = g_before + (e_before < need_eq ? e_before : need_eq);
-            s_sup_idx[pos] = src.x(i);
-            s_sup_key[pos] = key;
+    const int ipt = (n + NT - 1) / NT;                 // NT is a power of two: a shift
+    const int lo = min(n, tid * ipt), hi = min(n, lo + ipt);
+    int2 cnt = make_int2(0, 0);
+    for (int i = lo; i < hi; ++i) {
+        const uint32_t key = src.k(i);
+        cnt.x += (int)(key > vstar);
+        cnt.y += (int)(key == vstar);
+    }
+    int2 total;
+    const int2 excl = block_excl_scan2<NT>(cnt, s_ws, total);
+    int g_before = excl.x, e_before = excl.y;
+    if (cnt.x | cnt.y) {
+        for (int i = lo; i < hi; ++i) {
+            const uint32_t key = src.k(i);
+            if (key > vstar) {
+                const int pos = g_before + (e_before < need_eq ? e_before : need_eq);
+                s_sup_idx[pos] = src.x(i);
+                s_sup_key[pos] = key;
+                ++g_before;
+            } else if (key == vstar) {
+                if (e_before < need_eq) {
+                    const int pos = g_before + e_before;
+                    s_sup_idx[pos] = src.x(i);
+                    s_sup_key[pos] = key;
+                }
+                ++e_before;
+            }
         }
-        gt_run += total & 0xffff;
-        eq_run += total >> 16;
     }
 }
 
 // Top-K of the n listed entries (ascending index order in, ascending index order out).
 // kmax_out: largest listed key when known (n > K), else 0 with *kmax_known = false.
+// s_hist: SCRATCH_WORDS words; s_ws: 64 ints.
 template <int NT>
 __device__ int select_listed(const uint32_t* s_key, const int32_t* s_idx, int n, int K,
                              int32_t* s_sup_idx, uint32_t* s_sup_key, uint32_t* s_hist, int* s_ws,
@@ -414,8 +570,7 @@ __device__ int select_listed(const uint32_t* s_key, const int32_t* s_idx, int n,
         kmax_known = false;
     } else {
         SmemSrc src{s_key, s_idx};
-        int* s_cnt = reinterpret_cast<int*>(s_hist);
-        const Threshold t = count_threshold<NT>(s_key, n, K, 0, s_cnt);
+        const Threshold t = bin_threshold<NT>(s_key, n, K, true, reinterpret_cast<int*>(s_hist));
         uint32_t vstar;
         int need_eq;
         if (t.count == K) { vstar = t.v - 1u; need_eq = 0; }            // exactly K keys are >= v
@@ -588,11 +743,15 @@ __device__ void attend(const uint16_t* vbase, int ns, const int32_t* s_sup_idx, 
 // Pieces of the recall stage (one block per head).
 // ------------------------------------------------------------------------------------
 
-// Eq. 6: rho_c = (qbar_c . q) / |q| for every cached entry c < fill into s_rho[c], and the
-// normalised query into s_q[0..D).  Every warp reads the query itself (four elements per
-// lane) next to its cache rows, so one memory latency covers both.  No barrier at the end.
-template <int D, int NT>
-__device__ __forceinline__ void cache_similarities(const StepArgs& a, int bh, float* s_q, float* s_rho) {
+// Eq. 6: rho_c = (qbar_c . q) / |q| for every cached entry c < fill into s_rho[c], the
+// normalised query into s_q[0..D) and, if asked for, the raw query as floats into s_qraw[0..D).
+// Every warp reads the query itself (four elements per lane) next to its cache rows, so one
+// memory latency covers both.  after_issue() runs once the first trip's loads are on their
+// way (a place to request other rows without delaying these).  No barrier at the end.
+struct NoHook { __device__ __forceinline__ void operator()() const {} };
+template <int D, int NT, class Hook = NoHook>
+__device__ __forceinline__ void cache_similarities(const StepArgs& a, int bh, float* s_q, float* s_rho,
+                                                   float* s_qraw = nullptr, Hook after_issue = Hook()) {
     constexpr int NW = NT / 32;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int M = a.M, fill = a.fill;
@@ -611,6 +770,7 @@ __device__ __forceinline__ void cache_similarities(const StepArgs& a, int bh, fl
                                               : make_float4(0.f, 0.f, 0.f, 0.f);
         }
         if (c0 == warp) {
+            after_issue();
             // first trip: the query norm while the loads fly
             float n2 = q4[0] * q4[0];
             n2 = fmaf(q4[1], q4[1], n2); n2 = fmaf(q4[2], q4[2], n2); n2 = fmaf(q4[3], q4[3], n2);
@@ -621,6 +781,10 @@ __device__ __forceinline__ void cache_similarities(const StepArgs& a, int bh, fl
             if (warp == 0 && lane < D / 4) {
 #pragma unroll
                 for (int e = 0; e < 4; ++e) s_q[4 * lane + e] = nrm > 0.f ? q4[e] / nrm : 0.f;
+                if (s_qraw) {
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) s_qraw[4 * lane + e] = q4[e];
+                }
             }
         }
 #pragma unroll
@@ -688,7 +852,8 @@ __device__ __forceinline__ int decide_path(const StepArgs& a, float rho_max) {
 }
 
 // Leave the decision of one head where the later kernels (and the caller) find it; a head
-// on the exact path flags its KV group for the scan.
+// on the exact path flags its KV group for the scan and takes a ticket in the step's list of
+// exact heads (one atomic add; nobody waits on the list inside this kernel).
 __device__ __forceinline__ void record_decision(const StepArgs& a, int bh, int bkv, const int* s_sel, int path,
                                                 float rho_max) {
     const int tid = threadIdx.x;
@@ -700,82 +865,64 @@ __device__ __forceinline__ void record_decision(const StepArgs& a, int bh, int b
             a.ws_gflag[bkv] = a.step_id;       // same value from every head of the group
             a.ws_gflag[a.B * a.Hkv] = a.step_id;   // "some group needs a scan in this step"
             a.ws_ncand[bh] = a.L;
+            a.ws_xlist[atomicAdd(a.ws_xcount + (a.step_id & 1), 1u)] = bh;
             if (!a.prefill) atomicAdd(a.counters + (size_t)bh * 4 + path, 1ull);   // no return value: not waited for
         }
     }
 }
 
 // ------------------------------------------------------------------------------------
-// recall_kernel: Eq. 6, Eq. 7, Eq. 13 and the insert of the normalised query, per head.
-// Leaves the recalled slots, rho_max and the path in global memory and flags the KV group
-// of every head that takes the exact path.
-// ------------------------------------------------------------------------------------
-template <int D>
-__global__ void __launch_bounds__(RECALL_THREADS, 1) recall_kernel(const StepArgs a) {
-    constexpr int NT = RECALL_THREADS;
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    // layout (words): q[D] rho[M + 3] sel[r] misc[4]
-    float* s_q = reinterpret_cast<float*>(smem_raw);
-    float* s_rho = s_q + D;
-    int* s_sel = reinterpret_cast<int*>(s_rho + ((a.M + 3) & ~3));
-    float* s_misc = reinterpret_cast<float*>(s_sel + a.r);
-
-    const int tid = threadIdx.x;
-    const int bh = blockIdx.x;
-    const int bkv = kv_group_of(bh, a);
-
-    pdl_wait();        // the caches were written by the step before; q by whatever ran before this call
-    RETOPK_PHASE(1, 0);
-    if (tid < a.r) s_sel[tid] = -1;
-    if (tid == 0) s_misc[0] = -CUDART_INF_F;
-    cache_similarities<D, NT>(a, bh, s_q, s_rho);
-    __syncthreads();
-    RETOPK_PHASE(1, 1);
-    const float rho_max = recall_slots<NT>(a, s_rho, s_sel, s_misc);
-    const int path = decide_path(a, rho_max);
-
-    // insert the normalised query now: every similarity of this step has been taken
-    if (tid < D) store_qbar(a, ((size_t)bh * a.M + a.slot) * D + tid, s_q[tid]);
-    record_decision(a, bh, bkv, s_sel, path, rho_max);
-    RETOPK_PHASE(1, 2);
-}
-
-// ------------------------------------------------------------------------------------
 // Pieces of the reuse path (one block per head).
 // ------------------------------------------------------------------------------------
 
-// Eq. 8-9: the sorted unique candidate list of head bh into s_idx; returns its length.
-// Recalled indices below the window go through a bitmap over key positions (ordered
-// extraction = sorted and deduplicated for free); the window itself is a contiguous run
-// appended behind them, whatever the supports held there.  The bitmap must be clear and
-// s_sel loaded (barrier before the call); no barrier at the end.
+// Eq. 8-9, first half: the recalled supports' indices below the window set their bit in a
+// bitmap over key positions (the window is a contiguous run added later, whatever the supports
+// held there).  The bitmap must be clear and s_sel loaded (barrier before the call).  `pre`
+// holds element tid of the first four recalled lists when have_pre (loaded ahead by the caller
+// so that other work overlaps their latency); everything else is loaded here.  No barrier at the end.
 template <int NT>
-__device__ __forceinline__ int candidate_union(const StepArgs& a, int bh, const int* s_sel, int n_sel,
-                                               uint32_t* s_bm, int32_t* s_idx, int* s_ws) {
+__device__ __forceinline__ void union_load_first(const StepArgs& a, int bh, const int* s_sel, int n_sel, int* pre) {
+    const int tid = threadIdx.x;
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+        const int c = u < n_sel ? s_sel[u] : -1;
+        pre[u] = (c >= 0 && tid < a.K) ? a.sup_cache[((size_t)bh * a.M + c) * a.K + tid] : -1;
+    }
+}
+template <int NT>
+__device__ __forceinline__ void union_mark(const StepArgs& a, int bh, const int* s_sel, int n_sel, uint32_t* s_bm,
+                                           const int* pre, bool have_pre) {
     const int tid = threadIdx.x;
     const int M = a.M, L = a.L, K = a.K;
     const int w_lo = L - a.W > 0 ? L - a.W : 0;
-    {
-        bool bad = false;
-        for (int s0 = 0; s0 < n_sel; s0 += 4)
-            for (int i = tid; i < K; i += NT) {
-                int idx[4];
+    bool bad = false;
+    for (int s0 = 0; s0 < n_sel; s0 += 4)
+        for (int i = tid; i < K; i += NT) {
+            int idx[4];
+            const bool use_pre = have_pre && s0 == 0 && i == tid;
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const int c = s0 + u < n_sel ? s_sel[s0 + u] : -1;
-                    idx[u] = c >= 0 ? a.sup_cache[((size_t)bh * M + c) * K + i] : -1;
-                }
-#pragma unroll
-                for (int u = 0; u < 4; ++u)
-                    if (idx[u] >= 0) {
-                        if (idx[u] < w_lo) atomicOr(&s_bm[idx[u] >> 5], 1u << (idx[u] & 31));
-                        else if (idx[u] >= L) bad = true;
-                    }
+            for (int u = 0; u < 4; ++u) {
+                const int c = s0 + u < n_sel ? s_sel[s0 + u] : -1;
+                idx[u] = use_pre ? pre[u] : (c >= 0 ? a.sup_cache[((size_t)bh * M + c) * K + i] : -1);
             }
-        if (bad) atomicOr(a.status, 1u);
-    }
-    __syncthreads();
-    RETOPK_PHASE(0, 4);
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (idx[u] >= 0) {
+                    if (idx[u] < w_lo) atomicOr(&s_bm[idx[u] >> 5], 1u << (idx[u] & 31));
+                    else if (idx[u] >= L) bad = true;
+                }
+        }
+    if (bad) atomicOr(a.status, 1u);
+}
+
+// Eq. 8-9, second half: ordered extraction of the bitmap (sorted and deduplicated for free)
+// into s_idx, the window appended behind as a run; returns the list's length.  The bitmap
+// must be complete (barrier before the call); no barrier at the end.  s_ws: WS_WORDS ints.
+template <int NT>
+__device__ __forceinline__ int union_extract(const StepArgs& a, const uint32_t* s_bm, int32_t* s_idx, int* s_ws) {
+    const int tid = threadIdx.x;
+    const int L = a.L;
+    const int w_lo = L - a.W > 0 ? L - a.W : 0;
     const int nw_lo = (w_lo + 31) >> 5;               // words that can hold bits below the window
     const int wpt = (nw_lo + NT - 1) / NT;
     const int w0 = tid * wpt;
@@ -784,16 +931,28 @@ __device__ __forceinline__ int candidate_union(const StepArgs& a, int bh, const 
     for (int w = w0; w < w1; ++w) cnt += __popc(s_bm[w]);
     int n_low;
     int pos = block_excl_scan<NT>(cnt, s_ws, n_low);
-    for (int w = w0; w < w1; ++w) {
-        uint32_t bits = s_bm[w];
-        while (bits) {
-            const int bit = __ffs(bits) - 1;
-            s_idx[pos++] = w * 32 + bit;
-            bits &= bits - 1;
+    if (cnt)
+        for (int w = w0; w < w1; ++w) {
+            uint32_t bits = s_bm[w];
+            while (bits) {
+                const int bit = __ffs(bits) - 1;
+                s_idx[pos++] = w * 32 + bit;
+                bits &= bits - 1;
+            }
         }
-    }
     for (int i = w_lo + tid; i < L; i += NT) s_idx[n_low + (i - w_lo)] = i;
     return n_low + (L - w_lo);
+}
+
+// Eq. 8-9 in one piece: the sorted unique candidate list of head bh into s_idx; returns its
+// length.  The bitmap must be clear and s_sel loaded (barrier before the call); no barrier at
+// the end.
+template <int NT>
+__device__ __forceinline__ int candidate_union(const StepArgs& a, int bh, const int* s_sel, int n_sel,
+                                               uint32_t* s_bm, int32_t* s_idx, int* s_ws) {
+    union_mark<NT>(a, bh, s_sel, n_sel, s_bm, nullptr, false);
+    __syncthreads();
+    return union_extract<NT>(a, s_bm, s_idx, s_ws);
 }
 
 // Eq. 10: exact current-query scores of n key rows as order-preserving keys into key_out.
@@ -844,24 +1003,76 @@ __device__ __forceinline__ void score_candidates(const uint16_t* kbase, const in
     }
 }
 
+// The recent window's key rows [first_row, first_row + n) requested into the landing zone at
+// kernel entry: row i lands in wave i / SLOTS, row slot i % SLOTS; every lane copies (and later
+// reads back) its own 16 bytes.  One commit group.
+template <int D, int NT>
+__device__ __forceinline__ void window_request(const uint16_t* kbase, int first_row, int n, uint4* s_stage) {
+    constexpr int LPR = D / 8, RPW = 32 / LPR, SLOTS = (NT / 32) * RPW;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int sub = lane % LPR, myslot = warp * RPW + lane / LPR;
+    const char* src = reinterpret_cast<const char*>(kbase) + (size_t)first_row * (D * 2) + sub * 16;
+    uint4* my_stage = s_stage + tid;
+    for (int i = myslot, u = 0; i < n; i += SLOTS, ++u) cp_async16(my_stage + u * NT, src + (size_t)i * (D * 2));
+    cp_async_commit();
+}
+
+// Eq. 10 for the rows window_request brought in (its copies complete: wait before the call):
+// order-preserving score keys into key_out[0..n).  Same per-row arithmetic as score_candidates.
+template <int D, int NT>
+__device__ __forceinline__ void window_score(const uint4* s_stage, int n, const float* s_qraw, float scale,
+                                             uint32_t* key_out) {
+    constexpr int LPR = D / 8, RPW = 32 / LPR, SLOTS = (NT / 32) * RPW;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int sub = lane % LPR, myslot = warp * RPW + lane / LPR;
+    float qf[8];
+    *reinterpret_cast<float4*>(qf) = *reinterpret_cast<const float4*>(s_qraw + sub * 8);
+    *reinterpret_cast<float4*>(qf + 4) = *reinterpret_cast<const float4*>(s_qraw + sub * 8 + 4);
+    const uint4* my_stage = s_stage + tid;
+    for (int u0 = 0; u0 * SLOTS < n; u0 += 8) {
+        float part[8];
+#pragma unroll
+        for (int uu = 0; uu < 8; ++uu) {
+            const int i = (u0 + uu) * SLOTS + myslot;
+            part[uu] = i < n ? dot8(my_stage[(u0 + uu) * NT], qf) : 0.f;
+        }
+        int row;
+        const float tot = reduce8_across<LPR>(part, sub, row);
+        const int i = (u0 + row) * SLOTS + myslot;
+        if ((LPR == 8 || (sub & 1) == 0) && i < n) key_out[i] = score_key(tot * scale);
+    }
+}
+
+// Shared-memory carve-up of step_kernel (the host mirrors it in step_smem_words):
+//   qraw[D] q[D] rho[M+] sel[r+] misc[8] ws[WS_WORDS] hist[SCRATCH_WORDS] sup_idx[K] sup_key[K] w[K] wkey[W+]
+//   | big: idx[cap] key[cap], aliased later by red[NW*D+NT] | bitmap | stage[depth*NT*4]     ("+": rounded up to 4)
+__host__ __device__ inline int step_head_words(int D, int M, int r, int K, int W) {
+    return (2 * D + ((M + 3) & ~3) + ((r + 3) & ~3) + 8 + WS_WORDS + SCRATCH_WORDS + 3 * K + ((W + 3) & ~3) + 3) & ~3;
+}
+
 // ------------------------------------------------------------------------------------
-// reuse path of finish_kernel: candidate union (Eq. 8-9), candidate scores (Eq. 10), Top-K
-// (Eq. 11), softmax.V (Eq. 12) and the support insert for one head, all in shared memory.
+// step_kernel: the recall stage for every head (Eq. 6, Eq. 7, Eq. 13, insert of the normalised
+// query) and, for a head that reuses, the whole rest of the step in the same CTA: candidate
+// union (Eq. 8-9), candidate scores (Eq. 10), Top-K (Eq. 11), softmax.V (Eq. 12), support
+// insert; candidate list and scores never leave shared memory.  A head on the exact path
+// leaves after the recall stage; scan_kernel and exact_finish_kernel serve it.
 // ------------------------------------------------------------------------------------
 template <int D, int NT>
-__device__ void reuse_path(const StepArgs& a, unsigned char* smem_raw) {
+__global__ void __launch_bounds__(NT, 1024 / NT) step_kernel(const StepArgs a) {
     constexpr int NW = NT / 32;
-    // layout (words): qraw[D] sel[r] ws[32] hist[SCRATCH_WORDS] sup_idx[K] sup_key[K] w[K]
-    //                 | big: idx[cap] key[cap], aliased later by red[NW*D+NT] | bitmap | stage[depth*NT*4]
+    extern __shared__ __align__(16) unsigned char smem_raw[];
     float* s_qraw = reinterpret_cast<float*>(smem_raw);
-    int* s_sel = reinterpret_cast<int*>(s_qraw + D);
-    int* s_ws = s_sel + a.r;
-    uint32_t* s_hist = reinterpret_cast<uint32_t*>(s_ws + 32);
+    float* s_q = s_qraw + D;
+    float* s_rho = s_q + D;
+    int* s_sel = reinterpret_cast<int*>(s_rho + ((a.M + 3) & ~3));
+    float* s_misc = reinterpret_cast<float*>(s_sel + ((a.r + 3) & ~3));
+    int* s_ws = reinterpret_cast<int*>(s_misc + 8);
+    uint32_t* s_hist = reinterpret_cast<uint32_t*>(s_ws + WS_WORDS);
     int32_t* s_sup_idx = reinterpret_cast<int32_t*>(s_hist + SCRATCH_WORDS);
     uint32_t* s_sup_key = reinterpret_cast<uint32_t*>(s_sup_idx + a.K);
     float* s_w = reinterpret_cast<float*>(s_sup_key + a.K);
-    const int head_words = (D + a.r + 32 + SCRATCH_WORDS + 3 * a.K + 3) & ~3;
-    int32_t* s_idx = reinterpret_cast<int32_t*>(smem_raw) + head_words;
+    uint32_t* s_wkey = reinterpret_cast<uint32_t*>(s_w + a.K);
+    int32_t* s_idx = reinterpret_cast<int32_t*>(smem_raw) + step_head_words(D, a.M, a.r, a.K, a.W);
     uint32_t* s_key = reinterpret_cast<uint32_t*>(s_idx + a.cap);
     float* s_red = reinterpret_cast<float*>(s_idx);
     const int big_words = (max(2 * a.cap, NW * D + NT) + 3) & ~3;
@@ -869,48 +1080,82 @@ __device__ void reuse_path(const StepArgs& a, unsigned char* smem_raw) {
     uint4* s_stage = reinterpret_cast<uint4*>(s_bm + ((((int)a.max_seq_len + 31) / 32 + 3) & ~3));
 
     const int tid = threadIdx.x;
-    const int bh = finish_head(a);
-    const int cl_rank = finish_rank(a), cl_size = 1 << a.cl_shift;
+    const int bh = cluster_slot(a);
+    const int cl_rank = cluster_rank(a), cl_size = 1 << a.cl_shift;
     const int bkv = kv_group_of(bh, a);
     const int M = a.M, fill = a.fill, L = a.L, K = a.K;
     const int n_sel = a.r < fill ? a.r : fill;
-    RETOPK_PHASE(0, 0);
-    // peers write into this CTA's shared memory later on: all of them must be running by then
-    if (cl_size > 1) cooperative_groups::this_cluster().sync();
+    const int w_lo = L - a.W > 0 ? L - a.W : 0, wn = L - w_lo;
+    const uint16_t* kbase = a.k + (size_t)bkv * a.max_seq_len * D;
+    const bool may_reuse = !a.refresh && fill > 0;          // known on the host: else every head is exact
+    const bool prefetch = may_reuse && a.win_prefetch && cl_size == 1;
 
-    // recalled slots and the raw query from global memory; clear the bitmap meanwhile
-    if (tid < a.r) s_sel[tid] = a.ws_sel[(size_t)bh * a.r + tid];
-    if (tid >= 32 && tid < 32 + D / 2) {
-        const uint32_t raw = reinterpret_cast<const uint32_t*>(a.q + (size_t)bh * D)[tid - 32];
-        s_qraw[2 * (tid - 32)] = bf16_lo(raw);
-        s_qraw[2 * (tid - 32) + 1] = bf16_hi(raw);
-    }
-    {
+    // nothing before the wait depends on an earlier kernel
+    if (tid < a.r) s_sel[tid] = -1;
+    if (tid == 0) s_misc[0] = -CUDART_INF_F;
+    if (may_reuse) {
         const int nwords = (L + 31) >> 5;
         uint4* bm4 = reinterpret_cast<uint4*>(s_bm);
         for (int w = tid; w < (nwords + 3) >> 2; w += NT) bm4[w] = make_uint4(0, 0, 0, 0);
     }
+    pdl_wait();        // the caches were written by the step before; q by whatever ran before this call
+    RETOPK_PHASE(1, 0);
+
+    // ---- recall stage: Eq. 6, Eq. 7, Eq. 13, insert of the normalised query
+    cache_similarities<D, NT>(a, bh, s_q, s_rho, s_qraw,
+                              [&]() { if (prefetch) window_request<D, NT>(kbase, w_lo, wn, s_stage); });
+    __syncthreads();
+    RETOPK_PHASE(1, 1);
+    const float rho_max = recall_slots<NT>(a, s_rho, s_sel, s_misc);
+    const int path = decide_path(a, rho_max);
+    if (cl_rank == 0) {
+        // every similarity of this step has been taken: the slot may be overwritten
+        if (tid < D) store_qbar(a, ((size_t)bh * M + a.slot) * D + tid, s_q[tid]);
+        record_decision(a, bh, bkv, s_sel, path, rho_max);
+    }
+    RETOPK_PHASE(1, 2);
+    if (path != PATH_REUSE) {
+        cp_async_wait_all();       // no copy may land in shared memory this CTA has given up
+        return;
+    }
+
+    // ---- reuse path
+    RETOPK_PHASE(0, 0);
+    // peers write into this CTA's shared memory later on: all of them must be running by then
+    if (cl_size > 1) cooperative_groups::this_cluster().sync();
+
+    // Eq. 8-9.  The first recalled lists are requested, then the window rows (long arrived)
+    // are scored while those lists travel.
+    int pre[4];
+    union_load_first<NT>(a, bh, s_sel, n_sel, pre);
+    if (prefetch) {
+        cp_async_wait_all();
+        window_score<D, NT>(s_stage, wn, s_qraw, a.scale, s_wkey);
+    }
+    RETOPK_PHASE(0, 1);
+    union_mark<NT>(a, bh, s_sel, n_sel, s_bm, pre, true);
+    __syncthreads();
+    RETOPK_PHASE(0, 2);
+    const int n = union_extract<NT>(a, s_bm, s_idx, s_ws);
+    const int n_low = n - wn;
+    if (prefetch)
+        for (int j = tid; j < wn; j += NT) s_key[n_low + j] = s_wkey[j];
     __syncthreads();
     RETOPK_PHASE(0, 3);
-
-    // Eq. 8-9
-    const int n = candidate_union<NT>(a, bh, s_sel, n_sel, s_bm, s_idx, s_ws);
-    __syncthreads();
-    RETOPK_PHASE(0, 5);
+    if (a.dbg_cand && cl_rank == 0)
+        for (int i = tid; i < n; i += NT) a.dbg_cand[(size_t)bh * a.cap + i] = s_idx[i];
 
     // Eq. 10.  In a cluster every CTA built the same list; each scores a contiguous share of
     // it and hands the keys to the others through distributed shared memory.
     if (cl_size == 1) {
-        score_candidates<D, NT, true>(a.k + (size_t)bkv * a.max_seq_len * D, s_idx, n, s_qraw, s_stage,
-                                      a.stage_depth, a.scale, s_key);
+        score_candidates<D, NT, true>(kbase, s_idx, prefetch ? n_low : n, s_qraw, s_stage, a.stage_depth, a.scale, s_key);
         __syncthreads();
     } else {
         namespace cg = cooperative_groups;
         cg::cluster_group cluster = cg::this_cluster();
         const int share = (n + cl_size - 1) / cl_size;
         const int lo = min(n, cl_rank * share), hi = min(n, lo + share);
-        score_candidates<D, NT, true>(a.k + (size_t)bkv * a.max_seq_len * D, s_idx + lo, hi - lo, s_qraw, s_stage,
-                                      a.stage_depth, a.scale, s_key + lo);
+        score_candidates<D, NT, true>(kbase, s_idx + lo, hi - lo, s_qraw, s_stage, a.stage_depth, a.scale, s_key + lo);
         __syncthreads();
         for (int r = 1; r < cl_size; ++r) {
             uint32_t* peer = cluster.map_shared_rank(s_key, (cl_rank + r) & (cl_size - 1));
@@ -918,13 +1163,13 @@ __device__ void reuse_path(const StepArgs& a, unsigned char* smem_raw) {
         }
         cluster.sync();
     }
-    RETOPK_PHASE(0, 6);
+    RETOPK_PHASE(0, 4);
 
     // Eq. 11: Top-K of the candidates; insert the support
     uint32_t kmax;
     bool kmax_known;
     const int ns = select_listed<NT>(s_key, s_idx, n, K, s_sup_idx, s_sup_key, s_hist, s_ws, kmax, kmax_known);
-    RETOPK_PHASE(0, 7);
+    RETOPK_PHASE(0, 5);
     if (cl_rank == 0) {
         int32_t* sup_out = a.sup_cache + ((size_t)bh * M + a.slot) * K;
         for (int i = tid; i < K; i += NT) sup_out[i] = i < ns ? s_sup_idx[i] : -1;
@@ -938,7 +1183,7 @@ __device__ void reuse_path(const StepArgs& a, unsigned char* smem_raw) {
         atomicAdd(a.counters + (size_t)bh * 4 + PATH_REUSE, 1ull);
         atomicAdd(a.counters + (size_t)bh * 4 + 3, (unsigned long long)n);
     }
-    RETOPK_PHASE(0, 8);
+    RETOPK_PHASE(0, 6);
 }
 
 // ------------------------------------------------------------------------------------
@@ -1117,12 +1362,11 @@ __global__ void __launch_bounds__(SCAN_THREADS) scan_kernel(const StepArgs a) {
 // lower-index tie rule is taken from that list.
 // ------------------------------------------------------------------------------------
 template <int D, int NT>
-__device__ void exact_path(const StepArgs& a, unsigned char* smem_raw) {
+__device__ void exact_path(const StepArgs& a, int bh, unsigned char* smem_raw) {
     // In a cluster every CTA of a head selects the same support on its own (the lists are short
     // and come from L2); only the value rows are shared out, and rank 0 writes the results.
-    const int bh = finish_head(a);
-    const int cl_rank = finish_rank(a), cl_size = 1 << a.cl_shift;
-    // layout (words): sup_idx[K] sup_key[K] w[K] cnt[SCRATCH_WORDS] ws[32] misc[8]
+    const int cl_rank = cluster_rank(a), cl_size = 1 << a.cl_shift;
+    // layout (words): sup_idx[K] sup_key[K] w[K] cnt[SCRATCH_WORDS] ws[WS_WORDS] misc[8]
     //                 | lists: key[NS] idx[NS] tile[tile_cap]; dead once the support is emitted and
     //                   then reused by attend: red[NW*D+NT], stage[depth*NT*4] (may run past the lists)
     constexpr int NW = NT / 32;
@@ -1131,8 +1375,8 @@ __device__ void exact_path(const StepArgs& a, unsigned char* smem_raw) {
     float* s_w = reinterpret_cast<float*>(s_sup_key + a.K);
     uint32_t* s_hist = reinterpret_cast<uint32_t*>(s_w + a.K);
     int* s_ws = reinterpret_cast<int*>(s_hist + SCRATCH_WORDS);
-    int* s_misc = s_ws + 32;
-    uint32_t* s_key = reinterpret_cast<uint32_t*>(smem_raw) + ((3 * a.K + SCRATCH_WORDS + 32 + 8 + 3) & ~3);
+    int* s_misc = s_ws + WS_WORDS;
+    uint32_t* s_key = reinterpret_cast<uint32_t*>(smem_raw) + ((3 * a.K + SCRATCH_WORDS + WS_WORDS + 8 + 3) & ~3);
     int32_t* s_idx = reinterpret_cast<int32_t*>(s_key + a.NS);
     int32_t* s_tile = s_idx + a.NS;
     float* s_red = reinterpret_cast<float*>(s_key);
@@ -1193,7 +1437,7 @@ __device__ void exact_path(const StepArgs& a, unsigned char* smem_raw) {
                 s_key[i2] = score_key(m);
             }
             __syncthreads();
-            thr_key = count_threshold<NT>(s_key, n2, K, 16, reinterpret_cast<int*>(s_hist)).v;
+            thr_key = n2 > K ? bin_threshold<NT>(s_key, n2, K, false, reinterpret_cast<int*>(s_hist)).v : 0u;
         }
         RETOPK_PHASE(2, 1);
         // 2. the tiles whose maximum reaches v, in ascending order: eight consecutive tile
@@ -1287,20 +1531,24 @@ __device__ void exact_path(const StepArgs& a, unsigned char* smem_raw) {
 }
 
 // ------------------------------------------------------------------------------------
-// finish_kernel: one CTA per (sequence, query head), launched behind the scan.  A head on
-// the reuse path never waited for the scan's results, a head on the exact path selects from
-// them; both end with softmax.V and the support insert.  Heads of one step run side by side.
+// exact_finish_kernel: launched behind the scan with one CTA (or cluster) per head; cluster
+// number i serves the i-th head of the step's list of exact heads and the rest leave at once
+// (the list's length is only known on the device).  For Exact Top-K attention every head is
+// served.  Which CTA serves a head does not matter to its result.
 // ------------------------------------------------------------------------------------
 template <int D, int NT>
-__global__ void __launch_bounds__(NT, 1024 / NT) finish_kernel(const StepArgs a) {
+__global__ void __launch_bounds__(NT, 1024 / NT) exact_finish_kernel(const StepArgs a) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    pdl_wait();        // scores and tile maxima come from the scan, recalled slots and paths from recall_kernel
-    if (blockIdx.x == 0 && threadIdx.x == 0) *a.scan_counter = 0u;      // the scan before this kernel is complete
-    if (a.mode == MODE_RETOPK && a.ws_path[finish_head(a)] == PATH_REUSE) {
-        if (!a.skip_reuse) reuse_path<D, NT>(a, smem_raw);
-    } else {
-        exact_path<D, NT>(a, smem_raw);
+    pdl_wait();        // scores and tile maxima come from the scan, the list from step_kernel
+    int n_listed = a.B * a.Hq;
+    if (a.mode == MODE_RETOPK) n_listed = (int)a.ws_xcount[a.step_id & 1];
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        *a.scan_counter = 0u;                                   // the scan before this kernel is complete
+        if (a.mode == MODE_RETOPK) a.ws_xcount[(a.step_id + 1) & 1] = 0u;   // the next step's list starts empty
     }
+    const int slot = cluster_slot(a);
+    if (slot >= n_listed) return;
+    exact_path<D, NT>(a, a.mode == MODE_RETOPK ? a.ws_xlist[slot] : slot, smem_raw);
 }
 
 // Host-buffer entry point, when the caller's buffers are pinned and mapped: one launch reads
@@ -1339,14 +1587,15 @@ __global__ void narrow_kernel(const float* src, uint16_t* dst, size_t n) {
 // Clear the caches (supports to -1, queries and counters to 0).
 __global__ void reset_kernel(float* qbar, size_t n_q, int32_t* sup, size_t n_sup, unsigned long long* counters,
                              size_t n_cnt, int32_t* gflag, size_t n_flag, unsigned int* status,
-                             unsigned long long* slow, unsigned long long* groups, unsigned int* scan_counter) {
+                             unsigned long long* slow, unsigned long long* groups, unsigned int* scan_counter,
+                             unsigned int* xcount) {
     const size_t stride = (size_t)gridDim.x * blockDim.x;
     const size_t t0 = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     for (size_t i = t0; i < n_q; i += stride) qbar[i] = 0.f;
     for (size_t i = t0; i < n_sup; i += stride) sup[i] = -1;
     for (size_t i = t0; i < n_cnt; i += stride) counters[i] = 0;
     for (size_t i = t0; i < n_flag; i += stride) gflag[i] = -1;
-    if (t0 == 0) { *status = 0u; *slow = 0ull; *groups = 0ull; *scan_counter = 0u; }
+    if (t0 == 0) { *status = 0u; *slow = 0ull; *groups = 0ull; *scan_counter = 0u; xcount[0] = 0u; xcount[1] = 0u; }
 }
 
 }  // namespace retopk

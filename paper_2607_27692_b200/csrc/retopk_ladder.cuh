@@ -9,12 +9,12 @@
 //   level 3  selection, sparse output and cache update fused into one kernel
 //   level 4  as level 3, with the intermediate buffers kept by the context instead of being
 //            allocated from a stream-ordered pool in every step (a host-side difference)
-//   level 5  candidate construction through output in one kernel: recall_kernel +
-//            finish_kernel, the production path
+//   level 5  candidate construction through output in one kernel: step_kernel, the
+//            production path
 //
 // Every level runs the same device functions on the same lanes as the production path, so
 // supports and outputs are bit-identical across levels.  Heads on the exact path are served
-// by scan_kernel + finish_kernel at every level.  One block of LADDER_THREADS per head.
+// by scan_kernel + exact_finish_kernel at every level.  One block of LADDER_THREADS per head.
 #pragma once
 
 #include "retopk_kernels.cuh"
@@ -57,7 +57,7 @@ __global__ void __launch_bounds__(LADDER_THREADS, 1) ladder_topr_kernel(const St
     record_decision(a, bh, kv_group_of(bh, a), s_sel, decide_path(a, rho_max), rho_max);
 }
 
-// Shared-memory carve-up of the union: sel[r] ws[32] | idx[cap] | bitmap
+// Shared-memory carve-up of the union: sel[r] ws[WS_WORDS] | idx[cap] | bitmap
 struct UnionSmem {
     int* sel;
     int* ws;
@@ -68,7 +68,7 @@ __device__ __forceinline__ UnionSmem union_smem(const StepArgs& a, unsigned char
     UnionSmem u;
     u.sel = reinterpret_cast<int*>(base);
     u.ws = u.sel + ((a.r + 3) & ~3);
-    u.idx = u.ws + 32;
+    u.idx = u.ws + WS_WORDS;
     u.bm = reinterpret_cast<uint32_t*>(u.idx + ((a.cap + 3) & ~3));
     return u;
 }
@@ -87,6 +87,8 @@ __device__ __forceinline__ void union_to_global(const StepArgs& a, int bh, const
     const int n = candidate_union<NT>(a, bh, u.sel, n_sel, u.bm, u.idx, u.ws);
     __syncthreads();
     for (int i = tid; i < n; i += NT) a.lw_cand[(size_t)bh * a.cap + i] = u.idx[i];
+    if (a.dbg_cand)
+        for (int i = tid; i < n; i += NT) a.dbg_cand[(size_t)bh * a.cap + i] = u.idx[i];
     if (tid == 0) a.ws_ncand[bh] = n;
 }
 
@@ -144,9 +146,9 @@ __global__ void __launch_bounds__(LADDER_THREADS, 1) ladder_score_kernel(const S
 __global__ void __launch_bounds__(LADDER_THREADS, 1) ladder_select_kernel(const StepArgs a) {
     constexpr int NT = LADDER_THREADS;
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    // layout (words): ws[32] hist[SCRATCH_WORDS] sup_idx[K] sup_key[K] idx[cap] key[cap]
+    // layout (words): ws[WS_WORDS] hist[SCRATCH_WORDS] sup_idx[K] sup_key[K] idx[cap] key[cap]
     int* s_ws = reinterpret_cast<int*>(smem_raw);
-    uint32_t* s_hist = reinterpret_cast<uint32_t*>(s_ws + 32);
+    uint32_t* s_hist = reinterpret_cast<uint32_t*>(s_ws + WS_WORDS);
     int32_t* s_sup_idx = reinterpret_cast<int32_t*>(s_hist + SCRATCH_WORDS);
     uint32_t* s_sup_key = reinterpret_cast<uint32_t*>(s_sup_idx + a.K);
     int32_t* s_idx = reinterpret_cast<int32_t*>(s_sup_key + a.K);
@@ -178,12 +180,12 @@ template <int D>
 __global__ void __launch_bounds__(LADDER_THREADS, 1) ladder_attend_kernel(const StepArgs a) {
     constexpr int NT = LADDER_THREADS, NW = NT / 32;
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    // layout (words): ws[32] sup_idx[K] sup_key[K] w[K] red[NW*D+NT] | stage[depth*NT*4]
+    // layout (words): ws[WS_WORDS] sup_idx[K] sup_key[K] w[K] red[NW*D+NT] | stage[depth*NT*4]
     int* s_ws = reinterpret_cast<int*>(smem_raw);
-    int32_t* s_sup_idx = reinterpret_cast<int32_t*>(s_ws + 32);
+    int32_t* s_sup_idx = reinterpret_cast<int32_t*>(s_ws + WS_WORDS);
     uint32_t* s_sup_key = reinterpret_cast<uint32_t*>(s_sup_idx + a.K);
     float* s_w = reinterpret_cast<float*>(s_sup_key + a.K);
-    float* s_red = reinterpret_cast<float*>(s_ws + 32 + ((3 * a.K + 3) & ~3));
+    float* s_red = reinterpret_cast<float*>(s_ws + WS_WORDS + ((3 * a.K + 3) & ~3));
     uint4* s_stage = reinterpret_cast<uint4*>(s_red + NW * D + NT);
     const int tid = threadIdx.x, bh = blockIdx.x;
     if (a.ws_path[bh] != PATH_REUSE) return;
@@ -218,7 +220,7 @@ __global__ void __launch_bounds__(LADDER_THREADS, 1) ladder_insert_kernel(const 
 
 // ---- level 2 --------------------------------------------------------------------------
 
-// Cache search and support union in one kernel: recall_kernel's work, then Eq. 8-9 for a
+// Cache search and support union in one kernel: the recall stage, then Eq. 8-9 for a
 // head that stays on the reuse path.
 template <int D>
 __global__ void __launch_bounds__(LADDER_THREADS, 1) ladder_discover_kernel(const StepArgs a) {
@@ -248,14 +250,14 @@ template <int D>
 __global__ void __launch_bounds__(LADDER_THREADS, 1) ladder_select_attend_insert_kernel(const StepArgs a) {
     constexpr int NT = LADDER_THREADS, NW = NT / 32;
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    // layout (words): ws[32] hist[SCRATCH_WORDS] sup_idx[K] sup_key[K] w[K]
+    // layout (words): ws[WS_WORDS] hist[SCRATCH_WORDS] sup_idx[K] sup_key[K] w[K]
     //                 | big: idx[cap] key[cap], aliased later by red[NW*D+NT] | stage[depth*NT*4]
     int* s_ws = reinterpret_cast<int*>(smem_raw);
-    uint32_t* s_hist = reinterpret_cast<uint32_t*>(s_ws + 32);
+    uint32_t* s_hist = reinterpret_cast<uint32_t*>(s_ws + WS_WORDS);
     int32_t* s_sup_idx = reinterpret_cast<int32_t*>(s_hist + SCRATCH_WORDS);
     uint32_t* s_sup_key = reinterpret_cast<uint32_t*>(s_sup_idx + a.K);
     float* s_w = reinterpret_cast<float*>(s_sup_key + a.K);
-    const int head_words = (32 + SCRATCH_WORDS + 3 * a.K + 3) & ~3;
+    const int head_words = (WS_WORDS + SCRATCH_WORDS + 3 * a.K + 3) & ~3;
     int32_t* s_idx = reinterpret_cast<int32_t*>(smem_raw) + head_words;
     uint32_t* s_key = reinterpret_cast<uint32_t*>(s_idx + a.cap);
     float* s_red = reinterpret_cast<float*>(s_idx);

@@ -51,6 +51,9 @@ SIGNATURES = {
     "retopk_stats": (_i32, [_vp, C.POINTER(_Stats)]),
     "retopk_last_step": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp]),
     "retopk_last_recall": (_i32, [_vp, _vp, _vp]),
+    "retopk_debug_candidates": (_i32, [_vp, _i32]),
+    "retopk_last_candidates": (_i32, [_vp, _vp, _vp]),
+    "retopk_debug_fail_next_launch": (_i32, [_vp, _i32]),
     "retopk_export_state": (_i32, [_vp, _vp, _vp, C.POINTER(_i64), C.POINTER(_i64), _vp]),
     "retopk_import_state": (_i32, [_vp, _vp, _vp, _i64, _i64, _vp]),
     "retopk_profile_begin": (_i32, [_vp, _i32]),
@@ -156,11 +159,11 @@ class ReTopK:
         _check(self.lib.retopk_set_qbar_format(self.h, fmt), "retopk_set_qbar_format")
 
     def set_cluster_size(self, ctas_per_head: int):
-        """CTAs (one SM each) per head in the finish kernel: 1, 2, 4 or 8."""
+        """CTAs (one SM each) per head in the per-head kernels: 1, 2, 4 or 8."""
         _check(self.lib.retopk_set_cluster_size(self.h, ctas_per_head), "retopk_set_cluster_size")
 
     def set_finish_threads(self, threads: int):
-        """Block shape of the finish kernel: 1024 (one CTA per SM) or 512 (two per SM)."""
+        """Block shape of the per-head kernels: 1024 (one CTA per SM) or 512 (two per SM)."""
         _check(self.lib.retopk_set_finish_threads(self.h, threads), "retopk_set_finish_threads")
 
     def set_fusion_level(self, level: int, dependent_launches: bool = False):
@@ -232,6 +235,16 @@ class ReTopK:
         _check(self.lib.retopk_last_recall(self.h, sel.data_ptr(), _stream()), "retopk_last_recall")
         return sel
 
+    def debug_candidates(self, enable: bool = True):
+        """Test hook: keep the candidate list (Eq. 9) of every head that reuses."""
+        _check(self.lib.retopk_debug_candidates(self.h, int(enable)), "retopk_debug_candidates")
+
+    def last_candidates(self):
+        """[B, H_q, r*K+W] int32: per reuse head of the last step, its first n_cand entries are the list."""
+        cand = torch.empty((self.B, self.H_q, self.r * self.K + self.W), dtype=torch.int32, device=self.device)
+        _check(self.lib.retopk_last_candidates(self.h, cand.data_ptr(), _stream()), "retopk_last_candidates")
+        return cand
+
     def export_state(self):
         dev = self.device
         qbar = torch.empty((self.B, self.H_q, self.M, self.d), dtype=torch.float32, device=dev)
@@ -255,7 +268,7 @@ class ReTopK:
         ms, n = (C.c_double * 3)(), (_i64 * 3)()
         _check(self.lib.retopk_profile_end(self.h, ms, n), "retopk_profile_end")
         return {name: dict(ms=float(ms[i]), launches=int(n[i]))
-                for i, name in enumerate(("recall", "scan", "finish"))}
+                for i, name in enumerate(("step", "scan", "finish"))}
 
     def last_launch_count(self) -> int:
         return int(self.lib.retopk_last_launch_count(self.h))

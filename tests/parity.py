@@ -40,19 +40,52 @@ def assert_support_matches(sup_gpu, sup_ref, q_bits, k_head_bits, kth_score, wha
     return len(diff)
 
 
+def synthetic_full_state(oracle, st, L0, rng, n_inserted=None, spread=0.35, dup_slots=()):
+    """A cache that is full before the first step: written into the oracle (import it into the
+    GPU context from there).  Cached queries are noisy unit-norm copies of the stream's first
+    queries (so that similarities spread around typical thresholds), supports are sorted random
+    index sets below ``L0``.  ``dup_slots``: pairs (a, b) of slots made identical, which ties
+    their similarities exactly.  ``n_inserted`` >= M places the ring's write position."""
+    B, H, M, d, K = oracle.B, oracle.H_q, oracle.M, oracle.d, oracle.K
+    q0 = wl.bf16_bits_to_f64(st.q[0])                       # [B, H, d]
+    q0 = q0 / np.maximum(np.linalg.norm(q0, axis=-1, keepdims=True), 1e-30)
+    qbar = q0[:, :, None, :] + spread * rng.standard_normal((B, H, M, d)) / np.sqrt(d) * np.linspace(0.2, 4.0, M)[None, None, :, None]
+    qbar /= np.linalg.norm(qbar, axis=-1, keepdims=True)
+    sup = np.empty((B, H, M, K), dtype=np.int32)
+    for b in range(B):
+        for h in range(H):
+            for c in range(M):
+                n = min(K, L0)
+                row = np.sort(rng.choice(L0, size=n, replace=False)).astype(np.int32)
+                sup[b, h, c, :n] = row
+                sup[b, h, c, n:] = -1
+    for a, b_ in dup_slots:
+        qbar[:, :, b_] = qbar[:, :, a]
+    if oracle_is_bf16(oracle):
+        qbar = wl.bf16_bits_to_f64(wl.f32_to_bf16_bits(qbar.astype(np.float32)))
+    oracle.import_state(qbar, sup, M + M // 2 if n_inserted is None else n_inserted, 0)
+
+
+def oracle_is_bf16(oracle):
+    return bool(getattr(oracle, "qbar_bf16", False))
+
+
 def teacher_forced_run(cfg, st, steps, oracle, gpu, k_dev, v_dev, b_map=None, check_out=True,
-                       full_stream=None):
+                       full_stream=None, check_candidates=True):
     """Step both sides with the GPU caches re-seeded from the oracle before every step.
 
     ``oracle`` may cover a subset of the GPU's sequences: ``b_map[i]`` is the GPU batch row of
     oracle row ``i`` (the stream ``st`` then holds the oracle's rows, ``full_stream`` the
-    queries of every GPU sequence).  Returns counts of excused events.
+    queries of every GPU sequence).  With ``check_candidates`` the candidate list (Eq. 9) of
+    every head that reuses is compared element by element.  Returns counts of excused events.
     """
     G = cfg.H_q // cfg.H_kv
     b_map = list(range(oracle.B)) if b_map is None else b_map
     full = len(b_map) == gpu.B
     excused_flips = excused_pos = 0
     q_full = None
+    if check_candidates:
+        gpu.debug_candidates(True)
     for t in range(steps):
         L = st.seq_len(t)
         qbar, sup, n_ins, t_dec = oracle.export_state()
@@ -80,6 +113,7 @@ def teacher_forced_run(cfg, st, steps, oracle, gpu, k_dev, v_dev, b_map=None, ch
         g_sup = lg["support"].cpu().numpy()
         g_rho = lg["rho_max"].cpu().numpy()
         g_nc = lg["n_cand"].cpu().numpy()
+        g_cand = gpu.last_candidates().cpu().numpy() if check_candidates else None
         for i, b in enumerate(b_map):
             for h in range(cfg.H_q):
                 what = f"step {t} seq {b} head {h}"
@@ -95,6 +129,9 @@ def teacher_forced_run(cfg, st, steps, oracle, gpu, k_dev, v_dev, b_map=None, ch
                     continue
                 if lo["path"][i, h] == 0:
                     assert g_nc[b, h] == lo["n_cand"][i, h], f"{what}: n_cand"
+                    if check_candidates:
+                        want = oracle.last_candidates(i, h)
+                        assert np.array_equal(g_cand[b, h, :len(want)], want), f"{what}: candidate list"
                 excused_pos += assert_support_matches(
                     g_sup[b, h], lo["support"][i, h], st.q[t, i, h], st.k[i, h // G],
                     lo["kth_score"][i, h], what)

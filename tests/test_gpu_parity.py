@@ -431,3 +431,34 @@ def test_bf16_query_cache_free_running_and_argument_checks(rt, P, oracle_mod):
     g.reset()
     assert lib.retopk_set_qbar_format(g.h, 2) == -1
     assert lib.retopk_set_qbar_format(g.h, 0) == 0
+
+
+def test_failed_launch_in_mid_step_is_sticky_until_reset(rt, P, oracle_mod):
+    """A launch that fails after the step's first kernel went out leaves the caches half
+    advanced: the step and every later one report the failure until the context is reset
+    (the failure is injected on the host; no kernel misbehaves)."""
+    cfg = wl.CONFIGS["tiny"].replace(B=1, H_q=2, H_kv=1, context=600, steps=12)
+    st, o, g, k, v = stream_case(rt, P, oracle_mod, cfg, 12)
+    lib = rt.load()
+    q = [P.to_dev(st.q[t]) for t in range(12)]
+    for t in range(3):
+        g.decode_step(q[t], k, v, st.seq_len(t))
+    # a failure of the FIRST launch leaves nothing enqueued: the context stays usable
+    assert lib.retopk_debug_fail_next_launch(g.h, 1) == 0
+    with pytest.raises(rt.RetopkError):
+        g.decode_step(q[3], k, v, st.seq_len(3))
+    g.decode_step(q[3], k, v, st.seq_len(3))
+    assert g.export_state()[2] == 4
+    # a failure of the scan or finish launch is sticky
+    for which in (2, 3):
+        assert lib.retopk_debug_fail_next_launch(g.h, which) == 0
+        with pytest.raises(rt.RetopkError):
+            g.decode_step(q[4], k, v, st.seq_len(4))
+        with pytest.raises(rt.RetopkError):
+            g.decode_step(q[4], k, v, st.seq_len(4))
+        g.reset()
+        torch.cuda.synchronize()
+        # after the reset the context runs the stream again and agrees with the oracle
+        o.reset()
+        P.teacher_forced_run(cfg, st, 8, o, g, k, v)
+    assert lib.retopk_debug_fail_next_launch(g.h, 9) == -1
