@@ -141,6 +141,7 @@ class Layers:
         self.qbar_bf16 = False
         self.cluster = 0
         self.finish_threads = 0
+        self.block_shape = None
 
     def make_contexts(self, **override):
         for c in self.ctx:
@@ -155,6 +156,9 @@ class Layers:
         if self.finish_threads:
             for c in self.ctx:
                 c.set_finish_threads(self.finish_threads)
+        if self.block_shape:
+            for c in self.ctx:
+                c.set_block_shape(*self.block_shape)
 
     def stats(self):
         tot = {}
@@ -433,6 +437,7 @@ def run_gpu(args):
     layers.qbar_bf16 = args.qbar_bf16
     layers.cluster = args.cluster
     layers.finish_threads = args.finish_threads
+    layers.block_shape = args.block_shape
     global QBAR_BYTES
     QBAR_BYTES = 2 if args.qbar_bf16 else 4
     peak, peak_kind = measured_peaks()
@@ -528,7 +533,7 @@ def run_gpu(args):
         "config": {"workload": cfg.name, "B": cfg.B, "H_q": cfg.H_q, "H_kv": cfg.H_kv, "d": cfg.d,
                    "context": cfg.context, "K": cfg.K, "M": cfg.M, "r": cfg.r, "W": cfg.W, "tau": cfg.tau,
                    "R": cfg.R, "qbar_cache": "bf16" if args.qbar_bf16 else "fp32",
-                   "ctas_per_head": args.cluster or "auto", "threads_per_cta": args.finish_threads or "auto",
+                   "ctas_per_head": args.cluster or "auto", "threads_per_cta": args.finish_threads or (args.block_shape and "x".join(map(str, args.block_shape))) or "auto",
                    "layers_rotated": n_layers, "decode_steps_per_layer": t_per_layer,
                    "preroll_steps_per_layer": preroll, "cache_fill_at_first_timed_call": fill_first,
                    "cache_fill_at_last_timed_call": fill_last,
@@ -604,6 +609,8 @@ def run_one_layer(args):
         ctx.set_cluster_size(args.cluster)
     if args.finish_threads:
         ctx.set_finish_threads(args.finish_threads)
+    if args.block_shape:
+        ctx.set_block_shape(*args.block_shape)
     for t in range(steps):
         flush.zero_()
         ctx.decode_step(q[t], k, v, st.seq_len(t))
@@ -612,10 +619,19 @@ def run_one_layer(args):
 
 
 PHASES = {
-    "recall stage (every head)": (1, [(0, 1, "similarities (Eq. 6) + window rows requested"), (1, 2, "Top-r, decision, records (Eq. 7, Eq. 13)")]),
+    "recall stage (every head)": (1, [(0, 1, "similarities (Eq. 6) + window rows requested"), (1, 2, "Top-r, decision, records (Eq. 7, Eq. 13)"),
+                                      (1, 3, "  Top-r alone"), (3, 2, "  decision and records")]),
     "reuse path": (0, [(0, 1, "first lists requested + window rows scored"), (1, 2, "bitmap marked (Eq. 8-9)"),
                        (2, 3, "ordered extraction"), (3, 4, "candidate rows gathered and scored (Eq. 10)"),
-                       (4, 5, "Top-K (Eq. 11)"), (5, 6, "softmax.V, inserts (Eq. 12)")]),
+                       (4, 5, "Top-K (Eq. 11)"), (5, 6, "softmax.V, inserts (Eq. 12)"),
+                       (8, 9, "  Top-K: span of the keys"), (9, 10, "  Top-K: histogram"), (10, 11, "  Top-K: boundary bin"),
+                       (11, 12, "  Top-K: its members"), (12, 13, "  Top-K: their ranks"), (13, 14, "  Top-K: ballots"),
+                       (14, 5, "  Top-K: placed"),
+                       (2, 7, "  extraction: counts and prefix"), (7, 19, "  extraction: listed"), (19, 3, "  extraction: window appended"),
+                       (3, 15, "  rows: requested"), (15, 16, "  rows: first half landed"), (16, 17, "  rows: first half scored"),
+                       (17, 18, "  rows: second half landed"), (18, 4, "  rows: second half scored"),
+                       (5, 20, "  attend: value rows requested"), (20, 21, "  attend: softmax weights"), (21, 22, "  attend: rows landed"),
+                       (22, 23, "  attend: weighted sum"), (23, 6, "  attend: reduction and output")]),
     "exact finish": (2, [(0, 1, "bound from the tile maxima"), (1, 2, "hit-tile list"), (2, 3, "read-back of hit tiles"),
                          (3, 4, "Top-K (Eq. 1)"), (4, 5, "softmax.V, insert (Eq. 12)")]),
 }
@@ -660,6 +676,8 @@ def run_phases(args):
             ctx.set_cluster_size(args.cluster)
         if args.finish_threads:
             ctx.set_finish_threads(args.finish_threads)
+        if args.block_shape:
+            ctx.set_block_shape(*args.block_shape)
         acc = {name: [] for name in tables}
         for t in range(steps):
             flush.zero_()
@@ -674,8 +692,8 @@ def run_phases(args):
         for name in tables:
             x = np.array(acc[name]).astype(np.float64)
             rows = {what: round(float((x[..., b] - x[..., a]).mean())) for a, b, what in PHASES[name][1]}
-            first, last = PHASES[name][1][0][0], PHASES[name][1][-1][1]
-            rows["total"] = round(float((x[..., last] - x[..., first]).mean()))
+            main = [p for p in PHASES[name][1] if not p[2].startswith("  ")]
+            rows["total"] = round(float((x[..., main[-1][1]] - x[..., main[0][0]]).mean()))
             rep[name] = rows
         out[label] = rep
         ctx.close()
@@ -750,6 +768,8 @@ def main():
                     help="CTAs per head in the per-head kernels (0: the library's own choice)")
     ap.add_argument("--finish-threads", type=int, default=0, choices=[0, 512, 1024],
                     help="block shape of the per-head kernels (0: the library's own choice)")
+    ap.add_argument("--block-shape", default=None, type=lambda v: tuple(int(x) for x in v.split("x")),
+                    help="THREADSxCTAS_PER_SM of the per-head kernels: 1024x1, 512x2, 512x1 or 256x1 (default: the library's own choice)")
     ap.add_argument("--qbar-bf16", action="store_true",
                     help="keep the cached normalised queries in bf16 (storage variant) in every pass")
     ap.add_argument("--ladder", action="store_true",

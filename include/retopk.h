@@ -140,6 +140,15 @@ int retopk_set_cluster_size(retopk_ctx* ctx, int ctas_per_head);
 int retopk_set_finish_threads(retopk_ctx* ctx, int threads);
 
 /*
+ * The same choice in full: (threads, CTAs per SM) is one of (1024, 1), (512, 2), (512, 1),
+ * (256, 1).  With one CTA per SM the CTA takes all of the SM's shared memory whatever its
+ * thread count; fewer threads per head mean fewer instructions spent on block-wide
+ * bookkeeping and more work per thread.  retopk_set_finish_threads(512) is (512, 2).
+ * EINVAL for other pairs or below fusion level 5, EUNSUPPORTED when the shape does not fit.
+ */
+int retopk_set_block_shape(retopk_ctx* ctx, int threads, int ctas_per_sm);
+
+/*
  * Fusion level of the reuse path, for measuring what kernel fusion buys (the paper's kernel
  * efficiency analysis, Table 4, reports five cumulative stages for its own kernels; the cut
  * points here follow its description of them and are this library's own).  Results do not

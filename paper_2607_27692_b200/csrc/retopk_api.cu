@@ -19,8 +19,10 @@ struct retopk_ctx {
     long long max_seq_len, score_stride, tmax_stride;
     long long n_ins, t_dec;
     int NS, tile_cap, stage_depth, exact_stage_depth, win_prefetch;      // of the block shape in use
-    int finish_threads;          // 1024, or 512 with two CTAs per SM when there are more heads than SMs
-    struct FinishShape { int ok, stage_depth, exact_stage_depth, win_prefetch; size_t smem_step, smem_exact; } shape[2];   // [0]: 1024, [1]: 512
+    int finish_threads;          // threads per CTA of the per-head kernels: that of the block shape in use
+    int shape_id;                // block shape in use (index into shape[])
+    // block shapes of the per-head kernels: (threads, CTAs per SM) = (1024,1) (512,2) (512,1) (256,1)
+    struct FinishShape { int nt, per_sm, ok, stage_depth, exact_stage_depth, win_prefetch, NS, tile_cap; size_t smem_step, smem_exact; } shape[4];
     int num_sms, scan_grid;
     int call_serial;
     int recall_recent;
@@ -145,16 +147,19 @@ int auto_cluster(long long heads, int num_sms) {
 
 // More heads than SMs: two narrower CTAs per SM, so that one head's selection overlaps
 // another's row copies.
-int auto_finish_threads(const retopk_ctx* c) {
-    return (long long)c->B * c->Hq > c->num_sms && c->shape[1].ok ? 512 : 1024;
+int auto_shape(const retopk_ctx* c) {
+    return (long long)c->B * c->Hq > c->num_sms && c->shape[1].ok ? 1 : 0;
 }
 
-void use_finish_shape(retopk_ctx* c, int threads) {
-    const retopk_ctx::FinishShape& sh = c->shape[threads == 512 ? 1 : 0];
-    c->finish_threads = threads;
+void use_finish_shape(retopk_ctx* c, int id) {
+    const retopk_ctx::FinishShape& sh = c->shape[id];
+    c->shape_id = id;
+    c->finish_threads = sh.nt;
     c->stage_depth = sh.stage_depth;
     c->exact_stage_depth = sh.exact_stage_depth;
     c->win_prefetch = sh.win_prefetch;
+    c->NS = sh.NS;
+    c->tile_cap = sh.tile_cap;
     c->smem_step = sh.smem_step;
     c->smem_exact = sh.smem_exact;
 }
@@ -195,12 +200,16 @@ bool injected_failure(const retopk_ctx* c, int which) {
 int launch_step(const retopk_ctx* c, const StepArgs& a, cudaStream_t s) {
     if (injected_failure(c, 1)) return RETOPK_ECUDA;
     const unsigned grid = (unsigned)(c->B * c->Hq * c->cluster);      // one cluster of CTAs per head
-    if (c->finish_threads == 512) {
-        if (c->d == 128) return launch_dependent(step_kernel<128, 512>, grid, 512, c->smem_step, s, a, c->dependent_launches, c->cluster);
-        return launch_dependent(step_kernel<64, 512>, grid, 512, c->smem_step, s, a, c->dependent_launches, c->cluster);
+    const unsigned nt = (unsigned)c->finish_threads;
+    const int dep = c->dependent_launches, cl = c->cluster;
+    if (c->d == 128) {
+        if (nt == 1024) return launch_dependent(step_kernel<128, 1024>, grid, nt, c->smem_step, s, a, dep, cl);
+        if (nt == 512) return launch_dependent(step_kernel<128, 512>, grid, nt, c->smem_step, s, a, dep, cl);
+        return launch_dependent(step_kernel<128, 256>, grid, nt, c->smem_step, s, a, dep, cl);
     }
-    if (c->d == 128) return launch_dependent(step_kernel<128, 1024>, grid, FINISH_THREADS, c->smem_step, s, a, c->dependent_launches, c->cluster);
-    return launch_dependent(step_kernel<64, 1024>, grid, FINISH_THREADS, c->smem_step, s, a, c->dependent_launches, c->cluster);
+    if (nt == 1024) return launch_dependent(step_kernel<64, 1024>, grid, nt, c->smem_step, s, a, dep, cl);
+    if (nt == 512) return launch_dependent(step_kernel<64, 512>, grid, nt, c->smem_step, s, a, dep, cl);
+    return launch_dependent(step_kernel<64, 256>, grid, nt, c->smem_step, s, a, dep, cl);
 }
 
 int launch_scan(const retopk_ctx* c, const StepArgs& a, cudaStream_t s) {
@@ -220,13 +229,17 @@ int launch_scan(const retopk_ctx* c, const StepArgs& a, cudaStream_t s) {
 int launch_finish(const retopk_ctx* c, const StepArgs& a, cudaStream_t s) {
     if (injected_failure(c, 3)) return RETOPK_ECUDA;
     const unsigned grid = (unsigned)(c->B * c->Hq * c->cluster);      // one cluster of CTAs per head
+    const unsigned nt = (unsigned)c->finish_threads;
+    const int dep = c->dependent_launches, cl = c->cluster;
     const size_t smem = c->smem_exact;
-    if (c->finish_threads == 512) {
-        if (c->d == 128) return launch_dependent(exact_finish_kernel<128, 512>, grid, 512, smem, s, a, c->dependent_launches, c->cluster);
-        return launch_dependent(exact_finish_kernel<64, 512>, grid, 512, smem, s, a, c->dependent_launches, c->cluster);
+    if (c->d == 128) {
+        if (nt == 1024) return launch_dependent(exact_finish_kernel<128, 1024>, grid, nt, smem, s, a, dep, cl);
+        if (nt == 512) return launch_dependent(exact_finish_kernel<128, 512>, grid, nt, smem, s, a, dep, cl);
+        return launch_dependent(exact_finish_kernel<128, 256>, grid, nt, smem, s, a, dep, cl);
     }
-    if (c->d == 128) return launch_dependent(exact_finish_kernel<128, 1024>, grid, FINISH_THREADS, smem, s, a, c->dependent_launches, c->cluster);
-    return launch_dependent(exact_finish_kernel<64, 1024>, grid, FINISH_THREADS, smem, s, a, c->dependent_launches, c->cluster);
+    if (nt == 1024) return launch_dependent(exact_finish_kernel<64, 1024>, grid, nt, smem, s, a, dep, cl);
+    if (nt == 512) return launch_dependent(exact_finish_kernel<64, 512>, grid, nt, smem, s, a, dep, cl);
+    return launch_dependent(exact_finish_kernel<64, 256>, grid, nt, smem, s, a, dep, cl);
 }
 
 // Measurement hook: event number `which` (0..3) of the current call, if recording.
@@ -238,11 +251,12 @@ void prof_done(retopk_ctx* c, int kind) {
     if (c->prof_events && c->prof_calls < c->prof_max) c->prof_kind[c->prof_calls++] = (unsigned char)kind;
 }
 
-// Sizes of the exact path's shared lists for a support size K.  The landing zone of the value
-// rows reuses their space, so they cost nothing up to the size of that zone; 8192 entries for
-// K <= 512 keep the narrow (two CTAs per SM) shape within half an SM's shared memory.
-void exact_list_sizes(int K, int* NS, int* tile_cap) {
-    if (K <= 512) { *NS = 8192; *tile_cap = 4096; }
+// Sizes of the exact path's shared lists.  The landing zone of the value rows reuses their
+// space, so they cost nothing up to the size of that zone.  16384 entries hold the maximum of
+// every 16-row tile of a history of up to 256 Ki keys (longer ones are bounded through groups
+// of tiles); the narrow shape (two CTAs per SM, half an SM's shared memory each) takes 8192.
+void exact_list_sizes(int K, bool narrow, int* NS, int* tile_cap) {
+    if (narrow && K <= 512) { *NS = 8192; *tile_cap = 4096; }
     else { *NS = 16384; *tile_cap = 8192; }
 }
 
@@ -260,7 +274,7 @@ size_t exact_smem(int K, int NS, int tile_cap, int d, int nt, size_t budget, int
     long long fit = (long long)((budget - (live + red) * 4) / wave);
     long long want = (K + slots - 1) / slots;
     long long dep = fit < want ? fit : want;
-    *depth = (int)(dep < 1 ? 1 : (dep > 16 ? 16 : dep));
+    *depth = (int)(dep < 1 ? 1 : (dep > 64 ? 64 : dep));
     const size_t tail = red + (size_t)*depth * wave / 4;
     return (live + (lists > tail ? lists : tail)) * 4;
 }
@@ -310,7 +324,7 @@ int ladder_prepare(retopk_ctx* c) {
     const size_t wave = (size_t)LADDER_THREADS * 16 * c->stage_depth;
     const size_t union_words = ((r + 3) & ~(size_t)3) + WS_WORDS + capp + bm_words;
     c->sm_sim = (d + Mp) * 4;
-    c->sm_topr = (Mp + r + 4) * 4;
+    c->sm_topr = (Mp + WS_WORDS + r + 4) * 4;
     c->sm_union = union_words * 4;
     c->sm_discover = (d + Mp + 4 + union_words) * 4;
     c->sm_score = (d + capp) * 4 + wave;
@@ -495,9 +509,6 @@ int retopk_create_batched(retopk_ctx** out, int B, int H_q, int H_kv, int d, int
     c->dependent_launches = 1;
     c->score_stride = (max_seq_len + TILE_ROWS - 1) / TILE_ROWS * TILE_ROWS;   // whole 16-row tiles
     c->tmax_stride = ((max_seq_len + TILE_ROWS - 1) / TILE_ROWS + 3) / 4 * 4;
-    // exact path: shared lists for the scores that reach the tile bound (about 1.1-1.4 K of them,
-    // or all of L when L is short) and for the tiles that hold them
-    exact_list_sizes(K, &c->NS, &c->tile_cap);
     int sms = 0;
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, c->device);
     c->num_sms = sms > 0 ? sms : 148;
@@ -506,64 +517,69 @@ int retopk_create_batched(retopk_ctx** out, int B, int H_q, int H_kv, int d, int
     int max_smem = 0, sm_smem = 0;
     cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, c->device);
     cudaDeviceGetAttribute(&sm_smem, cudaDevAttrMaxSharedMemoryPerMultiprocessor, c->device);
-    for (int v = 0; v < 2; ++v) {
-        // v = 0: one CTA of 1024 threads per SM; v = 1: two of 512, each with half of the SM's
-        // shared memory (1 KB per CTA is the system's)
-        const int nt = v == 0 ? 1024 : 512;
-        const size_t budget = v == 0 ? (size_t)max_smem : (size_t)(sm_smem / 2 - 1024);
+    static const int kShapeThreads[4] = {1024, 512, 512, 256}, kShapePerSm[4] = {1, 2, 1, 1};
+    for (int v = 0; v < 4; ++v) {
+        // a CTA that shares its SM gets half of the SM's shared memory (1 KB per CTA is the system's)
+        const int nt = kShapeThreads[v];
+        const bool narrow = kShapePerSm[v] == 2;
+        const size_t budget = narrow ? (size_t)(sm_smem / 2 - 1024) : (size_t)max_smem;
         retopk_ctx::FinishShape& sh = c->shape[v];
+        sh.nt = nt;
+        sh.per_sm = kShapePerSm[v];
         const size_t red_words = (size_t)(nt / 32) * d + nt;
         const size_t head_words = (size_t)step_head_words(d, M, r, K, W);
         const size_t big_words = (((size_t)2 * c->cap > red_words ? (size_t)2 * c->cap : red_words) + 3) & ~(size_t)3;
         const size_t bm_words = (((size_t)max_seq_len + 31) / 32 + 3) & ~(size_t)3;
         const size_t fixed = (head_words + big_words + bm_words) * 4;
-        sh.smem_exact = exact_smem(K, c->NS, c->tile_cap, d, nt, budget, v == 0 ? 1 : 3, &sh.exact_stage_depth);
+        // exact path: shared lists for the tile maxima (then for the scores that reach the bound,
+        // about 1.1-1.4 K of them) and for the tiles that hold them
+        exact_list_sizes(K, narrow, &sh.NS, &sh.tile_cap);
+        sh.smem_exact = exact_smem(K, sh.NS, sh.tile_cap, d, nt, budget, narrow ? 3 : 1, &sh.exact_stage_depth);
         // the rest of shared memory is the landing zone of the asynchronous row copies: one
         // 16-byte piece per thread per row kept in flight per row slot
         const size_t wave = (size_t)nt * 16;
         // the narrow shape only pays with a few waves of rows in flight on either path
-        const size_t min_waves = v == 0 ? 1 : 3;
+        const size_t min_waves = narrow ? 3 : 1;
         sh.ok = budget >= fixed + min_waves * wave && sh.smem_exact > 0;
         if (!sh.ok) continue;
         const int slots = nt / (d / 8);
         const long long fit = (long long)((budget - fixed) / wave);
         auto waves_for = [&](int rows) { return (long long)((rows + slots - 1) / slots); };
         // enough for the candidates below the window (typically K and a bit), the K value rows
-        // and the window's rows, whichever is most; 16 waves at the very most
+        // and the window's rows, whichever is most
         long long want = waves_for(K + K / 4 > c->cap ? c->cap : K + K / 4);
         if (waves_for(K) > want) want = waves_for(K);
         if (waves_for(W) > want) want = waves_for(W);
         long long dep = fit < want ? fit : want;
-        sh.stage_depth = (int)(dep < 1 ? 1 : (dep > 16 ? 16 : dep));
+        sh.stage_depth = (int)(dep < 1 ? 1 : (dep > 64 ? 64 : dep));
         // the window's rows are requested at kernel entry when they fit the landing zone
         sh.win_prefetch = W > 0 && waves_for(W) <= sh.stage_depth;
         sh.smem_step = fixed + (size_t)sh.stage_depth * wave;
     }
     if (!c->shape[0].ok) { delete c; return RETOPK_EUNSUPPORTED; }
     // opt in to the device maximum once; contexts of different sizes then coexist
-    cudaError_t e1, e2 = cudaSuccess, e3, e4 = cudaSuccess;
+    bool attr_ok = true;
+    auto opt = [&](auto kernel) {
+        attr_ok = attr_ok && cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem) == cudaSuccess;
+    };
     int occ = 0;
     const int ntile = (c->G + 7) / 8;
     if (d == 128) {
-        e1 = cudaFuncSetAttribute(step_kernel<128, 1024>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
-        e2 = cudaFuncSetAttribute(step_kernel<128, 512>, cudaFuncAttributeMaxDynamicSharedMemorySize, sm_smem / 2 - 1024);
-        e3 = cudaFuncSetAttribute(exact_finish_kernel<128, 1024>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
-        e4 = cudaFuncSetAttribute(exact_finish_kernel<128, 512>, cudaFuncAttributeMaxDynamicSharedMemorySize, sm_smem / 2 - 1024);
+        opt(step_kernel<128, 1024>); opt(step_kernel<128, 512>); opt(step_kernel<128, 256>);
+        opt(exact_finish_kernel<128, 1024>); opt(exact_finish_kernel<128, 512>); opt(exact_finish_kernel<128, 256>);
         if (ntile == 1) cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, scan_kernel<128, 1>, SCAN_THREADS, 0);
         else cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, scan_kernel<128, 2>, SCAN_THREADS, 0);
     } else {
-        e1 = cudaFuncSetAttribute(step_kernel<64, 1024>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
-        e2 = cudaFuncSetAttribute(step_kernel<64, 512>, cudaFuncAttributeMaxDynamicSharedMemorySize, sm_smem / 2 - 1024);
-        e3 = cudaFuncSetAttribute(exact_finish_kernel<64, 1024>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
-        e4 = cudaFuncSetAttribute(exact_finish_kernel<64, 512>, cudaFuncAttributeMaxDynamicSharedMemorySize, sm_smem / 2 - 1024);
+        opt(step_kernel<64, 1024>); opt(step_kernel<64, 512>); opt(step_kernel<64, 256>);
+        opt(exact_finish_kernel<64, 1024>); opt(exact_finish_kernel<64, 512>); opt(exact_finish_kernel<64, 256>);
         if (ntile == 1) cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, scan_kernel<64, 1>, SCAN_THREADS, 0);
         else cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, scan_kernel<64, 2>, SCAN_THREADS, 0);
     }
-    if (e1 != cudaSuccess || e2 != cudaSuccess || e3 != cudaSuccess || e4 != cudaSuccess) { cudaGetLastError(); delete c; return RETOPK_ECUDA; }
+    if (!attr_ok) { cudaGetLastError(); delete c; return RETOPK_ECUDA; }
     c->scan_grid = c->num_sms * (occ > 0 ? occ : 2);
     // with few heads, a cluster of CTAs (one SM each) per head, as many as fit one wave
     c->cluster = auto_cluster((long long)B * H_q, c->num_sms);
-    use_finish_shape(c, auto_finish_threads(c));
+    use_finish_shape(c, auto_shape(c));
 
 
     const size_t nh = (size_t)B * H_q;
@@ -611,13 +627,16 @@ int retopk_set_cluster_size(retopk_ctx* c, int ctas_per_head) {
     if (ctas_per_head > 1) {
         // checked here, so that a size the device cannot schedule fails now and not in the middle of a step
         DeviceGuard g(c->device);
+        const int nt = c->finish_threads;
         bool ok;
-        if (c->finish_threads == 512)
-            ok = c->d == 128 ? cluster_fits(step_kernel<128, 512>, 512, c->smem_step, ctas_per_head) && cluster_fits(exact_finish_kernel<128, 512>, 512, c->smem_exact, ctas_per_head)
-                             : cluster_fits(step_kernel<64, 512>, 512, c->smem_step, ctas_per_head) && cluster_fits(exact_finish_kernel<64, 512>, 512, c->smem_exact, ctas_per_head);
+        if (c->d == 128)
+            ok = nt == 1024 ? cluster_fits(step_kernel<128, 1024>, nt, c->smem_step, ctas_per_head) && cluster_fits(exact_finish_kernel<128, 1024>, nt, c->smem_exact, ctas_per_head)
+               : nt == 512 ? cluster_fits(step_kernel<128, 512>, nt, c->smem_step, ctas_per_head) && cluster_fits(exact_finish_kernel<128, 512>, nt, c->smem_exact, ctas_per_head)
+                           : cluster_fits(step_kernel<128, 256>, nt, c->smem_step, ctas_per_head) && cluster_fits(exact_finish_kernel<128, 256>, nt, c->smem_exact, ctas_per_head);
         else
-            ok = c->d == 128 ? cluster_fits(step_kernel<128, 1024>, 1024, c->smem_step, ctas_per_head) && cluster_fits(exact_finish_kernel<128, 1024>, 1024, c->smem_exact, ctas_per_head)
-                             : cluster_fits(step_kernel<64, 1024>, 1024, c->smem_step, ctas_per_head) && cluster_fits(exact_finish_kernel<64, 1024>, 1024, c->smem_exact, ctas_per_head);
+            ok = nt == 1024 ? cluster_fits(step_kernel<64, 1024>, nt, c->smem_step, ctas_per_head) && cluster_fits(exact_finish_kernel<64, 1024>, nt, c->smem_exact, ctas_per_head)
+               : nt == 512 ? cluster_fits(step_kernel<64, 512>, nt, c->smem_step, ctas_per_head) && cluster_fits(exact_finish_kernel<64, 512>, nt, c->smem_exact, ctas_per_head)
+                           : cluster_fits(step_kernel<64, 256>, nt, c->smem_step, ctas_per_head) && cluster_fits(exact_finish_kernel<64, 256>, nt, c->smem_exact, ctas_per_head);
         if (!ok) return RETOPK_EUNSUPPORTED;
     }
     c->cluster = ctas_per_head;
@@ -630,12 +649,21 @@ int retopk_debug_fail_next_launch(retopk_ctx* c, int which) {
     return RETOPK_OK;
 }
 
+int retopk_set_block_shape(retopk_ctx* c, int threads, int ctas_per_sm) {
+    if (!c) return RETOPK_EINVAL;
+    int id = -1;
+    for (int v = 0; v < 4; ++v)
+        if (c->shape[v].nt == threads && c->shape[v].per_sm == ctas_per_sm) id = v;
+    if (id < 0) return RETOPK_EINVAL;
+    if (!c->shape[id].ok) return RETOPK_EUNSUPPORTED;
+    if (id != 0 && c->fusion_level < 5) return RETOPK_EINVAL;
+    use_finish_shape(c, id);
+    return RETOPK_OK;
+}
+
 int retopk_set_finish_threads(retopk_ctx* c, int threads) {
     if (!c || (threads != 1024 && threads != 512)) return RETOPK_EINVAL;
-    if (threads == 512 && !c->shape[1].ok) return RETOPK_EUNSUPPORTED;
-    if (threads == 512 && c->fusion_level < 5) return RETOPK_EINVAL;
-    use_finish_shape(c, threads);
-    return RETOPK_OK;
+    return retopk_set_block_shape(c, threads, threads == 512 ? 2 : 1);
 }
 
 int retopk_set_fusion_level(retopk_ctx* c, int level, int dependent_launches) {
@@ -643,7 +671,7 @@ int retopk_set_fusion_level(retopk_ctx* c, int level, int dependent_launches) {
     if (dependent_launches && level != 5) return RETOPK_EINVAL;   // the unfused kernels are plain launches
     DeviceGuard g(c->device);
     // the unfused kernels are sized for the wide finish shape; level 5 goes back to the default
-    use_finish_shape(c, level < 5 ? 1024 : auto_finish_threads(c));
+    use_finish_shape(c, level < 5 ? 0 : auto_shape(c));
     if (level < 5) {
         int rc = ladder_prepare(c);
         if (rc != RETOPK_OK) return rc;
@@ -1069,7 +1097,7 @@ int exact_topk_decode_static(int B, int H_q, int H_kv, int d, int K, int64_t max
     if (rc != RETOPK_OK) return rc;
 
     int NS = 0, tile_cap = 0;
-    exact_list_sizes(K, &NS, &tile_cap);
+    exact_list_sizes(K, false, &NS, &tile_cap);
     int depth = 1;
     const size_t smem = exact_smem(K, NS, tile_cap, d, FINISH_THREADS, (size_t)st->max_smem, 1, &depth);
     if (smem == 0) return RETOPK_EUNSUPPORTED;

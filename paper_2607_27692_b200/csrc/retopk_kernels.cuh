@@ -52,7 +52,7 @@ constexpr int SCAN_TILE_ROWS = 256;  // key rows per scan work item
 constexpr int MAX_GROUPS = 4096;     // B * H_kv limit (shared list in scan_kernel)
 constexpr int SEL_BINS = 2048;       // histogram bins of the threshold search
 constexpr int SEL_LIST = 256;        // members of the boundary bin ranked exhaustively
-constexpr int SCRATCH_WORDS = SEL_BINS + 2 * SEL_LIST + 128;  // bins | boundary list (key, position) | totals
+constexpr int SCRATCH_WORDS = SEL_BINS + 2 * SEL_LIST + 160;  // bins | boundary list (key, position) | totals, coarse bins, results
 constexpr int WS_WORDS = 64;         // scratch of the block-wide prefix sums
 constexpr int TILE_ROWS = 16;        // rows per score tile whose maximum the scan records
 
@@ -164,6 +164,16 @@ __device__ __forceinline__ void stg_hint(float* p, float v, uint64_t policy) {
     asm volatile("st.global.L2::cache_hint.f32 [%0], %1, %2;" :: "l"(p), "f"(v), "l"(policy) : "memory");
 }
 
+// One tensor-core step of a dot product: 16 rows x 16 bf16 values against 16 x 8 (fp32 accumulate).
+__device__ __forceinline__ void mma_bf16_16816(float* c, uint32_t a0, uint32_t a1, uint32_t a2,
+                                               uint32_t a3, uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, "
+        "{%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
 __device__ __forceinline__ float dot8(const uint4& x, const float* qf) {
     float a = bf16_lo(x.x) * qf[0];
     a = fmaf(bf16_hi(x.x), qf[1], a);
@@ -207,7 +217,7 @@ __device__ __forceinline__ int kv_group_of(int bh, const StepArgs& a) {
 // Exclusive prefix sum of v over the block in thread order; `total` gets the block sum.
 // s_ws: NT/32 ints of shared scratch.  Every thread of the block must call.
 template <int NT>
-__device__ __forceinline__ int block_excl_scan(int v, int* s_ws, int& total) {
+__device__ __noinline__ int block_excl_scan(int v, int* s_ws, int& total) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     int inc = v;
 #pragma unroll
@@ -233,7 +243,7 @@ __device__ __forceinline__ int block_excl_scan(int v, int* s_ws, int& total) {
 // Same for two counters at once: .x and .y are scanned side by side (totals may pass 2^16).
 // s_ws: 2 * NT/32 ints.
 template <int NT>
-__device__ __forceinline__ int2 block_excl_scan2(int2 v, int* s_ws, int2& total) {
+__device__ __noinline__ int2 block_excl_scan2(int2 v, int* s_ws, int2& total) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     int2 inc = v;
 #pragma unroll
@@ -276,7 +286,7 @@ struct ScoreSrc {
 // Returns the key value v and `need_eq` = how many elements equal to v belong to the top K.
 // s_hist: 256 words, s_misc: 2 ints.
 template <int NT, class Src>
-__device__ void radix_select(const Src& src, int n, int K, uint32_t* s_hist, int* s_misc,
+__device__ __noinline__ void radix_select(const Src& src, int n, int K, uint32_t* s_hist, int* s_misc,
                              uint32_t& vstar, int& need_eq) {
     const int tid = threadIdx.x, lane = tid & 31;
     uint32_t prefix = 0, mask = 0;
@@ -340,12 +350,13 @@ struct Threshold {
     uint32_t v;
     int count;
     int need;
+    int ties;       // bin_threshold only: keys equal to v in all (-1: not known)
     uint32_t kmax;
 };
 
 template <int NT>
-__device__ Threshold count_threshold(const uint32_t* key, int n, int K, int low_bit, int* s_h) {
-    static_assert(NT == 1024 || NT == 512, "32 digits are shared out over NT / 32 warps");
+__device__ __noinline__ Threshold count_threshold(const uint32_t* key, int n, int K, int low_bit, int* s_h) {
+    static_assert(NT % 32 == 0 && NT >= 256, "32 digits are shared out over NT / 32 warps");
     constexpr int NW = NT / 32;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     // scratch: two histograms of 32 x 32 words used alternately, then 96 words of totals
@@ -364,6 +375,7 @@ __device__ Threshold count_threshold(const uint32_t* key, int n, int K, int low_
     Threshold res;
     res.kmax = kmax;
     res.count = n;
+    res.ties = -1;
     int hi = 32 - __clz(kmin ^ kmax);                 // bits [hi-1:0] may differ
     uint32_t prefix = hi >= 32 ? 0u : (kmax >> hi) << hi;
     int kk = K;                                       // rank wanted among the keys matching prefix
@@ -408,32 +420,52 @@ __device__ Threshold count_threshold(const uint32_t* key, int n, int K, int low_
     return res;
 }
 
+// Cost model of the block-wide pieces below (measured on B200, 1024 threads): a shuffle, a
+// warp reduction or a shared-memory atomic costs about one cycle per WARP that executes it, a
+// barrier about 80 cycles.  So each phase keeps idle warps out of the loop bodies and leaves
+// serial bookkeeping to one warp.
+
+// Per-warp counts cnt (one per warp, written by lane 0 into s_cnt[warp]) -> the number of
+// items in the warps before this one, and the block total.  Call after a barrier.
+template <int NT>
+__device__ __forceinline__ int warp_base(const int* s_cnt, int& total) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int v = lane < NT / 32 ? s_cnt[lane] : 0;
+    total = __reduce_add_sync(0xffffffffu, v);
+    return __reduce_add_sync(0xffffffffu, lane < warp ? v : 0);
+}
+
 // Threshold by ONE histogram over the span of the scores.  Key i falls into bin
 // floor((score_i - min) / (max - min) * (SEL_BINS - 1)): a monotone map, so every key in a bin
 // above the bin b* that holds the K-th largest key belongs to the top K, and only b*'s members
-// (a handful when the scores are spread) need ranking.  n > K >= 1.
+// (a handful when the scores are spread) need ranking.  n >= K >= 1.
 //   exact = false: v = the smallest key of the bins b* and above, so at least K keys are >= v
 //                  (a lower bound for the K-th largest key); count = keys >= v.
 //   exact = true : b*'s members are ranked exhaustively by (key desc, position asc): v is the
-//                  K-th largest key and `need` of the keys equal to it belong to the top K;
-//                  count = K + 1 marks that form.  More than SEL_LIST members (heavy ties, an
-//                  outlier that flattens the bins): the radix bisection decides instead.
-// s_h: SCRATCH_WORDS ints.  Every thread returns the same result; kmax = largest key.
+//                  K-th largest key, `need` of the keys equal to it belong to the top K and
+//                  `ties` keys equal it in all; count = K + 1 marks that form.  More than
+//                  SEL_LIST members (heavy ties, an outlier that flattens the bins): the radix
+//                  bisection decides instead (ties = -1: not known).
+// A coarse histogram (one bin per 32 fine ones) is kept beside the fine one so that ONE warp
+// finds b* with two 32-lane prefix sums.  s_h: SCRATCH_WORDS ints.  Every thread returns the
+// same result; kmax = largest key.
 template <int NT>
 __device__ Threshold bin_threshold(const uint32_t* key, int n, int K, bool exact, int* s_h) {
-    constexpr int NW = NT / 32, BPT = SEL_BINS / NT;
+    constexpr int NW = NT / 32, NC = SEL_BINS / 32;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     int* s_bl = s_h + SEL_BINS;                      // boundary list: key[SEL_LIST] position[SEL_LIST]
-    int* s_tot = s_h + SEL_BINS + 2 * SEL_LIST;      // [0,32) minima [32,64) maxima [64,96) scan scratch [96,104) results
-    int* s_res = s_tot + 96;
+    int* s_tot = s_h + SEL_BINS + 2 * SEL_LIST;      // [0,32) minima [32,64) maxima [64,128) coarse bins
+    int* s_res = s_bl;                               // results live in the list's first words until it is filled
     uint32_t kmin = 0xffffffffu, kmax = 0u;
-    for (int i = tid; i < n; i += NT) { const uint32_t k = key[i]; kmin = min(kmin, k); kmax = max(kmax, k); }
-    kmin = __reduce_min_sync(0xffffffffu, kmin);
-    kmax = __reduce_max_sync(0xffffffffu, kmax);
+    if (warp * 32 < n) {                             // warps without keys skip the reductions
+        for (int i = tid; i < n; i += NT) { const uint32_t k = key[i]; kmin = min(kmin, k); kmax = max(kmax, k); }
+        kmin = __reduce_min_sync(0xffffffffu, kmin);
+        kmax = __reduce_max_sync(0xffffffffu, kmax);
+    }
     if (lane == 0) { s_tot[warp] = (int)kmin; s_tot[32 + warp] = (int)kmax; }
 #pragma unroll
     for (int i = tid; i < SEL_BINS; i += NT) s_h[i] = 0;
-    if (tid == 0) { s_res[3] = 0; s_res[4] = (int)0xffffffffu; }
+    if (tid < NC) s_tot[64 + tid] = 0;
     __syncthreads();
     kmin = __reduce_min_sync(0xffffffffu, lane < NW ? (uint32_t)s_tot[lane] : 0xffffffffu);
     kmax = __reduce_max_sync(0xffffffffu, lane < NW ? (uint32_t)s_tot[32 + lane] : 0u);
@@ -442,6 +474,7 @@ __device__ Threshold bin_threshold(const uint32_t* key, int n, int K, bool exact
     res.v = kmax;
     res.count = n;
     res.need = K;
+    res.ties = n;
     if (kmin == kmax) {          // every key equal: v is the K-th largest, the first K in order are taken
         __syncthreads();
         return res;
@@ -452,64 +485,89 @@ __device__ Threshold bin_threshold(const uint32_t* key, int n, int K, bool exact
         const int b = __float2int_rd((key_score(k) - smin) * scale);
         return min(max(b, 0), SEL_BINS - 1);          // also tames non-finite scores
     };
-    for (int i = tid; i < n; i += NT) atomicAdd(&s_h[bin_of(key[i])], 1);
-    __syncthreads();
-    // bins from the top: thread t owns bins SEL_BINS-1 - (t*BPT + j)
-    int c[BPT], local = 0;
-#pragma unroll
-    for (int j = 0; j < BPT; ++j) { c[j] = s_h[SEL_BINS - 1 - (tid * BPT + j)]; local += c[j]; }
-    int total;
-    int above = block_excl_scan<NT>(local, s_tot + 64, total);
-    if (above < K && K <= above + local) {            // exactly one thread holds b*
-#pragma unroll
-        for (int j = 0; j < BPT; ++j) {
-            if (K <= above + c[j]) { s_res[0] = SEL_BINS - 1 - (tid * BPT + j); s_res[1] = above; s_res[2] = c[j]; break; }
-            above += c[j];
+    if (warp * 32 < n)
+        for (int i = tid; i < n; i += NT) {
+            const int b = bin_of(key[i]);
+            atomicAdd(&s_h[b], 1);
+            atomicAdd(&s_tot[64 + (b >> 5)], 1);
         }
+    __syncthreads();
+    if (warp == 0) {
+        // coarse bins from the top, two per lane, then the 32 fine bins of the coarse bin found
+        const int c0 = s_tot[64 + NC - 1 - 2 * lane], c1 = s_tot[64 + NC - 2 - 2 * lane];
+        int inc = c0 + c1;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) { const int t = __shfl_up_sync(0xffffffffu, inc, o); if (lane >= o) inc += t; }
+        int above = inc - c0 - c1;
+        const unsigned hit = __ballot_sync(0xffffffffu, above < K && K <= inc);
+        const int src = __ffs(hit) - 1;
+        const int first = above < K && K <= above + c0;       // the upper of the lane's two coarse bins
+        int cb = NC - 1 - 2 * lane - (first ? 0 : 1);
+        above += first ? 0 : c0;
+        cb = __shfl_sync(0xffffffffu, cb, src);
+        above = __shfl_sync(0xffffffffu, above, src);
+        const int f = s_h[cb * 32 + 31 - lane];               // fine bins of cb, from the top
+        int finc = f;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) { const int t = __shfl_up_sync(0xffffffffu, finc, o); if (lane >= o) finc += t; }
+        const int fabove = above + finc - f;
+        if (fabove < K && K <= fabove + f) { s_res[0] = cb * 32 + 31 - lane; s_res[1] = fabove; s_res[2] = f; }
+        if (lane == 0) { s_res[3] = 0; s_res[4] = (int)0xffffffffu; }
     }
     __syncthreads();
-    const int bstar = s_res[0], m = s_res[2];
-    above = s_res[1];
+    const int bstar = s_res[0], above = s_res[1], m = s_res[2];
     if (!exact) {
         uint32_t lo = 0xffffffffu;
-        for (int i = tid; i < n; i += NT) { const uint32_t k = key[i]; if (bin_of(k) == bstar) lo = min(lo, k); }
-        lo = __reduce_min_sync(0xffffffffu, lo);
-        if (lane == 0 && lo != 0xffffffffu) atomicMin(reinterpret_cast<unsigned int*>(&s_res[4]), lo);
+        if (warp * 32 < n) {
+            for (int i = tid; i < n; i += NT) { const uint32_t k = key[i]; if (bin_of(k) == bstar) lo = min(lo, k); }
+            lo = __reduce_min_sync(0xffffffffu, lo);
+            if (lane == 0 && lo != 0xffffffffu) atomicMin(reinterpret_cast<unsigned int*>(&s_res[4]), lo);
+        }
         __syncthreads();
         res.v = (uint32_t)s_res[4];
         res.count = above + m;
         res.need = K - above;
+        res.ties = -1;
         __syncthreads();
         return res;
     }
-    if (m > SEL_LIST) {
+    if (m > SEL_LIST - 8) {
         __syncthreads();
-        return count_threshold<NT>(key, n, K, 0, s_h);
+        res = count_threshold<NT>(key, n, K, 0, s_h);
+        res.ties = -1;
+        return res;
     }
     const int need = K - above;                       // 1..m of b*'s members belong to the top K
-    for (int i = tid; i < n; i += NT) {
-        const uint32_t k = key[i];
-        if (bin_of(k) == bstar) {
-            const int p = atomicAdd(&s_res[3], 1);
-            s_bl[p] = (int)k;
-            s_bl[SEL_LIST + p] = i;
+    __syncthreads();                                  // s_res is about to be overwritten by the list
+    int* s_len = s_tot + 64;                          // (the coarse bins are dead now)
+    if (tid == 0) s_len[0] = 0;
+    __syncthreads();
+    if (warp * 32 < n)
+        for (int i = tid; i < n; i += NT) {
+            const uint32_t k = key[i];
+            if (bin_of(k) == bstar) {
+                const int p = atomicAdd(&s_len[0], 1);
+                s_bl[p] = (int)k;
+                s_bl[SEL_LIST + p] = i;
+            }
         }
-    }
     __syncthreads();
     if (tid < m) {
         const uint32_t mine = (uint32_t)s_bl[tid];
         const int pos = s_bl[SEL_LIST + tid];
-        int gt = 0, eq_before = 0;
+        int gt = 0, eq = 0, eq_before = 0;
         for (int j = 0; j < m; ++j) {
             const uint32_t o = (uint32_t)s_bl[j];
             gt += (int)(o > mine);
+            eq += (int)(o == mine);
             eq_before += (int)(o == mine) & (int)(s_bl[SEL_LIST + j] < pos);
         }
-        if (gt + eq_before == need - 1) { s_res[5] = (int)mine; s_res[6] = need - gt; }
+        if (gt + eq_before == need - 1) { s_len[1] = (int)mine; s_len[2] = need - gt; s_len[3] = eq; }
     }
     __syncthreads();
-    res.v = (uint32_t)s_res[5];
-    res.need = s_res[6];
+    res.v = (uint32_t)s_len[1];
+    res.need = s_len[2];
+    res.ties = s_len[3];
     res.count = K + 1;
     __syncthreads();
     return res;
@@ -518,10 +576,10 @@ __device__ Threshold bin_threshold(const uint32_t* key, int n, int K, bool exact
 // Write, in source order, every element with key > v and the first need_eq elements with
 // key == v into s_sup_idx / s_sup_key.  Source order is ascending index, so the output is
 // the support in ascending index order with ties resolved to the lower index.  Every thread
-// takes one contiguous run of the source, so a single prefix sum places them all.
-// s_ws: 64 ints.
+// takes one contiguous run of the source, so a single prefix sum places them all.  The general
+// form (any number of ties at v); s_ws: WS_WORDS ints.
 template <int NT, class Src>
-__device__ void ordered_emit(const Src& src, int n, uint32_t vstar, int need_eq, int32_t* s_sup_idx,
+__device__ __noinline__ void ordered_emit(const Src& src, int n, uint32_t vstar, int need_eq, int32_t* s_sup_idx,
                              uint32_t* s_sup_key, int* s_ws) {
     const int tid = threadIdx.x;
     const int ipt = (n + NT - 1) / NT;                 // NT is a power of two: a shift
@@ -555,9 +613,203 @@ __device__ void ordered_emit(const Src& src, int n, uint32_t vstar, int need_eq,
     }
 }
 
+// The common case of ordered_emit: every key >= v is taken (no tie at v is left out), the
+// source sits in shared memory.  Keys are visited in rounds of NT (key r*NT + tid), a ballot
+// gives each lane its place within the warp, per-(round, warp) counts go through a small
+// table: no shuffle chains.  s_tab: rounds * NT/32 ints (rounds = ceil(n / NT)); needs a barrier
+// before the call if s_tab was in use.
+template <int NT>
+__device__ void ordered_emit_ge(const uint32_t* s_key, const int32_t* s_idx, int n, uint32_t v,
+                                int32_t* s_sup_idx, uint32_t* s_sup_key, int* s_tab) {
+    constexpr int NW = NT / 32;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int rounds = (n + NT - 1) / NT;
+    for (int r = 0; r < rounds; ++r) {
+        const int i = r * NT + tid;
+        const unsigned bal = __ballot_sync(0xffffffffu, i < n && s_key[i] >= v);
+        if (lane == 0) s_tab[r * NW + warp] = __popc(bal);
+    }
+    __syncthreads();
+    int run = 0;                                       // taken in the rounds before r
+    for (int r = 0; r < rounds; ++r) {
+        int total;
+        const int base = run + warp_base<NT>(s_tab + r * NW, total);
+        const int i = r * NT + tid;
+        const uint32_t key = i < n ? s_key[i] : 0u;
+        const bool take = i < n && key >= v;
+        const unsigned bal = __ballot_sync(0xffffffffu, take);
+        if (take) {
+            const int pos = base + __popc(bal & ((1u << lane) - 1u));
+            s_sup_idx[pos] = s_idx[i];
+            s_sup_key[pos] = key;
+        }
+        run += total;
+    }
+}
+
+// ------------------------------------------------------------------------------------
+// The same threshold search and emit for lists of at most R * NT keys, written without loops:
+// every thread keeps its (at most R) keys and bins in registers and all accesses are
+// predicated.  On this hardware a taken branch to code that was not just executed costs about
+// a hundred cycles, a barrier about eighty, a straight-line instruction a few: the block-wide
+// phases of a decode step are short, so their cost is the number of branches and barriers on
+// the path, and this form has five barriers and next to no branches.
+//   EXACT = true : Top-K of (s_key, s_idx)[0..n) into s_sup_idx / s_sup_key in ascending index
+//                  order; returns 1, or 0 (nothing written) when the list needs the general
+//                  code: all keys equal, or a boundary bin with too many members.
+//   EXACT = false: returns 1 with *v_out = the smallest key of the bins from the boundary bin
+//                  up (at least K keys are >= it), or 0 when all keys are equal.
+// n > K >= 1 (EXACT) or n >= K (bound).  s_h: SCRATCH_WORDS ints.  *kmax_out = largest key.
+// ------------------------------------------------------------------------------------
+template <int NT, int R, bool EXACT>
+__device__ __forceinline__ int select_small(const uint32_t* s_key, const int32_t* s_idx, int n, int K,
+                                            int32_t* s_sup_idx, uint32_t* s_sup_key, int* s_h,
+                                            uint32_t* kmax_out, uint32_t* v_out) {
+    constexpr int NW = NT / 32, NC = SEL_BINS / 32;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    int* s_bl = s_h + SEL_BINS;                      // boundary list: key[SEL_LIST] position[SEL_LIST]
+    int* s_tot = s_h + SEL_BINS + 2 * SEL_LIST;      // [0,32) minima [32,64) maxima [64,128) coarse bins [128,136) results
+    int* s_res = s_tot + 128;
+    uint32_t k[R];
+    bool in[R];
+    uint32_t kmin = 0xffffffffu, kmax = 0u;
+    if (EXACT) RETOPK_PHASE(0, 8);
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+        const int i = r * NT + tid;
+        in[r] = i < n;
+        k[r] = in[r] ? s_key[i] : 0u;
+        kmin = min(kmin, in[r] ? k[r] : 0xffffffffu);
+        kmax = max(kmax, k[r]);
+    }
+    kmin = __reduce_min_sync(0xffffffffu, kmin);
+    kmax = __reduce_max_sync(0xffffffffu, kmax);
+    if (lane == 0) { s_tot[warp] = (int)kmin; s_tot[32 + warp] = (int)kmax; }
+#pragma unroll
+    for (int j = 0; j < SEL_BINS / NT; ++j) s_h[j * NT + tid] = 0;
+    if (tid < NC) s_tot[64 + tid] = 0;
+    if (tid < 8) s_res[tid] = tid == 4 ? (int)0xffffffffu : 0;
+    __syncthreads();
+    if (EXACT) RETOPK_PHASE(0, 9);
+    kmin = __reduce_min_sync(0xffffffffu, lane < NW ? (uint32_t)s_tot[lane] : 0xffffffffu);
+    kmax = __reduce_max_sync(0xffffffffu, lane < NW ? (uint32_t)s_tot[32 + lane] : 0u);
+    *kmax_out = kmax;
+    if (__builtin_expect(kmin == kmax, 0)) return 0;
+    const float smin = key_score(kmin);
+    const float scale = (float)(SEL_BINS - 1) / (key_score(kmax) - smin);
+    int b[R];
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+        const int raw = __float2int_rd((key_score(k[r]) - smin) * scale);
+        b[r] = min(max(raw, 0), SEL_BINS - 1);          // also tames non-finite scores
+        if (in[r]) {
+            atomicAdd(&s_h[b[r]], 1);
+            atomicAdd(&s_tot[64 + (b[r] >> 5)], 1);
+        }
+    }
+    __syncthreads();
+    if (EXACT) RETOPK_PHASE(0, 10);
+    // Every warp finds the boundary bin for itself (a lone warp runs several times slower than
+    // 32 in step, and this way no barrier is needed to spread the result): coarse bins from the
+    // top, two per lane, then the 32 fine bins of the coarse bin found.
+    int bstar, above, m;
+    {
+        const int c0 = s_tot[64 + NC - 1 - 2 * lane], c1 = s_tot[64 + NC - 2 - 2 * lane];
+        int inc = c0 + c1;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) { const int t = __shfl_up_sync(0xffffffffu, inc, o); inc += lane >= o ? t : 0; }
+        int ab = inc - c0 - c1;
+        const unsigned hit = __ballot_sync(0xffffffffu, ab < K && K <= inc);
+        const int src = __ffs(hit) - 1;
+        const bool first = ab < K && K <= ab + c0;            // the upper of the lane's two coarse bins
+        int cb = NC - 1 - 2 * lane - (first ? 0 : 1);
+        ab += first ? 0 : c0;
+        cb = __shfl_sync(0xffffffffu, cb, src);
+        ab = __shfl_sync(0xffffffffu, ab, src);
+        const int f = s_h[cb * 32 + 31 - lane];               // fine bins of cb, from the top
+        int finc = f;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) { const int t = __shfl_up_sync(0xffffffffu, finc, o); finc += lane >= o ? t : 0; }
+        const int fabove = ab + finc - f;
+        const unsigned fhit = __ballot_sync(0xffffffffu, fabove < K && K <= fabove + f);
+        const int fsrc = __ffs(fhit) - 1;
+        bstar = cb * 32 + 31 - fsrc;
+        above = __shfl_sync(0xffffffffu, fabove, fsrc);
+        m = __shfl_sync(0xffffffffu, f, fsrc);
+    }
+    if (EXACT) RETOPK_PHASE(0, 11);
+    if (!EXACT) {
+        uint32_t lo = 0xffffffffu;
+#pragma unroll
+        for (int r = 0; r < R; ++r) lo = min(lo, in[r] && b[r] == bstar ? k[r] : 0xffffffffu);
+        lo = __reduce_min_sync(0xffffffffu, lo);
+        if (lane == 0 && lo != 0xffffffffu) atomicMin(reinterpret_cast<unsigned int*>(&s_res[4]), lo);
+        __syncthreads();
+        *v_out = (uint32_t)s_res[4];
+        return 1;
+    }
+    if (__builtin_expect(m > SEL_LIST - 8, 0)) return 0;
+    const int need = K - above;                       // 1..m of the boundary bin's members belong to the top K
+    bool member = false;
+#pragma unroll
+    for (int r = 0; r < R; ++r)
+        if (in[r] && b[r] == bstar) {
+            member = true;
+            const int p = atomicAdd(&s_res[3], 1);
+            s_bl[p] = (int)k[r];
+            s_bl[SEL_LIST + p] = r * NT + tid;
+        }
+    __syncthreads();
+    if (EXACT) RETOPK_PHASE(0, 12);
+    // each owner ranks its own member(s) among the boundary bin's members by (key desc, position
+    // asc) and keeps those of rank < need; keys in the bins above are all taken
+    bool take[R];
+#pragma unroll
+    for (int r = 0; r < R; ++r) take[r] = in[r] && b[r] > bstar;
+    if (member) {
+#pragma unroll
+        for (int r = 0; r < R; ++r)
+            if (in[r] && b[r] == bstar) {
+                const int pos = r * NT + tid;
+                int rank = 0;
+                for (int j = 0; j < m; ++j) {
+                    const uint32_t o = (uint32_t)s_bl[j];
+                    rank += (int)(o > k[r]) | ((int)(o == k[r]) & (int)(s_bl[SEL_LIST + j] < pos));
+                }
+                take[r] = rank < need;
+            }
+    }
+    if (EXACT) RETOPK_PHASE(0, 13);
+    // places from ballots and a small table of per-(round, warp) counts
+    int* s_tab = s_h;                                 // (the fine bins are dead: every warp passed the barrier above)
+    unsigned bal[R];
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+        bal[r] = __ballot_sync(0xffffffffu, take[r]);
+        if (lane == 0) s_tab[r * NW + warp] = __popc(bal[r]);
+    }
+    __syncthreads();
+    if (EXACT) RETOPK_PHASE(0, 14);
+    int run = 0;
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+        const int c = lane < NW ? s_tab[r * NW + lane] : 0;
+        const int total = __reduce_add_sync(0xffffffffu, c);
+        const int base = run + __reduce_add_sync(0xffffffffu, lane < warp ? c : 0);
+        if (take[r]) {
+            const int pos = base + __popc(bal[r] & ((1u << lane) - 1u));
+            s_sup_idx[pos] = s_idx[r * NT + tid];
+            s_sup_key[pos] = k[r];
+        }
+        run += total;
+    }
+    return 1;
+}
+
 // Top-K of the n listed entries (ascending index order in, ascending index order out).
 // kmax_out: largest listed key when known (n > K), else 0 with *kmax_known = false.
-// s_hist: SCRATCH_WORDS words; s_ws: 64 ints.
+// s_hist: SCRATCH_WORDS words; s_ws: WS_WORDS ints; s_tab: ceil(n / NT) * NT/32 ints that may
+// alias nothing the call reads (the bins of s_hist are used for it when they are large enough).
 template <int NT>
 __device__ int select_listed(const uint32_t* s_key, const int32_t* s_idx, int n, int K,
                              int32_t* s_sup_idx, uint32_t* s_sup_key, uint32_t* s_hist, int* s_ws,
@@ -568,14 +820,25 @@ __device__ int select_listed(const uint32_t* s_key, const int32_t* s_idx, int n,
         ns = n;
         kmax = 0;
         kmax_known = false;
+    } else if (n <= 3 * NT && select_small<NT, 3, true>(s_key, s_idx, n, K, s_sup_idx, s_sup_key,
+                                                           reinterpret_cast<int*>(s_hist), &kmax, nullptr)) {
+        ns = K;
+        kmax_known = true;
     } else {
-        SmemSrc src{s_key, s_idx};
+        __syncthreads();                               // (the short form may have left the scratch in use)
         const Threshold t = bin_threshold<NT>(s_key, n, K, true, reinterpret_cast<int*>(s_hist));
-        uint32_t vstar;
-        int need_eq;
-        if (t.count == K) { vstar = t.v - 1u; need_eq = 0; }            // exactly K keys are >= v
-        else { vstar = t.v; need_eq = t.need; }                          // v = K-th largest key
-        ordered_emit<NT>(src, n, vstar, need_eq, s_sup_idx, s_sup_key, s_ws);
+        const int rounds = (n + NT - 1) / NT;
+        if (t.count != K && t.ties == t.need && rounds * (NT / 32) <= SEL_BINS) {
+            // every key equal to the K-th largest is taken: plain ">= v" (the histogram bins are free again)
+            ordered_emit_ge<NT>(s_key, s_idx, n, t.v, s_sup_idx, s_sup_key, reinterpret_cast<int*>(s_hist));
+        } else {
+            SmemSrc src{s_key, s_idx};
+            uint32_t vstar;
+            int need_eq;
+            if (t.count == K) { vstar = t.v - 1u; need_eq = 0; }            // exactly K keys are >= v
+            else { vstar = t.v; need_eq = t.need; }                          // v = K-th largest key
+            ordered_emit<NT>(src, n, vstar, need_eq, s_sup_idx, s_sup_key, s_ws);
+        }
         ns = K;
         kmax = t.kmax;
         kmax_known = true;
@@ -651,8 +914,9 @@ __device__ void attend(const uint16_t* vbase, int ns, const int32_t* s_sup_idx, 
         cp_async_commit();
     };
     issue(i_lo);
+    RETOPK_PHASE(0, 20);
 
-    if (!kmax_known) {
+    if (__builtin_expect(!kmax_known, 0)) {
         kmax = 0;
         for (int i = tid; i < ns; i += NT) kmax = max(kmax, s_sup_key[i]);
         kmax = __reduce_max_sync(0xffffffffu, kmax);
@@ -672,16 +936,21 @@ __device__ void attend(const uint16_t* vbase, int ns, const int32_t* s_sup_idx, 
     for (int o = 16; o > 0; o >>= 1) wsum += __shfl_xor_sync(0xffffffffu, wsum, o);
     float* s_wsf = reinterpret_cast<float*>(s_ws);
     if (lane == 0) s_wsf[warp] = wsum;
-    __syncthreads();
-    float denom = lane < NW ? s_wsf[lane] : 0.f;         // fixed tree: the same sum on every lane and run
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) denom += __shfl_xor_sync(0xffffffffu, denom, o);
+    RETOPK_PHASE(0, 21);
 
     float acc[8];
 #pragma unroll
     for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+    float denom = 0.f;
     for (int base = i_lo;;) {
         cp_async_wait_all();
+        if (base == i_lo) {
+            __syncthreads();                                     // weights and their partial sums are complete
+            denom = lane < NW ? s_wsf[lane] : 0.f;               // fixed tree: the same sum on every lane and run
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) denom += __shfl_xor_sync(0xffffffffu, denom, o);
+        }
+        RETOPK_PHASE(0, 22);
         for (int u = 0; u < depth; ++u) {
             const int i = base + u * SLOTS + myslot;
             if (i < i_hi) {
@@ -697,6 +966,7 @@ __device__ void attend(const uint16_t* vbase, int ns, const int32_t* s_sup_idx, 
         issue(base);
     }
     // fixed-order reduction: row slots of a warp, then warps in groups, then groups
+    RETOPK_PHASE(0, 23);
 #pragma unroll
     for (int o = LPR; o < 32; o <<= 1)
 #pragma unroll
@@ -743,28 +1013,48 @@ __device__ void attend(const uint16_t* vbase, int ns, const int32_t* s_sup_idx, 
 // Pieces of the recall stage (one block per head).
 // ------------------------------------------------------------------------------------
 
+// Four per-lane partials a[0..3] (one per cache row) summed over the 32 lanes of a warp with
+// 6 shuffles instead of 20: lanes trade values as the tree narrows.  Returns the total of row
+// (lane >> 3) & 3 ... precisely: row = ((lane >> 4) & 1) * 2 + ((lane >> 3) & 1), on every lane.
+__device__ __forceinline__ float reduce4_across32(const float* a, int lane, int& row) {
+    const bool h16 = lane & 16, h8 = lane & 8;
+    float b[2];
+#pragma unroll
+    for (int j = 0; j < 2; ++j)
+        b[j] = (h16 ? a[j + 2] : a[j]) + __shfl_xor_sync(0xffffffffu, h16 ? a[j] : a[j + 2], 16);
+    float c = (h8 ? b[1] : b[0]) + __shfl_xor_sync(0xffffffffu, h8 ? b[0] : b[1], 8);
+    c += __shfl_xor_sync(0xffffffffu, c, 4);
+    c += __shfl_xor_sync(0xffffffffu, c, 2);
+    c += __shfl_xor_sync(0xffffffffu, c, 1);
+    row = (h16 ? 2 : 0) + (h8 ? 1 : 0);
+    return c;
+}
+
 // Eq. 6: rho_c = (qbar_c . q) / |q| for every cached entry c < fill into s_rho[c], the
-// normalised query into s_q[0..D) and, if asked for, the raw query as floats into s_qraw[0..D).
-// Every warp reads the query itself (four elements per lane) next to its cache rows, so one
-// memory latency covers both.  after_issue() runs once the first trip's loads are on their
-// way (a place to request other rows without delaying these).  No barrier at the end.
+// normalised query into s_q[0..D) and, if asked for, the raw query as packed bf16 pairs into
+// s_qpk[0..D/2) (the B operand of the tensor-core candidate scores).  Every warp reads the
+// query itself (four elements per lane) next to its cache rows, so one memory latency covers
+// both.  after_issue() runs once the first trip's loads are on their way (a place to request
+// other rows without delaying these).  No barrier at the end.
 struct NoHook { __device__ __forceinline__ void operator()() const {} };
 template <int D, int NT, class Hook = NoHook>
 __device__ __forceinline__ void cache_similarities(const StepArgs& a, int bh, float* s_q, float* s_rho,
-                                                   float* s_qraw = nullptr, Hook after_issue = Hook()) {
+                                                   uint32_t* s_qpk = nullptr, Hook after_issue = Hook()) {
     constexpr int NW = NT / 32;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int M = a.M, fill = a.fill;
     float q4[4] = {0.f, 0.f, 0.f, 0.f};
+    uint2 raw = make_uint2(0u, 0u);
     if (lane < D / 4) {
-        const uint2 raw = *reinterpret_cast<const uint2*>(a.q + (size_t)bh * D + 4 * lane);
+        raw = *reinterpret_cast<const uint2*>(a.q + (size_t)bh * D + 4 * lane);
         q4[0] = bf16_lo(raw.x); q4[1] = bf16_hi(raw.x); q4[2] = bf16_lo(raw.y); q4[3] = bf16_hi(raw.y);
     }
     float inv_nrm = 0.f;
-    for (int c0 = warp; c0 < fill || c0 == warp; c0 += NW * 4) {
-        float4 x[4];
+    constexpr int U = NT >= 1024 ? 4 : 8;            // cache rows per warp and trip, all requested before any is used
+    for (int c0 = warp; c0 < fill || c0 == warp; c0 += NW * U) {
+        float4 x[U];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
+        for (int u = 0; u < U; ++u) {
             const int c = c0 + NW * u;
             x[u] = (c < fill && lane < D / 4) ? load_qbar4(a, ((size_t)bh * M + c) * D, lane)
                                               : make_float4(0.f, 0.f, 0.f, 0.f);
@@ -781,36 +1071,81 @@ __device__ __forceinline__ void cache_similarities(const StepArgs& a, int bh, fl
             if (warp == 0 && lane < D / 4) {
 #pragma unroll
                 for (int e = 0; e < 4; ++e) s_q[4 * lane + e] = nrm > 0.f ? q4[e] / nrm : 0.f;
-                if (s_qraw) {
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) s_qraw[4 * lane + e] = q4[e];
-                }
+                if (s_qpk) { s_qpk[2 * lane] = raw.x; s_qpk[2 * lane + 1] = raw.y; }
             }
         }
+        if (c0 >= fill) continue;                      // (warp-uniform) nothing cached for this warp
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const int c = c0 + NW * u;
-            float acc = x[u].x * q4[0];
-            acc = fmaf(x[u].y, q4[1], acc);
-            acc = fmaf(x[u].z, q4[2], acc);
-            acc = fmaf(x[u].w, q4[3], acc);
+        for (int u0 = 0; u0 < U; u0 += 4) {
+            float part[4];
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-            if (lane == 0 && c < fill) s_rho[c] = acc * inv_nrm;
+            for (int u = 0; u < 4; ++u) {
+                float acc = x[u0 + u].x * q4[0];
+                acc = fmaf(x[u0 + u].y, q4[1], acc);
+                acc = fmaf(x[u0 + u].z, q4[2], acc);
+                acc = fmaf(x[u0 + u].w, q4[3], acc);
+                part[u] = acc;
+            }
+            int row;
+            const float tot = reduce4_across32(part, lane, row);
+            const int c = c0 + NW * (u0 + row);
+            if ((lane & 7) == 0 && c < fill) s_rho[c] = tot * inv_nrm;
         }
     }
 }
 
 // Eq. 7: rho_max and the min(r, fill) most similar slots into s_sel (places beyond that keep
-// the -1 the caller put there; s_misc[0] must hold -inf).  Every cached entry ranks itself
-// against the others (larger rho first, ties -> lower slot).  P threads share an entry (P a
-// power of two <= 32): each counts the better entries in its slice of the cache, a shuffle
-// tree adds the slices.  s_rho must be complete (barrier before the call).
+// the -1 the caller put there; s_misc[0] must hold -inf): larger rho first, ties -> lower slot.
+// Up to 256 cached entries and r <= 8 (the common case) are ranked in registers, eight entries
+// per lane, one argmax round per recalled slot; larger caches by one warp per 256 entries and
+// a merge of their short lists by warp 0.  The first eight recalled slots also come back in
+// sel8 (-1 beyond min(r, fill)), the same on every thread.  s_rho must be complete (barrier
+// before the call); s_sel is complete at the block's next barrier.  s_ws: WS_WORDS ints.
+__device__ __forceinline__ void warp_top_slots(const float* s_rho, int lo, int hi, int n_take, int lane,
+                                               uint32_t* out_key, int* out_slot) {
+    // entry lo + v*32 + lane in value v; taken entries drop out by key 0 / slot INT_MAX
+    uint32_t key[8];
+#pragma unroll
+    for (int v = 0; v < 8; ++v) {
+        const int c = lo + v * 32 + lane;
+        key[v] = c < hi ? score_key(s_rho[c]) : 0u;            // a live key is 0 only for one NaN pattern
+    }
+    for (int j = 0; j < n_take; ++j) {
+        uint32_t best = 0u;
+        int best_c = 0x7fffffff;
+#pragma unroll
+        for (int v = 0; v < 8; ++v)
+            if (key[v] > best) { best = key[v]; best_c = lo + v * 32 + lane; }      // ascending c: the first maximum is the lowest slot
+        const uint32_t top = __reduce_max_sync(0xffffffffu, best);
+        const int c_star = __reduce_min_sync(0xffffffffu, best == top && top != 0u ? best_c : 0x7fffffff);
+#pragma unroll
+        for (int v = 0; v < 8; ++v)
+            if (lo + v * 32 + lane == c_star) key[v] = 0u;
+        if (lane == 0) { out_key[j] = top; out_slot[j] = c_star == 0x7fffffff ? -1 : c_star; }
+    }
+}
+
 template <int NT>
-__device__ __forceinline__ float recall_slots(const StepArgs& a, const float* s_rho, int* s_sel, float* s_misc) {
-    const int tid = threadIdx.x, lane = tid & 31;
+__device__ __forceinline__ float recall_slots(const StepArgs& a, const float* s_rho, int* s_sel, float* s_misc, int* s_ws,
+                                              int* sel8) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int M = a.M, fill = a.fill;
     const int n_sel = a.r < fill ? a.r : fill;
+    if (__builtin_expect(!a.recall_recent && n_sel <= 8 && fill <= 256 && fill > 0, 1)) {
+        // The common case: one warp, up to eight entries per lane, one argmax round per recalled
+        // slot (two warp reductions each).  (Having every warp do it for itself was tried: it
+        // saves the barrier but costs several times more issue slots than it saves.)
+        if (warp == 0) {
+            uint32_t* k_out = reinterpret_cast<uint32_t*>(s_ws);
+            warp_top_slots(s_rho, 0, fill, n_sel, lane, k_out, s_sel);
+            __syncwarp();
+            if (lane == 0 && s_sel[0] >= 0) s_misc[0] = s_rho[s_sel[0]];
+        }
+        __syncthreads();
+#pragma unroll
+        for (int j = 0; j < 8; ++j) sel8[j] = j < a.r ? s_sel[j] : -1;
+        return s_misc[0];
+    }
     if (a.recall_recent) {
         // Recent-R ablation: the newest n_sel entries (newest first), rho_max over those only
         if (tid < 32) {
@@ -824,24 +1159,52 @@ __device__ __forceinline__ float recall_slots(const StepArgs& a, const float* s_
             for (int o = 16; o > 0; o >>= 1) best = fmaxf(best, __shfl_xor_sync(0xffffffffu, best, o));
             if (lane == 0) s_misc[0] = best;
         }
-    } else {
+    } else if (n_sel > 8) {
+        // many recalled slots: every cached entry ranks itself against the others.  P threads
+        // share an entry (P a power of two <= 32): each counts the better entries in its slice
+        // of the cache, a shuffle tree adds the slices.
         int lp = 5;
         while (lp > 0 && (fill << lp) > NT) --lp;
-        const int P = 1 << lp, me = tid >> lp, part = tid & (P - 1);
-        const bool live = me < fill;
-        const float mine = live ? s_rho[me] : 0.f;
-        int rank = 0;
-        for (int c = part; c < fill; c += P) {
-            const float o = s_rho[c];
-            rank += (int)(o > mine) | ((int)(o == mine) & (int)(c < me));
+        const int P = 1 << lp, part = tid & (P - 1);
+        for (int me = tid >> lp; me < ((fill + (NT >> lp) - 1) / (NT >> lp)) * (NT >> lp); me += NT >> lp) {
+            const bool live = me < fill;
+            const float mine = live ? s_rho[me] : 0.f;
+            int rank = 0;
+            for (int c = part; c < fill; c += P) {
+                const float o = s_rho[c];
+                rank += (int)(o > mine) | ((int)(o == mine) & (int)(c < me));
+            }
+            for (int o = P >> 1; o > 0; o >>= 1) rank += __shfl_xor_sync(0xffffffffu, rank, o);
+            if (live && part == 0) {
+                if (rank < n_sel) s_sel[rank] = me;
+                if (rank == 0) s_misc[0] = mine;
+            }
         }
-        for (int o = P >> 1; o > 0; o >>= 1) rank += __shfl_xor_sync(0xffffffffu, rank, o);
-        if (live && part == 0) {
-            if (rank < n_sel) s_sel[rank] = me;
-            if (rank == 0) s_misc[0] = mine;
+    } else if (fill > 256) {
+        // one warp per 256 entries leaves its n_sel best in s_ws (keys in [g*16, g*16+8), slots behind them);
+        // at most four such warps (M <= 1024)
+        const int groups = (fill + 255) >> 8;
+        if (warp < groups)
+            warp_top_slots(s_rho, warp << 8, min(fill, (warp + 1) << 8), n_sel, lane,
+                           reinterpret_cast<uint32_t*>(s_ws) + warp * 16, s_ws + warp * 16 + 8);
+        __syncthreads();
+        if (warp == 0) {
+            // lane l holds candidate (group l >> 3, place l & 7); groups' lists are in rank order already
+            const int g = lane >> 3, j = lane & 7;
+            uint32_t key = (g < groups && j < n_sel) ? reinterpret_cast<uint32_t*>(s_ws)[g * 16 + j] : 0u;
+            int slot = (g < groups && j < n_sel) ? s_ws[g * 16 + 8 + j] : 0x7fffffff;
+            if (slot < 0) { slot = 0x7fffffff; key = 0u; }
+            for (int t = 0; t < n_sel; ++t) {
+                const uint32_t top = __reduce_max_sync(0xffffffffu, key);
+                const int c_star = __reduce_min_sync(0xffffffffu, key == top && top != 0u ? slot : 0x7fffffff);
+                if (slot == c_star) key = 0u;
+                if (lane == 0 && c_star != 0x7fffffff) { s_sel[t] = c_star; if (t == 0) s_misc[0] = s_rho[c_star]; }
+            }
         }
     }
     __syncthreads();
+#pragma unroll
+    for (int j = 0; j < 8; ++j) sel8[j] = j < a.r ? s_sel[j] : -1;
     return s_misc[0];
 }
 
@@ -881,13 +1244,30 @@ __device__ __forceinline__ void record_decision(const StepArgs& a, int bh, int b
 // holds element tid of the first four recalled lists when have_pre (loaded ahead by the caller
 // so that other work overlaps their latency); everything else is loaded here.  No barrier at the end.
 template <int NT>
-__device__ __forceinline__ void union_load_first(const StepArgs& a, int bh, const int* s_sel, int n_sel, int* pre) {
+__device__ __forceinline__ void union_load_first(const StepArgs& a, int bh, const int* sel8, int* pre) {
     const int tid = threadIdx.x;
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
-        const int c = u < n_sel ? s_sel[u] : -1;
+        const int c = sel8[u];
         pre[u] = (c >= 0 && tid < a.K) ? a.sup_cache[((size_t)bh * a.M + c) * a.K + tid] : -1;
     }
+}
+// The whole of union_mark when the four lists of union_load_first are all there is (at most
+// four recalled slots, K <= NT): no loops.  Returns false (nothing done) otherwise.
+template <int NT>
+__device__ __forceinline__ bool union_mark_short(const StepArgs& a, int n_sel, uint32_t* s_bm, const int* pre) {
+    if (__builtin_expect(n_sel > 4 || a.K > NT, 0)) return false;
+    const int L = a.L;
+    const int w_lo = L - a.W > 0 ? L - a.W : 0;
+    bool bad = false;
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+        const int x = pre[u];
+        if (x >= 0 && x < w_lo) atomicOr(&s_bm[x >> 5], 1u << (x & 31));
+        bad = bad || x >= L;
+    }
+    if (__builtin_expect(bad, 0)) atomicOr(a.status, 1u);
+    return true;
 }
 template <int NT>
 __device__ __forceinline__ void union_mark(const StepArgs& a, int bh, const int* s_sel, int n_sel, uint32_t* s_bm,
@@ -917,29 +1297,48 @@ __device__ __forceinline__ void union_mark(const StepArgs& a, int bh, const int*
 
 // Eq. 8-9, second half: ordered extraction of the bitmap (sorted and deduplicated for free)
 // into s_idx, the window appended behind as a run; returns the list's length.  The bitmap
-// must be complete (barrier before the call); no barrier at the end.  s_ws: WS_WORDS ints.
+// must be complete (barrier before the call); no barrier at the end.  Every thread that takes
+// part owns a whole number of 16-byte pieces of the bitmap; only the warps that own words run
+// the prefix sum.  s_ws: WS_WORDS ints.
 template <int NT>
 __device__ __forceinline__ int union_extract(const StepArgs& a, const uint32_t* s_bm, int32_t* s_idx, int* s_ws) {
-    const int tid = threadIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int L = a.L;
     const int w_lo = L - a.W > 0 ? L - a.W : 0;
-    const int nw_lo = (w_lo + 31) >> 5;               // words that can hold bits below the window
-    const int wpt = (nw_lo + NT - 1) / NT;
-    const int w0 = tid * wpt;
-    const int w1 = (w0 + wpt < nw_lo) ? w0 + wpt : nw_lo;
-    int cnt = 0;
-    for (int w = w0; w < w1; ++w) cnt += __popc(s_bm[w]);
+    const int nq = (((w_lo + 31) >> 5) + 3) >> 2;     // 16-byte pieces that can hold bits below the window
+    const int qpt = (nq + NT - 1) / NT;               // pieces per thread
+    const int q0 = tid * qpt;
+    const int q1 = (q0 + qpt < nq) ? q0 + qpt : nq;
+    const uint4* bm4 = reinterpret_cast<const uint4*>(s_bm);
+    int cnt = 0, inc = 0;
+    if (warp * 32 * qpt < nq) {                        // (warp-uniform) this warp owns words
+        for (int p = q0; p < q1; ++p) {
+            const uint4 x = bm4[p];
+            cnt += __popc(x.x) + __popc(x.y) + __popc(x.z) + __popc(x.w);
+        }
+        inc = cnt;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) { const int t = __shfl_up_sync(0xffffffffu, inc, o); if (lane >= o) inc += t; }
+    }
+    if (lane == 31) s_ws[warp] = inc;
+    __syncthreads();
+    RETOPK_PHASE(0, 7);
     int n_low;
-    int pos = block_excl_scan<NT>(cnt, s_ws, n_low);
+    int pos = warp_base<NT>(s_ws, n_low) + inc - cnt;
     if (cnt)
-        for (int w = w0; w < w1; ++w) {
-            uint32_t bits = s_bm[w];
-            while (bits) {
-                const int bit = __ffs(bits) - 1;
-                s_idx[pos++] = w * 32 + bit;
-                bits &= bits - 1;
+        for (int p = q0; p < q1; ++p) {
+            uint4 x = bm4[p];
+            // one trip per set bit, lowest first: the word is picked with selects, not branches
+            for (int left = __popc(x.x) + __popc(x.y) + __popc(x.z) + __popc(x.w); left > 0; --left) {
+                const int e = x.x ? 0 : x.y ? 1 : x.z ? 2 : 3;
+                const uint32_t w = e == 0 ? x.x : e == 1 ? x.y : e == 2 ? x.z : x.w;
+                const int bit = __ffs(w) - 1;
+                s_idx[pos++] = (p * 4 + e) * 32 + bit;
+                const uint32_t rest = w & (w - 1);
+                x.x = e == 0 ? rest : x.x; x.y = e == 1 ? rest : x.y; x.z = e == 2 ? rest : x.z; x.w = e == 3 ? rest : x.w;
             }
         }
+    RETOPK_PHASE(0, 19);
     for (int i = w_lo + tid; i < L; i += NT) s_idx[n_low + (i - w_lo)] = i;
     return n_low + (L - w_lo);
 }
@@ -955,99 +1354,132 @@ __device__ __forceinline__ int candidate_union(const StepArgs& a, int bh, const 
     return union_extract<NT>(a, s_bm, s_idx, s_ws);
 }
 
+// ------------------------------------------------------------------------------------
+// Eq. 10 on the tensor cores.  Gathered key rows are staged in tiles of 16 rows, the A operand
+// of mma.m16n8k16 (bf16 -> fp32); the query is column 0 of the B operand.  A dot product does
+// not care in which order its terms are paired, so each thread reads 16 contiguous bytes of a
+// staged row straight into its A-fragment registers and the query fragment is permuted to
+// match - the same fragment trick, MMA order and scaling as scan_kernel, so a key scores the
+// same bits on either path.  The 16-byte piece c of tile row rho sits at
+//     tile * 16 * PITCH + rho * PITCH + ((c ^ ((rho & 1) << 2)) << 4),   PITCH = 2 * D bytes,
+// which keeps the fragment reads of a quarter warp (rows g and g + 1, pieces t + 4j) on
+// distinct banks.
+// ------------------------------------------------------------------------------------
+template <int D>
+__device__ __forceinline__ unsigned tile_piece_offset(int row, int c) {
+    const int rho = row & 15;
+    return (unsigned)(row >> 4) * (32 * D) + rho * (2 * D) + ((c ^ ((rho & 1) << 2)) << 4);
+}
+
+// Request rows [r0, r1) of a chunk (row i of the chunk is kbase[row_of[i]] or kbase[first + i])
+// into the staging tiles; every lane copies one 16-byte piece per trip.  No commit.
+template <int D, int NT, bool INDEXED>
+__device__ __forceinline__ void rows_request(const uint16_t* kbase, const int32_t* row_of, int first, int r0, int r1,
+                                             unsigned char* s_stage) {
+    constexpr int LPR = D / 8, RPW = 32 / LPR, SLOTS = (NT / 32) * RPW;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int sub = lane % LPR, myslot = warp * RPW + lane / LPR;
+    const char* src = reinterpret_cast<const char*>(kbase) + sub * 16;
+    for (int i = r0 + myslot; i < r1; i += SLOTS)
+        cp_async16(s_stage + tile_piece_offset<D>(i, sub), src + (size_t)(INDEXED ? row_of[i] : first + i) * (D * 2));
+}
+
+// Scores of the staged rows [r0, r1) of a chunk (r0 a multiple of 16; their copies complete and
+// visible to the block: wait + barrier before the call) as order-preserving keys into
+// key_out[r0..r1).  One warp per tile.  s_qpk: the raw query as D/2 packed bf16 pairs.
+template <int D, int NT>
+__device__ __forceinline__ void rows_score(const unsigned char* s_stage, int r0, int r1, const uint32_t* s_qpk,
+                                           float scale, uint32_t* key_out) {
+    constexpr int NJ = D / 32, NW = NT / 32;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int g = lane >> 2, t = lane & 3;
+    if ((r0 >> 4) + warp >= (r1 + 15) >> 4) return;          // no tile for this warp
+    uint32_t bq[NJ][2][2];
+#pragma unroll
+    for (int j = 0; j < NJ; ++j)
+#pragma unroll
+        for (int p = 0; p < 2; ++p) {
+            const int w = j * 16 + t * 4 + 2 * p;
+            bq[j][p][0] = g == 0 ? s_qpk[w] : 0u;            // the query is column 0 of B
+            bq[j][p][1] = g == 0 ? s_qpk[w + 1] : 0u;
+        }
+    const unsigned swz = (unsigned)(g & 1) << 2;
+    for (int tile = (r0 >> 4) + warp; tile * 16 < r1; tile += NW) {
+        const unsigned char* base = s_stage + (size_t)tile * (32 * D);
+        uint4 x[NJ], y[NJ];
+#pragma unroll
+        for (int j = 0; j < NJ; ++j) {
+            const unsigned piece = ((unsigned)(t + 4 * j) ^ swz) << 4;
+            x[j] = *reinterpret_cast<const uint4*>(base + g * (2 * D) + piece);
+            y[j] = *reinterpret_cast<const uint4*>(base + (g + 8) * (2 * D) + piece);
+        }
+        float c[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int j = 0; j < NJ; ++j) {
+            mma_bf16_16816(c, x[j].x, y[j].x, x[j].y, y[j].y, bq[j][0][0], bq[j][0][1]);
+            mma_bf16_16816(c, x[j].z, y[j].z, x[j].w, y[j].w, bq[j][1][0], bq[j][1][1]);
+        }
+        if (t == 0) {                                         // c0: row g, c2: row g + 8, column 0
+            const int i0 = tile * 16 + g, i1 = i0 + 8;
+            if (i0 < r1) key_out[i0] = score_key(c[0] * scale);
+            if (i1 < r1) key_out[i1] = score_key(c[2] * scale);
+        }
+    }
+}
+
 // Eq. 10: exact current-query scores of n key rows as order-preserving keys into key_out.
-// Row i is kbase[row_of[i]] (INDEXED) or kbase[i] (rows already packed).  Every lane copies
-// its 16 bytes of each row asynchronously into its own landing zone and reads them back
-// itself, so a whole wave of rows is in flight with no registers held and no barrier.
-// s_qraw: the raw query as D floats; s_stage: depth * NT uint4.  No barrier at the end.
+// Row i is kbase[row_of[i]] (INDEXED) or kbase[i] (rows already packed).  The rows go through
+// the staging tiles in chunks of depth * SLOTS rows; each chunk is requested as two groups of
+// copies so that the first half is scored while the second half is still arriving (measured
+// against one group per chunk: 8.3K against 10.3K cycles for 306 rows).
+// s_stage: depth * NT * 16 bytes.  Ends with a barrier.
 template <int D, int NT, bool INDEXED>
 __device__ __forceinline__ void score_candidates(const uint16_t* kbase, const int32_t* row_of, int n,
-                                                 const float* s_qraw, uint4* s_stage, int depth, float scale,
+                                                 const uint32_t* s_qpk, uint4* s_stage4, int depth, float scale,
                                                  uint32_t* key_out) {
     constexpr int LPR = D / 8, RPW = 32 / LPR, SLOTS = (NT / 32) * RPW;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int sub = lane % LPR, myslot = warp * RPW + lane / LPR;
-    const char* ksrc = reinterpret_cast<const char*>(kbase) + sub * 16;
-    float qf[8];
-    *reinterpret_cast<float4*>(qf) = *reinterpret_cast<const float4*>(s_qraw + sub * 8);
-    *reinterpret_cast<float4*>(qf + 4) = *reinterpret_cast<const float4*>(s_qraw + sub * 8 + 4);
-    uint4* my_stage = s_stage + tid;
-    // each wave goes out as two groups of copies, so that the dot products of the first
-    // half run while the second half is still arriving
-    const int half = (depth + 1) / 2;
-    for (int base = 0; base < n; base += SLOTS * depth) {
-#pragma unroll 4
-        for (int u = 0; u < depth; ++u) {
-            const int i = base + u * SLOTS + myslot;
-            if (i < n) cp_async16(my_stage + u * NT, ksrc + (size_t)(INDEXED ? row_of[i] : i) * (D * 2));
-            if (u == half - 1) cp_async_commit();
-        }
+    unsigned char* s_stage = reinterpret_cast<unsigned char*>(s_stage4);
+    const int cap = depth * SLOTS;                           // a multiple of 16
+    for (int base = 0; base < n; base += cap) {
+        const int m = min(cap, n - base);
+        const int half = min(m, ((m >> 1) + 15) & ~15);
+        rows_request<D, NT, INDEXED>(kbase, row_of + (INDEXED ? base : 0), base, 0, half, s_stage);
         cp_async_commit();
-        for (int g2 = 0; g2 < 2; ++g2) {
-            if (g2 == 0) cp_async_wait_but_one();
-            else cp_async_wait_all();
-            const int u_begin = g2 == 0 ? 0 : half, u_end = g2 == 0 ? half : depth;
-            for (int u0 = u_begin; u0 < u_end; u0 += 8) {
-                float part[8];
-#pragma unroll
-                for (int uu = 0; uu < 8; ++uu) {
-                    const int i = base + (u0 + uu) * SLOTS + myslot;
-                    part[uu] = (u0 + uu < u_end && i < n) ? dot8(my_stage[(u0 + uu) * NT], qf) : 0.f;
-                }
-                int row;
-                const float tot = reduce8_across<LPR>(part, sub, row);
-                const int i = base + (u0 + row) * SLOTS + myslot;
-                if ((LPR == 8 || (sub & 1) == 0) && u0 + row < u_end && i < n) key_out[i] = score_key(tot * scale);
-            }
-        }
+        rows_request<D, NT, INDEXED>(kbase, row_of + (INDEXED ? base : 0), base, half, m, s_stage);
+        cp_async_commit();
+        RETOPK_PHASE(0, 15);
+        cp_async_wait_but_one();
+        __syncthreads();
+        RETOPK_PHASE(0, 16);
+        rows_score<D, NT>(s_stage, 0, half, s_qpk, scale, key_out + base);
+        RETOPK_PHASE(0, 17);
+        cp_async_wait_all();
+        __syncthreads();
+        RETOPK_PHASE(0, 18);
+        rows_score<D, NT>(s_stage, half, m, s_qpk, scale, key_out + base);
+        __syncthreads();                                     // keys complete; the tiles may be overwritten
     }
 }
 
-// The recent window's key rows [first_row, first_row + n) requested into the landing zone at
-// kernel entry: row i lands in wave i / SLOTS, row slot i % SLOTS; every lane copies (and later
-// reads back) its own 16 bytes.  One commit group.
+// The recent window's key rows [first_row, first_row + n) requested into the staging tiles at
+// kernel entry (one commit group), and their scores once the copies are complete and visible
+// (wait + barrier before window_score).
 template <int D, int NT>
 __device__ __forceinline__ void window_request(const uint16_t* kbase, int first_row, int n, uint4* s_stage) {
-    constexpr int LPR = D / 8, RPW = 32 / LPR, SLOTS = (NT / 32) * RPW;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int sub = lane % LPR, myslot = warp * RPW + lane / LPR;
-    const char* src = reinterpret_cast<const char*>(kbase) + (size_t)first_row * (D * 2) + sub * 16;
-    uint4* my_stage = s_stage + tid;
-    for (int i = myslot, u = 0; i < n; i += SLOTS, ++u) cp_async16(my_stage + u * NT, src + (size_t)i * (D * 2));
+    rows_request<D, NT, false>(kbase, nullptr, first_row, 0, n, reinterpret_cast<unsigned char*>(s_stage));
     cp_async_commit();
 }
-
-// Eq. 10 for the rows window_request brought in (its copies complete: wait before the call):
-// order-preserving score keys into key_out[0..n).  Same per-row arithmetic as score_candidates.
 template <int D, int NT>
-__device__ __forceinline__ void window_score(const uint4* s_stage, int n, const float* s_qraw, float scale,
+__device__ __forceinline__ void window_score(const uint4* s_stage, int n, const uint32_t* s_qpk, float scale,
                                              uint32_t* key_out) {
-    constexpr int LPR = D / 8, RPW = 32 / LPR, SLOTS = (NT / 32) * RPW;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int sub = lane % LPR, myslot = warp * RPW + lane / LPR;
-    float qf[8];
-    *reinterpret_cast<float4*>(qf) = *reinterpret_cast<const float4*>(s_qraw + sub * 8);
-    *reinterpret_cast<float4*>(qf + 4) = *reinterpret_cast<const float4*>(s_qraw + sub * 8 + 4);
-    const uint4* my_stage = s_stage + tid;
-    for (int u0 = 0; u0 * SLOTS < n; u0 += 8) {
-        float part[8];
-#pragma unroll
-        for (int uu = 0; uu < 8; ++uu) {
-            const int i = (u0 + uu) * SLOTS + myslot;
-            part[uu] = i < n ? dot8(my_stage[(u0 + uu) * NT], qf) : 0.f;
-        }
-        int row;
-        const float tot = reduce8_across<LPR>(part, sub, row);
-        const int i = (u0 + row) * SLOTS + myslot;
-        if ((LPR == 8 || (sub & 1) == 0) && i < n) key_out[i] = score_key(tot * scale);
-    }
+    rows_score<D, NT>(reinterpret_cast<const unsigned char*>(s_stage), 0, n, s_qpk, scale, key_out);
 }
 
 // Shared-memory carve-up of step_kernel (the host mirrors it in step_smem_words):
-//   qraw[D] q[D] rho[M+] sel[r+] misc[8] ws[WS_WORDS] hist[SCRATCH_WORDS] sup_idx[K] sup_key[K] w[K] wkey[W+]
+//   qpk[D/2] q[D] rho[M+] sel[r+] misc[8] ws[WS_WORDS] hist[SCRATCH_WORDS] sup_idx[K] sup_key[K] w[K] wkey[W+]
 //   | big: idx[cap] key[cap], aliased later by red[NW*D+NT] | bitmap | stage[depth*NT*4]     ("+": rounded up to 4)
 __host__ __device__ inline int step_head_words(int D, int M, int r, int K, int W) {
-    return (2 * D + ((M + 3) & ~3) + ((r + 3) & ~3) + 8 + WS_WORDS + SCRATCH_WORDS + 3 * K + ((W + 3) & ~3) + 3) & ~3;
+    return (D / 2 + D + ((M + 3) & ~3) + ((r + 3) & ~3) + 8 + WS_WORDS + SCRATCH_WORDS + 3 * K + ((W + 3) & ~3) + 3) & ~3;
 }
 
 // ------------------------------------------------------------------------------------
@@ -1061,8 +1493,8 @@ template <int D, int NT>
 __global__ void __launch_bounds__(NT, 1024 / NT) step_kernel(const StepArgs a) {
     constexpr int NW = NT / 32;
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    float* s_qraw = reinterpret_cast<float*>(smem_raw);
-    float* s_q = s_qraw + D;
+    uint32_t* s_qpk = reinterpret_cast<uint32_t*>(smem_raw);
+    float* s_q = reinterpret_cast<float*>(s_qpk + D / 2);
     float* s_rho = s_q + D;
     int* s_sel = reinterpret_cast<int*>(s_rho + ((a.M + 3) & ~3));
     float* s_misc = reinterpret_cast<float*>(s_sel + ((a.r + 3) & ~3));
@@ -1102,11 +1534,13 @@ __global__ void __launch_bounds__(NT, 1024 / NT) step_kernel(const StepArgs a) {
     RETOPK_PHASE(1, 0);
 
     // ---- recall stage: Eq. 6, Eq. 7, Eq. 13, insert of the normalised query
-    cache_similarities<D, NT>(a, bh, s_q, s_rho, s_qraw,
+    cache_similarities<D, NT>(a, bh, s_q, s_rho, s_qpk,
                               [&]() { if (prefetch) window_request<D, NT>(kbase, w_lo, wn, s_stage); });
     __syncthreads();
     RETOPK_PHASE(1, 1);
-    const float rho_max = recall_slots<NT>(a, s_rho, s_sel, s_misc);
+    int sel8[8];
+    const float rho_max = recall_slots<NT>(a, s_rho, s_sel, s_misc, s_ws, sel8);
+    RETOPK_PHASE(1, 3);
     const int path = decide_path(a, rho_max);
     if (cl_rank == 0) {
         // every similarity of this step has been taken: the slot may be overwritten
@@ -1127,13 +1561,17 @@ __global__ void __launch_bounds__(NT, 1024 / NT) step_kernel(const StepArgs a) {
     // Eq. 8-9.  The first recalled lists are requested, then the window rows (long arrived)
     // are scored while those lists travel.
     int pre[4];
-    union_load_first<NT>(a, bh, s_sel, n_sel, pre);
+    union_load_first<NT>(a, bh, sel8, pre);
     if (prefetch) {
         cp_async_wait_all();
-        window_score<D, NT>(s_stage, wn, s_qraw, a.scale, s_wkey);
+        __syncthreads();           // every thread's pieces have landed
+        window_score<D, NT>(s_stage, wn, s_qpk, a.scale, s_wkey);
     }
     RETOPK_PHASE(0, 1);
-    union_mark<NT>(a, bh, s_sel, n_sel, s_bm, pre, true);
+    if (!union_mark_short<NT>(a, n_sel, s_bm, pre)) {
+        __syncthreads();           // s_sel complete
+        union_mark<NT>(a, bh, s_sel, n_sel, s_bm, pre, true);
+    }
     __syncthreads();
     RETOPK_PHASE(0, 2);
     const int n = union_extract<NT>(a, s_bm, s_idx, s_ws);
@@ -1148,15 +1586,13 @@ __global__ void __launch_bounds__(NT, 1024 / NT) step_kernel(const StepArgs a) {
     // Eq. 10.  In a cluster every CTA built the same list; each scores a contiguous share of
     // it and hands the keys to the others through distributed shared memory.
     if (cl_size == 1) {
-        score_candidates<D, NT, true>(kbase, s_idx, prefetch ? n_low : n, s_qraw, s_stage, a.stage_depth, a.scale, s_key);
-        __syncthreads();
+        score_candidates<D, NT, true>(kbase, s_idx, prefetch ? n_low : n, s_qpk, s_stage, a.stage_depth, a.scale, s_key);
     } else {
         namespace cg = cooperative_groups;
         cg::cluster_group cluster = cg::this_cluster();
         const int share = (n + cl_size - 1) / cl_size;
         const int lo = min(n, cl_rank * share), hi = min(n, lo + share);
-        score_candidates<D, NT, true>(kbase, s_idx + lo, hi - lo, s_qraw, s_stage, a.stage_depth, a.scale, s_key + lo);
-        __syncthreads();
+        score_candidates<D, NT, true>(kbase, s_idx + lo, hi - lo, s_qpk, s_stage, a.stage_depth, a.scale, s_key + lo);
         for (int r = 1; r < cl_size; ++r) {
             uint32_t* peer = cluster.map_shared_rank(s_key, (cl_rank + r) & (cl_size - 1));
             for (int i = lo + tid; i < hi; i += NT) peer[i] = s_key[i];
@@ -1196,27 +1632,16 @@ __global__ void __launch_bounds__(NT, 1024 / NT) step_kernel(const StepArgs a) {
 // CTAs are persistent: the flagged groups' rows are cut into 256-row work items and every
 // CTA takes one contiguous share of them.
 // ------------------------------------------------------------------------------------
-__device__ __forceinline__ void mma_bf16_16816(float* c, uint32_t a0, uint32_t a1, uint32_t a2,
-                                               uint32_t a3, uint32_t b0, uint32_t b1) {
-    asm volatile(
-        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, "
-        "{%8,%9}, {%0,%1,%2,%3};"
-        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
 
 template <int D, int NTILE>   // NTILE = ceil(G / 8) head tiles
-__global__ void __launch_bounds__(SCAN_THREADS) scan_kernel(const StepArgs a) {
+__device__ __forceinline__ void scan_body(const StepArgs& a) {
     constexpr int NJ = D / 32;   // 64-byte column groups per row
-    __shared__ int s_list[MAX_GROUPS];
+    __shared__ unsigned short s_list[MAX_GROUPS];
     __shared__ int s_ws[SCAN_THREADS / 32];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int g = lane >> 2, t = lane & 3;
     const int G = a.G, L = a.L;
     const int n_groups = a.B * a.Hkv;
-    // No trigger for the dependent launch behind this kernel: its CTAs take a whole SM each
-    // and start as this kernel's CTAs exit; that already hides its launch latency.
-    pdl_wait();        // group flags and paths come from recall_kernel
 
     // nothing flagged in this step: leave at once (the common case on the reuse path)
     if (a.mode != MODE_EXACT && a.ws_gflag[n_groups] != a.step_id) return;
@@ -1230,7 +1655,7 @@ __global__ void __launch_bounds__(SCAN_THREADS) scan_kernel(const StepArgs a) {
             const int f = (i < n_groups) && a.ws_gflag[i] == a.step_id;
             int total;
             const int pos = n_act + block_excl_scan<SCAN_THREADS>(f, s_ws, total);
-            if (f) s_list[pos] = i;
+            if (f) s_list[pos] = (unsigned short)i;
             n_act += total;
         }
     if (n_act == 0) return;
@@ -1351,6 +1776,16 @@ __global__ void __launch_bounds__(SCAN_THREADS) scan_kernel(const StepArgs a) {
     }
 }
 
+// scan_kernel: the launch around scan_body, a dependent launch behind step_kernel (or, for
+// Exact Top-K, behind whatever ran before).  (Letting it come up beside step_kernel and wait for
+// the decisions only was tried: its CTAs then share SMs whose shared memory is carved up for
+// the per-head CTAs, and with that little L1 the scan streams 1.6x slower.)
+template <int D, int NTILE>
+__global__ void __launch_bounds__(SCAN_THREADS) scan_kernel(const StepArgs a) {
+    pdl_wait();        // group flags and paths come from step_kernel
+    scan_body<D, NTILE>(a);
+}
+
 // ------------------------------------------------------------------------------------
 // exact path of finish_kernel
 //
@@ -1382,7 +1817,7 @@ __device__ void exact_path(const StepArgs& a, int bh, unsigned char* smem_raw) {
     float* s_red = reinterpret_cast<float*>(s_key);
     uint4* s_stage = reinterpret_cast<uint4*>(s_key + ((NW * D + NT + 3) & ~3));
 
-    const int tid = threadIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int bkv = kv_group_of(bh, a);
     const int K = a.K, L = a.L, NS = a.NS;
     const float* sc = a.ws_scores + (size_t)bh * a.score_stride;
@@ -1400,72 +1835,131 @@ __device__ void exact_path(const StepArgs& a, int bh, unsigned char* smem_raw) {
     } else {
         const int ntile = (L + TILE_ROWS - 1) / TILE_ROWS;
         const int tcap = a.tile_cap;
-        // 1. lower bound v for the K-th score from the tile maxima (grouped so the list is short)
+        // 1. lower bound v for the K-th score: the K-th largest of the tile maxima (of groups of
+        //    2^sh tiles when there are more tiles than list entries).  The keys of the maxima stay
+        //    in shared memory for step 2.
         uint32_t thr_key = 0;
-        int sh = 0;                                  // groups of g2 = 2^sh tiles
-        while (((ntile + (1 << sh) - 1) >> sh) > 1024 && (ntile >> (sh + 1)) >= 2 * K) ++sh;
+        int sh = 0;
         while (((ntile + (1 << sh) - 1) >> sh) > NS) ++sh;
         const int g2 = 1 << sh;
         const int n2 = (ntile + g2 - 1) >> sh;
-        if (n2 >= K) {
-            for (int i2 = tid; i2 < n2; i2 += NT) {
-                const int t0 = i2 << sh;
-                float m;
-                if (g2 >= 4) {
-                    // g2 is a power of two: whole float4 chunks, all requested before any is used
-                    m = -CUDART_INF_F;
-                    for (int c0 = 0; c0 < g2; c0 += 16) {
-                        float4 x[4];
+        if (sh == 0) {
+            // four consecutive maxima per thread and trip, all trips requested before any is used
+            const int nq = (ntile + 3) >> 2;
+            for (int p0 = tid; p0 < nq; p0 += 4 * NT) {
+                float4 x[4];
 #pragma unroll
-                        for (int u = 0; u < 4; ++u)
-                            x[u] = (c0 + 4 * u < g2 && t0 + c0 + 4 * u < ntile)
-                                ? *reinterpret_cast<const float4*>(tm + t0 + c0 + 4 * u)
-                                : make_float4(-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F);
+                for (int u = 0; u < 4; ++u)
+                    x[u] = p0 + u * NT < nq ? *reinterpret_cast<const float4*>(tm + 4 * (p0 + u * NT))
+                                            : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-                        for (int u = 0; u < 4; ++u) {
-                            const int tt = t0 + c0 + 4 * u;
-                            m = fmaxf(m, x[u].x);
-                            if (tt + 1 < ntile) m = fmaxf(m, x[u].y);
-                            if (tt + 2 < ntile) m = fmaxf(m, x[u].z);
-                            if (tt + 3 < ntile) m = fmaxf(m, x[u].w);
-                        }
+                for (int u = 0; u < 4; ++u)
+                    if (p0 + u * NT < nq) {
+                        const int t0 = 4 * (p0 + u * NT);
+                        // (maxima past the last tile are padding of the row: keyed as the smallest key)
+                        const uint4 kq = make_uint4(score_key(x[u].x), t0 + 1 < ntile ? score_key(x[u].y) : 0u,
+                                                    t0 + 2 < ntile ? score_key(x[u].z) : 0u, t0 + 3 < ntile ? score_key(x[u].w) : 0u);
+                        *reinterpret_cast<uint4*>(s_key + t0) = kq;
                     }
-                } else {
-                    m = tm[t0];
-                    if (g2 == 2 && t0 + 1 < ntile) m = fmaxf(m, tm[t0 + 1]);
+            }
+        } else {
+            // groups of g2 tiles (very long histories only): 16-byte loads, g2 / 4 of them per group
+            // (or 4 / g2 groups per load)
+            const int nq = (ntile + 3) >> 2;
+            if (g2 < 4) {                                   // g2 == 2: two groups per load
+                for (int p = tid; p < nq; p += NT) {
+                    const float4 x = *reinterpret_cast<const float4*>(tm + 4 * p);
+                    const int t0 = 4 * p;
+                    s_key[2 * p] = score_key(t0 + 1 < ntile ? fmaxf(x.x, x.y) : x.x);
+                    if (t0 + 2 < ntile) s_key[2 * p + 1] = score_key(t0 + 3 < ntile ? fmaxf(x.z, x.w) : x.z);
                 }
-                s_key[i2] = score_key(m);
+            } else {
+                const int lpg = g2 >> 2;                    // loads per group
+                for (int i2 = tid; i2 < n2; i2 += NT) {
+                    float m = -CUDART_INF_F;
+                    for (int u = 0; u < lpg; ++u) {
+                        const int p = i2 * lpg + u;
+                        if (p >= nq) break;
+                        const float4 x = *reinterpret_cast<const float4*>(tm + 4 * p);
+                        const int t0 = 4 * p;
+                        m = fmaxf(m, x.x);
+                        if (t0 + 1 < ntile) m = fmaxf(m, x.y);
+                        if (t0 + 2 < ntile) m = fmaxf(m, x.z);
+                        if (t0 + 3 < ntile) m = fmaxf(m, x.w);
+                    }
+                    s_key[i2] = score_key(m);
+                }
             }
-            __syncthreads();
-            thr_key = n2 > K ? bin_threshold<NT>(s_key, n2, K, false, reinterpret_cast<int*>(s_hist)).v : 0u;
-        }
-        RETOPK_PHASE(2, 1);
-        // 2. the tiles whose maximum reaches v, in ascending order: eight consecutive tile
-        //    maxima per thread and one prefix sum per 8 * NT tiles
-        int nhit = 0;
-        for (int base = 0; base < ntile; base += NT * 8) {
-            const int t0 = base + tid * 8;
-            float4 m4[2];
-#pragma unroll
-            for (int u = 0; u < 2; ++u)
-                m4[u] = t0 + 4 * u < ntile ? *reinterpret_cast<const float4*>(tm + t0 + 4 * u)
-                                           : make_float4(0.f, 0.f, 0.f, 0.f);
-            const float mv[8] = {m4[0].x, m4[0].y, m4[0].z, m4[0].w, m4[1].x, m4[1].y, m4[1].z, m4[1].w};
-            unsigned hits = 0;
-#pragma unroll
-            for (int e = 0; e < 8; ++e)
-                if (t0 + e < ntile && score_key(mv[e]) >= thr_key) hits |= 1u << e;
-            int total;
-            int pos = nhit + block_excl_scan<NT>(__popc(hits), s_ws, total);
-            while (hits) {
-                const int e = __ffs(hits) - 1;
-                if (pos < tcap) s_tile[pos] = t0 + e;
-                ++pos;
-                hits &= hits - 1;
-            }
-            nhit += total;
         }
         __syncthreads();
+        if (n2 >= K) {
+            uint32_t kmax_unused;
+            if (!(n2 <= 9 * NT && select_small<NT, 9, false>(s_key, nullptr, n2, K, nullptr, nullptr, reinterpret_cast<int*>(s_hist),
+                                                             &kmax_unused, &thr_key))) {
+                __syncthreads();
+                thr_key = bin_threshold<NT>(s_key, n2, K, false, reinterpret_cast<int*>(s_hist)).v;
+            }
+        }
+        RETOPK_PHASE(2, 1);
+        // 2. the tiles whose maximum reaches v, in ascending order.  Ungrouped: straight from the
+        //    keys in shared memory, one 16-byte piece (four tiles) per thread and round.
+        int nhit = 0;
+        if (sh == 0) {
+            const int nq = (ntile + 3) >> 2;
+            for (int base = 0; base < nq; base += NT) {
+                const int p = base + tid;
+                unsigned hits = 0;
+                if (p < nq) {
+                    const uint4 kq = *reinterpret_cast<const uint4*>(s_key + 4 * p);
+                    const uint32_t kv[4] = {kq.x, kq.y, kq.z, kq.w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e)
+                        if (4 * p + e < ntile && kv[e] >= thr_key) hits |= 1u << e;
+                }
+                const int cnt = __popc(hits);
+                int inc = cnt;
+                if (base + warp * 32 < nq) {               // (warp-uniform) this warp looks at tiles in this round
+#pragma unroll
+                    for (int o = 1; o < 32; o <<= 1) { const int t = __shfl_up_sync(0xffffffffu, inc, o); if (lane >= o) inc += t; }
+                }
+                if (lane == 31) s_ws[warp] = inc;
+                __syncthreads();
+                int total;
+                int pos = nhit + warp_base<NT>(s_ws, total) + inc - cnt;
+                while (hits) {
+                    const int e = __ffs(hits) - 1;
+                    if (pos < tcap) s_tile[pos] = 4 * p + e;
+                    ++pos;
+                    hits &= hits - 1;
+                }
+                nhit += total;
+                __syncthreads();                            // s_ws is reused by the next round
+            }
+        } else {
+            for (int base = 0; base < ntile; base += NT * 8) {
+                const int t0 = base + tid * 8;
+                float4 m4[2];
+#pragma unroll
+                for (int u = 0; u < 2; ++u)
+                    m4[u] = t0 + 4 * u < ntile ? *reinterpret_cast<const float4*>(tm + t0 + 4 * u)
+                                               : make_float4(0.f, 0.f, 0.f, 0.f);
+                const float mv[8] = {m4[0].x, m4[0].y, m4[0].z, m4[0].w, m4[1].x, m4[1].y, m4[1].z, m4[1].w};
+                unsigned hits = 0;
+#pragma unroll
+                for (int e = 0; e < 8; ++e)
+                    if (t0 + e < ntile && score_key(mv[e]) >= thr_key) hits |= 1u << e;
+                int total;
+                int pos = nhit + block_excl_scan<NT>(__popc(hits), s_ws, total);
+                while (hits) {
+                    const int e = __ffs(hits) - 1;
+                    if (pos < tcap) s_tile[pos] = t0 + e;
+                    ++pos;
+                    hits &= hits - 1;
+                }
+                nhit += total;
+            }
+            __syncthreads();
+        }
         RETOPK_PHASE(2, 2);
         if (nhit > tcap) slow = true;
         else {
@@ -1487,8 +1981,16 @@ __device__ void exact_path(const StepArgs& a, int bh, unsigned char* smem_raw) {
                             if (row0 + 4 * u + e < L && score_key(v4[e]) >= thr_key) fl |= 1u << (4 * u + e);
                     }
                 }
+                const int cnt = __popc(fl);
+                int inc = cnt;
+                if (base + warp * 32 < nhit) {             // (warp-uniform) this warp visits tiles in this round
+#pragma unroll
+                    for (int o = 1; o < 32; o <<= 1) { const int t = __shfl_up_sync(0xffffffffu, inc, o); if (lane >= o) inc += t; }
+                }
+                if (lane == 31) s_ws[warp] = inc;
+                __syncthreads();
                 int total;
-                int pos = n + block_excl_scan<NT>(__popc(fl), s_ws, total);
+                int pos = n + warp_base<NT>(s_ws, total) + inc - cnt;
                 while (fl) {
                     const int e = __ffs(fl) - 1;
                     if (pos < NS) { s_key[pos] = score_key(sc[row0 + e]); s_idx[pos] = row0 + e; }
@@ -1496,8 +1998,8 @@ __device__ void exact_path(const StepArgs& a, int bh, unsigned char* smem_raw) {
                     fl &= fl - 1;
                 }
                 n += total;
+                __syncthreads();                            // s_ws is reused by the next round
             }
-            __syncthreads();
             if (n > NS) slow = true;
         }
     }

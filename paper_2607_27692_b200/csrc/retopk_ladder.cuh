@@ -44,16 +44,18 @@ __global__ void __launch_bounds__(LADDER_THREADS, 1) ladder_similarity_kernel(co
 __global__ void __launch_bounds__(LADDER_THREADS, 1) ladder_topr_kernel(const StepArgs a) {
     constexpr int NT = LADDER_THREADS;
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    // layout (words): rho[M + 3] sel[r] misc[4]
+    // layout (words): rho[M + 3] ws[WS_WORDS] sel[r] misc[4]
     float* s_rho = reinterpret_cast<float*>(smem_raw);
-    int* s_sel = reinterpret_cast<int*>(s_rho + ((a.M + 3) & ~3));
+    int* s_ws = reinterpret_cast<int*>(s_rho + ((a.M + 3) & ~3));
+    int* s_sel = s_ws + WS_WORDS;
     float* s_misc = reinterpret_cast<float*>(s_sel + a.r);
     const int tid = threadIdx.x, bh = blockIdx.x;
     if (tid < a.r) s_sel[tid] = -1;
     if (tid == 0) s_misc[0] = -CUDART_INF_F;
     for (int c = tid; c < a.fill; c += NT) s_rho[c] = a.lw_rho[(size_t)bh * a.M + c];
     __syncthreads();
-    const float rho_max = recall_slots<NT>(a, s_rho, s_sel, s_misc);
+    int sel8[8];
+    const float rho_max = recall_slots<NT>(a, s_rho, s_sel, s_misc, s_ws, sel8);
     record_decision(a, bh, kv_group_of(bh, a), s_sel, decide_path(a, rho_max), rho_max);
 }
 
@@ -121,24 +123,21 @@ template <int D, bool INDEXED>
 __global__ void __launch_bounds__(LADDER_THREADS, 1) ladder_score_kernel(const StepArgs a) {
     constexpr int NT = LADDER_THREADS;
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    // layout (words): qraw[D] idx[cap] | stage[depth*NT*4]
-    float* s_qraw = reinterpret_cast<float*>(smem_raw);
-    int32_t* s_idx = reinterpret_cast<int32_t*>(s_qraw + D);
+    // layout (words): qpk[D] (the packed query in its first half) idx[cap] | stage[depth*NT*4]
+    uint32_t* s_qpk = reinterpret_cast<uint32_t*>(smem_raw);
+    int32_t* s_idx = reinterpret_cast<int32_t*>(s_qpk + D);
     uint4* s_stage = reinterpret_cast<uint4*>(s_idx + ((a.cap + 3) & ~3));
     const int tid = threadIdx.x, bh = blockIdx.x;
     if (a.ws_path[bh] != PATH_REUSE) return;
     const int n = a.ws_ncand[bh];
-    if (tid < D / 2) {
-        const uint32_t raw = reinterpret_cast<const uint32_t*>(a.q + (size_t)bh * D)[tid];
-        s_qraw[2 * tid] = bf16_lo(raw);
-        s_qraw[2 * tid + 1] = bf16_hi(raw);
-    }
+    if (tid < D / 2) s_qpk[tid] = reinterpret_cast<const uint32_t*>(a.q + (size_t)bh * D)[tid];
     if (INDEXED)
         for (int i = tid; i < n; i += NT) s_idx[i] = a.lw_cand[(size_t)bh * a.cap + i];
     __syncthreads();
     const uint16_t* rows = INDEXED ? a.k + (size_t)kv_group_of(bh, a) * a.max_seq_len * D
                                    : a.lw_rows + (size_t)bh * a.cap * D;
-    score_candidates<D, NT, INDEXED>(rows, s_idx, n, s_qraw, s_stage, a.stage_depth, a.scale,
+    // (keys to shared memory first: the scoring warps write them one tile at a time)
+    score_candidates<D, NT, INDEXED>(rows, s_idx, n, s_qpk, s_stage, a.stage_depth, a.scale,
                                      a.lw_key + (size_t)bh * a.cap);
 }
 
@@ -226,7 +225,7 @@ template <int D>
 __global__ void __launch_bounds__(LADDER_THREADS, 1) ladder_discover_kernel(const StepArgs a) {
     constexpr int NT = LADDER_THREADS;
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    // layout (words): q[D] rho[M + 3] misc[4] | union carve-up (its sel[] is the recall's)
+    // layout (words): q[D] rho[M + 3] misc[4] | union carve-up (its sel[] and ws[] are the recall's)
     float* s_q = reinterpret_cast<float*>(smem_raw);
     float* s_rho = s_q + D;
     float* s_misc = s_rho + ((a.M + 3) & ~3);
@@ -236,7 +235,8 @@ __global__ void __launch_bounds__(LADDER_THREADS, 1) ladder_discover_kernel(cons
     if (tid == 0) s_misc[0] = -CUDART_INF_F;
     cache_similarities<D, NT>(a, bh, s_q, s_rho);
     __syncthreads();
-    const float rho_max = recall_slots<NT>(a, s_rho, u.sel, s_misc);
+    int sel8[8];
+    const float rho_max = recall_slots<NT>(a, s_rho, u.sel, s_misc, u.ws, sel8);
     const int path = decide_path(a, rho_max);
     if (tid < D) store_qbar(a, ((size_t)bh * a.M + a.slot) * D + tid, s_q[tid]);
     record_decision(a, bh, kv_group_of(bh, a), u.sel, path, rho_max);

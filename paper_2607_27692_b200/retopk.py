@@ -40,6 +40,7 @@ SIGNATURES = {
     "retopk_set_qbar_format": (_i32, [_vp, _i32]),
     "retopk_set_cluster_size": (_i32, [_vp, _i32]),
     "retopk_set_finish_threads": (_i32, [_vp, _i32]),
+    "retopk_set_block_shape": (_i32, [_vp, _i32, _i32]),
     "retopk_set_fusion_level": (_i32, [_vp, _i32, _i32]),
     "retopk_destroy": (_i32, [_vp]),
     "retopk_reset": (_i32, [_vp, _vp]),
@@ -165,6 +166,10 @@ class ReTopK:
     def set_finish_threads(self, threads: int):
         """Block shape of the per-head kernels: 1024 (one CTA per SM) or 512 (two per SM)."""
         _check(self.lib.retopk_set_finish_threads(self.h, threads), "retopk_set_finish_threads")
+
+    def set_block_shape(self, threads: int, ctas_per_sm: int):
+        """Block shape of the per-head kernels: (1024, 1), (512, 2), (512, 1) or (256, 1)."""
+        _check(self.lib.retopk_set_block_shape(self.h, threads, ctas_per_sm), "retopk_set_block_shape")
 
     def set_fusion_level(self, level: int, dependent_launches: bool = False):
         """Fusion level 1..5 of the reuse path (Table 4's ladder); results do not depend on it."""

@@ -134,3 +134,21 @@ def test_headline_shape_from_a_full_cache(rt, P, oracle_mod):
     so, sg = o.stats(), g.stats()
     assert so["reuse"] > 0 and so["cand_sum"] / so["reuse"] > 1500
     assert sg["status"] == 0 and sg["slow_select"] == 0
+
+
+@pytest.mark.parametrize("threads,per_sm", [(512, 1), (256, 1), (512, 2)])
+@pytest.mark.parametrize("d", [64, 128])
+def test_block_shapes_against_the_oracle(rt, P, oracle_mod, threads, per_sm, d):
+    """Every block shape of the per-head kernels, full cache, both paths (tau in the middle of the similarities)."""
+    M, r, steps = 128, 4, 24
+    cfg = wl.CONFIGS["tiny"].replace(B=2, H_q=4, H_kv=2, d=d, context=5000, steps=steps, K=128, W=48, M=M, r=r,
+                                     tau=0.9, R=8)
+    st = wl.make_stream(cfg, steps=steps)
+    o = oracle_mod.Oracle.from_config(cfg)
+    g = rt.ReTopK.from_config(cfg)
+    g.set_block_shape(threads, per_sm)
+    P.synthetic_full_state(o, st, cfg.context, np.random.default_rng(threads + d), n_inserted=M + 100)
+    ex = P.teacher_forced_run(cfg, st, steps, o, g, P.to_dev(st.k), P.to_dev(st.v))
+    so, sg = o.stats(), g.stats()
+    assert so["reuse"] > 0 and so["fallback"] + so["refresh"] > 0
+    assert abs(sg["reuse"] - so["reuse"]) <= ex["flips"] and sg["status"] == 0
