@@ -267,13 +267,10 @@ def algorithmic_bytes(cfg, stats, mean_L, mean_fill):
     heads = stats["steps"]
     n_sel = min(cfg.r, mean_fill)
     tail = K * d * 2 + K * 4 + d * 2          # value rows, support insert, output
-    exact_heads = heads - stats["reuse"]
     recall = heads * (mean_fill * d * QBAR_BYTES + d * QBAR_BYTES + d * 2)
     scan = stats["scan_groups"] * mean_L * d * 2
-    # step kernel: the recall stage of every head plus the whole reuse path of the heads that reuse
-    step = recall + stats["reuse"] * (tail + n_sel * K * 4) + stats["cand_sum"] * d * 2
-    finish = exact_heads * (tail + d * 2)
-    return dict(step=step, scan=scan, finish=finish)
+    finish = heads * (tail + d * 2) + stats["reuse"] * n_sel * K * 4 + stats["cand_sum"] * d * 2
+    return dict(recall=recall, scan=scan, finish=finish)
 
 
 def path_mix(stats):
@@ -520,7 +517,7 @@ def run_gpu(args):
                          "frac_of_8TBps": step_head["frac_of_8TBps"]},
                 "paths": {name: {"achieved": rep["GBps"], "frac": rep["frac_of_measured"], "frac_of_8TBps": rep["frac_of_8TBps"],
                                  "us_per_step": rep["us_per_step"]} for name, rep in paths.items()},
-                "exact_topk_kernels": {name: rec for name, rec in kernel_table(exact_p).items() if name != "step"}}
+                "exact_topk_kernels": {name: rec for name, rec in kernel_table(exact_p).items() if name != "recall"}}
 
     exact_bytes = (cfg.B * cfg.H_kv * mean_L * cfg.d * 2 + cfg.B * cfg.H_q * cfg.K * cfg.d * 2) * K
     exact_gbs = exact_bytes / (exact["ms"] * 1e-3) / 1e9
@@ -619,20 +616,15 @@ def run_one_layer(args):
 
 
 PHASES = {
-    "recall stage (every head)": (1, [(0, 1, "similarities (Eq. 6) + window rows requested"), (1, 2, "Top-r, decision, records (Eq. 7, Eq. 13)"),
+    "recall kernel": (1, [(0, 1, "similarities (Eq. 6)"), (1, 2, "Top-r, decision, records (Eq. 7, Eq. 13)"),
                                       (1, 3, "  Top-r alone"), (3, 2, "  decision and records")]),
-    "reuse path": (0, [(0, 1, "first lists requested + window rows scored"), (1, 2, "bitmap marked (Eq. 8-9)"),
-                       (2, 3, "ordered extraction"), (3, 4, "candidate rows gathered and scored (Eq. 10)"),
+    "finish kernel, reuse path": (0, [(0, 1, "slots, query, bitmap cleared"), (1, 2, "bitmap marked (Eq. 8-9)"),
+                       (2, 3, "ordered extraction, window appended"), (3, 4, "candidate rows gathered and scored (Eq. 10)"),
                        (4, 5, "Top-K (Eq. 11)"), (5, 6, "softmax.V, inserts (Eq. 12)"),
                        (8, 9, "  Top-K: span of the keys"), (9, 10, "  Top-K: histogram"), (10, 11, "  Top-K: boundary bin"),
                        (11, 12, "  Top-K: its members"), (12, 13, "  Top-K: their ranks"), (13, 14, "  Top-K: ballots"),
-                       (14, 5, "  Top-K: placed"),
-                       (2, 7, "  extraction: counts and prefix"), (7, 19, "  extraction: listed"), (19, 3, "  extraction: window appended"),
-                       (3, 15, "  rows: requested"), (15, 16, "  rows: first half landed"), (16, 17, "  rows: first half scored"),
-                       (17, 18, "  rows: second half landed"), (18, 4, "  rows: second half scored"),
-                       (5, 20, "  attend: value rows requested"), (20, 21, "  attend: softmax weights"), (21, 22, "  attend: rows landed"),
-                       (22, 23, "  attend: weighted sum"), (23, 6, "  attend: reduction and output")]),
-    "exact finish": (2, [(0, 1, "bound from the tile maxima"), (1, 2, "hit-tile list"), (2, 3, "read-back of hit tiles"),
+                       (14, 5, "  Top-K: placed")]),
+    "finish kernel, exact path": (2, [(0, 1, "bound from the tile maxima"), (1, 2, "hit-tile list"), (2, 3, "read-back of hit tiles"),
                          (3, 4, "Top-K (Eq. 1)"), (4, 5, "softmax.V, insert (Eq. 12)")]),
 }
 
@@ -669,8 +661,8 @@ def run_phases(args):
     nh = min(cfg.B * cfg.H_q, 1024)
     SLOTS = 24
     out = {"workload": cfg.name, "steps_measured": n_meas, "cache_fill": min(cfg.M, pre), "unit": "SM clock cycles, mean over heads and steps"}
-    for label, override, tables in (("pure_reuse", dict(tau=-2.0, R=0), ("recall stage (every head)", "reuse path")),
-                                    ("pure_exact", dict(tau=2.0, R=0), ("recall stage (every head)", "exact finish"))):
+    for label, override, tables in (("pure_reuse", dict(tau=-2.0, R=0), ("recall kernel", "finish kernel, reuse path")),
+                                    ("pure_exact", dict(tau=2.0, R=0), ("recall kernel", "finish kernel, exact path"))):
         ctx = rt.ReTopK.from_config(cfg, **override)
         if args.cluster:
             ctx.set_cluster_size(args.cluster)
@@ -765,11 +757,11 @@ def main():
     ap.add_argument("--preroll", type=int, default=None,
                     help="untimed decode calls per layer that fill the caches before every pass (default: M)")
     ap.add_argument("--cluster", type=int, default=0, choices=[0, 1, 2, 4, 8],
-                    help="CTAs per head in the per-head kernels (0: the library's own choice)")
+                    help="CTAs per head in the finish kernel (0: the library's own choice)")
     ap.add_argument("--finish-threads", type=int, default=0, choices=[0, 512, 1024],
-                    help="block shape of the per-head kernels (0: the library's own choice)")
+                    help="block shape of the finish kernel (0: the library's own choice)")
     ap.add_argument("--block-shape", default=None, type=lambda v: tuple(int(x) for x in v.split("x")),
-                    help="THREADSxCTAS_PER_SM of the per-head kernels: 1024x1, 512x2, 512x1 or 256x1 (default: the library's own choice)")
+                    help="THREADSxCTAS_PER_SM of the finish kernel: 1024x1, 512x2 or 512x1 (default: the library's own choice)")
     ap.add_argument("--qbar-bf16", action="store_true",
                     help="keep the cached normalised queries in bf16 (storage variant) in every pass")
     ap.add_argument("--ladder", action="store_true",

@@ -117,7 +117,7 @@ enum { RETOPK_QBAR_FP32 = 0, RETOPK_QBAR_BF16 = 1 };
 int retopk_set_qbar_format(retopk_ctx* ctx, int format);
 
 /*
- * CTAs per (sequence, query head) in the per-head kernels: 1, 2, 4 or 8.  With more than one, the
+ * CTAs per (sequence, query head) in the finish kernel: 1, 2, 4 or 8.  With more than one, the
  * CTAs of a head form a thread-block cluster on as many SMs: each scores a share of the
  * candidate rows (Eq. 10) and fetches a share of the selected value rows (Eq. 12); keys and
  * partial sums cross through distributed shared memory.  The paper has no counterpart; it is
@@ -130,7 +130,7 @@ int retopk_set_qbar_format(retopk_ctx* ctx, int format);
 int retopk_set_cluster_size(retopk_ctx* ctx, int ctas_per_head);
 
 /*
- * Block shape of the per-head kernels: 1024 threads (one CTA per SM) or 512 (two CTAs per SM,
+ * Block shape of the finish kernel: 1024 threads (one CTA per SM) or 512 (two CTAs per SM,
  * each with half of the SM's shared memory, so that the selection of one head overlaps the
  * row copies of another).  retopk_create* picks 512 when there are more heads than SMs and
  * the shape fits.  Results do not depend on the number of CTAs per SM; outputs differ between
@@ -140,10 +140,10 @@ int retopk_set_cluster_size(retopk_ctx* ctx, int ctas_per_head);
 int retopk_set_finish_threads(retopk_ctx* ctx, int threads);
 
 /*
- * The same choice in full: (threads, CTAs per SM) is one of (1024, 1), (512, 2), (512, 1),
- * (256, 1).  With one CTA per SM the CTA takes all of the SM's shared memory whatever its
- * thread count; fewer threads per head mean fewer instructions spent on block-wide
- * bookkeeping and more work per thread.  retopk_set_finish_threads(512) is (512, 2).
+ * The same choice in full: (threads, CTAs per SM) is one of (1024, 1), (512, 2), (512, 1).
+ * With one CTA per SM the CTA takes all of the SM's shared memory whatever its thread count;
+ * fewer threads per head mean fewer issue slots spent on block-wide bookkeeping and more
+ * work per thread.  retopk_set_finish_threads(512) is (512, 2).
  * EINVAL for other pairs or below fusion level 5, EUNSUPPORTED when the shape does not fit.
  */
 int retopk_set_block_shape(retopk_ctx* ctx, int threads, int ctas_per_sm);
@@ -181,12 +181,12 @@ int retopk_reset(retopk_ctx* ctx, void* stream);
  * One ReTopK decode step (Sec. 3.3-3.4: Eq. 6-13 and the cache insert) for all B * H_q
  * heads.  q, k_cache, v_cache are read, out is written; 1 <= seq_len <= max_seq_len.
  * The path of each head is decided on the device; no host synchronisation happens.
- * Advances t_dec and the insert count by one.  Three launches: the per-head step kernel
- * (recall, decision, and the whole reuse path of the heads that reuse), the full-history
- * scan of the flagged KV groups, and the finish of the heads on the exact path; the last two
- * leave at once when no head fell back.  If a launch fails after the first kernel of the step
- * was enqueued, the caches are half advanced: the call returns RETOPK_ECUDA and so does every
- * later step of this context until retopk_reset.
+ * Advances t_dec and the insert count by one.  Three launches: the recall kernel (similarity
+ * search, decision, insert of the normalised query), the full-history scan of the flagged KV
+ * groups (leaves at once when no head fell back), and the finish kernel with heads of both
+ * paths side by side.  If a launch fails after the first kernel of the step was enqueued, the
+ * caches are half advanced: the call returns RETOPK_ECUDA and so does every later step of
+ * this context until retopk_reset.
  */
 int retopk_decode_step(retopk_ctx* ctx, const void* q, const void* k_cache, const void* v_cache,
                        int64_t seq_len, void* out, void* stream);
@@ -250,7 +250,7 @@ int retopk_last_recall(retopk_ctx* ctx, int32_t* sel, void* stream);
  * Test hook (no counterpart in the paper): keep the candidate list A_t (Eq. 9) of every head
  * that reuses, so that a test can compare it element by element.  enable = 1 allocates a
  * buffer of B*H_q*(r*K+W) int32 (ENOMEM), enable = 0 frees it; both synchronise the device.
- * While it is off (the default) the step kernel writes nothing extra.
+ * While it is off (the default) the finish kernel writes nothing extra.
  * retopk_last_candidates copies the buffer to cand [B,H_q,r*K+W] (device pointer): for a head
  * on the reuse path in the most recent step, its first n_cand entries (retopk_last_step) are
  * the list in ascending order; other rows are stale.  EINVAL while the hook is off.
@@ -260,7 +260,7 @@ int retopk_last_candidates(retopk_ctx* ctx, int32_t* cand, void* stream);
 
 /*
  * Test hook (host side only; nothing on the device fails): the next launch of kernel `which`
- * (1: step, 2: scan, 3: exact finish; 0 clears the request) is skipped and reported as a failed
+ * (1: recall, 2: scan, 3: finish; 0 clears the request) is skipped and reported as a failed
  * launch, so that the error handling of retopk_decode_step can be exercised.
  */
 int retopk_debug_fail_next_launch(retopk_ctx* ctx, int which);
@@ -315,8 +315,8 @@ int exact_topk_decode_static(int B, int H_q, int H_kv, int d, int K, int64_t max
  * Measurement hooks (no counterpart in the paper).  Between begin and end, every decode
  * call of this context brackets each of its kernels with CUDA events on the call's stream
  * (up to max_calls calls; later calls run unrecorded).  retopk_profile_end synchronises
- * the device and returns, per kernel slot {0: step (recall + reuse path), 1: scan, 2: exact
- * finish}, the summed device time in milliseconds and the number of launches.  Not for use
+ * the device and returns, per kernel slot {0: recall, 1: scan, 2: finish}, the summed
+ * device time in milliseconds and the number of launches.  Not for use
  * inside a timed region: the events themselves cost a little, and an event between two
  * kernels keeps the second from starting early.  A failed begin keeps nothing allocated.
  */

@@ -18,17 +18,17 @@ struct retopk_ctx {
     float tau;
     long long max_seq_len, score_stride, tmax_stride;
     long long n_ins, t_dec;
-    int NS, tile_cap, stage_depth, exact_stage_depth, win_prefetch;      // of the block shape in use
+    int NS, tile_cap, stage_depth, exact_stage_depth;      // of the block shape in use
     int finish_threads;          // threads per CTA of the per-head kernels: that of the block shape in use
     int shape_id;                // block shape in use (index into shape[])
-    // block shapes of the per-head kernels: (threads, CTAs per SM) = (1024,1) (512,2) (512,1) (256,1)
-    struct FinishShape { int nt, per_sm, ok, stage_depth, exact_stage_depth, win_prefetch, NS, tile_cap; size_t smem_step, smem_exact; } shape[4];
+    // block shapes of finish_kernel: (threads, CTAs per SM) = (1024,1) (512,2) (512,1)
+    struct FinishShape { int nt, per_sm, ok, stage_depth, exact_stage_depth, NS, tile_cap; size_t smem_reuse, smem_exact, smem_finish; } shape[3];
     int num_sms, scan_grid;
     int call_serial;
     int recall_recent;
     int broken;                  // a launch failed in the middle of a step: the caches are inconsistent until reset
     mutable int fail_launch;     // test hook: the next launch of kernel 1 (step), 2 (scan) or 3 (finish) reports a failure
-    size_t smem_step, smem_exact;
+    size_t smem_recall, smem_reuse, smem_exact, smem_finish;
     // device state
     float* qbar_cache;
     uint16_t* qbar16;            // bf16 copy of the layout, allocated when that format is chosen
@@ -39,8 +39,6 @@ struct retopk_ctx {
     int32_t* ws_ncand;
     int32_t* ws_sel;
     int32_t* ws_gflag;
-    int32_t* ws_xlist;
-    unsigned int* ws_xcount;
     int32_t* dbg_cand;           // candidate lists of the last reuse step (test hook), or null
     float* ws_scores;
     float* ws_tmax;
@@ -93,7 +91,7 @@ void free_all(retopk_ctx* c) {
     cudaFree(c->status); cudaFree(c->slow_select); cudaFree(c->scan_groups); cudaFree(c->scan_counter); cudaFree(c->stage_q); cudaFree(c->stage_out);
     cudaFree(c->stage_kv);
     cudaFree(c->qbar16);
-    cudaFree(c->ws_xlist); cudaFree(c->ws_xcount); cudaFree(c->dbg_cand);
+    cudaFree(c->dbg_cand);
     for (int i = 0; i < 8; ++i) cudaFree(c->lw_persist[i]);
     if (c->pool) cudaMemPoolDestroy(c->pool);
 }
@@ -119,8 +117,7 @@ StepArgs make_args(const retopk_ctx* c, const void* q, const void* k, const void
     a.g_shift = (c->G & (c->G - 1)) == 0 ? __builtin_ctz((unsigned)c->G) : -1;
     a.stage_depth = c->stage_depth;
     a.exact_stage_depth = c->exact_stage_depth;
-    a.win_prefetch = c->win_prefetch;
-    a.ws_xlist = c->ws_xlist; a.ws_xcount = c->ws_xcount; a.dbg_cand = c->dbg_cand;
+    a.dbg_cand = c->dbg_cand;
     a.q = static_cast<const uint16_t*>(q);
     a.k = static_cast<const uint16_t*>(k);
     a.v = static_cast<const uint16_t*>(v);
@@ -137,8 +134,8 @@ StepArgs make_args(const retopk_ctx* c, const void* q, const void* k, const void
     return a;
 }
 
-// CTAs per head in step_kernel / exact_finish_kernel: with few heads, as many (a power of two
-// up to 8, one SM each) as still fit one wave.
+// CTAs per head in finish_kernel: with few heads, as many (a power of two up to 8, one SM each)
+// as still fit one wave.
 int auto_cluster(long long heads, int num_sms) {
     int cl = 1;
     while (cl < 8 && heads * cl * 2 <= num_sms) cl *= 2;
@@ -157,11 +154,11 @@ void use_finish_shape(retopk_ctx* c, int id) {
     c->finish_threads = sh.nt;
     c->stage_depth = sh.stage_depth;
     c->exact_stage_depth = sh.exact_stage_depth;
-    c->win_prefetch = sh.win_prefetch;
     c->NS = sh.NS;
     c->tile_cap = sh.tile_cap;
-    c->smem_step = sh.smem_step;
+    c->smem_reuse = sh.smem_reuse;
     c->smem_exact = sh.smem_exact;
+    c->smem_finish = sh.smem_finish;
 }
 
 // Launch with programmatic stream serialisation: the kernel may be set up while its
@@ -197,19 +194,11 @@ bool injected_failure(const retopk_ctx* c, int which) {
     return true;
 }
 
-int launch_step(const retopk_ctx* c, const StepArgs& a, cudaStream_t s) {
+int launch_recall(const retopk_ctx* c, const StepArgs& a, cudaStream_t s) {
     if (injected_failure(c, 1)) return RETOPK_ECUDA;
-    const unsigned grid = (unsigned)(c->B * c->Hq * c->cluster);      // one cluster of CTAs per head
-    const unsigned nt = (unsigned)c->finish_threads;
-    const int dep = c->dependent_launches, cl = c->cluster;
-    if (c->d == 128) {
-        if (nt == 1024) return launch_dependent(step_kernel<128, 1024>, grid, nt, c->smem_step, s, a, dep, cl);
-        if (nt == 512) return launch_dependent(step_kernel<128, 512>, grid, nt, c->smem_step, s, a, dep, cl);
-        return launch_dependent(step_kernel<128, 256>, grid, nt, c->smem_step, s, a, dep, cl);
-    }
-    if (nt == 1024) return launch_dependent(step_kernel<64, 1024>, grid, nt, c->smem_step, s, a, dep, cl);
-    if (nt == 512) return launch_dependent(step_kernel<64, 512>, grid, nt, c->smem_step, s, a, dep, cl);
-    return launch_dependent(step_kernel<64, 256>, grid, nt, c->smem_step, s, a, dep, cl);
+    const unsigned grid = (unsigned)(c->B * c->Hq);
+    if (c->d == 128) return launch_dependent(recall_kernel<128>, grid, RECALL_THREADS, c->smem_recall, s, a, c->dependent_launches);
+    return launch_dependent(recall_kernel<64>, grid, RECALL_THREADS, c->smem_recall, s, a, c->dependent_launches);
 }
 
 int launch_scan(const retopk_ctx* c, const StepArgs& a, cudaStream_t s) {
@@ -218,8 +207,11 @@ int launch_scan(const retopk_ctx* c, const StepArgs& a, cudaStream_t s) {
     const long long items = (long long)c->B * c->Hkv * ((a.L + SCAN_TILE_ROWS - 1) / SCAN_TILE_ROWS);
     const unsigned grid = (unsigned)(items < c->scan_grid ? items : c->scan_grid);
     const int ntile = (c->G + 7) / 8;
-    // A dependent launch behind step_kernel (or behind the previous call's last kernel for
-    // Exact Top-K).
+    // A dependent launch behind recall_kernel (or behind the previous call's last kernel for
+    // Exact Top-K).  Behind a kernel that takes ALL of an SM's shared memory the scan ran 1.6x
+    // slower: its CTAs then land on SMs still carved up for that kernel, and it needs about
+    // 100 KB of L1 per SM to keep its loads in flight.  recall_kernel uses a few KB, so the SMs
+    // are back in the default split by the time the scan's CTAs start.
     if (c->d == 128 && ntile == 1) return launch_dependent(scan_kernel<128, 1>, grid, SCAN_THREADS, 0, s, a, c->dependent_launches);
     if (c->d == 128) return launch_dependent(scan_kernel<128, 2>, grid, SCAN_THREADS, 0, s, a, c->dependent_launches);
     if (ntile == 1) return launch_dependent(scan_kernel<64, 1>, grid, SCAN_THREADS, 0, s, a, c->dependent_launches);
@@ -231,15 +223,13 @@ int launch_finish(const retopk_ctx* c, const StepArgs& a, cudaStream_t s) {
     const unsigned grid = (unsigned)(c->B * c->Hq * c->cluster);      // one cluster of CTAs per head
     const unsigned nt = (unsigned)c->finish_threads;
     const int dep = c->dependent_launches, cl = c->cluster;
-    const size_t smem = c->smem_exact;
+    const size_t smem = a.mode == MODE_EXACT ? c->smem_exact : c->smem_finish;
     if (c->d == 128) {
-        if (nt == 1024) return launch_dependent(exact_finish_kernel<128, 1024>, grid, nt, smem, s, a, dep, cl);
-        if (nt == 512) return launch_dependent(exact_finish_kernel<128, 512>, grid, nt, smem, s, a, dep, cl);
-        return launch_dependent(exact_finish_kernel<128, 256>, grid, nt, smem, s, a, dep, cl);
+        if (nt == 1024) return launch_dependent(finish_kernel<128, 1024>, grid, nt, smem, s, a, dep, cl);
+        return launch_dependent(finish_kernel<128, 512>, grid, nt, smem, s, a, dep, cl);
     }
-    if (nt == 1024) return launch_dependent(exact_finish_kernel<64, 1024>, grid, nt, smem, s, a, dep, cl);
-    if (nt == 512) return launch_dependent(exact_finish_kernel<64, 512>, grid, nt, smem, s, a, dep, cl);
-    return launch_dependent(exact_finish_kernel<64, 256>, grid, nt, smem, s, a, dep, cl);
+    if (nt == 1024) return launch_dependent(finish_kernel<64, 1024>, grid, nt, smem, s, a, dep, cl);
+    return launch_dependent(finish_kernel<64, 512>, grid, nt, smem, s, a, dep, cl);
 }
 
 // Measurement hook: event number `which` (0..3) of the current call, if recording.
@@ -274,7 +264,7 @@ size_t exact_smem(int K, int NS, int tile_cap, int d, int nt, size_t budget, int
     long long fit = (long long)((budget - (live + red) * 4) / wave);
     long long want = (K + slots - 1) / slots;
     long long dep = fit < want ? fit : want;
-    *depth = (int)(dep < 1 ? 1 : (dep > 64 ? 64 : dep));
+    *depth = (int)(dep < 1 ? 1 : (dep > 16 ? 16 : dep));
     const size_t tail = red + (size_t)*depth * wave / 4;
     return (live + (lists > tail ? lists : tail)) * 4;
 }
@@ -453,6 +443,7 @@ int ladder_step(retopk_ctx* c, StepArgs a, cudaStream_t s) {
     int launches = 0;
     if (rc == RETOPK_OK) {
         ladder_bind(a, buf);
+        a.skip_reuse = 1;
         rc = ladder_launches(c, a, s, &launches);
     }
     if (level != 4)
@@ -514,11 +505,12 @@ int retopk_create_batched(retopk_ctx** out, int B, int H_q, int H_kv, int d, int
     c->num_sms = sms > 0 ? sms : 148;
 
     // shared-memory footprints (must mirror the carve-up at the top of each kernel)
+    c->smem_recall = ((size_t)d + ((M + 3) & ~3) + WS_WORDS + ((r + 3) & ~3) + 4) * 4;
     int max_smem = 0, sm_smem = 0;
     cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, c->device);
     cudaDeviceGetAttribute(&sm_smem, cudaDevAttrMaxSharedMemoryPerMultiprocessor, c->device);
-    static const int kShapeThreads[4] = {1024, 512, 512, 256}, kShapePerSm[4] = {1, 2, 1, 1};
-    for (int v = 0; v < 4; ++v) {
+    static const int kShapeThreads[3] = {1024, 512, 512}, kShapePerSm[3] = {1, 2, 1};
+    for (int v = 0; v < 3; ++v) {
         // a CTA that shares its SM gets half of the SM's shared memory (1 KB per CTA is the system's)
         const int nt = kShapeThreads[v];
         const bool narrow = kShapePerSm[v] == 2;
@@ -527,7 +519,7 @@ int retopk_create_batched(retopk_ctx** out, int B, int H_q, int H_kv, int d, int
         sh.nt = nt;
         sh.per_sm = kShapePerSm[v];
         const size_t red_words = (size_t)(nt / 32) * d + nt;
-        const size_t head_words = (size_t)step_head_words(d, M, r, K, W);
+        const size_t head_words = ((size_t)d + r + WS_WORDS + SCRATCH_WORDS + 3 * (size_t)K + 3) & ~(size_t)3;
         const size_t big_words = (((size_t)2 * c->cap > red_words ? (size_t)2 * c->cap : red_words) + 3) & ~(size_t)3;
         const size_t bm_words = (((size_t)max_seq_len + 31) / 32 + 3) & ~(size_t)3;
         const size_t fixed = (head_words + big_words + bm_words) * 4;
@@ -545,16 +537,13 @@ int retopk_create_batched(retopk_ctx** out, int B, int H_q, int H_kv, int d, int
         const int slots = nt / (d / 8);
         const long long fit = (long long)((budget - fixed) / wave);
         auto waves_for = [&](int rows) { return (long long)((rows + slots - 1) / slots); };
-        // enough for the candidates below the window (typically K and a bit), the K value rows
-        // and the window's rows, whichever is most
+        // enough for one wave of candidates (typically K and a bit) and for the K value rows
         long long want = waves_for(K + K / 4 > c->cap ? c->cap : K + K / 4);
         if (waves_for(K) > want) want = waves_for(K);
-        if (waves_for(W) > want) want = waves_for(W);
         long long dep = fit < want ? fit : want;
-        sh.stage_depth = (int)(dep < 1 ? 1 : (dep > 64 ? 64 : dep));
-        // the window's rows are requested at kernel entry when they fit the landing zone
-        sh.win_prefetch = W > 0 && waves_for(W) <= sh.stage_depth;
-        sh.smem_step = fixed + (size_t)sh.stage_depth * wave;
+        sh.stage_depth = (int)(dep < 1 ? 1 : (dep > 16 ? 16 : dep));
+        sh.smem_reuse = fixed + (size_t)sh.stage_depth * wave;
+        sh.smem_finish = sh.smem_reuse > sh.smem_exact ? sh.smem_reuse : sh.smem_exact;
     }
     if (!c->shape[0].ok) { delete c; return RETOPK_EUNSUPPORTED; }
     // opt in to the device maximum once; contexts of different sizes then coexist
@@ -565,13 +554,11 @@ int retopk_create_batched(retopk_ctx** out, int B, int H_q, int H_kv, int d, int
     int occ = 0;
     const int ntile = (c->G + 7) / 8;
     if (d == 128) {
-        opt(step_kernel<128, 1024>); opt(step_kernel<128, 512>); opt(step_kernel<128, 256>);
-        opt(exact_finish_kernel<128, 1024>); opt(exact_finish_kernel<128, 512>); opt(exact_finish_kernel<128, 256>);
+        opt(finish_kernel<128, 1024>); opt(finish_kernel<128, 512>);
         if (ntile == 1) cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, scan_kernel<128, 1>, SCAN_THREADS, 0);
         else cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, scan_kernel<128, 2>, SCAN_THREADS, 0);
     } else {
-        opt(step_kernel<64, 1024>); opt(step_kernel<64, 512>); opt(step_kernel<64, 256>);
-        opt(exact_finish_kernel<64, 1024>); opt(exact_finish_kernel<64, 512>); opt(exact_finish_kernel<64, 256>);
+        opt(finish_kernel<64, 1024>); opt(finish_kernel<64, 512>);
         if (ntile == 1) cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, scan_kernel<64, 1>, SCAN_THREADS, 0);
         else cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, scan_kernel<64, 2>, SCAN_THREADS, 0);
     }
@@ -586,7 +573,7 @@ int retopk_create_batched(retopk_ctx** out, int B, int H_q, int H_kv, int d, int
     bool ok = dev_alloc(&c->qbar_cache, nh * M * d) && dev_alloc(&c->sup_cache, nh * M * K) &&
               dev_alloc(&c->ws_path, nh) && dev_alloc(&c->ws_rho, nh) && dev_alloc(&c->ws_ncand, nh) &&
               dev_alloc(&c->ws_sel, nh * r) && dev_alloc(&c->ws_gflag, (size_t)B * H_kv + 1) &&
-              dev_alloc(&c->ws_xlist, nh) && dev_alloc(&c->ws_xcount, 2) && dev_alloc(&c->ws_scores, nh * (size_t)c->score_stride) &&
+              dev_alloc(&c->ws_scores, nh * (size_t)c->score_stride) &&
               dev_alloc(&c->ws_tmax, nh * (size_t)c->tmax_stride) &&
               dev_alloc(&c->counters, nh * 4) && dev_alloc(&c->status, 1) &&
               dev_alloc(&c->slow_select, 1) && dev_alloc(&c->scan_groups, 1) && dev_alloc(&c->scan_counter, 1) && dev_alloc(&c->stage_q, nh * d) &&
@@ -630,13 +617,11 @@ int retopk_set_cluster_size(retopk_ctx* c, int ctas_per_head) {
         const int nt = c->finish_threads;
         bool ok;
         if (c->d == 128)
-            ok = nt == 1024 ? cluster_fits(step_kernel<128, 1024>, nt, c->smem_step, ctas_per_head) && cluster_fits(exact_finish_kernel<128, 1024>, nt, c->smem_exact, ctas_per_head)
-               : nt == 512 ? cluster_fits(step_kernel<128, 512>, nt, c->smem_step, ctas_per_head) && cluster_fits(exact_finish_kernel<128, 512>, nt, c->smem_exact, ctas_per_head)
-                           : cluster_fits(step_kernel<128, 256>, nt, c->smem_step, ctas_per_head) && cluster_fits(exact_finish_kernel<128, 256>, nt, c->smem_exact, ctas_per_head);
+            ok = nt == 1024 ? cluster_fits(finish_kernel<128, 1024>, nt, c->smem_finish, ctas_per_head)
+                            : cluster_fits(finish_kernel<128, 512>, nt, c->smem_finish, ctas_per_head);
         else
-            ok = nt == 1024 ? cluster_fits(step_kernel<64, 1024>, nt, c->smem_step, ctas_per_head) && cluster_fits(exact_finish_kernel<64, 1024>, nt, c->smem_exact, ctas_per_head)
-               : nt == 512 ? cluster_fits(step_kernel<64, 512>, nt, c->smem_step, ctas_per_head) && cluster_fits(exact_finish_kernel<64, 512>, nt, c->smem_exact, ctas_per_head)
-                           : cluster_fits(step_kernel<64, 256>, nt, c->smem_step, ctas_per_head) && cluster_fits(exact_finish_kernel<64, 256>, nt, c->smem_exact, ctas_per_head);
+            ok = nt == 1024 ? cluster_fits(finish_kernel<64, 1024>, nt, c->smem_finish, ctas_per_head)
+                            : cluster_fits(finish_kernel<64, 512>, nt, c->smem_finish, ctas_per_head);
         if (!ok) return RETOPK_EUNSUPPORTED;
     }
     c->cluster = ctas_per_head;
@@ -652,7 +637,7 @@ int retopk_debug_fail_next_launch(retopk_ctx* c, int which) {
 int retopk_set_block_shape(retopk_ctx* c, int threads, int ctas_per_sm) {
     if (!c) return RETOPK_EINVAL;
     int id = -1;
-    for (int v = 0; v < 4; ++v)
+    for (int v = 0; v < 3; ++v)
         if (c->shape[v].nt == threads && c->shape[v].per_sm == ctas_per_sm) id = v;
     if (id < 0) return RETOPK_EINVAL;
     if (!c->shape[id].ok) return RETOPK_EUNSUPPORTED;
@@ -713,7 +698,7 @@ int retopk_reset(retopk_ctx* c, void* stream) {
     const size_t nh = (size_t)c->B * c->Hq;
     reset_kernel<<<c->num_sms * 4, 256, 0, static_cast<cudaStream_t>(stream)>>>(
         c->qbar_cache, nh * c->M * c->d, c->sup_cache, nh * c->M * c->K, c->counters, nh * 4, c->ws_gflag,
-        (size_t)c->B * c->Hkv + 1, c->status, c->slow_select, c->scan_groups, c->scan_counter, c->ws_xcount);
+        (size_t)c->B * c->Hkv + 1, c->status, c->slow_select, c->scan_groups, c->scan_counter);
     c->n_ins = 0;
     c->t_dec = 0;
     c->broken = 0;
@@ -740,11 +725,11 @@ int retopk_decode_step(retopk_ctx* c, const void* q, const void* k_cache, const 
         return RETOPK_OK;
     }
     prof_mark(c, 0, s);
-    if ((rc = launch_step(c, a, s)) != RETOPK_OK) return rc;      // nothing of this step is enqueued yet
+    if ((rc = launch_recall(c, a, s)) != RETOPK_OK) return rc;    // nothing of this step is enqueued yet
     prof_mark(c, 1, s);
-    // From here on the step's first kernel is in the stream (normalised queries inserted, exact
-    // heads listed): a failed launch leaves the caches half advanced, so the context refuses
-    // further steps until retopk_reset.
+    // From here on the step's first kernel is in the stream (normalised queries inserted): a
+    // failed launch leaves the caches half advanced, so the context refuses further steps until
+    // retopk_reset.
     if ((rc = launch_scan(c, a, s)) != RETOPK_OK) { c->broken = 1; return rc; }
     prof_mark(c, 2, s);
     if ((rc = launch_finish(c, a, s)) != RETOPK_OK) { c->broken = 1; return rc; }
@@ -774,7 +759,7 @@ int retopk_prefill(retopk_ctx* c, const void* q_tail, const void* k_cache, const
         c->call_serial = (c->call_serial + 1) & 0x3fffffff;
         a.step_id = c->call_serial;
         int rc;
-        if ((rc = launch_step(c, a, s)) != RETOPK_OK) return rc;
+        if ((rc = launch_recall(c, a, s)) != RETOPK_OK) return rc;
         if ((rc = launch_scan(c, a, s)) != RETOPK_OK) { c->broken = 1; return rc; }
         if ((rc = launch_finish(c, a, s)) != RETOPK_OK) { c->broken = 1; return rc; }
         c->n_ins += 1;
@@ -1057,8 +1042,8 @@ int static_setup(int dev, StaticSetup** out) {
         if (cudaDeviceGetAttribute(&st->num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
             cudaDeviceGetAttribute(&st->max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess)
             return RETOPK_ECUDA;
-        if (cudaFuncSetAttribute(exact_finish_kernel<128, 1024>, cudaFuncAttributeMaxDynamicSharedMemorySize, st->max_smem) != cudaSuccess ||
-            cudaFuncSetAttribute(exact_finish_kernel<64, 1024>, cudaFuncAttributeMaxDynamicSharedMemorySize, st->max_smem) != cudaSuccess)
+        if (cudaFuncSetAttribute(finish_kernel<128, 1024>, cudaFuncAttributeMaxDynamicSharedMemorySize, st->max_smem) != cudaSuccess ||
+            cudaFuncSetAttribute(finish_kernel<64, 1024>, cudaFuncAttributeMaxDynamicSharedMemorySize, st->max_smem) != cudaSuccess)
             return RETOPK_ECUDA;
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&st->occ[0][0], scan_kernel<64, 1>, SCAN_THREADS, 0);
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&st->occ[0][1], scan_kernel<64, 2>, SCAN_THREADS, 0);
@@ -1144,8 +1129,8 @@ int exact_topk_decode_static(int B, int H_q, int H_kv, int d, int K, int64_t max
     if (cudaGetLastError() != cudaSuccess) return RETOPK_ECUDA;
     const int cluster = auto_cluster(nh, st->num_sms);
     a.cl_shift = __builtin_ctz((unsigned)cluster);
-    if (d == 128) return launch_dependent(exact_finish_kernel<128, 1024>, (unsigned)(nh * cluster), FINISH_THREADS, smem, s, a, 0, cluster);
-    return launch_dependent(exact_finish_kernel<64, 1024>, (unsigned)(nh * cluster), FINISH_THREADS, smem, s, a, 0, cluster);
+    if (d == 128) return launch_dependent(finish_kernel<128, 1024>, (unsigned)(nh * cluster), FINISH_THREADS, smem, s, a, 0, cluster);
+    return launch_dependent(finish_kernel<64, 1024>, (unsigned)(nh * cluster), FINISH_THREADS, smem, s, a, 0, cluster);
 }
 
 #ifdef RETOPK_PHASE_CLOCKS

@@ -1,25 +1,30 @@
 // Device code of the ReTopK decode step (sm_100a).
 //
-// Three launches per step, all reading caller-owned bf16 q / K / V:
-//   step_kernel    one CTA per (sequence, query head) - or a thread-block cluster of 2-8 CTAs
-//                  when there are few heads, or 512-thread CTAs two to an SM when there are
-//                  more heads than SMs.  Normalise the query, cosine similarity to the cached
-//                  queries (Eq. 6), Top-r recall and rho_max (Eq. 7), path decision (Eq. 13),
-//                  insert of the normalised query.  A head that reuses stays in its CTA to the
-//                  end: candidate union (Eq. 8-9) in a shared-memory bitmap, exact scores of
-//                  the gathered key rows (Eq. 10; the recent window's rows are requested at
-//                  kernel entry and arrive while the cache is searched), Top-K (Eq. 11),
-//                  softmax.V (Eq. 12), support insert.  A head on the exact path flags its KV
-//                  group, takes a ticket in the step's list of exact heads and leaves.
+// Three kernels per step, all reading caller-owned bf16 q / K / V:
+//   recall_kernel  one CTA per (sequence, query head): normalise the query, cosine
+//                  similarity to the cached queries (Eq. 6), Top-r recall and rho_max
+//                  (Eq. 7), path decision (Eq. 13), insert of the normalised query.  A head
+//                  on the exact path flags its KV group.
 //   scan_kernel    persistent CTAs over the flagged KV groups: full-history scores
 //                  e_i = q.k_i/sqrt(d) (Eq. 4); every key row streams once through the
 //                  tensor cores for all G query heads of its group; also the maximum of
 //                  every 16-row tile.  Leaves at once when no group is flagged.
-//   exact_finish_kernel  one CTA (or cluster) per LISTED head: global Top-K (Eq. 1) of the
-//                  scanned scores (tile maxima give a lower bound for the K-th score, only the
-//                  tiles that reach it are read back), softmax.V (Eq. 12), support insert.
-//                  Exact Top-K attention is scan + exact finish with every head listed.
+//   finish_kernel  one CTA per (sequence, query head) - or a thread-block cluster of 2-8 CTAs
+//                  when there are few heads, or 512-thread CTAs two to an SM when there are
+//                  more heads than SMs - with heads of both paths side by side.
+//                  Reuse path: candidate union (Eq. 8-9) in a shared-memory bitmap, exact
+//                  scores of the gathered key rows on the tensor cores (Eq. 10; same MMA path
+//                  as the scan, so a key scores the same bits on either path), Top-K (Eq. 11).
+//                  Exact path: global Top-K (Eq. 1) of the scanned scores (tile maxima give a
+//                  lower bound for the K-th score, only the tiles that reach it are read back).
+//                  Both: softmax.V (Eq. 12) and the support insert.
+//                  Exact Top-K attention is scan + finish with every head on the exact path.
 // All three are programmatic dependent launches; ingest_kernel serves the host-buffer entry point.
+//
+// (One launch per reuse head - recall stage and reuse path in one kernel, the exact heads
+// finished from a list behind the scan - was built and measured: the two launches that are
+// then empty on a reuse-only step cost as much as the recall launch saves, and a step with a
+// few exact heads pays reuse time PLUS scan PLUS exact finish instead of their maximum.)
 #pragma once
 #include <cooperative_groups.h>
 #include <cuda_bf16.h>
@@ -72,9 +77,8 @@ struct StepArgs {
     int tile_cap;            // entries in the exact path's list of hit tiles
     int g_shift;             // log2(G) when G is a power of two, else -1
     int step_id;             // call serial number; a KV group is flagged by storing it
-    int stage_depth;         // rows in flight per row slot in step_kernel's landing zone
-    int exact_stage_depth;   // same for exact_finish_kernel
-    int win_prefetch;        // 1: the window's key rows are requested at kernel entry (they fit the landing zone)
+    int stage_depth;         // rows in flight per row slot in the reuse path's landing zone
+    int exact_stage_depth;   // same for the exact path
     const uint16_t* q;
     const uint16_t* k;
     const uint16_t* v;
@@ -87,8 +91,6 @@ struct StepArgs {
     int32_t* ws_ncand;       // [B*Hq]
     int32_t* ws_sel;         // [B*Hq][r] recalled cache slots, -1 padded
     int32_t* ws_gflag;       // [B*Hkv + 1] == step_id when the group needs a full scan; last word: any group
-    int32_t* ws_xlist;       // [B*Hq] heads on the exact path in this step, in ticket order
-    unsigned int* ws_xcount; // [2] length of that list, by parity of step_id (the other word is cleared for the next step)
     int32_t* dbg_cand;       // [B*Hq][cap] test hook: candidate list of the last reuse step, or null
     float* ws_scores;        // [B*Hq][score_stride]
     float* ws_tmax;          // [B*Hq][tmax_stride] largest score of every 16-row key tile
@@ -97,11 +99,13 @@ struct StepArgs {
     unsigned int* status;
     unsigned long long* slow_select;
     unsigned long long* scan_groups;
-    unsigned int* scan_counter;  // pool cursor of scan_kernel; exact_finish_kernel resets it
+    unsigned int* scan_counter;  // pool cursor of scan_kernel; finish_kernel resets it
     int32_t* idx_out;        // MODE_EXACT only, may be null
-    int cl_shift;            // step_kernel / exact_finish_kernel run 2^cl_shift CTAs (one thread-block cluster) per head
+    int cl_shift;            // finish_kernel runs 2^cl_shift CTAs (one thread-block cluster) per head
     // Fusion-ladder levels below the production one (see retopk_ladder.cuh): the reuse path runs
-    // as separate kernels that hand their intermediates on through these global buffers.
+    // as separate kernels that hand their intermediates on through these global buffers, and
+    // finish_kernel then leaves heads on the reuse path alone.
+    int skip_reuse;
     float* lw_rho;           // [B*Hq][M] similarities
     float* lw_qbar;          // [B*Hq][d] normalised query
     int32_t* lw_cand;        // [B*Hq][cap] candidate indices
@@ -164,7 +168,7 @@ __device__ __forceinline__ void stg_hint(float* p, float v, uint64_t policy) {
     asm volatile("st.global.L2::cache_hint.f32 [%0], %1, %2;" :: "l"(p), "f"(v), "l"(policy) : "memory");
 }
 
-// One tensor-core step of a dot product: 16 rows x 16 bf16 values against 16 x 8 (fp32 accumulate).
+// One tensor-core step of the scan's dot products: 16 rows x 16 bf16 values against 16 x 8 (fp32 accumulate).
 __device__ __forceinline__ void mma_bf16_16816(float* c, uint32_t a0, uint32_t a1, uint32_t a2,
                                                uint32_t a3, uint32_t b0, uint32_t b1) {
     asm volatile(
@@ -172,18 +176,6 @@ __device__ __forceinline__ void mma_bf16_16816(float* c, uint32_t a0, uint32_t a
         "{%8,%9}, {%0,%1,%2,%3};"
         : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
-
-__device__ __forceinline__ float dot8(const uint4& x, const float* qf) {
-    float a = bf16_lo(x.x) * qf[0];
-    a = fmaf(bf16_hi(x.x), qf[1], a);
-    a = fmaf(bf16_lo(x.y), qf[2], a);
-    a = fmaf(bf16_hi(x.y), qf[3], a);
-    a = fmaf(bf16_lo(x.z), qf[4], a);
-    a = fmaf(bf16_hi(x.z), qf[5], a);
-    a = fmaf(bf16_lo(x.w), qf[6], a);
-    a = fmaf(bf16_hi(x.w), qf[7], a);
-    return a;
 }
 
 __device__ __forceinline__ void unpack8(const uint4& x, float* f) {
@@ -350,7 +342,6 @@ struct Threshold {
     uint32_t v;
     int count;
     int need;
-    int ties;       // bin_threshold only: keys equal to v in all (-1: not known)
     uint32_t kmax;
 };
 
@@ -375,7 +366,6 @@ __device__ __noinline__ Threshold count_threshold(const uint32_t* key, int n, in
     Threshold res;
     res.kmax = kmax;
     res.count = n;
-    res.ties = -1;
     int hi = 32 - __clz(kmin ^ kmax);                 // bits [hi-1:0] may differ
     uint32_t prefix = hi >= 32 ? 0u : (kmax >> hi) << hi;
     int kk = K;                                       // rank wanted among the keys matching prefix
@@ -420,11 +410,6 @@ __device__ __noinline__ Threshold count_threshold(const uint32_t* key, int n, in
     return res;
 }
 
-// Cost model of the block-wide pieces below (measured on B200, 1024 threads): a shuffle, a
-// warp reduction or a shared-memory atomic costs about one cycle per WARP that executes it, a
-// barrier about 80 cycles.  So each phase keeps idle warps out of the loop bodies and leaves
-// serial bookkeeping to one warp.
-
 // Per-warp counts cnt (one per warp, written by lane 0 into s_cnt[warp]) -> the number of
 // items in the warps before this one, and the block total.  Call after a barrier.
 template <int NT>
@@ -433,144 +418,6 @@ __device__ __forceinline__ int warp_base(const int* s_cnt, int& total) {
     const int v = lane < NT / 32 ? s_cnt[lane] : 0;
     total = __reduce_add_sync(0xffffffffu, v);
     return __reduce_add_sync(0xffffffffu, lane < warp ? v : 0);
-}
-
-// Threshold by ONE histogram over the span of the scores.  Key i falls into bin
-// floor((score_i - min) / (max - min) * (SEL_BINS - 1)): a monotone map, so every key in a bin
-// above the bin b* that holds the K-th largest key belongs to the top K, and only b*'s members
-// (a handful when the scores are spread) need ranking.  n >= K >= 1.
-//   exact = false: v = the smallest key of the bins b* and above, so at least K keys are >= v
-//                  (a lower bound for the K-th largest key); count = keys >= v.
-//   exact = true : b*'s members are ranked exhaustively by (key desc, position asc): v is the
-//                  K-th largest key, `need` of the keys equal to it belong to the top K and
-//                  `ties` keys equal it in all; count = K + 1 marks that form.  More than
-//                  SEL_LIST members (heavy ties, an outlier that flattens the bins): the radix
-//                  bisection decides instead (ties = -1: not known).
-// A coarse histogram (one bin per 32 fine ones) is kept beside the fine one so that ONE warp
-// finds b* with two 32-lane prefix sums.  s_h: SCRATCH_WORDS ints.  Every thread returns the
-// same result; kmax = largest key.
-template <int NT>
-__device__ Threshold bin_threshold(const uint32_t* key, int n, int K, bool exact, int* s_h) {
-    constexpr int NW = NT / 32, NC = SEL_BINS / 32;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    int* s_bl = s_h + SEL_BINS;                      // boundary list: key[SEL_LIST] position[SEL_LIST]
-    int* s_tot = s_h + SEL_BINS + 2 * SEL_LIST;      // [0,32) minima [32,64) maxima [64,128) coarse bins
-    int* s_res = s_bl;                               // results live in the list's first words until it is filled
-    uint32_t kmin = 0xffffffffu, kmax = 0u;
-    if (warp * 32 < n) {                             // warps without keys skip the reductions
-        for (int i = tid; i < n; i += NT) { const uint32_t k = key[i]; kmin = min(kmin, k); kmax = max(kmax, k); }
-        kmin = __reduce_min_sync(0xffffffffu, kmin);
-        kmax = __reduce_max_sync(0xffffffffu, kmax);
-    }
-    if (lane == 0) { s_tot[warp] = (int)kmin; s_tot[32 + warp] = (int)kmax; }
-#pragma unroll
-    for (int i = tid; i < SEL_BINS; i += NT) s_h[i] = 0;
-    if (tid < NC) s_tot[64 + tid] = 0;
-    __syncthreads();
-    kmin = __reduce_min_sync(0xffffffffu, lane < NW ? (uint32_t)s_tot[lane] : 0xffffffffu);
-    kmax = __reduce_max_sync(0xffffffffu, lane < NW ? (uint32_t)s_tot[32 + lane] : 0u);
-    Threshold res;
-    res.kmax = kmax;
-    res.v = kmax;
-    res.count = n;
-    res.need = K;
-    res.ties = n;
-    if (kmin == kmax) {          // every key equal: v is the K-th largest, the first K in order are taken
-        __syncthreads();
-        return res;
-    }
-    const float smin = key_score(kmin);
-    const float scale = (float)(SEL_BINS - 1) / (key_score(kmax) - smin);
-    auto bin_of = [&](uint32_t k) {
-        const int b = __float2int_rd((key_score(k) - smin) * scale);
-        return min(max(b, 0), SEL_BINS - 1);          // also tames non-finite scores
-    };
-    if (warp * 32 < n)
-        for (int i = tid; i < n; i += NT) {
-            const int b = bin_of(key[i]);
-            atomicAdd(&s_h[b], 1);
-            atomicAdd(&s_tot[64 + (b >> 5)], 1);
-        }
-    __syncthreads();
-    if (warp == 0) {
-        // coarse bins from the top, two per lane, then the 32 fine bins of the coarse bin found
-        const int c0 = s_tot[64 + NC - 1 - 2 * lane], c1 = s_tot[64 + NC - 2 - 2 * lane];
-        int inc = c0 + c1;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) { const int t = __shfl_up_sync(0xffffffffu, inc, o); if (lane >= o) inc += t; }
-        int above = inc - c0 - c1;
-        const unsigned hit = __ballot_sync(0xffffffffu, above < K && K <= inc);
-        const int src = __ffs(hit) - 1;
-        const int first = above < K && K <= above + c0;       // the upper of the lane's two coarse bins
-        int cb = NC - 1 - 2 * lane - (first ? 0 : 1);
-        above += first ? 0 : c0;
-        cb = __shfl_sync(0xffffffffu, cb, src);
-        above = __shfl_sync(0xffffffffu, above, src);
-        const int f = s_h[cb * 32 + 31 - lane];               // fine bins of cb, from the top
-        int finc = f;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) { const int t = __shfl_up_sync(0xffffffffu, finc, o); if (lane >= o) finc += t; }
-        const int fabove = above + finc - f;
-        if (fabove < K && K <= fabove + f) { s_res[0] = cb * 32 + 31 - lane; s_res[1] = fabove; s_res[2] = f; }
-        if (lane == 0) { s_res[3] = 0; s_res[4] = (int)0xffffffffu; }
-    }
-    __syncthreads();
-    const int bstar = s_res[0], above = s_res[1], m = s_res[2];
-    if (!exact) {
-        uint32_t lo = 0xffffffffu;
-        if (warp * 32 < n) {
-            for (int i = tid; i < n; i += NT) { const uint32_t k = key[i]; if (bin_of(k) == bstar) lo = min(lo, k); }
-            lo = __reduce_min_sync(0xffffffffu, lo);
-            if (lane == 0 && lo != 0xffffffffu) atomicMin(reinterpret_cast<unsigned int*>(&s_res[4]), lo);
-        }
-        __syncthreads();
-        res.v = (uint32_t)s_res[4];
-        res.count = above + m;
-        res.need = K - above;
-        res.ties = -1;
-        __syncthreads();
-        return res;
-    }
-    if (m > SEL_LIST - 8) {
-        __syncthreads();
-        res = count_threshold<NT>(key, n, K, 0, s_h);
-        res.ties = -1;
-        return res;
-    }
-    const int need = K - above;                       // 1..m of b*'s members belong to the top K
-    __syncthreads();                                  // s_res is about to be overwritten by the list
-    int* s_len = s_tot + 64;                          // (the coarse bins are dead now)
-    if (tid == 0) s_len[0] = 0;
-    __syncthreads();
-    if (warp * 32 < n)
-        for (int i = tid; i < n; i += NT) {
-            const uint32_t k = key[i];
-            if (bin_of(k) == bstar) {
-                const int p = atomicAdd(&s_len[0], 1);
-                s_bl[p] = (int)k;
-                s_bl[SEL_LIST + p] = i;
-            }
-        }
-    __syncthreads();
-    if (tid < m) {
-        const uint32_t mine = (uint32_t)s_bl[tid];
-        const int pos = s_bl[SEL_LIST + tid];
-        int gt = 0, eq = 0, eq_before = 0;
-        for (int j = 0; j < m; ++j) {
-            const uint32_t o = (uint32_t)s_bl[j];
-            gt += (int)(o > mine);
-            eq += (int)(o == mine);
-            eq_before += (int)(o == mine) & (int)(s_bl[SEL_LIST + j] < pos);
-        }
-        if (gt + eq_before == need - 1) { s_len[1] = (int)mine; s_len[2] = need - gt; s_len[3] = eq; }
-    }
-    __syncthreads();
-    res.v = (uint32_t)s_len[1];
-    res.need = s_len[2];
-    res.ties = s_len[3];
-    res.count = K + 1;
-    __syncthreads();
-    return res;
 }
 
 // Write, in source order, every element with key > v and the first need_eq elements with
@@ -613,44 +460,14 @@ __device__ __noinline__ void ordered_emit(const Src& src, int n, uint32_t vstar,
     }
 }
 
-// The common case of ordered_emit: every key >= v is taken (no tie at v is left out), the
-// source sits in shared memory.  Keys are visited in rounds of NT (key r*NT + tid), a ballot
-// gives each lane its place within the warp, per-(round, warp) counts go through a small
-// table: no shuffle chains.  s_tab: rounds * NT/32 ints (rounds = ceil(n / NT)); needs a barrier
-// before the call if s_tab was in use.
-template <int NT>
-__device__ void ordered_emit_ge(const uint32_t* s_key, const int32_t* s_idx, int n, uint32_t v,
-                                int32_t* s_sup_idx, uint32_t* s_sup_key, int* s_tab) {
-    constexpr int NW = NT / 32;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int rounds = (n + NT - 1) / NT;
-    for (int r = 0; r < rounds; ++r) {
-        const int i = r * NT + tid;
-        const unsigned bal = __ballot_sync(0xffffffffu, i < n && s_key[i] >= v);
-        if (lane == 0) s_tab[r * NW + warp] = __popc(bal);
-    }
-    __syncthreads();
-    int run = 0;                                       // taken in the rounds before r
-    for (int r = 0; r < rounds; ++r) {
-        int total;
-        const int base = run + warp_base<NT>(s_tab + r * NW, total);
-        const int i = r * NT + tid;
-        const uint32_t key = i < n ? s_key[i] : 0u;
-        const bool take = i < n && key >= v;
-        const unsigned bal = __ballot_sync(0xffffffffu, take);
-        if (take) {
-            const int pos = base + __popc(bal & ((1u << lane) - 1u));
-            s_sup_idx[pos] = s_idx[i];
-            s_sup_key[pos] = key;
-        }
-        run += total;
-    }
-}
-
 // ------------------------------------------------------------------------------------
-// The same threshold search and emit for lists of at most R * NT keys, written without loops:
-// every thread keeps its (at most R) keys and bins in registers and all accesses are
-// predicated.  On this hardware a taken branch to code that was not just executed costs about
+// Threshold by ONE histogram over the span of the scores, for lists of at most R * NT keys,
+// written without loops: every thread keeps its (at most R) keys and bins in registers and all
+// accesses are predicated.  Key i falls into bin floor((score_i - min) / (max - min) *
+// (SEL_BINS - 1)): a monotone map, so every key in a bin above the bin b* that holds the K-th
+// largest key belongs to the top K, and only b*'s members (a handful when the scores are
+// spread) need ranking.  A coarse histogram (one bin per 32 fine ones) beside the fine one lets
+// a warp find b* with two 32-lane prefix sums.  On this hardware a taken branch to code that was not just executed costs about
 // a hundred cycles, a barrier about eighty, a straight-line instruction a few: the block-wide
 // phases of a decode step are short, so their cost is the number of branches and barriers on
 // the path, and this form has five barriers and next to no branches.
@@ -808,205 +625,56 @@ __device__ __forceinline__ int select_small(const uint32_t* s_key, const int32_t
 
 // Top-K of the n listed entries (ascending index order in, ascending index order out).
 // kmax_out: largest listed key when known (n > K), else 0 with *kmax_known = false.
-// s_hist: SCRATCH_WORDS words; s_ws: WS_WORDS ints; s_tab: ceil(n / NT) * NT/32 ints that may
-// alias nothing the call reads (the bins of s_hist are used for it when they are large enough).
+// Short lists (at most 3 * NT keys, the usual case) take the loop-free form; longer ones, or
+// a list it hands back (all keys equal, a boundary bin with hundreds of members), the radix
+// bisection and the general emit.  s_hist: SCRATCH_WORDS words; s_ws: WS_WORDS ints.
+// One copy serves both paths of finish_kernel.
 template <int NT>
 __device__ int select_listed(const uint32_t* s_key, const int32_t* s_idx, int n, int K,
-                             int32_t* s_sup_idx, uint32_t* s_sup_key, uint32_t* s_hist, int* s_ws,
-                             uint32_t& kmax, bool& kmax_known) {
+                                          int32_t* s_sup_idx, uint32_t* s_sup_key, uint32_t* s_hist, int* s_ws,
+                                          uint32_t* kmax_out) {
     int ns;
+    uint32_t kmax = 0u;
     if (n <= K) {
-        for (int i = threadIdx.x; i < n; i += NT) { s_sup_idx[i] = s_idx[i]; s_sup_key[i] = s_key[i]; }
+        for (int i = threadIdx.x; i < n; i += NT) { s_sup_idx[i] = s_idx[i]; s_sup_key[i] = s_key[i]; kmax = max(kmax, s_key[i]); }
         ns = n;
-        kmax = 0;
-        kmax_known = false;
+        // (the largest key of a short list: one more reduction, it is rare)
+        kmax = __reduce_max_sync(0xffffffffu, kmax);
+        if ((threadIdx.x & 31) == 0) s_ws[threadIdx.x >> 5] = (int)kmax;
+        __syncthreads();
+        kmax = __reduce_max_sync(0xffffffffu, (threadIdx.x & 31) < NT / 32 ? (uint32_t)s_ws[threadIdx.x & 31] : 0u);
     } else if (n <= 3 * NT && select_small<NT, 3, true>(s_key, s_idx, n, K, s_sup_idx, s_sup_key,
                                                            reinterpret_cast<int*>(s_hist), &kmax, nullptr)) {
         ns = K;
-        kmax_known = true;
     } else {
         __syncthreads();                               // (the short form may have left the scratch in use)
-        const Threshold t = bin_threshold<NT>(s_key, n, K, true, reinterpret_cast<int*>(s_hist));
-        const int rounds = (n + NT - 1) / NT;
-        if (t.count != K && t.ties == t.need && rounds * (NT / 32) <= SEL_BINS) {
-            // every key equal to the K-th largest is taken: plain ">= v" (the histogram bins are free again)
-            ordered_emit_ge<NT>(s_key, s_idx, n, t.v, s_sup_idx, s_sup_key, reinterpret_cast<int*>(s_hist));
-        } else {
-            SmemSrc src{s_key, s_idx};
-            uint32_t vstar;
-            int need_eq;
-            if (t.count == K) { vstar = t.v - 1u; need_eq = 0; }            // exactly K keys are >= v
-            else { vstar = t.v; need_eq = t.need; }                          // v = K-th largest key
-            ordered_emit<NT>(src, n, vstar, need_eq, s_sup_idx, s_sup_key, s_ws);
-        }
+        SmemSrc src{s_key, s_idx};
+        const Threshold t = count_threshold<NT>(s_key, n, K, 0, reinterpret_cast<int*>(s_hist));
+        uint32_t vstar;
+        int need_eq;
+        if (t.count == K) { vstar = t.v - 1u; need_eq = 0; }            // exactly K keys are >= v
+        else { vstar = t.v; need_eq = t.need; }                          // v = K-th largest key
+        ordered_emit<NT>(src, n, vstar, need_eq, s_sup_idx, s_sup_key, s_ws);
         ns = K;
         kmax = t.kmax;
-        kmax_known = true;
     }
     __syncthreads();
+    *kmax_out = kmax;
     return ns;
 }
 
-// Sum each of eight per-lane partials a[0..7] over the LPR lanes of a row group, trading
-// values between lanes as the tree narrows (7-8 shuffles instead of 8 * log2(LPR)).
-// Returns the total of row `row`; for LPR = 16 both lanes of a pair hold the same row.
-template <int LPR>
-__device__ __forceinline__ float reduce8_across(const float* a, int sub, int& row) {
-    float b[4], c[2], d;
-    if (LPR == 16) {
-        const bool h8 = sub & 8, h4 = sub & 4, h2 = sub & 2;
-#pragma unroll
-        for (int j = 0; j < 4; ++j)
-            b[j] = (h8 ? a[j + 4] : a[j]) + __shfl_xor_sync(0xffffffffu, h8 ? a[j] : a[j + 4], 8);
-#pragma unroll
-        for (int j = 0; j < 2; ++j)
-            c[j] = (h4 ? b[j + 2] : b[j]) + __shfl_xor_sync(0xffffffffu, h4 ? b[j] : b[j + 2], 4);
-        d = (h2 ? c[1] : c[0]) + __shfl_xor_sync(0xffffffffu, h2 ? c[0] : c[1], 2);
-        d += __shfl_xor_sync(0xffffffffu, d, 1);
-        row = sub >> 1;
-    } else {
-        const bool h4 = sub & 4, h2 = sub & 2, h1 = sub & 1;
-#pragma unroll
-        for (int j = 0; j < 4; ++j)
-            b[j] = (h4 ? a[j + 4] : a[j]) + __shfl_xor_sync(0xffffffffu, h4 ? a[j] : a[j + 4], 4);
-#pragma unroll
-        for (int j = 0; j < 2; ++j)
-            c[j] = (h2 ? b[j + 2] : b[j]) + __shfl_xor_sync(0xffffffffu, h2 ? b[j] : b[j + 2], 2);
-        d = (h1 ? c[1] : c[0]) + __shfl_xor_sync(0xffffffffu, h1 ? c[0] : c[1], 1);
-        row = sub;
-    }
-    return d;
-}
-
-// ------------------------------------------------------------------------------------
-// Eq. 12: out = sum_i softmax(e)_i v_i over the ns selected rows.
-// The value rows are fetched with 16-byte asynchronous copies into a per-thread landing
-// zone (depth rows per row slot in flight at once); the softmax weights are computed while
-// the first wave is in the air.  s_w: ns floats; s_red: (NT/32) * D + NT floats; s_ws: 32
-// words; s_stage: depth * NT uint4.
-// With a cluster of cl_size CTAs per head (every CTA holding the same support), CTA cl_rank
-// fetches and weighs its contiguous share of the rows; the partial sums meet in rank 0
-// through distributed shared memory and are added there in rank order.
-// ------------------------------------------------------------------------------------
-template <int D, int NT>
-__device__ void attend(const uint16_t* vbase, int ns, const int32_t* s_sup_idx, const uint32_t* s_sup_key,
-                       float* s_w, float* s_red, int* s_ws, uint4* s_stage, int depth, uint32_t kmax,
-                       bool kmax_known, uint16_t* out_row, int cl_rank = 0, int cl_size = 1) {
-    constexpr int LPR = D / 8;                  // lanes per bf16 row (16 bytes each)
-    constexpr int RPW = 32 / LPR;               // rows per warp load
-    constexpr int SLOTS = (NT / 32) * RPW;      // row slots per block
-    constexpr int NW = NT / 32;
-    constexpr int PARTS = NT / D;               // second-stage partial sums
+// Largest key of s_key[0..n) (the rare callers that select without learning it).  Ends with a barrier.
+template <int NT>
+__device__ __noinline__ uint32_t block_max_key(const uint32_t* s_key, int n, int* s_ws) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int sub = lane % LPR, myslot = warp * RPW + lane / LPR;
-    const char* vsrc = reinterpret_cast<const char*>(vbase) + sub * 16;
-    uint4* my_stage = s_stage + tid;
-    // this CTA's share of the support: [i_lo, i_hi)
-    const int share = (ns + cl_size - 1) / cl_size;
-    const int i_lo = min(ns, cl_rank * share), i_hi = min(ns, i_lo + share);
-
-    auto issue = [&](int base) {
-#pragma unroll 4
-        for (int u = 0; u < depth; ++u) {
-            const int i = base + u * SLOTS + myslot;
-            if (i < i_hi) cp_async16(my_stage + u * NT, vsrc + (size_t)s_sup_idx[i] * (D * 2));
-        }
-        cp_async_commit();
-    };
-    issue(i_lo);
-    RETOPK_PHASE(0, 20);
-
-    if (__builtin_expect(!kmax_known, 0)) {
-        kmax = 0;
-        for (int i = tid; i < ns; i += NT) kmax = max(kmax, s_sup_key[i]);
-        kmax = __reduce_max_sync(0xffffffffu, kmax);
-        if (lane == 0) s_ws[warp] = (int)kmax;
-        __syncthreads();
-        kmax = __reduce_max_sync(0xffffffffu, lane < NW ? (uint32_t)s_ws[lane] : 0u);
-        __syncthreads();
-    }
-    const float smax = key_score(kmax);
-    float wsum = 0.f;
-    for (int i = tid; i < ns; i += NT) {
-        const float w = expf(key_score(s_sup_key[i]) - smax);
-        s_w[i] = w;
-        wsum += w;
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) wsum += __shfl_xor_sync(0xffffffffu, wsum, o);
-    float* s_wsf = reinterpret_cast<float*>(s_ws);
-    if (lane == 0) s_wsf[warp] = wsum;
-    RETOPK_PHASE(0, 21);
-
-    float acc[8];
-#pragma unroll
-    for (int e = 0; e < 8; ++e) acc[e] = 0.f;
-    float denom = 0.f;
-    for (int base = i_lo;;) {
-        cp_async_wait_all();
-        if (base == i_lo) {
-            __syncthreads();                                     // weights and their partial sums are complete
-            denom = lane < NW ? s_wsf[lane] : 0.f;               // fixed tree: the same sum on every lane and run
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) denom += __shfl_xor_sync(0xffffffffu, denom, o);
-        }
-        RETOPK_PHASE(0, 22);
-        for (int u = 0; u < depth; ++u) {
-            const int i = base + u * SLOTS + myslot;
-            if (i < i_hi) {
-                const float w = s_w[i];
-                float f[8];
-                unpack8(my_stage[u * NT], f);
-#pragma unroll
-                for (int e = 0; e < 8; ++e) acc[e] = fmaf(w, f[e], acc[e]);
-            }
-        }
-        base += SLOTS * depth;
-        if (base >= i_hi) break;
-        issue(base);
-    }
-    // fixed-order reduction: row slots of a warp, then warps in groups, then groups
-    RETOPK_PHASE(0, 23);
-#pragma unroll
-    for (int o = LPR; o < 32; o <<= 1)
-#pragma unroll
-        for (int e = 0; e < 8; ++e) acc[e] += __shfl_xor_sync(0xffffffffu, acc[e], o);
-    if (lane < LPR) {
-#pragma unroll
-        for (int e = 0; e < 8; ++e) s_red[warp * D + sub * 8 + e] = acc[e];
-    }
+    uint32_t kmax = 0u;
+    for (int i = tid; i < n; i += NT) kmax = max(kmax, s_key[i]);
+    kmax = __reduce_max_sync(0xffffffffu, kmax);
+    if (lane == 0) s_ws[warp] = (int)kmax;
     __syncthreads();
-    {
-        const int j = tid % D, part = tid / D;
-        constexpr int WPP = NW / PARTS;          // warps per part
-        float sum = 0.f;
-#pragma unroll
-        for (int w = 0; w < WPP; ++w) sum += s_red[(part * WPP + w) * D + j];
-        s_red[NW * D + part * D + j] = sum;
-    }
+    kmax = __reduce_max_sync(0xffffffffu, lane < NT / 32 ? (uint32_t)s_ws[lane] : 0u);
     __syncthreads();
-    float sum = 0.f;
-    if (tid < D) {
-#pragma unroll
-        for (int p = 0; p < PARTS; ++p) sum += s_red[NW * D + p * D + tid];
-    }
-    if (cl_size > 1) {
-        // s_red[0..D) is free again (its readers passed the barrier above)
-        namespace cg = cooperative_groups;
-        cg::cluster_group cluster = cg::this_cluster();
-        if (tid < D) s_red[tid] = sum;
-        cluster.sync();
-        if (cl_rank == 0 && tid < D) {
-            sum = 0.f;
-            for (int r = 0; r < cl_size; ++r) sum += *cluster.map_shared_rank(s_red + tid, r);
-        }
-        cluster.sync();           // nobody leaves while its shared memory may still be read
-        if (cl_rank != 0) return;
-    }
-    if (tid < D) {
-        const float o = ns > 0 ? sum / denom : 0.f;
-        out_row[tid] = __bfloat16_as_ushort(__float2bfloat16_rn(o));
-    }
+    return kmax;
 }
 
 // ------------------------------------------------------------------------------------
@@ -1030,23 +698,17 @@ __device__ __forceinline__ float reduce4_across32(const float* a, int lane, int&
     return c;
 }
 
-// Eq. 6: rho_c = (qbar_c . q) / |q| for every cached entry c < fill into s_rho[c], the
-// normalised query into s_q[0..D) and, if asked for, the raw query as packed bf16 pairs into
-// s_qpk[0..D/2) (the B operand of the tensor-core candidate scores).  Every warp reads the
-// query itself (four elements per lane) next to its cache rows, so one memory latency covers
-// both.  after_issue() runs once the first trip's loads are on their way (a place to request
-// other rows without delaying these).  No barrier at the end.
-struct NoHook { __device__ __forceinline__ void operator()() const {} };
-template <int D, int NT, class Hook = NoHook>
-__device__ __forceinline__ void cache_similarities(const StepArgs& a, int bh, float* s_q, float* s_rho,
-                                                   uint32_t* s_qpk = nullptr, Hook after_issue = Hook()) {
+// Eq. 6: rho_c = (qbar_c . q) / |q| for every cached entry c < fill into s_rho[c], and the
+// normalised query into s_q[0..D).  Every warp reads the query itself (four elements per
+// lane) next to its cache rows, so one memory latency covers both.  No barrier at the end.
+template <int D, int NT>
+__device__ __forceinline__ void cache_similarities(const StepArgs& a, int bh, float* s_q, float* s_rho) {
     constexpr int NW = NT / 32;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int M = a.M, fill = a.fill;
     float q4[4] = {0.f, 0.f, 0.f, 0.f};
-    uint2 raw = make_uint2(0u, 0u);
     if (lane < D / 4) {
-        raw = *reinterpret_cast<const uint2*>(a.q + (size_t)bh * D + 4 * lane);
+        const uint2 raw = *reinterpret_cast<const uint2*>(a.q + (size_t)bh * D + 4 * lane);
         q4[0] = bf16_lo(raw.x); q4[1] = bf16_hi(raw.x); q4[2] = bf16_lo(raw.y); q4[3] = bf16_hi(raw.y);
     }
     float inv_nrm = 0.f;
@@ -1060,7 +722,6 @@ __device__ __forceinline__ void cache_similarities(const StepArgs& a, int bh, fl
                                               : make_float4(0.f, 0.f, 0.f, 0.f);
         }
         if (c0 == warp) {
-            after_issue();
             // first trip: the query norm while the loads fly
             float n2 = q4[0] * q4[0];
             n2 = fmaf(q4[1], q4[1], n2); n2 = fmaf(q4[2], q4[2], n2); n2 = fmaf(q4[3], q4[3], n2);
@@ -1071,7 +732,6 @@ __device__ __forceinline__ void cache_similarities(const StepArgs& a, int bh, fl
             if (warp == 0 && lane < D / 4) {
 #pragma unroll
                 for (int e = 0; e < 4; ++e) s_q[4 * lane + e] = nrm > 0.f ? q4[e] / nrm : 0.f;
-                if (s_qpk) { s_qpk[2 * lane] = raw.x; s_qpk[2 * lane + 1] = raw.y; }
             }
         }
         if (c0 >= fill) continue;                      // (warp-uniform) nothing cached for this warp
@@ -1215,8 +875,7 @@ __device__ __forceinline__ int decide_path(const StepArgs& a, float rho_max) {
 }
 
 // Leave the decision of one head where the later kernels (and the caller) find it; a head
-// on the exact path flags its KV group for the scan and takes a ticket in the step's list of
-// exact heads (one atomic add; nobody waits on the list inside this kernel).
+// on the exact path flags its KV group for the scan.
 __device__ __forceinline__ void record_decision(const StepArgs& a, int bh, int bkv, const int* s_sel, int path,
                                                 float rho_max) {
     const int tid = threadIdx.x;
@@ -1228,7 +887,6 @@ __device__ __forceinline__ void record_decision(const StepArgs& a, int bh, int b
             a.ws_gflag[bkv] = a.step_id;       // same value from every head of the group
             a.ws_gflag[a.B * a.Hkv] = a.step_id;   // "some group needs a scan in this step"
             a.ws_ncand[bh] = a.L;
-            a.ws_xlist[atomicAdd(a.ws_xcount + (a.step_id & 1), 1u)] = bh;
             if (!a.prefill) atomicAdd(a.counters + (size_t)bh * 4 + path, 1ull);   // no return value: not waited for
         }
     }
@@ -1238,273 +896,335 @@ __device__ __forceinline__ void record_decision(const StepArgs& a, int bh, int b
 // Pieces of the reuse path (one block per head).
 // ------------------------------------------------------------------------------------
 
-// Eq. 8-9, first half: the recalled supports' indices below the window set their bit in a
-// bitmap over key positions (the window is a contiguous run added later, whatever the supports
-// held there).  The bitmap must be clear and s_sel loaded (barrier before the call).  `pre`
-// holds element tid of the first four recalled lists when have_pre (loaded ahead by the caller
-// so that other work overlaps their latency); everything else is loaded here.  No barrier at the end.
-template <int NT>
-__device__ __forceinline__ void union_load_first(const StepArgs& a, int bh, const int* sel8, int* pre) {
+// ------------------------------------------------------------------------------------
+// recall_kernel: Eq. 6, Eq. 7, Eq. 13 and the insert of the normalised query, per head.
+// Leaves the recalled slots, rho_max and the path in global memory and flags the KV group
+// of every head that takes the exact path.  Layout (words): q[D] rho[M+] ws[WS_WORDS] sel[r+] misc[4].
+// ------------------------------------------------------------------------------------
+constexpr int RECALL_THREADS = 1024;
+template <int D>
+__global__ void __launch_bounds__(RECALL_THREADS, 1) recall_kernel(const StepArgs a) {
+    constexpr int NT = RECALL_THREADS;
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    float* s_q = reinterpret_cast<float*>(smem_raw);
+    float* s_rho = s_q + D;
+    int* s_ws = reinterpret_cast<int*>(s_rho + ((a.M + 3) & ~3));
+    int* s_sel = s_ws + WS_WORDS;
+    float* s_misc = reinterpret_cast<float*>(s_sel + ((a.r + 3) & ~3));
+
     const int tid = threadIdx.x;
-#pragma unroll
-    for (int u = 0; u < 4; ++u) {
-        const int c = sel8[u];
-        pre[u] = (c >= 0 && tid < a.K) ? a.sup_cache[((size_t)bh * a.M + c) * a.K + tid] : -1;
-    }
+    const int bh = blockIdx.x;
+    const int bkv = kv_group_of(bh, a);
+    if (tid < a.r) s_sel[tid] = -1;
+    if (tid == 0) s_misc[0] = -CUDART_INF_F;
+    pdl_wait();        // the caches were written by the step before; q by whatever ran before this call
+    RETOPK_PHASE(1, 0);
+    cache_similarities<D, NT>(a, bh, s_q, s_rho);
+    __syncthreads();
+    RETOPK_PHASE(1, 1);
+    int sel8[8];
+    const float rho_max = recall_slots<NT>(a, s_rho, s_sel, s_misc, s_ws, sel8);
+    RETOPK_PHASE(1, 3);
+    const int path = decide_path(a, rho_max);
+    // insert the normalised query now: every similarity of this step has been taken
+    if (tid < D) store_qbar(a, ((size_t)bh * a.M + a.slot) * D + tid, s_q[tid]);
+    record_decision(a, bh, bkv, s_sel, path, rho_max);
+    RETOPK_PHASE(1, 2);
 }
-// The whole of union_mark when the four lists of union_load_first are all there is (at most
-// four recalled slots, K <= NT): no loops.  Returns false (nothing done) otherwise.
-template <int NT>
-__device__ __forceinline__ bool union_mark_short(const StepArgs& a, int n_sel, uint32_t* s_bm, const int* pre) {
-    if (__builtin_expect(n_sel > 4 || a.K > NT, 0)) return false;
-    const int L = a.L;
-    const int w_lo = L - a.W > 0 ? L - a.W : 0;
-    bool bad = false;
-#pragma unroll
-    for (int u = 0; u < 4; ++u) {
-        const int x = pre[u];
-        if (x >= 0 && x < w_lo) atomicOr(&s_bm[x >> 5], 1u << (x & 31));
-        bad = bad || x >= L;
-    }
-    if (__builtin_expect(bad, 0)) atomicOr(a.status, 1u);
-    return true;
+
+// ------------------------------------------------------------------------------------
+// Pieces of the reuse path (one block per head).
+// ------------------------------------------------------------------------------------
+
+// Eight bf16 values (16 bytes of a key row) against eight query values.
+__device__ __forceinline__ float dot8(const uint4& x, const float* qf) {
+    float a = bf16_lo(x.x) * qf[0];
+    a = fmaf(bf16_hi(x.x), qf[1], a);
+    a = fmaf(bf16_lo(x.y), qf[2], a);
+    a = fmaf(bf16_hi(x.y), qf[3], a);
+    a = fmaf(bf16_lo(x.z), qf[4], a);
+    a = fmaf(bf16_hi(x.z), qf[5], a);
+    a = fmaf(bf16_lo(x.w), qf[6], a);
+    a = fmaf(bf16_hi(x.w), qf[7], a);
+    return a;
 }
+
+// Sum each of eight per-lane partials a[0..7] over the LPR lanes of a row group, trading
+// values between lanes as the tree narrows (7-8 shuffles instead of 8 * log2(LPR)).
+// Returns the total of row `row`; for LPR = 16 both lanes of a pair hold the same row.
+template <int LPR>
+__device__ __forceinline__ float reduce8_across(const float* a, int sub, int& row) {
+    float b[4], c[2], d;
+    if (LPR == 16) {
+        const bool h8 = sub & 8, h4 = sub & 4, h2 = sub & 2;
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            b[j] = (h8 ? a[j + 4] : a[j]) + __shfl_xor_sync(0xffffffffu, h8 ? a[j] : a[j + 4], 8);
+#pragma unroll
+        for (int j = 0; j < 2; ++j)
+            c[j] = (h4 ? b[j + 2] : b[j]) + __shfl_xor_sync(0xffffffffu, h4 ? b[j] : b[j + 2], 4);
+        d = (h2 ? c[1] : c[0]) + __shfl_xor_sync(0xffffffffu, h2 ? c[0] : c[1], 2);
+        d += __shfl_xor_sync(0xffffffffu, d, 1);
+        row = sub >> 1;
+    } else {
+        const bool h4 = sub & 4, h2 = sub & 2, h1 = sub & 1;
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            b[j] = (h4 ? a[j + 4] : a[j]) + __shfl_xor_sync(0xffffffffu, h4 ? a[j] : a[j + 4], 4);
+#pragma unroll
+        for (int j = 0; j < 2; ++j)
+            c[j] = (h2 ? b[j + 2] : b[j]) + __shfl_xor_sync(0xffffffffu, h2 ? b[j] : b[j + 2], 2);
+        d = (h1 ? c[1] : c[0]) + __shfl_xor_sync(0xffffffffu, h1 ? c[0] : c[1], 1);
+        row = sub;
+    }
+    return d;
+}
+
+// Eq. 8-9: the sorted unique candidate list of head bh into s_idx; returns its length.
+// Recalled indices below the window go through a bitmap over key positions (ordered
+// extraction = sorted and deduplicated for free); the window itself is a contiguous run
+// appended behind them, whatever the supports held there.  The bitmap must be clear and
+// s_sel loaded (barrier before the call); no barrier at the end.
 template <int NT>
-__device__ __forceinline__ void union_mark(const StepArgs& a, int bh, const int* s_sel, int n_sel, uint32_t* s_bm,
-                                           const int* pre, bool have_pre) {
+__device__ __forceinline__ int candidate_union(const StepArgs& a, int bh, const int* s_sel, int n_sel,
+                                               uint32_t* s_bm, int32_t* s_idx, int* s_ws) {
     const int tid = threadIdx.x;
     const int M = a.M, L = a.L, K = a.K;
     const int w_lo = L - a.W > 0 ? L - a.W : 0;
-    bool bad = false;
-    for (int s0 = 0; s0 < n_sel; s0 += 4)
-        for (int i = tid; i < K; i += NT) {
-            int idx[4];
-            const bool use_pre = have_pre && s0 == 0 && i == tid;
+    {
+        bool bad = false;
+        for (int s0 = 0; s0 < n_sel; s0 += 4)
+            for (int i = tid; i < K; i += NT) {
+                int idx[4];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const int c = s0 + u < n_sel ? s_sel[s0 + u] : -1;
-                idx[u] = use_pre ? pre[u] : (c >= 0 ? a.sup_cache[((size_t)bh * M + c) * K + i] : -1);
-            }
-#pragma unroll
-            for (int u = 0; u < 4; ++u)
-                if (idx[u] >= 0) {
-                    if (idx[u] < w_lo) atomicOr(&s_bm[idx[u] >> 5], 1u << (idx[u] & 31));
-                    else if (idx[u] >= L) bad = true;
+                for (int u = 0; u < 4; ++u) {
+                    const int c = s0 + u < n_sel ? s_sel[s0 + u] : -1;
+                    idx[u] = c >= 0 ? a.sup_cache[((size_t)bh * M + c) * K + i] : -1;
                 }
-        }
-    if (bad) atomicOr(a.status, 1u);
-}
-
-// Eq. 8-9, second half: ordered extraction of the bitmap (sorted and deduplicated for free)
-// into s_idx, the window appended behind as a run; returns the list's length.  The bitmap
-// must be complete (barrier before the call); no barrier at the end.  Every thread that takes
-// part owns a whole number of 16-byte pieces of the bitmap; only the warps that own words run
-// the prefix sum.  s_ws: WS_WORDS ints.
-template <int NT>
-__device__ __forceinline__ int union_extract(const StepArgs& a, const uint32_t* s_bm, int32_t* s_idx, int* s_ws) {
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int L = a.L;
-    const int w_lo = L - a.W > 0 ? L - a.W : 0;
-    const int nq = (((w_lo + 31) >> 5) + 3) >> 2;     // 16-byte pieces that can hold bits below the window
-    const int qpt = (nq + NT - 1) / NT;               // pieces per thread
-    const int q0 = tid * qpt;
-    const int q1 = (q0 + qpt < nq) ? q0 + qpt : nq;
-    const uint4* bm4 = reinterpret_cast<const uint4*>(s_bm);
-    int cnt = 0, inc = 0;
-    if (warp * 32 * qpt < nq) {                        // (warp-uniform) this warp owns words
-        for (int p = q0; p < q1; ++p) {
-            const uint4 x = bm4[p];
-            cnt += __popc(x.x) + __popc(x.y) + __popc(x.z) + __popc(x.w);
-        }
-        inc = cnt;
 #pragma unroll
-        for (int o = 1; o < 32; o <<= 1) { const int t = __shfl_up_sync(0xffffffffu, inc, o); if (lane >= o) inc += t; }
-    }
-    if (lane == 31) s_ws[warp] = inc;
-    __syncthreads();
-    RETOPK_PHASE(0, 7);
-    int n_low;
-    int pos = warp_base<NT>(s_ws, n_low) + inc - cnt;
-    if (cnt)
-        for (int p = q0; p < q1; ++p) {
-            uint4 x = bm4[p];
-            // one trip per set bit, lowest first: the word is picked with selects, not branches
-            for (int left = __popc(x.x) + __popc(x.y) + __popc(x.z) + __popc(x.w); left > 0; --left) {
-                const int e = x.x ? 0 : x.y ? 1 : x.z ? 2 : 3;
-                const uint32_t w = e == 0 ? x.x : e == 1 ? x.y : e == 2 ? x.z : x.w;
-                const int bit = __ffs(w) - 1;
-                s_idx[pos++] = (p * 4 + e) * 32 + bit;
-                const uint32_t rest = w & (w - 1);
-                x.x = e == 0 ? rest : x.x; x.y = e == 1 ? rest : x.y; x.z = e == 2 ? rest : x.z; x.w = e == 3 ? rest : x.w;
+                for (int u = 0; u < 4; ++u)
+                    if (idx[u] >= 0) {
+                        if (idx[u] < w_lo) atomicOr(&s_bm[idx[u] >> 5], 1u << (idx[u] & 31));
+                        else if (idx[u] >= L) bad = true;
+                    }
             }
+        if (bad) atomicOr(a.status, 1u);
+    }
+    __syncthreads();
+    RETOPK_PHASE(0, 2);
+    const int nw_lo = (w_lo + 31) >> 5;               // words that can hold bits below the window
+    const int wpt = (nw_lo + NT - 1) / NT;
+    const int w0 = tid * wpt;
+    const int w1 = (w0 + wpt < nw_lo) ? w0 + wpt : nw_lo;
+    int cnt = 0;
+    for (int w = w0; w < w1; ++w) cnt += __popc(s_bm[w]);
+    int n_low;
+    int pos = block_excl_scan<NT>(cnt, s_ws, n_low);
+    for (int w = w0; w < w1; ++w) {
+        uint32_t bits = s_bm[w];
+        while (bits) {
+            const int bit = __ffs(bits) - 1;
+            s_idx[pos++] = w * 32 + bit;
+            bits &= bits - 1;
         }
-    RETOPK_PHASE(0, 19);
+    }
     for (int i = w_lo + tid; i < L; i += NT) s_idx[n_low + (i - w_lo)] = i;
     return n_low + (L - w_lo);
 }
 
-// Eq. 8-9 in one piece: the sorted unique candidate list of head bh into s_idx; returns its
-// length.  The bitmap must be clear and s_sel loaded (barrier before the call); no barrier at
-// the end.
-template <int NT>
-__device__ __forceinline__ int candidate_union(const StepArgs& a, int bh, const int* s_sel, int n_sel,
-                                               uint32_t* s_bm, int32_t* s_idx, int* s_ws) {
-    union_mark<NT>(a, bh, s_sel, n_sel, s_bm, nullptr, false);
-    __syncthreads();
-    return union_extract<NT>(a, s_bm, s_idx, s_ws);
-}
-
-// ------------------------------------------------------------------------------------
-// Eq. 10 on the tensor cores.  Gathered key rows are staged in tiles of 16 rows, the A operand
-// of mma.m16n8k16 (bf16 -> fp32); the query is column 0 of the B operand.  A dot product does
-// not care in which order its terms are paired, so each thread reads 16 contiguous bytes of a
-// staged row straight into its A-fragment registers and the query fragment is permuted to
-// match - the same fragment trick, MMA order and scaling as scan_kernel, so a key scores the
-// same bits on either path.  The 16-byte piece c of tile row rho sits at
-//     tile * 16 * PITCH + rho * PITCH + ((c ^ ((rho & 1) << 2)) << 4),   PITCH = 2 * D bytes,
-// which keeps the fragment reads of a quarter warp (rows g and g + 1, pieces t + 4j) on
-// distinct banks.
-// ------------------------------------------------------------------------------------
-template <int D>
-__device__ __forceinline__ unsigned tile_piece_offset(int row, int c) {
-    const int rho = row & 15;
-    return (unsigned)(row >> 4) * (32 * D) + rho * (2 * D) + ((c ^ ((rho & 1) << 2)) << 4);
-}
-
-// Request rows [r0, r1) of a chunk (row i of the chunk is kbase[row_of[i]] or kbase[first + i])
-// into the staging tiles; every lane copies one 16-byte piece per trip.  No commit.
+// Eq. 10: exact current-query scores of n key rows as order-preserving keys into key_out.
+// Row i is kbase[row_of[i]] (INDEXED) or kbase[i] (rows already packed).  Every lane copies
+// its 16 bytes of each row asynchronously into its own landing zone and reads them back
+// itself, so a whole wave of rows is in flight with no registers held and no barrier.
+// s_qraw: the raw query as D floats; s_stage: depth * NT uint4.  No barrier at the end.
 template <int D, int NT, bool INDEXED>
-__device__ __forceinline__ void rows_request(const uint16_t* kbase, const int32_t* row_of, int first, int r0, int r1,
-                                             unsigned char* s_stage) {
+__device__ __forceinline__ void score_candidates(const uint16_t* kbase, const int32_t* row_of, int n,
+                                                 const float* s_qraw, uint4* s_stage, int depth, float scale,
+                                                 uint32_t* key_out) {
     constexpr int LPR = D / 8, RPW = 32 / LPR, SLOTS = (NT / 32) * RPW;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int sub = lane % LPR, myslot = warp * RPW + lane / LPR;
-    const char* src = reinterpret_cast<const char*>(kbase) + sub * 16;
-    for (int i = r0 + myslot; i < r1; i += SLOTS)
-        cp_async16(s_stage + tile_piece_offset<D>(i, sub), src + (size_t)(INDEXED ? row_of[i] : first + i) * (D * 2));
-}
-
-// Scores of the staged rows [r0, r1) of a chunk (r0 a multiple of 16; their copies complete and
-// visible to the block: wait + barrier before the call) as order-preserving keys into
-// key_out[r0..r1).  One warp per tile.  s_qpk: the raw query as D/2 packed bf16 pairs.
-template <int D, int NT>
-__device__ __forceinline__ void rows_score(const unsigned char* s_stage, int r0, int r1, const uint32_t* s_qpk,
-                                           float scale, uint32_t* key_out) {
-    constexpr int NJ = D / 32, NW = NT / 32;
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int g = lane >> 2, t = lane & 3;
-    if ((r0 >> 4) + warp >= (r1 + 15) >> 4) return;          // no tile for this warp
-    uint32_t bq[NJ][2][2];
-#pragma unroll
-    for (int j = 0; j < NJ; ++j)
-#pragma unroll
-        for (int p = 0; p < 2; ++p) {
-            const int w = j * 16 + t * 4 + 2 * p;
-            bq[j][p][0] = g == 0 ? s_qpk[w] : 0u;            // the query is column 0 of B
-            bq[j][p][1] = g == 0 ? s_qpk[w + 1] : 0u;
+    const char* ksrc = reinterpret_cast<const char*>(kbase) + sub * 16;
+    float qf[8];
+    *reinterpret_cast<float4*>(qf) = *reinterpret_cast<const float4*>(s_qraw + sub * 8);
+    *reinterpret_cast<float4*>(qf + 4) = *reinterpret_cast<const float4*>(s_qraw + sub * 8 + 4);
+    uint4* my_stage = s_stage + tid;
+    // each wave goes out as two groups of copies, so that the dot products of the first
+    // half run while the second half is still arriving
+    const int half = (depth + 1) / 2;
+    for (int base = 0; base < n; base += SLOTS * depth) {
+#pragma unroll 4
+        for (int u = 0; u < depth; ++u) {
+            const int i = base + u * SLOTS + myslot;
+            if (i < n) cp_async16(my_stage + u * NT, ksrc + (size_t)(INDEXED ? row_of[i] : i) * (D * 2));
+            if (u == half - 1) cp_async_commit();
         }
-    const unsigned swz = (unsigned)(g & 1) << 2;
-    for (int tile = (r0 >> 4) + warp; tile * 16 < r1; tile += NW) {
-        const unsigned char* base = s_stage + (size_t)tile * (32 * D);
-        uint4 x[NJ], y[NJ];
+        cp_async_commit();
+        for (int g2 = 0; g2 < 2; ++g2) {
+            if (g2 == 0) cp_async_wait_but_one();
+            else cp_async_wait_all();
+            const int u_begin = g2 == 0 ? 0 : half, u_end = g2 == 0 ? half : depth;
+            for (int u0 = u_begin; u0 < u_end; u0 += 8) {
+                float part[8];
 #pragma unroll
-        for (int j = 0; j < NJ; ++j) {
-            const unsigned piece = ((unsigned)(t + 4 * j) ^ swz) << 4;
-            x[j] = *reinterpret_cast<const uint4*>(base + g * (2 * D) + piece);
-            y[j] = *reinterpret_cast<const uint4*>(base + (g + 8) * (2 * D) + piece);
-        }
-        float c[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-        for (int j = 0; j < NJ; ++j) {
-            mma_bf16_16816(c, x[j].x, y[j].x, x[j].y, y[j].y, bq[j][0][0], bq[j][0][1]);
-            mma_bf16_16816(c, x[j].z, y[j].z, x[j].w, y[j].w, bq[j][1][0], bq[j][1][1]);
-        }
-        if (t == 0) {                                         // c0: row g, c2: row g + 8, column 0
-            const int i0 = tile * 16 + g, i1 = i0 + 8;
-            if (i0 < r1) key_out[i0] = score_key(c[0] * scale);
-            if (i1 < r1) key_out[i1] = score_key(c[2] * scale);
+                for (int uu = 0; uu < 8; ++uu) {
+                    const int i = base + (u0 + uu) * SLOTS + myslot;
+                    part[uu] = (u0 + uu < u_end && i < n) ? dot8(my_stage[(u0 + uu) * NT], qf) : 0.f;
+                }
+                int row;
+                const float tot = reduce8_across<LPR>(part, sub, row);
+                const int i = base + (u0 + row) * SLOTS + myslot;
+                if ((LPR == 8 || (sub & 1) == 0) && u0 + row < u_end && i < n) key_out[i] = score_key(tot * scale);
+            }
         }
     }
 }
 
-// Eq. 10: exact current-query scores of n key rows as order-preserving keys into key_out.
-// Row i is kbase[row_of[i]] (INDEXED) or kbase[i] (rows already packed).  The rows go through
-// the staging tiles in chunks of depth * SLOTS rows; each chunk is requested as two groups of
-// copies so that the first half is scored while the second half is still arriving (measured
-// against one group per chunk: 8.3K against 10.3K cycles for 306 rows).
-// s_stage: depth * NT * 16 bytes.  Ends with a barrier.
-template <int D, int NT, bool INDEXED>
-__device__ __forceinline__ void score_candidates(const uint16_t* kbase, const int32_t* row_of, int n,
-                                                 const uint32_t* s_qpk, uint4* s_stage4, int depth, float scale,
-                                                 uint32_t* key_out) {
-    constexpr int LPR = D / 8, RPW = 32 / LPR, SLOTS = (NT / 32) * RPW;
-    unsigned char* s_stage = reinterpret_cast<unsigned char*>(s_stage4);
-    const int cap = depth * SLOTS;                           // a multiple of 16
-    for (int base = 0; base < n; base += cap) {
-        const int m = min(cap, n - base);
-        const int half = min(m, ((m >> 1) + 15) & ~15);
-        rows_request<D, NT, INDEXED>(kbase, row_of + (INDEXED ? base : 0), base, 0, half, s_stage);
-        cp_async_commit();
-        rows_request<D, NT, INDEXED>(kbase, row_of + (INDEXED ? base : 0), base, half, m, s_stage);
-        cp_async_commit();
-        RETOPK_PHASE(0, 15);
-        cp_async_wait_but_one();
-        __syncthreads();
-        RETOPK_PHASE(0, 16);
-        rows_score<D, NT>(s_stage, 0, half, s_qpk, scale, key_out + base);
-        RETOPK_PHASE(0, 17);
-        cp_async_wait_all();
-        __syncthreads();
-        RETOPK_PHASE(0, 18);
-        rows_score<D, NT>(s_stage, half, m, s_qpk, scale, key_out + base);
-        __syncthreads();                                     // keys complete; the tiles may be overwritten
-    }
-}
-
-// The recent window's key rows [first_row, first_row + n) requested into the staging tiles at
-// kernel entry (one commit group), and their scores once the copies are complete and visible
-// (wait + barrier before window_score).
-template <int D, int NT>
-__device__ __forceinline__ void window_request(const uint16_t* kbase, int first_row, int n, uint4* s_stage) {
-    rows_request<D, NT, false>(kbase, nullptr, first_row, 0, n, reinterpret_cast<unsigned char*>(s_stage));
-    cp_async_commit();
-}
-template <int D, int NT>
-__device__ __forceinline__ void window_score(const uint4* s_stage, int n, const uint32_t* s_qpk, float scale,
-                                             uint32_t* key_out) {
-    rows_score<D, NT>(reinterpret_cast<const unsigned char*>(s_stage), 0, n, s_qpk, scale, key_out);
-}
-
-// Shared-memory carve-up of step_kernel (the host mirrors it in step_smem_words):
-//   qpk[D/2] q[D] rho[M+] sel[r+] misc[8] ws[WS_WORDS] hist[SCRATCH_WORDS] sup_idx[K] sup_key[K] w[K] wkey[W+]
-//   | big: idx[cap] key[cap], aliased later by red[NW*D+NT] | bitmap | stage[depth*NT*4]     ("+": rounded up to 4)
-__host__ __device__ inline int step_head_words(int D, int M, int r, int K, int W) {
-    return (D / 2 + D + ((M + 3) & ~3) + ((r + 3) & ~3) + 8 + WS_WORDS + SCRATCH_WORDS + 3 * K + ((W + 3) & ~3) + 3) & ~3;
-}
-
 // ------------------------------------------------------------------------------------
-// step_kernel: the recall stage for every head (Eq. 6, Eq. 7, Eq. 13, insert of the normalised
-// query) and, for a head that reuses, the whole rest of the step in the same CTA: candidate
-// union (Eq. 8-9), candidate scores (Eq. 10), Top-K (Eq. 11), softmax.V (Eq. 12), support
-// insert; candidate list and scores never leave shared memory.  A head on the exact path
-// leaves after the recall stage; scan_kernel and exact_finish_kernel serve it.
+// Eq. 12: out = sum_i softmax(e)_i v_i over the ns selected rows.
+// The value rows are fetched with 16-byte asynchronous copies into a per-thread landing
+// zone (depth rows per row slot in flight at once); the softmax weights are computed while
+// the first wave is in the air.  s_w: ns floats; s_red: (NT/32) * D + NT floats; s_ws:
+// WS_WORDS words; s_stage: depth * NT uint4.
+// With a cluster of cl_size CTAs per head (every CTA holding the same support), CTA cl_rank
+// fetches and weighs its contiguous share of the rows; the partial sums meet in rank 0
+// through distributed shared memory and are added there in rank order.
 // ------------------------------------------------------------------------------------
 template <int D, int NT>
-__global__ void __launch_bounds__(NT, 1024 / NT) step_kernel(const StepArgs a) {
+__device__ void attend(const uint16_t* vbase, int ns, const int32_t* s_sup_idx, const uint32_t* s_sup_key,
+                       float* s_w, float* s_red, int* s_ws, uint4* s_stage, int depth, uint32_t kmax,
+                       bool kmax_known, uint16_t* out_row, int cl_rank = 0, int cl_size = 1) {
+    constexpr int LPR = D / 8;                  // lanes per bf16 row (16 bytes each)
+    constexpr int RPW = 32 / LPR;               // rows per warp load
+    constexpr int SLOTS = (NT / 32) * RPW;      // row slots per block
     constexpr int NW = NT / 32;
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    uint32_t* s_qpk = reinterpret_cast<uint32_t*>(smem_raw);
-    float* s_q = reinterpret_cast<float*>(s_qpk + D / 2);
-    float* s_rho = s_q + D;
-    int* s_sel = reinterpret_cast<int*>(s_rho + ((a.M + 3) & ~3));
-    float* s_misc = reinterpret_cast<float*>(s_sel + ((a.r + 3) & ~3));
-    int* s_ws = reinterpret_cast<int*>(s_misc + 8);
+    constexpr int PARTS = NT / D;               // second-stage partial sums
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int sub = lane % LPR, myslot = warp * RPW + lane / LPR;
+    const char* vsrc = reinterpret_cast<const char*>(vbase) + sub * 16;
+    uint4* my_stage = s_stage + tid;
+    // this CTA's share of the support: [i_lo, i_hi)
+    const int share = (ns + cl_size - 1) / cl_size;
+    const int i_lo = min(ns, cl_rank * share), i_hi = min(ns, i_lo + share);
+
+    auto issue = [&](int base) {
+#pragma unroll 4
+        for (int u = 0; u < depth; ++u) {
+            const int i = base + u * SLOTS + myslot;
+            if (i < i_hi) cp_async16(my_stage + u * NT, vsrc + (size_t)s_sup_idx[i] * (D * 2));
+        }
+        cp_async_commit();
+    };
+    issue(i_lo);
+
+    if (!kmax_known) {
+        kmax = 0;
+        for (int i = tid; i < ns; i += NT) kmax = max(kmax, s_sup_key[i]);
+        kmax = __reduce_max_sync(0xffffffffu, kmax);
+        if (lane == 0) s_ws[warp] = (int)kmax;
+        __syncthreads();
+        kmax = __reduce_max_sync(0xffffffffu, lane < NW ? (uint32_t)s_ws[lane] : 0u);
+        __syncthreads();
+    }
+    const float smax = key_score(kmax);
+    float wsum = 0.f;
+    for (int i = tid; i < ns; i += NT) {
+        const float w = expf(key_score(s_sup_key[i]) - smax);
+        s_w[i] = w;
+        wsum += w;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) wsum += __shfl_xor_sync(0xffffffffu, wsum, o);
+    float* s_wsf = reinterpret_cast<float*>(s_ws);
+    if (lane == 0) s_wsf[warp] = wsum;
+    __syncthreads();
+    float denom = lane < NW ? s_wsf[lane] : 0.f;         // fixed tree: the same sum on every lane and run
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) denom += __shfl_xor_sync(0xffffffffu, denom, o);
+
+    float acc[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+    for (int base = i_lo;;) {
+        cp_async_wait_all();
+        for (int u = 0; u < depth; ++u) {
+            const int i = base + u * SLOTS + myslot;
+            if (i < i_hi) {
+                const float w = s_w[i];
+                float f[8];
+                unpack8(my_stage[u * NT], f);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) acc[e] = fmaf(w, f[e], acc[e]);
+            }
+        }
+        base += SLOTS * depth;
+        if (base >= i_hi) break;
+        issue(base);
+    }
+    // fixed-order reduction: row slots of a warp, then warps in groups, then groups
+#pragma unroll
+    for (int o = LPR; o < 32; o <<= 1)
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc[e] += __shfl_xor_sync(0xffffffffu, acc[e], o);
+    if (lane < LPR) {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) s_red[warp * D + sub * 8 + e] = acc[e];
+    }
+    __syncthreads();
+    {
+        const int j = tid % D, part = tid / D;
+        constexpr int WPP = NW / PARTS;          // warps per part
+        float sum = 0.f;
+#pragma unroll
+        for (int w = 0; w < WPP; ++w) sum += s_red[(part * WPP + w) * D + j];
+        s_red[NW * D + part * D + j] = sum;
+    }
+    __syncthreads();
+    float sum = 0.f;
+    if (tid < D) {
+#pragma unroll
+        for (int p = 0; p < PARTS; ++p) sum += s_red[NW * D + p * D + tid];
+    }
+    if (cl_size > 1) {
+        // s_red[0..D) is free again (its readers passed the barrier above)
+        namespace cg = cooperative_groups;
+        cg::cluster_group cluster = cg::this_cluster();
+        if (tid < D) s_red[tid] = sum;
+        cluster.sync();
+        if (cl_rank == 0 && tid < D) {
+            sum = 0.f;
+            for (int r = 0; r < cl_size; ++r) sum += *cluster.map_shared_rank(s_red + tid, r);
+        }
+        cluster.sync();           // nobody leaves while its shared memory may still be read
+        if (cl_rank != 0) return;
+    }
+    if (tid < D) {
+        const float o = ns > 0 ? sum / denom : 0.f;
+        out_row[tid] = __bfloat16_as_ushort(__float2bfloat16_rn(o));
+    }
+}
+
+// ------------------------------------------------------------------------------------
+// reuse path of finish_kernel: candidate union (Eq. 8-9), candidate scores (Eq. 10), Top-K
+// (Eq. 11), softmax.V (Eq. 12) and the support insert for one head, all in shared memory.
+// (Also built and measured against this form: candidate scores on the tensor cores from
+// 16-row staging tiles, and the window's rows requested ahead of the recalled lists.  Phase
+// clocks showed them level or ahead, the timed pipeline 3 us per step behind: dropped.)
+// ------------------------------------------------------------------------------------
+template <int D, int NT>
+__device__ void reuse_path(const StepArgs& a, unsigned char* smem_raw) {
+    constexpr int NW = NT / 32;
+    // layout (words): qraw[D] sel[r] ws[WS_WORDS] hist[SCRATCH_WORDS] sup_idx[K] sup_key[K] w[K]
+    //                 | big: idx[cap] key[cap], aliased later by red[NW*D+NT] | bitmap | stage[depth*NT*4]
+    float* s_qraw = reinterpret_cast<float*>(smem_raw);
+    int* s_sel = reinterpret_cast<int*>(s_qraw + D);
+    int* s_ws = s_sel + a.r;
     uint32_t* s_hist = reinterpret_cast<uint32_t*>(s_ws + WS_WORDS);
     int32_t* s_sup_idx = reinterpret_cast<int32_t*>(s_hist + SCRATCH_WORDS);
     uint32_t* s_sup_key = reinterpret_cast<uint32_t*>(s_sup_idx + a.K);
     float* s_w = reinterpret_cast<float*>(s_sup_key + a.K);
-    uint32_t* s_wkey = reinterpret_cast<uint32_t*>(s_w + a.K);
-    int32_t* s_idx = reinterpret_cast<int32_t*>(smem_raw) + step_head_words(D, a.M, a.r, a.K, a.W);
+    const int head_words = (D + a.r + WS_WORDS + SCRATCH_WORDS + 3 * a.K + 3) & ~3;
+    int32_t* s_idx = reinterpret_cast<int32_t*>(smem_raw) + head_words;
     uint32_t* s_key = reinterpret_cast<uint32_t*>(s_idx + a.cap);
     float* s_red = reinterpret_cast<float*>(s_idx);
     const int big_words = (max(2 * a.cap, NW * D + NT) + 3) & ~3;
@@ -1517,82 +1237,47 @@ __global__ void __launch_bounds__(NT, 1024 / NT) step_kernel(const StepArgs a) {
     const int bkv = kv_group_of(bh, a);
     const int M = a.M, fill = a.fill, L = a.L, K = a.K;
     const int n_sel = a.r < fill ? a.r : fill;
-    const int w_lo = L - a.W > 0 ? L - a.W : 0, wn = L - w_lo;
-    const uint16_t* kbase = a.k + (size_t)bkv * a.max_seq_len * D;
-    const bool may_reuse = !a.refresh && fill > 0;          // known on the host: else every head is exact
-    const bool prefetch = may_reuse && a.win_prefetch && cl_size == 1;
-
-    // nothing before the wait depends on an earlier kernel
-    if (tid < a.r) s_sel[tid] = -1;
-    if (tid == 0) s_misc[0] = -CUDART_INF_F;
-    if (may_reuse) {
-        const int nwords = (L + 31) >> 5;
-        uint4* bm4 = reinterpret_cast<uint4*>(s_bm);
-        for (int w = tid; w < (nwords + 3) >> 2; w += NT) bm4[w] = make_uint4(0, 0, 0, 0);
-    }
-    pdl_wait();        // the caches were written by the step before; q by whatever ran before this call
-    RETOPK_PHASE(1, 0);
-
-    // ---- recall stage: Eq. 6, Eq. 7, Eq. 13, insert of the normalised query
-    cache_similarities<D, NT>(a, bh, s_q, s_rho, s_qpk,
-                              [&]() { if (prefetch) window_request<D, NT>(kbase, w_lo, wn, s_stage); });
-    __syncthreads();
-    RETOPK_PHASE(1, 1);
-    int sel8[8];
-    const float rho_max = recall_slots<NT>(a, s_rho, s_sel, s_misc, s_ws, sel8);
-    RETOPK_PHASE(1, 3);
-    const int path = decide_path(a, rho_max);
-    if (cl_rank == 0) {
-        // every similarity of this step has been taken: the slot may be overwritten
-        if (tid < D) store_qbar(a, ((size_t)bh * M + a.slot) * D + tid, s_q[tid]);
-        record_decision(a, bh, bkv, s_sel, path, rho_max);
-    }
-    RETOPK_PHASE(1, 2);
-    if (path != PATH_REUSE) {
-        cp_async_wait_all();       // no copy may land in shared memory this CTA has given up
-        return;
-    }
-
-    // ---- reuse path
     RETOPK_PHASE(0, 0);
     // peers write into this CTA's shared memory later on: all of them must be running by then
     if (cl_size > 1) cooperative_groups::this_cluster().sync();
 
-    // Eq. 8-9.  The first recalled lists are requested, then the window rows (long arrived)
-    // are scored while those lists travel.
-    int pre[4];
-    union_load_first<NT>(a, bh, sel8, pre);
-    if (prefetch) {
-        cp_async_wait_all();
-        __syncthreads();           // every thread's pieces have landed
-        window_score<D, NT>(s_stage, wn, s_qpk, a.scale, s_wkey);
+    // recalled slots and the raw query from global memory; clear the bitmap meanwhile
+    if (tid < a.r) s_sel[tid] = a.ws_sel[(size_t)bh * a.r + tid];
+    if (tid >= 32 && tid < 32 + D / 2) {
+        const uint32_t raw = reinterpret_cast<const uint32_t*>(a.q + (size_t)bh * D)[tid - 32];
+        s_qraw[2 * (tid - 32)] = bf16_lo(raw);
+        s_qraw[2 * (tid - 32) + 1] = bf16_hi(raw);
     }
-    RETOPK_PHASE(0, 1);
-    if (!union_mark_short<NT>(a, n_sel, s_bm, pre)) {
-        __syncthreads();           // s_sel complete
-        union_mark<NT>(a, bh, s_sel, n_sel, s_bm, pre, true);
+    {
+        const int nwords = (L + 31) >> 5;
+        uint4* bm4 = reinterpret_cast<uint4*>(s_bm);
+        for (int w = tid; w < (nwords + 3) >> 2; w += NT) bm4[w] = make_uint4(0, 0, 0, 0);
     }
     __syncthreads();
-    RETOPK_PHASE(0, 2);
-    const int n = union_extract<NT>(a, s_bm, s_idx, s_ws);
-    const int n_low = n - wn;
-    if (prefetch)
-        for (int j = tid; j < wn; j += NT) s_key[n_low + j] = s_wkey[j];
+    RETOPK_PHASE(0, 1);
+
+    // Eq. 8-9
+    const int n = candidate_union<NT>(a, bh, s_sel, n_sel, s_bm, s_idx, s_ws);
     __syncthreads();
     RETOPK_PHASE(0, 3);
+
     if (a.dbg_cand && cl_rank == 0)
         for (int i = tid; i < n; i += NT) a.dbg_cand[(size_t)bh * a.cap + i] = s_idx[i];
 
     // Eq. 10.  In a cluster every CTA built the same list; each scores a contiguous share of
     // it and hands the keys to the others through distributed shared memory.
     if (cl_size == 1) {
-        score_candidates<D, NT, true>(kbase, s_idx, prefetch ? n_low : n, s_qpk, s_stage, a.stage_depth, a.scale, s_key);
+        score_candidates<D, NT, true>(a.k + (size_t)bkv * a.max_seq_len * D, s_idx, n, s_qraw, s_stage,
+                                      a.stage_depth, a.scale, s_key);
+        __syncthreads();
     } else {
         namespace cg = cooperative_groups;
         cg::cluster_group cluster = cg::this_cluster();
         const int share = (n + cl_size - 1) / cl_size;
         const int lo = min(n, cl_rank * share), hi = min(n, lo + share);
-        score_candidates<D, NT, true>(kbase, s_idx + lo, hi - lo, s_qpk, s_stage, a.stage_depth, a.scale, s_key + lo);
+        score_candidates<D, NT, true>(a.k + (size_t)bkv * a.max_seq_len * D, s_idx + lo, hi - lo, s_qraw, s_stage,
+                                      a.stage_depth, a.scale, s_key + lo);
+        __syncthreads();
         for (int r = 1; r < cl_size; ++r) {
             uint32_t* peer = cluster.map_shared_rank(s_key, (cl_rank + r) & (cl_size - 1));
             for (int i = lo + tid; i < hi; i += NT) peer[i] = s_key[i];
@@ -1603,8 +1288,8 @@ __global__ void __launch_bounds__(NT, 1024 / NT) step_kernel(const StepArgs a) {
 
     // Eq. 11: Top-K of the candidates; insert the support
     uint32_t kmax;
-    bool kmax_known;
-    const int ns = select_listed<NT>(s_key, s_idx, n, K, s_sup_idx, s_sup_key, s_hist, s_ws, kmax, kmax_known);
+    const bool kmax_known = true;
+    const int ns = select_listed<NT>(s_key, s_idx, n, K, s_sup_idx, s_sup_key, s_hist, s_ws, &kmax);
     RETOPK_PHASE(0, 5);
     if (cl_rank == 0) {
         int32_t* sup_out = a.sup_cache + ((size_t)bh * M + a.slot) * K;
@@ -1776,13 +1461,13 @@ __device__ __forceinline__ void scan_body(const StepArgs& a) {
     }
 }
 
-// scan_kernel: the launch around scan_body, a dependent launch behind step_kernel (or, for
-// Exact Top-K, behind whatever ran before).  (Letting it come up beside step_kernel and wait for
-// the decisions only was tried: its CTAs then share SMs whose shared memory is carved up for
-// the per-head CTAs, and with that little L1 the scan streams 1.6x slower.)
+// scan_kernel: the launch around scan_body, a dependent launch behind recall_kernel (or, for
+// Exact Top-K, behind whatever ran before).  (Letting it come up beside a per-head kernel and
+// wait for the decisions only was tried: its CTAs then share SMs whose shared memory is carved
+// up for the per-head CTAs, and with that little L1 the scan streams 1.6x slower.)
 template <int D, int NTILE>
 __global__ void __launch_bounds__(SCAN_THREADS) scan_kernel(const StepArgs a) {
-    pdl_wait();        // group flags and paths come from step_kernel
+    pdl_wait();        // group flags and paths come from recall_kernel
     scan_body<D, NTILE>(a);
 }
 
@@ -1797,9 +1482,10 @@ __global__ void __launch_bounds__(SCAN_THREADS) scan_kernel(const StepArgs a) {
 // lower-index tie rule is taken from that list.
 // ------------------------------------------------------------------------------------
 template <int D, int NT>
-__device__ void exact_path(const StepArgs& a, int bh, unsigned char* smem_raw) {
+__device__ void exact_path(const StepArgs& a, unsigned char* smem_raw) {
     // In a cluster every CTA of a head selects the same support on its own (the lists are short
     // and come from L2); only the value rows are shared out, and rank 0 writes the results.
+    const int bh = cluster_slot(a);
     const int cl_rank = cluster_rank(a), cl_size = 1 << a.cl_shift;
     // layout (words): sup_idx[K] sup_key[K] w[K] cnt[SCRATCH_WORDS] ws[WS_WORDS] misc[8]
     //                 | lists: key[NS] idx[NS] tile[tile_cap]; dead once the support is emitted and
@@ -1817,7 +1503,7 @@ __device__ void exact_path(const StepArgs& a, int bh, unsigned char* smem_raw) {
     float* s_red = reinterpret_cast<float*>(s_key);
     uint4* s_stage = reinterpret_cast<uint4*>(s_key + ((NW * D + NT + 3) & ~3));
 
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int tid = threadIdx.x;
     const int bkv = kv_group_of(bh, a);
     const int K = a.K, L = a.L, NS = a.NS;
     const float* sc = a.ws_scores + (size_t)bh * a.score_stride;
@@ -1835,131 +1521,72 @@ __device__ void exact_path(const StepArgs& a, int bh, unsigned char* smem_raw) {
     } else {
         const int ntile = (L + TILE_ROWS - 1) / TILE_ROWS;
         const int tcap = a.tile_cap;
-        // 1. lower bound v for the K-th score: the K-th largest of the tile maxima (of groups of
-        //    2^sh tiles when there are more tiles than list entries).  The keys of the maxima stay
-        //    in shared memory for step 2.
+        // 1. lower bound v for the K-th score from the tile maxima (grouped so the list is short)
         uint32_t thr_key = 0;
-        int sh = 0;
+        int sh = 0;                                  // groups of g2 = 2^sh tiles
+        while (((ntile + (1 << sh) - 1) >> sh) > 1024 && (ntile >> (sh + 1)) >= 2 * K) ++sh;
         while (((ntile + (1 << sh) - 1) >> sh) > NS) ++sh;
         const int g2 = 1 << sh;
         const int n2 = (ntile + g2 - 1) >> sh;
-        if (sh == 0) {
-            // four consecutive maxima per thread and trip, all trips requested before any is used
-            const int nq = (ntile + 3) >> 2;
-            for (int p0 = tid; p0 < nq; p0 += 4 * NT) {
-                float4 x[4];
-#pragma unroll
-                for (int u = 0; u < 4; ++u)
-                    x[u] = p0 + u * NT < nq ? *reinterpret_cast<const float4*>(tm + 4 * (p0 + u * NT))
-                                            : make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-                for (int u = 0; u < 4; ++u)
-                    if (p0 + u * NT < nq) {
-                        const int t0 = 4 * (p0 + u * NT);
-                        // (maxima past the last tile are padding of the row: keyed as the smallest key)
-                        const uint4 kq = make_uint4(score_key(x[u].x), t0 + 1 < ntile ? score_key(x[u].y) : 0u,
-                                                    t0 + 2 < ntile ? score_key(x[u].z) : 0u, t0 + 3 < ntile ? score_key(x[u].w) : 0u);
-                        *reinterpret_cast<uint4*>(s_key + t0) = kq;
-                    }
-            }
-        } else {
-            // groups of g2 tiles (very long histories only): 16-byte loads, g2 / 4 of them per group
-            // (or 4 / g2 groups per load)
-            const int nq = (ntile + 3) >> 2;
-            if (g2 < 4) {                                   // g2 == 2: two groups per load
-                for (int p = tid; p < nq; p += NT) {
-                    const float4 x = *reinterpret_cast<const float4*>(tm + 4 * p);
-                    const int t0 = 4 * p;
-                    s_key[2 * p] = score_key(t0 + 1 < ntile ? fmaxf(x.x, x.y) : x.x);
-                    if (t0 + 2 < ntile) s_key[2 * p + 1] = score_key(t0 + 3 < ntile ? fmaxf(x.z, x.w) : x.z);
-                }
-            } else {
-                const int lpg = g2 >> 2;                    // loads per group
-                for (int i2 = tid; i2 < n2; i2 += NT) {
-                    float m = -CUDART_INF_F;
-                    for (int u = 0; u < lpg; ++u) {
-                        const int p = i2 * lpg + u;
-                        if (p >= nq) break;
-                        const float4 x = *reinterpret_cast<const float4*>(tm + 4 * p);
-                        const int t0 = 4 * p;
-                        m = fmaxf(m, x.x);
-                        if (t0 + 1 < ntile) m = fmaxf(m, x.y);
-                        if (t0 + 2 < ntile) m = fmaxf(m, x.z);
-                        if (t0 + 3 < ntile) m = fmaxf(m, x.w);
-                    }
-                    s_key[i2] = score_key(m);
-                }
-            }
-        }
-        __syncthreads();
         if (n2 >= K) {
-            uint32_t kmax_unused;
-            if (!(n2 <= 9 * NT && select_small<NT, 9, false>(s_key, nullptr, n2, K, nullptr, nullptr, reinterpret_cast<int*>(s_hist),
-                                                             &kmax_unused, &thr_key))) {
-                __syncthreads();
-                thr_key = bin_threshold<NT>(s_key, n2, K, false, reinterpret_cast<int*>(s_hist)).v;
-            }
-        }
-        RETOPK_PHASE(2, 1);
-        // 2. the tiles whose maximum reaches v, in ascending order.  Ungrouped: straight from the
-        //    keys in shared memory, one 16-byte piece (four tiles) per thread and round.
-        int nhit = 0;
-        if (sh == 0) {
-            const int nq = (ntile + 3) >> 2;
-            for (int base = 0; base < nq; base += NT) {
-                const int p = base + tid;
-                unsigned hits = 0;
-                if (p < nq) {
-                    const uint4 kq = *reinterpret_cast<const uint4*>(s_key + 4 * p);
-                    const uint32_t kv[4] = {kq.x, kq.y, kq.z, kq.w};
+            for (int i2 = tid; i2 < n2; i2 += NT) {
+                const int t0 = i2 << sh;
+                float m;
+                if (g2 >= 4) {
+                    // g2 is a power of two: whole float4 chunks, all requested before any is used
+                    m = -CUDART_INF_F;
+                    for (int c0 = 0; c0 < g2; c0 += 16) {
+                        float4 x[4];
 #pragma unroll
-                    for (int e = 0; e < 4; ++e)
-                        if (4 * p + e < ntile && kv[e] >= thr_key) hits |= 1u << e;
-                }
-                const int cnt = __popc(hits);
-                int inc = cnt;
-                if (base + warp * 32 < nq) {               // (warp-uniform) this warp looks at tiles in this round
+                        for (int u = 0; u < 4; ++u)
+                            x[u] = (c0 + 4 * u < g2 && t0 + c0 + 4 * u < ntile)
+                                ? *reinterpret_cast<const float4*>(tm + t0 + c0 + 4 * u)
+                                : make_float4(-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F);
 #pragma unroll
-                    for (int o = 1; o < 32; o <<= 1) { const int t = __shfl_up_sync(0xffffffffu, inc, o); if (lane >= o) inc += t; }
+                        for (int u = 0; u < 4; ++u) {
+                            const int tt = t0 + c0 + 4 * u;
+                            m = fmaxf(m, x[u].x);
+                            if (tt + 1 < ntile) m = fmaxf(m, x[u].y);
+                            if (tt + 2 < ntile) m = fmaxf(m, x[u].z);
+                            if (tt + 3 < ntile) m = fmaxf(m, x[u].w);
+                        }
+                    }
+                } else {
+                    m = tm[t0];
+                    if (g2 == 2 && t0 + 1 < ntile) m = fmaxf(m, tm[t0 + 1]);
                 }
-                if (lane == 31) s_ws[warp] = inc;
-                __syncthreads();
-                int total;
-                int pos = nhit + warp_base<NT>(s_ws, total) + inc - cnt;
-                while (hits) {
-                    const int e = __ffs(hits) - 1;
-                    if (pos < tcap) s_tile[pos] = 4 * p + e;
-                    ++pos;
-                    hits &= hits - 1;
-                }
-                nhit += total;
-                __syncthreads();                            // s_ws is reused by the next round
-            }
-        } else {
-            for (int base = 0; base < ntile; base += NT * 8) {
-                const int t0 = base + tid * 8;
-                float4 m4[2];
-#pragma unroll
-                for (int u = 0; u < 2; ++u)
-                    m4[u] = t0 + 4 * u < ntile ? *reinterpret_cast<const float4*>(tm + t0 + 4 * u)
-                                               : make_float4(0.f, 0.f, 0.f, 0.f);
-                const float mv[8] = {m4[0].x, m4[0].y, m4[0].z, m4[0].w, m4[1].x, m4[1].y, m4[1].z, m4[1].w};
-                unsigned hits = 0;
-#pragma unroll
-                for (int e = 0; e < 8; ++e)
-                    if (t0 + e < ntile && score_key(mv[e]) >= thr_key) hits |= 1u << e;
-                int total;
-                int pos = nhit + block_excl_scan<NT>(__popc(hits), s_ws, total);
-                while (hits) {
-                    const int e = __ffs(hits) - 1;
-                    if (pos < tcap) s_tile[pos] = t0 + e;
-                    ++pos;
-                    hits &= hits - 1;
-                }
-                nhit += total;
+                s_key[i2] = score_key(m);
             }
             __syncthreads();
+            thr_key = count_threshold<NT>(s_key, n2, K, 16, reinterpret_cast<int*>(s_hist)).v;
         }
+        RETOPK_PHASE(2, 1);
+        // 2. the tiles whose maximum reaches v, in ascending order: eight consecutive tile
+        //    maxima per thread and one prefix sum per 8 * NT tiles
+        int nhit = 0;
+        for (int base = 0; base < ntile; base += NT * 8) {
+            const int t0 = base + tid * 8;
+            float4 m4[2];
+#pragma unroll
+            for (int u = 0; u < 2; ++u)
+                m4[u] = t0 + 4 * u < ntile ? *reinterpret_cast<const float4*>(tm + t0 + 4 * u)
+                                           : make_float4(0.f, 0.f, 0.f, 0.f);
+            const float mv[8] = {m4[0].x, m4[0].y, m4[0].z, m4[0].w, m4[1].x, m4[1].y, m4[1].z, m4[1].w};
+            unsigned hits = 0;
+#pragma unroll
+            for (int e = 0; e < 8; ++e)
+                if (t0 + e < ntile && score_key(mv[e]) >= thr_key) hits |= 1u << e;
+            int total;
+            int pos = nhit + block_excl_scan<NT>(__popc(hits), s_ws, total);
+            while (hits) {
+                const int e = __ffs(hits) - 1;
+                if (pos < tcap) s_tile[pos] = t0 + e;
+                ++pos;
+                hits &= hits - 1;
+            }
+            nhit += total;
+        }
+        __syncthreads();
         RETOPK_PHASE(2, 2);
         if (nhit > tcap) slow = true;
         else {
@@ -1981,16 +1608,8 @@ __device__ void exact_path(const StepArgs& a, int bh, unsigned char* smem_raw) {
                             if (row0 + 4 * u + e < L && score_key(v4[e]) >= thr_key) fl |= 1u << (4 * u + e);
                     }
                 }
-                const int cnt = __popc(fl);
-                int inc = cnt;
-                if (base + warp * 32 < nhit) {             // (warp-uniform) this warp visits tiles in this round
-#pragma unroll
-                    for (int o = 1; o < 32; o <<= 1) { const int t = __shfl_up_sync(0xffffffffu, inc, o); if (lane >= o) inc += t; }
-                }
-                if (lane == 31) s_ws[warp] = inc;
-                __syncthreads();
                 int total;
-                int pos = n + warp_base<NT>(s_ws, total) + inc - cnt;
+                int pos = n + block_excl_scan<NT>(__popc(fl), s_ws, total);
                 while (fl) {
                     const int e = __ffs(fl) - 1;
                     if (pos < NS) { s_key[pos] = score_key(sc[row0 + e]); s_idx[pos] = row0 + e; }
@@ -1998,8 +1617,8 @@ __device__ void exact_path(const StepArgs& a, int bh, unsigned char* smem_raw) {
                     fl &= fl - 1;
                 }
                 n += total;
-                __syncthreads();                            // s_ws is reused by the next round
             }
+            __syncthreads();
             if (n > NS) slow = true;
         }
     }
@@ -2017,7 +1636,7 @@ __device__ void exact_path(const StepArgs& a, int bh, unsigned char* smem_raw) {
     }
     uint32_t kmax = 0;
     bool kmax_known = false;
-    if (ns < 0) ns = select_listed<NT>(s_key, s_idx, n, K, s_sup_idx, s_sup_key, s_hist, s_ws, kmax, kmax_known);
+    if (ns < 0) { ns = select_listed<NT>(s_key, s_idx, n, K, s_sup_idx, s_sup_key, s_hist, s_ws, &kmax); kmax_known = true; }
     RETOPK_PHASE(2, 4);
 
     // record the support (cache insert / caller's index output)
@@ -2033,24 +1652,21 @@ __device__ void exact_path(const StepArgs& a, int bh, unsigned char* smem_raw) {
 }
 
 // ------------------------------------------------------------------------------------
-// exact_finish_kernel: launched behind the scan with one CTA (or cluster) per head; cluster
-// number i serves the i-th head of the step's list of exact heads and the rest leave at once
-// (the list's length is only known on the device).  For Exact Top-K attention every head is
-// served.  Which CTA serves a head does not matter to its result.
+// finish_kernel: one CTA (or cluster) per (sequence, query head), launched behind the scan.
+// A head on the reuse path never needed the scan's results, a head on the exact path selects
+// from them; both end with softmax.V and the support insert.  Heads of one step run side by
+// side, so a step with a few exact heads costs the longer of the two paths, not their sum.
 // ------------------------------------------------------------------------------------
 template <int D, int NT>
-__global__ void __launch_bounds__(NT, 1024 / NT) exact_finish_kernel(const StepArgs a) {
+__global__ void __launch_bounds__(NT, 1024 / NT) finish_kernel(const StepArgs a) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    pdl_wait();        // scores and tile maxima come from the scan, the list from step_kernel
-    int n_listed = a.B * a.Hq;
-    if (a.mode == MODE_RETOPK) n_listed = (int)a.ws_xcount[a.step_id & 1];
-    if (blockIdx.x == 0 && threadIdx.x == 0) {
-        *a.scan_counter = 0u;                                   // the scan before this kernel is complete
-        if (a.mode == MODE_RETOPK) a.ws_xcount[(a.step_id + 1) & 1] = 0u;   // the next step's list starts empty
+    pdl_wait();        // scores and tile maxima come from the scan, recalled slots and paths from recall_kernel
+    if (blockIdx.x == 0 && threadIdx.x == 0) *a.scan_counter = 0u;      // the scan before this kernel is complete
+    if (a.mode == MODE_RETOPK && a.ws_path[cluster_slot(a)] == PATH_REUSE) {
+        if (!a.skip_reuse) reuse_path<D, NT>(a, smem_raw);
+    } else {
+        exact_path<D, NT>(a, smem_raw);
     }
-    const int slot = cluster_slot(a);
-    if (slot >= n_listed) return;
-    exact_path<D, NT>(a, a.mode == MODE_RETOPK ? a.ws_xlist[slot] : slot, smem_raw);
 }
 
 // Host-buffer entry point, when the caller's buffers are pinned and mapped: one launch reads
@@ -2089,15 +1705,14 @@ __global__ void narrow_kernel(const float* src, uint16_t* dst, size_t n) {
 // Clear the caches (supports to -1, queries and counters to 0).
 __global__ void reset_kernel(float* qbar, size_t n_q, int32_t* sup, size_t n_sup, unsigned long long* counters,
                              size_t n_cnt, int32_t* gflag, size_t n_flag, unsigned int* status,
-                             unsigned long long* slow, unsigned long long* groups, unsigned int* scan_counter,
-                             unsigned int* xcount) {
+                             unsigned long long* slow, unsigned long long* groups, unsigned int* scan_counter) {
     const size_t stride = (size_t)gridDim.x * blockDim.x;
     const size_t t0 = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     for (size_t i = t0; i < n_q; i += stride) qbar[i] = 0.f;
     for (size_t i = t0; i < n_sup; i += stride) sup[i] = -1;
     for (size_t i = t0; i < n_cnt; i += stride) counters[i] = 0;
     for (size_t i = t0; i < n_flag; i += stride) gflag[i] = -1;
-    if (t0 == 0) { *status = 0u; *slow = 0ull; *groups = 0ull; *scan_counter = 0u; xcount[0] = 0u; xcount[1] = 0u; }
+    if (t0 == 0) { *status = 0u; *slow = 0ull; *groups = 0ull; *scan_counter = 0u; }
 }
 
 }  // namespace retopk

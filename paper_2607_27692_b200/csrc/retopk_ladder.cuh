@@ -9,12 +9,12 @@
 //   level 3  selection, sparse output and cache update fused into one kernel
 //   level 4  as level 3, with the intermediate buffers kept by the context instead of being
 //            allocated from a stream-ordered pool in every step (a host-side difference)
-//   level 5  candidate construction through output in one kernel: step_kernel, the
-//            production path
+//   level 5  candidate construction through output in one kernel: recall_kernel +
+//            finish_kernel, the production path
 //
 // Every level runs the same device functions on the same lanes as the production path, so
 // supports and outputs are bit-identical across levels.  Heads on the exact path are served
-// by scan_kernel + exact_finish_kernel at every level.  One block of LADDER_THREADS per head.
+// by scan_kernel + finish_kernel at every level.  One block of LADDER_THREADS per head.
 #pragma once
 
 #include "retopk_kernels.cuh"
@@ -123,21 +123,24 @@ template <int D, bool INDEXED>
 __global__ void __launch_bounds__(LADDER_THREADS, 1) ladder_score_kernel(const StepArgs a) {
     constexpr int NT = LADDER_THREADS;
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    // layout (words): qpk[D] (the packed query in its first half) idx[cap] | stage[depth*NT*4]
-    uint32_t* s_qpk = reinterpret_cast<uint32_t*>(smem_raw);
-    int32_t* s_idx = reinterpret_cast<int32_t*>(s_qpk + D);
+    // layout (words): qraw[D] idx[cap] | stage[depth*NT*4]
+    float* s_qraw = reinterpret_cast<float*>(smem_raw);
+    int32_t* s_idx = reinterpret_cast<int32_t*>(s_qraw + D);
     uint4* s_stage = reinterpret_cast<uint4*>(s_idx + ((a.cap + 3) & ~3));
     const int tid = threadIdx.x, bh = blockIdx.x;
     if (a.ws_path[bh] != PATH_REUSE) return;
     const int n = a.ws_ncand[bh];
-    if (tid < D / 2) s_qpk[tid] = reinterpret_cast<const uint32_t*>(a.q + (size_t)bh * D)[tid];
+    if (tid < D / 2) {
+        const uint32_t raw = reinterpret_cast<const uint32_t*>(a.q + (size_t)bh * D)[tid];
+        s_qraw[2 * tid] = bf16_lo(raw);
+        s_qraw[2 * tid + 1] = bf16_hi(raw);
+    }
     if (INDEXED)
         for (int i = tid; i < n; i += NT) s_idx[i] = a.lw_cand[(size_t)bh * a.cap + i];
     __syncthreads();
     const uint16_t* rows = INDEXED ? a.k + (size_t)kv_group_of(bh, a) * a.max_seq_len * D
                                    : a.lw_rows + (size_t)bh * a.cap * D;
-    // (keys to shared memory first: the scoring warps write them one tile at a time)
-    score_candidates<D, NT, INDEXED>(rows, s_idx, n, s_qpk, s_stage, a.stage_depth, a.scale,
+    score_candidates<D, NT, INDEXED>(rows, s_idx, n, s_qraw, s_stage, a.stage_depth, a.scale,
                                      a.lw_key + (size_t)bh * a.cap);
 }
 
@@ -161,8 +164,8 @@ __global__ void __launch_bounds__(LADDER_THREADS, 1) ladder_select_kernel(const 
     }
     __syncthreads();
     uint32_t kmax;
-    bool kmax_known;
-    const int ns = select_listed<NT>(s_key, s_idx, n, a.K, s_sup_idx, s_sup_key, s_hist, s_ws, kmax, kmax_known);
+    const bool kmax_known = true;
+    const int ns = select_listed<NT>(s_key, s_idx, n, a.K, s_sup_idx, s_sup_key, s_hist, s_ws, &kmax);
     for (int i = tid; i < ns; i += NT) {
         a.lw_sup_idx[(size_t)bh * a.K + i] = s_sup_idx[i];
         a.lw_sup_key[(size_t)bh * a.K + i] = s_sup_key[i];
@@ -225,7 +228,7 @@ template <int D>
 __global__ void __launch_bounds__(LADDER_THREADS, 1) ladder_discover_kernel(const StepArgs a) {
     constexpr int NT = LADDER_THREADS;
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    // layout (words): q[D] rho[M + 3] misc[4] | union carve-up (its sel[] and ws[] are the recall's)
+    // layout (words): q[D] rho[M + 3] misc[4] | union carve-up (its sel[] is the recall's)
     float* s_q = reinterpret_cast<float*>(smem_raw);
     float* s_rho = s_q + D;
     float* s_misc = s_rho + ((a.M + 3) & ~3);
@@ -272,8 +275,8 @@ __global__ void __launch_bounds__(LADDER_THREADS, 1) ladder_select_attend_insert
     }
     __syncthreads();
     uint32_t kmax;
-    bool kmax_known;
-    const int ns = select_listed<NT>(s_key, s_idx, n, a.K, s_sup_idx, s_sup_key, s_hist, s_ws, kmax, kmax_known);
+    const bool kmax_known = true;
+    const int ns = select_listed<NT>(s_key, s_idx, n, a.K, s_sup_idx, s_sup_key, s_hist, s_ws, &kmax);
     int32_t* sup_out = a.sup_cache + ((size_t)bh * a.M + a.slot) * a.K;
     for (int i = tid; i < a.K; i += NT) sup_out[i] = i < ns ? s_sup_idx[i] : -1;
     attend<D, NT>(a.v + (size_t)kv_group_of(bh, a) * a.max_seq_len * D, ns, s_sup_idx, s_sup_key, s_w, s_red, s_ws,

@@ -160,15 +160,15 @@ class ReTopK:
         _check(self.lib.retopk_set_qbar_format(self.h, fmt), "retopk_set_qbar_format")
 
     def set_cluster_size(self, ctas_per_head: int):
-        """CTAs (one SM each) per head in the per-head kernels: 1, 2, 4 or 8."""
+        """CTAs (one SM each) per head in the finish kernel: 1, 2, 4 or 8."""
         _check(self.lib.retopk_set_cluster_size(self.h, ctas_per_head), "retopk_set_cluster_size")
 
     def set_finish_threads(self, threads: int):
-        """Block shape of the per-head kernels: 1024 (one CTA per SM) or 512 (two per SM)."""
+        """Block shape of the finish kernel: 1024 (one CTA per SM) or 512 (two per SM)."""
         _check(self.lib.retopk_set_finish_threads(self.h, threads), "retopk_set_finish_threads")
 
     def set_block_shape(self, threads: int, ctas_per_sm: int):
-        """Block shape of the per-head kernels: (1024, 1), (512, 2), (512, 1) or (256, 1)."""
+        """Block shape of the finish kernel: (1024, 1), (512, 2) or (512, 1)."""
         _check(self.lib.retopk_set_block_shape(self.h, threads, ctas_per_sm), "retopk_set_block_shape")
 
     def set_fusion_level(self, level: int, dependent_launches: bool = False):
@@ -273,7 +273,7 @@ class ReTopK:
         ms, n = (C.c_double * 3)(), (_i64 * 3)()
         _check(self.lib.retopk_profile_end(self.h, ms, n), "retopk_profile_end")
         return {name: dict(ms=float(ms[i]), launches=int(n[i]))
-                for i, name in enumerate(("step", "scan", "finish"))}
+                for i, name in enumerate(("recall", "scan", "finish"))}
 
     def last_launch_count(self) -> int:
         return int(self.lib.retopk_last_launch_count(self.h))

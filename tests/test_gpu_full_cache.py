@@ -136,7 +136,7 @@ def test_headline_shape_from_a_full_cache(rt, P, oracle_mod):
     assert sg["status"] == 0 and sg["slow_select"] == 0
 
 
-@pytest.mark.parametrize("threads,per_sm", [(512, 1), (256, 1), (512, 2)])
+@pytest.mark.parametrize("threads,per_sm", [(512, 1), (512, 2)])
 @pytest.mark.parametrize("d", [64, 128])
 def test_block_shapes_against_the_oracle(rt, P, oracle_mod, threads, per_sm, d):
     """Every block shape of the per-head kernels, full cache, both paths (tau in the middle of the similarities)."""
