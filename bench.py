@@ -623,9 +623,13 @@ PHASES = {
                        (4, 5, "Top-K (Eq. 11)"), (5, 6, "softmax.V, inserts (Eq. 12)"),
                        (8, 9, "  Top-K: span of the keys"), (9, 10, "  Top-K: histogram"), (10, 11, "  Top-K: boundary bin"),
                        (11, 12, "  Top-K: its members"), (12, 13, "  Top-K: their ranks"), (13, 14, "  Top-K: ballots"),
-                       (14, 5, "  Top-K: placed")]),
+                       (14, 5, "  Top-K: placed"),
+                       (16, 17, "  softmax.V: value rows requested"), (17, 18, "  softmax.V: weights"),
+                       (18, 19, "  softmax.V: rows landed"), (19, 20, "  softmax.V: weighted sum"), (20, 6, "  softmax.V: reduction, output")]),
     "finish kernel, exact path": (2, [(0, 1, "bound from the tile maxima"), (1, 2, "hit-tile list"), (2, 3, "read-back of hit tiles"),
-                         (3, 4, "Top-K (Eq. 1)"), (4, 5, "softmax.V, insert (Eq. 12)")]),
+                         (3, 4, "Top-K (Eq. 1)"), (4, 5, "softmax.V, insert (Eq. 12)"),
+                       (16, 17, "  softmax.V: value rows requested"), (17, 18, "  softmax.V: weights"),
+                       (18, 19, "  softmax.V: rows landed"), (19, 20, "  softmax.V: weighted sum"), (20, 5, "  softmax.V: reduction, output")]),
 }
 
 

@@ -224,6 +224,14 @@ int launch_finish(const retopk_ctx* c, const StepArgs& a, cudaStream_t s) {
     const unsigned nt = (unsigned)c->finish_threads;
     const int dep = c->dependent_launches, cl = c->cluster;
     const size_t smem = a.mode == MODE_EXACT ? c->smem_exact : c->smem_finish;
+    if (a.mode == MODE_EXACT) {      // the variant without the reuse path's code
+        if (c->d == 128) {
+            if (nt == 1024) return launch_dependent(finish_kernel<128, 1024, false>, grid, nt, smem, s, a, dep, cl);
+            return launch_dependent(finish_kernel<128, 512, false>, grid, nt, smem, s, a, dep, cl);
+        }
+        if (nt == 1024) return launch_dependent(finish_kernel<64, 1024, false>, grid, nt, smem, s, a, dep, cl);
+        return launch_dependent(finish_kernel<64, 512, false>, grid, nt, smem, s, a, dep, cl);
+    }
     if (c->d == 128) {
         if (nt == 1024) return launch_dependent(finish_kernel<128, 1024>, grid, nt, smem, s, a, dep, cl);
         return launch_dependent(finish_kernel<128, 512>, grid, nt, smem, s, a, dep, cl);
@@ -555,10 +563,12 @@ int retopk_create_batched(retopk_ctx** out, int B, int H_q, int H_kv, int d, int
     const int ntile = (c->G + 7) / 8;
     if (d == 128) {
         opt(finish_kernel<128, 1024>); opt(finish_kernel<128, 512>);
+        opt(finish_kernel<128, 1024, false>); opt(finish_kernel<128, 512, false>);
         if (ntile == 1) cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, scan_kernel<128, 1>, SCAN_THREADS, 0);
         else cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, scan_kernel<128, 2>, SCAN_THREADS, 0);
     } else {
         opt(finish_kernel<64, 1024>); opt(finish_kernel<64, 512>);
+        opt(finish_kernel<64, 1024, false>); opt(finish_kernel<64, 512, false>);
         if (ntile == 1) cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, scan_kernel<64, 1>, SCAN_THREADS, 0);
         else cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, scan_kernel<64, 2>, SCAN_THREADS, 0);
     }
@@ -1042,8 +1052,8 @@ int static_setup(int dev, StaticSetup** out) {
         if (cudaDeviceGetAttribute(&st->num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
             cudaDeviceGetAttribute(&st->max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess)
             return RETOPK_ECUDA;
-        if (cudaFuncSetAttribute(finish_kernel<128, 1024>, cudaFuncAttributeMaxDynamicSharedMemorySize, st->max_smem) != cudaSuccess ||
-            cudaFuncSetAttribute(finish_kernel<64, 1024>, cudaFuncAttributeMaxDynamicSharedMemorySize, st->max_smem) != cudaSuccess)
+        if (cudaFuncSetAttribute(finish_kernel<128, 1024, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, st->max_smem) != cudaSuccess ||
+            cudaFuncSetAttribute(finish_kernel<64, 1024, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, st->max_smem) != cudaSuccess)
             return RETOPK_ECUDA;
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&st->occ[0][0], scan_kernel<64, 1>, SCAN_THREADS, 0);
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&st->occ[0][1], scan_kernel<64, 2>, SCAN_THREADS, 0);
@@ -1129,8 +1139,8 @@ int exact_topk_decode_static(int B, int H_q, int H_kv, int d, int K, int64_t max
     if (cudaGetLastError() != cudaSuccess) return RETOPK_ECUDA;
     const int cluster = auto_cluster(nh, st->num_sms);
     a.cl_shift = __builtin_ctz((unsigned)cluster);
-    if (d == 128) return launch_dependent(finish_kernel<128, 1024>, (unsigned)(nh * cluster), FINISH_THREADS, smem, s, a, 0, cluster);
-    return launch_dependent(finish_kernel<64, 1024>, (unsigned)(nh * cluster), FINISH_THREADS, smem, s, a, 0, cluster);
+    if (d == 128) return launch_dependent(finish_kernel<128, 1024, false>, (unsigned)(nh * cluster), FINISH_THREADS, smem, s, a, 0, cluster);
+    return launch_dependent(finish_kernel<64, 1024, false>, (unsigned)(nh * cluster), FINISH_THREADS, smem, s, a, 0, cluster);
 }
 
 #ifdef RETOPK_PHASE_CLOCKS

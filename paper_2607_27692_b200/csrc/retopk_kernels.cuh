@@ -113,7 +113,7 @@ struct StepArgs {
     uint16_t* lw_rows;       // [B*Hq][cap][d] packed candidate key rows (level 1 only)
     int32_t* lw_sup_idx;     // [B*Hq][K] selected indices
     uint32_t* lw_sup_key;    // [B*Hq][K] their score keys
-    int32_t* lw_meta;        // [B*Hq][4] ns, kmax, kmax_known, -
+    int32_t* lw_meta;        // [B*Hq][4] ns, kmax, -, -
 };
 
 // ------------------------------------------------------------------------------------
@@ -262,73 +262,20 @@ __device__ __noinline__ int2 block_excl_scan2(int2 v, int* s_ws, int2& total) {
 // ------------------------------------------------------------------------------------
 // selection primitives
 // ------------------------------------------------------------------------------------
-struct SmemSrc {
+// Where the general (rarely taken) selection code reads its keys: a list in shared memory
+// (key, idx) or, with key == nullptr, the score array of a head in global memory (entry i is
+// row i).  One type, so there is one copy of that code: the size of a kernel's code costs time
+// on every launch that follows a long scan, whether the code runs or not.
+struct KeySrc {
     const uint32_t* key;
     const int32_t* idx;
-    __device__ __forceinline__ uint32_t k(int i) const { return key[i]; }
-    __device__ __forceinline__ int x(int i) const { return idx[i]; }
-};
-struct ScoreSrc {
     const float* sc;
-    __device__ __forceinline__ uint32_t k(int i) const { return score_key(sc[i]); }
-    __device__ __forceinline__ int x(int i) const { return i; }
+    __device__ __forceinline__ uint32_t k(int i) const { return key ? key[i] : score_key(sc[i]); }
+    __device__ __forceinline__ int x(int i) const { return key ? idx[i] : i; }
 };
-
-// K-th largest key of src[0..n) (n > K >= 1) by four 8-bit radix passes.
-// Returns the key value v and `need_eq` = how many elements equal to v belong to the top K.
-// s_hist: 256 words, s_misc: 2 ints.
-template <int NT, class Src>
-__device__ __noinline__ void radix_select(const Src& src, int n, int K, uint32_t* s_hist, int* s_misc,
-                             uint32_t& vstar, int& need_eq) {
-    const int tid = threadIdx.x, lane = tid & 31;
-    uint32_t prefix = 0, mask = 0;
-    int kk = K;
-    for (int shift = 24; shift >= 0; shift -= 8) {
-        for (int i = tid; i < 256; i += NT) s_hist[i] = 0;
-        __syncthreads();
-        for (int base = 0; base < n; base += NT) {
-            const int i = base + tid;
-            const uint32_t key = i < n ? src.k(i) : 0u;
-            const bool in = i < n && (key & mask) == prefix;
-            const unsigned dgt = in ? (key >> shift) & 255u : 256u;     // 256 = not counted
-            const unsigned peers = __match_any_sync(0xffffffffu, dgt);  // one add per distinct digit
-            if (in && lane == __ffs(peers) - 1) atomicAdd(&s_hist[dgt], (uint32_t)__popc(peers));
-        }
-        __syncthreads();
-        if (tid < 32) {
-            // lane l owns digits 255-8l .. 248-8l (descending)
-            int c = 0;
-#pragma unroll
-            for (int u = 0; u < 8; ++u) c += (int)s_hist[255 - 8 * lane - u];
-            int inc = c;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                int tt = __shfl_up_sync(0xffffffffu, inc, o);
-                if (lane >= o) inc += tt;
-            }
-            int above = inc - c;
-            if (above < kk && kk <= above + c) {
-                int acc = above;
-                for (int u = 0; u < 8; ++u) {
-                    const int dgt = 255 - 8 * lane - u;
-                    const int h = (int)s_hist[dgt];
-                    if (kk <= acc + h) { s_misc[0] = dgt; s_misc[1] = kk - acc; break; }
-                    acc += h;
-                }
-            }
-        }
-        __syncthreads();
-        prefix |= (uint32_t)s_misc[0] << shift;
-        mask |= 255u << shift;
-        kk = s_misc[1];
-        __syncthreads();
-    }
-    vstar = prefix;
-    need_eq = kk;
-}
 
 // Threshold by radix bisection.  Finds v, a multiple of 2^low_bit, with at least K of
-// key[0..n) >= v (n >= K >= 1), five key bits per round, starting at the first bit in
+// the keys of src[0..n) >= v (n >= K >= 1), five key bits per round, starting at the first bit in
 // which the keys differ at all.  Each round histograms the next digit of the keys that
 // still match the prefix into 32 bins x 32 lane columns (a lane only ever adds to its own
 // column, so clustered keys do not serialise), sums the columns, and descends into the
@@ -346,7 +293,7 @@ struct Threshold {
 };
 
 template <int NT>
-__device__ __noinline__ Threshold count_threshold(const uint32_t* key, int n, int K, int low_bit, int* s_h) {
+__device__ __noinline__ Threshold count_threshold(const KeySrc src, int n, int K, int low_bit, int* s_h) {
     static_assert(NT % 32 == 0 && NT >= 256, "32 digits are shared out over NT / 32 warps");
     constexpr int NW = NT / 32;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -354,7 +301,7 @@ __device__ __noinline__ Threshold count_threshold(const uint32_t* key, int n, in
     int* s_tot = s_h + 2048;
     // common leading bits of all keys
     uint32_t kmin = 0xffffffffu, kmax = 0u;
-    for (int i = tid; i < n; i += NT) { const uint32_t k = key[i]; kmin = min(kmin, k); kmax = max(kmax, k); }
+    for (int i = tid; i < n; i += NT) { const uint32_t k = src.k(i); kmin = min(kmin, k); kmax = max(kmax, k); }
     kmin = __reduce_min_sync(0xffffffffu, kmin);
     kmax = __reduce_max_sync(0xffffffffu, kmax);
     if (lane == 0) { s_tot[warp] = (int)kmin; s_tot[32 + warp] = (int)kmax; }
@@ -375,7 +322,7 @@ __device__ __noinline__ Threshold count_threshold(const uint32_t* key, int n, in
         const int shift = hi - width;
         const uint32_t himask = hi >= 32 ? 0u : 0xffffffffu << hi;
         for (int i = tid; i < n; i += NT) {
-            const uint32_t k = key[i];
+            const uint32_t k = src.k(i);
             if ((k & himask) == prefix) atomicAdd(&hist[(((k >> shift) & ((1u << width) - 1u)) << 5) + lane], 1);
         }
         __syncthreads();
@@ -425,8 +372,8 @@ __device__ __forceinline__ int warp_base(const int* s_cnt, int& total) {
 // the support in ascending index order with ties resolved to the lower index.  Every thread
 // takes one contiguous run of the source, so a single prefix sum places them all.  The general
 // form (any number of ties at v); s_ws: WS_WORDS ints.
-template <int NT, class Src>
-__device__ __noinline__ void ordered_emit(const Src& src, int n, uint32_t vstar, int need_eq, int32_t* s_sup_idx,
+template <int NT>
+__device__ __noinline__ void ordered_emit(const KeySrc src, int n, uint32_t vstar, int need_eq, int32_t* s_sup_idx,
                              uint32_t* s_sup_key, int* s_ws) {
     const int tid = threadIdx.x;
     const int ipt = (n + NT - 1) / NT;                 // NT is a power of two: a shift
@@ -589,6 +536,7 @@ __device__ __forceinline__ int select_small(const uint32_t* s_key, const int32_t
             if (in[r] && b[r] == bstar) {
                 const int pos = r * NT + tid;
                 int rank = 0;
+#pragma unroll 4
                 for (int j = 0; j < m; ++j) {
                     const uint32_t o = (uint32_t)s_bl[j];
                     rank += (int)(o > k[r]) | ((int)(o == k[r]) & (int)(s_bl[SEL_LIST + j] < pos));
@@ -623,19 +571,34 @@ __device__ __forceinline__ int select_small(const uint32_t* s_key, const int32_t
     return 1;
 }
 
+// Top-K of src[0..n) (n > K) by radix bisection and the general emit, for any number of ties:
+// ascending index order out, ties to the lower index.  Returns the largest key.
+template <int NT>
+__device__ __forceinline__ uint32_t select_general(const KeySrc src, int n, int K, int32_t* s_sup_idx,
+                                                   uint32_t* s_sup_key, uint32_t* s_hist, int* s_ws) {
+    const Threshold t = count_threshold<NT>(src, n, K, 0, reinterpret_cast<int*>(s_hist));
+    uint32_t vstar;
+    int need_eq;
+    if (t.count == K) { vstar = t.v - 1u; need_eq = 0; }            // exactly K keys are >= v
+    else { vstar = t.v; need_eq = t.need; }                          // v = K-th largest key
+    ordered_emit<NT>(src, n, vstar, need_eq, s_sup_idx, s_sup_key, s_ws);
+    return t.kmax;
+}
+
 // Top-K of the n listed entries (ascending index order in, ascending index order out).
-// kmax_out: largest listed key when known (n > K), else 0 with *kmax_known = false.
+// *kmax_out: the largest listed key.
 // Short lists (at most 3 * NT keys, the usual case) take the loop-free form; longer ones, or
 // a list it hands back (all keys equal, a boundary bin with hundreds of members), the radix
 // bisection and the general emit.  s_hist: SCRATCH_WORDS words; s_ws: WS_WORDS ints.
 // One copy serves both paths of finish_kernel.
 template <int NT>
-__device__ int select_listed(const uint32_t* s_key, const int32_t* s_idx, int n, int K,
+__device__ __forceinline__ int select_listed_body(const uint32_t* s_key, const int32_t* s_idx, int n, int K,
                                           int32_t* s_sup_idx, uint32_t* s_sup_key, uint32_t* s_hist, int* s_ws,
                                           uint32_t* kmax_out) {
     int ns;
     uint32_t kmax = 0u;
     if (n <= K) {
+#pragma unroll 1
         for (int i = threadIdx.x; i < n; i += NT) { s_sup_idx[i] = s_idx[i]; s_sup_key[i] = s_key[i]; kmax = max(kmax, s_key[i]); }
         ns = n;
         // (the largest key of a short list: one more reduction, it is rare)
@@ -648,19 +611,19 @@ __device__ int select_listed(const uint32_t* s_key, const int32_t* s_idx, int n,
         ns = K;
     } else {
         __syncthreads();                               // (the short form may have left the scratch in use)
-        SmemSrc src{s_key, s_idx};
-        const Threshold t = count_threshold<NT>(s_key, n, K, 0, reinterpret_cast<int*>(s_hist));
-        uint32_t vstar;
-        int need_eq;
-        if (t.count == K) { vstar = t.v - 1u; need_eq = 0; }            // exactly K keys are >= v
-        else { vstar = t.v; need_eq = t.need; }                          // v = K-th largest key
-        ordered_emit<NT>(src, n, vstar, need_eq, s_sup_idx, s_sup_key, s_ws);
+        kmax = select_general<NT>(KeySrc{s_key, s_idx, nullptr}, n, K, s_sup_idx, s_sup_key, s_hist, s_ws);
         ns = K;
-        kmax = t.kmax;
     }
     __syncthreads();
     *kmax_out = kmax;
     return ns;
+}
+
+template <int NT>
+__device__ __noinline__ int select_listed(const uint32_t* s_key, const int32_t* s_idx, int n, int K,
+                                          int32_t* s_sup_idx, uint32_t* s_sup_key, uint32_t* s_hist, int* s_ws,
+                                          uint32_t* kmax_out) {
+    return select_listed_body<NT>(s_key, s_idx, n, K, s_sup_idx, s_sup_key, s_hist, s_ws, kmax_out);
 }
 
 // Largest key of s_key[0..n) (the rare callers that select without learning it).  Ends with a barrier.
@@ -668,6 +631,7 @@ template <int NT>
 __device__ __noinline__ uint32_t block_max_key(const uint32_t* s_key, int n, int* s_ws) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     uint32_t kmax = 0u;
+#pragma unroll 1
     for (int i = tid; i < n; i += NT) kmax = max(kmax, s_key[i]);
     kmax = __reduce_max_sync(0xffffffffu, kmax);
     if (lane == 0) s_ws[warp] = (int)kmax;
@@ -713,6 +677,7 @@ __device__ __forceinline__ void cache_similarities(const StepArgs& a, int bh, fl
     }
     float inv_nrm = 0.f;
     constexpr int U = NT >= 1024 ? 4 : 8;            // cache rows per warp and trip, all requested before any is used
+#pragma unroll 1
     for (int c0 = warp; c0 < fill || c0 == warp; c0 += NW * U) {
         float4 x[U];
 #pragma unroll
@@ -770,6 +735,7 @@ __device__ __forceinline__ void warp_top_slots(const float* s_rho, int lo, int h
         const int c = lo + v * 32 + lane;
         key[v] = c < hi ? score_key(s_rho[c]) : 0u;            // a live key is 0 only for one NaN pattern
     }
+#pragma unroll 1
     for (int j = 0; j < n_take; ++j) {
         uint32_t best = 0u;
         int best_c = 0x7fffffff;
@@ -785,33 +751,21 @@ __device__ __forceinline__ void warp_top_slots(const float* s_rho, int lo, int h
     }
 }
 
+// The cases beside the common one (Recent-R, more than eight recalled slots, more than 256
+// cached entries), kept out of line so the common path stays short.  Ends without a barrier.
 template <int NT>
-__device__ __forceinline__ float recall_slots(const StepArgs& a, const float* s_rho, int* s_sel, float* s_misc, int* s_ws,
-                                              int* sel8) {
+__device__ __noinline__ void recall_slots_general(bool recent, int r, int M, int fill, int slot, const float* s_rho,
+                                                  int* s_sel, float* s_misc, int* s_ws) {
+    // (scalars, not the argument block: a reference to it would force a copy in local memory)
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int M = a.M, fill = a.fill;
-    const int n_sel = a.r < fill ? a.r : fill;
-    if (__builtin_expect(!a.recall_recent && n_sel <= 8 && fill <= 256 && fill > 0, 1)) {
-        // The common case: one warp, up to eight entries per lane, one argmax round per recalled
-        // slot (two warp reductions each).  (Having every warp do it for itself was tried: it
-        // saves the barrier but costs several times more issue slots than it saves.)
-        if (warp == 0) {
-            uint32_t* k_out = reinterpret_cast<uint32_t*>(s_ws);
-            warp_top_slots(s_rho, 0, fill, n_sel, lane, k_out, s_sel);
-            __syncwarp();
-            if (lane == 0 && s_sel[0] >= 0) s_misc[0] = s_rho[s_sel[0]];
-        }
-        __syncthreads();
-#pragma unroll
-        for (int j = 0; j < 8; ++j) sel8[j] = j < a.r ? s_sel[j] : -1;
-        return s_misc[0];
-    }
-    if (a.recall_recent) {
+    const int n_sel = r < fill ? r : fill;
+    if (recent) {
         // Recent-R ablation: the newest n_sel entries (newest first), rho_max over those only
         if (tid < 32) {
             float best = -CUDART_INF_F;
+#pragma unroll 1
             for (int j = lane; j < n_sel; j += 32) {
-                const int c = ((a.slot - 1 - j) % M + M) % M;
+                const int c = ((slot - 1 - j) % M + M) % M;
                 s_sel[j] = c;
                 best = fmaxf(best, s_rho[c]);
             }
@@ -826,10 +780,12 @@ __device__ __forceinline__ float recall_slots(const StepArgs& a, const float* s_
         int lp = 5;
         while (lp > 0 && (fill << lp) > NT) --lp;
         const int P = 1 << lp, part = tid & (P - 1);
+#pragma unroll 1
         for (int me = tid >> lp; me < ((fill + (NT >> lp) - 1) / (NT >> lp)) * (NT >> lp); me += NT >> lp) {
             const bool live = me < fill;
             const float mine = live ? s_rho[me] : 0.f;
             int rank = 0;
+#pragma unroll 2
             for (int c = part; c < fill; c += P) {
                 const float o = s_rho[c];
                 rank += (int)(o > mine) | ((int)(o == mine) & (int)(c < me));
@@ -854,6 +810,7 @@ __device__ __forceinline__ float recall_slots(const StepArgs& a, const float* s_
             uint32_t key = (g < groups && j < n_sel) ? reinterpret_cast<uint32_t*>(s_ws)[g * 16 + j] : 0u;
             int slot = (g < groups && j < n_sel) ? s_ws[g * 16 + 8 + j] : 0x7fffffff;
             if (slot < 0) { slot = 0x7fffffff; key = 0u; }
+#pragma unroll 1
             for (int t = 0; t < n_sel; ++t) {
                 const uint32_t top = __reduce_max_sync(0xffffffffu, key);
                 const int c_star = __reduce_min_sync(0xffffffffu, key == top && top != 0u ? slot : 0x7fffffff);
@@ -861,6 +818,27 @@ __device__ __forceinline__ float recall_slots(const StepArgs& a, const float* s_
                 if (lane == 0 && c_star != 0x7fffffff) { s_sel[t] = c_star; if (t == 0) s_misc[0] = s_rho[c_star]; }
             }
         }
+    }
+}
+
+template <int NT>
+__device__ __forceinline__ float recall_slots(const StepArgs& a, const float* s_rho, int* s_sel, float* s_misc, int* s_ws,
+                                              int* sel8) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int fill = a.fill;
+    const int n_sel = a.r < fill ? a.r : fill;
+    if (__builtin_expect(!a.recall_recent && n_sel <= 8 && fill <= 256 && fill > 0, 1)) {
+        // The common case: one warp, up to eight entries per lane, one argmax round per recalled
+        // slot (two warp reductions each).  (Having every warp do it for itself was tried: it
+        // saves the barrier but costs several times more issue slots than it saves.)
+        if (warp == 0) {
+            uint32_t* k_out = reinterpret_cast<uint32_t*>(s_ws);
+            warp_top_slots(s_rho, 0, fill, n_sel, lane, k_out, s_sel);
+            __syncwarp();
+            if (lane == 0 && s_sel[0] >= 0) s_misc[0] = s_rho[s_sel[0]];
+        }
+    } else {
+        recall_slots_general<NT>(a.recall_recent != 0, a.r, a.M, fill, a.slot, s_rho, s_sel, s_misc, s_ws);
     }
     __syncthreads();
 #pragma unroll
@@ -994,6 +972,7 @@ __device__ __forceinline__ int candidate_union(const StepArgs& a, int bh, const 
     {
         bool bad = false;
         for (int s0 = 0; s0 < n_sel; s0 += 4)
+#pragma unroll 1
             for (int i = tid; i < K; i += NT) {
                 int idx[4];
 #pragma unroll
@@ -1017,9 +996,11 @@ __device__ __forceinline__ int candidate_union(const StepArgs& a, int bh, const 
     const int w0 = tid * wpt;
     const int w1 = (w0 + wpt < nw_lo) ? w0 + wpt : nw_lo;
     int cnt = 0;
+#pragma unroll 4
     for (int w = w0; w < w1; ++w) cnt += __popc(s_bm[w]);
     int n_low;
     int pos = block_excl_scan<NT>(cnt, s_ws, n_low);
+#pragma unroll 1
     for (int w = w0; w < w1; ++w) {
         uint32_t bits = s_bm[w];
         while (bits) {
@@ -1028,6 +1009,7 @@ __device__ __forceinline__ int candidate_union(const StepArgs& a, int bh, const 
             bits &= bits - 1;
         }
     }
+#pragma unroll 1
     for (int i = w_lo + tid; i < L; i += NT) s_idx[n_low + (i - w_lo)] = i;
     return n_low + (L - w_lo);
 }
@@ -1091,9 +1073,9 @@ __device__ __forceinline__ void score_candidates(const uint16_t* kbase, const in
 // through distributed shared memory and are added there in rank order.
 // ------------------------------------------------------------------------------------
 template <int D, int NT>
-__device__ void attend(const uint16_t* vbase, int ns, const int32_t* s_sup_idx, const uint32_t* s_sup_key,
-                       float* s_w, float* s_red, int* s_ws, uint4* s_stage, int depth, uint32_t kmax,
-                       bool kmax_known, uint16_t* out_row, int cl_rank = 0, int cl_size = 1) {
+__device__ __forceinline__ void attend_body(const uint16_t* vbase, int ns, const int32_t* s_sup_idx, const uint32_t* s_sup_key,
+                                    float* s_w, float* s_red, int* s_ws, uint4* s_stage, int depth, uint32_t kmax,
+                                    uint16_t* out_row, int cl_rank, int cl_size, int ptab) {
     constexpr int LPR = D / 8;                  // lanes per bf16 row (16 bytes each)
     constexpr int RPW = 32 / LPR;               // rows per warp load
     constexpr int SLOTS = (NT / 32) * RPW;      // row slots per block
@@ -1106,47 +1088,44 @@ __device__ void attend(const uint16_t* vbase, int ns, const int32_t* s_sup_idx, 
     // this CTA's share of the support: [i_lo, i_hi)
     const int share = (ns + cl_size - 1) / cl_size;
     const int i_lo = min(ns, cl_rank * share), i_hi = min(ns, i_lo + share);
-
-    auto issue = [&](int base) {
+    float denom = 0.f;
+    float acc[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+    RETOPK_PHASE(ptab, 16);
+    for (int base = i_lo;;) {
+        // (code kept compact on purpose: loops, not unrolled copies)
 #pragma unroll 4
         for (int u = 0; u < depth; ++u) {
             const int i = base + u * SLOTS + myslot;
             if (i < i_hi) cp_async16(my_stage + u * NT, vsrc + (size_t)s_sup_idx[i] * (D * 2));
         }
         cp_async_commit();
-    };
-    issue(i_lo);
-
-    if (!kmax_known) {
-        kmax = 0;
-        for (int i = tid; i < ns; i += NT) kmax = max(kmax, s_sup_key[i]);
-        kmax = __reduce_max_sync(0xffffffffu, kmax);
-        if (lane == 0) s_ws[warp] = (int)kmax;
-        __syncthreads();
-        kmax = __reduce_max_sync(0xffffffffu, lane < NW ? (uint32_t)s_ws[lane] : 0u);
-        __syncthreads();
-    }
-    const float smax = key_score(kmax);
-    float wsum = 0.f;
-    for (int i = tid; i < ns; i += NT) {
-        const float w = expf(key_score(s_sup_key[i]) - smax);
-        s_w[i] = w;
-        wsum += w;
-    }
+        if (base == i_lo) {
+            // the softmax weights (all ns of them: the denominator is the whole sum) while the
+            // first wave of rows is in the air
+            RETOPK_PHASE(ptab, 17);
+            const float smax = key_score(kmax);
+            float wsum = 0.f;
+#pragma unroll 1
+            for (int i = tid; i < ns; i += NT) {
+                const float w = expf(key_score(s_sup_key[i]) - smax);
+                s_w[i] = w;
+                wsum += w;
+            }
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) wsum += __shfl_xor_sync(0xffffffffu, wsum, o);
-    float* s_wsf = reinterpret_cast<float*>(s_ws);
-    if (lane == 0) s_wsf[warp] = wsum;
-    __syncthreads();
-    float denom = lane < NW ? s_wsf[lane] : 0.f;         // fixed tree: the same sum on every lane and run
+            for (int o = 16; o > 0; o >>= 1) wsum += __shfl_xor_sync(0xffffffffu, wsum, o);
+            float* s_wsf = reinterpret_cast<float*>(s_ws);
+            if (lane == 0) s_wsf[warp] = wsum;
+            __syncthreads();
+            denom = lane < NW ? s_wsf[lane] : 0.f;         // fixed tree: the same sum on every lane and run
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) denom += __shfl_xor_sync(0xffffffffu, denom, o);
-
-    float acc[8];
-#pragma unroll
-    for (int e = 0; e < 8; ++e) acc[e] = 0.f;
-    for (int base = i_lo;;) {
+            for (int o = 16; o > 0; o >>= 1) denom += __shfl_xor_sync(0xffffffffu, denom, o);
+            RETOPK_PHASE(ptab, 18);
+        }
         cp_async_wait_all();
+        if (base == i_lo) RETOPK_PHASE(ptab, 19);
+#pragma unroll 4
         for (int u = 0; u < depth; ++u) {
             const int i = base + u * SLOTS + myslot;
             if (i < i_hi) {
@@ -1159,8 +1138,8 @@ __device__ void attend(const uint16_t* vbase, int ns, const int32_t* s_sup_idx, 
         }
         base += SLOTS * depth;
         if (base >= i_hi) break;
-        issue(base);
     }
+    RETOPK_PHASE(ptab, 20);
     // fixed-order reduction: row slots of a warp, then warps in groups, then groups
 #pragma unroll
     for (int o = LPR; o < 32; o <<= 1)
@@ -1193,6 +1172,7 @@ __device__ void attend(const uint16_t* vbase, int ns, const int32_t* s_sup_idx, 
         cluster.sync();
         if (cl_rank == 0 && tid < D) {
             sum = 0.f;
+#pragma unroll 1
             for (int r = 0; r < cl_size; ++r) sum += *cluster.map_shared_rank(s_red + tid, r);
         }
         cluster.sync();           // nobody leaves while its shared memory may still be read
@@ -1204,6 +1184,13 @@ __device__ void attend(const uint16_t* vbase, int ns, const int32_t* s_sup_idx, 
     }
 }
 
+template <int D, int NT>
+__device__ __noinline__ void attend(const uint16_t* vbase, int ns, const int32_t* s_sup_idx, const uint32_t* s_sup_key,
+                                    float* s_w, float* s_red, int* s_ws, uint4* s_stage, int depth, uint32_t kmax,
+                                    uint16_t* out_row, int cl_rank = 0, int cl_size = 1, int ptab = 1) {
+    attend_body<D, NT>(vbase, ns, s_sup_idx, s_sup_key, s_w, s_red, s_ws, s_stage, depth, kmax, out_row, cl_rank, cl_size, ptab);
+}
+
 // ------------------------------------------------------------------------------------
 // reuse path of finish_kernel: candidate union (Eq. 8-9), candidate scores (Eq. 10), Top-K
 // (Eq. 11), softmax.V (Eq. 12) and the support insert for one head, all in shared memory.
@@ -1212,7 +1199,7 @@ __device__ void attend(const uint16_t* vbase, int ns, const int32_t* s_sup_idx, 
 // clocks showed them level or ahead, the timed pipeline 3 us per step behind: dropped.)
 // ------------------------------------------------------------------------------------
 template <int D, int NT>
-__device__ void reuse_path(const StepArgs& a, unsigned char* smem_raw) {
+__device__ __forceinline__ void reuse_path(const StepArgs& a, unsigned char* smem_raw) {
     constexpr int NW = NT / 32;
     // layout (words): qraw[D] sel[r] ws[WS_WORDS] hist[SCRATCH_WORDS] sup_idx[K] sup_key[K] w[K]
     //                 | big: idx[cap] key[cap], aliased later by red[NW*D+NT] | bitmap | stage[depth*NT*4]
@@ -1251,6 +1238,7 @@ __device__ void reuse_path(const StepArgs& a, unsigned char* smem_raw) {
     {
         const int nwords = (L + 31) >> 5;
         uint4* bm4 = reinterpret_cast<uint4*>(s_bm);
+#pragma unroll 1
         for (int w = tid; w < (nwords + 3) >> 2; w += NT) bm4[w] = make_uint4(0, 0, 0, 0);
     }
     __syncthreads();
@@ -1262,43 +1250,53 @@ __device__ void reuse_path(const StepArgs& a, unsigned char* smem_raw) {
     RETOPK_PHASE(0, 3);
 
     if (a.dbg_cand && cl_rank == 0)
+#pragma unroll 1
         for (int i = tid; i < n; i += NT) a.dbg_cand[(size_t)bh * a.cap + i] = s_idx[i];
 
     // Eq. 10.  In a cluster every CTA built the same list; each scores a contiguous share of
     // it and hands the keys to the others through distributed shared memory.
-    if (cl_size == 1) {
-        score_candidates<D, NT, true>(a.k + (size_t)bkv * a.max_seq_len * D, s_idx, n, s_qraw, s_stage,
-                                      a.stage_depth, a.scale, s_key);
-        __syncthreads();
-    } else {
-        namespace cg = cooperative_groups;
-        cg::cluster_group cluster = cg::this_cluster();
+    {
         const int share = (n + cl_size - 1) / cl_size;
         const int lo = min(n, cl_rank * share), hi = min(n, lo + share);
         score_candidates<D, NT, true>(a.k + (size_t)bkv * a.max_seq_len * D, s_idx + lo, hi - lo, s_qraw, s_stage,
                                       a.stage_depth, a.scale, s_key + lo);
         __syncthreads();
-        for (int r = 1; r < cl_size; ++r) {
-            uint32_t* peer = cluster.map_shared_rank(s_key, (cl_rank + r) & (cl_size - 1));
-            for (int i = lo + tid; i < hi; i += NT) peer[i] = s_key[i];
+        if (cl_size > 1) {
+            namespace cg = cooperative_groups;
+            cg::cluster_group cluster = cg::this_cluster();
+#pragma unroll 1
+            for (int r = 1; r < cl_size; ++r) {
+                uint32_t* peer = cluster.map_shared_rank(s_key, (cl_rank + r) & (cl_size - 1));
+#pragma unroll 1
+                for (int i = lo + tid; i < hi; i += NT) peer[i] = s_key[i];
+            }
+            cluster.sync();
         }
-        cluster.sync();
     }
     RETOPK_PHASE(0, 4);
 
     // Eq. 11: Top-K of the candidates; insert the support
     uint32_t kmax;
-    const bool kmax_known = true;
+#ifdef RETOPK_REUSE_INLINE
+    const int ns = select_listed_body<NT>(s_key, s_idx, n, K, s_sup_idx, s_sup_key, s_hist, s_ws, &kmax);
+#else
     const int ns = select_listed<NT>(s_key, s_idx, n, K, s_sup_idx, s_sup_key, s_hist, s_ws, &kmax);
+#endif
     RETOPK_PHASE(0, 5);
     if (cl_rank == 0) {
         int32_t* sup_out = a.sup_cache + ((size_t)bh * M + a.slot) * K;
+#pragma unroll 1
         for (int i = tid; i < K; i += NT) sup_out[i] = i < ns ? s_sup_idx[i] : -1;
     }
 
     // Eq. 12 (s_red aliases the candidate lists, which are dead now)
+#ifdef RETOPK_REUSE_INLINE
+    attend_body<D, NT>(a.v + (size_t)bkv * a.max_seq_len * D, ns, s_sup_idx, s_sup_key, s_w, s_red, s_ws, s_stage,
+                  a.stage_depth, kmax, a.out + (size_t)bh * D, cl_rank, cl_size, 0);
+#else
     attend<D, NT>(a.v + (size_t)bkv * a.max_seq_len * D, ns, s_sup_idx, s_sup_key, s_w, s_red, s_ws, s_stage,
-                  a.stage_depth, kmax, kmax_known, a.out + (size_t)bh * D, cl_rank, cl_size);
+                  a.stage_depth, kmax, a.out + (size_t)bh * D, cl_rank, cl_size, 0);
+#endif
     if (tid == 0 && cl_rank == 0) {      // the step record is written last: nothing in this kernel waits for it
         a.ws_ncand[bh] = n;
         atomicAdd(a.counters + (size_t)bh * 4 + PATH_REUSE, 1ull);
@@ -1442,8 +1440,16 @@ __device__ __forceinline__ void scan_body(const StepArgs& a) {
                     m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 16));
                     if (head < G && ((need >> head) & 1u)) {
                         float* srow = a.ws_scores + (size_t)(head0 + head) * a.score_stride;
+#if RETOPK_SCORE_POLICY == 1
+                        if (r0 < L) srow[r0] = c[e] * scale;
+                        if (r1 < L) srow[r1] = c[2 + e] * scale;
+#elif RETOPK_SCORE_POLICY == 2
+                        if (r0 < L) stg_hint(srow + r0, c[e] * scale, pol_first);
+                        if (r1 < L) stg_hint(srow + r1, c[2 + e] * scale, pol_first);
+#else
                         if (r0 < L) stg_hint(srow + r0, c[e] * scale, pol_last);
                         if (r1 < L) stg_hint(srow + r1, c[2 + e] * scale, pol_last);
+#endif
                         if (g == 0 && tile_row < L)
                             stg_hint(a.ws_tmax + (size_t)(head0 + head) * a.tmax_stride + (tile_row >> 4), m * scale, pol_last);
                     }
@@ -1482,7 +1488,7 @@ __global__ void __launch_bounds__(SCAN_THREADS) scan_kernel(const StepArgs a) {
 // lower-index tie rule is taken from that list.
 // ------------------------------------------------------------------------------------
 template <int D, int NT>
-__device__ void exact_path(const StepArgs& a, unsigned char* smem_raw) {
+__device__ __forceinline__ void exact_path(const StepArgs& a, unsigned char* smem_raw) {
     // In a cluster every CTA of a head selects the same support on its own (the lists are short
     // and come from L2); only the value rows are shared out, and rank 0 writes the results.
     const int bh = cluster_slot(a);
@@ -1515,6 +1521,7 @@ __device__ void exact_path(const StepArgs& a, unsigned char* smem_raw) {
     RETOPK_PHASE(2, 0);
 
     if (L <= K) {
+#pragma unroll 1
         for (int i = tid; i < L; i += NT) { s_sup_idx[i] = i; s_sup_key[i] = score_key(sc[i]); }
         ns = L;
         __syncthreads();
@@ -1528,7 +1535,27 @@ __device__ void exact_path(const StepArgs& a, unsigned char* smem_raw) {
         while (((ntile + (1 << sh) - 1) >> sh) > NS) ++sh;
         const int g2 = 1 << sh;
         const int n2 = (ntile + g2 - 1) >> sh;
-        if (n2 >= K) {
+        // the usual shape: eight tile maxima per thread, kept in registers for step 2
+        const bool regs8 = sh == 3 && n2 <= NT;
+        float mv[8];
+        if (regs8) {
+            const int t0 = tid * 8;
+            float4 m4[2];
+#pragma unroll
+            for (int u = 0; u < 2; ++u)
+                m4[u] = t0 + 4 * u < ntile ? *reinterpret_cast<const float4*>(tm + t0 + 4 * u)
+                                           : make_float4(0.f, 0.f, 0.f, 0.f);
+            const float raw[8] = {m4[0].x, m4[0].y, m4[0].z, m4[0].w, m4[1].x, m4[1].y, m4[1].z, m4[1].w};
+            float m = -CUDART_INF_F;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                mv[e] = t0 + e < ntile ? raw[e] : -CUDART_INF_F;
+                m = fmaxf(m, mv[e]);
+            }
+            if (tid < n2) s_key[tid] = score_key(m);
+            __syncthreads();
+        } else if (n2 >= K) {
+#pragma unroll 1
             for (int i2 = tid; i2 < n2; i2 += NT) {
                 const int t0 = i2 << sh;
                 float m;
@@ -1558,31 +1585,46 @@ __device__ void exact_path(const StepArgs& a, unsigned char* smem_raw) {
                 s_key[i2] = score_key(m);
             }
             __syncthreads();
-            thr_key = count_threshold<NT>(s_key, n2, K, 16, reinterpret_cast<int*>(s_hist)).v;
+        }
+        if (n2 >= K) {
+            // one histogram over the span of the maxima when they fit the loop-free form (the
+            // bound it gives is a key of the list, tighter than a truncated one), else bisection
+            uint32_t unused;
+            const int done = n2 <= NT
+                ? select_small<NT, 1, false>(s_key, nullptr, n2, K, nullptr, nullptr, reinterpret_cast<int*>(s_hist), &unused, &thr_key)
+                : 0;
+            if (!done) {
+                __syncthreads();
+                thr_key = count_threshold<NT>(KeySrc{s_key, nullptr, nullptr}, n2, K, 16, reinterpret_cast<int*>(s_hist)).v;
+            }
         }
         RETOPK_PHASE(2, 1);
         // 2. the tiles whose maximum reaches v, in ascending order: eight consecutive tile
         //    maxima per thread and one prefix sum per 8 * NT tiles
         int nhit = 0;
+#pragma unroll 1
         for (int base = 0; base < ntile; base += NT * 8) {
             const int t0 = base + tid * 8;
-            float4 m4[2];
+            if (!regs8) {
+                float4 m4[2];
 #pragma unroll
-            for (int u = 0; u < 2; ++u)
-                m4[u] = t0 + 4 * u < ntile ? *reinterpret_cast<const float4*>(tm + t0 + 4 * u)
-                                           : make_float4(0.f, 0.f, 0.f, 0.f);
-            const float mv[8] = {m4[0].x, m4[0].y, m4[0].z, m4[0].w, m4[1].x, m4[1].y, m4[1].z, m4[1].w};
+                for (int u = 0; u < 2; ++u)
+                    m4[u] = t0 + 4 * u < ntile ? *reinterpret_cast<const float4*>(tm + t0 + 4 * u)
+                                               : make_float4(0.f, 0.f, 0.f, 0.f);
+                mv[0] = m4[0].x; mv[1] = m4[0].y; mv[2] = m4[0].z; mv[3] = m4[0].w;
+                mv[4] = m4[1].x; mv[5] = m4[1].y; mv[6] = m4[1].z; mv[7] = m4[1].w;
+            }
             unsigned hits = 0;
 #pragma unroll
             for (int e = 0; e < 8; ++e)
                 if (t0 + e < ntile && score_key(mv[e]) >= thr_key) hits |= 1u << e;
             int total;
             int pos = nhit + block_excl_scan<NT>(__popc(hits), s_ws, total);
-            while (hits) {
-                const int e = __ffs(hits) - 1;
-                if (pos < tcap) s_tile[pos] = t0 + e;
-                ++pos;
-                hits &= hits - 1;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {               // predicated, no loop: a few hits per thread at most
+                const bool hit = (hits >> e) & 1u;
+                if (hit && pos < tcap) s_tile[pos] = t0 + e;
+                pos += hit ? 1 : 0;
             }
             nhit += total;
         }
@@ -1591,6 +1633,7 @@ __device__ void exact_path(const StepArgs& a, unsigned char* smem_raw) {
         if (nhit > tcap) slow = true;
         else {
             // 3. one thread per hit tile: its 16 scores, those >= v listed in index order
+#pragma unroll 1
             for (int base = 0; base < nhit; base += NT) {
                 const int it = base + tid;
                 float4 x[4];
@@ -1600,21 +1643,22 @@ __device__ void exact_path(const StepArgs& a, unsigned char* smem_raw) {
                     row0 = s_tile[it] * TILE_ROWS;
 #pragma unroll
                     for (int u = 0; u < 4; ++u) x[u] = *reinterpret_cast<const float4*>(sc + row0 + 4 * u);
+                } else {
 #pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        const float v4[4] = {x[u].x, x[u].y, x[u].z, x[u].w};
-#pragma unroll
-                        for (int e = 0; e < 4; ++e)
-                            if (row0 + 4 * u + e < L && score_key(v4[e]) >= thr_key) fl |= 1u << (4 * u + e);
-                    }
+                    for (int u = 0; u < 4; ++u) x[u] = make_float4(0.f, 0.f, 0.f, 0.f);
                 }
+                const float v16[16] = {x[0].x, x[0].y, x[0].z, x[0].w, x[1].x, x[1].y, x[1].z, x[1].w,
+                                       x[2].x, x[2].y, x[2].z, x[2].w, x[3].x, x[3].y, x[3].z, x[3].w};
+#pragma unroll
+                for (int e = 0; e < 16; ++e)
+                    if (it < nhit && row0 + e < L && score_key(v16[e]) >= thr_key) fl |= 1u << e;
                 int total;
                 int pos = n + block_excl_scan<NT>(__popc(fl), s_ws, total);
-                while (fl) {
-                    const int e = __ffs(fl) - 1;
-                    if (pos < NS) { s_key[pos] = score_key(sc[row0 + e]); s_idx[pos] = row0 + e; }
-                    ++pos;
-                    fl &= fl - 1;
+#pragma unroll
+                for (int e = 0; e < 16; ++e) {          // from the registers, predicated
+                    const bool hit = (fl >> e) & 1u;
+                    if (hit && pos < NS) { s_key[pos] = score_key(v16[e]); s_idx[pos] = row0 + e; }
+                    pos += hit ? 1 : 0;
                 }
                 n += total;
             }
@@ -1623,20 +1667,18 @@ __device__ void exact_path(const StepArgs& a, unsigned char* smem_raw) {
         }
     }
     RETOPK_PHASE(2, 3);
+    uint32_t kmax;
     if (slow) {
-        // multi-pass select straight from the score array (heavy ties, odd distributions)
-        ScoreSrc src{sc};
-        uint32_t vstar;
-        int need_eq;
-        radix_select<NT>(src, L, K, s_hist, s_misc, vstar, need_eq);
-        ordered_emit<NT>(src, L, vstar, need_eq, s_sup_idx, s_sup_key, s_ws);
+        // straight from the score array (heavy ties, odd distributions)
+        kmax = select_general<NT>(KeySrc{nullptr, nullptr, sc}, L, K, s_sup_idx, s_sup_key, s_hist, s_ws);
         ns = K;
         if (tid == 0 && cl_rank == 0) atomicAdd(a.slow_select, 1ull);
         __syncthreads();
+    } else if (ns < 0) {
+        ns = select_listed<NT>(s_key, s_idx, n, K, s_sup_idx, s_sup_key, s_hist, s_ws, &kmax);
+    } else {
+        kmax = block_max_key<NT>(s_sup_key, ns, s_ws);      // L <= K: everything is selected
     }
-    uint32_t kmax = 0;
-    bool kmax_known = false;
-    if (ns < 0) { ns = select_listed<NT>(s_key, s_idx, n, K, s_sup_idx, s_sup_key, s_hist, s_ws, &kmax); kmax_known = true; }
     RETOPK_PHASE(2, 4);
 
     // record the support (cache insert / caller's index output)
@@ -1644,10 +1686,11 @@ __device__ void exact_path(const StepArgs& a, unsigned char* smem_raw) {
     if (a.mode == MODE_RETOPK) sup_out = a.sup_cache + ((size_t)bh * a.M + a.slot) * K;
     else if (a.idx_out) sup_out = a.idx_out + (size_t)bh * K;
     if (sup_out && cl_rank == 0)
+#pragma unroll 1
         for (int i = tid; i < K; i += NT) sup_out[i] = i < ns ? s_sup_idx[i] : -1;
 
     attend<D, NT>(a.v + (size_t)bkv * a.max_seq_len * D, ns, s_sup_idx, s_sup_key, s_w, s_red, s_ws, s_stage,
-                  a.exact_stage_depth, kmax, kmax_known, a.out + (size_t)bh * D, cl_rank, cl_size);
+                  a.exact_stage_depth, kmax, a.out + (size_t)bh * D, cl_rank, cl_size, 2);
     RETOPK_PHASE(2, 5);
 }
 
@@ -1657,12 +1700,14 @@ __device__ void exact_path(const StepArgs& a, unsigned char* smem_raw) {
 // from them; both end with softmax.V and the support insert.  Heads of one step run side by
 // side, so a step with a few exact heads costs the longer of the two paths, not their sum.
 // ------------------------------------------------------------------------------------
-template <int D, int NT>
+// WITH_REUSE = false leaves the reuse path out: the kernel of the Exact Top-K entry points
+// (the size of a kernel's code costs time at every launch behind a long scan).
+template <int D, int NT, bool WITH_REUSE = true>
 __global__ void __launch_bounds__(NT, 1024 / NT) finish_kernel(const StepArgs a) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     pdl_wait();        // scores and tile maxima come from the scan, recalled slots and paths from recall_kernel
     if (blockIdx.x == 0 && threadIdx.x == 0) *a.scan_counter = 0u;      // the scan before this kernel is complete
-    if (a.mode == MODE_RETOPK && a.ws_path[cluster_slot(a)] == PATH_REUSE) {
+    if (WITH_REUSE && a.mode == MODE_RETOPK && a.ws_path[cluster_slot(a)] == PATH_REUSE) {
         if (!a.skip_reuse) reuse_path<D, NT>(a, smem_raw);
     } else {
         exact_path<D, NT>(a, smem_raw);

@@ -164,7 +164,6 @@ __global__ void __launch_bounds__(LADDER_THREADS, 1) ladder_select_kernel(const 
     }
     __syncthreads();
     uint32_t kmax;
-    const bool kmax_known = true;
     const int ns = select_listed<NT>(s_key, s_idx, n, a.K, s_sup_idx, s_sup_key, s_hist, s_ws, &kmax);
     for (int i = tid; i < ns; i += NT) {
         a.lw_sup_idx[(size_t)bh * a.K + i] = s_sup_idx[i];
@@ -173,7 +172,7 @@ __global__ void __launch_bounds__(LADDER_THREADS, 1) ladder_select_kernel(const 
     if (tid == 0) {
         a.lw_meta[bh * 4 + 0] = ns;
         a.lw_meta[bh * 4 + 1] = (int32_t)kmax;
-        a.lw_meta[bh * 4 + 2] = kmax_known ? 1 : 0;
+        a.lw_meta[bh * 4 + 2] = 1;
     }
 }
 
@@ -193,14 +192,13 @@ __global__ void __launch_bounds__(LADDER_THREADS, 1) ladder_attend_kernel(const 
     if (a.ws_path[bh] != PATH_REUSE) return;
     const int ns = a.lw_meta[bh * 4 + 0];
     const uint32_t kmax = (uint32_t)a.lw_meta[bh * 4 + 1];
-    const bool kmax_known = a.lw_meta[bh * 4 + 2] != 0;
     for (int i = tid; i < ns; i += NT) {
         s_sup_idx[i] = a.lw_sup_idx[(size_t)bh * a.K + i];
         s_sup_key[i] = a.lw_sup_key[(size_t)bh * a.K + i];
     }
     __syncthreads();
     attend<D, NT>(a.v + (size_t)kv_group_of(bh, a) * a.max_seq_len * D, ns, s_sup_idx, s_sup_key, s_w, s_red, s_ws,
-                  s_stage, a.stage_depth, kmax, kmax_known, a.out + (size_t)bh * D);
+                  s_stage, a.stage_depth, kmax, a.out + (size_t)bh * D);
     if (tid == 0) {
         const int n = a.ws_ncand[bh];
         atomicAdd(a.counters + (size_t)bh * 4 + PATH_REUSE, 1ull);
@@ -275,12 +273,11 @@ __global__ void __launch_bounds__(LADDER_THREADS, 1) ladder_select_attend_insert
     }
     __syncthreads();
     uint32_t kmax;
-    const bool kmax_known = true;
     const int ns = select_listed<NT>(s_key, s_idx, n, a.K, s_sup_idx, s_sup_key, s_hist, s_ws, &kmax);
     int32_t* sup_out = a.sup_cache + ((size_t)bh * a.M + a.slot) * a.K;
     for (int i = tid; i < a.K; i += NT) sup_out[i] = i < ns ? s_sup_idx[i] : -1;
     attend<D, NT>(a.v + (size_t)kv_group_of(bh, a) * a.max_seq_len * D, ns, s_sup_idx, s_sup_key, s_w, s_red, s_ws,
-                  s_stage, a.stage_depth, kmax, kmax_known, a.out + (size_t)bh * D);
+                  s_stage, a.stage_depth, kmax, a.out + (size_t)bh * D);
     if (tid == 0) {
         atomicAdd(a.counters + (size_t)bh * 4 + PATH_REUSE, 1ull);
         atomicAdd(a.counters + (size_t)bh * 4 + 3, (unsigned long long)n);
