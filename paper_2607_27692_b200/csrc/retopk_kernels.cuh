@@ -592,7 +592,7 @@ __device__ __forceinline__ uint32_t select_general(const KeySrc src, int n, int 
 // bisection and the general emit.  s_hist: SCRATCH_WORDS words; s_ws: WS_WORDS ints.
 // One copy serves both paths of finish_kernel.
 template <int NT>
-__device__ __forceinline__ int select_listed_body(const uint32_t* s_key, const int32_t* s_idx, int n, int K,
+__device__ __noinline__ int select_listed(const uint32_t* s_key, const int32_t* s_idx, int n, int K,
                                           int32_t* s_sup_idx, uint32_t* s_sup_key, uint32_t* s_hist, int* s_ws,
                                           uint32_t* kmax_out) {
     int ns;
@@ -617,13 +617,6 @@ __device__ __forceinline__ int select_listed_body(const uint32_t* s_key, const i
     __syncthreads();
     *kmax_out = kmax;
     return ns;
-}
-
-template <int NT>
-__device__ __noinline__ int select_listed(const uint32_t* s_key, const int32_t* s_idx, int n, int K,
-                                          int32_t* s_sup_idx, uint32_t* s_sup_key, uint32_t* s_hist, int* s_ws,
-                                          uint32_t* kmax_out) {
-    return select_listed_body<NT>(s_key, s_idx, n, K, s_sup_idx, s_sup_key, s_hist, s_ws, kmax_out);
 }
 
 // Largest key of s_key[0..n) (the rare callers that select without learning it).  Ends with a barrier.
@@ -1073,9 +1066,9 @@ __device__ __forceinline__ void score_candidates(const uint16_t* kbase, const in
 // through distributed shared memory and are added there in rank order.
 // ------------------------------------------------------------------------------------
 template <int D, int NT>
-__device__ __forceinline__ void attend_body(const uint16_t* vbase, int ns, const int32_t* s_sup_idx, const uint32_t* s_sup_key,
+__device__ __noinline__ void attend(const uint16_t* vbase, int ns, const int32_t* s_sup_idx, const uint32_t* s_sup_key,
                                     float* s_w, float* s_red, int* s_ws, uint4* s_stage, int depth, uint32_t kmax,
-                                    uint16_t* out_row, int cl_rank, int cl_size, int ptab) {
+                                    uint16_t* out_row, int cl_rank = 0, int cl_size = 1, int ptab = 1) {
     constexpr int LPR = D / 8;                  // lanes per bf16 row (16 bytes each)
     constexpr int RPW = 32 / LPR;               // rows per warp load
     constexpr int SLOTS = (NT / 32) * RPW;      // row slots per block
@@ -1184,13 +1177,6 @@ __device__ __forceinline__ void attend_body(const uint16_t* vbase, int ns, const
     }
 }
 
-template <int D, int NT>
-__device__ __noinline__ void attend(const uint16_t* vbase, int ns, const int32_t* s_sup_idx, const uint32_t* s_sup_key,
-                                    float* s_w, float* s_red, int* s_ws, uint4* s_stage, int depth, uint32_t kmax,
-                                    uint16_t* out_row, int cl_rank = 0, int cl_size = 1, int ptab = 1) {
-    attend_body<D, NT>(vbase, ns, s_sup_idx, s_sup_key, s_w, s_red, s_ws, s_stage, depth, kmax, out_row, cl_rank, cl_size, ptab);
-}
-
 // ------------------------------------------------------------------------------------
 // reuse path of finish_kernel: candidate union (Eq. 8-9), candidate scores (Eq. 10), Top-K
 // (Eq. 11), softmax.V (Eq. 12) and the support insert for one head, all in shared memory.
@@ -1198,8 +1184,32 @@ __device__ __noinline__ void attend(const uint16_t* vbase, int ns, const int32_t
 // 16-row staging tiles, and the window's rows requested ahead of the recalled lists.  Phase
 // clocks showed them level or ahead, the timed pipeline 3 us per step behind: dropped.)
 // ------------------------------------------------------------------------------------
+// What either path reads first from global memory, requested at kernel entry together with the
+// head's path so that one memory latency covers both: the recalled slot and the two query
+// elements this thread will stage (reuse path), eight tile maxima (exact path; a reuse head
+// drops them unused, 32 KB of L2 reads per head).
+struct FirstLoads {
+    int sel;
+    uint32_t qraw;
+    float4 m4[2];
+};
 template <int D, int NT>
-__device__ __forceinline__ void reuse_path(const StepArgs& a, unsigned char* smem_raw) {
+__device__ __forceinline__ FirstLoads first_loads(const StepArgs& a, int bh, bool want_reuse) {
+    const int tid = threadIdx.x;
+    FirstLoads f;
+    f.sel = (want_reuse && tid < a.r) ? a.ws_sel[(size_t)bh * a.r + tid] : -1;
+    f.qraw = (want_reuse && tid >= 32 && tid < 32 + D / 2) ? reinterpret_cast<const uint32_t*>(a.q + (size_t)bh * D)[tid - 32] : 0u;
+    const int ntile = (a.L + TILE_ROWS - 1) / TILE_ROWS;
+    const float* tm = a.ws_tmax + (size_t)bh * a.tmax_stride;
+#pragma unroll
+    for (int u = 0; u < 2; ++u)
+        f.m4[u] = tid * 8 + 4 * u < ntile ? *reinterpret_cast<const float4*>(tm + tid * 8 + 4 * u)
+                                          : make_float4(0.f, 0.f, 0.f, 0.f);
+    return f;
+}
+
+template <int D, int NT>
+__device__ __forceinline__ void reuse_path(const StepArgs& a, unsigned char* smem_raw, const FirstLoads& first) {
     constexpr int NW = NT / 32;
     // layout (words): qraw[D] sel[r] ws[WS_WORDS] hist[SCRATCH_WORDS] sup_idx[K] sup_key[K] w[K]
     //                 | big: idx[cap] key[cap], aliased later by red[NW*D+NT] | bitmap | stage[depth*NT*4]
@@ -1228,12 +1238,11 @@ __device__ __forceinline__ void reuse_path(const StepArgs& a, unsigned char* sme
     // peers write into this CTA's shared memory later on: all of them must be running by then
     if (cl_size > 1) cooperative_groups::this_cluster().sync();
 
-    // recalled slots and the raw query from global memory; clear the bitmap meanwhile
-    if (tid < a.r) s_sel[tid] = a.ws_sel[(size_t)bh * a.r + tid];
+    // recalled slots and the raw query (requested at kernel entry); clear the bitmap meanwhile
+    if (tid < a.r) s_sel[tid] = first.sel;
     if (tid >= 32 && tid < 32 + D / 2) {
-        const uint32_t raw = reinterpret_cast<const uint32_t*>(a.q + (size_t)bh * D)[tid - 32];
-        s_qraw[2 * (tid - 32)] = bf16_lo(raw);
-        s_qraw[2 * (tid - 32) + 1] = bf16_hi(raw);
+        s_qraw[2 * (tid - 32)] = bf16_lo(first.qraw);
+        s_qraw[2 * (tid - 32) + 1] = bf16_hi(first.qraw);
     }
     {
         const int nwords = (L + 31) >> 5;
@@ -1277,11 +1286,7 @@ __device__ __forceinline__ void reuse_path(const StepArgs& a, unsigned char* sme
 
     // Eq. 11: Top-K of the candidates; insert the support
     uint32_t kmax;
-#ifdef RETOPK_REUSE_INLINE
-    const int ns = select_listed_body<NT>(s_key, s_idx, n, K, s_sup_idx, s_sup_key, s_hist, s_ws, &kmax);
-#else
     const int ns = select_listed<NT>(s_key, s_idx, n, K, s_sup_idx, s_sup_key, s_hist, s_ws, &kmax);
-#endif
     RETOPK_PHASE(0, 5);
     if (cl_rank == 0) {
         int32_t* sup_out = a.sup_cache + ((size_t)bh * M + a.slot) * K;
@@ -1290,13 +1295,8 @@ __device__ __forceinline__ void reuse_path(const StepArgs& a, unsigned char* sme
     }
 
     // Eq. 12 (s_red aliases the candidate lists, which are dead now)
-#ifdef RETOPK_REUSE_INLINE
-    attend_body<D, NT>(a.v + (size_t)bkv * a.max_seq_len * D, ns, s_sup_idx, s_sup_key, s_w, s_red, s_ws, s_stage,
-                  a.stage_depth, kmax, a.out + (size_t)bh * D, cl_rank, cl_size, 0);
-#else
     attend<D, NT>(a.v + (size_t)bkv * a.max_seq_len * D, ns, s_sup_idx, s_sup_key, s_w, s_red, s_ws, s_stage,
                   a.stage_depth, kmax, a.out + (size_t)bh * D, cl_rank, cl_size, 0);
-#endif
     if (tid == 0 && cl_rank == 0) {      // the step record is written last: nothing in this kernel waits for it
         a.ws_ncand[bh] = n;
         atomicAdd(a.counters + (size_t)bh * 4 + PATH_REUSE, 1ull);
@@ -1326,7 +1326,9 @@ __device__ __forceinline__ void scan_body(const StepArgs& a) {
     const int G = a.G, L = a.L;
     const int n_groups = a.B * a.Hkv;
 
-    // nothing flagged in this step: leave at once (the common case on the reuse path)
+    // nothing flagged in this step: leave at once (the common case on the reuse path).  (Reading
+    // the flags straight away instead saves a memory latency in front of a short scan, 0.3 us on
+    // a mixed step, and costs 0.5 us on every step that scans nothing: measured, not kept.)
     if (a.mode != MODE_EXACT && a.ws_gflag[n_groups] != a.step_id) return;
 
     // the groups to scan, in ascending order (all of them for Exact Top-K attention)
@@ -1440,16 +1442,8 @@ __device__ __forceinline__ void scan_body(const StepArgs& a) {
                     m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 16));
                     if (head < G && ((need >> head) & 1u)) {
                         float* srow = a.ws_scores + (size_t)(head0 + head) * a.score_stride;
-#if RETOPK_SCORE_POLICY == 1
-                        if (r0 < L) srow[r0] = c[e] * scale;
-                        if (r1 < L) srow[r1] = c[2 + e] * scale;
-#elif RETOPK_SCORE_POLICY == 2
-                        if (r0 < L) stg_hint(srow + r0, c[e] * scale, pol_first);
-                        if (r1 < L) stg_hint(srow + r1, c[2 + e] * scale, pol_first);
-#else
                         if (r0 < L) stg_hint(srow + r0, c[e] * scale, pol_last);
                         if (r1 < L) stg_hint(srow + r1, c[2 + e] * scale, pol_last);
-#endif
                         if (g == 0 && tile_row < L)
                             stg_hint(a.ws_tmax + (size_t)(head0 + head) * a.tmax_stride + (tile_row >> 4), m * scale, pol_last);
                     }
@@ -1488,12 +1482,12 @@ __global__ void __launch_bounds__(SCAN_THREADS) scan_kernel(const StepArgs a) {
 // lower-index tie rule is taken from that list.
 // ------------------------------------------------------------------------------------
 template <int D, int NT>
-__device__ __forceinline__ void exact_path(const StepArgs& a, unsigned char* smem_raw) {
+__device__ __forceinline__ void exact_path(const StepArgs& a, unsigned char* smem_raw, const FirstLoads& first) {
     // In a cluster every CTA of a head selects the same support on its own (the lists are short
     // and come from L2); only the value rows are shared out, and rank 0 writes the results.
     const int bh = cluster_slot(a);
     const int cl_rank = cluster_rank(a), cl_size = 1 << a.cl_shift;
-    // layout (words): sup_idx[K] sup_key[K] w[K] cnt[SCRATCH_WORDS] ws[WS_WORDS] misc[8]
+    // layout (words): sup_idx[K] sup_key[K] w[K] cnt[SCRATCH_WORDS] ws[WS_WORDS] (8 spare)
     //                 | lists: key[NS] idx[NS] tile[tile_cap]; dead once the support is emitted and
     //                   then reused by attend: red[NW*D+NT], stage[depth*NT*4] (may run past the lists)
     constexpr int NW = NT / 32;
@@ -1502,7 +1496,6 @@ __device__ __forceinline__ void exact_path(const StepArgs& a, unsigned char* sme
     float* s_w = reinterpret_cast<float*>(s_sup_key + a.K);
     uint32_t* s_hist = reinterpret_cast<uint32_t*>(s_w + a.K);
     int* s_ws = reinterpret_cast<int*>(s_hist + SCRATCH_WORDS);
-    int* s_misc = s_ws + WS_WORDS;
     uint32_t* s_key = reinterpret_cast<uint32_t*>(smem_raw) + ((3 * a.K + SCRATCH_WORDS + WS_WORDS + 8 + 3) & ~3);
     int32_t* s_idx = reinterpret_cast<int32_t*>(s_key + a.NS);
     int32_t* s_tile = s_idx + a.NS;
@@ -1539,13 +1532,9 @@ __device__ __forceinline__ void exact_path(const StepArgs& a, unsigned char* sme
         const bool regs8 = sh == 3 && n2 <= NT;
         float mv[8];
         if (regs8) {
-            const int t0 = tid * 8;
-            float4 m4[2];
-#pragma unroll
-            for (int u = 0; u < 2; ++u)
-                m4[u] = t0 + 4 * u < ntile ? *reinterpret_cast<const float4*>(tm + t0 + 4 * u)
-                                           : make_float4(0.f, 0.f, 0.f, 0.f);
-            const float raw[8] = {m4[0].x, m4[0].y, m4[0].z, m4[0].w, m4[1].x, m4[1].y, m4[1].z, m4[1].w};
+            const int t0 = tid * 8;                 // (the maxima first_loads() asked for)
+            const float raw[8] = {first.m4[0].x, first.m4[0].y, first.m4[0].z, first.m4[0].w,
+                                  first.m4[1].x, first.m4[1].y, first.m4[1].z, first.m4[1].w};
             float m = -CUDART_INF_F;
 #pragma unroll
             for (int e = 0; e < 8; ++e) {
@@ -1707,10 +1696,14 @@ __global__ void __launch_bounds__(NT, 1024 / NT) finish_kernel(const StepArgs a)
     extern __shared__ __align__(16) unsigned char smem_raw[];
     pdl_wait();        // scores and tile maxima come from the scan, recalled slots and paths from recall_kernel
     if (blockIdx.x == 0 && threadIdx.x == 0) *a.scan_counter = 0u;      // the scan before this kernel is complete
-    if (WITH_REUSE && a.mode == MODE_RETOPK && a.ws_path[cluster_slot(a)] == PATH_REUSE) {
-        if (!a.skip_reuse) reuse_path<D, NT>(a, smem_raw);
+    const int bh = cluster_slot(a);
+    const bool retopk = WITH_REUSE && a.mode == MODE_RETOPK;
+    const int path = retopk ? (int)a.ws_path[bh] : (int)PATH_FALLBACK;
+    const FirstLoads first = first_loads<D, NT>(a, bh, retopk);
+    if (path == PATH_REUSE) {
+        if (!a.skip_reuse) reuse_path<D, NT>(a, smem_raw, first);
     } else {
-        exact_path<D, NT>(a, smem_raw);
+        exact_path<D, NT>(a, smem_raw, first);
     }
 }
 
