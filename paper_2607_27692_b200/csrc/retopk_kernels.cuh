@@ -12,9 +12,8 @@
 //   finish_kernel  one CTA per (sequence, query head) - or a thread-block cluster of 2-8 CTAs
 //                  when there are few heads, or 512-thread CTAs two to an SM when there are
 //                  more heads than SMs - with heads of both paths side by side.
-//                  Reuse path: candidate union (Eq. 8-9) in a shared-memory bitmap, exact
-//                  scores of the gathered key rows on the tensor cores (Eq. 10; same MMA path
-//                  as the scan, so a key scores the same bits on either path), Top-K (Eq. 11).
+//                  Reuse path: candidate union (Eq. 8-9) in a shared-memory bitmap, fp32 scores
+//                  of the gathered key rows (Eq. 10), Top-K by one histogram (Eq. 11).
 //                  Exact path: global Top-K (Eq. 1) of the scanned scores (tile maxima give a
 //                  lower bound for the K-th score, only the tiles that reach it are read back).
 //                  Both: softmax.V (Eq. 12) and the support insert.
@@ -25,6 +24,13 @@
 // finished from a list behind the scan - was built and measured: the two launches that are
 // then empty on a reuse-only step cost as much as the recall launch saves, and a step with a
 // few exact heads pays reuse time PLUS scan PLUS exact finish instead of their maximum.)
+//
+// Code size matters here: behind a full-history scan the per-head kernels start with cold
+// instruction caches, and the fetch cost grows with the size of a kernel's code whether that
+// code runs or not.  So: softmax.V and the listed Top-K exist once, out of line, for both paths;
+// one general selection; no automatic unrolling of loops that run once; rare cases out of line
+// (taking scalars, never the argument block by reference: that would force a copy of it into
+// local memory at kernel entry).
 #pragma once
 #include <cooperative_groups.h>
 #include <cuda_bf16.h>
