@@ -55,3 +55,38 @@ def test_gpu_arm_line():
     assert {"sm_mhz", "sm_max_mhz", "reasons"} <= set(line["clocks"])
     cb = line["cpu_baseline"]
     assert cb["kind"] == "oracle" and cb["value"] > 0 and cb["cores"] >= 1
+
+
+@pytest.mark.gpu
+def test_gpu_arm_reports_the_steady_state_and_every_path():
+    """Caches are filled before the warm-up, and the step-level and per-path fractions are in the line."""
+    line = run_bench("--config", "tiny", "--steps", "12", "--warmup", "4", "--layers", "2", "--no-cpu-baseline")
+    cfg = line["config"]
+    assert cfg["preroll_steps_per_layer"] >= 16 and cfg["cache_fill_at_first_timed_call"] == 16      # tiny: M = 16
+    assert cfg["cache_fill_at_last_timed_call"] == 16
+    roof = line["roofline"]
+    assert {"recall", "scan", "finish"} <= set(roof["kernels"]) and roof["step"]["frac"] > 0
+    for name in ("configured_tau", "pure_reuse", "pure_exact", "tau_0.85"):
+        assert line["paths"][name]["us_per_step"] > 0 and roof["paths"][name]["frac"] > 0
+    assert abs(line["paths"]["configured_tau"]["us_per_step"] - line["value"]) < 0.02
+    assert "met_at_configured_tau" in line["targets"]
+    assert line["prefill_seed"]["n_tail"] == 16 and line["prefill_seed"]["ms"] > 0
+
+
+@pytest.mark.gpu
+def test_profiler_case_and_phase_table_run():
+    """The small case profiler captures use, and the per-phase clock table of an instrumented
+    build (compiled into a temporary directory by the benchmark itself)."""
+    env = dict(os.environ, PYTHONPATH=ROOT)
+    res = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--config", "tiny", "--one-layer", "mix",
+                          "--steps", "4", "--preroll", "4"], capture_output=True, text=True, env=env, cwd=ROOT, timeout=600)
+    assert res.returncode == 0, res.stderr[-2000:]
+    rec = json.loads([ln for ln in res.stdout.splitlines() if ln.startswith("{")][-1])
+    assert rec["one_layer"] == "mix" and rec["steps"] == 8 and rec["stats"]["status"] == 0
+    res = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--config", "tiny", "--phases", "--steps", "6",
+                          "--preroll", "6"], capture_output=True, text=True, env=env, cwd=ROOT, timeout=900)
+    assert res.returncode == 0, res.stderr[-2000:]
+    table = json.loads(res.stdout[res.stdout.index("{"):])
+    assert table["pure_reuse"]["recall kernel"]["total"] > 0
+    assert table["pure_reuse"]["finish kernel, reuse path"]["total"] > 0
+    assert table["pure_exact"]["finish kernel, exact path"]["total"] > 0
