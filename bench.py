@@ -139,6 +139,7 @@ class Layers:
         self.out_host = torch.empty((cfg.B, cfg.H_q, cfg.d), dtype=torch.bfloat16).pin_memory()
         self.ctx = []
         self.qbar_bf16 = False
+        self.recall_recent = False
         self.cluster = 0
         self.finish_threads = 0
         self.block_shape = None
@@ -150,6 +151,9 @@ class Layers:
         if self.qbar_bf16:
             for c in self.ctx:
                 c.set_qbar_format(1)
+        if self.recall_recent:
+            for c in self.ctx:
+                c.set_recall_mode(1)
         if self.cluster:
             for c in self.ctx:
                 c.set_cluster_size(self.cluster)
@@ -451,6 +455,7 @@ def run_gpu(args):
         cfg = cfg.replace(steps=t_per_layer)
     layers = Layers(cfg, n_layers, t_per_layer, rank, torch, rt, preroll=preroll)
     layers.qbar_bf16 = args.qbar_bf16
+    layers.recall_recent = args.recall_recent
     layers.cluster = args.cluster
     layers.finish_threads = args.finish_threads
     layers.block_shape = args.block_shape
@@ -549,7 +554,7 @@ def run_gpu(args):
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": cfg.name, "B": cfg.B, "H_q": cfg.H_q, "H_kv": cfg.H_kv, "d": cfg.d,
                    "context": cfg.context, "K": cfg.K, "M": cfg.M, "r": cfg.r, "W": cfg.W, "tau": cfg.tau,
-                   "R": cfg.R, "qbar_cache": "bf16" if args.qbar_bf16 else "fp32",
+                   "R": cfg.R, "qbar_cache": "bf16" if args.qbar_bf16 else "fp32", "recall": "recent" if args.recall_recent else "similar",
                    "ctas_per_head": args.cluster or "auto", "threads_per_cta": args.finish_threads or (args.block_shape and "x".join(map(str, args.block_shape))) or "auto",
                    "layers_rotated": n_layers, "decode_steps_per_layer": t_per_layer,
                    "preroll_steps_per_layer": preroll, "cache_fill_at_first_timed_call": fill_first,
@@ -787,6 +792,8 @@ def main():
                     help="block shape of the finish kernel (0: the library's own choice)")
     ap.add_argument("--block-shape", default=None, type=lambda v: tuple(int(x) for x in v.split("x")),
                     help="THREADSxCTAS_PER_SM of the finish kernel: 1024x1, 512x2 or 512x1 (default: the library's own choice)")
+    ap.add_argument("--recall-recent", action="store_true",
+                    help="recall the most recent cached entries instead of the most similar (the Recent-R ablation row)")
     ap.add_argument("--qbar-bf16", action="store_true",
                     help="keep the cached normalised queries in bf16 (storage variant) in every pass")
     ap.add_argument("--ladder", action="store_true",
