@@ -650,6 +650,8 @@ PHASES = {
                        (8, 9, "  Top-K: span of the keys"), (9, 10, "  Top-K: histogram"), (10, 11, "  Top-K: boundary bin"),
                        (11, 12, "  Top-K: its members"), (12, 13, "  Top-K: their ranks"), (13, 14, "  Top-K: ballots"),
                        (14, 5, "  Top-K: placed"),
+                       (3, 21, "  rows: requested"), (21, 22, "  rows: first half landed"), (22, 23, "  rows: first half scored"),
+                       (23, 7, "  rows: second half landed"), (7, 4, "  rows: second half scored"),
                        (16, 17, "  softmax.V: value rows requested"), (17, 18, "  softmax.V: weights"),
                        (18, 19, "  softmax.V: rows landed"), (19, 20, "  softmax.V: weighted sum"), (20, 6, "  softmax.V: reduction, output")]),
     "finish kernel, exact path": (2, [(0, 1, "bound from the tile maxima"), (1, 2, "hit-tile list"), (2, 3, "read-back of hit tiles"),

@@ -1041,9 +1041,11 @@ __device__ __forceinline__ void score_candidates(const uint16_t* kbase, const in
             if (u == half - 1) cp_async_commit();
         }
         cp_async_commit();
+        if (base == 0) RETOPK_PHASE(0, 21);
         for (int g2 = 0; g2 < 2; ++g2) {
             if (g2 == 0) cp_async_wait_but_one();
             else cp_async_wait_all();
+            if (base == 0) { if (g2 == 0) RETOPK_PHASE(0, 22); else RETOPK_PHASE(0, 7); }
             const int u_begin = g2 == 0 ? 0 : half, u_end = g2 == 0 ? half : depth;
             for (int u0 = u_begin; u0 < u_end; u0 += 8) {
                 float part[8];
@@ -1057,6 +1059,7 @@ __device__ __forceinline__ void score_candidates(const uint16_t* kbase, const in
                 const int i = base + (u0 + row) * SLOTS + myslot;
                 if ((LPR == 8 || (sub & 1) == 0) && u0 + row < u_end && i < n) key_out[i] = score_key(tot * scale);
             }
+            if (base == 0 && g2 == 0) RETOPK_PHASE(0, 23);
         }
     }
 }
